@@ -1,0 +1,161 @@
+/*
+ * dragon.h -- C ABI of the B200 graph virtual machine (libdragon.so).
+ *
+ * The library evaluates a compiled function  f = function(inputs, outputs)  (Sec. 2.1 of
+ * "Dragon: A Computation Graph Virtual Machine Based Deep Learning Framework",
+ * arXiv 1707.08265) over large tensors on one GPU: the forward pass and the generated
+ * gradient pass of a tensor-as-node DAG, after the forward prune (Sec. 2.2, Algorithm 1)
+ * and the backward prune (Sec. 2.3, Algorithm 2).
+ *
+ * Conventions that hold for every entry point
+ *   - Tensor ids and operator ids are dense non-negative ints in creation order; this is
+ *     the "creating order" of Sec. 3.2.  A negative return value is an error code.
+ *   - All host pointers are read during the call only; nothing is retained.
+ *   - All device memory (feeds, fetches, workspace) belongs to the caller.  The library
+ *     allocates device memory only for its own immutable instruction streams, on the first
+ *     dragon_run() of a function, and frees it in dragon_function_destroy().
+ *   - Tensors are row-major and contiguous, rank 0..2.  Device pointers must be 16-byte
+ *     aligned.
+ *   - Every entry point returns an error code (or NULL) instead of launching on bad
+ *     arguments; dragon_last_error() gives the message.  No call synchronises the device
+ *     except dragon_function_status().
+ */
+#ifndef DRAGON_H_
+#define DRAGON_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct dragon_graph dragon_graph_t;       /* host-only graph under construction   */
+typedef struct dragon_function dragon_function_t; /* pruned + compiled function           */
+typedef int32_t dragon_id;
+
+enum {
+  DRAGON_OK = 0,
+  DRAGON_ERR_INVALID_ARG = -1,
+  DRAGON_ERR_SHAPE = -2,         /* declared output shape differs from the inferred one, or operands do not broadcast */
+  DRAGON_ERR_DTYPE = -3,
+  DRAGON_ERR_NOT_SSA = -4,       /* output already has a producer, or an operator reads its own output */
+  DRAGON_ERR_MISSING_INPUT = -5, /* a marked source tensor is not among the function's inputs */
+  DRAGON_ERR_NO_PATH = -6,       /* gradient requested but no chain objective -> derivative target */
+  DRAGON_ERR_UNSUPPORTED = -7,
+  DRAGON_ERR_WORKSPACE = -8,     /* workspace missing, misaligned or too small */
+  DRAGON_ERR_CUDA = -9,
+  DRAGON_ERR_TIMEOUT = -10       /* a bounded device-side wait ran out (reported by dragon_function_status) */
+};
+
+enum { DRAGON_F32 = 0, DRAGON_BF16 = 1, DRAGON_I32 = 2 };
+
+/* Operator types.  The paper names Sigmoid, Tanh, ReLU (Sec. 2.4) and uses mul, add, sin in
+ * its example (Sec. 2.2); the remaining semantics are this library's:
+ *   ADD, SUB, MUL          a+b, a-b, a*b with right-aligned broadcasting among [], [C], [R,C]
+ *   DIV                    a / (1 + |b|)
+ *   EXP                    exp(min(max(x, -10), 10))
+ *   SUM, MEAN              over the last axis, result broadcast back to the operand's shape
+ *   INNER_PRODUCT(X, W)    Y[m,n] = sum_k X[m,k] * W[n,k]; operands are consumed as bf16,
+ *                          accumulation is fp32
+ *   BIAS_ADD(Y, b)         Y[m,n] + b[n]
+ *   SOFTMAX_CROSS_ENTROPY(Z, labels)  scalar -(1/M) sum_m log softmax(Z[m,:])[labels[m]],
+ *                          labels int32 in [0, N); an out-of-range label contributes 0 and
+ *                          sets the function status to DRAGON_ERR_INVALID_ARG (no fault)
+ */
+enum {
+  DRAGON_OP_ADD = 0, DRAGON_OP_SUB = 1, DRAGON_OP_MUL = 2, DRAGON_OP_DIV = 3,
+  DRAGON_OP_SIN = 4, DRAGON_OP_EXP = 5, DRAGON_OP_TANH = 6, DRAGON_OP_SIGMOID = 7,
+  DRAGON_OP_RELU = 8, DRAGON_OP_SUM = 9, DRAGON_OP_MEAN = 10,
+  DRAGON_OP_INNER_PRODUCT = 11, DRAGON_OP_BIAS_ADD = 12, DRAGON_OP_SOFTMAX_CROSS_ENTROPY = 13,
+  DRAGON_OP_COUNT_ = 14
+};
+
+/* ---- graph capture (Sec. 2.1: tensors are nodes; an operator connects each of its inputs
+ *      to each of its outputs, Sec. 2.2) -------------------------------------------------- */
+
+dragon_graph_t* dragon_graph_create(void);
+void dragon_graph_destroy(dragon_graph_t* g); /* NULL is allowed */
+
+/* Declares a tensor.  name: unique, NUL-terminated (Sec. 3.1: each tensor has a unique name).
+ * rank 0..2, shape[rank] > 0 (host pointer, may be NULL for rank 0).  Returns the new id. */
+dragon_id dragon_add_tensor(dragon_graph_t* g, const char* name, int dtype, int rank, const int64_t* shape);
+
+/* Appends an operator.  in/out: host arrays of tensor ids declared earlier.  Every output must
+ * have no producer yet, must not be among the inputs and must not have been read already; its
+ * declared shape must equal the inferred one (Sec. 4.3: a mistaken shape is caught before
+ * executing).  attrs is reserved (pass NULL, 0).  Returns the operator id. */
+dragon_id dragon_add_op(dragon_graph_t* g, int op_type, const dragon_id* in, int n_in,
+                        const dragon_id* out, int n_out, const double* attrs, int n_attrs);
+
+/* theano.tensor.grad analogue (Sec. 4.1): attaches one gradient stage for the derivative pairs
+ * objs x wrts (Sec. 2.3).  The stage computes the gradient of the sum of all elements of all
+ * objs.  For each wrts[j] a new f32 tensor of the same shape is declared and its id written to
+ * out_grad_tensor_ids[j] (host array of n_wrt ids).  DRAGON_ERR_NO_PATH if some wrts[j] has no
+ * chain to any objective.  Gradient tensors can be fetched but not consumed by operators. */
+int dragon_add_grad(dragon_graph_t* g, const dragon_id* objs, int n_obj, const dragon_id* wrts, int n_wrt,
+                    dragon_id* out_grad_tensor_ids);
+
+int dragon_graph_num_tensors(const dragon_graph_t* g);
+int dragon_graph_num_ops(const dragon_graph_t* g);
+
+/* ---- compile: prune + instruction streams (Sec. 2.2, 2.3, 3.2) -------------------------- */
+
+/* Builds f = function(inputs, outputs).  inputs must be source tensors (no producer); an input
+ * that the targets do not need is legal, is reported as pruned, and its feed pointer is never
+ * read (the redundant b of Sec. 2.2).  Works without a GPU.  The graph may be destroyed
+ * afterwards.  Returns NULL on error. */
+dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, int n_in,
+                                   const dragon_id* outputs, int n_out);
+void dragon_function_destroy(dragon_function_t* f); /* NULL is allowed */
+
+/* Marked flags M of Algorithm 1 run over the two-stage DAG from the fetched targets: one byte
+ * per tensor id (n_tensors must equal the graph's tensor count at compile time). */
+int dragon_function_marked(const dragon_function_t* f, uint8_t* flag_per_tensor, int n_tensors);
+
+/* Kept operators.  fwd_ops: kept forward operator ids in creation order.  grad_ops: for every
+ * kept gradient operator the id of its forward operator, stage by stage, inverse creation
+ * order inside a stage (Sec. 3.2); grad_input_mask (may be NULL): bit p set iff the gradient
+ * with respect to operand position p is produced (first occurrence of a repeated operand).
+ * The counts are always written; the arrays are filled up to their capacities. */
+int dragon_function_kept_ops(const dragon_function_t* f, dragon_id* fwd_ops, int cap_f, int* n_f,
+                             dragon_id* grad_ops, uint32_t* grad_input_mask, int cap_g, int* n_g);
+
+/* One byte per listed input: 1 if the pruned function reads it. */
+int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flag_per_input, int n_in);
+
+/* Number of kernel launches one dragon_run() issues, and a short human-readable plan
+ * (NUL-terminated, truncated to cap). */
+int dragon_function_num_launches(const dragon_function_t* f);
+int dragon_function_describe(const dragon_function_t* f, char* buf, int cap);
+
+/* Scratch memory (partial sums, tensors that cross kernels, spilled values, a status word).
+ * dev_ptr: device memory, 256-byte aligned, at least dragon_function_workspace_bytes() long,
+ * owned by the caller and not touched by anyone else while a run is in flight. */
+size_t dragon_function_workspace_bytes(const dragon_function_t* f);
+int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t bytes);
+
+/* ---- run (Sec. 2.1: push inputs, get outputs) ------------------------------------------ */
+
+/* feeds: host array of n_in device pointers in the order of inputs (entries of pruned inputs
+ * may be NULL); fetches: host array of n_out device pointers; cuda_stream: a cudaStream_t.
+ * Asynchronous; launches nothing on error.  Each needed input is read and each fetched output
+ * written by the kernels of the plan; a fetch that is itself an input is copied. */
+int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetches, void* cuda_stream);
+
+/* Synchronises the stream of the last run and returns the device status word: DRAGON_OK,
+ * DRAGON_ERR_TIMEOUT (a bounded wait gave up) or DRAGON_ERR_INVALID_ARG (bad label). */
+int dragon_function_status(dragon_function_t* f);
+
+/* Host instantiation of the VM's elementary functions (fn: DRAGON_OP_SIN, _EXP, _TANH,
+ * _SIGMOID; DRAGON_OP_DIV evaluates 1/(1+|x|); 100 + DRAGON_OP_SIN evaluates the cosine),
+ * for accuracy sweeps on machines without a GPU.  x, y: host arrays of n floats. */
+int dragon_host_math(int fn, const float* x, float* y, int n);
+
+/* Thread-local message of the last failing call on this thread. */
+const char* dragon_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DRAGON_H_ */
