@@ -1,0 +1,412 @@
+// Host compiler, part 2: one fused segment of micro-operations -> VM instruction stream.
+//
+// The VM is an accumulator machine (vm_isa.h).  Values that outlive the accumulator get a
+// home: a register slot, then a shared-memory slot, then a per-CTA spill slot in the workspace;
+// the victim of an eviction is the value whose next use is farthest away.  Tensors that are
+// memory operands can be re-read instead of being kept; scalars and constants live in the
+// uniform table.
+#include <algorithm>
+#include <cstring>
+#include <map>
+
+#include "plan.h"
+
+namespace dragon {
+namespace {
+
+using namespace vm;
+
+enum HomeKind { H_NONE, H_REG, H_SMEM, H_SPILL };
+constexpr int kFar = 1 << 30;
+
+struct VInfo {
+  std::vector<int> uses;   // positions (index into the segment's item list), ascending
+  int home = H_NONE, home_idx = -1;
+  int uni = -1;            // uniform-table index (scalars, constants)
+  int operand = -1;        // operand-table index (memory tensors that are not scalars)
+};
+
+struct Gen {
+  const std::vector<Item>& items;
+  const std::vector<int>& idx;
+  const std::vector<Value>& vals;
+  const std::vector<MemRef>& mems;
+  VmSegment* seg;
+  Shape dom;
+  std::vector<int> canon;
+  std::map<int, VInfo> info;
+  std::vector<uint32_t> pro, body, epi;
+  int reg_owner[kVmRegs];        // value id, -1 free, -2 pinned accumulator
+  int smem_owner[kVmSmemSlots];
+  std::vector<int> free_spill;
+  int n_uni = 0;
+  int acc_val = -1;
+  std::vector<bool> done;        // item already produced by a fused instruction
+  int err = DRAGON_OK;
+
+  Gen(const std::vector<Item>& it, const std::vector<int>& ix, const std::vector<Value>& v,
+      const std::vector<MemRef>& m, VmSegment* s)
+      : items(it), idx(ix), vals(v), mems(m), seg(s) {}
+
+  int C(int v) const { return v < 0 ? v : canon[v]; }
+
+  int class_of(const Shape& s) const {
+    if (s == dom) return K_FULL;
+    if (s.numel() == 1) return K_SCALAR;
+    if (dom.rank == 2 && s.rows() == 1 && s.cols() == dom.cols()) return K_ROW;
+    return -1;
+  }
+  int operand_for(int mem, int kind) {
+    for (size_t i = 0; i < seg->operand_mem.size(); ++i)
+      if (seg->operand_mem[i] == mem && seg->operand_kind[i] == (uint32_t)kind) return (int)i;
+    seg->operand_mem.push_back(mem);
+    seg->operand_kind.push_back((uint32_t)kind);
+    return (int)seg->operand_mem.size() - 1;
+  }
+  int next_use(int v, int pos) const {  // first use strictly after pos
+    auto it = info.find(v);
+    if (it == info.end()) return kFar;
+    auto u = std::upper_bound(it->second.uses.begin(), it->second.uses.end(), pos);
+    return u == it->second.uses.end() ? kFar : *u;
+  }
+  bool is_input(int v) const { auto it = info.find(v); return it != info.end() && it->second.operand >= 0; }
+  bool addressable(int v) { VInfo& f = info[v]; return f.uni >= 0 || f.home == H_REG || f.home == H_SMEM; }
+
+  void emit(int c, int r = 0, uint32_t arg = 0) { body.push_back(encode(c, r, arg)); }
+  void emit_str(int k) { emit(J_STR * kJointStride + k); }
+
+  void release(int v) {
+    VInfo& f = info[v];
+    if (f.home == H_REG) reg_owner[f.home_idx] = -1;
+    else if (f.home == H_SMEM) smem_owner[f.home_idx] = -1;
+    else if (f.home == H_SPILL) free_spill.push_back(f.home_idx);
+    f.home = H_NONE;
+  }
+  void release_dead(int v, int pos) {
+    if (v >= 0 && next_use(v, pos) == kFar) {
+      release(v);
+      if (acc_val == v) acc_val = -1;
+    }
+  }
+  int new_spill() {
+    if (!free_spill.empty()) { int g = free_spill.back(); free_spill.pop_back(); return g; }
+    return seg->n_spill++;
+  }
+  int free_smem() {
+    for (int s = 0; s < kVmSmemSlots; ++s)
+      if (smem_owner[s] == -1) { seg->n_smem = std::max(seg->n_smem, s + 1); return s; }
+    return -1;
+  }
+  int free_reg() const {
+    for (int k = 0; k < kVmRegs; ++k)
+      if (reg_owner[k] == -1) return k;
+    return -1;
+  }
+  // a free register slot; may evict the resident value whose next use is farthest
+  int alloc_reg(int pos, int keep1 = -1, int keep2 = -1) {
+    int k0 = free_reg();
+    if (k0 >= 0) return k0;
+    int best = -1, best_use = -1;
+    for (int k = 0; k < kVmRegs; ++k) {
+      int v = reg_owner[k];
+      if (v < 0 || v == keep1 || v == keep2) continue;
+      int u = next_use(v, pos - 1);
+      if (is_input(v)) u = kFar - 1;  // a cached memory operand is dropped for free
+      if (u > best_use) { best_use = u; best = k; }
+    }
+    if (best < 0) { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: out of register slots"); return 0; }
+    int v = reg_owner[best];
+    VInfo& f = info[v];
+    if (is_input(v)) {
+      f.home = H_NONE;
+    } else {
+      int s = free_smem();
+      if (s >= 0) { emit(P_RTOS, best, s); f.home = H_SMEM; f.home_idx = s; smem_owner[s] = v; }
+      else { int gsl = new_spill(); emit(P_SPILL, best, gsl); f.home = H_SPILL; f.home_idx = gsl; }
+    }
+    reg_owner[best] = -1;
+    return best;
+  }
+  void give_reg(int v, int k) { VInfo& f = info[v]; f.home = H_REG; f.home_idx = k; reg_owner[k] = v; }
+
+  // the accumulator is about to be overwritten: keep its value if it is used after position pos
+  void save_acc(int pos, int keep1 = -1, int keep2 = -1) {
+    int v = acc_val;
+    if (v < 0) return;
+    VInfo& f = info[v];
+    if (f.uni >= 0 || f.home != H_NONE) return;
+    int nu = next_use(v, pos);
+    if (nu == kFar) return;
+    const bool have_free = free_reg() >= 0;
+    if (is_input(v) && !have_free) return;  // re-read later
+    if (!have_free) {
+      // if every register holds something needed sooner, the accumulator itself goes down a level
+      int farthest = -1;
+      for (int k = 0; k < kVmRegs; ++k) {
+        int w = reg_owner[k];
+        if (w < 0 || w == keep1 || w == keep2) continue;
+        farthest = std::max(farthest, is_input(w) ? kFar - 1 : next_use(w, pos));
+      }
+      if (farthest >= 0 && farthest <= nu) {
+        int s = free_smem();
+        if (s >= 0) { emit(P_STS, 0, s); f.home = H_SMEM; f.home_idx = s; smem_owner[s] = v; }
+        else { int gsl = new_spill(); emit(P_SPILL, kAccSlot, gsl); f.home = H_SPILL; f.home_idx = gsl; }
+        return;
+      }
+    }
+    int k = alloc_reg(pos + 1, keep1, keep2);
+    emit_str(k);
+    give_reg(v, k);
+  }
+  void load_acc(int v, int pos, int keep1 = -1, int keep2 = -1) {
+    if (acc_val == v) return;
+    save_acc(pos - 1, keep1, keep2);
+    VInfo& f = info[v];
+    if (f.uni >= 0) emit(P_LDU, 0, f.uni);
+    else if (f.home == H_REG) emit(J_LDR * kJointStride + f.home_idx);
+    else if (f.home == H_SMEM) emit(P_LDS, 0, f.home_idx);
+    else if (f.home == H_SPILL) emit(P_FILL, kAccSlot, f.home_idx);
+    else if (f.operand >= 0) emit(P_GLD, kAccSlot, f.operand);
+    else { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: value has no location"); }
+    acc_val = v;
+  }
+  void make_addressable(int v, int pos, int keep1, int keep2) {
+    if (addressable(v)) return;
+    VInfo& f = info[v];
+    int k = alloc_reg(pos, keep1, keep2);
+    if (f.home == H_SPILL) { emit(P_FILL, k, f.home_idx); free_spill.push_back(f.home_idx); }
+    else if (f.operand >= 0) emit(P_GLD, k, f.operand);
+    else { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: operand has no location"); }
+    give_reg(v, k);
+  }
+  // acc holds x and is about to be overwritten by a result: give x a home if it is needed again
+  // (a memory operand only while a register slot is free; it can be re-read otherwise)
+  void keep_operand(int x, int pos, int other) {
+    if (next_use(x, pos) == kFar || addressable(x) || info[x].home != H_NONE) return;
+    if (!is_input(x)) {
+      int k = alloc_reg(pos, x, other);
+      emit_str(k);
+      give_reg(x, k);
+      return;
+    }
+    int k = free_reg();
+    if (k >= 0) { emit_str(k); give_reg(x, k); }
+  }
+
+  void binary(const Item& it, int pos) {
+    static const int jop[4] = {J_ADD, J_SUB, J_MUL, J_DIVP}, jrev[4] = {J_ADD, J_RSUB, J_MUL, J_RDIVP};
+    static const int uop[4] = {P_ADDU, P_SUBU, P_MULU, P_DIVPU}, urev[4] = {P_ADDU, P_RSUBU, P_MULU, P_RDIVPU};
+    static const int sop[4] = {P_ADDS, P_SUBS, P_MULS, P_DIVPS}, srev[4] = {P_ADDS, P_RSUBS, P_MULS, P_RDIVPS};
+    const int a = C(it.a), b = C(it.b), d = C(it.dst);
+    int x, y;  // x goes through the accumulator, y is addressed
+    if (a == b) { x = a; y = a; }
+    else if (acc_val == a) { x = a; y = b; }
+    else if (acc_val == b) { x = b; y = a; }
+    else {
+      bool aa = addressable(a), ab = addressable(b);
+      if (aa && !ab) { x = b; y = a; }
+      else if (ab && !aa) { x = a; y = b; }
+      else if (aa && ab) {
+        // keep the one that is needed again where it is
+        bool a_dies = next_use(a, pos) == kFar, b_dies = next_use(b, pos) == kFar;
+        if (b_dies && !a_dies) { x = b; y = a; } else { x = a; y = b; }
+      } else { x = a; y = b; }
+    }
+    if (a == b) {
+      load_acc(x, pos, x);
+      if (!addressable(x)) { int k = alloc_reg(pos, x); emit_str(k); give_reg(x, k); }
+    } else {
+      if (!addressable(y)) make_addressable(y, pos, x, y);
+      load_acc(x, pos, x, y);
+      keep_operand(x, pos, y);
+    }
+    const bool rev = (x == b && a != b);
+    const int o = it.opc - M_ADD;
+    VInfo& fy = info[y];
+    if (fy.uni >= 0) emit(rev ? urev[o] : uop[o], 0, fy.uni);
+    else if (fy.home == H_REG) emit((rev ? jrev[o] : jop[o]) * kJointStride + fy.home_idx);
+    else emit(rev ? srev[o] : sop[o], 0, fy.home_idx);
+    acc_val = d;
+    release_dead(a, pos);
+    if (b != a) release_dead(b, pos);
+  }
+
+  void unary(const Item& it, int pos) {
+    static const std::map<int, int> op = {{M_SIN, P_SIN}, {M_COS, P_COS}, {M_EXPC, P_EXPC}, {M_TANH, P_TANH},
+      {M_SIGMOID, P_SIGMOID}, {M_RELU, P_RELU}, {M_NEG, P_NEG}, {M_STEP, P_STEP}, {M_CLAMPMASK, P_CLAMPMASK},
+      {M_ONEMSQ, P_ONEMSQ}, {M_YOMY, P_YOMY}, {M_DIVPGB, P_DIVPGB}, {M_RBF16, P_RBF16}, {M_ROWSUM, P_ROWSUM}};
+    const int a = C(it.a), d = C(it.dst);
+    load_acc(a, pos, a);
+    keep_operand(a, pos, -1);
+    // sin and cos of the same value share one range reduction
+    if (it.opc == M_SIN || it.opc == M_COS) {
+      for (int q = pos + 1; q < (int)idx.size(); ++q) {
+        const Item& o2 = items[idx[q]];
+        if (done[q] || o2.kind != IT_MOP || (o2.opc != M_SIN && o2.opc != M_COS) || o2.opc == it.opc || C(o2.a) != a) continue;
+        int k = alloc_reg(pos, a);
+        emit(P_SINCOS, k, 0);
+        int dsin = it.opc == M_SIN ? d : C(o2.dst), dcos = it.opc == M_SIN ? C(o2.dst) : d;
+        give_reg(dcos, k);
+        acc_val = dsin;
+        done[q] = true;
+        auto& u = info[a].uses;  // the partner's use of a is consumed here
+        u.erase(std::remove(u.begin(), u.end(), q), u.end());
+        release_dead(a, pos);
+        if (next_use(dcos, pos) == kFar) release(dcos);
+        if (next_use(dsin, pos) == kFar) acc_val = -1;
+        return;
+      }
+    }
+    emit(op.at(it.opc));
+    acc_val = d;
+    release_dead(a, pos);
+  }
+
+  int run() {
+    // 1. aliases (WIDEN) and the fused domain
+    canon.resize(vals.size());
+    for (size_t v = 0; v < vals.size(); ++v) canon[v] = (int)v;
+    bool has_dom = false, any_rowsum = false;
+    auto join = [&](const Shape& s) {
+      if (!has_dom) { dom = s; has_dom = true; return; }
+      Shape o;
+      if (broadcast_shapes(dom, s, &o)) dom = o;
+    };
+    for (int i : idx) {
+      const Item& it = items[i];
+      if (it.opc == M_WIDEN) canon[it.dst] = canon[it.a];
+      if (it.opc == M_STORE || it.opc == M_ACCUM) join(vals[it.a].shape);
+      else join(vals[it.dst].shape);
+      any_rowsum |= it.opc == M_ROWSUM;
+    }
+    // 2. uses and static locations
+    std::fill(reg_owner, reg_owner + kVmRegs, -1);
+    std::fill(smem_owner, smem_owner + kVmSmemSlots, -1);
+    bool any_row_class = false;
+    auto note = [&](int v, int pos) {
+      if (v < 0) return;
+      v = C(v);
+      VInfo& f = info[v];
+      f.uses.push_back(pos);
+      const Value& val = vals[v];
+      if (val.kind == VK_CONST && f.uni < 0) {
+        f.uni = n_uni++;
+        pro.push_back(encode(P_UCONST, 0, f.uni));
+        uint32_t bits; std::memcpy(&bits, &val.c, 4);
+        pro.push_back(bits);
+      } else if (val.kind == VK_MEM && f.uni < 0 && f.operand < 0) {
+        int cls = class_of(mems[val.mem].shape);
+        if (cls < 0) { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: operand shape does not fit the fused domain"); return; }
+        if (cls == K_SCALAR) {
+          f.uni = n_uni++;
+          pro.push_back(encode(P_ULOAD, 0, (uint32_t)f.uni | ((uint32_t)operand_for(val.mem, K_SCALAR) << 9)));
+        } else {
+          f.operand = operand_for(val.mem, cls);
+          any_row_class |= cls == K_ROW;
+        }
+      }
+    };
+    for (int p = 0; p < (int)idx.size(); ++p) {
+      const Item& it = items[idx[p]];
+      if (it.opc == M_WIDEN) continue;
+      note(it.a, p);
+      note(it.b, p);
+      if ((it.opc == M_STORE || it.opc == M_ACCUM) && class_of(mems[it.mem].shape) == K_ROW) any_row_class = true;
+    }
+    if (err) return err;
+    if (n_uni > 511) { set_error("graph VM: too many scalars and constants"); return DRAGON_ERR_UNSUPPORTED; }
+    seg->row_mode = any_rowsum || any_row_class;
+    if (seg->row_mode) {
+      seg->n = dom.rows();
+      seg->cols = (int)dom.cols();
+      if (dom.cols() > kVmTile) { set_error("graph VM: rows longer than %d elements are not supported", kVmTile); return DRAGON_ERR_UNSUPPORTED; }
+    } else {
+      seg->n = dom.numel();
+      seg->cols = 0;
+    }
+    // 3. accumulators get pinned registers
+    std::vector<std::pair<int, int>> accs;  // (item position, register)
+    for (int p = 0; p < (int)idx.size(); ++p)
+      if (items[idx[p]].opc == M_ACCUM) {
+        int k = (int)accs.size();
+        if (k >= kVmRegs - 4) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+        reg_owner[k] = -2;
+        accs.emplace_back(p, k);
+      }
+    // 4. body
+    done.assign(idx.size(), false);
+    for (int p = 0; p < (int)idx.size() && !err; ++p) {
+      if (done[p]) continue;
+      const Item& it = items[idx[p]];
+      if (it.opc == M_WIDEN) continue;
+      if (is_binary(it.opc)) binary(it, p);
+      else if (it.opc == M_STORE) {
+        int v = C(it.a);
+        int cls = class_of(mems[it.mem].shape);
+        if (cls < 0) { set_error("graph VM: store shape does not fit the fused domain"); return DRAGON_ERR_UNSUPPORTED; }
+        int opd = operand_for(it.mem, cls);
+        VInfo& f = info[v];
+        if (acc_val == v) emit(P_GST, kAccSlot, opd);
+        else if (f.home == H_REG) emit(P_GST, f.home_idx, opd);
+        else { load_acc(v, p, v); emit(P_GST, kAccSlot, opd); }
+        release_dead(v, p);
+      } else if (it.opc == M_ACCUM) {
+        int v = C(it.a), k = -1;
+        for (auto& a : accs) if (a.first == p) k = a.second;
+        load_acc(v, p, v);
+        emit(J_ACCUM * kJointStride + k);
+        release_dead(v, p);
+      } else unary(it, p);
+    }
+    if (err) return err;
+    // 5. peephole: multiply by a uniform followed by an add fuses into one instruction
+    std::vector<uint32_t> fused;
+    for (size_t i = 0; i < body.size(); ++i) {
+      uint32_t w = body[i];
+      if ((w & 1023u) == (uint32_t)P_MULU && i + 1 < body.size()) {
+        uint32_t nx = body[i + 1], ncase = nx & 1023u, ui = w >> 14;
+        if (ncase == (uint32_t)P_ADDU && ui < 512 && (nx >> 14) < 512) { fused.push_back(encode(P_FMAU, 0, ui | ((nx >> 14) << 9))); ++i; continue; }
+        if (ncase >= (uint32_t)(J_ADD * kJointStride) && ncase < (uint32_t)(J_ADD * kJointStride + kVmRegs)) {
+          fused.push_back(encode(J_FMAUR * kJointStride + (int)(ncase - J_ADD * kJointStride), 0, ui)); ++i; continue;
+        }
+      }
+      fused.push_back(w);
+    }
+    body.swap(fused);
+    // 6. epilogue: accumulators leave as per-CTA partial sums
+    for (auto& a : accs) {
+      const Item& it = items[idx[a.first]];
+      int cls = class_of(mems[it.mem].shape);
+      FinishJob job; job.mem = it.mem;
+      if (cls == K_SCALAR) { job.kind = 1; job.acc = seg->n_scalacc++; epi.push_back(encode(P_SCALOUT, a.second, job.acc)); }
+      else if (cls == K_ROW) { job.kind = 0; job.acc = seg->n_colacc++; epi.push_back(encode(P_COLOUT, a.second, job.acc)); }
+      else { set_error("graph VM: reduction target shape is not supported"); return DRAGON_ERR_UNSUPPORTED; }
+      seg->finish.push_back(job);
+    }
+    seg->code = pro;
+    seg->code.push_back(encode(P_LOOP_BEGIN, 0, 0));
+    seg->code.insert(seg->code.end(), body.begin(), body.end());
+    seg->code.push_back(encode(P_LOOP_END, 0, 0));
+    seg->code.insert(seg->code.end(), epi.begin(), epi.end());
+    seg->code.push_back(encode(P_END, 0, 0));
+    seg->code.push_back(encode(P_END, 0, 0));  // the interpreter prefetches one word ahead
+    seg->n_instr_body = (int)body.size();
+    if ((int)seg->code.size() > kVmCodeMaxWords) { set_error("graph VM: instruction stream too long (%d words)", (int)seg->code.size()); return DRAGON_ERR_UNSUPPORTED; }
+    if ((int)seg->operand_mem.size() > kMaxOperands) { set_error("graph VM: too many memory operands in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+    return DRAGON_OK;
+  }
+};
+
+}  // namespace
+
+int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx, const std::vector<Value>& vals,
+                    const std::vector<MemRef>& mems, int sm_count, VmSegment* seg) {
+  Gen gen(items, idx, vals, mems, seg);
+  int rc = gen.run();
+  if (rc) return rc;
+  long long tiles = seg->row_mode ? seg->n : (seg->n + kVmTile - 1) / kVmTile;
+  seg->grid = (int)std::max<long long>(1, std::min<long long>(tiles, sm_count));
+  return DRAGON_OK;
+}
+
+}  // namespace dragon

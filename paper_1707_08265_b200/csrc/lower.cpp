@@ -1,0 +1,487 @@
+// Host compiler, part 1: kept operators -> micro-operations -> fused segments -> launch plan.
+//
+// Forward operators are lowered in creating order, gradient operators in inverse order
+// (Sec. 3.2).  A gradient operator reads forward values through its anchor (Sec. 3.3); inside
+// one fused segment those are simply values that stay live, across segments they are
+// workspace tensors.  Gradients with respect to broadcast operands are kept per domain element
+// (the reverse sweep is linear in dy) and summed once, where the gradient tensor is written.
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <map>
+
+#include "plan.h"
+
+namespace dragon {
+namespace {
+
+struct Lowerer {
+  const Graph& g;
+  const PruneResult& pr;
+  Plan* plan;
+  std::vector<Item> items;
+  std::vector<Value> vals;
+  std::vector<int> fval;                      // forward tensor -> value id
+  std::vector<std::map<int, int>> gval;       // per stage: tensor -> gradient value id
+  std::vector<int> fetch_of;                  // tensor -> fetch position or -1
+  std::map<int, int> transposed;              // memref -> memref of its transpose
+  int err = DRAGON_OK;
+
+  Lowerer(const Graph& g_, const PruneResult& pr_, Plan* p) : g(g_), pr(pr_), plan(p) {}
+
+  int new_mem(int where, int index, int dtype, const Shape& s) {
+    MemRef m;
+    m.where = where; m.index = index; m.dtype = dtype; m.shape = s;
+    plan->mems.push_back(m);
+    return (int)plan->mems.size() - 1;
+  }
+  int new_val(int kind, const Shape& s, int mem = -1, float c = 0.f) {
+    Value v; v.kind = kind; v.shape = s; v.mem = mem; v.c = c;
+    vals.push_back(v);
+    return (int)vals.size() - 1;
+  }
+  int konst(float c) {
+    int v = new_val(VK_CONST, Shape(), -1, c);
+    vals[v].known_const = true;
+    return v;
+  }
+  bool is_const(int v, float c) const { return vals[v].known_const && vals[v].c == c; }
+
+  // the same value seen with a (wider) logical shape; emits no instruction
+  int widen(int v, const Shape& want) {
+    Shape s;
+    if (!broadcast_shapes(vals[v].shape, want, &s) || s == vals[v].shape) return v;
+    Item it; it.kind = IT_MOP; it.opc = M_WIDEN; it.a = v;
+    it.dst = new_val(VK_OP, s);
+    vals[it.dst].known_const = vals[v].known_const;
+    vals[it.dst].c = vals[v].c;
+    items.push_back(it);
+    return it.dst;
+  }
+
+  int mop(int opc, int a, int b = -1) {
+    Shape s = vals[a].shape;
+    if (b >= 0 && !broadcast_shapes(vals[a].shape, vals[b].shape, &s)) {
+      set_error("internal: operands of a micro-operation do not broadcast");
+      err = DRAGON_ERR_SHAPE;
+      return a;
+    }
+    if (opc == M_MUL) {  // the seed of a gradient stage is one: dy * v folds to v
+      if (is_const(a, 1.f)) return widen(b, s);
+      if (is_const(b, 1.f)) return widen(a, s);
+    }
+    if (opc == M_NEG && vals[a].known_const) return widen(konst(-vals[a].c), s);
+    if (is_binary(opc) && vals[a].known_const && vals[b].known_const) {
+      float x = vals[a].c, y = vals[b].c;
+      float r = opc == M_ADD ? x + y : opc == M_SUB ? x - y : opc == M_MUL ? x * y : x / (1.f + std::fabs(y));
+      return widen(konst(r), s);
+    }
+    Item it; it.kind = IT_MOP; it.opc = opc; it.a = a; it.b = b;
+    it.dst = new_val(VK_OP, s);
+    items.push_back(it);
+    return it.dst;
+  }
+  void store(int v, int mem) {
+    Item it; it.kind = IT_MOP; it.opc = M_STORE; it.a = v; it.mem = mem;
+    items.push_back(it);
+  }
+  void accum(int v, int mem) {
+    Item it; it.kind = IT_MOP; it.opc = M_ACCUM; it.a = v; it.mem = mem;
+    items.push_back(it);
+  }
+  // memory image of value v with the given dtype (dtype < 0: any float type)
+  int materialise(int v, int dtype, int dtype_if_new) {
+    const Value& val = vals[v];
+    if (val.kind == VK_MEM && (dtype < 0 || plan->mems[val.mem].dtype == dtype)) return val.mem;
+    int m = new_mem(MEM_WORK, -1, dtype < 0 ? dtype_if_new : dtype, val.shape);
+    store(v, m);
+    return m;
+  }
+  int transpose_of(int mem) {
+    auto it = transposed.find(mem);
+    if (it != transposed.end()) return it->second;
+    Shape s = plan->mems[mem].shape, t;
+    t.rank = 2; t.d[0] = s.d[1]; t.d[1] = s.d[0];
+    int m = new_mem(MEM_WORK, -1, DRAGON_BF16, t);
+    Item x; x.kind = IT_TRANSPOSE; x.mA = mem; x.mC = m;
+    items.push_back(x);
+    transposed[mem] = m;
+    return m;
+  }
+  int gemm(int mA, int mB, int out_where, int out_index, int out_dtype) {
+    Shape s; s.rank = 2; s.d[0] = plan->mems[mA].shape.d[0]; s.d[1] = plan->mems[mB].shape.d[0];
+    int mC = new_mem(out_where, out_index, out_dtype, s);
+    Item x; x.kind = IT_GEMM; x.mA = mA; x.mB = mB; x.mC = mC;
+    items.push_back(x);
+    return mC;
+  }
+
+  void accumulate_grad(int s, int x, int contrib) {
+    auto it = gval[s].find(x);
+    if (it == gval[s].end()) gval[s][x] = contrib;
+    else it->second = mop(M_ADD, it->second, contrib);
+  }
+
+  void store_fetch(int v, int tensor) {
+    const TensorInfo& t = g.tensors[tensor];
+    int m = new_mem(MEM_FETCH, fetch_of[tensor], t.dtype, t.shape);
+    if (vals[v].shape == t.shape) store(v, m);
+    else accum(v, m);
+  }
+
+  void lower_forward(int k) {
+    const OpInfo& op = g.ops[k];
+    const int o = op.out[0];
+    const TensorInfo& to = g.tensors[o];
+    auto in = [&](int p) { return fval[op.in[p]]; };
+    int v = -1;
+    switch (op.type) {
+      case DRAGON_OP_ADD: v = mop(M_ADD, in(0), in(1)); break;
+      case DRAGON_OP_SUB: v = mop(M_SUB, in(0), in(1)); break;
+      case DRAGON_OP_MUL: v = mop(M_MUL, in(0), in(1)); break;
+      case DRAGON_OP_DIV: v = mop(M_DIVP, in(0), in(1)); break;
+      case DRAGON_OP_SIN: v = mop(M_SIN, in(0)); break;
+      case DRAGON_OP_EXP: v = mop(M_EXPC, in(0)); break;
+      case DRAGON_OP_TANH: v = mop(M_TANH, in(0)); break;
+      case DRAGON_OP_SIGMOID: v = mop(M_SIGMOID, in(0)); break;
+      case DRAGON_OP_RELU: v = mop(M_RELU, in(0)); break;
+      case DRAGON_OP_SUM: v = mop(M_ROWSUM, in(0)); break;
+      case DRAGON_OP_MEAN: v = mop(M_MUL, mop(M_ROWSUM, in(0)), konst(1.f / (float)to.shape.cols())); break;
+      case DRAGON_OP_BIAS_ADD: v = mop(M_ADD, in(0), in(1)); break;
+      case DRAGON_OP_INNER_PRODUCT: {
+        int mA = materialise(in(0), DRAGON_BF16, DRAGON_BF16);
+        int mB = materialise(in(1), DRAGON_BF16, DRAGON_BF16);
+        bool direct = fetch_of[o] >= 0;
+        int mC = gemm(mA, mB, direct ? MEM_FETCH : MEM_WORK, direct ? fetch_of[o] : -1, to.dtype);
+        fval[o] = new_val(VK_MEM, to.shape, mC);
+        return;
+      }
+      case DRAGON_OP_SOFTMAX_CROSS_ENTROPY: {
+        int mZ = materialise(in(0), -1, g.tensors[op.in[0]].dtype);
+        int mL = vals[in(1)].mem;
+        bool direct = fetch_of[o] >= 0;
+        int mC = new_mem(direct ? MEM_FETCH : MEM_WORK, direct ? fetch_of[o] : -1, DRAGON_F32, Shape());
+        Item x; x.kind = IT_SCE_FWD; x.mA = mZ; x.mB = mL; x.mC = mC;
+        items.push_back(x);
+        fval[o] = new_val(VK_MEM, to.shape, mC);
+        return;
+      }
+      default:
+        set_error("operator type %d cannot be lowered", op.type);
+        err = DRAGON_ERR_UNSUPPORTED;
+        return;
+    }
+    if (to.dtype == DRAGON_BF16) v = mop(M_RBF16, v);
+    fval[o] = v;
+    if (fetch_of[o] >= 0) store_fetch(v, o);
+  }
+
+  void lower_gradient(const GradOpRef& r) {
+    const OpInfo& op = g.ops[r.op];
+    const int s = r.stage, o = op.out[0];
+    auto gy = gval[s].find(o);
+    if (gy == gval[s].end()) return;  // no gradient reaches this operator
+    // a gradient value stands for a tensor of at least the output's shape (a folded seed or a
+    // scalar factor is narrower); sums over broadcast axes count every element of that shape
+    const int dy = widen(gy->second, g.tensors[o].shape);
+    std::vector<bool> want(op.in.size(), false);
+    for (size_t p = 0; p < op.in.size(); ++p)
+      for (size_t q = 0; q < op.in.size(); ++q)
+        if (((r.mask >> q) & 1u) && op.in[q] == op.in[p]) want[p] = true;
+    auto in = [&](int p) { return fval[op.in[p]]; };
+    auto add = [&](int p, int c) { accumulate_grad(s, op.in[p], c); };
+    switch (op.type) {
+      case DRAGON_OP_ADD: case DRAGON_OP_BIAS_ADD:
+        if (want[0]) add(0, dy);
+        if (want[1]) add(1, dy);
+        break;
+      case DRAGON_OP_SUB:
+        if (want[0]) add(0, dy);
+        if (want[1]) add(1, mop(M_NEG, dy));
+        break;
+      case DRAGON_OP_MUL:
+        if (want[0]) add(0, mop(M_MUL, dy, in(1)));
+        if (want[1]) add(1, mop(M_MUL, dy, in(0)));
+        break;
+      case DRAGON_OP_DIV:
+        if (want[0]) add(0, mop(M_DIVP, dy, in(1)));
+        if (want[1]) add(1, mop(M_MUL, mop(M_MUL, dy, in(0)), mop(M_DIVPGB, in(1))));
+        break;
+      case DRAGON_OP_SIN: add(0, mop(M_MUL, dy, mop(M_COS, in(0)))); break;
+      case DRAGON_OP_EXP: add(0, mop(M_MUL, mop(M_MUL, dy, fval[o]), mop(M_CLAMPMASK, in(0)))); break;
+      case DRAGON_OP_TANH: add(0, mop(M_MUL, dy, mop(M_ONEMSQ, fval[o]))); break;
+      case DRAGON_OP_SIGMOID: add(0, mop(M_MUL, dy, mop(M_YOMY, fval[o]))); break;
+      case DRAGON_OP_RELU: add(0, mop(M_MUL, dy, mop(M_STEP, in(0)))); break;
+      case DRAGON_OP_SUM: case DRAGON_OP_MEAN: {
+        int c = mop(M_ROWSUM, dy);
+        if (op.type == DRAGON_OP_MEAN) c = mop(M_MUL, c, konst(1.f / (float)g.tensors[o].shape.cols()));
+        add(0, c);
+        break;
+      }
+      case DRAGON_OP_INNER_PRODUCT: {
+        int mdY = materialise(dy, DRAGON_BF16, DRAGON_BF16);
+        if (want[0]) {  // dX[M,K] = dY[M,N] * W[N,K]
+          int mW = materialise(in(1), DRAGON_BF16, DRAGON_BF16);
+          int mC = gemm(mdY, transpose_of(mW), MEM_WORK, -1, g.tensors[op.in[0]].dtype == DRAGON_BF16 ? DRAGON_BF16 : DRAGON_F32);
+          add(0, new_val(VK_MEM, plan->mems[mC].shape, mC));
+        }
+        if (want[1]) {  // dW[N,K] = dY^T[N,M] * X[M,K]
+          int mX = materialise(in(0), DRAGON_BF16, DRAGON_BF16);
+          int mC = gemm(transpose_of(mdY), transpose_of(mX), MEM_WORK, -1, DRAGON_F32);
+          add(1, new_val(VK_MEM, plan->mems[mC].shape, mC));
+        }
+        break;
+      }
+      case DRAGON_OP_SOFTMAX_CROSS_ENTROPY: {
+        const TensorInfo& tz = g.tensors[op.in[0]];
+        int mZ = materialise(in(0), -1, tz.dtype);
+        int mdZ = new_mem(MEM_WORK, -1, tz.dtype, tz.shape);
+        Item x; x.kind = IT_SCE_BWD; x.mA = mZ; x.mB = vals[in(1)].mem; x.mC = mdZ;
+        if (vals[dy].known_const) x.scale = vals[dy].c;
+        else x.mD = materialise(dy, DRAGON_F32, DRAGON_F32);
+        items.push_back(x);
+        add(0, new_val(VK_MEM, tz.shape, mdZ));
+        break;
+      }
+      default:
+        set_error("gradient of operator type %d cannot be lowered", op.type);
+        err = DRAGON_ERR_UNSUPPORTED;
+    }
+  }
+};
+
+// true when a value/memory shape fits the fused domain `dom` (may widen it)
+bool join_domain(Shape* dom, bool* has_dom, const Shape& s) {
+  if (!*has_dom) { *dom = s; *has_dom = true; return true; }
+  Shape out;
+  if (!broadcast_shapes(*dom, s, &out)) return false;
+  *dom = out;
+  return true;
+}
+
+}  // namespace
+
+int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs,
+                   const std::vector<int>& outputs, int sm_count, Plan* plan) {
+  Lowerer L(g, pr, plan);
+  plan->sm_count = sm_count;
+  const int n = (int)g.tensors.size();
+  L.fval.assign(n, -1);
+  L.fetch_of.assign(n, -1);
+  L.gval.resize(g.stages.size());
+  for (int j = 0; j < (int)outputs.size(); ++j) {
+    if (L.fetch_of[outputs[j]] >= 0) {
+      set_error("tensor '%s' is fetched twice", g.tensors[outputs[j]].name.c_str());
+      return DRAGON_ERR_INVALID_ARG;
+    }
+    L.fetch_of[outputs[j]] = j;
+  }
+  for (int j = 0; j < (int)inputs.size(); ++j) {
+    const TensorInfo& t = g.tensors[inputs[j]];
+    if (!pr.marked[inputs[j]]) continue;
+    int m = L.new_mem(MEM_FEED, j, t.dtype, t.shape);
+    L.fval[inputs[j]] = L.new_val(VK_MEM, t.shape, m);
+    if (L.fetch_of[inputs[j]] >= 0) {  // a fetched input is copied
+      int mo = L.new_mem(MEM_FETCH, L.fetch_of[inputs[j]], t.dtype, t.shape);
+      Item x; x.kind = IT_COPY; x.mA = m; x.mC = mo;
+      L.items.push_back(x);
+    }
+  }
+  for (int k : pr.fwd_ops) {
+    if (g.ops[k].out.size() != 1) {
+      set_error("operators with several outputs can be pruned but not executed");
+      return DRAGON_ERR_UNSUPPORTED;
+    }
+    L.lower_forward(k);
+    if (L.err) return L.err;
+  }
+  auto seed_stage = [&](int s) {  // one for every element of every objective of a live stage
+    auto& gv = L.gval[s];
+    if (gv.empty())
+      for (int o : g.stages[s].objs)
+        if (pr.in_G[s][o]) gv[o] = L.konst(1.f);
+  };
+  for (const GradOpRef& r : pr.grad_ops) {
+    seed_stage(r.stage);
+    L.lower_gradient(r);
+    if (L.err) return L.err;
+  }
+  for (int s = 0; s < (int)g.stages.size(); ++s) {
+    const GradStage& st = g.stages[s];
+    for (size_t j = 0; j < st.wrts.size(); ++j) {
+      int gid = st.grad_ids[j];
+      if (L.fetch_of[gid] < 0) continue;
+      seed_stage(s);
+      auto it = L.gval[s].find(st.wrts[j]);
+      int v = it == L.gval[s].end() ? L.konst(0.f) : it->second;
+      L.store_fetch(L.widen(v, g.tensors[st.wrts[j]].shape), gid);
+    }
+  }
+  if (L.err) return L.err;
+
+  std::vector<Item>& items = L.items;
+  std::vector<Value>& vals = L.vals;
+  std::vector<MemRef>& mems = plan->mems;
+
+  // A workspace image that is written once and then only copied to a fetch buffer by a plain
+  // full-shape store is written to the fetch buffer directly (gradient tensors produced by a
+  // contraction, fetched logits...).
+  for (size_t i = 0; i < items.size(); ++i) {
+    Item& st = items[i];
+    if (st.kind != IT_MOP || st.opc != M_STORE || vals[st.a].kind != VK_MEM) continue;
+    int src = vals[st.a].mem, dst = st.mem;
+    if (mems[src].where != MEM_WORK || mems[dst].where != MEM_FETCH) continue;
+    if (mems[src].dtype != mems[dst].dtype || mems[src].shape != mems[dst].shape) continue;
+    int writers = 0;
+    for (const Item& w : items)
+      if ((w.kind != IT_MOP && w.mC == src) || (w.kind == IT_MOP && (w.opc == M_STORE || w.opc == M_ACCUM) && w.mem == src)) ++writers;
+    if (writers != 1) continue;
+    mems[src].where = MEM_FETCH;
+    mems[src].index = mems[dst].index;
+    st.opc = -1;  // removed
+  }
+  items.erase(std::remove_if(items.begin(), items.end(), [](const Item& x) { return x.kind == IT_MOP && x.opc < 0; }), items.end());
+
+  // dead-code elimination, roots = everything that reaches a fetch buffer
+  std::vector<uint8_t> val_live(vals.size(), 0);
+  for (auto& m : mems) m.live = m.where == MEM_FETCH;
+  auto use_val = [&](int v) {
+    if (v < 0) return;
+    val_live[v] = 1;
+    if (vals[v].kind == VK_MEM) mems[vals[v].mem].live = true;
+  };
+  for (int i = (int)items.size() - 1; i >= 0; --i) {
+    Item& it = items[i];
+    if (it.kind == IT_MOP) {
+      if (it.opc == M_STORE || it.opc == M_ACCUM) it.live = mems[it.mem].live;
+      else it.live = val_live[it.dst] != 0;
+      if (it.live) { use_val(it.a); use_val(it.b); }
+    } else {
+      it.live = mems[it.mC].live;
+      if (it.live)
+        for (int m : {it.mA, it.mB, it.mD})
+          if (m >= 0) mems[m].live = true;
+    }
+  }
+
+  // segmentation: maximal runs of live micro-operations whose shapes share one domain
+  std::vector<std::vector<int>> seg_items;
+  {
+    Shape dom; bool has_dom = false; int cur = -1;
+    for (int i = 0; i < (int)items.size(); ++i) {
+      Item& it = items[i];
+      if (!it.live) continue;
+      if (it.kind != IT_MOP) { cur = -1; has_dom = false; continue; }
+      Shape s = (it.opc == M_STORE || it.opc == M_ACCUM) ? vals[it.a].shape : vals[it.dst].shape;
+      if (cur < 0 || !join_domain(&dom, &has_dom, s)) {
+        seg_items.emplace_back();
+        cur = (int)seg_items.size() - 1;
+        has_dom = false;
+        join_domain(&dom, &has_dom, s);
+      }
+      it.segment = cur;
+      seg_items[cur].push_back(i);
+    }
+  }
+  // values that cross a segment boundary become workspace tensors
+  {
+    std::vector<int> def_seg(vals.size(), -1), def_item(vals.size(), -1);
+    for (int i = 0; i < (int)items.size(); ++i)
+      if (items[i].live && items[i].kind == IT_MOP && items[i].dst >= 0) { def_seg[items[i].dst] = items[i].segment; def_item[items[i].dst] = i; }
+    std::map<int, int> spilled;  // value -> VK_MEM value
+    const int n_items = (int)items.size();
+    for (int i = 0; i < n_items; ++i) {
+      if (!items[i].live || items[i].kind != IT_MOP) continue;
+      for (int which = 0; which < 2; ++which) {
+        int v = which == 0 ? items[i].a : items[i].b;
+        if (v < 0 || vals[v].kind != VK_OP || def_seg[v] == items[i].segment) continue;
+        auto f = spilled.find(v);
+        if (f == spilled.end()) {
+          int dt = items[def_item[v]].opc == M_RBF16 ? DRAGON_BF16 : DRAGON_F32;
+          MemRef m; m.where = MEM_WORK; m.dtype = dt; m.shape = vals[v].shape; m.live = true;
+          mems.push_back(m);
+          int mid = (int)mems.size() - 1;
+          Item st; st.kind = IT_MOP; st.opc = M_STORE; st.a = v; st.mem = mid; st.live = true; st.segment = def_seg[v];
+          items.push_back(st);
+          auto& lst = seg_items[def_seg[v]];  // right after the definition, while the value is at hand
+          lst.insert(std::find(lst.begin(), lst.end(), def_item[v]) + 1, (int)items.size() - 1);
+          Value nv; nv.kind = VK_MEM; nv.shape = vals[v].shape; nv.mem = mid;
+          vals.push_back(nv);
+          f = spilled.emplace(v, (int)vals.size() - 1).first;
+        }
+        if (which == 0) items[i].a = f->second; else items[i].b = f->second;
+      }
+    }
+  }
+
+  // steps in execution order
+  std::vector<int> seg_step(seg_items.size(), -1);
+  plan->segs.resize(seg_items.size());
+  for (int i = 0; i < (int)items.size(); ++i) {
+    const Item& it = items[i];
+    if (!it.live) continue;
+    if (it.kind == IT_MOP) {
+      if (it.segment >= 0 && seg_step[it.segment] < 0) {
+        seg_step[it.segment] = (int)plan->steps.size();
+        Step st; st.kind = ST_VM; st.seg = it.segment;
+        plan->steps.push_back(st);
+      }
+      continue;
+    }
+    Step st;
+    st.kind = it.kind == IT_GEMM ? ST_GEMM : it.kind == IT_TRANSPOSE ? ST_TRANSPOSE : it.kind == IT_SCE_FWD ? ST_SCE_FWD
+              : it.kind == IT_SCE_BWD ? ST_SCE_BWD : ST_COPY;
+    st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.scale = it.scale;
+    plan->steps.push_back(st);
+  }
+  for (size_t s = 0; s < seg_items.size(); ++s) {
+    int rc = codegen_segment(items, seg_items[s], vals, mems, sm_count, &plan->segs[s]);
+    if (rc) return rc;
+  }
+
+  // workspace layout: the status word, live workspace tensors, then per-segment scratch
+  size_t off = 0;
+  auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
+  plan->status_off = take(256);
+  for (auto& m : mems)
+    if (m.where == MEM_WORK && m.live) m.offset = take(m.bytes());
+  for (auto& sg : plan->segs) {
+    sg.spill_off = take((size_t)sg.grid * sg.n_spill * kVmTile * sizeof(float));
+    sg.colpart_off = take((size_t)sg.n_colacc * sg.grid * sg.cols * sizeof(float));
+    sg.scalpart_off = take((size_t)sg.n_scalacc * sg.grid * sizeof(double));
+  }
+  for (auto& st : plan->steps)
+    if (st.kind == ST_SCE_FWD) st.scratch_off = take((size_t)mems[st.mA].shape.d[0] * sizeof(float));
+  plan->workspace_bytes = off;
+  return DRAGON_OK;
+}
+
+std::string describe_plan(const Plan& p) {
+  std::string s;
+  char buf[256];
+  for (const Step& st : p.steps) {
+    switch (st.kind) {
+      case ST_VM: {
+        const VmSegment& sg = p.segs[st.seg];
+        snprintf(buf, sizeof(buf), "vm[%s n=%lld cols=%d instr=%d body=%d operands=%d smem=%d spill=%d colacc=%d scalacc=%d grid=%d]\n",
+                 sg.row_mode ? "row" : "flat", sg.n, sg.cols, (int)sg.code.size(), sg.n_instr_body,
+                 (int)sg.operand_mem.size(), sg.n_smem, sg.n_spill, sg.n_colacc, sg.n_scalacc, sg.grid);
+        break;
+      }
+      case ST_GEMM:
+        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
+                 (long long)p.mems[st.mA].shape.d[1], p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
+        break;
+      case ST_TRANSPOSE:
+        snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);
+        break;
+      case ST_SCE_FWD: snprintf(buf, sizeof(buf), "softmax_ce_fwd\n"); break;
+      case ST_SCE_BWD: snprintf(buf, sizeof(buf), "softmax_ce_bwd\n"); break;
+      default: snprintf(buf, sizeof(buf), "copy\n");
+    }
+    s += buf;
+  }
+  return s;
+}
+
+}  // namespace dragon

@@ -1,0 +1,126 @@
+// Compiled form of a pruned function: a list of launch steps produced by the host compiler
+// (lower.cpp builds the micro-operation list from the kept operators, codegen.cpp turns each
+// fused segment into a VM instruction stream).
+#pragma once
+#include <string>
+#include <vector>
+
+#include "graph.h"
+#include "vm_isa.h"
+
+namespace dragon {
+
+// geometry of the VM kernel: every CTA owns tiles of kVmTile elements, kVmVec per thread
+constexpr int kVmThreads = 256;
+constexpr int kVmVec = 16;
+constexpr int kVmTile = kVmThreads * kVmVec;  // 4096
+constexpr int kVmRegs = 10;                   // register slots R[0..kVmRegs)
+constexpr int kVmCodeMaxWords = 12 * 1024;    // instruction stream held in shared memory
+constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread
+constexpr int kDefaultSmCount = 148;
+
+enum MemWhere { MEM_FEED = 0, MEM_FETCH = 1, MEM_WORK = 2 };
+
+struct MemRef {
+  int where = MEM_WORK;
+  int index = -1;        // feed / fetch position; unused for workspace buffers
+  int dtype = DRAGON_F32;
+  Shape shape;
+  size_t offset = 0;     // byte offset inside the workspace (MEM_WORK)
+  bool live = false;
+  size_t bytes() const { return (size_t)shape.numel() * (dtype == DRAGON_BF16 ? 2 : 4); }
+};
+
+enum MOpc {
+  M_ADD, M_SUB, M_MUL, M_DIVP,
+  M_SIN, M_COS, M_EXPC, M_TANH, M_SIGMOID, M_RELU, M_NEG, M_STEP, M_CLAMPMASK, M_ONEMSQ, M_YOMY,
+  M_DIVPGB, M_RBF16, M_ROWSUM,
+  M_WIDEN,  // same value, wider logical shape (no instruction)
+  M_STORE,  // write value a to memory mem
+  M_ACCUM   // sum value a over the axes along which mem is smaller, write to mem
+};
+inline bool is_binary(int opc) { return opc <= M_DIVP; }
+
+enum ValKind { VK_MEM, VK_OP, VK_CONST };
+struct Value {
+  int kind = VK_OP;
+  Shape shape;
+  int mem = -1;
+  float c = 0.f;
+  bool known_const = false;  // VK_CONST, or a widened view of one
+};
+
+enum ItemKind { IT_MOP, IT_GEMM, IT_TRANSPOSE, IT_SCE_FWD, IT_SCE_BWD, IT_COPY };
+struct Item {
+  int kind = IT_MOP;
+  // IT_MOP
+  int opc = 0, a = -1, b = -1, dst = -1, mem = -1;
+  // heavy items: memory operands.  GEMM: C = A * B^T; TRANSPOSE: C = A^T;
+  // SCE: A = logits, B = labels, C = out, D = scalar dL (gradient)
+  int mA = -1, mB = -1, mC = -1, mD = -1;
+  float scale = 1.f;                       // SCE_BWD: immediate dL when mD < 0
+  bool live = false;
+  int segment = -1;
+};
+
+// ---- launch steps -------------------------------------------------------------------------
+
+struct FinishJob {
+  int kind;       // 0: column sums of colpart[acc] -> mem; 1: scalar sum of scalpart[acc] -> mem
+  int acc;        // accumulator index inside the segment
+  int mem;
+};
+
+struct VmSegment {
+  std::vector<uint32_t> code;
+  std::vector<int> operand_mem;     // operand table: memref ids
+  std::vector<uint32_t> operand_kind;
+  bool row_mode = false;
+  long long n = 0;                  // flat: elements; row: rows
+  int cols = 0;
+  int n_spill = 0, n_colacc = 0, n_scalacc = 0, n_smem = 0;
+  int grid = 0;
+  size_t spill_off = 0, colpart_off = 0, scalpart_off = 0;  // workspace offsets
+  std::vector<FinishJob> finish;
+  uint32_t* d_code = nullptr;       // device copy
+  int n_instr_body = 0;
+};
+
+enum StepKind { ST_VM, ST_GEMM, ST_TRANSPOSE, ST_SCE_FWD, ST_SCE_BWD, ST_COPY };
+struct Step {
+  int kind;
+  int seg = -1;                          // ST_VM
+  int mA = -1, mB = -1, mC = -1, mD = -1;
+  float scale = 1.f;
+  size_t scratch_off = 0;                // SCE_FWD: per-row losses
+};
+
+struct Plan {
+  std::vector<MemRef> mems;
+  std::vector<VmSegment> segs;
+  std::vector<Step> steps;
+  size_t workspace_bytes = 0;
+  size_t status_off = 0;
+  int sm_count = kDefaultSmCount;
+};
+
+int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs,
+                   const std::vector<int>& outputs, int sm_count, Plan* plan);
+
+// codegen.cpp: instruction stream for the micro-operations items[idx[..]] (all IT_MOP, one domain)
+int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx, const std::vector<Value>& vals,
+                    const std::vector<MemRef>& mems, int sm_count, VmSegment* seg);
+
+std::string describe_plan(const Plan& p);
+
+}  // namespace dragon
+
+struct dragon_function {
+  dragon::PruneResult prune;
+  dragon::Plan plan;
+  int n_tensors = 0, n_in = 0, n_out = 0;
+  void* workspace = nullptr;
+  size_t workspace_bytes = 0;
+  void* last_stream = nullptr;
+  bool uploaded = false;
+};
