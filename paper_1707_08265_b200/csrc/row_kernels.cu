@@ -1,0 +1,118 @@
+// Row kernels around the contraction: SoftmaxCrossEntropy forward / gradient (one CTA per
+// row: warp-shuffle + shared-memory reductions), the mean of the per-row losses, and the bf16
+// transpose that feeds K-major operands to the tensor-core GEMM.
+#include <cuda_runtime.h>
+
+#include "plan.h"
+#include "vm_math.h"
+
+namespace dragon {
+namespace {
+
+constexpr int kRowThreads = 256;
+
+__device__ __forceinline__ float load_logit(const void* z, int dtype, size_t i) {
+  return dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(z) + i)
+                             : __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(z) + i) << 16);
+}
+
+template <bool kMax>
+__device__ __forceinline__ float block_reduce(float v, float* sh) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float w = __shfl_xor_sync(0xffffffffu, v, o);
+    v = kMax ? fmaxf(v, w) : v + w;
+  }
+  if ((threadIdx.x & 31) == 0) sh[threadIdx.x >> 5] = v;
+  __syncthreads();
+  float r = sh[0];
+#pragma unroll
+  for (int i = 1; i < kRowThreads / 32; ++i) r = kMax ? fmaxf(r, sh[i]) : r + sh[i];
+  __syncthreads();
+  return r;
+}
+
+// mode 0: rowloss[m] = logsumexp(z[m,:]) - z[m,label];  mode 1: dz[m,j] = dL/M * (softmax - onehot)
+template <int kMode>
+__global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdtype, const int* labels, int rows, int cols,
+                                                          float* rowloss, void* dz, int dzdtype, const float* dl_ptr,
+                                                          float dl_imm, int* status) {
+  __shared__ float sh[kRowThreads / 32];
+  const int m = blockIdx.x;
+  const size_t off = (size_t)m * cols;
+  float mx = -INFINITY;
+  for (int j = threadIdx.x; j < cols; j += kRowThreads) mx = fmaxf(mx, load_logit(z, zdtype, off + j));
+  mx = block_reduce<true>(mx, sh);
+  float se = 0.f;
+  for (int j = threadIdx.x; j < cols; j += kRowThreads) se += vmmath::exp_wide(load_logit(z, zdtype, off + j) - mx);
+  se = block_reduce<false>(se, sh);
+  const int lab = __ldg(labels + m);
+  const bool ok = lab >= 0 && lab < cols;
+  if (!ok && threadIdx.x == 0) atomicExch(status, DRAGON_ERR_INVALID_ARG);
+  if (kMode == 0) {
+    if (threadIdx.x == 0) rowloss[m] = ok ? (logf(se) + mx - load_logit(z, zdtype, off + lab)) : 0.f;
+  } else {
+    const float dl = dl_ptr ? __ldg(dl_ptr) : dl_imm;
+    const float sc = dl / (float)rows, inv = 1.f / se;
+    for (int j = threadIdx.x; j < cols; j += kRowThreads) {
+      float g = vmmath::exp_wide(load_logit(z, zdtype, off + j) - mx) * inv;
+      if (ok && j == lab) g -= 1.f;
+      g = ok ? g * sc : 0.f;
+      if (dzdtype == DRAGON_F32) reinterpret_cast<float*>(dz)[off + j] = g;
+      else reinterpret_cast<unsigned short*>(dz)[off + j] = (unsigned short)vmmath::bf16_bits(g);
+    }
+  }
+}
+
+__global__ void __launch_bounds__(kRowThreads) mean_kernel(const float* v, int n, float* out) {
+  __shared__ double sh[kRowThreads];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n; i += kRowThreads) s += (double)v[i];
+  sh[threadIdx.x] = s;
+  __syncthreads();
+  for (int o = kRowThreads / 2; o > 0; o >>= 1) {
+    if (threadIdx.x < o) sh[threadIdx.x] += sh[threadIdx.x + o];
+    __syncthreads();
+  }
+  if (threadIdx.x == 0) *out = (float)(sh[0] / (double)n);
+}
+
+// out[c, r] = in[r, c], 16-bit elements, 64x64 tiles through shared memory
+__global__ void __launch_bounds__(256) transpose16_kernel(const unsigned short* __restrict__ in, unsigned short* __restrict__ out,
+                                                           int rows, int cols) {
+  __shared__ unsigned short tile[64][64 + 2];
+  const int r0 = blockIdx.y * 64, c0 = blockIdx.x * 64;
+  const int tx = threadIdx.x & 63, ty = threadIdx.x >> 6;
+  for (int i = ty; i < 64; i += 4) {
+    const int r = r0 + i, c = c0 + tx;
+    tile[i][tx] = (r < rows && c < cols) ? in[(size_t)r * cols + c] : (unsigned short)0;
+  }
+  __syncthreads();
+  for (int i = ty; i < 64; i += 4) {
+    const int c = c0 + i, r = r0 + tx;
+    if (c < cols && r < rows) out[(size_t)c * rows + r] = tile[tx][i];
+  }
+}
+
+}  // namespace
+
+cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
+                           int* status, cudaStream_t st) {
+  sce_kernel<0><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
+  mean_kernel<<<1, kRowThreads, 0, st>>>(rowloss, rows, out);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
+                           const float* dl_ptr, float dl_imm, int* status, cudaStream_t st) {
+  sce_kernel<1><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cudaStream_t st) {
+  dim3 grid((cols + 63) / 64, (rows + 63) / 64);
+  transpose16_kernel<<<grid, 256, 0, st>>>(reinterpret_cast<const unsigned short*>(in), reinterpret_cast<unsigned short*>(out), rows, cols);
+  return cudaGetLastError();
+}
+
+}  // namespace dragon

@@ -1,0 +1,394 @@
+// The graph-VM kernel: interprets the instruction stream of one fused segment (vm_isa.h).
+//
+// Geometry: 256 threads per CTA, one CTA per SM (the whole register file belongs to it), 16
+// elements per thread held as four 128-bit vectors that are each contiguous across the warp,
+// so a tile is 4096 elements.  Flat mode walks the element range tile by tile (grid-stride);
+// row mode gives every tile one row of the [rows, cols] domain, which makes a row reduction a
+// CTA-wide reduction and a column reduction a per-thread running sum.  The instruction stream
+// and the uniforms sit in shared memory; the accumulator and the register slots are C arrays
+// that are only ever indexed with compile-time constants (every register-operand instruction
+// is its own switch case), so they live in registers.  One decoded instruction is amortised
+// over 16 element operations per thread, and the next instruction word is fetched before the
+// current one executes.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+
+#include "plan.h"
+#include "vm_math.h"
+
+namespace dragon {
+namespace vm {
+
+constexpr int NT = kVmThreads;
+constexpr int V = kVmVec;
+constexpr int NV4 = V / 4;
+constexpr int NR = kVmRegs;
+constexpr int TILE = kVmTile;
+static_assert(V == 16 && NR == 10 && NT == 256, "the case tables below are written for 16 lanes and 10 register slots");
+
+#define FORV _Pragma("unroll") for (int j = 0; j < V; ++j)
+
+struct TileCtx {
+  long long base;   // element offset of this tile for FULL operands
+  int limit;        // valid elements in the tile (TILE when full)
+  bool full;        // limit == TILE
+  bool vec_ok;      // 4-element groups are 16-byte aligned
+  bool first;       // tile 0 (stores of ROW / SCALAR shaped outputs happen here)
+};
+
+__device__ __forceinline__ int lane_pos(int tid, int j) { return (j >> 2) * (NT * 4) + tid * 4 + (j & 3); }
+
+__device__ __forceinline__ void load_operand(const Operand& o, const TileCtx& tc, int tid, float* t) {
+  const long long base = o.kind == K_FULL ? tc.base : 0;
+  if (o.dtype == DRAGON_F32) {
+    const float* p = reinterpret_cast<const float*>(o.ptr) + base;
+#pragma unroll
+    for (int h = 0; h < NV4; ++h) {
+      const int pos = h * NT * 4 + tid * 4;
+      if (tc.vec_ok && pos + 3 < tc.limit) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p + pos));
+        t[4 * h + 0] = v.x; t[4 * h + 1] = v.y; t[4 * h + 2] = v.z; t[4 * h + 3] = v.w;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) t[4 * h + e] = (pos + e < tc.limit) ? __ldg(p + pos + e) : 0.f;
+      }
+    }
+  } else {
+    const unsigned short* p = reinterpret_cast<const unsigned short*>(o.ptr) + base;
+#pragma unroll
+    for (int h = 0; h < NV4; ++h) {
+      const int pos = h * NT * 4 + tid * 4;
+      if (tc.vec_ok && pos + 3 < tc.limit) {
+        const uint2 v = __ldg(reinterpret_cast<const uint2*>(p + pos));
+        t[4 * h + 0] = __uint_as_float(v.x << 16); t[4 * h + 1] = __uint_as_float(v.x & 0xffff0000u);
+        t[4 * h + 2] = __uint_as_float(v.y << 16); t[4 * h + 3] = __uint_as_float(v.y & 0xffff0000u);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          t[4 * h + e] = (pos + e < tc.limit) ? __uint_as_float((unsigned)__ldg(p + pos + e) << 16) : 0.f;
+      }
+    }
+  }
+}
+
+__device__ __forceinline__ void store_operand(const Operand& o, const TileCtx& tc, int tid, const float* t) {
+  if (o.kind == K_SCALAR) {
+    if (tc.first && tid == 0) {
+      if (o.dtype == DRAGON_F32) *reinterpret_cast<float*>(o.ptr) = t[0];
+      else *reinterpret_cast<unsigned short*>(o.ptr) = (unsigned short)vmmath::bf16_bits(t[0]);
+    }
+    return;
+  }
+  if (o.kind == K_ROW && !tc.first) return;
+  const long long base = o.kind == K_FULL ? tc.base : 0;
+  if (o.dtype == DRAGON_F32) {
+    float* p = reinterpret_cast<float*>(o.ptr) + base;
+#pragma unroll
+    for (int h = 0; h < NV4; ++h) {
+      const int pos = h * NT * 4 + tid * 4;
+      if (tc.vec_ok && pos + 3 < tc.limit) {
+        *reinterpret_cast<float4*>(p + pos) = make_float4(t[4 * h], t[4 * h + 1], t[4 * h + 2], t[4 * h + 3]);
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (pos + e < tc.limit) p[pos + e] = t[4 * h + e];
+      }
+    }
+  } else {
+    unsigned short* p = reinterpret_cast<unsigned short*>(o.ptr) + base;
+#pragma unroll
+    for (int h = 0; h < NV4; ++h) {
+      const int pos = h * NT * 4 + tid * 4;
+      if (tc.vec_ok && pos + 3 < tc.limit) {
+        uint2 v;
+        v.x = vmmath::bf16_bits(t[4 * h]) | (vmmath::bf16_bits(t[4 * h + 1]) << 16);
+        v.y = vmmath::bf16_bits(t[4 * h + 2]) | (vmmath::bf16_bits(t[4 * h + 3]) << 16);
+        *reinterpret_cast<uint2*>(p + pos) = v;
+      } else {
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (pos + e < tc.limit) p[pos + e] = (unsigned short)vmmath::bf16_bits(t[4 * h + e]);
+      }
+    }
+  }
+}
+
+// every joint instruction for register slot K
+#define JOINT_CASES(K)                                                                            \
+  case J_LDR * kJointStride + K: FORV acc[j] = R[K][j]; break;                                    \
+  case J_STR * kJointStride + K: FORV R[K][j] = acc[j]; break;                                    \
+  case J_ADD * kJointStride + K: FORV acc[j] = acc[j] + R[K][j]; break;                           \
+  case J_SUB * kJointStride + K: FORV acc[j] = acc[j] - R[K][j]; break;                           \
+  case J_RSUB * kJointStride + K: FORV acc[j] = R[K][j] - acc[j]; break;                          \
+  case J_MUL * kJointStride + K: FORV acc[j] = acc[j] * R[K][j]; break;                           \
+  case J_DIVP * kJointStride + K: FORV acc[j] = vmmath::divp_f(acc[j], R[K][j]); break;           \
+  case J_RDIVP * kJointStride + K: FORV acc[j] = vmmath::divp_f(R[K][j], acc[j]); break;          \
+  case J_ADDTO * kJointStride + K: FORV R[K][j] += acc[j]; break;                                 \
+  case J_ACCUM * kJointStride + K:                                                                \
+    if (tc.full) { FORV R[K][j] += acc[j]; }                                                      \
+    else { FORV R[K][j] += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }                        \
+    break;                                                                                        \
+  case J_FMAUR * kJointStride + K: { const float u_ = U[arg]; FORV acc[j] = fmaf(acc[j], u_, R[K][j]); } break;
+
+#define ALL_SLOTS(M) M(0) M(1) M(2) M(3) M(4) M(5) M(6) M(7) M(8) M(9)
+
+#define SEL_TO_T_CASE(K) case K: FORV t[j] = R[K][j]; break;
+#define SEL_FROM_T_CASE(K) case K: FORV R[K][j] = t[j]; break;
+#define SELECT_TO_T(r)                       \
+  switch (r) {                               \
+    ALL_SLOTS(SEL_TO_T_CASE)                 \
+    default: FORV t[j] = acc[j]; break;      \
+  }
+#define SELECT_FROM_T(r)                     \
+  switch (r) {                               \
+    ALL_SLOTS(SEL_FROM_T_CASE)               \
+    default: FORV acc[j] = t[j]; break;      \
+  }
+
+#define T_FROM_VEC4(h, v) { t[4 * (h)] = (v).x; t[4 * (h) + 1] = (v).y; t[4 * (h) + 2] = (v).z; t[4 * (h) + 3] = (v).w; }
+#define VEC4_FROM_T(h) make_float4(t[4 * (h)], t[4 * (h) + 1], t[4 * (h) + 2], t[4 * (h) + 3])
+
+__global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Params p) {
+  extern __shared__ __align__(16) unsigned char smem_raw[];
+  // layout: code | uniforms | reduction scratch | V-wide slots
+  uint32_t* code = reinterpret_cast<uint32_t*>(smem_raw);
+  const int code_words = (p.n_code + 3) & ~3;
+  float* U = reinterpret_cast<float*>(code + code_words);
+  double* red = reinterpret_cast<double*>(U + kMaxUniforms);
+  float4* slots = reinterpret_cast<float4*>(red + 64);
+
+  const int tid = threadIdx.x;
+  for (int i = tid; i < p.n_code; i += NT) code[i] = p.code[i];
+  __syncthreads();
+
+  float acc[V], t[V], R[NR][V];
+  FORV { acc[j] = 0.f; t[j] = 0.f; }
+#pragma unroll
+  for (int k = 0; k < NR; ++k) FORV R[k][j] = 0.f;
+
+  const long long ntiles = p.row_mode ? p.n : (p.n + TILE - 1) / TILE;
+  long long tile = blockIdx.x;
+  TileCtx tc;
+  int loop_pc = 0;
+  auto set_tile = [&]() {
+    if (p.row_mode) {
+      tc.base = tile * (long long)p.cols;
+      tc.limit = p.cols;
+      tc.vec_ok = (p.cols & 3) == 0;
+    } else {
+      tc.base = tile * (long long)TILE;
+      const long long left = p.n - tc.base;
+      tc.limit = left < TILE ? (int)left : TILE;
+      tc.vec_ok = true;
+    }
+    tc.full = tc.limit == TILE;
+    tc.first = tile == 0;
+  };
+  set_tile();
+  float* spill = p.spill + (size_t)blockIdx.x * p.n_spill * TILE;
+
+  int pc = 0;
+  uint32_t w = code[0];
+  for (;;) {
+    uint32_t wn = code[pc + 1];  // fetched ahead of the dispatch below
+    ++pc;
+    const int cs = w & 1023u;
+    const int r = (w >> 10) & 15u;
+    const uint32_t arg = w >> 14;
+    switch (cs) {
+      ALL_SLOTS(JOINT_CASES)
+      case P_LDU: { const float u = U[arg]; FORV acc[j] = u; } break;
+      case P_ADDU: { const float u = U[arg]; FORV acc[j] += u; } break;
+      case P_SUBU: { const float u = U[arg]; FORV acc[j] -= u; } break;
+      case P_RSUBU: { const float u = U[arg]; FORV acc[j] = u - acc[j]; } break;
+      case P_MULU: { const float u = U[arg]; FORV acc[j] *= u; } break;
+      case P_DIVPU: { const float u = vmmath::f_rcp(1.f + fabsf(U[arg])); FORV acc[j] *= u; } break;
+      case P_RDIVPU: { const float u = U[arg]; FORV acc[j] = vmmath::divp_f(u, acc[j]); } break;
+      case P_FMAU: { const float a = U[arg & 511u], b = U[arg >> 9]; FORV acc[j] = fmaf(acc[j], a, b); } break;
+      case P_LDS: case P_ADDS: case P_SUBS: case P_RSUBS: case P_MULS: case P_DIVPS: case P_RDIVPS: case P_STOR: {
+#pragma unroll
+        for (int h = 0; h < NV4; ++h) { const float4 v = slots[(arg * NV4 + h) * NT + tid]; T_FROM_VEC4(h, v) }
+        switch (cs) {
+          case P_LDS: FORV acc[j] = t[j]; break;
+          case P_ADDS: FORV acc[j] += t[j]; break;
+          case P_SUBS: FORV acc[j] -= t[j]; break;
+          case P_RSUBS: FORV acc[j] = t[j] - acc[j]; break;
+          case P_MULS: FORV acc[j] *= t[j]; break;
+          case P_DIVPS: FORV acc[j] = vmmath::divp_f(acc[j], t[j]); break;
+          case P_RDIVPS: FORV acc[j] = vmmath::divp_f(t[j], acc[j]); break;
+          default: SELECT_FROM_T(r) break;
+        }
+      } break;
+      case P_STS: case P_RTOS: {
+        if (cs == P_STS) { FORV t[j] = acc[j]; } else { SELECT_TO_T(r) }
+#pragma unroll
+        for (int h = 0; h < NV4; ++h) slots[(arg * NV4 + h) * NT + tid] = VEC4_FROM_T(h);
+      } break;
+      case P_SIN: FORV acc[j] = vmmath::sin_f(acc[j]); break;
+      case P_COS: FORV acc[j] = vmmath::cos_f(acc[j]); break;
+      case P_SINCOS: {
+        FORV { float s_, c_; vmmath::sincos_f(acc[j], &s_, &c_); acc[j] = s_; t[j] = c_; }
+        SELECT_FROM_T(r)
+      } break;
+      case P_EXPC: FORV acc[j] = vmmath::exp_clamped10(acc[j]); break;
+      case P_TANH: FORV acc[j] = vmmath::tanh_f(acc[j]); break;
+      case P_SIGMOID: FORV acc[j] = vmmath::sigmoid_f(acc[j]); break;
+      case P_RELU: FORV acc[j] = fmaxf(acc[j], 0.f); break;
+      case P_NEG: FORV acc[j] = -acc[j]; break;
+      case P_STEP: FORV acc[j] = acc[j] > 0.f ? 1.f : 0.f; break;
+      case P_CLAMPMASK: FORV acc[j] = (acc[j] >= -10.f && acc[j] <= 10.f) ? 1.f : 0.f; break;
+      case P_ONEMSQ: FORV acc[j] = fmaf(-acc[j], acc[j], 1.f); break;
+      case P_YOMY: FORV acc[j] = acc[j] * (1.f - acc[j]); break;
+      case P_DIVPGB: FORV acc[j] = vmmath::divp_grad_b(acc[j]); break;
+      case P_RBF16: FORV acc[j] = vmmath::round_bf16(acc[j]); break;
+      case P_ROWSUM: {
+        float s = 0.f;
+        if (tc.full) { FORV s += acc[j]; }
+        else { FORV s += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        float* redf = reinterpret_cast<float*>(red);
+        if ((tid & 31) == 0) redf[tid >> 5] = s;
+        __syncthreads();
+        float tot = 0.f;
+#pragma unroll
+        for (int i = 0; i < NT / 32; ++i) tot += redf[i];
+        __syncthreads();
+        FORV acc[j] = tot;
+      } break;
+      case P_GLD: {
+        load_operand(p.operand[arg], tc, tid, t);
+        SELECT_FROM_T(r)
+      } break;
+      case P_GST: {
+        SELECT_TO_T(r)
+        store_operand(p.operand[arg], tc, tid, t);
+      } break;
+      case P_FILL: {
+        const float4* s4 = reinterpret_cast<const float4*>(spill + (size_t)arg * TILE);
+#pragma unroll
+        for (int h = 0; h < NV4; ++h) { const float4 v = s4[h * NT + tid]; T_FROM_VEC4(h, v) }
+        SELECT_FROM_T(r)
+      } break;
+      case P_SPILL: {
+        SELECT_TO_T(r)
+        float4* s4 = reinterpret_cast<float4*>(spill + (size_t)arg * TILE);
+#pragma unroll
+        for (int h = 0; h < NV4; ++h) s4[h * NT + tid] = VEC4_FROM_T(h);
+      } break;
+      case P_ULOAD: {
+        if (tid == 0) {
+          const Operand& o = p.operand[arg >> 9];
+          U[arg & 511u] = o.dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(o.ptr))
+                                                : __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(o.ptr)) << 16);
+        }
+      } break;
+      case P_UCONST: {
+        if (tid == 0) U[arg] = __uint_as_float(wn);
+        ++pc;
+        wn = code[pc];
+      } break;
+      case P_LOOP_BEGIN:
+        __syncthreads();  // uniforms written by thread 0 are visible from here on
+        loop_pc = pc;
+        break;
+      case P_LOOP_END:
+        tile += gridDim.x;
+        if (tile < ntiles) { set_tile(); pc = loop_pc; wn = code[pc]; }
+        break;
+      case P_COLOUT: {
+        SELECT_TO_T(r)
+        float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
+        FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = t[j]; }
+      } break;
+      case P_SCALOUT: {
+        SELECT_TO_T(r)
+        double s = 0.0;
+        FORV s += (double)t[j];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+        if ((tid & 31) == 0) red[tid >> 5] = s;
+        __syncthreads();
+        if (tid == 0) {
+          double tot = 0.0;
+          for (int i = 0; i < NT / 32; ++i) tot += red[i];
+          p.scalpart[(size_t)arg * gridDim.x + blockIdx.x] = tot;
+        }
+        __syncthreads();
+      } break;
+      default:  // P_END and anything unknown
+        return;
+    }
+    w = wn;
+  }
+}
+
+// ---- finishing reductions: per-CTA partials -> tensors (fixed order, fp64) ------------------
+
+struct FinishParams {
+  int n_jobs;
+  struct Job {
+    int kind;          // 0 column sums, 1 scalar
+    const void* part;  // float [grid][cols] or double [grid]
+    void* out;
+    int dtype, cols, grid;
+  } job[8];
+};
+
+__global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
+  const FinishParams::Job& jb = fp.job[blockIdx.y];
+  if (jb.kind == 0) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= jb.cols) return;
+    const float* part = reinterpret_cast<const float*>(jb.part);
+    double s = 0.0;
+    for (int g = 0; g < jb.grid; ++g) s += (double)part[(size_t)g * jb.cols + c];
+    if (jb.dtype == DRAGON_F32) reinterpret_cast<float*>(jb.out)[c] = (float)s;
+    else reinterpret_cast<unsigned short*>(jb.out)[c] = (unsigned short)vmmath::bf16_bits((float)s);
+  } else if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const double* part = reinterpret_cast<const double*>(jb.part);
+    double s = 0.0;
+    for (int g = 0; g < jb.grid; ++g) s += part[g];
+    if (jb.dtype == DRAGON_F32) *reinterpret_cast<float*>(jb.out) = (float)s;
+    else *reinterpret_cast<unsigned short*>(jb.out) = (unsigned short)vmmath::bf16_bits((float)s);
+  }
+}
+
+size_t vm_smem_bytes(int n_code, int n_smem_slots) {
+  return (size_t)((n_code + 3) & ~3) * 4 + kMaxUniforms * 4 + 64 * 8 + (size_t)n_smem_slots * NV4 * NT * 16;
+}
+
+}  // namespace vm
+
+// launch helpers used by api.cu
+cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, cudaStream_t st) {
+  const size_t smem = vm::vm_smem_bytes(p.n_code, n_smem_slots);
+  cudaError_t e = cudaFuncSetAttribute(vm::vm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  if (e != cudaSuccess) return e;
+  vm::vm_kernel<<<grid, vm::NT, smem, st>>>(p);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st) {
+  if (sg.finish.empty()) return cudaSuccess;
+  vm::FinishParams fp;
+  fp.n_jobs = (int)sg.finish.size();
+  int max_cols = 1;
+  for (int i = 0; i < fp.n_jobs; ++i) {
+    const FinishJob& j = sg.finish[i];
+    auto& o = fp.job[i];
+    o.kind = j.kind;
+    o.grid = sg.grid;
+    o.cols = sg.cols;
+    o.dtype = mems[j.mem].dtype;
+    o.out = mem_ptr[j.mem];
+    if (j.kind == 0) { o.part = ws + sg.colpart_off + (size_t)j.acc * sg.grid * sg.cols * sizeof(float); max_cols = std::max(max_cols, sg.cols); }
+    else o.part = ws + sg.scalpart_off + (size_t)j.acc * sg.grid * sizeof(double);
+  }
+  dim3 grid((max_cols + 127) / 128, fp.n_jobs);
+  vm::finish_kernel<<<grid, 128, 0, st>>>(fp);
+  return cudaGetLastError();
+}
+
+}  // namespace dragon

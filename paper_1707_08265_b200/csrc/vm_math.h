@@ -1,0 +1,157 @@
+// Elementary functions of the graph VM, fp32, written for a few-ulp relative error so that
+// compositions of many operators stay within 1e-5 of an fp64 evaluation.
+//
+//   sin/cos : three-constant Cody-Waite reduction by pi/2 (fused multiply-adds), odd/even
+//             polynomials on [-pi/4, pi/4]
+//   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), scaled by 2^n
+//   tanh    : x + x^3*T(x^2) below 0.6, 1 - 2/(exp(2|x|)+1) above
+//   sigmoid : 1/(1+exp(-x))
+// Polynomial coefficients are weighted least-squares fits on Chebyshev nodes, iteratively
+// re-weighted towards the minimax error (relative errors 4e-9, 1e-10, 3e-9, 3e-9).
+//
+// The header also compiles for the host so that the accuracy of the polynomials can be swept
+// against fp64 without a GPU (the reciprocal is then an exact division).
+#pragma once
+#include <cmath>
+#include <cstdint>
+#include <cstring>
+
+#if defined(__CUDACC__)
+#define VM_HD __host__ __device__ __forceinline__
+#else
+#define VM_HD inline
+#endif
+
+namespace dragon {
+namespace vmmath {
+
+VM_HD float f_rcp(float x) {
+#if defined(__CUDA_ARCH__)
+  float r;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+#else
+  return 1.0f / x;
+#endif
+}
+
+VM_HD float f_from_bits(uint32_t u) {
+#if defined(__CUDA_ARCH__)
+  return __uint_as_float(u);
+#else
+  float f; std::memcpy(&f, &u, 4); return f;
+#endif
+}
+VM_HD uint32_t f_bits(float f) {
+#if defined(__CUDA_ARCH__)
+  return __float_as_uint(f);
+#else
+  uint32_t u; std::memcpy(&u, &f, 4); return u;
+#endif
+}
+
+VM_HD float sin_poly(float r) {
+  const float z = r * r;
+  float p = fmaf(z, -1.9515285269243e-4f, 8.33216077944338e-3f);
+  p = fmaf(z, p, -1.6666654609873324e-1f);
+  return fmaf(r * z, p, r);
+}
+VM_HD float cos_poly(float r) {
+  const float z = r * r;
+  float p = fmaf(z, 2.4433150705502356e-5f, -1.3887316189460366e-3f);
+  p = fmaf(z, p, 4.1666645681363114e-2f);
+  return fmaf(z * z, p, fmaf(z, -0.5f, 1.0f));
+}
+
+// r = x - k*pi/2 with |r| <= pi/4 (approximately), q = k mod 4.  Each step is one fused
+// multiply-add, so the first difference is exact while k*fl(pi/2) stays within 24 bits of x
+// (|x| < 2^24*pi/2); the later steps add an absolute error of a few 1e-7 at the largest
+// arguments, far below the spacing of fp32 numbers of that size.  Beyond that range (and for
+// inf/NaN) x - x is returned: 0, or NaN.
+VM_HD float reduce_pio2(float x, int* q) {
+  float k = rintf(x * 0.636619772367581343f);
+  float r = fmaf(-k, 1.57079637050628662109375f, x);        // fl(pi/2)
+  r = fmaf(-k, -4.371138828673793e-8f, r);                  // fl(pi/2 - c1)
+  r = fmaf(-k, -1.7151245100058819e-15f, r);                // fl(pi/2 - c1 - c2)
+  if (!(fabsf(x) <= 2.5e7f)) { r = x - x; k = 0.f; }
+  *q = (int)k;
+  return r;
+}
+
+VM_HD void sincos_f(float x, float* s, float* c) {
+  int q;
+  const float r = reduce_pio2(x, &q);
+  const float ps = sin_poly(r), pc = cos_poly(r);
+  float ss = (q & 1) ? pc : ps;
+  float cc = (q & 1) ? ps : pc;
+  if (q & 2) ss = -ss;
+  if ((q + 1) & 2) cc = -cc;
+  *s = ss;
+  *c = cc;
+}
+VM_HD float sin_f(float x) {
+  int q;
+  const float r = reduce_pio2(x, &q);
+  const float v = (q & 1) ? cos_poly(r) : sin_poly(r);
+  return (q & 2) ? -v : v;
+}
+VM_HD float cos_f(float x) {
+  int q;
+  const float r = reduce_pio2(x, &q);
+  const float v = (q & 1) ? sin_poly(r) : cos_poly(r);
+  return ((q + 1) & 2) ? -v : v;
+}
+
+// exp for -100 <= x <= 88.7 (callers clamp)
+VM_HD float exp_core(float x) {
+  const float n = rintf(x * 1.44269504088896341f);
+  float r = fmaf(-n, 0.693145751953125f, x);                   // ln2, high part with a short mantissa
+  r = fmaf(-n, 1.428606765330187e-6f, r);                      // ln2 - high part
+  float e = fmaf(r, 1.3814663108745e-3f, 8.36871131029872e-3f);
+  e = fmaf(r, e, 4.16683865189979e-2f);
+  e = fmaf(r, e, 1.6666520673866728e-1f);
+  e = fmaf(r, e, 4.9999993454926206e-1f);
+  const float p = fmaf(r * r, e, r) + 1.0f;
+  // 2^n in two factors so that n = 128 and n below -126 stay in range
+  const int ni = (int)n;
+  const int h = ni / 2;
+  const float s1 = f_from_bits((uint32_t)(h + 127) << 23), s2 = f_from_bits((uint32_t)(ni - h + 127) << 23);
+  return p * s1 * s2;
+}
+VM_HD float exp_clamped10(float x) { return exp_core(fminf(fmaxf(x, -10.0f), 10.0f)); }
+VM_HD float exp_wide(float x) { return exp_core(fminf(fmaxf(x, -100.0f), 88.7f)); }
+
+VM_HD float sigmoid_f(float x) { return f_rcp(1.0f + exp_wide(-x)); }
+
+VM_HD float tanh_f(float x) {
+  const float ax = fabsf(x);
+  const float z = x * x;
+  float p = fmaf(z, -5.89516999486988e-3f, 2.079598263424288e-2f);
+  p = fmaf(z, p, -5.378383380013826e-2f);
+  p = fmaf(z, p, 1.333192417199396e-1f);
+  p = fmaf(z, p, -3.3333298003965545e-1f);
+  const float small = fmaf(x * z, p, x);
+  const float e = exp_wide(2.0f * fminf(ax, 20.0f));
+  const float big = copysignf(fmaf(-2.0f, f_rcp(e + 1.0f), 1.0f), x);
+  return ax < 0.6f ? small : big;
+}
+
+VM_HD float divp_f(float a, float b) { return a * f_rcp(1.0f + fabsf(b)); }
+
+// -sgn(b) / (1 + |b|)^2 with sgn(0) = 0
+VM_HD float divp_grad_b(float b) {
+  const float r = f_rcp(1.0f + fabsf(b));
+  const float sg = b > 0.0f ? 1.0f : (b < 0.0f ? -1.0f : 0.0f);
+  return -sg * r * r;
+}
+
+// float -> bfloat16 (round to nearest even) -> float
+VM_HD uint32_t bf16_bits(float f) {
+  uint32_t u = f_bits(f);
+  if ((u & 0x7fffffffu) > 0x7f800000u) return (u >> 16) | 0x40u;  // quiet NaN
+  return (u + 0x7fffu + ((u >> 16) & 1u)) >> 16;
+}
+VM_HD float round_bf16(float f) { return f_from_bits(bf16_bits(f) << 16); }
+
+}  // namespace vmmath
+}  // namespace dragon
