@@ -1,0 +1,373 @@
+// C ABI of libdragon.so: graph capture, compile (prune + lower), run.
+#include <cuda_runtime.h>
+
+#include <cstring>
+#include <new>
+
+#include "plan.h"
+#include "vm_math.h"
+
+namespace dragon {
+cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, cudaStream_t st);
+cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st);
+cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
+                           int* status, cudaStream_t st);
+cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
+                           const float* dl_ptr, float dl_imm, int* status, cudaStream_t st);
+cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cudaStream_t st);
+int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, int* status, cudaStream_t st);
+}  // namespace dragon
+
+using namespace dragon;
+
+namespace {
+
+bool valid_tensor(const dragon_graph_t* g, dragon_id t) { return t >= 0 && t < (int)g->g.tensors.size(); }
+
+int infer_shape(const Graph& g, int type, const dragon_id* in, int n_in, Shape* out) {
+  auto T = [&](int p) -> const TensorInfo& { return g.tensors[in[p]]; };
+  auto is_float = [&](int p) { return T(p).dtype == DRAGON_F32 || T(p).dtype == DRAGON_BF16; };
+  switch (type) {
+    case DRAGON_OP_ADD: case DRAGON_OP_SUB: case DRAGON_OP_MUL: case DRAGON_OP_DIV:
+      if (n_in != 2) { set_error("binary operator takes 2 inputs"); return DRAGON_ERR_INVALID_ARG; }
+      if (!is_float(0) || !is_float(1)) { set_error("elementwise operators take f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+      if (!broadcast_shapes(T(0).shape, T(1).shape, out)) { set_error("operands '%s' and '%s' do not broadcast", T(0).name.c_str(), T(1).name.c_str()); return DRAGON_ERR_SHAPE; }
+      return DRAGON_OK;
+    case DRAGON_OP_SIN: case DRAGON_OP_EXP: case DRAGON_OP_TANH: case DRAGON_OP_SIGMOID: case DRAGON_OP_RELU:
+    case DRAGON_OP_SUM: case DRAGON_OP_MEAN:
+      if (n_in != 1) { set_error("unary operator takes 1 input"); return DRAGON_ERR_INVALID_ARG; }
+      if (!is_float(0)) { set_error("elementwise operators take f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+      if ((type == DRAGON_OP_SUM || type == DRAGON_OP_MEAN) && T(0).shape.rank == 0) { set_error("Sum/Mean need rank >= 1"); return DRAGON_ERR_SHAPE; }
+      *out = T(0).shape;
+      return DRAGON_OK;
+    case DRAGON_OP_INNER_PRODUCT:
+      if (n_in != 2) { set_error("InnerProduct takes 2 inputs"); return DRAGON_ERR_INVALID_ARG; }
+      if (!is_float(0) || !is_float(1)) { set_error("InnerProduct takes f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+      if (T(0).shape.rank != 2 || T(1).shape.rank != 2 || T(0).shape.d[1] != T(1).shape.d[1]) { set_error("InnerProduct needs X[M,K], W[N,K]"); return DRAGON_ERR_SHAPE; }
+      out->rank = 2; out->d[0] = T(0).shape.d[0]; out->d[1] = T(1).shape.d[0];
+      return DRAGON_OK;
+    case DRAGON_OP_BIAS_ADD:
+      if (n_in != 2) { set_error("BiasAdd takes 2 inputs"); return DRAGON_ERR_INVALID_ARG; }
+      if (!is_float(0) || !is_float(1)) { set_error("BiasAdd takes f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+      if (T(0).shape.rank != 2 || T(1).shape.rank != 1 || T(0).shape.d[1] != T(1).shape.d[0]) { set_error("BiasAdd needs Y[M,N], b[N]"); return DRAGON_ERR_SHAPE; }
+      *out = T(0).shape;
+      return DRAGON_OK;
+    case DRAGON_OP_SOFTMAX_CROSS_ENTROPY:
+      if (n_in != 2) { set_error("SoftmaxCrossEntropy takes 2 inputs"); return DRAGON_ERR_INVALID_ARG; }
+      if (!is_float(0) || T(1).dtype != DRAGON_I32) { set_error("SoftmaxCrossEntropy takes float logits and int32 labels"); return DRAGON_ERR_DTYPE; }
+      if (T(0).shape.rank != 2 || T(1).shape.rank != 1 || T(0).shape.d[0] != T(1).shape.d[0]) { set_error("SoftmaxCrossEntropy needs Z[M,N], labels[M]"); return DRAGON_ERR_SHAPE; }
+      *out = Shape();
+      return DRAGON_OK;
+    default:
+      set_error("unknown operator type %d", type);
+      return DRAGON_ERR_INVALID_ARG;
+  }
+}
+
+int query_sm_count() {
+  int n = 0;
+  if (cudaGetDeviceCount(&n) != cudaSuccess || n <= 0) { cudaGetLastError(); return kDefaultSmCount; }
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) {
+    cudaGetLastError();
+    return kDefaultSmCount;
+  }
+  return sms;
+}
+
+}  // namespace
+
+extern "C" {
+
+dragon_graph_t* dragon_graph_create(void) { return new (std::nothrow) dragon_graph_t(); }
+void dragon_graph_destroy(dragon_graph_t* g) { delete g; }
+
+dragon_id dragon_add_tensor(dragon_graph_t* g, const char* name, int dtype, int rank, const int64_t* shape) {
+  if (!g || !name || rank < 0 || rank > 2 || (rank > 0 && !shape)) { set_error("dragon_add_tensor: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  if (dtype != DRAGON_F32 && dtype != DRAGON_BF16 && dtype != DRAGON_I32) { set_error("dragon_add_tensor: unknown dtype %d", dtype); return DRAGON_ERR_DTYPE; }
+  TensorInfo t;
+  t.name = name;
+  t.dtype = dtype;
+  t.shape.rank = rank;
+  for (int i = 0; i < rank; ++i) {
+    if (shape[i] <= 0) { set_error("dragon_add_tensor: dimension %d of '%s' is not positive", i, name); return DRAGON_ERR_SHAPE; }
+    t.shape.d[i] = shape[i];
+  }
+  if (!g->g.names.insert(t.name).second) { set_error("dragon_add_tensor: name '%s' is already taken", name); return DRAGON_ERR_INVALID_ARG; }
+  g->g.tensors.push_back(t);
+  return (dragon_id)g->g.tensors.size() - 1;
+}
+
+dragon_id dragon_add_op(dragon_graph_t* g, int op_type, const dragon_id* in, int n_in, const dragon_id* out, int n_out,
+                        const double* attrs, int n_attrs) {
+  (void)attrs;
+  if (!g || !in || !out || n_in <= 0 || n_out <= 0 || n_attrs < 0) { set_error("dragon_add_op: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  for (int i = 0; i < n_in; ++i)
+    if (!valid_tensor(g, in[i])) { set_error("dragon_add_op: input id %d is not a tensor", in[i]); return DRAGON_ERR_INVALID_ARG; }
+  for (int i = 0; i < n_out; ++i)
+    if (!valid_tensor(g, out[i])) { set_error("dragon_add_op: output id %d is not a tensor", out[i]); return DRAGON_ERR_INVALID_ARG; }
+  if (n_out != 1) { set_error("dragon_add_op: every operator type of this library has one output"); return DRAGON_ERR_INVALID_ARG; }
+  for (int i = 0; i < n_in; ++i)
+    if (g->g.tensors[in[i]].grad_stage >= 0) { set_error("dragon_add_op: gradient tensors cannot be consumed by operators"); return DRAGON_ERR_UNSUPPORTED; }
+  TensorInfo& to = g->g.tensors[out[0]];
+  if (to.producer >= 0 || to.grad_stage >= 0) { set_error("dragon_add_op: tensor '%s' already has a producer", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+  for (int i = 0; i < n_in; ++i)
+    if (in[i] == out[0]) { set_error("dragon_add_op: operator reads its own output '%s'", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+  // a tensor that was read before it got a producer would let the new operator close a cycle
+  if (to.consumed) { set_error("dragon_add_op: tensor '%s' is already read by an earlier operator", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+  Shape s;
+  int rc = infer_shape(g->g, op_type, in, n_in, &s);
+  if (rc != DRAGON_OK) return rc;
+  if (s != to.shape) { set_error("dragon_add_op: declared shape of '%s' differs from the inferred one", to.name.c_str()); return DRAGON_ERR_SHAPE; }
+  if (to.dtype == DRAGON_I32) { set_error("dragon_add_op: operators produce f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+  OpInfo op;
+  op.type = op_type;
+  op.in.assign(in, in + n_in);
+  op.out.assign(out, out + n_out);
+  g->g.ops.push_back(op);
+  for (int i = 0; i < n_in; ++i) g->g.tensors[in[i]].consumed = true;
+  g->g.tensors[out[0]].producer = (int)g->g.ops.size() - 1;
+  return (dragon_id)g->g.ops.size() - 1;
+}
+
+int dragon_add_grad(dragon_graph_t* g, const dragon_id* objs, int n_obj, const dragon_id* wrts, int n_wrt,
+                    dragon_id* out_grad_tensor_ids) {
+  if (!g || !objs || !wrts || !out_grad_tensor_ids || n_obj <= 0 || n_wrt <= 0) { set_error("dragon_add_grad: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  GradStage st;
+  for (int i = 0; i < n_obj; ++i) {
+    if (!valid_tensor(g, objs[i]) || g->g.tensors[objs[i]].grad_stage >= 0) { set_error("dragon_add_grad: bad objective id %d", objs[i]); return DRAGON_ERR_INVALID_ARG; }
+    if (g->g.tensors[objs[i]].dtype == DRAGON_I32) { set_error("dragon_add_grad: objective must be a float tensor"); return DRAGON_ERR_DTYPE; }
+    st.objs.push_back(objs[i]);
+  }
+  for (int i = 0; i < n_wrt; ++i) {
+    if (!valid_tensor(g, wrts[i]) || g->g.tensors[wrts[i]].grad_stage >= 0) { set_error("dragon_add_grad: bad derivative target id %d", wrts[i]); return DRAGON_ERR_INVALID_ARG; }
+    if (g->g.tensors[wrts[i]].dtype == DRAGON_I32) { set_error("dragon_add_grad: derivative target must be a float tensor"); return DRAGON_ERR_DTYPE; }
+    st.wrts.push_back(wrts[i]);
+  }
+  std::vector<uint8_t> G = backward_chain_marks(g->g, st.objs, st.wrts);
+  for (int w : st.wrts)
+    if (!G[w]) { set_error("dragon_add_grad: no chain from '%s' to any objective", g->g.tensors[w].name.c_str()); return DRAGON_ERR_NO_PATH; }
+  const int s = (int)g->g.stages.size();
+  for (int i = 0; i < n_wrt; ++i) {
+    TensorInfo t;
+    t.name = "grad" + std::to_string(s) + "/" + g->g.tensors[wrts[i]].name;
+    while (!g->g.names.insert(t.name).second) t.name += "'";
+    t.dtype = DRAGON_F32;
+    t.shape = g->g.tensors[wrts[i]].shape;
+    t.grad_stage = s;
+    t.grad_wrt = wrts[i];
+    g->g.tensors.push_back(t);
+    st.grad_ids.push_back((int)g->g.tensors.size() - 1);
+    out_grad_tensor_ids[i] = st.grad_ids.back();
+  }
+  g->g.stages.push_back(st);
+  return DRAGON_OK;
+}
+
+int dragon_graph_num_tensors(const dragon_graph_t* g) { return g ? (int)g->g.tensors.size() : DRAGON_ERR_INVALID_ARG; }
+int dragon_graph_num_ops(const dragon_graph_t* g) { return g ? (int)g->g.ops.size() : DRAGON_ERR_INVALID_ARG; }
+
+dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, int n_in, const dragon_id* outputs, int n_out) {
+  if (!g || (n_in > 0 && !inputs) || !outputs || n_in < 0 || n_out <= 0) { set_error("dragon_function: bad argument"); return nullptr; }
+  std::vector<int> in(inputs, inputs + n_in), out(outputs, outputs + n_out);
+  std::vector<uint8_t> seen(g->g.tensors.size(), 0);
+  for (int t : in) {
+    if (!valid_tensor(g, t)) { set_error("dragon_function: input id %d is not a tensor", t); return nullptr; }
+    if (g->g.tensors[t].producer >= 0 || g->g.tensors[t].grad_stage >= 0) { set_error("dragon_function: input '%s' is not a source tensor", g->g.tensors[t].name.c_str()); return nullptr; }
+    if (seen[t]) { set_error("dragon_function: input '%s' is listed twice", g->g.tensors[t].name.c_str()); return nullptr; }
+    seen[t] = 1;
+  }
+  for (int t : out)
+    if (!valid_tensor(g, t)) { set_error("dragon_function: output id %d is not a tensor", t); return nullptr; }
+  dragon_function_t* f = new (std::nothrow) dragon_function_t();
+  if (!f) return nullptr;
+  f->n_tensors = (int)g->g.tensors.size();
+  f->n_in = n_in;
+  f->n_out = n_out;
+  if (prune_function(g->g, in, out, &f->prune) != DRAGON_OK) { delete f; return nullptr; }
+  if (lower_function(g->g, f->prune, in, out, query_sm_count(), &f->plan) != DRAGON_OK) { delete f; return nullptr; }
+  return f;
+}
+
+void dragon_function_destroy(dragon_function_t* f) {
+  if (!f) return;
+  for (auto& sg : f->plan.segs)
+    if (sg.d_code) cudaFree(sg.d_code);
+  delete f;
+}
+
+int dragon_function_marked(const dragon_function_t* f, uint8_t* flags, int n_tensors) {
+  if (!f || !flags || n_tensors != f->n_tensors) { set_error("dragon_function_marked: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  std::memcpy(flags, f->prune.marked.data(), (size_t)n_tensors);
+  return DRAGON_OK;
+}
+
+int dragon_function_kept_ops(const dragon_function_t* f, dragon_id* fwd_ops, int cap_f, int* n_f, dragon_id* grad_ops,
+                             uint32_t* grad_input_mask, int cap_g, int* n_g) {
+  if (!f || !n_f || !n_g || cap_f < 0 || cap_g < 0) { set_error("dragon_function_kept_ops: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  *n_f = (int)f->prune.fwd_ops.size();
+  *n_g = (int)f->prune.grad_ops.size();
+  for (int i = 0; i < *n_f && i < cap_f && fwd_ops; ++i) fwd_ops[i] = f->prune.fwd_ops[i];
+  for (int i = 0; i < *n_g && i < cap_g; ++i) {
+    if (grad_ops) grad_ops[i] = f->prune.grad_ops[i].op;
+    if (grad_input_mask) grad_input_mask[i] = f->prune.grad_ops[i].mask;
+  }
+  return DRAGON_OK;
+}
+
+int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flags, int n_in) {
+  if (!f || (n_in > 0 && !flags) || n_in != f->n_in) { set_error("dragon_function_used_inputs: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  if (n_in) std::memcpy(flags, f->prune.used_inputs.data(), (size_t)n_in);
+  return DRAGON_OK;
+}
+
+int dragon_function_num_launches(const dragon_function_t* f) {
+  if (!f) return DRAGON_ERR_INVALID_ARG;
+  int n = 0;
+  for (const Step& st : f->plan.steps) {
+    if (st.kind == ST_VM) n += 1 + (f->plan.segs[st.seg].finish.empty() ? 0 : 1);
+    else if (st.kind == ST_SCE_FWD) n += 2;
+    else if (st.kind != ST_COPY) n += 1;
+  }
+  return n;
+}
+
+int dragon_function_describe(const dragon_function_t* f, char* buf, int cap) {
+  if (!f || !buf || cap <= 0) return DRAGON_ERR_INVALID_ARG;
+  std::string s = describe_plan(f->plan);
+  std::strncpy(buf, s.c_str(), (size_t)cap - 1);
+  buf[cap - 1] = 0;
+  return DRAGON_OK;
+}
+
+size_t dragon_function_workspace_bytes(const dragon_function_t* f) { return f ? f->plan.workspace_bytes : 0; }
+
+int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t bytes) {
+  if (!f) { set_error("dragon_function_set_workspace: NULL function"); return DRAGON_ERR_INVALID_ARG; }
+  if (!dev_ptr || ((uintptr_t)dev_ptr & 255) || bytes < f->plan.workspace_bytes) {
+    set_error("workspace must be 256-byte aligned device memory of at least %zu bytes", f->plan.workspace_bytes);
+    return DRAGON_ERR_WORKSPACE;
+  }
+  f->workspace = dev_ptr;
+  f->workspace_bytes = bytes;
+  return DRAGON_OK;
+}
+
+int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetches, void* cuda_stream) {
+  if (!f || !fetches || (f->n_in > 0 && !feeds)) { set_error("dragon_run: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  Plan& P = f->plan;
+  if (!f->workspace) { set_error("dragon_run: no workspace set (need %zu bytes)", P.workspace_bytes); return DRAGON_ERR_WORKSPACE; }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  char* ws = reinterpret_cast<char*>(f->workspace);
+  std::vector<void*> ptr(P.mems.size(), nullptr);
+  for (size_t m = 0; m < P.mems.size(); ++m) {
+    const MemRef& mr = P.mems[m];
+    if (mr.where == MEM_WORK) { ptr[m] = ws + mr.offset; continue; }
+    if (!mr.live) continue;
+    void* q = mr.where == MEM_FEED ? const_cast<void*>(feeds[mr.index]) : fetches[mr.index];
+    if (!q || ((uintptr_t)q & 15)) {
+      set_error("dragon_run: %s %d is NULL or not 16-byte aligned", mr.where == MEM_FEED ? "feed" : "fetch", mr.index);
+      return DRAGON_ERR_INVALID_ARG;
+    }
+    ptr[m] = q;
+  }
+  if (!f->uploaded) {  // first run: device copies of the instruction streams
+    for (auto& sg : P.segs) {
+      if (cudaMalloc(&sg.d_code, sg.code.size() * 4) != cudaSuccess ||
+          cudaMemcpy(sg.d_code, sg.code.data(), sg.code.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
+        set_error("dragon_run: cannot upload the instruction stream: %s", cudaGetErrorString(cudaGetLastError()));
+        return DRAGON_ERR_CUDA;
+      }
+    }
+    f->uploaded = true;
+  }
+  int* status = reinterpret_cast<int*>(ws + P.status_off);
+  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
+  for (const Step& s : P.steps) {
+    if (e != cudaSuccess) break;
+    switch (s.kind) {
+      case ST_VM: {
+        VmSegment& sg = P.segs[s.seg];
+        vm::Params p;
+        std::memset(&p, 0, sizeof(p));
+        p.code = sg.d_code;
+        p.n_code = (int)sg.code.size();
+        p.row_mode = sg.row_mode;
+        p.n = sg.n;
+        p.cols = sg.cols;
+        p.n_spill = sg.n_spill;
+        p.spill = reinterpret_cast<float*>(ws + sg.spill_off);
+        p.colpart = reinterpret_cast<float*>(ws + sg.colpart_off);
+        p.scalpart = reinterpret_cast<double*>(ws + sg.scalpart_off);
+        p.status = status;
+        for (size_t i = 0; i < sg.operand_mem.size(); ++i) {
+          p.operand[i].ptr = ptr[sg.operand_mem[i]];
+          p.operand[i].kind = sg.operand_kind[i];
+          p.operand[i].dtype = (uint32_t)P.mems[sg.operand_mem[i]].dtype;
+        }
+        e = launch_vm(p, sg.grid, sg.n_smem, st);
+        if (e == cudaSuccess) e = launch_finish(sg, P.mems, ptr.data(), ws, st);
+        break;
+      }
+      case ST_GEMM: {
+        const MemRef &A = P.mems[s.mA], &C = P.mems[s.mC];
+        int rc = launch_gemm_bf16(ptr[s.mA], ptr[s.mB], ptr[s.mC], C.dtype, (int)C.shape.d[0], (int)C.shape.d[1], (int)A.shape.d[1], status, st);
+        if (rc != DRAGON_OK) return rc;
+        break;
+      }
+      case ST_TRANSPOSE:
+        e = launch_transpose16(ptr[s.mA], ptr[s.mC], (int)P.mems[s.mA].shape.d[0], (int)P.mems[s.mA].shape.d[1], st);
+        break;
+      case ST_SCE_FWD:
+        e = launch_sce_fwd(ptr[s.mA], P.mems[s.mA].dtype, reinterpret_cast<const int*>(ptr[s.mB]), (int)P.mems[s.mA].shape.d[0],
+                           (int)P.mems[s.mA].shape.d[1], reinterpret_cast<float*>(ws + s.scratch_off), reinterpret_cast<float*>(ptr[s.mC]), status, st);
+        break;
+      case ST_SCE_BWD:
+        e = launch_sce_bwd(ptr[s.mA], P.mems[s.mA].dtype, reinterpret_cast<const int*>(ptr[s.mB]), (int)P.mems[s.mA].shape.d[0],
+                           (int)P.mems[s.mA].shape.d[1], ptr[s.mC], P.mems[s.mC].dtype,
+                           s.mD >= 0 ? reinterpret_cast<const float*>(ptr[s.mD]) : nullptr, s.scale, status, st);
+        break;
+      case ST_COPY:
+        e = cudaMemcpyAsync(ptr[s.mC], ptr[s.mA], P.mems[s.mA].bytes(), cudaMemcpyDeviceToDevice, st);
+        break;
+    }
+  }
+  if (e != cudaSuccess) {
+    set_error("dragon_run: CUDA error: %s", cudaGetErrorString(e));
+    return DRAGON_ERR_CUDA;
+  }
+  f->last_stream = cuda_stream;
+  return DRAGON_OK;
+}
+
+int dragon_function_status(dragon_function_t* f) {
+  if (!f || !f->workspace) { set_error("dragon_function_status: no run yet"); return DRAGON_ERR_INVALID_ARG; }
+  int v = 0;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(f->last_stream);
+  if (cudaStreamSynchronize(st) != cudaSuccess ||
+      cudaMemcpy(&v, reinterpret_cast<char*>(f->workspace) + f->plan.status_off, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    set_error("dragon_function_status: CUDA error: %s", cudaGetErrorString(cudaGetLastError()));
+    return DRAGON_ERR_CUDA;
+  }
+  return v;
+}
+
+int dragon_host_math(int fn, const float* x, float* y, int n) {
+  if (!x || !y || n < 0) { set_error("dragon_host_math: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  for (int i = 0; i < n; ++i) {
+    switch (fn) {
+      case DRAGON_OP_SIN: y[i] = vmmath::sin_f(x[i]); break;
+      case 100 + DRAGON_OP_SIN: y[i] = vmmath::cos_f(x[i]); break;
+      case DRAGON_OP_EXP: y[i] = vmmath::exp_clamped10(x[i]); break;
+      case DRAGON_OP_TANH: y[i] = vmmath::tanh_f(x[i]); break;
+      case DRAGON_OP_SIGMOID: y[i] = vmmath::sigmoid_f(x[i]); break;
+      case DRAGON_OP_DIV: y[i] = vmmath::divp_f(1.f, x[i]); break;
+      default: set_error("dragon_host_math: unknown function %d", fn); return DRAGON_ERR_INVALID_ARG;
+    }
+  }
+  return DRAGON_OK;
+}
+
+const char* dragon_last_error(void) { return dragon::last_error(); }
+
+}  // extern "C"
