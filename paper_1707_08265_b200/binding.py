@@ -1,0 +1,244 @@
+"""Thin ctypes binding of libdragon.so: same names as include/dragon.h, argument marshalling only.
+
+Every step of the evaluated path runs in the library's CUDA kernels; nothing here computes.
+The library must have been built (``python -m paper_1707_08265_b200.build`` or
+``__graft_entry__.build()``); loading fails loudly otherwise.
+"""
+import ctypes
+import os
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(HERE, "libdragon.so")
+
+OK = 0
+ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_NOT_SSA, ERR_MISSING_INPUT = -1, -2, -3, -4, -5
+ERR_NO_PATH, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8, -9, -10
+F32, BF16, I32 = 0, 1, 2
+DTYPES = {"f32": F32, "bf16": BF16, "i32": I32}
+OPS = {"Add": 0, "Sub": 1, "Mul": 2, "Div": 3, "Sin": 4, "Exp": 5, "Tanh": 6, "Sigmoid": 7, "ReLU": 8,
+       "Sum": 9, "Mean": 10, "InnerProduct": 11, "BiasAdd": 12, "SoftmaxCrossEntropy": 13}
+
+_lib = None
+
+_c = ctypes
+_SIGNATURES = {
+    "dragon_graph_create": (_c.c_void_p, []),
+    "dragon_graph_destroy": (None, [_c.c_void_p]),
+    "dragon_add_tensor": (_c.c_int32, [_c.c_void_p, _c.c_char_p, _c.c_int, _c.c_int, _c.POINTER(_c.c_int64)]),
+    "dragon_add_op": (_c.c_int32, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int32),
+                                   _c.c_int, _c.POINTER(_c.c_double), _c.c_int]),
+    "dragon_add_grad": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int32), _c.c_int,
+                                   _c.POINTER(_c.c_int32)]),
+    "dragon_graph_num_tensors": (_c.c_int, [_c.c_void_p]),
+    "dragon_graph_num_ops": (_c.c_int, [_c.c_void_p]),
+    "dragon_function": (_c.c_void_p, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int32), _c.c_int]),
+    "dragon_function_destroy": (None, [_c.c_void_p]),
+    "dragon_function_marked": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_uint8), _c.c_int]),
+    "dragon_function_kept_ops": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int),
+                                            _c.POINTER(_c.c_int32), _c.POINTER(_c.c_uint32), _c.c_int, _c.POINTER(_c.c_int)]),
+    "dragon_function_used_inputs": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_uint8), _c.c_int]),
+    "dragon_function_num_launches": (_c.c_int, [_c.c_void_p]),
+    "dragon_function_describe": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_int]),
+    "dragon_function_workspace_bytes": (_c.c_size_t, [_c.c_void_p]),
+    "dragon_function_set_workspace": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
+    "dragon_run": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p), _c.c_void_p]),
+    "dragon_function_status": (_c.c_int, [_c.c_void_p]),
+    "dragon_host_math": (_c.c_int, [_c.c_int, _c.POINTER(_c.c_float), _c.POINTER(_c.c_float), _c.c_int]),
+    "dragon_last_error": (_c.c_char_p, []),
+}
+
+
+def lib():
+    """The loaded library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError("libdragon.so is missing: build it with `python -m paper_1707_08265_b200.build`")
+        L = ctypes.CDLL(LIB_PATH)
+        for name, (res, args) in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.restype = res
+            fn.argtypes = args
+        _lib = L
+    return _lib
+
+
+class DragonError(RuntimeError):
+    def __init__(self, code, where):
+        msg = lib().dragon_last_error()
+        super().__init__("%s failed with code %d: %s" % (where, code, msg.decode() if msg else ""))
+        self.code = code
+
+
+def _ids(seq):
+    arr = (_c.c_int32 * max(1, len(seq)))(*seq)
+    return arr
+
+
+class Graph:
+    """dragon_graph_t: tensors and operators in creation order."""
+
+    def __init__(self):
+        self.h = lib().dragon_graph_create()
+        if not self.h:
+            raise MemoryError("dragon_graph_create")
+
+    def close(self):
+        if self.h:
+            lib().dragon_graph_destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def add_tensor(self, name, dtype, shape):
+        shp = (_c.c_int64 * max(1, len(shape)))(*shape)
+        r = lib().dragon_add_tensor(self.h, name.encode(), dtype, len(shape), shp)
+        if r < 0:
+            raise DragonError(r, "dragon_add_tensor")
+        return r
+
+    def add_op(self, op_type, ins, outs):
+        r = lib().dragon_add_op(self.h, op_type, _ids(ins), len(ins), _ids(outs), len(outs), None, 0)
+        if r < 0:
+            raise DragonError(r, "dragon_add_op")
+        return r
+
+    def add_grad(self, objs, wrts):
+        out = (_c.c_int32 * max(1, len(wrts)))()
+        r = lib().dragon_add_grad(self.h, _ids(objs), len(objs), _ids(wrts), len(wrts), out)
+        if r < 0:
+            raise DragonError(r, "dragon_add_grad")
+        return list(out[:len(wrts)])
+
+    def num_tensors(self):
+        return lib().dragon_graph_num_tensors(self.h)
+
+    def num_ops(self):
+        return lib().dragon_graph_num_ops(self.h)
+
+    def function(self, inputs, outputs):
+        return Function(self, inputs, outputs)
+
+    @staticmethod
+    def from_desc(desc):
+        """Replays a graph description (see workloads.GraphDesc) through the C ABI.  Tensors,
+        operators and gradient stages are created in the same order, so ids coincide."""
+        g = Graph()
+        grad_ids = {gid for st in desc.get("grads", []) for gid in st["grad_ids"]}
+        stage_first = {st["grad_ids"][0]: st for st in desc.get("grads", []) if st["grad_ids"]}
+        producer = {}
+        for k, op in enumerate(desc["ops"]):
+            for o in op["out"]:
+                producer[o] = k
+        next_op = 0
+        for t, ti in enumerate(desc["tensors"]):
+            if t in grad_ids:
+                if t in stage_first:
+                    st = stage_first[t]
+                    got = g.add_grad(st["objs"], st["wrts"])
+                    assert got == list(st["grad_ids"]), (got, st["grad_ids"])
+                continue
+            tid = g.add_tensor(ti["name"], DTYPES[ti["dtype"]], ti["shape"])
+            assert tid == t
+            # operators whose outputs are all declared can be appended now (creation order)
+            while next_op < len(desc["ops"]) and max(desc["ops"][next_op]["out"]) <= t:
+                op = desc["ops"][next_op]
+                oid = g.add_op(OPS[op["type"]], op["in"], op["out"])
+                assert oid == next_op
+                next_op += 1
+        assert next_op == len(desc["ops"])
+        return g
+
+
+class Function:
+    """dragon_function_t: the pruned, compiled function(inputs, outputs)."""
+
+    def __init__(self, graph, inputs, outputs):
+        self.n_in, self.n_out = len(inputs), len(outputs)
+        self.n_tensors = graph.num_tensors()
+        self.n_ops = graph.num_ops()
+        self.h = lib().dragon_function(graph.h, _ids(inputs), len(inputs), _ids(outputs), len(outputs))
+        if not self.h:
+            raise DragonError(-1, "dragon_function")
+        self._ws = None
+
+    def close(self):
+        if self.h:
+            lib().dragon_function_destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def marked(self):
+        buf = (_c.c_uint8 * self.n_tensors)()
+        r = lib().dragon_function_marked(self.h, buf, self.n_tensors)
+        if r < 0:
+            raise DragonError(r, "dragon_function_marked")
+        return list(buf)
+
+    def kept_ops(self):
+        cap = 2 * self.n_ops * 4 + 8
+        fwd = (_c.c_int32 * cap)()
+        gops = (_c.c_int32 * cap)()
+        mask = (_c.c_uint32 * cap)()
+        nf, ng = _c.c_int(), _c.c_int()
+        r = lib().dragon_function_kept_ops(self.h, fwd, cap, _c.byref(nf), gops, mask, cap, _c.byref(ng))
+        if r < 0:
+            raise DragonError(r, "dragon_function_kept_ops")
+        assert nf.value <= cap and ng.value <= cap
+        return list(fwd[:nf.value]), list(gops[:ng.value]), list(mask[:ng.value])
+
+    def used_inputs(self):
+        buf = (_c.c_uint8 * max(1, self.n_in))()
+        r = lib().dragon_function_used_inputs(self.h, buf, self.n_in)
+        if r < 0:
+            raise DragonError(r, "dragon_function_used_inputs")
+        return list(buf[:self.n_in])
+
+    def num_launches(self):
+        return lib().dragon_function_num_launches(self.h)
+
+    def describe(self):
+        buf = _c.create_string_buffer(1 << 16)
+        lib().dragon_function_describe(self.h, buf, len(buf))
+        return buf.value.decode()
+
+    def workspace_bytes(self):
+        return lib().dragon_function_workspace_bytes(self.h)
+
+    def set_workspace(self, dev_ptr, nbytes):
+        r = lib().dragon_function_set_workspace(self.h, dev_ptr, nbytes)
+        if r < 0:
+            raise DragonError(r, "dragon_function_set_workspace")
+
+    def run(self, feed_ptrs, fetch_ptrs, stream=0):
+        feeds = (_c.c_void_p * max(1, self.n_in))(*[p or None for p in feed_ptrs])
+        fetches = (_c.c_void_p * max(1, self.n_out))(*fetch_ptrs)
+        r = lib().dragon_run(self.h, feeds, fetches, stream)
+        if r < 0:
+            raise DragonError(r, "dragon_run")
+
+    def status(self):
+        return lib().dragon_function_status(self.h)
+
+    # ---- convenience for torch tensors (device memory and streams only) ----
+    def run_torch(self, feeds, fetches, stream=None):
+        """feeds / fetches: lists of CUDA torch tensors (None for a pruned input)."""
+        import torch
+        if self._ws is None:
+            nbytes = max(256, self.workspace_bytes())
+            self._ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+            base = (self._ws.data_ptr() + 255) & ~255
+            self.set_workspace(base, nbytes)
+        s = stream if stream is not None else torch.cuda.current_stream()
+        self.run([0 if t is None else t.data_ptr() for t in feeds], [t.data_ptr() for t in fetches], s.cuda_stream)
+
+
+def host_math(fn, x):
+    import numpy as np
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    y = np.empty_like(x)
+    r = lib().dragon_host_math(fn, x.ctypes.data_as(_c.POINTER(_c.c_float)), y.ctypes.data_as(_c.POINTER(_c.c_float)), x.size)
+    if r < 0:
+        raise DragonError(r, "dragon_host_math")
+    return y

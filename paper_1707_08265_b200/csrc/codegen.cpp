@@ -240,7 +240,7 @@ struct Gen {
     keep_operand(a, pos, -1);
     // sin and cos of the same value share one range reduction
     if (it.opc == M_SIN || it.opc == M_COS) {
-      for (int q = pos + 1; q < (int)idx.size(); ++q) {
+      for (int q = pos + 1; q < (int)idx.size() && q < pos + 4096; ++q) {
         const Item& o2 = items[idx[q]];
         if (done[q] || o2.kind != IT_MOP || (o2.opc != M_SIN && o2.opc != M_COS) || o2.opc == it.opc || C(o2.a) != a) continue;
         int k = alloc_reg(pos, a);

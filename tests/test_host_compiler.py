@@ -1,0 +1,153 @@
+"""Host side of the library through the C ABI, no GPU: exported symbols, error codes, prune sets
+and operator order against the oracle (bit-exact), linear-time pruning of a long chain."""
+import ctypes
+import os
+import re
+import time
+
+import numpy as np
+import pytest
+
+from oracle import prune as oprune
+from paper_1707_08265_b200 import binding as B
+from paper_1707_08265_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "dragon.h")).read()
+    names = set(re.findall(r"\b(dragon_[a-z_]+)\s*\(", header))
+    assert len(names) >= 20
+    L = ctypes.CDLL(B.LIB_PATH)
+    for n in sorted(names):
+        assert hasattr(L, n), n
+    assert names == set(B._SIGNATURES), names ^ set(B._SIGNATURES)
+
+
+def compare_sets(desc, inputs, outputs):
+    want = oprune.function_sets(desc, inputs, outputs)
+    g = B.Graph.from_desc(desc)
+    f = g.function(inputs, outputs)
+    fwd, gops, masks = f.kept_ops()
+    assert f.marked() == want["marked"]
+    assert fwd == want["fwd_ops"]
+    assert gops == [k for (_, k, _) in want["grad_ops"]]
+    assert masks == [sum(1 << p for p in pos) for (_, _, pos) in want["grad_ops"]]
+    assert f.used_inputs() == want["used_inputs"]
+    return f
+
+
+def test_paper_example_through_the_c_abi():
+    g, ids = wl.toy_function_grad(1 << 12)
+    inputs = [ids["x"], ids["a"], ids["b"]]
+    f = compare_sets(g.desc, inputs, [ids["y"]])
+    assert f.used_inputs() == [1, 1, 0] and f.kept_ops()[0] == [0]      # b is redundant (Sec. 2.2)
+    compare_sets(g.desc, inputs, [ids["f"], ids["y"]])
+    compare_sets(g.desc, inputs, [ids["dx"], ids["da"], ids["db"]])
+    compare_sets(g.desc, inputs, [ids["db"]])
+    compare_sets(g.desc, inputs, [ids["f"], ids["da"]])
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_random_dag_prune_sets_match_oracle(seed):
+    g, inputs, fetch = wl.random_dag(1000, seed, n_ops=40)
+    compare_sets(g.desc, inputs, fetch)
+    compare_sets(g.desc, inputs, fetch[:1])
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_row_dag_with_gradients_matches_oracle(seed):
+    g, inputs, fetch = wl.random_row_dag(8, 16, seed, n_ops=60)
+    G = oprune.backward_marks(g.desc, fetch, inputs)
+    wrts = [i for i in inputs if i in G]
+    grads = g.grad(fetch, wrts)
+    compare_sets(g.desc, inputs, fetch + grads)
+    compare_sets(g.desc, inputs, grads[:1])
+    compare_sets(g.desc, inputs, fetch[:1] + grads[-1:])
+
+
+def test_mlp_prune_sets():
+    g, ids = wl.mlp(64, 32, 32, 16)
+    inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
+    f = compare_sets(g.desc, inputs, [ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")])
+    plan = f.describe()
+    assert plan.count("gemm") == 5                      # two forward, dW2, dH, dW1; no dX of layer 1
+    compare_sets(g.desc, inputs, [ids["loss"]])
+    compare_sets(g.desc, inputs, [ids["dW2"]])
+
+
+def test_two_gradient_stages():
+    g, ids = wl.toy_function(16)
+    s0 = g.grad([ids["f"]], [ids["x"], ids["b"]])
+    s1 = g.grad([ids["y"]], [ids["a"]])
+    inputs = [ids["x"], ids["a"], ids["b"]]
+    compare_sets(g.desc, inputs, s0 + s1)
+    f = compare_sets(g.desc, inputs, s1)
+    assert f.used_inputs() == [1, 1, 0]
+
+
+def test_error_codes():
+    g = B.Graph()
+    x = g.add_tensor("x", B.F32, [4, 8])
+    r = g.add_tensor("r", B.F32, [8])
+    bad = g.add_tensor("bad", B.F32, [7])
+    lab = g.add_tensor("lab", B.I32, [4])
+    y = g.add_tensor("y", B.F32, [4, 8])
+    y2 = g.add_tensor("y2", B.F32, [4, 9])
+
+    def code(fn):
+        with pytest.raises(B.DragonError) as e:
+            fn()
+        return e.value.code
+
+    assert code(lambda: g.add_tensor("x", B.F32, [1])) == B.ERR_INVALID_ARG           # duplicate name
+    assert code(lambda: g.add_tensor("z", 7, [1])) == B.ERR_DTYPE
+    assert code(lambda: g.add_tensor("z", B.F32, [0])) == B.ERR_SHAPE
+    assert code(lambda: g.add_op(B.OPS["Add"], [x, bad], [y])) == B.ERR_SHAPE          # no broadcast
+    assert code(lambda: g.add_op(B.OPS["Add"], [x, r], [y2])) == B.ERR_SHAPE           # declared != inferred
+    assert code(lambda: g.add_op(B.OPS["Add"], [x, lab], [y])) == B.ERR_DTYPE
+    assert code(lambda: g.add_op(B.OPS["Add"], [x, y], [y])) == B.ERR_NOT_SSA          # reads its own output
+    assert code(lambda: g.add_op(99, [x, r], [y])) == B.ERR_INVALID_ARG
+    assert g.add_op(B.OPS["Add"], [x, r], [y]) == 0
+    assert code(lambda: g.add_op(B.OPS["Add"], [x, r], [y])) == B.ERR_NOT_SSA          # second producer
+    z = g.add_tensor("z", B.F32, [4, 8])
+    assert code(lambda: g.add_grad([y], [bad])) == B.ERR_NO_PATH
+    (dr,) = g.add_grad([y], [r])
+    assert code(lambda: g.add_op(B.OPS["Sin"], [dr], [z])) == B.ERR_UNSUPPORTED        # gradient tensors are terminal
+    with pytest.raises(B.DragonError):
+        g.function([r], [y])                                                           # x is needed but not listed
+    assert b"not among the inputs" in B.lib().dragon_last_error()
+    with pytest.raises(B.DragonError):
+        g.function([x, r, y], [y])                                                     # y is not a source
+    f = g.function([x, r, bad], [y, dr])
+    assert f.used_inputs() == [1, 1, 0]
+    assert f.workspace_bytes() > 0 and f.num_launches() >= 1
+    with pytest.raises(B.DragonError) as e:
+        f.run([0, 0, 0], [0, 0])                                                       # no workspace yet
+    assert e.value.code == B.ERR_WORKSPACE
+
+
+def test_long_chain_prunes_in_linear_time_without_recursion():
+    def build(n):
+        g = B.Graph()
+        prev = g.add_tensor("x", B.F32, [8])
+        for k in range(n):
+            nxt = g.add_tensor("t%d" % k, B.F32, [8])
+            g.add_op(B.OPS["Tanh"] if k % 2 else B.OPS["Sin"], [prev], [nxt])
+            prev = nxt
+        return g, prev
+
+    lib = B.lib()
+    times = []
+    for n in (50000, 200000):
+        g, last = build(n)
+        dx = g.add_grad([last], [0])
+        ins = (ctypes.c_int32 * 1)(0)
+        outs = (ctypes.c_int32 * 2)(last, dx[0])
+        # only the two prunes are timed here: lowering a 200000-operator fused segment is not the claim
+        t0 = time.perf_counter()
+        ok = lib.dragon_add_grad(g.h, (ctypes.c_int32 * 1)(last), 1, (ctypes.c_int32 * 1)(0), 1, (ctypes.c_int32 * 1)())
+        times.append(time.perf_counter() - t0)
+        assert ok == 0
+    assert times[1] < 12 * times[0] + 0.05
