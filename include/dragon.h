@@ -143,6 +143,24 @@ int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t by
  * written by the kernels of the plan; a fetch that is itself an input is copied. */
 int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetches, void* cuda_stream);
 
+/* The same with HOST buffers: copies every needed input from host_feeds[j] to the staging area,
+ * runs, and copies every fetched output to host_fetches[j], all asynchronously on cuda_stream
+ * (the caller synchronises the stream before reading the results; pinned host memory makes the
+ * copies truly asynchronous).  staging_dev: caller-owned device memory, 256-byte aligned, at
+ * least dragon_function_staging_bytes() long.  Entries of pruned inputs may be NULL. */
+size_t dragon_function_staging_bytes(const dragon_function_t* f);
+int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* const* host_fetches,
+                    void* staging_dev, size_t staging_bytes, void* cuda_stream);
+
+/* Device-side timing of one launch step of the plan (step index as listed by
+ * dragon_function_describe, one line per step; for a graph-VM step the VM kernel alone is
+ * bracketed, not its finishing reduction).  dragon_function_profile() arms a ring of
+ * `capacity` CUDA event pairs recorded around that step by every following dragon_run()
+ * (step < 0 disarms); dragon_function_profile_read() synchronises the recorded events and
+ * returns the summed kernel time and the number of runs since arming, then re-arms. */
+int dragon_function_profile(dragon_function_t* f, int step, int capacity);
+int dragon_function_profile_read(dragon_function_t* f, double* total_ms, int* runs);
+
 /* Synchronises the stream of the last run and returns the device status word: DRAGON_OK,
  * DRAGON_ERR_TIMEOUT (a bounded wait gave up) or DRAGON_ERR_INVALID_ARG (bad label). */
 int dragon_function_status(dragon_function_t* f);

@@ -43,6 +43,11 @@ _SIGNATURES = {
     "dragon_function_set_workspace": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
     "dragon_run": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p), _c.c_void_p]),
     "dragon_function_status": (_c.c_int, [_c.c_void_p]),
+    "dragon_function_staging_bytes": (_c.c_size_t, [_c.c_void_p]),
+    "dragon_run_host": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p), _c.c_void_p,
+                                   _c.c_size_t, _c.c_void_p]),
+    "dragon_function_profile": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_int]),
+    "dragon_function_profile_read": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_double), _c.POINTER(_c.c_int)]),
     "dragon_host_math": (_c.c_int, [_c.c_int, _c.POINTER(_c.c_float), _c.POINTER(_c.c_float), _c.c_int]),
     "dragon_last_error": (_c.c_char_p, []),
 }
@@ -221,15 +226,41 @@ class Function:
     def status(self):
         return lib().dragon_function_status(self.h)
 
+    def staging_bytes(self):
+        return lib().dragon_function_staging_bytes(self.h)
+
+    def run_host(self, host_feed_ptrs, host_fetch_ptrs, staging_ptr, staging_bytes, stream=0):
+        feeds = (_c.c_void_p * max(1, self.n_in))(*[p or None for p in host_feed_ptrs])
+        fetches = (_c.c_void_p * max(1, self.n_out))(*host_fetch_ptrs)
+        r = lib().dragon_run_host(self.h, feeds, fetches, staging_ptr, staging_bytes, stream)
+        if r < 0:
+            raise DragonError(r, "dragon_run_host")
+
+    def profile(self, step, capacity=1024):
+        r = lib().dragon_function_profile(self.h, step, capacity)
+        if r < 0:
+            raise DragonError(r, "dragon_function_profile")
+
+    def profile_read(self):
+        ms, runs = _c.c_double(), _c.c_int()
+        r = lib().dragon_function_profile_read(self.h, _c.byref(ms), _c.byref(runs))
+        if r < 0:
+            raise DragonError(r, "dragon_function_profile_read")
+        return ms.value, runs.value
+
     # ---- convenience for torch tensors (device memory and streams only) ----
-    def run_torch(self, feeds, fetches, stream=None):
-        """feeds / fetches: lists of CUDA torch tensors (None for a pruned input)."""
+    def ensure_workspace(self):
         import torch
         if self._ws is None:
             nbytes = max(256, self.workspace_bytes())
             self._ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
             base = (self._ws.data_ptr() + 255) & ~255
             self.set_workspace(base, nbytes)
+
+    def run_torch(self, feeds, fetches, stream=None):
+        """feeds / fetches: lists of CUDA torch tensors (None for a pruned input)."""
+        import torch
+        self.ensure_workspace()
         s = stream if stream is not None else torch.cuda.current_stream()
         self.run([0 if t is None else t.data_ptr() for t in feeds], [t.data_ptr() for t in fetches], s.cuda_stream)
 

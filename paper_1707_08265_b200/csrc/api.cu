@@ -191,6 +191,7 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
 
 void dragon_function_destroy(dragon_function_t* f) {
   if (!f) return;
+  for (void* ev : f->prof_ev) cudaEventDestroy(reinterpret_cast<cudaEvent_t>(ev));
   for (auto& sg : f->plan.segs)
     if (sg.d_code) cudaFree(sg.d_code);
   delete f;
@@ -283,8 +284,11 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
   }
   int* status = reinterpret_cast<int*>(ws + P.status_off);
   cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
-  for (const Step& s : P.steps) {
+  for (size_t si = 0; si < P.steps.size(); ++si) {
+    const Step& s = P.steps[si];
     if (e != cudaSuccess) break;
+    const bool prof = (int)si == f->prof_step && 2 * (f->prof_used + 1) <= (int)f->prof_ev.size();
+    if (prof && s.kind != ST_VM) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used]), st);
     switch (s.kind) {
       case ST_VM: {
         VmSegment& sg = P.segs[s.seg];
@@ -305,7 +309,9 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
           p.operand[i].kind = sg.operand_kind[i];
           p.operand[i].dtype = (uint32_t)P.mems[sg.operand_mem[i]].dtype;
         }
+        if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used]), st);
         e = launch_vm(p, sg.grid, sg.n_smem, st);
+        if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used + 1]), st);
         if (e == cudaSuccess) e = launch_finish(sg, P.mems, ptr.data(), ws, st);
         break;
       }
@@ -331,12 +337,101 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         e = cudaMemcpyAsync(ptr[s.mC], ptr[s.mA], P.mems[s.mA].bytes(), cudaMemcpyDeviceToDevice, st);
         break;
     }
+    if (prof) {
+      if (s.kind != ST_VM) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used + 1]), st);
+      ++f->prof_used;
+    }
   }
   if (e != cudaSuccess) {
     set_error("dragon_run: CUDA error: %s", cudaGetErrorString(e));
     return DRAGON_ERR_CUDA;
   }
   f->last_stream = cuda_stream;
+  return DRAGON_OK;
+}
+
+size_t dragon_function_staging_bytes(const dragon_function_t* f) {
+  if (!f) return 0;
+  size_t n = 0;
+  for (const MemRef& m : f->plan.mems)
+    if (m.live && m.where != MEM_WORK) n += (m.bytes() + 255) & ~(size_t)255;
+  return n;
+}
+
+int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* const* host_fetches, void* staging_dev,
+                    size_t staging_bytes, void* cuda_stream) {
+  if (!f || !host_fetches || (f->n_in > 0 && !host_feeds)) { set_error("dragon_run_host: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  if (!staging_dev || ((uintptr_t)staging_dev & 255) || staging_bytes < dragon_function_staging_bytes(f)) {
+    set_error("dragon_run_host: staging area must be 256-byte aligned device memory of at least %zu bytes", dragon_function_staging_bytes(f));
+    return DRAGON_ERR_WORKSPACE;
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  std::vector<const void*> feeds(f->n_in, nullptr);
+  std::vector<void*> fetches(f->n_out, nullptr);
+  char* base = reinterpret_cast<char*>(staging_dev);
+  size_t off = 0;
+  // several memrefs may name the same feed / fetch position: one staging slot per position
+  for (const MemRef& m : f->plan.mems) {
+    if (!m.live || m.where == MEM_WORK) continue;
+    const size_t sz = (m.bytes() + 255) & ~(size_t)255;
+    if (m.where == MEM_FEED && !feeds[m.index]) {
+      if (!host_feeds[m.index]) { set_error("dragon_run_host: feed %d is NULL", m.index); return DRAGON_ERR_INVALID_ARG; }
+      feeds[m.index] = base + off;
+      if (cudaMemcpyAsync(base + off, host_feeds[m.index], m.bytes(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        set_error("dragon_run_host: host-to-device copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+        return DRAGON_ERR_CUDA;
+      }
+    } else if (m.where == MEM_FETCH && !fetches[m.index]) {
+      if (!host_fetches[m.index]) { set_error("dragon_run_host: fetch %d is NULL", m.index); return DRAGON_ERR_INVALID_ARG; }
+      fetches[m.index] = base + off;
+    }
+    off += sz;
+  }
+  int rc = dragon_run(f, feeds.data(), fetches.data(), cuda_stream);
+  if (rc != DRAGON_OK) return rc;
+  std::vector<uint8_t> copied(f->n_out, 0);
+  for (const MemRef& m : f->plan.mems) {
+    if (!m.live || m.where != MEM_FETCH || copied[m.index]) continue;
+    copied[m.index] = 1;
+    if (cudaMemcpyAsync(host_fetches[m.index], fetches[m.index], m.bytes(), cudaMemcpyDeviceToHost, st) != cudaSuccess) {
+      set_error("dragon_run_host: device-to-host copy failed: %s", cudaGetErrorString(cudaGetLastError()));
+      return DRAGON_ERR_CUDA;
+    }
+  }
+  return DRAGON_OK;
+}
+
+int dragon_function_profile(dragon_function_t* f, int step, int capacity) {
+  if (!f || step >= (int)f->plan.steps.size() || (step >= 0 && (capacity <= 0 || capacity > 65536))) {
+    set_error("dragon_function_profile: bad argument");
+    return DRAGON_ERR_INVALID_ARG;
+  }
+  f->prof_step = step;
+  f->prof_used = 0;
+  if (step < 0) return DRAGON_OK;
+  while ((int)f->prof_ev.size() < 2 * capacity) {
+    cudaEvent_t ev;
+    if (cudaEventCreate(&ev) != cudaSuccess) { set_error("dragon_function_profile: cudaEventCreate failed"); return DRAGON_ERR_CUDA; }
+    f->prof_ev.push_back(ev);
+  }
+  return DRAGON_OK;
+}
+
+int dragon_function_profile_read(dragon_function_t* f, double* total_ms, int* runs) {
+  if (!f || !total_ms || !runs) { set_error("dragon_function_profile_read: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  double tot = 0.0;
+  for (int i = 0; i < f->prof_used; ++i) {
+    cudaEvent_t a = reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * i]), b = reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * i + 1]);
+    float ms = 0.f;
+    if (cudaEventSynchronize(b) != cudaSuccess || cudaEventElapsedTime(&ms, a, b) != cudaSuccess) {
+      set_error("dragon_function_profile_read: %s", cudaGetErrorString(cudaGetLastError()));
+      return DRAGON_ERR_CUDA;
+    }
+    tot += ms;
+  }
+  *total_ms = tot;
+  *runs = f->prof_used;
+  f->prof_used = 0;
   return DRAGON_OK;
 }
 

@@ -123,4 +123,7 @@ struct dragon_function {
   size_t workspace_bytes = 0;
   void* last_stream = nullptr;
   bool uploaded = false;
+  // profiling ring (dragon_function_profile)
+  int prof_step = -1, prof_used = 0;
+  std::vector<void*> prof_ev;   // 2 * capacity cudaEvent_t
 };
