@@ -9,7 +9,7 @@ LIB = os.path.join(HERE, "libdragon.so")
 SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "api.cu", "vm_kernel.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
-         "--expt-relaxed-constexpr", "-Xcompiler", "-Wall"]
+         "--expt-relaxed-constexpr", "-Xcompiler", "-Wall"] + os.environ.get("DRAGON_NVCC_DEFS", "").split()
 
 
 def _stale(target, deps):

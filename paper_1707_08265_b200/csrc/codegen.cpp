@@ -121,8 +121,8 @@ struct Gen {
       f.home = H_NONE;
     } else {
       int s = free_smem();
-      if (s >= 0) { emit(P_RTOS, best, s); f.home = H_SMEM; f.home_idx = s; smem_owner[s] = v; }
-      else { int gsl = new_spill(); emit(P_SPILL, best, gsl); f.home = H_SPILL; f.home_idx = gsl; }
+      if (s >= 0) { emit(J_RTOS * kJointStride + best, 0, s); f.home = H_SMEM; f.home_idx = s; smem_owner[s] = v; }
+      else { int gsl = new_spill(); emit(J_SPILL * kJointStride + best, 0, gsl); f.home = H_SPILL; f.home_idx = gsl; }
     }
     reg_owner[best] = -1;
     return best;
@@ -150,7 +150,7 @@ struct Gen {
       if (farthest >= 0 && farthest <= nu) {
         int s = free_smem();
         if (s >= 0) { emit(P_STS, 0, s); f.home = H_SMEM; f.home_idx = s; smem_owner[s] = v; }
-        else { int gsl = new_spill(); emit(P_SPILL, kAccSlot, gsl); f.home = H_SPILL; f.home_idx = gsl; }
+        else { int gsl = new_spill(); emit(P_SPILL, 0, gsl); f.home = H_SPILL; f.home_idx = gsl; }
         return;
       }
     }
@@ -165,18 +165,25 @@ struct Gen {
     if (f.uni >= 0) emit(P_LDU, 0, f.uni);
     else if (f.home == H_REG) emit(J_LDR * kJointStride + f.home_idx);
     else if (f.home == H_SMEM) emit(P_LDS, 0, f.home_idx);
-    else if (f.home == H_SPILL) emit(P_FILL, kAccSlot, f.home_idx);
-    else if (f.operand >= 0) emit(P_GLD, kAccSlot, f.operand);
+    else if (f.home == H_SPILL) emit(P_FILL, 0, f.home_idx);
+    else if (f.operand >= 0) emit(P_GLD, 0, f.operand);
     else { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: value has no location"); }
     acc_val = v;
   }
-  void make_addressable(int v, int pos, int keep1, int keep2) {
-    if (addressable(v)) return;
+  // a spilled value comes back into a register slot without touching the accumulator
+  bool fill_to_reg(int v, int pos, int keep1, int keep2) {
     VInfo& f = info[v];
+    if (f.home != H_SPILL) return false;
     int k = alloc_reg(pos, keep1, keep2);
-    if (f.home == H_SPILL) { emit(P_FILL, k, f.home_idx); free_spill.push_back(f.home_idx); }
-    else if (f.operand >= 0) emit(P_GLD, k, f.operand);
-    else { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: operand has no location"); }
+    emit(J_FILL * kJointStride + k, 0, f.home_idx);
+    free_spill.push_back(f.home_idx);
+    give_reg(v, k);
+    return true;
+  }
+  // acc holds v: give it a register home now
+  void home_acc(int v, int pos, int keep1, int keep2) {
+    int k = alloc_reg(pos, keep1, keep2);
+    emit_str(k);
     give_reg(v, k);
   }
   // acc holds x and is about to be overwritten by a result: give x a home if it is needed again
@@ -214,9 +221,19 @@ struct Gen {
     }
     if (a == b) {
       load_acc(x, pos, x);
-      if (!addressable(x)) { int k = alloc_reg(pos, x); emit_str(k); give_reg(x, k); }
+      if (!addressable(x)) home_acc(x, pos, x, -1);
     } else {
-      if (!addressable(y)) make_addressable(y, pos, x, y);
+      if (!addressable(y)) fill_to_reg(y, pos, x, y);
+      if (!addressable(y)) {
+        // y is a memory operand: it has to pass through the accumulator, so the roles swap
+        if (acc_val == x) {
+          if (!addressable(x)) home_acc(x, pos, x, y);
+        } else if (!addressable(x) && !fill_to_reg(x, pos, x, y)) {
+          load_acc(x, pos, x, y);
+          home_acc(x, pos, x, y);
+        }
+        std::swap(x, y);
+      }
       load_acc(x, pos, x, y);
       keep_operand(x, pos, y);
     }
@@ -243,10 +260,11 @@ struct Gen {
       for (int q = pos + 1; q < (int)idx.size() && q < pos + 4096; ++q) {
         const Item& o2 = items[idx[q]];
         if (done[q] || o2.kind != IT_MOP || (o2.opc != M_SIN && o2.opc != M_COS) || o2.opc == it.opc || C(o2.a) != a) continue;
-        int k = alloc_reg(pos, a);
-        emit(P_SINCOS, k, 0);
+        int sl = free_smem();
+        if (sl < 0) break;  // no slot for the cosine: two separate instructions
+        emit(P_SINCOS, 0, sl);
         int dsin = it.opc == M_SIN ? d : C(o2.dst), dcos = it.opc == M_SIN ? C(o2.dst) : d;
-        give_reg(dcos, k);
+        info[dcos].home = H_SMEM; info[dcos].home_idx = sl; smem_owner[sl] = dcos;
         acc_val = dsin;
         done[q] = true;
         auto& u = info[a].uses;  // the partner's use of a is consumed here
@@ -345,10 +363,8 @@ struct Gen {
         int cls = class_of(mems[it.mem].shape);
         if (cls < 0) { set_error("graph VM: store shape does not fit the fused domain"); return DRAGON_ERR_UNSUPPORTED; }
         int opd = operand_for(it.mem, cls);
-        VInfo& f = info[v];
-        if (acc_val == v) emit(P_GST, kAccSlot, opd);
-        else if (f.home == H_REG) emit(P_GST, f.home_idx, opd);
-        else { load_acc(v, p, v); emit(P_GST, kAccSlot, opd); }
+        load_acc(v, p, v);
+        emit(P_GST, 0, opd);
         release_dead(v, p);
       } else if (it.opc == M_ACCUM) {
         int v = C(it.a), k = -1;
@@ -378,8 +394,9 @@ struct Gen {
       const Item& it = items[idx[a.first]];
       int cls = class_of(mems[it.mem].shape);
       FinishJob job; job.mem = it.mem;
-      if (cls == K_SCALAR) { job.kind = 1; job.acc = seg->n_scalacc++; epi.push_back(encode(P_SCALOUT, a.second, job.acc)); }
-      else if (cls == K_ROW) { job.kind = 0; job.acc = seg->n_colacc++; epi.push_back(encode(P_COLOUT, a.second, job.acc)); }
+      epi.push_back(encode(J_LDR * kJointStride + a.second, 0, 0));
+      if (cls == K_SCALAR) { job.kind = 1; job.acc = seg->n_scalacc++; epi.push_back(encode(P_SCALOUT, 0, job.acc)); }
+      else if (cls == K_ROW) { job.kind = 0; job.acc = seg->n_colacc++; epi.push_back(encode(P_COLOUT, 0, job.acc)); }
       else { set_error("graph VM: reduction target shape is not supported"); return DRAGON_ERR_UNSUPPORTED; }
       seg->finish.push_back(job);
     }

@@ -11,10 +11,17 @@
 namespace dragon {
 
 // geometry of the VM kernel: every CTA owns tiles of kVmTile elements, kVmVec per thread
-constexpr int kVmThreads = 256;
-constexpr int kVmVec = 16;
+#ifndef DRAGON_VM_REGS
+#define DRAGON_VM_REGS 7
+#endif
+#ifndef DRAGON_VM_THREADS
+#define DRAGON_VM_THREADS 512
+#define DRAGON_VM_VEC 8
+#endif
+constexpr int kVmThreads = DRAGON_VM_THREADS;
+constexpr int kVmVec = DRAGON_VM_VEC;
 constexpr int kVmTile = kVmThreads * kVmVec;  // 4096
-constexpr int kVmRegs = 10;                   // register slots R[0..kVmRegs)
+constexpr int kVmRegs = DRAGON_VM_REGS;       // register slots R[0..kVmRegs)
 constexpr int kVmCodeMaxWords = 12 * 1024;    // instruction stream held in shared memory
 constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread
 constexpr int kDefaultSmCount = 148;

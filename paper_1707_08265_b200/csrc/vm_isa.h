@@ -1,6 +1,6 @@
 // Instruction set of the graph-VM kernel.  One 32-bit word per instruction:
 //   bits 0..9   case id (for register-operand instructions: base + register slot)
-//   bits 10..13 r   (register slot, or kAccSlot for the accumulator) of the two-level instructions
+//   bits 10..13 reserved
 //   bits 14..31 arg (uniform / shared-memory slot / operand / spill index)
 // The machine is an accumulator machine: every thread owns V elements of the current tile;
 // "acc" and the register slots R[0..NR) are V-wide and live in registers, shared-memory slots
@@ -13,7 +13,6 @@ namespace vm {
 
 constexpr int kMaxOperands = 40;   // memory operands per kernel launch
 constexpr int kMaxUniforms = 512;
-constexpr int kAccSlot = 15;       // value of the r field that names the accumulator
 
 enum Joint : int {  // each occupies kJointStride consecutive case ids, one per register slot
   J_LDR = 0,   // acc = R
@@ -27,6 +26,10 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   J_ADDTO,     // R = R + acc
   J_ACCUM,     // R = R + (lane valid ? acc : 0)   (loop-carried accumulators)
   J_FMAUR,     // acc = acc * U[arg] + R
+  J_RTOS,      // S[arg] = R
+  J_STOR,      // R = S[arg]
+  J_SPILL,     // spill[arg] = R
+  J_FILL,      // R = spill[arg]
   J_COUNT
 };
 constexpr int kJointStride = 16;
@@ -39,10 +42,8 @@ enum Plain : int {
   P_LDS,                // acc = S[arg]
   P_STS,                // S[arg] = acc
   P_ADDS, P_SUBS, P_RSUBS, P_MULS, P_DIVPS, P_RDIVPS,
-  P_RTOS,               // S[arg] = R[r]
-  P_STOR,               // R[r] = S[arg]
   P_SIN, P_COS,
-  P_SINCOS,             // R[r] = cos(acc); acc = sin(acc)
+  P_SINCOS,             // S[arg] = cos(acc); acc = sin(acc)
   P_EXPC, P_TANH, P_SIGMOID, P_RELU, P_NEG,
   P_STEP,               // acc = acc > 0 ? 1 : 0
   P_CLAMPMASK,          // acc = (-10 <= acc <= 10) ? 1 : 0
@@ -51,16 +52,16 @@ enum Plain : int {
   P_DIVPGB,             // acc = -sgn(acc) / (1 + |acc|)^2
   P_RBF16,              // acc = float(bf16(acc)), round to nearest even
   P_ROWSUM,             // acc = sum of acc over the whole row (all lanes, all threads), row mode only
-  P_GLD,                // {R[r] | acc} = operand[arg] at this tile
-  P_GST,                // operand[arg] at this tile = {R[r] | acc}
-  P_FILL,               // {R[r] | acc} = spill[arg]
-  P_SPILL,              // spill[arg] = {R[r] | acc}
+  P_GLD,                // acc = operand[arg] at this tile
+  P_GST,                // operand[arg] at this tile = acc
+  P_FILL,               // acc = spill[arg]
+  P_SPILL,              // spill[arg] = acc
   P_ULOAD,              // U[arg & 511] = scalar operand[arg >> 9]   (prologue)
   P_UCONST,             // U[arg] = next word reinterpreted as float (prologue)
   P_LOOP_BEGIN,         // start of the per-tile body
   P_LOOP_END,           // next tile; jumps back to the body or falls through to the epilogue
-  P_COLOUT,             // column partial sums: colpart[arg][cta][c] = {R[r] | acc}
-  P_SCALOUT,            // scalar partial sum: scalpart[arg][cta] = block sum of {R[r] | acc} in fp64
+  P_COLOUT,             // column partial sums: colpart[arg][cta][c] = acc
+  P_SCALOUT,            // scalar partial sum: scalpart[arg][cta] = block sum of acc in fp64
   P_END,
   P_COUNT_
 };

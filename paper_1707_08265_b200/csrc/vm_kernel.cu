@@ -25,7 +25,7 @@ constexpr int V = kVmVec;
 constexpr int NV4 = V / 4;
 constexpr int NR = kVmRegs;
 constexpr int TILE = kVmTile;
-static_assert(V == 16 && NR == 10 && NT == 256, "the case tables below are written for 16 lanes and 10 register slots");
+static_assert(V % 4 == 0 && NR >= 6 && NR <= 12, "the case tables below are written for 6..12 register slots");
 
 #define FORV _Pragma("unroll") for (int j = 0; j < V; ++j)
 
@@ -129,41 +129,65 @@ __device__ __forceinline__ void store_operand(const Operand& o, const TileCtx& t
     if (tc.full) { FORV R[K][j] += acc[j]; }                                                      \
     else { FORV R[K][j] += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }                        \
     break;                                                                                        \
-  case J_FMAUR * kJointStride + K: { const float u_ = U[arg]; FORV acc[j] = fmaf(acc[j], u_, R[K][j]); } break;
+  case J_FMAUR * kJointStride + K: { const float u_ = U[arg]; FORV acc[j] = fmaf(acc[j], u_, R[K][j]); } break; \
+  case J_RTOS * kJointStride + K: VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, R[K]) break;       \
+  case J_STOR * kJointStride + K: VEC_LOAD(R[K], slots + (size_t)arg * NV4 * NT + tid) break;        \
+  case J_SPILL * kJointStride + K: VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, R[K]) break; \
+  case J_FILL * kJointStride + K: VEC_LOAD(R[K], reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) break;
 
-#define ALL_SLOTS(M) M(0) M(1) M(2) M(3) M(4) M(5) M(6) M(7) M(8) M(9)
+#if DRAGON_VM_REGS > 6
+#define SLOT6(M) M(6)
+#else
+#define SLOT6(M)
+#endif
+#if DRAGON_VM_REGS > 7
+#define SLOT7(M) M(7)
+#else
+#define SLOT7(M)
+#endif
+#if DRAGON_VM_REGS > 8
+#define SLOT8(M) M(8)
+#else
+#define SLOT8(M)
+#endif
+#if DRAGON_VM_REGS > 9
+#define SLOT9(M) M(9)
+#else
+#define SLOT9(M)
+#endif
+#if DRAGON_VM_REGS > 10
+#define SLOT10(M) M(10)
+#else
+#define SLOT10(M)
+#endif
+#if DRAGON_VM_REGS > 11
+#define SLOT11(M) M(11)
+#else
+#define SLOT11(M)
+#endif
+#define ALL_SLOTS(M) M(0) M(1) M(2) M(3) M(4) M(5) SLOT6(M) SLOT7(M) SLOT8(M) SLOT9(M) SLOT10(M) SLOT11(M)
 
-#define SEL_TO_T_CASE(K) case K: FORV t[j] = R[K][j]; break;
-#define SEL_FROM_T_CASE(K) case K: FORV R[K][j] = t[j]; break;
-#define SELECT_TO_T(r)                       \
-  switch (r) {                               \
-    ALL_SLOTS(SEL_TO_T_CASE)                 \
-    default: FORV t[j] = acc[j]; break;      \
-  }
-#define SELECT_FROM_T(r)                     \
-  switch (r) {                               \
-    ALL_SLOTS(SEL_FROM_T_CASE)               \
-    default: FORV acc[j] = t[j]; break;      \
-  }
+// a V-wide value <-> NV4 float4 cells spaced NT apart (one column per thread)
+#define VEC_STORE(ptr, X) { float4* p_ = (ptr); _Pragma("unroll") for (int h = 0; h < NV4; ++h) p_[h * NT] = make_float4((X)[4 * h], (X)[4 * h + 1], (X)[4 * h + 2], (X)[4 * h + 3]); }
+#define VEC_LOAD(X, ptr) { const float4* p_ = (ptr); _Pragma("unroll") for (int h = 0; h < NV4; ++h) { const float4 v_ = p_[h * NT]; (X)[4 * h] = v_.x; (X)[4 * h + 1] = v_.y; (X)[4 * h + 2] = v_.z; (X)[4 * h + 3] = v_.w; } }
 
-#define T_FROM_VEC4(h, v) { t[4 * (h)] = (v).x; t[4 * (h) + 1] = (v).y; t[4 * (h) + 2] = (v).z; t[4 * (h) + 3] = (v).w; }
-#define VEC4_FROM_T(h) make_float4(t[4 * (h)], t[4 * (h) + 1], t[4 * (h) + 2], t[4 * (h) + 3])
 
 __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Params p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // layout: code | uniforms | reduction scratch | V-wide slots
+  // layout: code | uniforms | reduction scratch | staging columns | V-wide slots
   uint32_t* code = reinterpret_cast<uint32_t*>(smem_raw);
   const int code_words = (p.n_code + 3) & ~3;
   float* U = reinterpret_cast<float*>(code + code_words);
   double* red = reinterpret_cast<double*>(U + kMaxUniforms);
-  float4* slots = reinterpret_cast<float4*>(red + 64);
+  float4* stage = reinterpret_cast<float4*>(red + 64) + threadIdx.x;   // [NV4][NT], one column per thread
+  float4* slots = reinterpret_cast<float4*>(red + 64) + NV4 * NT;      // [slot][NV4][NT]
 
   const int tid = threadIdx.x;
   for (int i = tid; i < p.n_code; i += NT) code[i] = p.code[i];
   __syncthreads();
 
-  float acc[V], t[V], R[NR][V];
-  FORV { acc[j] = 0.f; t[j] = 0.f; }
+  float acc[V], R[NR][V];
+  FORV acc[j] = 0.f;
 #pragma unroll
   for (int k = 0; k < NR; ++k) FORV R[k][j] = 0.f;
 
@@ -194,7 +218,6 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
     uint32_t wn = code[pc + 1];  // fetched ahead of the dispatch below
     ++pc;
     const int cs = w & 1023u;
-    const int r = (w >> 10) & 15u;
     const uint32_t arg = w >> 14;
     switch (cs) {
       ALL_SLOTS(JOINT_CASES)
@@ -206,34 +229,44 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
       case P_DIVPU: { const float u = vmmath::f_rcp(1.f + fabsf(U[arg])); FORV acc[j] *= u; } break;
       case P_RDIVPU: { const float u = U[arg]; FORV acc[j] = vmmath::divp_f(u, acc[j]); } break;
       case P_FMAU: { const float a = U[arg & 511u], b = U[arg >> 9]; FORV acc[j] = fmaf(acc[j], a, b); } break;
-      case P_LDS: case P_ADDS: case P_SUBS: case P_RSUBS: case P_MULS: case P_DIVPS: case P_RDIVPS: case P_STOR: {
-#pragma unroll
-        for (int h = 0; h < NV4; ++h) { const float4 v = slots[(arg * NV4 + h) * NT + tid]; T_FROM_VEC4(h, v) }
+      case P_LDS: VEC_LOAD(acc, slots + (size_t)arg * NV4 * NT + tid) break;
+      case P_STS: VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, acc) break;
+      case P_ADDS: case P_SUBS: case P_RSUBS: case P_MULS: case P_DIVPS: case P_RDIVPS: {
+        float t[V];
+        VEC_LOAD(t, slots + (size_t)arg * NV4 * NT + tid)
         switch (cs) {
-          case P_LDS: FORV acc[j] = t[j]; break;
           case P_ADDS: FORV acc[j] += t[j]; break;
           case P_SUBS: FORV acc[j] -= t[j]; break;
           case P_RSUBS: FORV acc[j] = t[j] - acc[j]; break;
           case P_MULS: FORV acc[j] *= t[j]; break;
           case P_DIVPS: FORV acc[j] = vmmath::divp_f(acc[j], t[j]); break;
-          case P_RDIVPS: FORV acc[j] = vmmath::divp_f(t[j], acc[j]); break;
-          default: SELECT_FROM_T(r) break;
+          default: FORV acc[j] = vmmath::divp_f(t[j], acc[j]); break;
         }
       } break;
-      case P_STS: case P_RTOS: {
-        if (cs == P_STS) { FORV t[j] = acc[j]; } else { SELECT_TO_T(r) }
-#pragma unroll
-        for (int h = 0; h < NV4; ++h) slots[(arg * NV4 + h) * NT + tid] = VEC4_FROM_T(h);
+      case P_SIN: case P_COS: case P_SINCOS: case P_EXPC: case P_TANH: case P_SIGMOID: {
+        // The expensive functions run four lanes at a time in a rolled loop over a per-thread
+        // staging column in shared memory: unrolled over all lanes, their temporaries would not
+        // fit in the register file beside the register slots.
+        VEC_STORE(stage, acc)
+#pragma unroll 1
+        for (int h = 0; h < NV4; ++h) {
+          float4 v = stage[h * NT], c4 = v;
+          switch (cs) {
+            case P_SIN: v.x = vmmath::sin_f(v.x); v.y = vmmath::sin_f(v.y); v.z = vmmath::sin_f(v.z); v.w = vmmath::sin_f(v.w); break;
+            case P_COS: v.x = vmmath::cos_f(v.x); v.y = vmmath::cos_f(v.y); v.z = vmmath::cos_f(v.z); v.w = vmmath::cos_f(v.w); break;
+            case P_SINCOS:
+              vmmath::sincos_f(c4.x, &v.x, &c4.x); vmmath::sincos_f(c4.y, &v.y, &c4.y);
+              vmmath::sincos_f(c4.z, &v.z, &c4.z); vmmath::sincos_f(c4.w, &v.w, &c4.w);
+              slots[((size_t)arg * NV4 + h) * NT + tid] = c4;
+              break;
+            case P_EXPC: v.x = vmmath::exp_clamped10(v.x); v.y = vmmath::exp_clamped10(v.y); v.z = vmmath::exp_clamped10(v.z); v.w = vmmath::exp_clamped10(v.w); break;
+            case P_TANH: v.x = vmmath::tanh_f(v.x); v.y = vmmath::tanh_f(v.y); v.z = vmmath::tanh_f(v.z); v.w = vmmath::tanh_f(v.w); break;
+            default: v.x = vmmath::sigmoid_f(v.x); v.y = vmmath::sigmoid_f(v.y); v.z = vmmath::sigmoid_f(v.z); v.w = vmmath::sigmoid_f(v.w); break;
+          }
+          stage[h * NT] = v;
+        }
+        VEC_LOAD(acc, stage)
       } break;
-      case P_SIN: FORV acc[j] = vmmath::sin_f(acc[j]); break;
-      case P_COS: FORV acc[j] = vmmath::cos_f(acc[j]); break;
-      case P_SINCOS: {
-        FORV { float s_, c_; vmmath::sincos_f(acc[j], &s_, &c_); acc[j] = s_; t[j] = c_; }
-        SELECT_FROM_T(r)
-      } break;
-      case P_EXPC: FORV acc[j] = vmmath::exp_clamped10(acc[j]); break;
-      case P_TANH: FORV acc[j] = vmmath::tanh_f(acc[j]); break;
-      case P_SIGMOID: FORV acc[j] = vmmath::sigmoid_f(acc[j]); break;
       case P_RELU: FORV acc[j] = fmaxf(acc[j], 0.f); break;
       case P_NEG: FORV acc[j] = -acc[j]; break;
       case P_STEP: FORV acc[j] = acc[j] > 0.f ? 1.f : 0.f; break;
@@ -257,26 +290,10 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
         __syncthreads();
         FORV acc[j] = tot;
       } break;
-      case P_GLD: {
-        load_operand(p.operand[arg], tc, tid, t);
-        SELECT_FROM_T(r)
-      } break;
-      case P_GST: {
-        SELECT_TO_T(r)
-        store_operand(p.operand[arg], tc, tid, t);
-      } break;
-      case P_FILL: {
-        const float4* s4 = reinterpret_cast<const float4*>(spill + (size_t)arg * TILE);
-#pragma unroll
-        for (int h = 0; h < NV4; ++h) { const float4 v = s4[h * NT + tid]; T_FROM_VEC4(h, v) }
-        SELECT_FROM_T(r)
-      } break;
-      case P_SPILL: {
-        SELECT_TO_T(r)
-        float4* s4 = reinterpret_cast<float4*>(spill + (size_t)arg * TILE);
-#pragma unroll
-        for (int h = 0; h < NV4; ++h) s4[h * NT + tid] = VEC4_FROM_T(h);
-      } break;
+      case P_GLD: load_operand(p.operand[arg], tc, tid, acc); break;
+      case P_GST: store_operand(p.operand[arg], tc, tid, acc); break;
+      case P_FILL: VEC_LOAD(acc, reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) break;
+      case P_SPILL: VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, acc) break;
       case P_ULOAD: {
         if (tid == 0) {
           const Operand& o = p.operand[arg >> 9];
@@ -298,14 +315,12 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
         if (tile < ntiles) { set_tile(); pc = loop_pc; wn = code[pc]; }
         break;
       case P_COLOUT: {
-        SELECT_TO_T(r)
         float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
-        FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = t[j]; }
+        FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = acc[j]; }
       } break;
       case P_SCALOUT: {
-        SELECT_TO_T(r)
         double s = 0.0;
-        FORV s += (double)t[j];
+        FORV s += (double)acc[j];
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
         if ((tid & 31) == 0) red[tid >> 5] = s;
@@ -356,7 +371,7 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
 }
 
 size_t vm_smem_bytes(int n_code, int n_smem_slots) {
-  return (size_t)((n_code + 3) & ~3) * 4 + kMaxUniforms * 4 + 64 * 8 + (size_t)n_smem_slots * NV4 * NT * 16;
+  return (size_t)((n_code + 3) & ~3) * 4 + kMaxUniforms * 4 + 64 * 8 + (size_t)(n_smem_slots + 1) * NV4 * NT * 16;
 }
 
 }  // namespace vm
