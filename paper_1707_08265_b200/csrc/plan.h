@@ -11,13 +11,6 @@
 namespace dragon {
 
 // geometry of the VM kernel: every CTA owns tiles of kVmTile elements, kVmVec per thread
-#ifndef DRAGON_VM_REGS
-#define DRAGON_VM_REGS 7
-#endif
-#ifndef DRAGON_VM_THREADS
-#define DRAGON_VM_THREADS 512
-#define DRAGON_VM_VEC 8
-#endif
 constexpr int kVmThreads = DRAGON_VM_THREADS;
 constexpr int kVmVec = DRAGON_VM_VEC;
 constexpr int kVmTile = kVmThreads * kVmVec;  // 4096

@@ -8,6 +8,15 @@
 #pragma once
 #include <cstdint>
 
+// geometry of the VM kernel (threads per CTA, elements per thread, register slots)
+#ifndef DRAGON_VM_REGS
+#define DRAGON_VM_REGS 7
+#endif
+#ifndef DRAGON_VM_THREADS
+#define DRAGON_VM_THREADS 512
+#define DRAGON_VM_VEC 8
+#endif
+
 namespace dragon {
 namespace vm {
 
@@ -32,7 +41,7 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   J_FILL,      // R = spill[arg]
   J_COUNT
 };
-constexpr int kJointStride = 16;
+constexpr int kJointStride = DRAGON_VM_REGS;  // case ids are dense, so the dispatch is one indexed jump
 constexpr int kFirstPlain = J_COUNT * kJointStride;
 
 enum Plain : int {

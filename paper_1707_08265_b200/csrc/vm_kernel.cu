@@ -13,6 +13,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <type_traits>
 
 #include "plan.h"
 #include "vm_math.h"
@@ -114,73 +115,31 @@ __device__ __forceinline__ void store_operand(const Operand& o, const TileCtx& t
   }
 }
 
-// every joint instruction for register slot K
-#define JOINT_CASES(K)                                                                            \
-  case J_LDR * kJointStride + K: FORV acc[j] = R[K][j]; break;                                    \
-  case J_STR * kJointStride + K: FORV R[K][j] = acc[j]; break;                                    \
-  case J_ADD * kJointStride + K: FORV acc[j] = acc[j] + R[K][j]; break;                           \
-  case J_SUB * kJointStride + K: FORV acc[j] = acc[j] - R[K][j]; break;                           \
-  case J_RSUB * kJointStride + K: FORV acc[j] = R[K][j] - acc[j]; break;                          \
-  case J_MUL * kJointStride + K: FORV acc[j] = acc[j] * R[K][j]; break;                           \
-  case J_DIVP * kJointStride + K: FORV acc[j] = vmmath::divp_f(acc[j], R[K][j]); break;           \
-  case J_RDIVP * kJointStride + K: FORV acc[j] = vmmath::divp_f(R[K][j], acc[j]); break;          \
-  case J_ADDTO * kJointStride + K: FORV R[K][j] += acc[j]; break;                                 \
-  case J_ACCUM * kJointStride + K:                                                                \
-    if (tc.full) { FORV R[K][j] += acc[j]; }                                                      \
-    else { FORV R[K][j] += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }                        \
-    break;                                                                                        \
-  case J_FMAUR * kJointStride + K: { const float u_ = U[arg]; FORV acc[j] = fmaf(acc[j], u_, R[K][j]); } break; \
-  case J_RTOS * kJointStride + K: VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, R[K]) break;       \
-  case J_STOR * kJointStride + K: VEC_LOAD(R[K], slots + (size_t)arg * NV4 * NT + tid) break;        \
-  case J_SPILL * kJointStride + K: VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, R[K]) break; \
-  case J_FILL * kJointStride + K: VEC_LOAD(R[K], reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) break;
-
-#if DRAGON_VM_REGS > 6
-#define SLOT6(M) M(6)
-#else
-#define SLOT6(M)
-#endif
-#if DRAGON_VM_REGS > 7
-#define SLOT7(M) M(7)
-#else
-#define SLOT7(M)
-#endif
-#if DRAGON_VM_REGS > 8
-#define SLOT8(M) M(8)
-#else
-#define SLOT8(M)
-#endif
-#if DRAGON_VM_REGS > 9
-#define SLOT9(M) M(9)
-#else
-#define SLOT9(M)
-#endif
-#if DRAGON_VM_REGS > 10
-#define SLOT10(M) M(10)
-#else
-#define SLOT10(M)
-#endif
-#if DRAGON_VM_REGS > 11
-#define SLOT11(M) M(11)
-#else
-#define SLOT11(M)
-#endif
-#define ALL_SLOTS(M) M(0) M(1) M(2) M(3) M(4) M(5) SLOT6(M) SLOT7(M) SLOT8(M) SLOT9(M) SLOT10(M) SLOT11(M)
-
 // a V-wide value <-> NV4 float4 cells spaced NT apart (one column per thread)
 #define VEC_STORE(ptr, X) { float4* p_ = (ptr); _Pragma("unroll") for (int h = 0; h < NV4; ++h) p_[h * NT] = make_float4((X)[4 * h], (X)[4 * h + 1], (X)[4 * h + 2], (X)[4 * h + 3]); }
 #define VEC_LOAD(X, ptr) { const float4* p_ = (ptr); _Pragma("unroll") for (int h = 0; h < NV4; ++h) { const float4 v_ = p_[h * NT]; (X)[4 * h] = v_.x; (X)[4 * h + 1] = v_.y; (X)[4 * h + 2] = v_.z; (X)[4 * h + 3] = v_.w; } }
 
 
+// balanced binary search over [LO, HI): calls f(integral_constant<LEAF>, arg) for the leaf equal to cs
+template <int LO, int HI, class F>
+__device__ __forceinline__ void dispatch_tree(const int cs, const uint32_t arg, F& f) {
+  if constexpr (HI - LO == 1) {
+    f(std::integral_constant<int, LO>{}, arg);
+  } else {
+    constexpr int MID = (LO + HI) / 2;
+    if (cs < MID) dispatch_tree<LO, MID>(cs, arg, f);
+    else dispatch_tree<MID, HI>(cs, arg, f);
+  }
+}
+
 __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Params p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
-  // layout: code | uniforms | reduction scratch | staging columns | V-wide slots
+  // layout: code | uniforms | reduction scratch | V-wide slots
   uint32_t* code = reinterpret_cast<uint32_t*>(smem_raw);
   const int code_words = (p.n_code + 3) & ~3;
   float* U = reinterpret_cast<float*>(code + code_words);
   double* red = reinterpret_cast<double*>(U + kMaxUniforms);
-  float4* stage = reinterpret_cast<float4*>(red + 64) + threadIdx.x;   // [NV4][NT], one column per thread
-  float4* slots = reinterpret_cast<float4*>(red + 64) + NV4 * NT;      // [slot][NV4][NT]
+  float4* slots = reinterpret_cast<float4*>(red + 64);                // [slot][NV4][NT]
 
   const int tid = threadIdx.x;
   for (int i = tid; i < p.n_code; i += NT) code[i] = p.code[i];
@@ -212,6 +171,95 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
   set_tile();
   float* spill = p.spill + (size_t)blockIdx.x * p.n_spill * TILE;
 
+  // One instruction = one leaf of a balanced binary decision tree over the case id (the
+  // compiler turns a switch of this size into a long compare chain, and indexed jumps are not
+  // available from CUDA C); every leaf is compiled for its own constant case id, so register
+  // slots are named statically.
+  auto exec = [&](auto cs_tag, const uint32_t arg) {
+    constexpr int CS = decltype(cs_tag)::value;
+#ifdef DRAGON_VM_EXPERIMENT_MINIMAL
+    if constexpr (!(CS == P_RELU || CS == P_GLD || CS == P_GST || CS / kJointStride == J_ADD || CS / kJointStride == J_STR)) { return; } else
+#endif
+    if constexpr (CS < kFirstPlain) {
+      constexpr int J = CS / kJointStride, K = CS % kJointStride;
+      if constexpr (J == J_LDR) { FORV acc[j] = R[K][j]; }
+      else if constexpr (J == J_STR) { FORV R[K][j] = acc[j]; }
+      else if constexpr (J == J_ADD) { FORV acc[j] = acc[j] + R[K][j]; }
+      else if constexpr (J == J_SUB) { FORV acc[j] = acc[j] - R[K][j]; }
+      else if constexpr (J == J_RSUB) { FORV acc[j] = R[K][j] - acc[j]; }
+      else if constexpr (J == J_MUL) { FORV acc[j] = acc[j] * R[K][j]; }
+      else if constexpr (J == J_DIVP) { FORV acc[j] = vmmath::divp_f(acc[j], R[K][j]); }
+      else if constexpr (J == J_RDIVP) { FORV acc[j] = vmmath::divp_f(R[K][j], acc[j]); }
+      else if constexpr (J == J_ADDTO) { FORV R[K][j] += acc[j]; }
+      else if constexpr (J == J_ACCUM) {
+        if (tc.full) { FORV R[K][j] += acc[j]; }
+        else { FORV R[K][j] += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }
+      }
+      else if constexpr (J == J_FMAUR) { const float u_ = U[arg]; FORV acc[j] = fmaf(acc[j], u_, R[K][j]); }
+      else if constexpr (J == J_RTOS) { VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, R[K]) }
+      else if constexpr (J == J_STOR) { VEC_LOAD(R[K], slots + (size_t)arg * NV4 * NT + tid) }
+      else if constexpr (J == J_SPILL) { VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, R[K]) }
+      else if constexpr (J == J_FILL) { VEC_LOAD(R[K], reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) }
+    }
+    else if constexpr (CS == P_LDU) { const float u = U[arg]; FORV acc[j] = u; }
+    else if constexpr (CS == P_ADDU) { const float u = U[arg]; FORV acc[j] += u; }
+    else if constexpr (CS == P_SUBU) { const float u = U[arg]; FORV acc[j] -= u; }
+    else if constexpr (CS == P_RSUBU) { const float u = U[arg]; FORV acc[j] = u - acc[j]; }
+    else if constexpr (CS == P_MULU) { const float u = U[arg]; FORV acc[j] *= u; }
+    else if constexpr (CS == P_DIVPU) { const float u = vmmath::f_rcp(1.f + fabsf(U[arg])); FORV acc[j] *= u; }
+    else if constexpr (CS == P_RDIVPU) { const float u = U[arg]; FORV acc[j] = vmmath::divp_f(u, acc[j]); }
+    else if constexpr (CS == P_FMAU) { const float a = U[arg & 511u], b = U[arg >> 9]; FORV acc[j] = fmaf(acc[j], a, b); }
+    else if constexpr (CS == P_LDS) { VEC_LOAD(acc, slots + (size_t)arg * NV4 * NT + tid) }
+    else if constexpr (CS == P_STS) { VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, acc) }
+    else if constexpr (CS >= P_ADDS && CS <= P_RDIVPS) {
+      float t[V];
+      VEC_LOAD(t, slots + (size_t)arg * NV4 * NT + tid)
+      if constexpr (CS == P_ADDS) { FORV acc[j] += t[j]; }
+      else if constexpr (CS == P_SUBS) { FORV acc[j] -= t[j]; }
+      else if constexpr (CS == P_RSUBS) { FORV acc[j] = t[j] - acc[j]; }
+      else if constexpr (CS == P_MULS) { FORV acc[j] *= t[j]; }
+      else if constexpr (CS == P_DIVPS) { FORV acc[j] = vmmath::divp_f(acc[j], t[j]); }
+      else { FORV acc[j] = vmmath::divp_f(t[j], acc[j]); }
+    }
+    else if constexpr (CS == P_SIN) { FORV acc[j] = vmmath::sin_f(acc[j]); }
+    else if constexpr (CS == P_COS) { FORV acc[j] = vmmath::cos_f(acc[j]); }
+    else if constexpr (CS == P_SINCOS) {
+      float t[V];
+      FORV { float s_, c_; vmmath::sincos_f(acc[j], &s_, &c_); acc[j] = s_; t[j] = c_; }
+      VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, t)
+    }
+    else if constexpr (CS == P_EXPC) { FORV acc[j] = vmmath::exp_clamped10(acc[j]); }
+    else if constexpr (CS == P_TANH) { FORV acc[j] = vmmath::tanh_f(acc[j]); }
+    else if constexpr (CS == P_SIGMOID) { FORV acc[j] = vmmath::sigmoid_f(acc[j]); }
+    else if constexpr (CS == P_RELU) { FORV acc[j] = fmaxf(acc[j], 0.f); }
+    else if constexpr (CS == P_NEG) { FORV acc[j] = -acc[j]; }
+    else if constexpr (CS == P_STEP) { FORV acc[j] = acc[j] > 0.f ? 1.f : 0.f; }
+    else if constexpr (CS == P_CLAMPMASK) { FORV acc[j] = (acc[j] >= -10.f && acc[j] <= 10.f) ? 1.f : 0.f; }
+    else if constexpr (CS == P_ONEMSQ) { FORV acc[j] = fmaf(-acc[j], acc[j], 1.f); }
+    else if constexpr (CS == P_YOMY) { FORV acc[j] = acc[j] * (1.f - acc[j]); }
+    else if constexpr (CS == P_DIVPGB) { FORV acc[j] = vmmath::divp_grad_b(acc[j]); }
+    else if constexpr (CS == P_RBF16) { FORV acc[j] = vmmath::round_bf16(acc[j]); }
+    else if constexpr (CS == P_ROWSUM) {
+      float sum = 0.f;
+      if (tc.full) { FORV sum += acc[j]; }
+      else { FORV sum += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      float* redf = reinterpret_cast<float*>(red);
+      if ((tid & 31) == 0) redf[tid >> 5] = sum;
+      __syncthreads();
+      float tot = 0.f;
+#pragma unroll
+      for (int i = 0; i < NT / 32; ++i) tot += redf[i];
+      __syncthreads();
+      FORV acc[j] = tot;
+    }
+    else if constexpr (CS == P_GLD) { load_operand(p.operand[arg], tc, tid, acc); }
+    else if constexpr (CS == P_GST) { store_operand(p.operand[arg], tc, tid, acc); }
+    else if constexpr (CS == P_FILL) { VEC_LOAD(acc, reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) }
+    else if constexpr (CS == P_SPILL) { VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, acc) }
+  };
+
   int pc = 0;
   uint32_t w = code[0];
   for (;;) {
@@ -219,121 +267,51 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
     ++pc;
     const int cs = w & 1023u;
     const uint32_t arg = w >> 14;
-    switch (cs) {
-      ALL_SLOTS(JOINT_CASES)
-      case P_LDU: { const float u = U[arg]; FORV acc[j] = u; } break;
-      case P_ADDU: { const float u = U[arg]; FORV acc[j] += u; } break;
-      case P_SUBU: { const float u = U[arg]; FORV acc[j] -= u; } break;
-      case P_RSUBU: { const float u = U[arg]; FORV acc[j] = u - acc[j]; } break;
-      case P_MULU: { const float u = U[arg]; FORV acc[j] *= u; } break;
-      case P_DIVPU: { const float u = vmmath::f_rcp(1.f + fabsf(U[arg])); FORV acc[j] *= u; } break;
-      case P_RDIVPU: { const float u = U[arg]; FORV acc[j] = vmmath::divp_f(u, acc[j]); } break;
-      case P_FMAU: { const float a = U[arg & 511u], b = U[arg >> 9]; FORV acc[j] = fmaf(acc[j], a, b); } break;
-      case P_LDS: VEC_LOAD(acc, slots + (size_t)arg * NV4 * NT + tid) break;
-      case P_STS: VEC_STORE(slots + (size_t)arg * NV4 * NT + tid, acc) break;
-      case P_ADDS: case P_SUBS: case P_RSUBS: case P_MULS: case P_DIVPS: case P_RDIVPS: {
-        float t[V];
-        VEC_LOAD(t, slots + (size_t)arg * NV4 * NT + tid)
-        switch (cs) {
-          case P_ADDS: FORV acc[j] += t[j]; break;
-          case P_SUBS: FORV acc[j] -= t[j]; break;
-          case P_RSUBS: FORV acc[j] = t[j] - acc[j]; break;
-          case P_MULS: FORV acc[j] *= t[j]; break;
-          case P_DIVPS: FORV acc[j] = vmmath::divp_f(acc[j], t[j]); break;
-          default: FORV acc[j] = vmmath::divp_f(t[j], acc[j]); break;
-        }
-      } break;
-      case P_SIN: case P_COS: case P_SINCOS: case P_EXPC: case P_TANH: case P_SIGMOID: {
-        // The expensive functions run four lanes at a time in a rolled loop over a per-thread
-        // staging column in shared memory: unrolled over all lanes, their temporaries would not
-        // fit in the register file beside the register slots.
-        VEC_STORE(stage, acc)
-#pragma unroll 1
-        for (int h = 0; h < NV4; ++h) {
-          float4 v = stage[h * NT], c4 = v;
-          switch (cs) {
-            case P_SIN: v.x = vmmath::sin_f(v.x); v.y = vmmath::sin_f(v.y); v.z = vmmath::sin_f(v.z); v.w = vmmath::sin_f(v.w); break;
-            case P_COS: v.x = vmmath::cos_f(v.x); v.y = vmmath::cos_f(v.y); v.z = vmmath::cos_f(v.z); v.w = vmmath::cos_f(v.w); break;
-            case P_SINCOS:
-              vmmath::sincos_f(c4.x, &v.x, &c4.x); vmmath::sincos_f(c4.y, &v.y, &c4.y);
-              vmmath::sincos_f(c4.z, &v.z, &c4.z); vmmath::sincos_f(c4.w, &v.w, &c4.w);
-              slots[((size_t)arg * NV4 + h) * NT + tid] = c4;
-              break;
-            case P_EXPC: v.x = vmmath::exp_clamped10(v.x); v.y = vmmath::exp_clamped10(v.y); v.z = vmmath::exp_clamped10(v.z); v.w = vmmath::exp_clamped10(v.w); break;
-            case P_TANH: v.x = vmmath::tanh_f(v.x); v.y = vmmath::tanh_f(v.y); v.z = vmmath::tanh_f(v.z); v.w = vmmath::tanh_f(v.w); break;
-            default: v.x = vmmath::sigmoid_f(v.x); v.y = vmmath::sigmoid_f(v.y); v.z = vmmath::sigmoid_f(v.z); v.w = vmmath::sigmoid_f(v.w); break;
+    if (cs < P_ULOAD) {
+      dispatch_tree<0, P_ULOAD>(cs, arg, exec);
+    } else {
+      switch (cs) {  // control and once-per-CTA instructions
+        case P_ULOAD: {
+          if (tid == 0) {
+            const Operand& o = p.operand[arg >> 9];
+            U[arg & 511u] = o.dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(o.ptr))
+                                                  : __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(o.ptr)) << 16);
           }
-          stage[h * NT] = v;
-        }
-        VEC_LOAD(acc, stage)
-      } break;
-      case P_RELU: FORV acc[j] = fmaxf(acc[j], 0.f); break;
-      case P_NEG: FORV acc[j] = -acc[j]; break;
-      case P_STEP: FORV acc[j] = acc[j] > 0.f ? 1.f : 0.f; break;
-      case P_CLAMPMASK: FORV acc[j] = (acc[j] >= -10.f && acc[j] <= 10.f) ? 1.f : 0.f; break;
-      case P_ONEMSQ: FORV acc[j] = fmaf(-acc[j], acc[j], 1.f); break;
-      case P_YOMY: FORV acc[j] = acc[j] * (1.f - acc[j]); break;
-      case P_DIVPGB: FORV acc[j] = vmmath::divp_grad_b(acc[j]); break;
-      case P_RBF16: FORV acc[j] = vmmath::round_bf16(acc[j]); break;
-      case P_ROWSUM: {
-        float s = 0.f;
-        if (tc.full) { FORV s += acc[j]; }
-        else { FORV s += (lane_pos(tid, j) < tc.limit) ? acc[j] : 0.f; }
+        } break;
+        case P_UCONST: {
+          if (tid == 0) U[arg] = __uint_as_float(wn);
+          ++pc;
+          wn = code[pc];
+        } break;
+        case P_LOOP_BEGIN:
+          __syncthreads();  // uniforms written by thread 0 are visible from here on
+          loop_pc = pc;
+          break;
+        case P_LOOP_END:
+          tile += gridDim.x;
+          if (tile < ntiles) { set_tile(); pc = loop_pc; wn = code[pc]; }
+          break;
+        case P_COLOUT: {
+          float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
+          FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = acc[j]; }
+        } break;
+        case P_SCALOUT: {
+          double sum = 0.0;
+          FORV sum += (double)acc[j];
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        float* redf = reinterpret_cast<float*>(red);
-        if ((tid & 31) == 0) redf[tid >> 5] = s;
-        __syncthreads();
-        float tot = 0.f;
-#pragma unroll
-        for (int i = 0; i < NT / 32; ++i) tot += redf[i];
-        __syncthreads();
-        FORV acc[j] = tot;
-      } break;
-      case P_GLD: load_operand(p.operand[arg], tc, tid, acc); break;
-      case P_GST: store_operand(p.operand[arg], tc, tid, acc); break;
-      case P_FILL: VEC_LOAD(acc, reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) break;
-      case P_SPILL: VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, acc) break;
-      case P_ULOAD: {
-        if (tid == 0) {
-          const Operand& o = p.operand[arg >> 9];
-          U[arg & 511u] = o.dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(o.ptr))
-                                                : __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(o.ptr)) << 16);
-        }
-      } break;
-      case P_UCONST: {
-        if (tid == 0) U[arg] = __uint_as_float(wn);
-        ++pc;
-        wn = code[pc];
-      } break;
-      case P_LOOP_BEGIN:
-        __syncthreads();  // uniforms written by thread 0 are visible from here on
-        loop_pc = pc;
-        break;
-      case P_LOOP_END:
-        tile += gridDim.x;
-        if (tile < ntiles) { set_tile(); pc = loop_pc; wn = code[pc]; }
-        break;
-      case P_COLOUT: {
-        float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
-        FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = acc[j]; }
-      } break;
-      case P_SCALOUT: {
-        double s = 0.0;
-        FORV s += (double)acc[j];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-        if ((tid & 31) == 0) red[tid >> 5] = s;
-        __syncthreads();
-        if (tid == 0) {
-          double tot = 0.0;
-          for (int i = 0; i < NT / 32; ++i) tot += red[i];
-          p.scalpart[(size_t)arg * gridDim.x + blockIdx.x] = tot;
-        }
-        __syncthreads();
-      } break;
-      default:  // P_END and anything unknown
-        return;
+          for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+          if ((tid & 31) == 0) red[tid >> 5] = sum;
+          __syncthreads();
+          if (tid == 0) {
+            double tot = 0.0;
+            for (int i = 0; i < NT / 32; ++i) tot += red[i];
+            p.scalpart[(size_t)arg * gridDim.x + blockIdx.x] = tot;
+          }
+          __syncthreads();
+        } break;
+        default:  // P_END and anything unknown
+          return;
+      }
     }
     w = wn;
   }
@@ -371,7 +349,7 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
 }
 
 size_t vm_smem_bytes(int n_code, int n_smem_slots) {
-  return (size_t)((n_code + 3) & ~3) * 4 + kMaxUniforms * 4 + 64 * 8 + (size_t)(n_smem_slots + 1) * NV4 * NT * 16;
+  return (size_t)((n_code + 3) & ~3) * 4 + kMaxUniforms * 4 + 64 * 8 + (size_t)n_smem_slots * NV4 * NT * 16;
 }
 
 }  // namespace vm
