@@ -1,14 +1,291 @@
-// InnerProduct contraction C[M,N] = A[M,K] * B[N,K]^T (bf16 operands, fp32 accumulate).
+// InnerProduct contraction C[M,N] = A[M,K] * B[N,K]^T: bf16 operands, fp32 accumulation in
+// tensor memory, fp32 or bf16 output.  Hand-written for sm_100a:
+//   - operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
+//     ring of shared-memory stages guarded by full/empty mbarriers;
+//   - one elected thread issues tcgen05.mma (cta_group::1, kind::f16, 128 x kTileN x 16) with the
+//     accumulator in TMEM; tcgen05.commit releases stages and finally signals the epilogue;
+//   - four epilogue warps read their 32-lane TMEM quadrants with tcgen05.ld and write C.
+// Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
+// warps 2..5 = epilogue.  Every mbarrier wait is bounded by a clock budget; when it runs out
+// the kernel records DRAGON_ERR_TIMEOUT in the status word, stops issuing work, frees its TMEM
+// and returns.
+#include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdint>
+#include <map>
+#include <mutex>
+
 #include "plan.h"
+#include "vm_math.h"
 
 namespace dragon {
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kTileN = 128;
+constexpr int kTileK = 64;          // one 128-byte swizzle row of bf16
+constexpr int kStages = 6;
+constexpr int kUmmaK = 16;
+constexpr int kGemmThreads = 192;
+constexpr uint32_t kStageBytesA = kTileM * kTileK * 2;
+constexpr uint32_t kStageBytesB = kTileN * kTileK * 2;
+constexpr uint32_t kStageBytes = kStageBytesA + kStageBytesB;
+constexpr size_t kGemmSmem = 1024 /*alignment slack*/ + (size_t)kStages * kStageBytes + 256 /*barriers*/;
+constexpr long long kWaitBudgetCycles = 4000000000LL;   // about two seconds
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.b32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+  return ok != 0;
+}
+// bounded wait: false when the clock budget ran out (the caller records the failure and unwinds)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try_wait(bar, parity)) return true;
+  const long long t0 = clock64();
+  for (;;) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (clock64() - t0 > kWaitBudgetCycles) return false;
+  }
+}
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+// shared-memory matrix descriptor: K-major tile, 128-byte swizzle, 8-row groups 1024 bytes apart
+__device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);          // start address
+  d |= (uint64_t)1 << 16;                            // leading byte offset (unused for swizzled K-major)
+  d |= (uint64_t)(1024 >> 4) << 32;                  // stride byte offset
+  d |= (uint64_t)1 << 46;                            // descriptor version of this architecture
+  d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
+  return d;
+}
+// instruction descriptor: D = f32, A = B = bf16, both K-major, M x N
+constexpr uint32_t make_idesc(int m, int n) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+
+struct GemmArgs {
+  void* C;
+  int c_dtype;
+  int M, N, K;
+  int* status;
+};
+
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
+  extern __shared__ unsigned char gemm_smem_raw[];
+  const uint32_t raw = smem_u32(gemm_smem_raw);
+  const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned operand stages
+  unsigned char* tiles_ptr = gemm_smem_raw + (tiles - raw);
+  uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + (size_t)kStages * kStageBytes);
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages, bar_accum = bar_empty + 8 * kStages;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * kTileN;
+  const int k_tiles = (g.K + kTileK - 1) / kTileK;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
+    mbar_init(bar_accum, 1);
+    abort_flag[0] = 0;
+    abort_flag[1] = 0;   // a flag nobody sets, for waits that must not be cut short
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {  // TMEM: kTileN fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    if (lane == 0) {  // TMA producer
+      int issued = 0;
+      for (int kt = 0; kt < k_tiles; ++kt) {
+        const int s = kt % kStages, it = kt / kStages;
+        if (!mbar_wait(bar_empty + 8 * s, (it & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); break; }
+        mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+        const uint32_t dst = tiles + (uint32_t)s * kStageBytes;
+        tma_load_2d(dst, &tmap_a, kt * kTileK, m0, bar_full + 8 * s);
+        tma_load_2d(dst + kStageBytesA, &tmap_b, kt * kTileK, n0, bar_full + 8 * s);
+        issued = kt + 1;
+      }
+      if (*abort_flag) {  // let the copies that are still in flight land before the CTA goes away
+        for (int kt = issued > kStages ? issued - kStages : 0; kt < issued; ++kt)
+          mbar_wait(bar_full + 8 * (kt % kStages), (kt / kStages) & 1, abort_flag + 1 /* never set */);
+      }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {  // MMA issuer
+      constexpr uint32_t idesc = make_idesc(kTileM, kTileN);
+      bool ok = true;
+      for (int kt = 0; kt < k_tiles && ok; ++kt) {
+        const int s = kt % kStages, it = kt / kStages;
+        if (!mbar_wait(bar_full + 8 * s, it & 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = tiles + (uint32_t)s * kStageBytes, b_addr = a_addr + kStageBytesA;
+        const uint64_t a_desc = make_smem_desc(a_addr), b_desc = make_smem_desc(b_addr);
+#pragma unroll
+        for (int k = 0; k < kTileK / kUmmaK; ++k) {
+          // advancing 16 elements along K inside the swizzle row = 32 bytes = 2 descriptor units
+          umma_f16(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+        }
+        umma_commit(bar_empty + 8 * s);   // the stage is free once these MMAs have read it
+      }
+      if (ok) umma_commit(bar_accum);     // accumulator complete
+    }
+  } else {
+    // epilogue: warp w owns TMEM lanes 32*(w%4) .. +31, i.e. rows m0 + 32*(w%4) + lane
+    const int q = warp & 3;
+    const bool ok = mbar_wait(bar_accum, 0, abort_flag);
+    if (!ok && lane == 0) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); }
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int row = m0 + q * 32 + lane;
+    if (ok) {
+#pragma unroll 1
+      for (int c = 0; c < kTileN; c += 32) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (row < g.M) {
+          const int col0 = n0 + c;
+          if (g.c_dtype == DRAGON_F32) {
+            float* out = reinterpret_cast<float*>(g.C) + (size_t)row * g.N + col0;
+            if ((g.N & 3) == 0 && col0 + 32 <= g.N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4)
+                *reinterpret_cast<float4*>(out + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < g.N) out[j] = __uint_as_float(v[j]);
+            }
+          } else {
+            unsigned short* out = reinterpret_cast<unsigned short*>(g.C) + (size_t)row * g.N + col0;
+            if ((g.N & 7) == 0 && col0 + 32 <= g.N) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 8) {
+                uint4 pk;
+                pk.x = vmmath::bf16_bits(__uint_as_float(v[j])) | (vmmath::bf16_bits(__uint_as_float(v[j + 1])) << 16);
+                pk.y = vmmath::bf16_bits(__uint_as_float(v[j + 2])) | (vmmath::bf16_bits(__uint_as_float(v[j + 3])) << 16);
+                pk.z = vmmath::bf16_bits(__uint_as_float(v[j + 4])) | (vmmath::bf16_bits(__uint_as_float(v[j + 5])) << 16);
+                pk.w = vmmath::bf16_bits(__uint_as_float(v[j + 6])) | (vmmath::bf16_bits(__uint_as_float(v[j + 7])) << 16);
+                *reinterpret_cast<uint4*>(out + j) = pk;
+              }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 32; ++j)
+                if (col0 + j < g.N) out[j] = (unsigned short)vmmath::bf16_bits(__uint_as_float(v[j]));
+            }
+          }
+        }
+      }
+    }
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTileN) : "memory");
+  }
+}
+
+// ---- host side ---------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess && q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// row-major bf16 [rows, cols] viewed as a 2-D tensor map with boxes of box_rows x 64 elements
+bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+  cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
 
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, int* status, cudaStream_t st) {
-  (void)A; (void)B; (void)C; (void)c_dtype; (void)M; (void)N; (void)K; (void)status; (void)st;
-  set_error("InnerProduct: the tensor-core contraction is not built into this library yet");
-  return DRAGON_ERR_UNSUPPORTED;
+  if (M <= 0 || N <= 0 || K <= 0 || (K & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
+    set_error("InnerProduct: K must be a multiple of 8 and all operands 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
+    return DRAGON_ERR_UNSUPPORTED;
+  }
+  CUtensorMap ta, tb;
+  if (!make_tmap(&ta, A, M, K, kTileM) || !make_tmap(&tb, B, N, K, kTileN)) {
+    set_error("InnerProduct: cannot encode the TMA descriptors (no CUDA driver?)");
+    return DRAGON_ERR_CUDA;
+  }
+  static std::once_flag once;
+  static cudaError_t attr_err = cudaSuccess;
+  std::call_once(once, [] { attr_err = cudaFuncSetAttribute(gemm_bf16_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem); });
+  if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
+  GemmArgs g{C, c_dtype, M, N, K, status};
+  dim3 grid((N + kTileN - 1) / kTileN, (M + kTileM - 1) / kTileM);
+  gemm_bf16_tcgen05<<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, g);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) { set_error("InnerProduct: launch failed: %s", cudaGetErrorString(e)); return DRAGON_ERR_CUDA; }
+  return DRAGON_OK;
 }
 
 }  // namespace dragon

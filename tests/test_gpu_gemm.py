@@ -1,0 +1,84 @@
+"""GPU parity of the tensor-core contraction and of the whole two-layer graph (InnerProduct, BiasAdd,
+ReLU, SoftmaxCrossEntropy, forward + backward) against the oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import interp
+from paper_1707_08265_b200 import workloads as wl
+from test_gpu_vm import run_gpu, check, TOLBF, TOL32
+
+pytestmark = pytest.mark.gpu
+
+
+def bf16able(a):
+    return torch.from_numpy(a.astype(np.float32)).to(torch.bfloat16).float().numpy()
+
+
+@pytest.mark.parametrize("m,n,k,dt", [(128, 128, 64, "f32"), (128, 128, 512, "f32"), (256, 384, 448, "bf16"),
+                                      (200, 136, 72, "f32"), (1, 8, 8, "f32"), (300, 520, 1000, "bf16"),
+                                      (1024, 1024, 2048, "f32")])
+def test_inner_product_forward(m, n, k, dt):
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16")
+    Y = gd.op("InnerProduct", [X, W], "Y", [m, n], dt)
+    rng = np.random.default_rng(m + n + k)
+    x = bf16able(rng.standard_normal((m, k))); w = bf16able(rng.standard_normal((n, k)) / np.sqrt(k))
+    (got,), f = run_gpu(gd.desc, [X, W], [Y], [x, w])
+    (ref,) = interp.run_function(gd.desc, [X, W], [Y], [x, w])
+    # fp32 accumulation of exact bf16 products: far inside the bf16-contraction tolerance
+    check(got, ref, TOLBF if dt == "bf16" else 2e-5, "Y")
+    # a transposed or shifted operand would not survive this: one-hot weights pick columns of X
+    if n <= k:
+        sel = np.zeros((n, k), dtype=np.float32)
+        sel[np.arange(n), (np.arange(n) * 7) % k] = 1
+        (got,), _ = run_gpu(gd.desc, [X, W], [Y], [x, sel])
+        assert np.array_equal(got, x[:, (np.arange(n) * 7) % k].astype(np.float64))
+
+
+@pytest.mark.parametrize("m,n,k", [(128, 128, 128), (96, 40, 72), (512, 256, 320)])
+def test_inner_product_gradients(m, n, k):
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); G = gd.tensor("G", [m, n], "f32")
+    Y = gd.op("InnerProduct", [X, W], "Y", [m, n], "f32")
+    obj = gd.op("Mul", [Y, G], "obj")
+    dX, dW = gd.grad([obj], [X, W])
+    rng = np.random.default_rng(k)
+    feeds = [bf16able(rng.standard_normal((m, k))), bf16able(rng.standard_normal((n, k))), bf16able(rng.standard_normal((m, n)))]
+    got, f = run_gpu(gd.desc, [X, W, G], [dX, dW], feeds)
+    ref = interp.run_function(gd.desc, [X, W, G], [dX, dW], feeds)
+    check(got[0], ref[0], 1e-4, "dX")
+    check(got[1], ref[1], 1e-4, "dW")
+
+
+def mlp_case(batch, d_in, d_hid, d_out, seed):
+    g, ids = wl.mlp(batch, d_in, d_hid, d_out)
+    feeds = list(wl.mlp_feeds(batch, d_in, d_hid, d_out, seed))
+    inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
+    outs = [ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")]
+    return g, ids, inputs, outs, feeds
+
+
+@pytest.mark.parametrize("shape", [(128, 128, 128, 128), (256, 192, 320, 136), (1024, 512, 512, 1000)])
+def test_mlp_forward_backward(shape):
+    g, ids, inputs, outs, feeds = mlp_case(*shape, seed=wl.BASE_SEED + 4)
+    got, f = run_gpu(g.desc, inputs, outs, feeds)
+    assert f.used_inputs() == [1] * 6 and f.marked()[ids["side"]] == 0       # Tanh(X) pruned
+    assert f.describe().count("gemm") == 5                                     # no dX of layer 1
+    ref = interp.run_function(g.desc, inputs, outs, feeds)
+    for gv, rv, name in zip(got, ref, ("loss", "dW1", "db1", "dW2", "db2")):
+        check(gv, rv, TOLBF, name)
+        scale = np.max(np.abs(rv))
+        assert np.max(np.abs(gv - rv)) <= 0.03 * scale + 1e-12, (name, np.max(np.abs(gv - rv)), scale)
+
+
+def test_mlp_out_of_range_label_sets_status_and_does_not_fault():
+    g, ids, inputs, outs, feeds = mlp_case(128, 128, 128, 128, seed=3)
+    feeds[5] = feeds[5].copy(); feeds[5][7] = 4096
+    from paper_1707_08265_b200 import binding as B
+    from test_gpu_vm import to_dev
+    fn = B.Graph.from_desc(g.desc).function(inputs, outs)
+    dev = [to_dev(a, g.desc["tensors"][i]["dtype"]) for i, a in zip(inputs, feeds)]
+    o = [torch.empty(tuple(g.shape(t)), dtype=torch.float32, device="cuda") for t in outs]
+    fn.run_torch(dev, o)
+    assert fn.status() == B.ERR_INVALID_ARG
