@@ -222,7 +222,12 @@ struct Lowerer {
         int mdY = materialise(dy, DRAGON_BF16, DRAGON_BF16);
         if (want[0]) {  // dX[M,K] = dY[M,N] * W[N,K]
           int mW = materialise(in(1), DRAGON_BF16, DRAGON_BF16);
-          int mC = gemm(mdY, transpose_of(mW), MEM_WORK, -1, g.tensors[op.in[0]].dtype == DRAGON_BF16 ? DRAGON_BF16 : DRAGON_F32);
+          // the gradient of a bf16 activation is kept in bf16 (it feeds the next contraction);
+          // a gradient that the caller asked for stays fp32
+          const auto& wr = g.stages[s].wrts;
+          const bool wanted = std::find(wr.begin(), wr.end(), op.in[0]) != wr.end();
+          int mC = gemm(mdY, transpose_of(mW), MEM_WORK, -1,
+                        (g.tensors[op.in[0]].dtype == DRAGON_BF16 && !wanted) ? DRAGON_BF16 : DRAGON_F32);
           add(0, new_val(VK_MEM, plan->mems[mC].shape, mC));
         }
         if (want[1]) {  // dW[N,K] = dY^T[N,M] * X[M,K]
