@@ -165,6 +165,31 @@ int dragon_function_profile_read(dragon_function_t* f, double* total_ms, int* ru
  * DRAGON_ERR_TIMEOUT (a bounded wait gave up) or DRAGON_ERR_INVALID_ARG (bad label). */
 int dragon_function_status(dragon_function_t* f);
 
+/* Mean softmax cross-entropy loss without any allocation.  The paper has no counterpart: this is
+ * a convenience of this library for callers that cannot give it a workspace.
+ *
+ * Who needs it: code that runs where device memory cannot be requested -- a plug-in inside a host
+ * application whose own pool already owns the whole GPU (a cudaMalloc from the plug-in would fail,
+ * or take memory the pool counts on), or a latency-bound loop that cannot afford the device-wide
+ * synchronisation an allocation or a free may imply.  Such a caller cannot use dragon_run(), which
+ * wants a caller-provided workspace and uploads instruction streams on first use.
+ *
+ * Computes  loss_out[0] = -(1/rows) * sum_m log softmax(logits[m,:])[labels[m]]  exactly like the
+ * SOFTMAX_CROSS_ENTROPY operator (same kernels).  logits: device, row-major [rows, cols], dtype
+ * DRAGON_F32 or DRAGON_BF16; labels: device int32[rows]; loss_out: device float[1]; all owned by
+ * the caller.  The per-row partial losses live in a fixed array inside the library image
+ * (257 KiB per GPU, held from library load to process exit), which limits rows to 65536:
+ * larger inputs are rejected with DRAGON_ERR_WORKSPACE.  The call allocates and frees nothing
+ * and is asynchronous on cuda_stream.
+ *
+ * The first call on each device looks up the array's device address (a one-time set-up under
+ * the current device); make that first call outside any stream capture.  All calls on a device
+ * share the one array: it keeps the previous call's contents (the function clears what has to
+ * start at zero), and two calls that overlap on the GPU -- different streams, no ordering --
+ * race on it and give wrong results.  An out-of-range label contributes 0, as in the operator. */
+int dragon_softmax_ce_loss_static(const void* logits, int dtype, const int32_t* labels, int rows, int cols,
+                                  float* loss_out, void* cuda_stream);
+
 /* Host instantiation of the VM's elementary functions (fn: DRAGON_OP_SIN, _EXP, _TANH,
  * _SIGMOID; DRAGON_OP_DIV evaluates 1/(1+|x|); 100 + DRAGON_OP_SIN evaluates the cosine),
  * for accuracy sweeps on machines without a GPU.  x, y: host arrays of n floats. */

@@ -48,6 +48,7 @@ _SIGNATURES = {
                                    _c.c_size_t, _c.c_void_p]),
     "dragon_function_profile": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_int]),
     "dragon_function_profile_read": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_double), _c.POINTER(_c.c_int)]),
+    "dragon_softmax_ce_loss_static": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_int, _c.c_int, _c.c_void_p, _c.c_void_p]),
     "dragon_host_math": (_c.c_int, [_c.c_int, _c.POINTER(_c.c_float), _c.POINTER(_c.c_float), _c.c_int]),
     "dragon_last_error": (_c.c_char_p, []),
 }
@@ -263,6 +264,13 @@ class Function:
         self.ensure_workspace()
         s = stream if stream is not None else torch.cuda.current_stream()
         self.run([0 if t is None else t.data_ptr() for t in feeds], [t.data_ptr() for t in fetches], s.cuda_stream)
+
+
+def softmax_ce_loss_static(logits_ptr, dtype, labels_ptr, rows, cols, loss_ptr, stream=0):
+    """dragon_softmax_ce_loss_static: allocation-free mean cross-entropy (device pointers)."""
+    r = lib().dragon_softmax_ce_loss_static(logits_ptr, dtype, labels_ptr, rows, cols, loss_ptr, stream)
+    if r < 0:
+        raise DragonError(r, "dragon_softmax_ce_loss_static")
 
 
 def host_math(fn, x):

@@ -115,4 +115,58 @@ cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cu
   return cudaGetLastError();
 }
 
+// ---- allocation-free loss ------------------------------------------------------------------------
+
+// Scratch of dragon_softmax_ce_loss_static(): one partial loss per row plus a status word.  It is
+// part of the library image, so every GPU that loads the library holds these 257 KiB until exit.
+constexpr int kStaticMaxRows = 65536;
+static __device__ __align__(256) float g_static_rowloss[kStaticMaxRows + 64];
+
+namespace {
+// device address of the scratch array, looked up once per device (index = CUDA device ordinal)
+float* static_scratch_for_current_device(int* err) {
+  static float* cache[64] = {};
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = DRAGON_ERR_CUDA; return nullptr; }
+  if (!cache[dev]) {
+    // in host code the array's name is only a handle; the kernels need the address on this device
+    float* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_static_rowloss);
+    if (e != cudaSuccess || !ptr) {
+      set_error("dragon_softmax_ce_loss_static: cudaGetSymbolAddress failed: %s", cudaGetErrorString(e));
+      *err = DRAGON_ERR_CUDA;
+      return nullptr;
+    }
+    cache[dev] = ptr;
+  }
+  return cache[dev];
+}
+}  // namespace
+
 }  // namespace dragon
+
+extern "C" int dragon_softmax_ce_loss_static(const void* logits, int dtype, const int32_t* labels, int rows, int cols,
+                                             float* loss_out, void* cuda_stream) {
+  using namespace dragon;
+  if (!logits || !labels || !loss_out || rows <= 0 || cols <= 0 || (dtype != DRAGON_F32 && dtype != DRAGON_BF16)) {
+    set_error("dragon_softmax_ce_loss_static: bad argument");
+    return DRAGON_ERR_INVALID_ARG;
+  }
+  if (rows > kStaticMaxRows) {
+    set_error("dragon_softmax_ce_loss_static: %d rows exceed the built-in scratch (at most %d rows)", rows, kStaticMaxRows);
+    return DRAGON_ERR_WORKSPACE;
+  }
+  int err = DRAGON_OK;
+  float* scratch = static_scratch_for_current_device(&err);
+  if (!scratch) return err;
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  int* status = reinterpret_cast<int*>(scratch + kStaticMaxRows);
+  // the status word must start at zero; the per-row losses are overwritten in full by every call
+  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
+  if (e == cudaSuccess) e = launch_sce_fwd(logits, dtype, labels, rows, cols, scratch, loss_out, status, st);
+  if (e != cudaSuccess) {
+    set_error("dragon_softmax_ce_loss_static: CUDA error: %s", cudaGetErrorString(e));
+    return DRAGON_ERR_CUDA;
+  }
+  return DRAGON_OK;
+}
