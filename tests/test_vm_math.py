@@ -1,0 +1,50 @@
+"""Accuracy sweep of the VM's elementary functions (host instantiation of csrc/vm_math.h, reached
+through dragon_host_math) against fp64.  The device build differs only in the reciprocal
+(rcp.approx, about one ulp); the polynomials, reductions and constants are the same code."""
+import numpy as np
+
+from paper_1707_08265_b200 import binding as B
+
+SIN, COS = B.OPS["Sin"], 100 + B.OPS["Sin"]
+
+
+def rel(y, r):
+    return np.abs(y.astype(np.float64) - r) / np.maximum(np.abs(r), 1e-300)
+
+
+def test_sin_cos_small_and_medium_arguments():
+    x = np.concatenate([np.linspace(-100, 100, 1_000_001), np.linspace(-1e-3, 1e-3, 10001), [0.0, -0.0]]).astype(np.float32)
+    xd = x.astype(np.float64)
+    for fn, ref in ((SIN, np.sin), (COS, np.cos)):
+        y, r = B.host_math(fn, x), ref(xd)
+        assert np.max(np.abs(y - r)) < 1.5e-7
+        big = np.abs(r) > 1e-3
+        assert np.max(rel(y, r)[big]) < 2.5e-7            # about two ulp
+    tiny = np.float32([1e-30, -3e-20, 1e-10])
+    assert np.array_equal(B.host_math(SIN, tiny), tiny)      # sin x = x to the last bit near zero
+    x = (np.float32(10) ** np.linspace(2, 5, 300001)).astype(np.float32)
+    for fn, ref in ((SIN, np.sin), (COS, np.cos)):
+        assert np.max(np.abs(B.host_math(fn, x) - ref(x.astype(np.float64)))) < 3e-7
+
+
+def test_sin_cos_huge_arguments_stay_bounded():
+    # beyond 2^22 the spacing of fp32 numbers exceeds 0.25: only boundedness and NaN behaviour are promised
+    x = (np.float32(10) ** np.linspace(5, 7.3, 100001)).astype(np.float32)
+    for fn, ref in ((SIN, np.sin), (COS, np.cos)):
+        assert np.max(np.abs(B.host_math(fn, x) - ref(x.astype(np.float64)))) < 1e-3
+    y = B.host_math(SIN, np.float32([1e30, np.inf, -np.inf, np.nan]))
+    assert y[0] == 0 and np.all(np.isnan(y[1:]))
+
+
+def test_exp_tanh_sigmoid_div():
+    x = np.linspace(-12, 12, 1_000_001).astype(np.float32)
+    assert np.max(rel(B.host_math(B.OPS["Exp"], x), np.exp(np.clip(x.astype(np.float64), -10, 10)))) < 2e-7
+    x = np.concatenate([np.linspace(-20, 20, 1_000_001), np.linspace(-1e-3, 1e-3, 10001)]).astype(np.float32)
+    r = np.tanh(x.astype(np.float64))
+    assert np.max(rel(B.host_math(B.OPS["Tanh"], x), r)[r != 0]) < 3e-7
+    x = np.linspace(-80, 80, 1_000_001).astype(np.float32)
+    assert np.max(rel(B.host_math(B.OPS["Sigmoid"], x), 1 / (1 + np.exp(-x.astype(np.float64))))) < 3e-7
+    y = B.host_math(B.OPS["Sigmoid"], np.float32([-200, 200]))
+    assert y[0] < 1e-37 and y[1] == 1
+    x = np.linspace(-50, 50, 100001).astype(np.float32)
+    assert np.max(rel(B.host_math(B.OPS["Div"], x), 1 / (1 + np.abs(x.astype(np.float64))))) < 2e-7
