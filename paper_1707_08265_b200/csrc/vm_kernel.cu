@@ -13,6 +13,9 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
+#include <mutex>
+#include <string>
 #include <type_traits>
 
 #include "plan.h"
@@ -177,9 +180,7 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
   // slots are named statically.
   auto exec = [&](auto cs_tag, const uint32_t arg) {
     constexpr int CS = decltype(cs_tag)::value;
-#ifdef DRAGON_VM_EXPERIMENT_MINIMAL
-    if constexpr (!(CS == P_RELU || CS == P_GLD || CS == P_GST || CS / kJointStride == J_ADD || CS / kJointStride == J_STR)) { return; } else
-#endif
+    asm volatile("// VMLEAF %0" ::"n"(CS));   // marks the leaf for the jump-table build step
     if constexpr (CS < kFirstPlain) {
       constexpr int J = CS / kJointStride, K = CS % kJointStride;
       if constexpr (J == J_LDR) { FORV acc[j] = R[K][j]; }
@@ -268,6 +269,7 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
     const int cs = w & 1023u;
     const uint32_t arg = w >> 14;
     if (cs < P_ULOAD) {
+      asm volatile("// VMDISPATCH %0" ::"r"(cs));   // the build step puts an indexed jump here
       dispatch_tree<0, P_ULOAD>(cs, arg, exec);
     } else {
       switch (cs) {  // control and once-per-CTA instructions
@@ -354,13 +356,44 @@ size_t vm_smem_bytes(int n_code, int n_smem_slots) {
 
 }  // namespace vm
 
+}  // namespace dragon
+
+// cubin of this same kernel with the dispatch tree replaced by one indexed jump (build step
+// ptx_jumptable.py); size 0 when that step refused
+extern "C" const unsigned long dragon_vm_jt_cubin_size;
+extern "C" const unsigned char dragon_vm_jt_cubin[];
+
+namespace dragon {
+
+// the kernel to launch: the jump-table build when it is there (and DRAGON_VM_DISPATCH != "tree"),
+// else the compiled-in tree kernel
+static const void* vm_entry() {
+  static const void* entry = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    entry = reinterpret_cast<const void*>(vm::vm_kernel);
+    const char* mode = std::getenv("DRAGON_VM_DISPATCH");
+    if (dragon_vm_jt_cubin_size == 0 || (mode && std::string(mode) == "tree")) return;
+    cudaLibrary_t lib;
+    cudaKernel_t k;
+    if (cudaLibraryLoadData(&lib, dragon_vm_jt_cubin, nullptr, nullptr, 0, nullptr, nullptr, 0) == cudaSuccess &&
+        cudaLibraryGetKernel(&k, lib, "_ZN6dragon2vm9vm_kernelENS0_6ParamsE") == cudaSuccess) {
+      entry = reinterpret_cast<const void*>(k);
+    } else {
+      cudaGetLastError();
+    }
+  });
+  return entry;
+}
+
 // launch helpers used by api.cu
 cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, cudaStream_t st) {
   const size_t smem = vm::vm_smem_bytes(p.n_code, n_smem_slots);
-  cudaError_t e = cudaFuncSetAttribute(vm::vm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+  const void* entry = vm_entry();
+  cudaError_t e = cudaFuncSetAttribute(entry, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
   if (e != cudaSuccess) return e;
-  vm::vm_kernel<<<grid, vm::NT, smem, st>>>(p);
-  return cudaGetLastError();
+  void* args[] = {const_cast<vm::Params*>(&p)};
+  return cudaLaunchKernel(entry, dim3(grid), dim3(vm::NT), args, smem, st);
 }
 
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st) {

@@ -1,0 +1,119 @@
+"""Build step: turns the VM kernel's dispatch tree into one indexed jump.
+
+nvcc emits no indexed branch for a C++ switch, so vm_kernel.cu dispatches through a balanced tree
+of compares.  Its PTX carries two kinds of markers (comments written by inline asm):
+``// VMDISPATCH %r<N>`` where the case id is known, and ``// VMLEAF <id>`` at the top of the code
+of every case.  This script gives every leaf block a label, checks that the tree between the
+dispatch point and the leaves consists of compares and branches only (so that skipping it skips
+no work; otherwise it refuses and the library keeps the tree), and replaces the dispatch point by
+``brx.idx`` over a ``.branchtargets`` table.  The result is assembled with ptxas and loaded at
+run time; the compiled-in tree kernel stays as the fallback.
+"""
+import re
+import sys
+
+LABEL = re.compile(r"^\s*(\$?[A-Za-z_][\w$]*):\s*$")
+BRANCH = re.compile(r"^\s*(@!?%p\d+\s+)?(bra(\.uni)?|brx\.idx|ret|exit|trap)\b")
+# compares, branches, and integer arithmetic on the case id (the compiler narrows and offsets it)
+TREE_OK = re.compile(r"^\s*(@!?%p\d+\s+)?(setp\.|bra\b|bra\.uni\b|cvt\.[us]\d+\.[us]\d+\s|and\.b(16|32)\s|(add|sub)\.s(16|32)\s|shr\.[us]32\s)")
+
+
+def rewrite(ptx, kernel_substr="vm_kernel"):
+    lines = ptx.split("\n")
+    # body of the kernel entry
+    start = next(i for i, l in enumerate(lines) if ".entry" in l and kernel_substr in l)
+    depth, body_lo, body_hi = 0, None, None
+    for i in range(start, len(lines)):
+        depth += lines[i].count("{") - lines[i].count("}")
+        if body_lo is None and "{" in lines[i]:
+            body_lo = i
+        if body_lo is not None and depth == 0:
+            body_hi = i
+            break
+    disp = [i for i in range(body_lo, body_hi) if "// VMDISPATCH" in lines[i]]
+    if len(disp) != 1:
+        raise RuntimeError("expected one dispatch marker, found %d" % len(disp))
+    disp = disp[0]
+    reg = re.search(r"VMDISPATCH\s+(%r\d+)", lines[disp]).group(1)
+    leaves = {}
+    for i in range(body_lo, body_hi):
+        m = re.search(r"// VMLEAF (\d+)", lines[i])
+        if m:
+            n = int(m.group(1))
+            if n in leaves:
+                raise RuntimeError("leaf %d appears twice" % n)
+            leaves[n] = i
+    n_leaves = max(leaves) + 1
+    if sorted(leaves) != list(range(n_leaves)):
+        raise RuntimeError("leaf ids are not dense")
+
+    def is_code(l):
+        s = l.strip()
+        return bool(s) and not s.startswith("//") and not s.startswith(".") and not LABEL.match(l) and s not in ("{", "}")
+
+    # label of the basic block that holds each leaf marker (insert one when the block is a fall-through)
+    inserts = {}          # line index -> label to insert before that line
+    leaf_label = {}
+    for n, at in leaves.items():
+        j = at - 1
+        while True:
+            if LABEL.match(lines[j]):
+                leaf_label[n] = LABEL.match(lines[j]).group(1)
+                break
+            if is_code(lines[j]) and BRANCH.match(lines[j]):
+                lab = "VMLEAF_%d" % n
+                inserts[j + 1] = lab
+                leaf_label[n] = lab
+                break
+            j -= 1
+            if j <= body_lo:
+                raise RuntimeError("no block start for leaf %d" % n)
+    # safety: from the dispatch marker to every leaf block only compares and branches may run
+    label_at = {LABEL.match(lines[i]).group(1): i for i in range(body_lo, body_hi) if LABEL.match(lines[i])}
+    leaf_starts = set()
+    for n, at in leaves.items():
+        j = at
+        while not (LABEL.match(lines[j]) or (is_code(lines[j]) and BRANCH.match(lines[j]))):
+            j -= 1
+        leaf_starts.add(j if LABEL.match(lines[j]) else j + 1)
+    seen, work = set(), [disp + 1]
+    while work:
+        i = work.pop()
+        if i in seen:
+            continue
+        seen.add(i)
+        while True:
+            if i in leaf_starts:
+                break
+            l = lines[i]
+            if "// VMLEAF" in l:
+                break
+            if is_code(l):
+                if not TREE_OK.match(l):
+                    raise RuntimeError("dispatch tree holds other work: %r (line %d)" % (l.strip(), i))
+                m = re.search(r"bra(\.uni)?\s+(\$?[\w$]+);", l)
+                if m:
+                    work.append(label_at[m.group(2)])
+                    if not l.strip().startswith("@"):
+                        break        # unconditional: no fall-through
+            i += 1
+            if i >= body_hi:
+                raise RuntimeError("ran off the kernel body while checking the tree")
+    # rewrite
+    out = []
+    for i, l in enumerate(lines):
+        if i in inserts:
+            out.append(inserts[i] + ":")
+        if i == disp:
+            out.append("\tVMJT: .branchtargets " + ", ".join(leaf_label[n] for n in range(n_leaves)) + ";")
+            out.append("\tbrx.idx " + reg + ", VMJT;")
+            continue
+        out.append(l)
+    return "\n".join(out), n_leaves
+
+
+if __name__ == "__main__":
+    src, dst = sys.argv[1], sys.argv[2]
+    text, n = rewrite(open(src).read())
+    open(dst, "w").write(text)
+    print("jump table over %d leaves written to %s" % (n, dst))
