@@ -63,18 +63,24 @@ VM_HD float cos_poly(float r) {
   return fmaf(z * z, p, fmaf(z, -0.5f, 1.0f));
 }
 
-// r = x - k*pi/2 with |r| <= pi/4 (approximately), q = k mod 4.  Each step is one fused
-// multiply-add, so the first difference is exact while k*fl(pi/2) stays within 24 bits of x
-// (|x| < 2^24*pi/2); the later steps add an absolute error of a few 1e-7 at the largest
-// arguments, far below the spacing of fp32 numbers of that size.  Beyond that range (and for
-// inf/NaN) x - x is returned: 0, or NaN.
+// r = x - k*pi/2 with |r| <= pi/4 (approximately), q = k mod 4.  k = round(x*2/pi) is taken
+// with the add-a-big-constant trick (1.5*2^23: the sum's low mantissa bits are the integer), which
+// costs two fused multiply-adds instead of a round and a float-to-int conversion on the
+// quarter-rate pipe; it is exact for |x*2/pi| < 2^22.  Each reduction step is one fused
+// multiply-add, so the first difference is exact while k*fl(pi/2) stays within 24 bits of x;
+// the later steps add an absolute error of a few 1e-7 at the largest arguments, far below the
+// spacing of fp32 numbers of that size.  Beyond |x| = 6.5e6 (and for inf/NaN) x - x is returned:
+// 0, or NaN.
 VM_HD float reduce_pio2(float x, int* q) {
-  float k = rintf(x * 0.636619772367581343f);
+  const float big = 12582912.0f;                                  // 1.5 * 2^23
+  const float kb = fmaf(x, 0.636619772367581343f, big);
+  float k = kb - big;
   float r = fmaf(-k, 1.57079637050628662109375f, x);        // fl(pi/2)
   r = fmaf(-k, -4.371138828673793e-8f, r);                  // fl(pi/2 - c1)
   r = fmaf(-k, -1.7151245100058819e-15f, r);                // fl(pi/2 - c1 - c2)
-  if (!(fabsf(x) <= 2.5e7f)) { r = x - x; k = 0.f; }
-  *q = (int)k;
+  int qi = (int)f_bits(kb);                                 // low bits = k (two's complement)
+  if (!(fabsf(x) <= 6.5e6f)) { r = x - x; qi = 0; }
+  *q = qi;
   return r;
 }
 
@@ -104,7 +110,8 @@ VM_HD float cos_f(float x) {
 
 // exp for -100 <= x <= 88.7 (callers clamp)
 VM_HD float exp_core(float x) {
-  const float n = rintf(x * 1.44269504088896341f);
+  const float nb = fmaf(x, 1.44269504088896341f, 12582912.0f);   // round(x*log2 e) in the low mantissa bits
+  const float n = nb - 12582912.0f;
   float r = fmaf(-n, 0.693145751953125f, x);                   // ln2, high part with a short mantissa
   r = fmaf(-n, 1.428606765330187e-6f, r);                      // ln2 - high part
   float e = fmaf(r, 1.3814663108745e-3f, 8.36871131029872e-3f);
@@ -113,8 +120,8 @@ VM_HD float exp_core(float x) {
   e = fmaf(r, e, 4.9999993454926206e-1f);
   const float p = fmaf(r * r, e, r) + 1.0f;
   // 2^n in two factors so that n = 128 and n below -126 stay in range
-  const int ni = (int)n;
-  const int h = ni / 2;
+  const int ni = (int)(f_bits(nb) << 10) >> 10;                   // sign-extended low 22 bits
+  const int h = ni >> 1;
   const float s1 = f_from_bits((uint32_t)(h + 127) << 23), s2 = f_from_bits((uint32_t)(ni - h + 127) << 23);
   return p * s1 * s2;
 }

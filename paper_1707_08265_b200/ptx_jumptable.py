@@ -18,7 +18,7 @@ BRANCH = re.compile(r"^\s*(@!?%p\d+\s+)?(bra(\.uni)?|brx\.idx|ret|exit|trap)\b")
 TREE_OK = re.compile(r"^\s*(@!?%p\d+\s+)?(setp\.|bra\b|bra\.uni\b|cvt\.[us]\d+\.[us]\d+\s|and\.b(16|32)\s|(add|sub)\.s(16|32)\s|shr\.[us]32\s)")
 
 
-def rewrite(ptx, kernel_substr="vm_kernel"):
+def rewrite(ptx, kernel_substr="vm_kernel", thread=True):
     lines = ptx.split("\n")
     # body of the kernel entry
     start = next(i for i, l in enumerate(lines) if ".entry" in l and kernel_substr in l)
@@ -99,14 +99,34 @@ def rewrite(ptx, kernel_substr="vm_kernel"):
             i += 1
             if i >= body_hi:
                 raise RuntimeError("ran off the kernel body while checking the tree")
+    # threaded dispatch: the decode of the next instruction (the loop head, a straight block that
+    # ends at the dispatch point) is copied to the end of every leaf in place of the jump back,
+    # so that it can be scheduled among the leaf's own arithmetic
+    h = disp
+    while not LABEL.match(lines[h]):
+        h -= 1
+        if h <= body_lo:
+            raise RuntimeError("no label at the loop head")
+    head_label = LABEL.match(lines[h]).group(1)
+    head = [l for l in lines[h + 1:disp] if is_code(l)]
+    for l in head:
+        if BRANCH.match(l) and not l.strip().startswith("@"):
+            raise RuntimeError("loop head is not a straight block")
+    back = re.compile(r"^\s*bra(\.uni)?\s+" + re.escape(head_label) + r";\s*$")
     # rewrite
     out = []
+    n_threaded = 0
     for i, l in enumerate(lines):
         if i in inserts:
             out.append(inserts[i] + ":")
         if i == disp:
             out.append("\tVMJT: .branchtargets " + ", ".join(leaf_label[n] for n in range(n_leaves)) + ";")
             out.append("\tbrx.idx " + reg + ", VMJT;")
+            continue
+        if thread and body_lo < i < body_hi and back.match(l) and i > disp:
+            out.extend(head)
+            out.append("\tbrx.idx " + reg + ", VMJT;")
+            n_threaded += 1
             continue
         out.append(l)
     return "\n".join(out), n_leaves
