@@ -129,6 +129,19 @@ int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flag_per_in
 int dragon_function_num_launches(const dragon_function_t* f);
 int dragon_function_describe(const dragon_function_t* f, char* buf, int cap);
 
+/* Introspection of one graph-VM step of the plan (step index = line of dragon_function_describe),
+ * for tools and tests that check the emitted instruction stream without a GPU.  info[0..8] =
+ * {number of code words, row mode (0/1), cols, number of operands, spill slots, shared-memory
+ * slots, rows or elements (low 32 bits), rows or elements (high 32 bits), number of reduced
+ * outputs}; code (may be NULL)
+ * receives up to cap_code words (encoding: csrc/vm_isa.h); operands (may be NULL) receives up to
+ * cap_operands quadruples {where (0 feed, 1 fetch, 2 workspace), position or workspace offset / 256,
+ * kind (0 full, 1 row, 2 scalar), dtype}; reduced (may be NULL) receives up to cap_reduced triples
+ * {0 column sums / 1 scalar sum, accumulator index, fetch position (or -1 for a workspace tensor)}.
+ * Returns DRAGON_ERR_INVALID_ARG if the step is not a graph-VM step. */
+int dragon_function_vm_step(const dragon_function_t* f, int step, int64_t* info, uint32_t* code, int cap_code,
+                            int64_t* operands, int cap_operands, int64_t* reduced, int cap_reduced);
+
 /* Scratch memory (partial sums, tensors that cross kernels, spilled values, a status word).
  * dev_ptr: device memory, 256-byte aligned, at least dragon_function_workspace_bytes() long,
  * owned by the caller and not touched by anyone else while a run is in flight. */

@@ -39,6 +39,8 @@ _SIGNATURES = {
     "dragon_function_used_inputs": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_uint8), _c.c_int]),
     "dragon_function_num_launches": (_c.c_int, [_c.c_void_p]),
     "dragon_function_describe": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_int]),
+    "dragon_function_vm_step": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64), _c.POINTER(_c.c_uint32), _c.c_int,
+                                           _c.POINTER(_c.c_int64), _c.c_int, _c.POINTER(_c.c_int64), _c.c_int]),
     "dragon_function_workspace_bytes": (_c.c_size_t, [_c.c_void_p]),
     "dragon_function_set_workspace": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.c_size_t]),
     "dragon_run": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p), _c.c_void_p]),
@@ -208,6 +210,20 @@ class Function:
         buf = _c.create_string_buffer(1 << 16)
         lib().dragon_function_describe(self.h, buf, len(buf))
         return buf.value.decode()
+
+    def vm_step(self, step):
+        """Instruction stream and operand table of a graph-VM step, or None for another kind of step."""
+        info = (_c.c_int64 * 9)()
+        if lib().dragon_function_vm_step(self.h, step, info, None, 0, None, 0, None, 0) < 0:
+            return None
+        code = (_c.c_uint32 * max(1, info[0]))()
+        ops = (_c.c_int64 * max(4, 4 * info[3]))()
+        red = (_c.c_int64 * max(3, 3 * info[8]))()
+        lib().dragon_function_vm_step(self.h, step, info, code, info[0], ops, info[3], red, info[8])
+        return {"code": list(code[:info[0]]), "row_mode": bool(info[1]), "cols": info[2], "n": info[6] | (info[7] << 32),
+                "n_spill": info[4], "n_smem": info[5],
+                "operands": [tuple(ops[4 * i:4 * i + 4]) for i in range(info[3])],
+                "reduced": [tuple(red[3 * i:3 * i + 3]) for i in range(info[8])]}
 
     def workspace_bytes(self):
         return lib().dragon_function_workspace_bytes(self.h)

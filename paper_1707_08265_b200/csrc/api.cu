@@ -241,6 +241,33 @@ int dragon_function_describe(const dragon_function_t* f, char* buf, int cap) {
   return DRAGON_OK;
 }
 
+int dragon_function_vm_step(const dragon_function_t* f, int step, int64_t* info, uint32_t* code, int cap_code,
+                            int64_t* operands, int cap_operands, int64_t* reduced, int cap_reduced) {
+  if (!f || !info || step < 0 || step >= (int)f->plan.steps.size() || f->plan.steps[step].kind != ST_VM || cap_code < 0 || cap_operands < 0) {
+    set_error("dragon_function_vm_step: not a graph-VM step");
+    return DRAGON_ERR_INVALID_ARG;
+  }
+  const VmSegment& sg = f->plan.segs[f->plan.steps[step].seg];
+  info[0] = (int64_t)sg.code.size(); info[1] = sg.row_mode; info[2] = sg.cols; info[3] = (int64_t)sg.operand_mem.size();
+  info[4] = sg.n_spill; info[5] = sg.n_smem; info[6] = sg.n & 0xffffffffLL; info[7] = sg.n >> 32;
+  info[8] = (int64_t)sg.finish.size();
+  for (int i = 0; reduced && i < cap_reduced && i < (int)sg.finish.size(); ++i) {
+    const MemRef& m = f->plan.mems[sg.finish[i].mem];
+    reduced[3 * i + 0] = sg.finish[i].kind;
+    reduced[3 * i + 1] = sg.finish[i].acc;
+    reduced[3 * i + 2] = m.where == MEM_FETCH ? m.index : -1;
+  }
+  for (int i = 0; code && i < cap_code && i < (int)sg.code.size(); ++i) code[i] = sg.code[i];
+  for (int i = 0; operands && i < cap_operands && i < (int)sg.operand_mem.size(); ++i) {
+    const MemRef& m = f->plan.mems[sg.operand_mem[i]];
+    operands[4 * i + 0] = m.where;
+    operands[4 * i + 1] = m.where == MEM_WORK ? (int64_t)(m.offset / 256) : m.index;
+    operands[4 * i + 2] = sg.operand_kind[i];
+    operands[4 * i + 3] = m.dtype;
+  }
+  return DRAGON_OK;
+}
+
 size_t dragon_function_workspace_bytes(const dragon_function_t* f) { return f ? f->plan.workspace_bytes : 0; }
 
 int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t bytes) {

@@ -42,6 +42,7 @@ struct Gen {
   int n_uni = 0;
   int acc_val = -1;
   std::vector<bool> done;        // item already produced by a fused instruction
+  std::vector<std::pair<int, int>> accs;  // (item position of an accumulation, its pinned register)
   int err = DRAGON_OK;
 
   Gen(const std::vector<Item>& it, const std::vector<int>& ix, const std::vector<Value>& v,
@@ -214,9 +215,12 @@ struct Gen {
       if (aa && !ab) { x = b; y = a; }
       else if (ab && !aa) { x = a; y = b; }
       else if (aa && ab) {
-        // keep the one that is needed again where it is
+        // a uniform stays the addressed operand (multiply-by-uniform then add fuses later);
+        // otherwise keep the one that is needed again where it is
         bool a_dies = next_use(a, pos) == kFar, b_dies = next_use(b, pos) == kFar;
-        if (b_dies && !a_dies) { x = b; y = a; } else { x = a; y = b; }
+        if (info[a].uni >= 0 && info[b].uni < 0) { x = b; y = a; }
+        else if (info[b].uni >= 0 && info[a].uni < 0) { x = a; y = b; }
+        else if (b_dies && !a_dies) { x = b; y = a; } else { x = a; y = b; }
       } else { x = a; y = b; }
     }
     if (a == b) {
@@ -254,7 +258,6 @@ struct Gen {
       {M_ONEMSQ, P_ONEMSQ}, {M_YOMY, P_YOMY}, {M_DIVPGB, P_DIVPGB}, {M_RBF16, P_RBF16}, {M_ROWSUM, P_ROWSUM}};
     const int a = C(it.a), d = C(it.dst);
     load_acc(a, pos, a);
-    keep_operand(a, pos, -1);
     // sin and cos of the same value share one range reduction
     if (it.opc == M_SIN || it.opc == M_COS) {
       for (int q = pos + 1; q < (int)idx.size() && q < pos + 4096; ++q) {
@@ -262,22 +265,50 @@ struct Gen {
         if (done[q] || o2.kind != IT_MOP || (o2.opc != M_SIN && o2.opc != M_COS) || o2.opc == it.opc || C(o2.a) != a) continue;
         int sl = free_smem();
         if (sl < 0) break;  // no slot for the cosine: two separate instructions
-        emit(P_SINCOS, 0, sl);
         int dsin = it.opc == M_SIN ? d : C(o2.dst), dcos = it.opc == M_SIN ? C(o2.dst) : d;
-        info[dcos].home = H_SMEM; info[dcos].home_idx = sl; smem_owner[sl] = dcos;
+        smem_owner[sl] = dcos;    // taken before anything below can evict a register into it
+        auto& ua = info[a].uses;  // the partner's use of a is consumed here
+        ua.erase(std::remove(ua.begin(), ua.end(), q), ua.end());
+        keep_operand(a, pos, -1);
+        emit(P_SINCOS, 0, sl);
+        info[dcos].home = H_SMEM; info[dcos].home_idx = sl;
         acc_val = dsin;
         done[q] = true;
-        auto& u = info[a].uses;  // the partner's use of a is consumed here
-        u.erase(std::remove(u.begin(), u.end(), q), u.end());
         release_dead(a, pos);
         if (next_use(dcos, pos) == kFar) release(dcos);
         if (next_use(dsin, pos) == kFar) acc_val = -1;
         return;
       }
     }
+    keep_operand(a, pos, -1);
     emit(op.at(it.opc));
     acc_val = d;
     release_dead(a, pos);
+  }
+
+  // the accumulator holds a fresh value: stores and accumulations of it that come later in the
+  // list are issued right away (they depend on nothing else), which saves a store/reload pair
+  void drain_acc(int pos) {
+    const int v = acc_val;
+    if (v < 0) return;
+    for (int q = pos + 1; q < (int)idx.size() && q < pos + 4096; ++q) {
+      const Item& o2 = items[idx[q]];
+      if (done[q] || (o2.opc != M_STORE && o2.opc != M_ACCUM) || C(o2.a) != v) continue;
+      if (o2.opc == M_STORE) {
+        int cls = class_of(mems[o2.mem].shape);
+        if (cls < 0) continue;
+        emit(P_GST, 0, operand_for(o2.mem, cls));
+      } else {
+        int k = -1;
+        for (auto& a : accs) if (a.first == q) k = a.second;
+        if (k < 0) continue;
+        emit(J_ACCUM * kJointStride + k);
+      }
+      done[q] = true;
+      auto& u = info[v].uses;
+      u.erase(std::remove(u.begin(), u.end(), q), u.end());
+    }
+    if (next_use(v, pos) == kFar) { release(v); acc_val = -1; }
   }
 
   int run() {
@@ -343,7 +374,6 @@ struct Gen {
       seg->cols = 0;
     }
     // 3. accumulators get pinned registers
-    std::vector<std::pair<int, int>> accs;  // (item position, register)
     for (int p = 0; p < (int)idx.size(); ++p)
       if (items[idx[p]].opc == M_ACCUM) {
         int k = (int)accs.size();
@@ -357,7 +387,7 @@ struct Gen {
       if (done[p]) continue;
       const Item& it = items[idx[p]];
       if (it.opc == M_WIDEN) continue;
-      if (is_binary(it.opc)) binary(it, p);
+      if (is_binary(it.opc)) { binary(it, p); drain_acc(p); }
       else if (it.opc == M_STORE) {
         int v = C(it.a);
         int cls = class_of(mems[it.mem].shape);
@@ -372,7 +402,7 @@ struct Gen {
         load_acc(v, p, v);
         emit(J_ACCUM * kJointStride + k);
         release_dead(v, p);
-      } else unary(it, p);
+      } else { unary(it, p); drain_acc(p); }
     }
     if (err) return err;
     // 5. peephole: multiply by a uniform followed by an add fuses into one instruction

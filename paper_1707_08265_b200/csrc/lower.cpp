@@ -461,6 +461,34 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
   return DRAGON_OK;
 }
 
+// one mnemonic per instruction word of a segment
+static std::string disassemble(const VmSegment& sg) {
+  static const char* jn[] = {"ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr"};
+  static const char* pn[] = {"ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls",
+                             "divps", "rdivps", "sin", "cos", "sincos", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq",
+                             "yomy", "divpgb", "rbf16", "rowsum", "gld", "gst", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout",
+                             "scalout", "end"};
+  std::string s;
+  char buf[64];
+  for (size_t i = 0; i < sg.code.size(); ++i) {
+    const uint32_t w = sg.code[i];
+    const int cs = (int)(w & 1023u);
+    const uint32_t arg = w >> 14;
+    if (cs < vm::kFirstPlain) snprintf(buf, sizeof(buf), "%s r%d", jn[cs / vm::kJointStride], cs % vm::kJointStride);
+    else if (cs < vm::P_COUNT_) snprintf(buf, sizeof(buf), "%s", pn[cs - vm::kFirstPlain]);
+    else snprintf(buf, sizeof(buf), "?%d", cs);
+    s += buf;
+    if (arg || (cs >= vm::kFirstPlain && cs != vm::P_LOOP_BEGIN && cs != vm::P_LOOP_END && cs != vm::P_END && !(cs >= vm::P_SIN && cs <= vm::P_ROWSUM && cs != vm::P_SINCOS))) {
+      snprintf(buf, sizeof(buf), " %u", arg);
+      s += buf;
+    }
+    s += "; ";
+    if (cs == vm::P_UCONST) ++i;
+    if (cs == vm::P_END) break;
+  }
+  return s;
+}
+
 std::string describe_plan(const Plan& p) {
   std::string s;
   char buf[256];
@@ -471,6 +499,9 @@ std::string describe_plan(const Plan& p) {
         snprintf(buf, sizeof(buf), "vm[%s n=%lld cols=%d instr=%d body=%d operands=%d smem=%d spill=%d colacc=%d scalacc=%d grid=%d]\n",
                  sg.row_mode ? "row" : "flat", sg.n, sg.cols, (int)sg.code.size(), sg.n_instr_body,
                  (int)sg.operand_mem.size(), sg.n_smem, sg.n_spill, sg.n_colacc, sg.n_scalacc, sg.grid);
+        s += buf;
+        if (sg.code.size() <= 96) s += "  code: " + disassemble(sg) + "\n";
+        buf[0] = 0;
         break;
       }
       case ST_GEMM:
