@@ -29,7 +29,7 @@ constexpr int V = kVmVec;
 constexpr int NV4 = V / 4;
 constexpr int NR = kVmRegs;
 constexpr int TILE = kVmTile;
-static_assert(V % 4 == 0 && NR >= 6 && NR <= 12, "the case tables below are written for 6..12 register slots");
+static_assert(V % 4 == 0 && NR >= 2 && NR <= 15, "register slot count out of range");
 
 #define FORV _Pragma("unroll") for (int j = 0; j < V; ++j)
 
@@ -39,6 +39,7 @@ struct TileCtx {
   bool full;        // limit == TILE
   bool vec_ok;      // 4-element groups are 16-byte aligned
   bool first;       // tile 0 (stores of ROW / SCALAR shaped outputs happen here)
+  long long next;   // element distance to this CTA's next tile, 0 when there is none (L2 prefetch)
 };
 
 __device__ __forceinline__ int lane_pos(int tid, int j) { return (j >> 2) * (NT * 4) + tid * 4 + (j & 3); }
@@ -47,6 +48,11 @@ __device__ __forceinline__ void load_operand(const Operand& o, const TileCtx& tc
   const long long base = o.kind == K_FULL ? tc.base : 0;
   if (o.dtype == DRAGON_F32) {
     const float* p = reinterpret_cast<const float*>(o.ptr) + base;
+    if (o.kind == K_FULL && tc.next) {  // pull this CTA's next tile into L2 while the current one is processed
+#pragma unroll
+      for (int h = 0; h < NV4; ++h)
+        if (h * NT * 4 + tid * 4 < tc.limit) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + tc.next + h * NT * 4 + tid * 4));
+    }
 #pragma unroll
     for (int h = 0; h < NV4; ++h) {
       const int pos = h * NT * 4 + tid * 4;
@@ -60,6 +66,11 @@ __device__ __forceinline__ void load_operand(const Operand& o, const TileCtx& tc
     }
   } else {
     const unsigned short* p = reinterpret_cast<const unsigned short*>(o.ptr) + base;
+    if (o.kind == K_FULL && tc.next) {
+#pragma unroll
+      for (int h = 0; h < NV4; ++h)
+        if (h * NT * 4 + tid * 4 < tc.limit) asm volatile("prefetch.global.L2 [%0];" ::"l"(p + tc.next + h * NT * 4 + tid * 4));
+    }
 #pragma unroll
     for (int h = 0; h < NV4; ++h) {
       const int pos = h * NT * 4 + tid * 4;
@@ -170,6 +181,11 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
     }
     tc.full = tc.limit == TILE;
     tc.first = tile == 0;
+    // the whole next tile must exist for the prefetch addresses to stay inside the tensor
+    const long long nt = tile + gridDim.x;
+    tc.next = 0;
+    if (p.row_mode) { if (nt < ntiles) tc.next = (long long)gridDim.x * p.cols; }
+    else if ((nt + 1) * TILE <= p.n) tc.next = (long long)gridDim.x * TILE;
   };
   set_tile();
   float* spill = p.spill + (size_t)blockIdx.x * p.n_spill * TILE;
