@@ -117,6 +117,65 @@ def run_reference(args):
     print(json.dumps(line), flush=True)
 
 
+def run_other_config(args):
+    """Device-resident timing of the other workloads (same step definition: one dragon_run)."""
+    import torch
+    from paper_1707_08265_b200 import binding as B
+    seeds = json.load(open(os.path.join(ROOT, "tests", "golden", "config_seeds.json")))
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32}
+    gen = torch.Generator("cuda").manual_seed(wl.BASE_SEED + args.config)
+
+    def dev_random(g, t):
+        ti = g.desc["tensors"][t]
+        if ti["dtype"] == "i32":
+            return torch.randint(0, 4096, tuple(ti["shape"]), generator=gen, device="cuda", dtype=torch.int32)
+        return torch.empty(tuple(ti["shape"]), dtype=torch.float32, device="cuda").normal_(generator=gen).to(tdt[ti["dtype"]])
+
+    if args.config == 1:
+        n = 1 << 20
+        g, ids = wl.toy_function(n)
+        inputs, outputs, units, what = [ids["x"], ids["a"], ids["b"]], [ids["f"], ids["y"]], n, "f and y of x*sin(a*x+b), x fp32[2^20] (L2-resident)"
+    elif args.config == 3:
+        n = 1 << 27
+        g, inputs, outputs = wl.random_dag(n, seeds["random_dag"]["seed"])
+        units, what = n, "random 64-operator elementwise DAG, 4 x fp32[2^27], 2 fetches"
+    elif args.config == 4:
+        g, ids = wl.mlp(8192, 4096, 4096, 4096)
+        inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
+        outputs = [ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")]
+        units, what = 8192, "MLP 8192 x 4096-4096-4096 bf16, forward + backward (batch rows per step)"
+    else:
+        from oracle import prune as oprune   # which inputs are connected is decided outside the generator
+        g, inputs, fetch = wl.random_row_dag(16384, 4096, seeds["random_row_dag"]["seed"])
+        G = oprune.backward_marks(g.desc, fetch, inputs)
+        outputs = fetch + g.grad(fetch, [i for i in inputs if i in G])
+        units, what = 16384 * 4096, "random 1024-operator row DAG on [16384,4096], forward + backward"
+    f = B.Graph.from_desc(g.desc).function(inputs, outputs)
+    feeds = [dev_random(g, t) if u else None for t, u in zip(inputs, f.used_inputs())]
+    if args.config == 4:
+        for j in (1, 2, 3, 4):
+            feeds[j] = (feeds[j].float() / 64).to(torch.bfloat16)
+    outs = [torch.empty(tuple(g.shape(t)), dtype=tdt[g.desc["tensors"][t]["dtype"]], device="cuda") for t in outputs]
+    for _ in range(max(3, args.warmup)):
+        f.run_torch(feeds, outs)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    steps = min(args.steps, 50)
+    e0.record()
+    for _ in range(steps):
+        f.run_torch(feeds, outs)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    assert f.status() == 0
+    nbytes = sum(t.numel() * t.element_size() for t in feeds if t is not None) + sum(t.numel() * t.element_size() for t in outs)
+    line = {"config": args.config, "workload": what, "ms_per_step": ms, "units_per_s": units / (ms * 1e-3),
+            "io_GBps": nbytes / ms / 1e6, "launches": f.num_launches(), "plan": f.describe().strip().split("\n")[:24]}
+    if args.config == 4:
+        line["gemm_TFLOPs_over_whole_step"] = 5 * 2 * 8192 * 4096 * 4096 / ms / 1e9
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -125,9 +184,13 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU (default: the benchmark's 2^26)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5],
+                    help="2 (default) is the benchmark workload; the others print one summary line each")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.config != 2:
+        return run_other_config(args)
 
     import torch
     import torch.distributed as dist
