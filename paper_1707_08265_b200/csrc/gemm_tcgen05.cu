@@ -2,9 +2,12 @@
 // tensor memory, fp32 or bf16 output.  Hand-written for sm_100a:
 //   - operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
 //     ring of shared-memory stages guarded by full/empty mbarriers;
-//   - one elected thread issues tcgen05.mma (cta_group::1, kind::f16, 128 x kTileN x 16) with the
-//     accumulator in TMEM; tcgen05.commit releases stages and finally signals the epilogue;
-//   - four epilogue warps read their 32-lane TMEM quadrants with tcgen05.ld and write C.
+//   - one elected thread issues tcgen05.mma (cta_group::1, kind::f16, 128 x 256 x 16) with the
+//     accumulator in TMEM; tcgen05.commit releases stages and signals the epilogue;
+//   - four epilogue warps read their 32-lane TMEM quadrants with tcgen05.ld and write C;
+//   - CTAs are persistent (one per SM) and walk the 128 x 256 output tiles in an L2-friendly
+//     order; two TMEM accumulators alternate, so the epilogue of one tile overlaps the main loop
+//     of the next.
 // Warp roles (192 threads): warp 0 = TMA producer, warp 1 = TMEM owner + MMA issuer,
 // warps 2..5 = epilogue.  Every mbarrier wait is bounded by a clock budget; when it runs out
 // the kernel records DRAGON_ERR_TIMEOUT in the status word, stops issuing work, frees its TMEM
@@ -12,8 +15,8 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdint>
-#include <map>
 #include <mutex>
 
 #include "plan.h"
@@ -23,10 +26,11 @@ namespace dragon {
 namespace {
 
 constexpr int kTileM = 128;
-constexpr int kTileN = 128;
+constexpr int kTileN = 256;
 constexpr int kTileK = 64;          // one 128-byte swizzle row of bf16
-constexpr int kStages = 6;
+constexpr int kStages = 4;
 constexpr int kUmmaK = 16;
+constexpr int kAccBufs = 2;         // double-buffered accumulators: 2 x 256 TMEM columns
 constexpr int kGemmThreads = 192;
 constexpr uint32_t kStageBytesA = kTileM * kTileK * 2;
 constexpr uint32_t kStageBytesB = kTileN * kTileK * 2;
@@ -109,8 +113,24 @@ struct GemmArgs {
   void* C;
   int c_dtype;
   int M, N, K;
+  int tiles_m, tiles_n;
   int* status;
 };
+
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+// tile order: groups of 8 row-blocks share their column sweep, so that the B tiles of a sweep
+// and the 8 A row-blocks stay in L2 while they are reused
+__device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int* tm, int* tn) {
+  const int group = 8 * tiles_n;
+  const int g0 = (t / group) * 8;
+  const int rows = min(8, tiles_m - g0);
+  const int r = t % group;
+  *tm = g0 + r % rows;
+  *tn = r / rows;
+}
 
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
@@ -119,23 +139,24 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   const uint32_t tiles = (raw + 1023u) & ~1023u;                 // 1024-byte aligned operand stages
   unsigned char* tiles_ptr = gemm_smem_raw + (tiles - raw);
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + (size_t)kStages * kStageBytes);
-  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages, bar_accum = bar_empty + 8 * kStages;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 1);
+  const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages;
+  const uint32_t bar_acc_full = bar_empty + 8 * kStages, bar_acc_empty = bar_acc_full + 8 * kAccBufs;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccBufs);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int m0 = blockIdx.y * kTileM, n0 = blockIdx.x * kTileN;
   const int k_tiles = (g.K + kTileK - 1) / kTileK;
+  const int n_tiles = g.tiles_m * g.tiles_n;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
-    mbar_init(bar_accum, 1);
+    for (int b = 0; b < kAccBufs; ++b) { mbar_init(bar_acc_full + 8 * b, 1); mbar_init(bar_acc_empty + 8 * b, 4); }
     abort_flag[0] = 0;
     abort_flag[1] = 0;   // a flag nobody sets, for waits that must not be cut short
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-  if (warp == 1) {  // TMEM: kTileN fp32 columns x 128 lanes
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)kTileN) : "memory");
+  if (warp == 1) {  // TMEM: two accumulators of kTileN fp32 columns x 128 lanes
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)(kAccBufs * kTileN)) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -144,56 +165,72 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    if (lane == 0) {  // TMA producer
+    if (lane == 0) {  // TMA producer: one running stage counter across all tiles of this CTA
       int issued = 0;
-      for (int kt = 0; kt < k_tiles; ++kt) {
-        const int s = kt % kStages, it = kt / kStages;
-        if (!mbar_wait(bar_empty + 8 * s, (it & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); break; }
-        mbar_expect_tx(bar_full + 8 * s, kStageBytes);
-        const uint32_t dst = tiles + (uint32_t)s * kStageBytes;
-        tma_load_2d(dst, &tmap_a, kt * kTileK, m0, bar_full + 8 * s);
-        tma_load_2d(dst + kStageBytesA, &tmap_b, kt * kTileK, n0, bar_full + 8 * s);
-        issued = kt + 1;
+      bool ok = true;
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        int tm, tn;
+        tile_coords(t, g.tiles_m, g.tiles_n, &tm, &tn);
+        for (int kt = 0; kt < k_tiles; ++kt, ++issued) {
+          const int s = issued % kStages, it = issued / kStages;
+          if (!mbar_wait(bar_empty + 8 * s, (it & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+          mbar_expect_tx(bar_full + 8 * s, kStageBytes);
+          const uint32_t dst = tiles + (uint32_t)s * kStageBytes;
+          tma_load_2d(dst, &tmap_a, kt * kTileK, tm * kTileM, bar_full + 8 * s);
+          tma_load_2d(dst + kStageBytesA, &tmap_b, kt * kTileK, tn * kTileN, bar_full + 8 * s);
+        }
       }
       if (*abort_flag) {  // let the copies that are still in flight land before the CTA goes away
-        for (int kt = issued > kStages ? issued - kStages : 0; kt < issued; ++kt)
-          mbar_wait(bar_full + 8 * (kt % kStages), (kt / kStages) & 1, abort_flag + 1 /* never set */);
+        for (int i = issued > kStages ? issued - kStages : 0; i < issued; ++i)
+          mbar_wait(bar_full + 8 * (i % kStages), (i / kStages) & 1, abort_flag + 1);
       }
     }
   } else if (warp == 1) {
     if (lane == 0) {  // MMA issuer
       constexpr uint32_t idesc = make_idesc(kTileM, kTileN);
+      int consumed = 0, local = 0;
       bool ok = true;
-      for (int kt = 0; kt < k_tiles && ok; ++kt) {
-        const int s = kt % kStages, it = kt / kStages;
-        if (!mbar_wait(bar_full + 8 * s, it & 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+      for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
+        const int buf = local % kAccBufs, use = local / kAccBufs;
+        // the epilogue must have drained this accumulator (first use passes at once)
+        if (!mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const uint32_t a_addr = tiles + (uint32_t)s * kStageBytes, b_addr = a_addr + kStageBytesA;
-        const uint64_t a_desc = make_smem_desc(a_addr), b_desc = make_smem_desc(b_addr);
+        const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
+        for (int kt = 0; kt < k_tiles; ++kt, ++consumed) {
+          const int s = consumed % kStages, it = consumed / kStages;
+          if (!mbar_wait(bar_full + 8 * s, it & 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+          asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+          const uint32_t a_addr = tiles + (uint32_t)s * kStageBytes, b_addr = a_addr + kStageBytesA;
+          const uint64_t a_desc = make_smem_desc(a_addr), b_desc = make_smem_desc(b_addr);
 #pragma unroll
-        for (int k = 0; k < kTileK / kUmmaK; ++k) {
-          // advancing 16 elements along K inside the swizzle row = 32 bytes = 2 descriptor units
-          umma_f16(tmem_base, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+          for (int k = 0; k < kTileK / kUmmaK; ++k) {
+            // advancing 16 elements along K inside the swizzle row = 32 bytes = 2 descriptor units
+            umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+          }
+          umma_commit(bar_empty + 8 * s);   // the stage is free once these MMAs have read it
         }
-        umma_commit(bar_empty + 8 * s);   // the stage is free once these MMAs have read it
+        if (ok) umma_commit(bar_acc_full + 8 * buf);   // accumulator complete
       }
-      if (ok) umma_commit(bar_accum);     // accumulator complete
     }
   } else {
-    // epilogue: warp w owns TMEM lanes 32*(w%4) .. +31, i.e. rows m0 + 32*(w%4) + lane
+    // epilogue: warp w owns TMEM lanes 32*(w%4) .. +31, i.e. rows 32*(w%4) + lane of the tile
     const int q = warp & 3;
-    const bool ok = mbar_wait(bar_accum, 0, abort_flag);
-    if (!ok && lane == 0) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); }
-    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int row = m0 + q * 32 + lane;
-    if (ok) {
+    int local = 0;
+    for (int t = blockIdx.x; t < n_tiles; t += gridDim.x, ++local) {
+      const int buf = local % kAccBufs, use = local / kAccBufs;
+      int tm, tn;
+      tile_coords(t, g.tiles_m, g.tiles_n, &tm, &tn);
+      const bool ok = mbar_wait(bar_acc_full + 8 * buf, use & 1, abort_flag);
+      if (!ok) { if (lane == 0) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); } break; }
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int row = tm * kTileM + q * 32 + lane;
 #pragma unroll 1
       for (int c = 0; c < kTileN; c += 32) {
         uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)c, v);
+        tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kTileN + c), v);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-        if (row < g.M) {
-          const int col0 = n0 + c;
+        const int col0 = tn * kTileN + c;
+        if (row < g.M && col0 < g.N) {
           if (g.c_dtype == DRAGON_F32) {
             float* out = reinterpret_cast<float*>(g.C) + (size_t)row * g.N + col0;
             if ((g.N & 3) == 0 && col0 + 32 <= g.N) {
@@ -225,12 +262,16 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
           }
         }
       }
+      // this warp is done reading the accumulator: hand it back to the MMA issuer
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(bar_acc_empty + 8 * buf);
     }
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)kTileN) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(kAccBufs * kTileN)) : "memory");
   }
 }
 
@@ -280,8 +321,14 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
   static cudaError_t attr_err = cudaSuccess;
   std::call_once(once, [] { attr_err = cudaFuncSetAttribute(gemm_bf16_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem); });
   if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
-  GemmArgs g{C, c_dtype, M, N, K, status};
-  dim3 grid((N + kTileN - 1) / kTileN, (M + kTileM - 1) / kTileM);
+  const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
+  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status};
+  static int sm_count = 0;
+  if (!sm_count) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0) sm_count = kDefaultSmCount;
+  }
+  const int grid = std::min(tiles_m * tiles_n, sm_count);   // persistent CTAs, one per SM
   gemm_bf16_tcgen05<<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, g);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_error("InnerProduct: launch failed: %s", cudaGetErrorString(e)); return DRAGON_ERR_CUDA; }
