@@ -25,6 +25,8 @@ struct Lowerer {
   std::vector<std::map<int, int>> gval;       // per stage: tensor -> gradient value id
   std::vector<int> fetch_of;                  // tensor -> fetch position or -1
   std::map<int, int> transposed;              // memref -> memref of its transpose
+  std::map<std::pair<int, int>, int> materialised;   // (value, dtype) -> memref
+  std::vector<std::map<int, int>> pending;    // per stage: tensor -> gradient contributions still to come
   int err = DRAGON_OK;
 
   Lowerer(const Graph& g_, const PruneResult& pr_, Plan* p) : g(g_), pr(pr_), plan(p) {}
@@ -93,8 +95,13 @@ struct Lowerer {
   int materialise(int v, int dtype, int dtype_if_new) {
     const Value& val = vals[v];
     if (val.kind == VK_MEM && (dtype < 0 || plan->mems[val.mem].dtype == dtype)) return val.mem;
-    int m = new_mem(MEM_WORK, -1, dtype < 0 ? dtype_if_new : dtype, val.shape);
+    const int want = dtype < 0 ? dtype_if_new : dtype;
+    auto key = std::make_pair(v, want);
+    auto it = materialised.find(key);
+    if (it != materialised.end()) return it->second;   // one image per value and type
+    int m = new_mem(MEM_WORK, -1, want, val.shape);
     store(v, m);
+    materialised[key] = m;
     return m;
   }
   int transpose_of(int mem) {
@@ -211,7 +218,8 @@ struct Lowerer {
       case DRAGON_OP_EXP: add(0, mop(M_MUL, mop(M_MUL, dy, fval[o]), mop(M_CLAMPMASK, in(0)))); break;
       case DRAGON_OP_TANH: add(0, mop(M_MUL, dy, mop(M_ONEMSQ, fval[o]))); break;
       case DRAGON_OP_SIGMOID: add(0, mop(M_MUL, dy, mop(M_YOMY, fval[o]))); break;
-      case DRAGON_OP_RELU: add(0, mop(M_MUL, dy, mop(M_STEP, in(0)))); break;
+      // [x > 0] = [relu(x) > 0]: reading the output keeps the input out of memory
+      case DRAGON_OP_RELU: add(0, mop(M_MUL, dy, mop(M_STEP, fval[o]))); break;
       case DRAGON_OP_SUM: case DRAGON_OP_MEAN: {
         int c = mop(M_ROWSUM, dy);
         if (op.type == DRAGON_OP_MEAN) c = mop(M_MUL, c, konst(1.f / (float)g.tensors[o].shape.cols()));
@@ -306,16 +314,40 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
       for (int o : g.stages[s].objs)
         if (pr.in_G[s][o]) gv[o] = L.konst(1.f);
   };
+  // a fetched gradient is written as soon as its last contribution is in (it then joins the
+  // segment that produced it instead of a trailing one that would re-read everything)
+  auto produced = [&](const GradOpRef& r) {
+    std::vector<int> t;
+    const OpInfo& op = g.ops[r.op];
+    for (size_t p = 0; p < op.in.size(); ++p)
+      if ((r.mask >> p) & 1u) t.push_back(op.in[p]);
+    return t;
+  };
+  L.pending.resize(g.stages.size());
+  for (const GradOpRef& r : pr.grad_ops)
+    for (int t : produced(r)) ++L.pending[r.stage][t];
+  std::vector<std::vector<uint8_t>> fetched_early(g.stages.size(), std::vector<uint8_t>(n, 0));
   for (const GradOpRef& r : pr.grad_ops) {
     seed_stage(r.stage);
     L.lower_gradient(r);
     if (L.err) return L.err;
+    for (int t : produced(r)) {
+      if (--L.pending[r.stage][t] != 0) continue;
+      const GradStage& st = g.stages[r.stage];
+      for (size_t j = 0; j < st.wrts.size(); ++j)
+        if (st.wrts[j] == t && L.fetch_of[st.grad_ids[j]] >= 0 && !fetched_early[r.stage][t]) {
+          auto it = L.gval[r.stage].find(t);
+          if (it == L.gval[r.stage].end()) continue;
+          L.store_fetch(L.widen(it->second, g.tensors[t].shape), st.grad_ids[j]);
+          fetched_early[r.stage][t] = 1;
+        }
+    }
   }
   for (int s = 0; s < (int)g.stages.size(); ++s) {
     const GradStage& st = g.stages[s];
     for (size_t j = 0; j < st.wrts.size(); ++j) {
       int gid = st.grad_ids[j];
-      if (L.fetch_of[gid] < 0) continue;
+      if (L.fetch_of[gid] < 0 || fetched_early[s][st.wrts[j]]) continue;
       seed_stage(s);
       auto it = L.gval[s].find(st.wrts[j]);
       int v = it == L.gval[s].end() ? L.konst(0.f) : it->second;
@@ -401,6 +433,22 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
         int v = which == 0 ? items[i].a : items[i].b;
         if (v < 0 || vals[v].kind != VK_OP || def_seg[v] == items[i].segment) continue;
         auto f = spilled.find(v);
+        if (f == spilled.end()) {
+          int dt = items[def_item[v]].opc == M_RBF16 ? DRAGON_BF16 : DRAGON_F32;
+          // an image of this value that its own segment already writes serves as well
+          auto have = L.materialised.find(std::make_pair(v, dt));
+          if (have != L.materialised.end() && mems[have->second].live) {
+            bool same_seg = false;
+            for (int j = 0; j < n_items; ++j)
+              if (items[j].live && items[j].kind == IT_MOP && items[j].opc == M_STORE && items[j].mem == have->second && items[j].a == v)
+                same_seg = items[j].segment == def_seg[v];
+            if (same_seg) {
+              Value nv; nv.kind = VK_MEM; nv.shape = vals[v].shape; nv.mem = have->second;
+              vals.push_back(nv);
+              f = spilled.emplace(v, (int)vals.size() - 1).first;
+            }
+          }
+        }
         if (f == spilled.end()) {
           int dt = items[def_item[v]].opc == M_RBF16 ? DRAGON_BF16 : DRAGON_F32;
           MemRef m; m.where = MEM_WORK; m.dtype = dt; m.shape = vals[v].shape; m.live = true;
