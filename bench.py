@@ -27,6 +27,9 @@ METRIC = "pruned-graph fwd+bwd elements/sec"
 UNIT = "elements/s"
 WORKLOAD = "config 2: f=x*sin(a*x+b), x fp32[2^26], fetch df/dx, df/da, df/db"
 ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
+# dram__bytes_read.sum + dram__bytes_write.sum of vm_kernel per element, from the ncu capture summarised in
+# profiles/vm_kernel_config2.md (taken at 2^25 elements; traffic is proportional to the element count)
+NCU_DRAM_BYTES_PER_ELEM = (134.384896e6 + 93.343488e6) / (1 << 25)
 
 
 def measured_peak_gbs():
@@ -302,7 +305,7 @@ def main():
                         "h2d_bytes_per_step": 4 * n + 8, "d2h_bytes_per_step": 4 * n + 8},
                 "gpu_launches": f.num_launches() * args.steps,
                 "roofline": {"bound": "hbm", "kernel": "vm_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": None,
+                             "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": NCU_DRAM_BYTES_PER_ELEM * n,
                              "kernel_ms": kern_avg_ms, "frac_of_nominal_8TBs": achieved / 8000.0}}
         if not args.skip_cpu_baseline and world == 1:
             rate, sample, _ = oracle_rate()
