@@ -15,7 +15,7 @@ constexpr int kVmThreads = DRAGON_VM_THREADS;
 constexpr int kVmVec = DRAGON_VM_VEC;
 constexpr int kVmTile = kVmThreads * kVmVec;  // 4096
 constexpr int kVmRegs = DRAGON_VM_REGS;       // register slots R[0..kVmRegs)
-constexpr int kVmCodeMaxWords = 12 * 1024;    // instruction stream held in shared memory
+constexpr int kVmCodeMaxWords = 8 * 1024;     // instruction stream held in shared memory (8 bytes per word once decoded)
 constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread
 constexpr int kDefaultSmCount = 148;
 

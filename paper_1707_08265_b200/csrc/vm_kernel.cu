@@ -149,14 +149,14 @@ __device__ __forceinline__ void dispatch_tree(const int cs, const uint32_t arg, 
 __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Params p) {
   extern __shared__ __align__(16) unsigned char smem_raw[];
   // layout: code | uniforms | reduction scratch | V-wide slots
-  uint32_t* code = reinterpret_cast<uint32_t*>(smem_raw);
+  uint2* code2 = reinterpret_cast<uint2*>(smem_raw);
   const int code_words = (p.n_code + 3) & ~3;
-  float* U = reinterpret_cast<float*>(code + code_words);
+  float* U = reinterpret_cast<float*>(code2 + code_words);
   double* red = reinterpret_cast<double*>(U + kMaxUniforms);
   float4* slots = reinterpret_cast<float4*>(red + 64);                // [slot][NV4][NT]
 
   const int tid = threadIdx.x;
-  for (int i = tid; i < p.n_code; i += NT) code[i] = p.code[i];
+  for (int i = tid; i < p.n_code; i += NT) { const uint32_t cw = p.code[i]; code2[i] = make_uint2(cw & 1023u, cw >> 14); }
   __syncthreads();
 
   float acc[V], R[NR][V];
@@ -167,7 +167,7 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
   const long long ntiles = p.row_mode ? p.n : (p.n + TILE - 1) / TILE;
   long long tile = blockIdx.x;
   TileCtx tc;
-  int loop_pc = 0;
+  const uint2* loop_ip = code2;
   auto set_tile = [&]() {
     if (p.row_mode) {
       tc.base = tile * (long long)p.cols;
@@ -277,13 +277,15 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
     else if constexpr (CS == P_SPILL) { VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, acc) }
   };
 
-  int pc = 0;
-  uint32_t w = code[0];
+  // Decoded instruction stream: one uint2 {case id, argument} per word, so that the decode of an
+  // instruction is a single 64-bit shared-memory load.  `ip` points at the entry after `w`.
+  const uint2* ip = code2 + 1;
+  uint2 w = code2[0];
   for (;;) {
-    uint32_t wn = code[pc + 1];  // fetched ahead of the dispatch below
-    ++pc;
-    const int cs = w & 1023u;
-    const uint32_t arg = w >> 14;
+    uint2 wn = *ip;   // fetched ahead of the dispatch below
+    ++ip;
+    const int cs = (int)w.x;
+    const uint32_t arg = w.y;
     if (cs < P_ULOAD) {
       asm volatile("// VMDISPATCH %0" ::"r"(cs));   // the build step puts an indexed jump here
       dispatch_tree<0, P_ULOAD>(cs, arg, exec);
@@ -297,17 +299,18 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
           }
         } break;
         case P_UCONST: {
-          if (tid == 0) U[arg] = __uint_as_float(wn);
-          ++pc;
-          wn = code[pc];
+          // the literal is the raw word that follows in the undecoded stream
+          if (tid == 0) U[arg] = __uint_as_float(p.code[(int)(ip - code2) - 1]);
+          wn = *ip;
+          ++ip;
         } break;
         case P_LOOP_BEGIN:
           __syncthreads();  // uniforms written by thread 0 are visible from here on
-          loop_pc = pc;
+          loop_ip = ip - 1;   // entry of the first body instruction (already in wn)
           break;
         case P_LOOP_END:
           tile += gridDim.x;
-          if (tile < ntiles) { set_tile(); pc = loop_pc; wn = code[pc]; }
+          if (tile < ntiles) { set_tile(); wn = *loop_ip; ip = loop_ip + 1; }
           break;
         case P_COLOUT: {
           float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
@@ -367,7 +370,7 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
 }
 
 size_t vm_smem_bytes(int n_code, int n_smem_slots) {
-  return (size_t)((n_code + 3) & ~3) * 4 + kMaxUniforms * 4 + 64 * 8 + (size_t)n_smem_slots * NV4 * NT * 16;
+  return (size_t)((n_code + 3) & ~3) * 8 + kMaxUniforms * 4 + 64 * 8 + (size_t)n_smem_slots * NV4 * NT * 16;
 }
 
 }  // namespace vm
