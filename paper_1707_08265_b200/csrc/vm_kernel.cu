@@ -168,6 +168,8 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
   long long tile = blockIdx.x;
   TileCtx tc;
   const uint2* loop_ip = code2;
+  const uint2* ip = code2;
+  uint2 wn = make_uint2(0u, 0u);
   auto set_tile = [&]() {
     if (p.row_mode) {
       tc.base = tile * (long long)p.cols;
@@ -275,65 +277,61 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
     else if constexpr (CS == P_GST) { store_operand(p.operand[arg], tc, tid, acc); }
     else if constexpr (CS == P_FILL) { VEC_LOAD(acc, reinterpret_cast<const float4*>(spill + (size_t)arg * TILE) + tid) }
     else if constexpr (CS == P_SPILL) { VEC_STORE(reinterpret_cast<float4*>(spill + (size_t)arg * TILE) + tid, acc) }
+    // ---- control and once-per-CTA instructions ----
+    else if constexpr (CS == P_ULOAD) {
+      if (tid == 0) {
+        const Operand& o = p.operand[arg >> 9];
+        U[arg & 511u] = o.dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(o.ptr))
+                                              : __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(o.ptr)) << 16);
+      }
+    }
+    else if constexpr (CS == P_UCONST) {
+      // the literal is the raw word that follows in the undecoded stream
+      if (tid == 0) U[arg] = __uint_as_float(p.code[(int)(ip - code2) - 1]);
+      wn = *ip;
+      ++ip;
+    }
+    else if constexpr (CS == P_LOOP_BEGIN) {
+      __syncthreads();    // uniforms written by thread 0 are visible from here on
+      loop_ip = ip - 1;   // entry of the first body instruction (already in wn)
+    }
+    else if constexpr (CS == P_LOOP_END) {
+      tile += gridDim.x;
+      if (tile < ntiles) { set_tile(); wn = *loop_ip; ip = loop_ip + 1; }
+    }
+    else if constexpr (CS == P_COLOUT) {
+      float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
+      FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = acc[j]; }
+    }
+    else if constexpr (CS == P_SCALOUT) {
+      double sum = 0.0;
+      FORV sum += (double)acc[j];
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+      if ((tid & 31) == 0) red[tid >> 5] = sum;
+      __syncthreads();
+      if (tid == 0) {
+        double tot = 0.0;
+        for (int i = 0; i < NT / 32; ++i) tot += red[i];
+        p.scalpart[(size_t)arg * gridDim.x + blockIdx.x] = tot;
+      }
+      __syncthreads();
+    }
+    else {  // P_END
+      asm volatile("exit;");
+    }
   };
 
   // Decoded instruction stream: one uint2 {case id, argument} per word, so that the decode of an
   // instruction is a single 64-bit shared-memory load.  `ip` points at the entry after `w`.
-  const uint2* ip = code2 + 1;
+  ip = code2 + 1;
   uint2 w = code2[0];
   for (;;) {
-    uint2 wn = *ip;   // fetched ahead of the dispatch below
+    wn = *ip;   // fetched ahead of the dispatch below
     ++ip;
-    const int cs = (int)w.x;
-    const uint32_t arg = w.y;
-    if (cs < P_ULOAD) {
-      asm volatile("// VMDISPATCH %0" ::"r"(cs));   // the build step puts an indexed jump here
-      dispatch_tree<0, P_ULOAD>(cs, arg, exec);
-    } else {
-      switch (cs) {  // control and once-per-CTA instructions
-        case P_ULOAD: {
-          if (tid == 0) {
-            const Operand& o = p.operand[arg >> 9];
-            U[arg & 511u] = o.dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(o.ptr))
-                                                  : __uint_as_float((unsigned)__ldg(reinterpret_cast<const unsigned short*>(o.ptr)) << 16);
-          }
-        } break;
-        case P_UCONST: {
-          // the literal is the raw word that follows in the undecoded stream
-          if (tid == 0) U[arg] = __uint_as_float(p.code[(int)(ip - code2) - 1]);
-          wn = *ip;
-          ++ip;
-        } break;
-        case P_LOOP_BEGIN:
-          __syncthreads();  // uniforms written by thread 0 are visible from here on
-          loop_ip = ip - 1;   // entry of the first body instruction (already in wn)
-          break;
-        case P_LOOP_END:
-          tile += gridDim.x;
-          if (tile < ntiles) { set_tile(); wn = *loop_ip; ip = loop_ip + 1; }
-          break;
-        case P_COLOUT: {
-          float* out = p.colpart + ((size_t)arg * gridDim.x + blockIdx.x) * p.cols;
-          FORV { const int c = lane_pos(tid, j); if (c < p.cols) out[c] = acc[j]; }
-        } break;
-        case P_SCALOUT: {
-          double sum = 0.0;
-          FORV sum += (double)acc[j];
-#pragma unroll
-          for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
-          if ((tid & 31) == 0) red[tid >> 5] = sum;
-          __syncthreads();
-          if (tid == 0) {
-            double tot = 0.0;
-            for (int i = 0; i < NT / 32; ++i) tot += red[i];
-            p.scalpart[(size_t)arg * gridDim.x + blockIdx.x] = tot;
-          }
-          __syncthreads();
-        } break;
-        default:  // P_END and anything unknown
-          return;
-      }
-    }
+    const int cs = min((int)w.x, (int)P_END);     // anything unknown ends the program
+    asm volatile("// VMDISPATCH %0" ::"r"(cs));   // the build step puts an indexed jump here
+    dispatch_tree<0, P_COUNT_>(cs, w.y, exec);
     w = wn;
   }
 }
