@@ -438,6 +438,12 @@ struct Gen {
     seg->code.push_back(encode(P_END, 0, 0));
     seg->code.push_back(encode(P_END, 0, 0));  // the interpreter prefetches one word ahead
     seg->n_instr_body = (int)body.size();
+    // the kernel jumps through a table indexed by the case id without a range check
+    for (size_t i = 0; i < seg->code.size(); ++i) {
+      const int cs = (int)(seg->code[i] & 1023u);
+      if (cs >= P_COUNT_) { set_error("graph VM: internal error, invalid case id %d", cs); return DRAGON_ERR_UNSUPPORTED; }
+      if (cs == P_UCONST) ++i;  // the next word is a literal
+    }
     if ((int)seg->code.size() > kVmCodeMaxWords) { set_error("graph VM: instruction stream too long (%d words)", (int)seg->code.size()); return DRAGON_ERR_UNSUPPORTED; }
     if ((int)seg->operand_mem.size() > kMaxOperands) { set_error("graph VM: too many memory operands in one segment"); return DRAGON_ERR_UNSUPPORTED; }
     return DRAGON_OK;

@@ -329,7 +329,7 @@ __global__ void __launch_bounds__(NT, 1) vm_kernel(const __grid_constant__ Param
   for (;;) {
     wn = *ip;   // fetched ahead of the dispatch below
     ++ip;
-    const int cs = min((int)w.x, (int)P_END);     // anything unknown ends the program
+    const int cs = (int)w.x;                      // < P_COUNT_: launch_vm() validates the stream once
     asm volatile("// VMDISPATCH %0" ::"r"(cs));   // the build step puts an indexed jump here
     dispatch_tree<0, P_COUNT_>(cs, w.y, exec);
     w = wn;
