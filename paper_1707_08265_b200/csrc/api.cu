@@ -15,7 +15,8 @@ cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int row
 cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
                            const float* dl_ptr, float dl_imm, int* status, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cudaStream_t st);
-int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, int* status, cudaStream_t st);
+int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
+                     cudaStream_t st);
 }  // namespace dragon
 
 using namespace dragon;
@@ -344,7 +345,8 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
       }
       case ST_GEMM: {
         const MemRef &A = P.mems[s.mA], &C = P.mems[s.mC];
-        int rc = launch_gemm_bf16(ptr[s.mA], ptr[s.mB], ptr[s.mC], C.dtype, (int)C.shape.d[0], (int)C.shape.d[1], (int)A.shape.d[1], status, st);
+        const int kc = (int)(s.tA ? A.shape.d[0] : A.shape.d[1]);
+        int rc = launch_gemm_bf16(ptr[s.mA], ptr[s.mB], ptr[s.mC], C.dtype, (int)C.shape.d[0], (int)C.shape.d[1], kc, s.tA, s.tB, status, st);
         if (rc != DRAGON_OK) return rc;
         break;
       }

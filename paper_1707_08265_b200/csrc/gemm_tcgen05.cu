@@ -82,9 +82,22 @@ __device__ __forceinline__ uint64_t make_smem_desc(uint32_t addr) {
   d |= (uint64_t)2 << 61;                            // SWIZZLE_128B
   return d;
 }
-// instruction descriptor: D = f32, A = B = bf16, both K-major, M x N
-constexpr uint32_t make_idesc(int m, int n) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+// the same for an MN-major operand (the memory matrix is [K, MN] row-major): the tile is stored as
+// chunks of 64 MN-elements; inside a chunk every K-row is one 128-byte swizzle row, 8 K-rows form a
+// 1024-byte group (stride byte offset) and chunks are 8192 bytes apart (leading byte offset)
+__device__ __forceinline__ uint64_t make_smem_desc_mn(uint32_t addr) {
+  uint64_t d = 0;
+  d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+  d |= (uint64_t)(8192 >> 4) << 16;
+  d |= (uint64_t)(1024 >> 4) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// instruction descriptor: D = f32, A = B = bf16, M x N; bits 15 / 16 select MN-major A / B
+constexpr uint32_t make_idesc(int m, int n, bool a_mn, bool b_mn) {
+  return (1u << 4) | (1u << 7) | (1u << 10) | ((a_mn ? 1u : 0u) << 15) | ((b_mn ? 1u : 0u) << 16) |
+         ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
 __device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
@@ -132,6 +145,7 @@ __device__ __forceinline__ void tile_coords(int t, int tiles_m, int tiles_n, int
   *tn = r / rows;
 }
 
+template <bool kAMn, bool kBMn>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b, const GemmArgs g) {
   extern __shared__ unsigned char gemm_smem_raw[];
@@ -176,8 +190,18 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
           if (!mbar_wait(bar_empty + 8 * s, (it & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
           mbar_expect_tx(bar_full + 8 * s, kStageBytes);
           const uint32_t dst = tiles + (uint32_t)s * kStageBytes;
-          tma_load_2d(dst, &tmap_a, kt * kTileK, tm * kTileM, bar_full + 8 * s);
-          tma_load_2d(dst + kStageBytesA, &tmap_b, kt * kTileK, tn * kTileN, bar_full + 8 * s);
+          if (!kAMn) {
+            tma_load_2d(dst, &tmap_a, kt * kTileK, tm * kTileM, bar_full + 8 * s);
+          } else {  // boxes of 64 MN-elements x 64 K-rows, one per chunk
+#pragma unroll
+            for (int c = 0; c < kTileM / 64; ++c) tma_load_2d(dst + c * 8192, &tmap_a, tm * kTileM + c * 64, kt * kTileK, bar_full + 8 * s);
+          }
+          if (!kBMn) {
+            tma_load_2d(dst + kStageBytesA, &tmap_b, kt * kTileK, tn * kTileN, bar_full + 8 * s);
+          } else {
+#pragma unroll
+            for (int c = 0; c < kTileN / 64; ++c) tma_load_2d(dst + kStageBytesA + c * 8192, &tmap_b, tn * kTileN + c * 64, kt * kTileK, bar_full + 8 * s);
+          }
         }
       }
       if (*abort_flag) {  // let the copies that are still in flight land before the CTA goes away
@@ -187,7 +211,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
     }
   } else if (warp == 1) {
     if (lane == 0) {  // MMA issuer
-      constexpr uint32_t idesc = make_idesc(kTileM, kTileN);
+      constexpr uint32_t idesc = make_idesc(kTileM, kTileN, kAMn, kBMn);
       int consumed = 0, local = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
@@ -201,11 +225,13 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
           if (!mbar_wait(bar_full + 8 * s, it & 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_addr = tiles + (uint32_t)s * kStageBytes, b_addr = a_addr + kStageBytesA;
-          const uint64_t a_desc = make_smem_desc(a_addr), b_desc = make_smem_desc(b_addr);
+          const uint64_t a_desc = kAMn ? make_smem_desc_mn(a_addr) : make_smem_desc(a_addr);
+          const uint64_t b_desc = kBMn ? make_smem_desc_mn(b_addr) : make_smem_desc(b_addr);
 #pragma unroll
           for (int k = 0; k < kTileK / kUmmaK; ++k) {
-            // advancing 16 elements along K inside the swizzle row = 32 bytes = 2 descriptor units
-            umma_f16(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+            // 16 elements along K: K-major = 32 bytes inside the swizzle row (2 descriptor units),
+            // MN-major = two 8-row groups = 2048 bytes (128 units)
+            umma_f16(d_tmem, a_desc + (kAMn ? 128 : 2) * k, b_desc + (kBMn ? 128 : 2) * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
           }
           umma_commit(bar_empty + 8 * s);   // the stage is free once these MMAs have read it
         }
@@ -294,6 +320,8 @@ EncodeTiledFn encode_fn() {
 }
 
 // row-major bf16 [rows, cols] viewed as a 2-D tensor map with boxes of box_rows x 64 elements
+// (K-major operand: rows = M or N, cols = K, box_rows = tile height; MN-major operand: rows = K,
+// cols = M or N, box_rows = 64)
 bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
@@ -307,19 +335,25 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_ro
 
 }  // namespace
 
-int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, int* status, cudaStream_t st) {
-  if (M <= 0 || N <= 0 || K <= 0 || (K & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
-    set_error("InnerProduct: K must be a multiple of 8 and all operands 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
+// C[M,N] = opA * opB^T with K the contraction length.  a_mn / b_mn: the operand is given as the
+// row-major matrix [K, M] (resp. [K, N]) instead of [M, K] (resp. [N, K]).
+int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
+                     cudaStream_t st) {
+  const int a_inner = a_mn ? M : K, b_inner = b_mn ? N : K;
+  if (M <= 0 || N <= 0 || K <= 0 || (a_inner & 7) || (b_inner & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
+    set_error("InnerProduct: the contiguous extent of every operand must be a multiple of 8 and all pointers 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
     return DRAGON_ERR_UNSUPPORTED;
   }
   CUtensorMap ta, tb;
-  if (!make_tmap(&ta, A, M, K, kTileM) || !make_tmap(&tb, B, N, K, kTileN)) {
+  const bool ok_a = a_mn ? make_tmap(&ta, A, K, M, 64) : make_tmap(&ta, A, M, K, kTileM);
+  const bool ok_b = b_mn ? make_tmap(&tb, B, K, N, 64) : make_tmap(&tb, B, N, K, kTileN);
+  if (!ok_a || !ok_b) {
     set_error("InnerProduct: cannot encode the TMA descriptors (no CUDA driver?)");
     return DRAGON_ERR_CUDA;
   }
-  static std::once_flag once;
-  static cudaError_t attr_err = cudaSuccess;
-  std::call_once(once, [] { attr_err = cudaFuncSetAttribute(gemm_bf16_tcgen05, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem); });
+  auto kern = a_mn ? gemm_bf16_tcgen05<true, true> : (b_mn ? gemm_bf16_tcgen05<false, true> : gemm_bf16_tcgen05<false, false>);
+  if (a_mn && !b_mn) { set_error("InnerProduct: this operand layout combination is not built"); return DRAGON_ERR_UNSUPPORTED; }
+  cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
   if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
   const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
   GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status};
@@ -329,7 +363,7 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
     if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0) sm_count = kDefaultSmCount;
   }
   const int grid = std::min(tiles_m * tiles_n, sm_count);   // persistent CTAs, one per SM
-  gemm_bf16_tcgen05<<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, g);
+  kern<<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, g);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) { set_error("InnerProduct: launch failed: %s", cudaGetErrorString(e)); return DRAGON_ERR_CUDA; }
   return DRAGON_OK;

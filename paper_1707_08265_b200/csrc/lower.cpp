@@ -24,7 +24,6 @@ struct Lowerer {
   std::vector<int> fval;                      // forward tensor -> value id
   std::vector<std::map<int, int>> gval;       // per stage: tensor -> gradient value id
   std::vector<int> fetch_of;                  // tensor -> fetch position or -1
-  std::map<int, int> transposed;              // memref -> memref of its transpose
   std::map<std::pair<int, int>, int> materialised;   // (value, dtype) -> memref
   std::vector<std::map<int, int>> pending;    // per stage: tensor -> gradient contributions still to come
   int err = DRAGON_OK;
@@ -104,21 +103,11 @@ struct Lowerer {
     materialised[key] = m;
     return m;
   }
-  int transpose_of(int mem) {
-    auto it = transposed.find(mem);
-    if (it != transposed.end()) return it->second;
-    Shape s = plan->mems[mem].shape, t;
-    t.rank = 2; t.d[0] = s.d[1]; t.d[1] = s.d[0];
-    int m = new_mem(MEM_WORK, -1, DRAGON_BF16, t);
-    Item x; x.kind = IT_TRANSPOSE; x.mA = mem; x.mC = m;
-    items.push_back(x);
-    transposed[mem] = m;
-    return m;
-  }
-  int gemm(int mA, int mB, int out_where, int out_index, int out_dtype) {
-    Shape s; s.rank = 2; s.d[0] = plan->mems[mA].shape.d[0]; s.d[1] = plan->mems[mB].shape.d[0];
+  // C = opA * opB^T; tA / tB: the memory matrix of the operand is its transpose ([K, M] / [K, N])
+  int gemm(int mA, int mB, int out_where, int out_index, int out_dtype, bool tA = false, bool tB = false) {
+    Shape s; s.rank = 2; s.d[0] = plan->mems[mA].shape.d[tA ? 1 : 0]; s.d[1] = plan->mems[mB].shape.d[tB ? 1 : 0];
     int mC = new_mem(out_where, out_index, out_dtype, s);
-    Item x; x.kind = IT_GEMM; x.mA = mA; x.mB = mB; x.mC = mC;
+    Item x; x.kind = IT_GEMM; x.mA = mA; x.mB = mB; x.mC = mC; x.tA = tA; x.tB = tB;
     items.push_back(x);
     return mC;
   }
@@ -234,13 +223,13 @@ struct Lowerer {
           // a gradient that the caller asked for stays fp32
           const auto& wr = g.stages[s].wrts;
           const bool wanted = std::find(wr.begin(), wr.end(), op.in[0]) != wr.end();
-          int mC = gemm(mdY, transpose_of(mW), MEM_WORK, -1,
-                        (g.tensors[op.in[0]].dtype == DRAGON_BF16 && !wanted) ? DRAGON_BF16 : DRAGON_F32);
+          int mC = gemm(mdY, mW, MEM_WORK, -1,
+                        (g.tensors[op.in[0]].dtype == DRAGON_BF16 && !wanted) ? DRAGON_BF16 : DRAGON_F32, false, true);
           add(0, new_val(VK_MEM, plan->mems[mC].shape, mC));
         }
         if (want[1]) {  // dW[N,K] = dY^T[N,M] * X[M,K]
           int mX = materialise(in(0), DRAGON_BF16, DRAGON_BF16);
-          int mC = gemm(transpose_of(mdY), transpose_of(mX), MEM_WORK, -1, DRAGON_F32);
+          int mC = gemm(mdY, mX, MEM_WORK, -1, DRAGON_F32, true, true);
           add(1, new_val(VK_MEM, plan->mems[mC].shape, mC));
         }
         break;
@@ -484,7 +473,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     Step st;
     st.kind = it.kind == IT_GEMM ? ST_GEMM : it.kind == IT_TRANSPOSE ? ST_TRANSPOSE : it.kind == IT_SCE_FWD ? ST_SCE_FWD
               : it.kind == IT_SCE_BWD ? ST_SCE_BWD : ST_COPY;
-    st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.scale = it.scale;
+    st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
     plan->steps.push_back(st);
   }
   for (size_t s = 0; s < seg_items.size(); ++s) {
@@ -553,8 +542,9 @@ std::string describe_plan(const Plan& p) {
         break;
       }
       case ST_GEMM:
-        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
-                 (long long)p.mems[st.mA].shape.d[1], p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
+        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
+                 (long long)p.mems[st.mA].shape.d[st.tA ? 0 : 1], st.tA ? " A^T" : "", st.tB ? " B^T" : "",
+                 p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
         break;
       case ST_TRANSPOSE:
         snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);

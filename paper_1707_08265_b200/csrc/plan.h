@@ -59,6 +59,7 @@ struct Item {
   // SCE: A = logits, B = labels, C = out, D = scalar dL (gradient)
   int mA = -1, mB = -1, mC = -1, mD = -1;
   float scale = 1.f;                       // SCE_BWD: immediate dL when mD < 0
+  bool tA = false, tB = false;             // GEMM: operand given transposed ([K, M] / [K, N] row-major)
   bool live = false;
   int segment = -1;
 };
@@ -92,6 +93,7 @@ struct Step {
   int seg = -1;                          // ST_VM
   int mA = -1, mB = -1, mC = -1, mD = -1;
   float scale = 1.f;
+  bool tA = false, tB = false;
   size_t scratch_off = 0;                // SCE_FWD: per-row losses
 };
 
