@@ -15,6 +15,7 @@ import sys
 LABEL = re.compile(r"^\s*(\$?[A-Za-z_][\w$]*):\s*$")
 BRANCH = re.compile(r"^\s*(@!?%p\d+\s+)?(bra(\.uni)?|brx\.idx|ret|exit|trap)\b")
 # compares, branches, and integer arithmetic on the case id (the compiler narrows and offsets it)
+SPECIAL = re.compile(r"^\s*mov\.u32\s+(%r\d+),\s*%(tid|ctaid|ntid|nctaid)\.[xyz];")
 TREE_OK = re.compile(r"^\s*(@!?%p\d+\s+)?(setp\.|bra\b|bra\.uni\b|cvt\.[us]\d+\.[us]\d+\s|and\.b(16|32)\s|(add|sub)\.s(16|32)\s|shr\.[us]32\s)")
 
 
@@ -76,6 +77,12 @@ def rewrite(ptx, kernel_substr="vm_kernel", thread=True):
         while not (LABEL.match(lines[j]) or (is_code(lines[j]) and BRANCH.match(lines[j]))):
             j -= 1
         leaf_starts.add(j if LABEL.match(lines[j]) else j + 1)
+    hoisted = set()
+
+    def n_defs(reg):
+        pat = re.compile(r"^\s*(@!?%p\d+\s+)?[a-z][\w.]*\s+(\{[^}]*)?" + re.escape(reg) + r"\b[,;}]")
+        return sum(1 for j in range(body_lo, body_hi) if pat.match(lines[j]))
+
     seen, work = set(), [disp + 1]
     while work:
         i = work.pop()
@@ -88,8 +95,11 @@ def rewrite(ptx, kernel_substr="vm_kernel", thread=True):
             l = lines[i]
             if "// VMLEAF" in l:
                 break
-            if is_code(l):
-                if not TREE_OK.match(l):
+            if is_code(l) and i not in hoisted:
+                m = SPECIAL.match(l)
+                if m and n_defs(m.group(1)) == 1:
+                    hoisted.add(i)      # a re-read of a special register: defined once, so it can move to the entry
+                elif not TREE_OK.match(l):
                     raise RuntimeError("dispatch tree holds other work: %r (line %d)" % (l.strip(), i))
                 m = re.search(r"bra(\.uni)?\s+(\$?[\w$]+);", l)
                 if m:
@@ -116,7 +126,13 @@ def rewrite(ptx, kernel_substr="vm_kernel", thread=True):
     # rewrite
     out = []
     n_threaded = 0
+    first_code = next(i for i in range(body_lo + 1, body_hi) if is_code(lines[i]))
+    head = [l for l in head if l not in [lines[j] for j in hoisted]]
     for i, l in enumerate(lines):
+        if i == first_code:
+            out.extend(lines[j] for j in sorted(hoisted))
+        if i in hoisted:
+            continue
         if i in inserts:
             out.append(inserts[i] + ":")
         if i == disp:
