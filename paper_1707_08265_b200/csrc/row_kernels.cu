@@ -32,7 +32,37 @@ __device__ __forceinline__ float block_reduce(float v, float* sh) {
   return r;
 }
 
-// mode 0: rowloss[m] = logsumexp(z[m,:]) - z[m,label];  mode 1: dz[m,j] = dL/M * (softmax - onehot)
+// eight consecutive logits at element index i (a multiple of 8) as floats
+__device__ __forceinline__ void load8(const void* z, int dtype, size_t i, float* v) {
+  if (dtype == DRAGON_F32) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(z) + i));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(reinterpret_cast<const float*>(z) + i) + 1);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+  } else {
+    const uint4 u = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(z) + i));
+    v[0] = __uint_as_float(u.x << 16); v[1] = __uint_as_float(u.x & 0xffff0000u);
+    v[2] = __uint_as_float(u.y << 16); v[3] = __uint_as_float(u.y & 0xffff0000u);
+    v[4] = __uint_as_float(u.z << 16); v[5] = __uint_as_float(u.z & 0xffff0000u);
+    v[6] = __uint_as_float(u.w << 16); v[7] = __uint_as_float(u.w & 0xffff0000u);
+  }
+}
+__device__ __forceinline__ void store8(void* z, int dtype, size_t i, const float* v) {
+  if (dtype == DRAGON_F32) {
+    float4* p = reinterpret_cast<float4*>(reinterpret_cast<float*>(z) + i);
+    p[0] = make_float4(v[0], v[1], v[2], v[3]);
+    p[1] = make_float4(v[4], v[5], v[6], v[7]);
+  } else {
+    uint4 u;
+    u.x = vmmath::bf16_bits(v[0]) | (vmmath::bf16_bits(v[1]) << 16);
+    u.y = vmmath::bf16_bits(v[2]) | (vmmath::bf16_bits(v[3]) << 16);
+    u.z = vmmath::bf16_bits(v[4]) | (vmmath::bf16_bits(v[5]) << 16);
+    u.w = vmmath::bf16_bits(v[6]) | (vmmath::bf16_bits(v[7]) << 16);
+    *reinterpret_cast<uint4*>(reinterpret_cast<unsigned short*>(z) + i) = u;
+  }
+}
+
+// mode 0: rowloss[m] = logsumexp(z[m,:]) - z[m,label];  mode 1: dz[m,j] = dL/M * (softmax - onehot).
+// Rows whose length is a multiple of 8 are read and written 8 elements (16 or 32 bytes) per thread.
 template <int kMode>
 __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdtype, const int* labels, int rows, int cols,
                                                           float* rowloss, void* dz, int dzdtype, const float* dl_ptr,
@@ -40,11 +70,30 @@ __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdt
   __shared__ float sh[kRowThreads / 32];
   const int m = blockIdx.x;
   const size_t off = (size_t)m * cols;
+  const bool vec = (cols & 7) == 0;
   float mx = -INFINITY;
-  for (int j = threadIdx.x; j < cols; j += kRowThreads) mx = fmaxf(mx, load_logit(z, zdtype, off + j));
+  if (vec) {
+    for (int j = threadIdx.x * 8; j < cols; j += kRowThreads * 8) {
+      float v[8];
+      load8(z, zdtype, off + j, v);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mx = fmaxf(mx, v[e]);
+    }
+  } else {
+    for (int j = threadIdx.x; j < cols; j += kRowThreads) mx = fmaxf(mx, load_logit(z, zdtype, off + j));
+  }
   mx = block_reduce<true>(mx, sh);
   float se = 0.f;
-  for (int j = threadIdx.x; j < cols; j += kRowThreads) se += vmmath::exp_wide(load_logit(z, zdtype, off + j) - mx);
+  if (vec) {
+    for (int j = threadIdx.x * 8; j < cols; j += kRowThreads * 8) {
+      float v[8];
+      load8(z, zdtype, off + j, v);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) se += vmmath::exp_wide(v[e] - mx);
+    }
+  } else {
+    for (int j = threadIdx.x; j < cols; j += kRowThreads) se += vmmath::exp_wide(load_logit(z, zdtype, off + j) - mx);
+  }
   se = block_reduce<false>(se, sh);
   const int lab = __ldg(labels + m);
   const bool ok = lab >= 0 && lab < cols;
@@ -54,12 +103,26 @@ __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdt
   } else {
     const float dl = dl_ptr ? __ldg(dl_ptr) : dl_imm;
     const float sc = dl / (float)rows, inv = 1.f / se;
-    for (int j = threadIdx.x; j < cols; j += kRowThreads) {
-      float g = vmmath::exp_wide(load_logit(z, zdtype, off + j) - mx) * inv;
-      if (ok && j == lab) g -= 1.f;
-      g = ok ? g * sc : 0.f;
-      if (dzdtype == DRAGON_F32) reinterpret_cast<float*>(dz)[off + j] = g;
-      else reinterpret_cast<unsigned short*>(dz)[off + j] = (unsigned short)vmmath::bf16_bits(g);
+    if (vec) {
+      for (int j = threadIdx.x * 8; j < cols; j += kRowThreads * 8) {
+        float v[8];
+        load8(z, zdtype, off + j, v);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float g = vmmath::exp_wide(v[e] - mx) * inv;
+          if (j + e == lab) g -= 1.f;
+          v[e] = ok ? g * sc : 0.f;
+        }
+        store8(dz, dzdtype, off + j, v);
+      }
+    } else {
+      for (int j = threadIdx.x; j < cols; j += kRowThreads) {
+        float g = vmmath::exp_wide(load_logit(z, zdtype, off + j) - mx) * inv;
+        if (ok && j == lab) g -= 1.f;
+        g = ok ? g * sc : 0.f;
+        if (dzdtype == DRAGON_F32) reinterpret_cast<float*>(dz)[off + j] = g;
+        else reinterpret_cast<unsigned short*>(dz)[off + j] = (unsigned short)vmmath::bf16_bits(g);
+      }
     }
   }
 }

@@ -82,3 +82,16 @@ def test_mlp_out_of_range_label_sets_status_and_does_not_fault():
     o = [torch.empty(tuple(g.shape(t)), dtype=torch.float32, device="cuda") for t in outs]
     fn.run_torch(dev, o)
     assert fn.status() == B.ERR_INVALID_ARG
+
+
+def test_unsupported_contraction_length_is_an_error_not_a_fault():
+    from paper_1707_08265_b200 import binding as B
+    from test_gpu_vm import to_dev
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [16, 12], "bf16"); W = gd.tensor("W", [8, 12], "bf16")     # K = 12 is not a multiple of 8
+    Y = gd.op("InnerProduct", [X, W], "Y", [16, 8], "f32")
+    f = B.Graph.from_desc(gd.desc).function([X, W], [Y])
+    out = torch.zeros(16, 8, device="cuda")
+    with pytest.raises(B.DragonError) as e:
+        f.run_torch([to_dev(np.zeros((16, 12), np.float32), "bf16"), to_dev(np.zeros((8, 12), np.float32), "bf16")], [out])
+    assert e.value.code == B.ERR_UNSUPPORTED

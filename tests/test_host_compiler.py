@@ -151,3 +151,24 @@ def test_long_chain_prunes_in_linear_time_without_recursion():
         times.append(time.perf_counter() - t0)
         assert ok == 0
     assert times[1] < 12 * times[0] + 0.05
+
+
+def test_limits_are_reported_not_faulted():
+    # a row reduction over rows longer than one tile is refused at compile time
+    g = B.Graph()
+    x = g.add_tensor("x", B.F32, [4, 5000])
+    y = g.add_tensor("y", B.F32, [4, 5000])
+    g.add_op(B.OPS["Sum"], [x], [y])
+    with pytest.raises(B.DragonError):
+        g.function([x], [y])
+    assert b"rows longer than" in B.lib().dragon_last_error()
+    # the same shape without a row operation is a flat elementwise function and compiles
+    g2 = B.Graph()
+    x2 = g2.add_tensor("x", B.F32, [4, 5000])
+    y2 = g2.add_tensor("y", B.F32, [4, 5000])
+    g2.add_op(B.OPS["Tanh"], [x2], [y2])
+    f = g2.function([x2], [y2])
+    assert "flat n=20000" in f.describe()
+    # fetching the same tensor twice is refused
+    with pytest.raises(B.DragonError):
+        g2.function([x2], [y2, y2])
