@@ -37,12 +37,39 @@ def build(verbose=False, force=False, ptxas_info=False):
                 print(" ".join(cmd), flush=True)
             subprocess.run(cmd, check=True)
     objs.append(_jump_table_object(objdir, headers, verbose, force or ptxas_info))
+    objs.append(_generated_kernel_object(objdir, verbose, force or ptxas_info))
     if force or _stale(LIB, objs):
         cmd = [NVCC, "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"]
         if verbose:
             print(" ".join(cmd), flush=True)
         subprocess.run(cmd, check=True)
     return LIB
+
+
+def _embed(cpp, obj, symbol, data, what):
+    with open(cpp, "w") as fh:
+        fh.write("// generated: %s\n" % what)
+        fh.write('extern "C" const unsigned long %s_size = %d;\n' % (symbol, len(data)))
+        fh.write('extern "C" const unsigned char %s[] = {' % symbol)
+        fh.write(",".join(str(b) for b in data) if data else "0")
+        fh.write("};\n")
+    subprocess.run(["g++", "-O1", "-fPIC", "-c", cpp, "-o", obj], check=True)
+
+
+def _generated_kernel_object(objdir, verbose, force):
+    """vm_ptxgen.py -> PTX -> cubin of the graph-VM kernel, embedded as a byte array."""
+    from paper_1707_08265_b200 import vm_ptxgen
+    ptx, cubin = os.path.join(objdir, "vm_gen.ptx"), os.path.join(objdir, "vm_gen.cubin")
+    cpp, obj = os.path.join(objdir, "vm_gen_cubin.cpp"), os.path.join(objdir, "vm_gen_cubin.o")
+    if not (force or _stale(obj, [vm_ptxgen.__file__])):
+        return obj
+    open(ptx, "w").write(vm_ptxgen.generate())
+    ptxas = os.path.join(os.path.dirname(NVCC), "ptxas")
+    r = subprocess.run([ptxas, "-arch=sm_100a", "-O3", "-v", ptx, "-o", cubin], check=True, capture_output=True, text=True)
+    if verbose:
+        print(r.stderr, flush=True)
+    _embed(cpp, obj, "dragon_vm_gen_cubin", open(cubin, "rb").read(), "cubin of the PTX-generated VM kernel")
+    return obj
 
 
 def _jump_table_object(objdir, headers, verbose, force):

@@ -368,7 +368,7 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
 }
 
 size_t vm_smem_bytes(int n_code, int n_smem_slots) {
-  return (size_t)((n_code + 3) & ~3) * 8 + kMaxUniforms * 4 + 64 * 8 + (size_t)n_smem_slots * NV4 * NT * 16;
+  return (size_t)((n_code + 3) & ~3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)n_smem_slots * NV4 * NT * 16;
 }
 
 }  // namespace vm
@@ -379,6 +379,8 @@ size_t vm_smem_bytes(int n_code, int n_smem_slots) {
 // ptx_jumptable.py); size 0 when that step refused
 extern "C" const unsigned long dragon_vm_jt_cubin_size;
 extern "C" const unsigned char dragon_vm_jt_cubin[];
+extern "C" const unsigned long dragon_vm_gen_cubin_size;
+extern "C" const unsigned char dragon_vm_gen_cubin[];
 
 namespace dragon {
 
@@ -390,6 +392,16 @@ static const void* vm_entry() {
   std::call_once(once, [] {
     entry = reinterpret_cast<const void*>(vm::vm_kernel);
     const char* mode = std::getenv("DRAGON_VM_DISPATCH");
+    if (mode && std::string(mode) == "gen") {
+      cudaLibrary_t lib;
+      cudaKernel_t k;
+      if (cudaLibraryLoadData(&lib, dragon_vm_gen_cubin, nullptr, nullptr, 0, nullptr, nullptr, 0) == cudaSuccess &&
+          cudaLibraryGetKernel(&k, lib, "dragon_vm_r7") == cudaSuccess) {
+        entry = reinterpret_cast<const void*>(k);
+        return;
+      }
+      cudaGetLastError();
+    }
     if (dragon_vm_jt_cubin_size == 0 || (mode && std::string(mode) == "tree")) return;
     cudaLibrary_t lib;
     cudaKernel_t k;

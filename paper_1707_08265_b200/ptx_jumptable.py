@@ -137,11 +137,11 @@ def rewrite(ptx, kernel_substr="vm_kernel", thread=True):
             out.append(inserts[i] + ":")
         if i == disp:
             out.append("\tVMJT: .branchtargets " + ", ".join(leaf_label[n] for n in range(n_leaves)) + ";")
-            out.append("\tbrx.idx " + reg + ", VMJT;")
+            out.append("\tbrx.idx.uni " + reg + ", VMJT;")
             continue
         if thread and body_lo < i < body_hi and back.match(l) and i > disp:
             out.extend(head)
-            out.append("\tbrx.idx " + reg + ", VMJT;")
+            out.append("\tbrx.idx.uni " + reg + ", VMJT;")
             n_threaded += 1
             continue
         out.append(l)
