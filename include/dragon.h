@@ -130,10 +130,10 @@ int dragon_function_num_launches(const dragon_function_t* f);
 int dragon_function_describe(const dragon_function_t* f, char* buf, int cap);
 
 /* Introspection of one graph-VM step of the plan (step index = line of dragon_function_describe),
- * for tools and tests that check the emitted instruction stream without a GPU.  info[0..8] =
+ * for tools and tests that check the emitted instruction stream without a GPU.  info[0..9] =
  * {number of code words, row mode (0/1), cols, number of operands, spill slots, shared-memory
  * slots, rows or elements (low 32 bits), rows or elements (high 32 bits), number of reduced
- * outputs}; code (may be NULL)
+ * outputs, register slots of the kernel build the program is for (3 dense, 7 wide)}; code (may be NULL)
  * receives up to cap_code words (encoding: csrc/vm_isa.h); operands (may be NULL) receives up to
  * cap_operands quadruples {where (0 feed, 1 fetch, 2 workspace), position or workspace offset / 256,
  * kind (0 full, 1 row, 2 scalar), dtype}; reduced (may be NULL) receives up to cap_reduced triples

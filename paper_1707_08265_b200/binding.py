@@ -213,7 +213,7 @@ class Function:
 
     def vm_step(self, step):
         """Instruction stream and operand table of a graph-VM step, or None for another kind of step."""
-        info = (_c.c_int64 * 9)()
+        info = (_c.c_int64 * 10)()
         if lib().dragon_function_vm_step(self.h, step, info, None, 0, None, 0, None, 0) < 0:
             return None
         code = (_c.c_uint32 * max(1, info[0]))()
@@ -221,7 +221,7 @@ class Function:
         red = (_c.c_int64 * max(3, 3 * info[8]))()
         lib().dragon_function_vm_step(self.h, step, info, code, info[0], ops, info[3], red, info[8])
         return {"code": list(code[:info[0]]), "row_mode": bool(info[1]), "cols": info[2], "n": info[6] | (info[7] << 32),
-                "n_spill": info[4], "n_smem": info[5],
+                "n_spill": info[4], "n_smem": info[5], "n_regs": info[9],
                 "operands": [tuple(ops[4 * i:4 * i + 4]) for i in range(info[3])],
                 "reduced": [tuple(red[3 * i:3 * i + 3]) for i in range(info[8])]}
 

@@ -8,7 +8,7 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdragon.so")
-SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "api.cu", "vm_kernel.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
+SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "api.cu", "vm_launch.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr", "-Xcompiler", "-Wall"] + os.environ.get("DRAGON_NVCC_DEFS", "").split()
@@ -36,7 +36,6 @@ def build(verbose=False, force=False, ptxas_info=False):
             if verbose:
                 print(" ".join(cmd), flush=True)
             subprocess.run(cmd, check=True)
-    objs.append(_jump_table_object(objdir, headers, verbose, force or ptxas_info))
     objs.append(_generated_kernel_object(objdir, verbose, force or ptxas_info))
     if force or _stale(LIB, objs):
         cmd = [NVCC, "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"]
@@ -69,38 +68,6 @@ def _generated_kernel_object(objdir, verbose, force):
     if verbose:
         print(r.stderr, flush=True)
     _embed(cpp, obj, "dragon_vm_gen_cubin", open(cubin, "rb").read(), "cubin of the PTX-generated VM kernel")
-    return obj
-
-
-def _jump_table_object(objdir, headers, verbose, force):
-    """vm_kernel.cu -> PTX -> indexed-jump dispatch (ptx_jumptable.py) -> cubin, embedded as a byte array.
-    If the rewrite refuses, the array is empty and the library keeps the compiled-in tree kernel."""
-    from paper_1707_08265_b200 import ptx_jumptable
-    src = os.path.join(CSRC, "vm_kernel.cu")
-    ptx, jt = os.path.join(objdir, "vm_kernel.ptx"), os.path.join(objdir, "vm_kernel_jt.ptx")
-    cubin, cpp, obj = os.path.join(objdir, "vm_kernel_jt.cubin"), os.path.join(objdir, "vm_jt_cubin.cpp"), os.path.join(objdir, "vm_jt_cubin.o")
-    if not (force or _stale(obj, [src, ptx_jumptable.__file__] + headers)):
-        return obj
-    data = b""
-    try:
-        arch = [a for a in FLAGS if not a.startswith("-Xcompiler") and a not in ("-fPIC", "-Wall")]
-        subprocess.run([NVCC] + arch + ["-ptx", src, "-o", ptx], check=True)
-        text, n = ptx_jumptable.rewrite(open(ptx).read())
-        open(jt, "w").write(text)
-        ptxas = os.path.join(os.path.dirname(NVCC), "ptxas")
-        r = subprocess.run([ptxas, "-arch=sm_100a", "-O3", "-lineinfo", "-v", jt, "-o", cubin], check=True, capture_output=True, text=True)
-        if verbose:
-            print("jump table over %d leaves\n%s" % (n, r.stderr), flush=True)
-        data = open(cubin, "rb").read()
-    except Exception as e:  # keep the tree kernel
-        print("warning: jump-table dispatch not built (%s); the dispatch tree stays" % e, flush=True)
-    with open(cpp, "w") as fh:
-        fh.write("// generated: cubin of the VM kernel with jump-table dispatch\n")
-        fh.write('extern "C" const unsigned long dragon_vm_jt_cubin_size = %d;\n' % len(data))
-        fh.write('extern "C" const unsigned char dragon_vm_jt_cubin[] = {')
-        fh.write(",".join(str(b) for b in data) if data else "0")
-        fh.write("};\n")
-    subprocess.run(["g++", "-O1", "-fPIC", "-c", cpp, "-o", obj], check=True)
     return obj
 
 

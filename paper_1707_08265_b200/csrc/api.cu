@@ -8,7 +8,7 @@
 #include "vm_math.h"
 
 namespace dragon {
-cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, cudaStream_t st);
+cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st);
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st);
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
                            int* status, cudaStream_t st);
@@ -252,6 +252,7 @@ int dragon_function_vm_step(const dragon_function_t* f, int step, int64_t* info,
   info[0] = (int64_t)sg.code.size(); info[1] = sg.row_mode; info[2] = sg.cols; info[3] = (int64_t)sg.operand_mem.size();
   info[4] = sg.n_spill; info[5] = sg.n_smem; info[6] = sg.n & 0xffffffffLL; info[7] = sg.n >> 32;
   info[8] = (int64_t)sg.finish.size();
+  info[9] = sg.dense ? vm::kVmRegsDense : vm::kVmRegsWide;
   for (int i = 0; reduced && i < cap_reduced && i < (int)sg.finish.size(); ++i) {
     const MemRef& m = f->plan.mems[sg.finish[i].mem];
     reduced[3 * i + 0] = sg.finish[i].kind;
@@ -328,6 +329,9 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         p.n = sg.n;
         p.cols = sg.cols;
         p.n_spill = sg.n_spill;
+        p.n_tiles = (uint32_t)(sg.row_mode ? sg.n : (sg.n + kVmTile - 1) / kVmTile);
+        p.loop_start = (uint32_t)sg.loop_start;
+        p.grid = (uint32_t)sg.grid;
         p.spill = reinterpret_cast<float*>(ws + sg.spill_off);
         p.colpart = reinterpret_cast<float*>(ws + sg.colpart_off);
         p.scalpart = reinterpret_cast<double*>(ws + sg.scalpart_off);
@@ -338,7 +342,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
           p.operand[i].dtype = (uint32_t)P.mems[sg.operand_mem[i]].dtype;
         }
         if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used]), st);
-        e = launch_vm(p, sg.grid, sg.n_smem, st);
+        e = launch_vm(p, sg.grid, sg.n_smem, sg.dense, st);
         if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used + 1]), st);
         if (e == cudaSuccess) e = launch_finish(sg, P.mems, ptr.data(), ws, st);
         break;

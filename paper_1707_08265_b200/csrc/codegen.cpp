@@ -6,8 +6,10 @@
 // memory operands can be re-read instead of being kept; scalars and constants live in the
 // uniform table.
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <map>
+#include <string>
 
 #include "plan.h"
 
@@ -36,18 +38,21 @@ struct Gen {
   std::vector<int> canon;
   std::map<int, VInfo> info;
   std::vector<uint32_t> pro, body, epi;
-  int reg_owner[kVmRegs];        // value id, -1 free, -2 pinned accumulator
+  const int nr;                  // register slots of the kernel build this program is for
+  const int n_smem_max;          // shared-memory slots that build can hold
+  int reg_owner[kJointStride];   // value id, -1 free, -2 pinned accumulator
   int smem_owner[kVmSmemSlots];
   std::vector<int> free_spill;
   int n_uni = 0;
   int acc_val = -1;
   std::vector<bool> done;        // item already produced by a fused instruction
   std::vector<std::pair<int, int>> accs;  // (item position of an accumulation, its pinned register)
+  std::vector<std::pair<int, int>> saccs; // (item position of an accumulation to a scalar, its scalar accumulator)
   int err = DRAGON_OK;
 
   Gen(const std::vector<Item>& it, const std::vector<int>& ix, const std::vector<Value>& v,
-      const std::vector<MemRef>& m, VmSegment* s)
-      : items(it), idx(ix), vals(v), mems(m), seg(s) {}
+      const std::vector<MemRef>& m, VmSegment* s, int n_regs, int n_smem)
+      : items(it), idx(ix), vals(v), mems(m), seg(s), nr(n_regs), n_smem_max(n_smem) {}
 
   int C(int v) const { return v < 0 ? v : canon[v]; }
 
@@ -75,6 +80,16 @@ struct Gen {
 
   void emit(int c, int r = 0, uint32_t arg = 0) { body.push_back(encode(c, r, arg)); }
   void emit_str(int k) { emit(J_STR * kJointStride + k); }
+  // the accumulation at item position q of the value in the accumulator
+  bool emit_accum(int q) {
+    for (auto& a : accs) if (a.first == q) { emit(J_ACCUM * kJointStride + a.second); return true; }
+    for (auto& a : saccs) if (a.first == q) { emit(P_SACC0 + a.second); return true; }
+    return false;
+  }
+  int scalar_acc_at(int q) const {
+    for (auto& a : saccs) if (a.first == q) return a.second;
+    return -1;
+  }
 
   void release(int v) {
     VInfo& f = info[v];
@@ -94,12 +109,12 @@ struct Gen {
     return seg->n_spill++;
   }
   int free_smem() {
-    for (int s = 0; s < kVmSmemSlots; ++s)
+    for (int s = 0; s < n_smem_max; ++s)
       if (smem_owner[s] == -1) { seg->n_smem = std::max(seg->n_smem, s + 1); return s; }
     return -1;
   }
   int free_reg() const {
-    for (int k = 0; k < kVmRegs; ++k)
+    for (int k = 0; k < nr; ++k)
       if (reg_owner[k] == -1) return k;
     return -1;
   }
@@ -108,7 +123,7 @@ struct Gen {
     int k0 = free_reg();
     if (k0 >= 0) return k0;
     int best = -1, best_use = -1;
-    for (int k = 0; k < kVmRegs; ++k) {
+    for (int k = 0; k < nr; ++k) {
       int v = reg_owner[k];
       if (v < 0 || v == keep1 || v == keep2) continue;
       int u = next_use(v, pos - 1);
@@ -143,7 +158,7 @@ struct Gen {
     if (!have_free) {
       // if every register holds something needed sooner, the accumulator itself goes down a level
       int farthest = -1;
-      for (int k = 0; k < kVmRegs; ++k) {
+      for (int k = 0; k < nr; ++k) {
         int w = reg_owner[k];
         if (w < 0 || w == keep1 || w == keep2) continue;
         farthest = std::max(farthest, is_input(w) ? kFar - 1 : next_use(w, pos));
@@ -201,6 +216,17 @@ struct Gen {
     if (k >= 0) { emit_str(k); give_reg(x, k); }
   }
 
+  // scalar accumulator that takes the product d = acc * y directly, or -1: d's only use must be a
+  // sum over the whole domain and y must sit in a register slot
+  int macc_target(const Item& it, int d, int y) {
+    if (it.opc != M_MUL) return -1;
+    const VInfo& fy = info[y];
+    if (fy.uni >= 0 || fy.home != H_REG || info[d].uses.size() != 1) return -1;
+    const int q = info[d].uses[0];
+    const Item& o2 = items[idx[q]];
+    return (!done[q] && o2.opc == M_ACCUM && C(o2.a) == d) ? scalar_acc_at(q) : -1;
+  }
+
   void binary(const Item& it, int pos) {
     static const int jop[4] = {J_ADD, J_SUB, J_MUL, J_DIVP}, jrev[4] = {J_ADD, J_RSUB, J_MUL, J_RDIVP};
     static const int uop[4] = {P_ADDU, P_SUBU, P_MULU, P_DIVPU}, urev[4] = {P_ADDU, P_RSUBU, P_MULU, P_RDIVPU};
@@ -239,11 +265,26 @@ struct Gen {
         std::swap(x, y);
       }
       load_acc(x, pos, x, y);
-      keep_operand(x, pos, y);
+      if (macc_target(it, d, y) < 0) keep_operand(x, pos, y);   // a fused multiply-accumulate leaves x in the accumulator
     }
     const bool rev = (x == b && a != b);
     const int o = it.opc - M_ADD;
     VInfo& fy = info[y];
+    // a product whose only use is a sum over the whole domain goes straight into the scalar
+    // accumulator; the accumulator register keeps x
+    {
+      const int sa = macc_target(it, d, y);
+      if (sa >= 0) {
+        const int q = info[d].uses[0];
+        emit((J_MACC0 + sa) * kJointStride + fy.home_idx);
+        done[q] = true;
+        info[d].uses.clear();
+        acc_val = x;
+        release_dead(a, pos);
+        if (b != a) release_dead(b, pos);
+        return;
+      }
+    }
     if (fy.uni >= 0) emit(rev ? urev[o] : uop[o], 0, fy.uni);
     else if (fy.home == H_REG) emit((rev ? jrev[o] : jop[o]) * kJointStride + fy.home_idx);
     else emit(rev ? srev[o] : sop[o], 0, fy.home_idx);
@@ -263,20 +304,30 @@ struct Gen {
       for (int q = pos + 1; q < (int)idx.size() && q < pos + 4096; ++q) {
         const Item& o2 = items[idx[q]];
         if (done[q] || o2.kind != IT_MOP || (o2.opc != M_SIN && o2.opc != M_COS) || o2.opc == it.opc || C(o2.a) != a) continue;
-        int sl = free_smem();
-        if (sl < 0) break;  // no slot for the cosine: two separate instructions
         int dsin = it.opc == M_SIN ? d : C(o2.dst), dcos = it.opc == M_SIN ? C(o2.dst) : d;
-        smem_owner[sl] = dcos;    // taken before anything below can evict a register into it
         auto& ua = info[a].uses;  // the partner's use of a is consumed here
         ua.erase(std::remove(ua.begin(), ua.end(), q), ua.end());
         keep_operand(a, pos, -1);
-        emit(P_SINCOS, 0, sl);
-        info[dcos].home = H_SMEM; info[dcos].home_idx = sl;
-        acc_val = dsin;
+        // the one needed first stays in the accumulator, the other goes to a register slot (a
+        // shared-memory slot when none is free)
+        const bool cos_first = next_use(dcos, pos) < next_use(dsin, pos);
+        const int dacc = cos_first ? dcos : dsin, dother = cos_first ? dsin : dcos;
+        const int k = free_reg();
+        if (k >= 0) {
+          emit((cos_first ? J_COSSINR : J_SINCOSR) * kJointStride + k);
+          give_reg(dother, k);
+        } else {
+          int sl = free_smem();
+          if (sl < 0) { ua.push_back(q); std::sort(ua.begin(), ua.end()); break; }  // two separate instructions
+          smem_owner[sl] = dother;
+          emit(cos_first ? P_COSSIN : P_SINCOS, 0, sl);
+          info[dother].home = H_SMEM; info[dother].home_idx = sl;
+        }
+        acc_val = dacc;
         done[q] = true;
         release_dead(a, pos);
-        if (next_use(dcos, pos) == kFar) release(dcos);
-        if (next_use(dsin, pos) == kFar) acc_val = -1;
+        if (next_use(dother, pos) == kFar) release(dother);
+        if (next_use(dacc, pos) == kFar) acc_val = -1;
         return;
       }
     }
@@ -298,11 +349,8 @@ struct Gen {
         int cls = class_of(mems[o2.mem].shape);
         if (cls < 0) continue;
         emit(P_GST, 0, operand_for(o2.mem, cls));
-      } else {
-        int k = -1;
-        for (auto& a : accs) if (a.first == q) k = a.second;
-        if (k < 0) continue;
-        emit(J_ACCUM * kJointStride + k);
+      } else if (!emit_accum(q)) {
+        continue;
       }
       done[q] = true;
       auto& u = info[v].uses;
@@ -329,7 +377,7 @@ struct Gen {
       any_rowsum |= it.opc == M_ROWSUM;
     }
     // 2. uses and static locations
-    std::fill(reg_owner, reg_owner + kVmRegs, -1);
+    std::fill(reg_owner, reg_owner + kJointStride, -1);
     std::fill(smem_owner, smem_owner + kVmSmemSlots, -1);
     bool any_row_class = false;
     auto note = [&](int v, int pos) {
@@ -376,8 +424,13 @@ struct Gen {
     // 3. accumulators get pinned registers
     for (int p = 0; p < (int)idx.size(); ++p)
       if (items[idx[p]].opc == M_ACCUM) {
+        // a sum over the whole domain needs one running value per thread; a column sum one per lane
+        if (class_of(mems[items[idx[p]].mem].shape) == K_SCALAR && (int)saccs.size() < kVmScalarAccs) {
+          saccs.emplace_back(p, (int)saccs.size());
+          continue;
+        }
         int k = (int)accs.size();
-        if (k >= kVmRegs - 4) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+        if (k >= nr - 2) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
         reg_owner[k] = -2;
         accs.emplace_back(p, k);
       }
@@ -397,10 +450,9 @@ struct Gen {
         emit(P_GST, 0, opd);
         release_dead(v, p);
       } else if (it.opc == M_ACCUM) {
-        int v = C(it.a), k = -1;
-        for (auto& a : accs) if (a.first == p) k = a.second;
+        int v = C(it.a);
         load_acc(v, p, v);
-        emit(J_ACCUM * kJointStride + k);
+        emit_accum(p);
         release_dead(v, p);
       } else { unary(it, p); drain_acc(p); }
     }
@@ -412,9 +464,28 @@ struct Gen {
       if ((w & 1023u) == (uint32_t)P_MULU && i + 1 < body.size()) {
         uint32_t nx = body[i + 1], ncase = nx & 1023u, ui = w >> 14;
         if (ncase == (uint32_t)P_ADDU && ui < 512 && (nx >> 14) < 512) { fused.push_back(encode(P_FMAU, 0, ui | ((nx >> 14) << 9))); ++i; continue; }
-        if (ncase >= (uint32_t)(J_ADD * kJointStride) && ncase < (uint32_t)(J_ADD * kJointStride + kVmRegs)) {
+        if (ncase >= (uint32_t)(J_ADD * kJointStride) && ncase < (uint32_t)(J_ADD * kJointStride + nr)) {
           fused.push_back(encode(J_FMAUR * kJointStride + (int)(ncase - J_ADD * kJointStride), 0, ui)); ++i; continue;
         }
+      }
+      fused.push_back(w);
+    }
+    body.swap(fused);
+    fused.clear();
+    // loads and stores of fp32 tensors of the full domain shape have their own, shorter instructions
+    auto plain_f32 = [&](uint32_t opd) {
+      return seg->operand_kind[opd] == (uint32_t)K_FULL && mems[seg->operand_mem[opd]].dtype == DRAGON_F32;
+    };
+    for (uint32_t& w : body) {
+      if ((w & 1023u) == (uint32_t)P_GLD && plain_f32(w >> 14)) w = encode(P_GLDF, 0, w >> 14);
+      else if ((w & 1023u) == (uint32_t)P_GST && plain_f32(w >> 14)) w = encode(P_GSTF, 0, w >> 14);
+    }
+    for (size_t i = 0; i < body.size(); ++i) {   // a load that is kept in a register slot is one instruction
+      const uint32_t w = body[i], nx = i + 1 < body.size() ? body[i + 1] : 0u, ncase = nx & 1023u;
+      if ((w & 1023u) == (uint32_t)P_GLDF && i + 1 < body.size() && ncase >= (uint32_t)(J_STR * kJointStride) && ncase < (uint32_t)(J_STR * kJointStride + nr)) {
+        fused.push_back(encode(J_GLDR * kJointStride + (int)(ncase - J_STR * kJointStride), 0, w >> 14));
+        ++i;
+        continue;
       }
       fused.push_back(w);
     }
@@ -430,8 +501,15 @@ struct Gen {
       else { set_error("graph VM: reduction target shape is not supported"); return DRAGON_ERR_UNSUPPORTED; }
       seg->finish.push_back(job);
     }
+    for (auto& a : saccs) {
+      const Item& it = items[idx[a.first]];
+      FinishJob job; job.mem = it.mem; job.kind = 1; job.acc = seg->n_scalacc++;
+      epi.push_back(encode(P_ASCAL0 + a.second, 0, job.acc));
+      seg->finish.push_back(job);
+    }
     seg->code = pro;
     seg->code.push_back(encode(P_LOOP_BEGIN, 0, 0));
+    seg->loop_start = (int)seg->code.size();
     seg->code.insert(seg->code.end(), body.begin(), body.end());
     seg->code.push_back(encode(P_LOOP_END, 0, 0));
     seg->code.insert(seg->code.end(), epi.begin(), epi.end());
@@ -454,11 +532,29 @@ struct Gen {
 
 int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx, const std::vector<Value>& vals,
                     const std::vector<MemRef>& mems, int sm_count, VmSegment* seg) {
-  Gen gen(items, idx, vals, mems, seg);
-  int rc = gen.run();
-  if (rc) return rc;
+  // the dense build (few register slots, two CTAs per SM) when the program keeps everything on
+  // chip with it, else the wide one; DRAGON_VM_BUILD=wide|dense forces the choice
+  const char* force = std::getenv("DRAGON_VM_BUILD");
+  const bool only_wide = force && std::string(force) == "wide", only_dense = force && std::string(force) == "dense";
+  int rc = DRAGON_ERR_UNSUPPORTED;
+  if (!only_wide) {
+    VmSegment trial = *seg;
+    Gen gen(items, idx, vals, mems, &trial, kVmRegsDense, kVmSmemSlotsDense);
+    rc = gen.run();
+    // it must keep everything on chip, within half an SM's shared memory
+    const size_t smem = (size_t)((trial.code.size() + 3) & ~(size_t)3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)trial.n_smem * kVmTile * 4;
+    if (rc == DRAGON_OK && trial.n_spill == 0 && smem <= 113 * 1024) { *seg = trial; seg->dense = true; }
+    else rc = DRAGON_ERR_UNSUPPORTED;
+  }
+  if (rc != DRAGON_OK) {
+    Gen gen(items, idx, vals, mems, seg, kVmRegsWide, kVmSmemSlots);
+    rc = gen.run();
+    if (rc) return rc;
+    seg->dense = false;
+  }
   long long tiles = seg->row_mode ? seg->n : (seg->n + kVmTile - 1) / kVmTile;
-  seg->grid = (int)std::max<long long>(1, std::min<long long>(tiles, sm_count));
+  if (tiles >= (1LL << 31)) { set_error("graph VM: more than 2^31 tiles"); return DRAGON_ERR_UNSUPPORTED; }
+  seg->grid = (int)std::max<long long>(1, std::min<long long>(tiles, (long long)sm_count * (seg->dense ? 2 : 1)));
   return DRAGON_OK;
 }
 

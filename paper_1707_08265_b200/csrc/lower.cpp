@@ -500,11 +500,12 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
 
 // one mnemonic per instruction word of a segment
 static std::string disassemble(const VmSegment& sg) {
-  static const char* jn[] = {"ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr"};
+  static const char* jn[] = {"ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
+                             "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3"};
   static const char* pn[] = {"ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls",
-                             "divps", "rdivps", "sin", "cos", "sincos", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq",
-                             "yomy", "divpgb", "rbf16", "rowsum", "gld", "gst", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout",
-                             "scalout", "end"};
+                             "divps", "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq",
+                             "yomy", "divpgb", "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout",
+                             "scalout", "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "end"};
   std::string s;
   char buf[64];
   for (size_t i = 0; i < sg.code.size(); ++i) {
@@ -515,7 +516,7 @@ static std::string disassemble(const VmSegment& sg) {
     else if (cs < vm::P_COUNT_) snprintf(buf, sizeof(buf), "%s", pn[cs - vm::kFirstPlain]);
     else snprintf(buf, sizeof(buf), "?%d", cs);
     s += buf;
-    if (arg || (cs >= vm::kFirstPlain && cs != vm::P_LOOP_BEGIN && cs != vm::P_LOOP_END && cs != vm::P_END && !(cs >= vm::P_SIN && cs <= vm::P_ROWSUM && cs != vm::P_SINCOS))) {
+    if (arg || (cs >= vm::kFirstPlain && cs != vm::P_LOOP_BEGIN && cs != vm::P_LOOP_END && cs != vm::P_END && !(cs >= vm::P_SIN && cs <= vm::P_ROWSUM && cs != vm::P_SINCOS && cs != vm::P_COSSIN) && !(cs >= vm::P_SACC0 && cs <= vm::P_SACC3))) {
       snprintf(buf, sizeof(buf), " %u", arg);
       s += buf;
     }
@@ -533,8 +534,8 @@ std::string describe_plan(const Plan& p) {
     switch (st.kind) {
       case ST_VM: {
         const VmSegment& sg = p.segs[st.seg];
-        snprintf(buf, sizeof(buf), "vm[%s n=%lld cols=%d instr=%d body=%d operands=%d smem=%d spill=%d colacc=%d scalacc=%d grid=%d]\n",
-                 sg.row_mode ? "row" : "flat", sg.n, sg.cols, (int)sg.code.size(), sg.n_instr_body,
+        snprintf(buf, sizeof(buf), "vm[%s %s n=%lld cols=%d instr=%d body=%d operands=%d smem=%d spill=%d colacc=%d scalacc=%d grid=%d]\n",
+                 sg.row_mode ? "row" : "flat", sg.dense ? "dense" : "wide", sg.n, sg.cols, (int)sg.code.size(), sg.n_instr_body,
                  (int)sg.operand_mem.size(), sg.n_smem, sg.n_spill, sg.n_colacc, sg.n_scalacc, sg.grid);
         s += buf;
         if (sg.code.size() <= 96) s += "  code: " + disassemble(sg) + "\n";

@@ -14,9 +14,9 @@ namespace dragon {
 constexpr int kVmThreads = DRAGON_VM_THREADS;
 constexpr int kVmVec = DRAGON_VM_VEC;
 constexpr int kVmTile = kVmThreads * kVmVec;  // 4096
-constexpr int kVmRegs = DRAGON_VM_REGS;       // register slots R[0..kVmRegs)
 constexpr int kVmCodeMaxWords = 8 * 1024;     // instruction stream held in shared memory (8 bytes per word once decoded)
-constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread
+constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread (wide build: one CTA per SM)
+constexpr int kVmSmemSlotsDense = 6;          // the same for the dense build (two CTAs share the SM's shared memory)
 constexpr int kDefaultSmCount = 148;
 
 enum MemWhere { MEM_FEED = 0, MEM_FETCH = 1, MEM_WORK = 2 };
@@ -77,6 +77,7 @@ struct VmSegment {
   std::vector<int> operand_mem;     // operand table: memref ids
   std::vector<uint32_t> operand_kind;
   bool row_mode = false;
+  bool dense = false;               // kernel build: dense (3 register slots, 2 CTAs per SM) or wide (7, 1)
   long long n = 0;                  // flat: elements; row: rows
   int cols = 0;
   int n_spill = 0, n_colacc = 0, n_scalacc = 0, n_smem = 0;
@@ -85,6 +86,7 @@ struct VmSegment {
   std::vector<FinishJob> finish;
   uint32_t* d_code = nullptr;       // device copy
   int n_instr_body = 0;
+  int loop_start = 0;               // index in code of the first instruction of the per-tile body
 };
 
 enum StepKind { ST_VM, ST_GEMM, ST_TRANSPOSE, ST_SCE_FWD, ST_SCE_BWD, ST_COPY };

@@ -8,14 +8,9 @@
 #pragma once
 #include <cstdint>
 
-// geometry of the VM kernel (threads per CTA, elements per thread, register slots)
-#ifndef DRAGON_VM_REGS
-#define DRAGON_VM_REGS 7
-#endif
-#ifndef DRAGON_VM_THREADS
+// geometry of the VM kernel (threads per CTA, elements per thread)
 #define DRAGON_VM_THREADS 512
 #define DRAGON_VM_VEC 8
-#endif
 
 namespace dragon {
 namespace vm {
@@ -39,9 +34,18 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   J_STOR,      // R = S[arg]
   J_SPILL,     // spill[arg] = R
   J_FILL,      // R = spill[arg]
+  J_GLDR,      // R = acc = operand[arg] at this tile
+  J_SINCOSR,   // R = cos(acc); acc = sin(acc)
+  J_COSSINR,   // R = sin(acc); acc = cos(acc)
+  J_MACC0, J_MACC1, J_MACC2, J_MACC3,   // A[i] += sum over this thread's valid lanes of acc * R   (acc unchanged)
   J_COUNT
 };
-constexpr int kJointStride = DRAGON_VM_REGS;  // case ids are dense, so the dispatch is one indexed jump
+// The kernel exists in two builds that share this encoding: "wide" (7 register slots, one CTA per
+// SM) and "dense" (3 register slots, two CTAs per SM, for programs with few live values: twice
+// the warps hide the latency of the dispatch).  A case id whose slot a build lacks is never emitted.
+constexpr int kJointStride = 8;
+constexpr int kVmRegsWide = 7, kVmRegsDense = 3;
+constexpr int kVmScalarAccs = 4;             // A[0..4): per-thread scalar accumulators (packed pair of partial sums)
 constexpr int kFirstPlain = J_COUNT * kJointStride;
 
 enum Plain : int {
@@ -53,6 +57,7 @@ enum Plain : int {
   P_ADDS, P_SUBS, P_RSUBS, P_MULS, P_DIVPS, P_RDIVPS,
   P_SIN, P_COS,
   P_SINCOS,             // S[arg] = cos(acc); acc = sin(acc)
+  P_COSSIN,             // S[arg] = sin(acc); acc = cos(acc)
   P_EXPC, P_TANH, P_SIGMOID, P_RELU, P_NEG,
   P_STEP,               // acc = acc > 0 ? 1 : 0
   P_CLAMPMASK,          // acc = (-10 <= acc <= 10) ? 1 : 0
@@ -63,6 +68,8 @@ enum Plain : int {
   P_ROWSUM,             // acc = sum of acc over the whole row (all lanes, all threads), row mode only
   P_GLD,                // acc = operand[arg] at this tile
   P_GST,                // operand[arg] at this tile = acc
+  P_GLDF,               // P_GLD for an fp32 operand of the full domain shape
+  P_GSTF,               // P_GST for an fp32 operand of the full domain shape
   P_FILL,               // acc = spill[arg]
   P_SPILL,              // spill[arg] = acc
   P_ULOAD,              // U[arg & 511] = scalar operand[arg >> 9]   (prologue)
@@ -71,6 +78,8 @@ enum Plain : int {
   P_LOOP_END,           // next tile; jumps back to the body or falls through to the epilogue
   P_COLOUT,             // column partial sums: colpart[arg][cta][c] = acc
   P_SCALOUT,            // scalar partial sum: scalpart[arg][cta] = block sum of acc in fp64
+  P_SACC0, P_SACC1, P_SACC2, P_SACC3,       // A[i] += sum over this thread's valid lanes of acc
+  P_ASCAL0, P_ASCAL1, P_ASCAL2, P_ASCAL3,   // scalpart[arg][cta] = block sum of A[i] in fp64
   P_END,
   P_COUNT_
 };
@@ -87,19 +96,25 @@ struct Operand {        // 16 bytes
   uint32_t dtype;       // DRAGON_F32 / DRAGON_BF16
 };
 
-struct Params {
-  const uint32_t* code;     // device copy of the instruction stream
-  int n_code;
-  int row_mode;             // 0: flat domain of n elements; 1: rows x cols, one row per tile
-  long long n;              // flat: element count; row mode: row count
-  int cols;                 // row mode: row length
-  int n_spill;              // spill slots per CTA
-  float* spill;             // [grid][n_spill][tile]
-  float* colpart;           // [n_colacc][grid][cols]
-  double* scalpart;         // [n_scalacc][grid]
-  int* status;
-  Operand operand[kMaxOperands];
+struct Params {             // kernel parameter block; the PTX generator (vm_ptxgen.py) uses the same offsets
+  const uint32_t* code;     //  0  device copy of the instruction stream
+  float* spill;             //  8  [grid][n_spill][tile]
+  float* colpart;           // 16  [n_colacc][grid][cols]
+  double* scalpart;         // 24  [n_scalacc][grid]
+  int* status;              // 32
+  long long n;              // 40  flat: element count; row mode: row count
+  int n_code;               // 48
+  int row_mode;             // 52  0: flat domain of n elements; 1: rows x cols, one row per tile
+  int cols;                 // 56  row mode: row length
+  int n_spill;              // 60  spill slots per CTA
+  uint32_t n_tiles;         // 64
+  uint32_t loop_start;      // 68  index of the first instruction of the per-tile body
+  uint32_t grid;            // 72  CTAs launched
+  uint32_t reserved;        // 76
+  Operand operand[kMaxOperands];   // 80
 };
+static_assert(sizeof(Operand) == 16 && sizeof(Params) == 80 + 16 * kMaxOperands, "layout shared with the PTX generator");
+
 
 }  // namespace vm
 }  // namespace dragon

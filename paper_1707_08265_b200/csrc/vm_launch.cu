@@ -1,0 +1,108 @@
+// Launch side of the graph VM.  The interpreter kernel itself is written in PTX by
+// vm_ptxgen.py (two builds: "wide" and "dense", see vm_isa.h); its cubin is embedded in the
+// library by the build and loaded here.  This file also holds the small finishing kernel that
+// turns per-CTA partial sums into tensors.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <mutex>
+
+#include "plan.h"
+#include "vm_math.h"
+
+// cubin assembled from the generated PTX (build.py)
+extern "C" const unsigned long dragon_vm_gen_cubin_size;
+extern "C" const unsigned char dragon_vm_gen_cubin[];
+
+namespace dragon {
+namespace vm {
+
+// ---- finishing reductions: per-CTA partials -> tensors (fixed order, fp64) ------------------
+
+struct FinishParams {
+  int n_jobs;
+  struct Job {
+    int kind;          // 0 column sums, 1 scalar
+    const void* part;  // float [grid][cols] or double [grid]
+    void* out;
+    int dtype, cols, grid;
+  } job[8];
+};
+
+__global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
+  const FinishParams::Job& jb = fp.job[blockIdx.y];
+  if (jb.kind == 0) {
+    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= jb.cols) return;
+    const float* part = reinterpret_cast<const float*>(jb.part);
+    double s = 0.0;
+    for (int g = 0; g < jb.grid; ++g) s += (double)part[(size_t)g * jb.cols + c];
+    if (jb.dtype == DRAGON_F32) reinterpret_cast<float*>(jb.out)[c] = (float)s;
+    else reinterpret_cast<unsigned short*>(jb.out)[c] = (unsigned short)vmmath::bf16_bits((float)s);
+  } else if (blockIdx.x == 0 && threadIdx.x == 0) {
+    const double* part = reinterpret_cast<const double*>(jb.part);
+    double s = 0.0;
+    for (int g = 0; g < jb.grid; ++g) s += part[g];
+    if (jb.dtype == DRAGON_F32) *reinterpret_cast<float*>(jb.out) = (float)s;
+    else *reinterpret_cast<unsigned short*>(jb.out) = (unsigned short)vmmath::bf16_bits((float)s);
+  }
+}
+
+// shared memory of one CTA: decoded instruction stream | uniforms | reduction scratch | operand table | slots
+size_t vm_smem_bytes(int n_code, int n_smem_slots) {
+  return (size_t)((n_code + 3) & ~3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)n_smem_slots * kVmTile * 4;
+}
+
+}  // namespace vm
+
+struct VmKernels {
+  cudaError_t err = cudaErrorUnknown;
+  cudaKernel_t wide = nullptr, dense = nullptr;
+};
+
+// loads the embedded cubin once per process (kernels of a cudaLibrary_t are usable on every device)
+static const VmKernels& vm_kernels() {
+  static VmKernels k;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    cudaLibrary_t lib;
+    k.err = cudaLibraryLoadData(&lib, dragon_vm_gen_cubin, nullptr, nullptr, 0, nullptr, nullptr, 0);
+    if (k.err == cudaSuccess) k.err = cudaLibraryGetKernel(&k.wide, lib, "dragon_vm_wide");
+    if (k.err == cudaSuccess) k.err = cudaLibraryGetKernel(&k.dense, lib, "dragon_vm_dense");
+    if (k.err == cudaSuccess) k.err = cudaFuncSetAttribute(k.wide, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (k.err == cudaSuccess) k.err = cudaFuncSetAttribute(k.dense, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024);
+  });
+  return k;
+}
+
+cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st) {
+  const VmKernels& k = vm_kernels();
+  if (k.err != cudaSuccess) return k.err;
+  const size_t smem = vm::vm_smem_bytes(p.n_code, n_smem_slots);
+  if (smem > (size_t)(dense ? 113 : 227) * 1024) return cudaErrorInvalidConfiguration;
+  void* args[] = {const_cast<vm::Params*>(&p)};
+  return cudaLaunchKernel(reinterpret_cast<const void*>(dense ? k.dense : k.wide), dim3(grid), dim3(kVmThreads), args, smem, st);
+}
+
+cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st) {
+  if (sg.finish.empty()) return cudaSuccess;
+  vm::FinishParams fp;
+  fp.n_jobs = (int)sg.finish.size();
+  int max_cols = 1;
+  for (int i = 0; i < fp.n_jobs; ++i) {
+    const FinishJob& j = sg.finish[i];
+    auto& o = fp.job[i];
+    o.kind = j.kind;
+    o.grid = sg.grid;
+    o.cols = sg.cols;
+    o.dtype = mems[j.mem].dtype;
+    o.out = mem_ptr[j.mem];
+    if (j.kind == 0) { o.part = ws + sg.colpart_off + (size_t)j.acc * sg.grid * sg.cols * sizeof(float); max_cols = std::max(max_cols, sg.cols); }
+    else o.part = ws + sg.scalpart_off + (size_t)j.acc * sg.grid * sizeof(double);
+  }
+  dim3 grid((max_cols + 127) / 128, fp.n_jobs);
+  vm::finish_kernel<<<grid, 128, 0, st>>>(fp);
+  return cudaGetLastError();
+}
+
+}  // namespace dragon

@@ -31,13 +31,20 @@ MAX_OPERANDS = 40
 MAX_UNIFORMS = 512
 
 # Params (csrc/vm_isa.h): byte offsets
-P_CODE, P_NCODE, P_ROWMODE, P_N, P_COLS, P_NSPILL, P_SPILL, P_COLPART, P_SCALPART, P_STATUS, P_OPERAND = 0, 8, 12, 16, 24, 28, 32, 40, 48, 56, 64
+P_CODE, P_SPILL, P_COLPART, P_SCALPART, P_STATUS, P_N = 0, 8, 16, 24, 32, 40
+P_NCODE, P_ROWMODE, P_COLS, P_NSPILL, P_NTILES, P_LOOPSTART, P_GRID, P_OPERAND = 48, 52, 56, 60, 64, 68, 72, 80
 P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
+# shared memory behind the decoded instruction stream: uniforms | reduction scratch | operand table | slots
+OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
 
-JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr"]
+JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
+         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3"]
+JOINT_STRIDE = 8    # case id of a joint instruction = index * JOINT_STRIDE + register slot
+N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
-         "rdivps", "sin", "cos", "sincos", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
-         "rbf16", "rowsum", "gld", "gst", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout", "end"]
+         "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
+         "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "end"]
 
 
 def f32bits(x):
@@ -57,6 +64,7 @@ class Kernel:
         self.kt = []          # packed constants (u64 words)
         self.A = ["%%A%d" % i for i in range(NP)]
         self.R = [["%%R%d_%d" % (k, i) for i in range(NP)] for k in range(nr)]
+        self.S = ["%%S%d" % i for i in range(N_SACC)]     # scalar accumulators (.f32)
 
     # ---- plumbing -------------------------------------------------------------------------
     def e(self, s):
@@ -147,6 +155,21 @@ class Kernel:
     def fetch(self):
         self.e("ld.shared.v2.u32 {%case, %arg}, [%ip];")
         self.e("add.u32 %ip, %ip, 8;")
+
+    def param(self, off, ty="u32"):
+        d = self.rd() if ty in ("u64", "s64") else self.r()
+        self.e("ld.param.%s %s, [VP+%d];" % (ty, d, off))
+        return d
+
+    def tx_is_zero(self):
+        pr = self.p()
+        self.e("setp.eq.u32 %s, %%pos0, 0;" % pr)
+        return pr
+
+    def pos0_64(self):
+        d = self.rd()
+        self.e("cvt.u64.u32 %s, %%pos0;" % d)
+        return d
 
     def jump(self):
         self.e("brx.idx.uni %%case, JT_%s;" % self.name)
@@ -341,36 +364,48 @@ class Kernel:
             self.mul2(num[i], self.pack(self.rcp1pabs(lo), self.rcp1pabs(hi)), dst[i])
 
     # ---- tile context -----------------------------------------------------------------------
+    # Kept per thread between instructions: %tile (index), %tb4 (byte offset of this thread's first
+    # element of the tile in an fp32 FULL tensor), %limit (valid elements in the tile), %tnext
+    # (elements to this CTA's next tile, 0 when there is none), %pfull (limit == TILE; then every
+    # 4-element group is whole and 16-byte aligned).
     def set_tile(self):
-        """from %tile: %tbase, %limit, %pfull, %pvec, %pfirst, %tnext, %pfast"""
         done, flat = self.newlabel("st"), self.newlabel("st")
-        nt, t0 = self.rd(), self.rd()
-        pr = self.p()
-        self.e("add.s64 %s, %%tile, %%gs;" % nt)
-        self.e("mov.s64 %tnext, 0;")
-        self.e("@!%%prow bra.uni %s;" % flat)
-        self.e("mul.lo.s64 %tbase, %tile, %cols64;")
-        self.e("mov.s32 %limit, %cols;")
-        t1 = self.r()
-        self.e("and.b32 %s, %%cols, 3;" % t1)
-        self.e("setp.eq.s32 %%pvec, %s, 0;" % t1)
-        self.e("setp.lt.s64 %s, %s, %%ntiles;" % (pr, nt))
-        self.e("@%s mul.lo.s64 %%tnext, %%gs, %%cols64;" % pr)
+        prow, pn = self.p(), self.p()
+        rowmode, gs, nt, tbase = self.param(P_ROWMODE), self.param(P_GRID), self.r(), self.rd()
+        self.e("setp.ne.s32 %s, %s, 0;" % (prow, rowmode))
+        self.e("add.u32 %s, %%tile, %s;" % (nt, gs))
+        self.e("mov.u32 %tnext, 0;")
+        self.e("@!%s bra.uni %s;" % (prow, flat))
+        cols, ntiles = self.param(P_COLS), self.param(P_NTILES)
+        self.e("mul.wide.u32 %s, %%tile, %s;" % (tbase, cols))
+        self.e("mov.u32 %%limit, %s;" % cols)
+        self.e("setp.lt.u32 %s, %s, %s;" % (pn, nt, ntiles))
+        self.e("@%s mul.lo.u32 %%tnext, %s, %s;" % (pn, gs, cols))
         self.e("bra.uni %s;" % done)
         self.label(flat)
-        self.e("shl.b64 %%tbase, %%tile, %d;" % 12)
-        self.e("sub.s64 %s, %%n, %%tbase;" % t0)
-        self.e("min.s64 %s, %s, %d;" % (t0, t0, TILE))
-        self.e("cvt.s32.s64 %%limit, %s;" % t0)
-        self.e("setp.eq.s32 %pvec, %limit, %limit;")
-        self.e("add.s64 %s, %s, 1;" % (nt, nt))
-        self.e("shl.b64 %s, %s, 12;" % (nt, nt))
-        self.e("setp.le.s64 %s, %s, %%n;" % (pr, nt))
-        self.e("@%s shl.b64 %%tnext, %%gs, 12;" % pr)
+        n, left, end = self.param(P_N, "s64"), self.rd(), self.rd()
+        self.e("mul.wide.u32 %s, %%tile, %d;" % (tbase, TILE))
+        self.e("sub.s64 %s, %s, %s;" % (left, n, tbase))
+        self.e("min.s64 %s, %s, %d;" % (left, left, TILE))
+        self.e("cvt.u32.u64 %%limit, %s;" % left)
+        self.e("add.u32 %s, %s, 1;" % (nt, nt))
+        self.e("mul.wide.u32 %s, %s, %d;" % (end, nt, TILE))     # the whole next tile must exist
+        self.e("setp.le.s64 %s, %s, %s;" % (pn, end, n))
+        self.e("@%s shl.b32 %%tnext, %s, 12;" % (pn, gs))
         self.label(done)
-        self.e("setp.eq.s32 %%pfull, %%limit, %d;" % TILE)
-        self.e("setp.eq.s64 %pfirst, %tile, 0;")
-        self.e("and.pred %pfast, %pfull, %pvec;")
+        self.e("setp.eq.u32 %%pfull, %%limit, %d;" % TILE)
+        p64 = self.pos0_64()
+        self.e("add.u64 %s, %s, %s;" % (tbase, tbase, p64))
+        self.e("shl.b64 %%tb4, %s, 2;" % tbase)
+
+    def pvec(self):
+        """4-element groups are 16-byte aligned: always in flat mode, in row mode when cols % 4 == 0"""
+        pr, p2, t = self.p(), self.p(), self.r()
+        self.e("setp.eq.s32 %s, %s, 0;" % (pr, self.param(P_ROWMODE)))
+        self.e("and.b32 %s, %s, 3;" % (t, self.param(P_COLS)))
+        self.e("setp.eq.u32 %s, %s, 0;" % (p2, t))
+        self.e("or.pred %s, %s, %s;" % (pr, pr, p2))
+        return pr
 
     # position of element j of this thread inside the tile
     def lane_pos(self, j):
@@ -383,88 +418,131 @@ class Kernel:
         out = []
         for j, s in enumerate(sc):
             pr, d = self.p(), self.f()
-            self.e("setp.lt.s32 %s, %s, %%limit;" % (pr, self.lane_pos(j)))
+            self.e("setp.lt.u32 %s, %s, %%limit;" % (pr, self.lane_pos(j)))
             self.e("selp.f32 %s, %s, 0f00000000, %s;" % (d, s, pr))
             out.append(d)
         return out
 
     # ---- global loads and stores of one operand ----------------------------------------------
-    def operand(self):
+    def operand(self, want_meta=True):
         """-> (ptr u64, kind u32, dtype u32) of operand[%arg] from the shared-memory copy of the table"""
-        a, ptr, kind, dt = self.r(), self.rd(), self.r(), self.r()
+        a, ptr = self.r(), self.rd()
         self.e("shl.b32 %s, %%arg, 4;" % a)
-        self.e("add.u32 %s, %s, %%opb;" % (a, a))
-        self.e("ld.shared.u64 %s, [%s];" % (ptr, a))
-        self.e("ld.shared.v2.u32 {%s, %s}, [%s+8];" % (kind, dt, a))
+        self.e("add.u32 %s, %s, %%ub;" % (a, a))
+        self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
+        if not want_meta:
+            return ptr, None, None
+        kind, dt = self.r(), self.r()
+        self.e("ld.shared.v2.u32 {%s, %s}, [%s+%d];" % (kind, dt, a, OFF_OPB + 8))
         return ptr, kind, dt
 
-    def leaf_gld(self):
-        ptr, kind, dt = self.operand()
-        self.fetch()
-        pfullk, pbf = self.p(), self.p()
-        base = self.rd()
-        self.e("setp.eq.u32 %s, %s, 0;" % (pfullk, kind))
-        self.e("selp.b64 %s, %%tbase, 0, %s;" % (base, pfullk))
-        self.e("setp.ne.u32 %s, %s, 0;" % (pbf, dt))
-        lbf, ldone, lslow = self.newlabel("gld"), self.newlabel("gld"), self.newlabel("gld")
-        self.e("@%s bra.uni %s;" % (pbf, lbf))
-        # ---- fp32 ----
-        adr = self.rd()
-        self.e("add.s64 %s, %s, %%pos0_64;" % (adr, base))
-        self.e("shl.b64 %s, %s, 2;" % (adr, adr))
-        self.e("add.u64 %s, %s, %s;" % (adr, adr, ptr))
-        self.prefetch(adr, pfullk, 4)
-        self.e("@!%%pfast bra.uni %s;" % lslow)
-        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s];" % (self.A[0], self.A[1], adr))
-        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (self.A[2], self.A[3], adr, HALF_BYTES))
-        self.jump()
-        self.label(lslow)
+    def prefetch(self, adr, esize, cond=None):
+        """pulls this CTA's next tile of a FULL operand into L2 while the current one is processed"""
+        pr, pa, off = self.p(), self.rd(), self.rd()
+        self.e("setp.ne.u32 %s, %%tnext, 0;" % pr)
+        if cond:
+            self.e("and.pred %s, %s, %s;" % (pr, pr, cond))
+        self.e("mul.wide.u32 %s, %%tnext, %d;" % (off, esize))
+        self.e("add.u64 %s, %s, %s;" % (pa, adr, off))
         for h in range(2):
-            lv, ln = self.newlabel("gld"), self.newlabel("gld")
+            ph, ps = self.p(), self.r()
+            self.e("add.u32 %s, %%pos0, %d;" % (ps, h * NT * 4))
+            self.e("setp.lt.u32 %s, %s, %%limit;" % (ph, ps))
+            self.e("and.pred %s, %s, %s;" % (ph, ph, pr))
+            self.e("@%s prefetch.global.L2 [%s+%d];" % (ph, pa, h * NT * 4 * esize))
+
+    def leaf_gldf(self, dst, copy_to=None):
+        """fp32 FULL operand -> dst (and copy_to)"""
+        ptr, _, _ = self.operand(False)
+        self.fetch()
+        adr = self.rd()
+        self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
+        slow = self.newlabel("gldf")
+        self.e("@!%%pfull bra.uni %s;" % slow)
+        pr, pa, off = self.p(), self.rd(), self.rd()
+        self.e("setp.ne.u32 %s, %%tnext, 0;" % pr)
+        self.e("mul.wide.u32 %s, %%tnext, 4;" % off)
+        self.e("add.u64 %s, %s, %s;" % (pa, adr, off))
+        self.e("@%s prefetch.global.L2 [%s];" % (pr, pa))
+        self.e("@%s prefetch.global.L2 [%s+%d];" % (pr, pa, HALF_BYTES))
+        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s];" % (dst[0], dst[1], adr))
+        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (dst[2], dst[3], adr, HALF_BYTES))
+        if copy_to:
+            self.mov_v(copy_to, dst)
+        self.jump()
+        self.label(slow)
+        self.prefetch(adr, 4)
+        self.load_f32_slow(adr, dst)
+        if copy_to:
+            self.mov_v(copy_to, dst)
+        self.jump()
+
+    def load_f32_slow(self, adr, dst):
+        pvec = self.pvec()
+        for h in range(2):
+            lv, ln = self.newlabel("ld"), self.newlabel("ld")
             pv, pos3 = self.p(), self.r()
             self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
-            self.e("setp.lt.s32 %s, %s, %%limit;" % (pv, pos3))
-            self.e("and.pred %s, %s, %%pvec;" % (pv, pv))
+            self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
+            self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
             sc = []
             for e_ in range(4):
                 pe, d = self.p(), self.f()
-                self.e("setp.lt.s32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
+                self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
                 self.e("mov.f32 %s, 0f00000000;" % d)
                 self.e("@%s ld.global.nc.f32 %s, [%s+%d];" % (pe, d, adr, h * HALF_BYTES + 4 * e_))
                 sc.append(d)
-            self.pack(sc[0], sc[1], self.A[2 * h])
-            self.pack(sc[2], sc[3], self.A[2 * h + 1])
+            self.pack(sc[0], sc[1], dst[2 * h])
+            self.pack(sc[2], sc[3], dst[2 * h + 1])
             self.e("bra %s;" % ln)
             self.label(lv)
-            self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (self.A[2 * h], self.A[2 * h + 1], adr, h * HALF_BYTES))
+            self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (dst[2 * h], dst[2 * h + 1], adr, h * HALF_BYTES))
             self.label(ln)
+
+    def leaf_gld(self):
+        """any operand -> acc"""
+        A = self.A
+        ptr, kind, dt = self.operand()
+        self.fetch()
+        pfullk, pbf = self.p(), self.p()
+        off, p64 = self.rd(), self.pos0_64()
+        self.e("setp.eq.u32 %s, %s, 0;" % (pfullk, kind))
+        self.e("shl.b64 %s, %s, 2;" % (p64, p64))
+        self.e("selp.b64 %s, %%tb4, %s, %s;" % (off, p64, pfullk))     # FULL: this tile; ROW: the row itself
+        self.e("setp.ne.u32 %s, %s, 0;" % (pbf, dt))
+        lbf = self.newlabel("gld")
+        self.e("@%s bra.uni %s;" % (pbf, lbf))
+        adr = self.rd()
+        self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        self.prefetch(adr, 4, pfullk)
+        self.load_f32_slow(adr, A)
         self.jump()
         # ---- bf16 ----
         self.label(lbf)
         adr = self.rd()
-        self.e("add.s64 %s, %s, %%pos0_64;" % (adr, base))
-        self.e("shl.b64 %s, %s, 1;" % (adr, adr))
-        self.e("add.u64 %s, %s, %s;" % (adr, adr, ptr))
-        self.prefetch(adr, pfullk, 2)
+        self.e("shr.u64 %s, %s, 1;" % (off, off))
+        self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        self.prefetch(adr, 2, pfullk)
+        pvec = self.pvec()
         for h in range(2):
             lv, ln = self.newlabel("gld"), self.newlabel("gld")
             pv, pos3 = self.p(), self.r()
             self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
-            self.e("setp.lt.s32 %s, %s, %%limit;" % (pv, pos3))
-            self.e("and.pred %s, %s, %%pvec;" % (pv, pv))
+            self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
+            self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
             sc = []
             for e_ in range(4):
                 pe, d, hh = self.p(), self.r(), self.t("h")
-                self.e("setp.lt.s32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
+                self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
                 self.e("mov.b16 %s, 0;" % hh)
                 self.e("@%s ld.global.nc.u16 %s, [%s+%d];" % (pe, hh, adr, h * NT * 8 + 2 * e_))
                 self.e("cvt.u32.u16 %s, %s;" % (d, hh))
                 self.e("shl.b32 %s, %s, 16;" % (d, d))
                 sc.append(d)
-            self.pack(sc[0], sc[1], self.A[2 * h])
-            self.pack(sc[2], sc[3], self.A[2 * h + 1])
+            self.pack(sc[0], sc[1], A[2 * h])
+            self.pack(sc[2], sc[3], A[2 * h + 1])
             self.e("bra %s;" % ln)
             self.label(lv)
             w0, w1 = self.r(), self.r()
@@ -473,86 +551,88 @@ class Kernel:
                 lo, hi = self.r(), self.r()
                 self.e("shl.b32 %s, %s, 16;" % (lo, w))
                 self.e("and.b32 %s, %s, 0xffff0000;" % (hi, w))
-                self.pack(lo, hi, self.A[2 * h + i])
+                self.pack(lo, hi, A[2 * h + i])
             self.label(ln)
         self.jump()
 
-    def prefetch(self, adr, pfullk, esize):
-        """pulls this CTA's next tile of a FULL operand into L2 while the current one is processed"""
-        skip = self.newlabel("pf")
-        pr, pa = self.p(), self.rd()
-        self.e("setp.ne.s64 %s, %%tnext, 0;" % pr)
-        self.e("and.pred %s, %s, %s;" % (pr, pr, pfullk))
-        self.e("@!%s bra.uni %s;" % (pr, skip))
-        self.e("mad.lo.s64 %s, %%tnext, %d, %s;" % (pa, esize, adr))
+    def store_f32_slow(self, adr):
+        A = self.A
+        pvec = self.pvec()
         for h in range(2):
-            ph, ps = self.p(), self.r()
-            self.e("add.u32 %s, %%pos0, %d;" % (ps, h * NT * 4))
-            self.e("setp.lt.s32 %s, %s, %%limit;" % (ph, ps))
-            self.e("@%s prefetch.global.L2 [%s+%d];" % (ph, pa, h * NT * 4 * esize))
-        self.label(skip)
-
-    def leaf_gst(self):
-        ptr, kind, dt = self.operand()
-        self.fetch()
-        lout = self.newlabel("gst")
-        pfullk, pscal, pbf, pr = self.p(), self.p(), self.p(), self.p()
-        base = self.rd()
-        self.e("setp.eq.u32 %s, %s, 0;" % (pfullk, kind))
-        self.e("setp.eq.u32 %s, %s, 2;" % (pscal, kind))
-        self.e("setp.ne.u32 %s, %s, 0;" % (pbf, dt))
-        self.e("selp.b64 %s, %%tbase, 0, %s;" % (base, pfullk))
-        # ROW and SCALAR shaped outputs are written by the first tile only
-        self.e("or.pred %s, %s, %%pfirst;" % (pr, pfullk))
-        self.e("@!%s bra.uni %s;" % (pr, lout))
-        lscal, lbf, lslow = self.newlabel("gst"), self.newlabel("gst"), self.newlabel("gst")
-        self.e("@%s bra.uni %s;" % (pscal, lscal))
-        self.e("@%s bra.uni %s;" % (pbf, lbf))
-        adr = self.rd()
-        self.e("add.s64 %s, %s, %%pos0_64;" % (adr, base))
-        self.e("shl.b64 %s, %s, 2;" % (adr, adr))
-        self.e("add.u64 %s, %s, %s;" % (adr, adr, ptr))
-        self.e("@!%%pfast bra.uni %s;" % lslow)
-        self.stg_v(adr, self.A)
-        self.jump()
-        self.label(lslow)
-        for h in range(2):
-            lv, ln = self.newlabel("gst"), self.newlabel("gst")
+            lv, ln = self.newlabel("st"), self.newlabel("st")
             pv, pos3 = self.p(), self.r()
             self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
-            self.e("setp.lt.s32 %s, %s, %%limit;" % (pv, pos3))
-            self.e("and.pred %s, %s, %%pvec;" % (pv, pv))
+            self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
+            self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
-            sc = self.unpack(self.A[2 * h]) + self.unpack(self.A[2 * h + 1])
+            sc = self.unpack(A[2 * h]) + self.unpack(A[2 * h + 1])
             for e_ in range(4):
                 pe = self.p()
-                self.e("setp.lt.s32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
+                self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
                 self.e("@%s st.global.f32 [%s+%d], %s;" % (pe, adr, h * HALF_BYTES + 4 * e_, sc[e_]))
             self.e("bra %s;" % ln)
             self.label(lv)
-            self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (adr, h * HALF_BYTES, self.A[2 * h], self.A[2 * h + 1]))
+            self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (adr, h * HALF_BYTES, A[2 * h], A[2 * h + 1]))
             self.label(ln)
+
+    def leaf_gstf(self):
+        """acc -> fp32 FULL operand"""
+        ptr, _, _ = self.operand(False)
+        self.fetch()
+        adr = self.rd()
+        self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
+        slow = self.newlabel("gstf")
+        self.e("@!%%pfull bra.uni %s;" % slow)
+        self.stg_v(adr, self.A)
+        self.jump()
+        self.label(slow)
+        self.store_f32_slow(adr)
+        self.jump()
+
+    def leaf_gst(self):
+        """acc -> any operand"""
+        A = self.A
+        ptr, kind, dt = self.operand()
+        self.fetch()
+        lout = self.newlabel("gst")
+        pfullk, pscal, pbf, pr, pfirst = self.p(), self.p(), self.p(), self.p(), self.p()
+        off, p64 = self.rd(), self.pos0_64()
+        self.e("setp.eq.u32 %s, %s, 0;" % (pfullk, kind))
+        self.e("setp.eq.u32 %s, %s, 2;" % (pscal, kind))
+        self.e("setp.ne.u32 %s, %s, 0;" % (pbf, dt))
+        self.e("shl.b64 %s, %s, 2;" % (p64, p64))
+        self.e("selp.b64 %s, %%tb4, %s, %s;" % (off, p64, pfullk))
+        # ROW and SCALAR shaped outputs are written by the first tile only
+        self.e("setp.eq.u32 %s, %%tile, 0;" % pfirst)
+        self.e("or.pred %s, %s, %s;" % (pr, pfullk, pfirst))
+        self.e("@!%s bra.uni %s;" % (pr, lout))
+        lscal, lbf = self.newlabel("gst"), self.newlabel("gst")
+        self.e("@%s bra.uni %s;" % (pscal, lscal))
+        self.e("@%s bra.uni %s;" % (pbf, lbf))
+        adr = self.rd()
+        self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        self.store_f32_slow(adr)
         self.jump()
         # bf16 tensors
         self.label(lbf)
         adr = self.rd()
-        self.e("add.s64 %s, %s, %%pos0_64;" % (adr, base))
-        self.e("shl.b64 %s, %s, 1;" % (adr, adr))
-        self.e("add.u64 %s, %s, %s;" % (adr, adr, ptr))
+        self.e("shr.u64 %s, %s, 1;" % (off, off))
+        self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        pvec = self.pvec()
         for h in range(2):
             lv, ln = self.newlabel("gst"), self.newlabel("gst")
             pv, pos3 = self.p(), self.r()
-            sc = self.unpack(self.A[2 * h]) + self.unpack(self.A[2 * h + 1])
+            sc = self.unpack(A[2 * h]) + self.unpack(A[2 * h + 1])
             w0, w1 = self.r(), self.r()
             self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w0, sc[1], sc[0]))
             self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w1, sc[3], sc[2]))
             self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
-            self.e("setp.lt.s32 %s, %s, %%limit;" % (pv, pos3))
-            self.e("and.pred %s, %s, %%pvec;" % (pv, pv))
+            self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
+            self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
             for e_ in range(4):
                 pe, hh, w = self.p(), self.t("h"), (w0, w1)[e_ >> 1]
-                self.e("setp.lt.s32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
+                self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
                 if e_ & 1:
                     self.e("{ .reg .b16 %%lo; mov.b32 {%%lo, %s}, %s; }" % (hh, w))
                 else:
@@ -565,12 +645,9 @@ class Kernel:
         self.jump()
         # one scalar, written by thread 0
         self.label(lscal)
-        skip = self.newlabel("gst")
-        p0 = self.p()
-        self.e("setp.ne.u32 %s, %%tx, 0;" % p0)
-        self.e("@%s bra %s;" % (p0, skip))
-        a0, _ = self.unpack(self.A[0])
-        sb = self.newlabel("gst")
+        skip, sb = self.newlabel("gst"), self.newlabel("gst")
+        self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
+        a0, _ = self.unpack(A[0])
         self.e("@%s bra.uni %s;" % (pbf, sb))
         self.e("st.global.f32 [%s], %s;" % (ptr, a0))
         self.e("bra %s;" % skip)
@@ -583,6 +660,13 @@ class Kernel:
         self.jump()
 
     # ---- leaves -------------------------------------------------------------------------------
+    def lane_sum(self, vals):
+        """sum of the 8 lanes of a packed V-wide value, as one scalar"""
+        lo, hi = self.unpack(self.add2(self.add2(vals[0], vals[1]), self.add2(vals[2], vals[3])))
+        d = self.f()
+        self.e("add.f32 %s, %s, %s;" % (d, lo, hi))
+        return d
+
     def leaf_joint(self, op, k):
         A, R = self.A, self.R[k]
         if op in ("rtos", "stor"):
@@ -599,6 +683,32 @@ class Kernel:
                 self.stg_v(a, R)
             else:
                 self.ldg_v(a, R)
+        elif op == "gldr":
+            self.leaf_gldf(R, A)
+            return
+        elif op in ("sincosr", "cossinr"):
+            self.fetch()
+            S, C = self.sincos(A)
+            self.mov_v(R, C if op == "sincosr" else S)
+            self.mov_v(A, S if op == "sincosr" else C)
+        elif op.startswith("macc"):
+            self.fetch()
+            acc = self.S[int(op[4])]
+            tail = self.newlabel("ma")
+            self.e("@!%%pfull bra.uni %s;" % tail)
+            t = self.mul2(A[0], R[0])
+            for i in range(1, NP): t = self.fma2(A[i], R[i], t)
+            lo, hi = self.unpack(t)
+            self.e("add.f32 %s, %s, %s;" % (lo, lo, hi))
+            self.e("add.f32 %s, %s, %s;" % (acc, acc, lo))
+            self.jump()
+            self.label(tail)
+            m = self.packs(self.mask_tail(self.scalars(A)))
+            t = self.mul2(m[0], R[0])
+            for i in range(1, NP): t = self.fma2(m[i], R[i], t)
+            lo, hi = self.unpack(t)
+            self.e("add.f32 %s, %s, %s;" % (lo, lo, hi))
+            self.e("add.f32 %s, %s, %s;" % (acc, acc, lo))
         elif op == "fmaur":
             u = self.uniform()
             self.fetch()
@@ -679,11 +789,11 @@ class Kernel:
             self.fetch(); S, _ = self.sincos(A, True, False); self.mov_v(A, S)
         elif op == "cos":
             self.fetch(); _, C = self.sincos(A, False, True); self.mov_v(A, C)
-        elif op == "sincos":
+        elif op in ("sincos", "cossin"):
             a = self.slot_addr(); self.fetch()
             S, C = self.sincos(A)
-            self.sts_v(a, C)
-            self.mov_v(A, S)
+            self.sts_v(a, C if op == "sincos" else S)
+            self.mov_v(A, S if op == "sincos" else C)
         elif op == "expc":
             self.fetch(); self.mov_v(A, self.expc(A))
         elif op == "tanh":
@@ -745,6 +855,10 @@ class Kernel:
             self.leaf_gld(); return
         elif op == "gst":
             self.leaf_gst(); return
+        elif op == "gldf":
+            self.leaf_gldf(A); return
+        elif op == "gstf":
+            self.leaf_gstf(); return
         elif op == "fill":
             a = self.spill_addr(); self.fetch(); self.ldg_v(a, A)
         elif op == "spill":
@@ -756,19 +870,36 @@ class Kernel:
         elif op == "loop_begin":
             self.fetch()
             self.e("bar.sync 0;")          # uniforms written by thread 0 are visible from here on
-            self.e("sub.u32 %loop_ip, %ip, 8;")   # entry of the first body instruction (just fetched)
         elif op == "loop_end":
             self.leaf_loop_end(); return
         elif op == "colout":
             self.leaf_colout()
         elif op == "scalout":
             self.leaf_scalout()
+        elif op.startswith("sacc"):
+            self.fetch()
+            acc = self.S[int(op[4])]
+            tail = self.newlabel("sa")
+            self.e("@!%%pfull bra.uni %s;" % tail)
+            self.e("add.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(A)))
+            self.jump()
+            self.label(tail)
+            self.e("add.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(self.packs(self.mask_tail(self.scalars(A))))))
+        elif op.startswith("ascal"):
+            self.leaf_scalout([self.S[int(op[5])]])
         elif op == "end":
             self.e("exit;")
             return
         else:
             raise ValueError(op)
         self.jump()
+
+    def warp_and_lane(self):
+        lane, warp, t = self.r(), self.r(), self.r()
+        self.e("shr.u32 %s, %%pos0, 2;" % t)
+        self.e("and.b32 %s, %s, 31;" % (lane, t))
+        self.e("shr.u32 %s, %s, 5;" % (warp, t))
+        return warp, lane
 
     def leaf_rowsum(self):
         A = self.A
@@ -788,17 +919,18 @@ class Kernel:
             t = self.f()
             self.e("shfl.sync.bfly.b32 %s, %s, %d, 0x1f, 0xffffffff;" % (t, s, o))
             self.e("add.f32 %s, %s, %s;" % (s, s, t))
+        warp, lane = self.warp_and_lane()
         pr, a = self.p(), self.r()
-        self.e("setp.eq.u32 %s, %%lane, 0;" % pr)
-        self.e("shl.b32 %s, %%warp, 2;" % a)
-        self.e("add.u32 %s, %s, %%redb;" % (a, a))
-        self.e("@%s st.shared.f32 [%s], %s;" % (pr, a, s))
+        self.e("setp.eq.u32 %s, %s, 0;" % (pr, lane))
+        self.e("shl.b32 %s, %s, 2;" % (a, warp))
+        self.e("add.u32 %s, %s, %%ub;" % (a, a))
+        self.e("@%s st.shared.f32 [%s+%d], %s;" % (pr, a, OFF_RED, s))
         self.e("bar.sync 0;")
         tot = self.f()
         self.e("mov.f32 %s, 0f00000000;" % tot)
         for i in range(NT // 128):
             q = [self.f() for _ in range(4)]
-            self.e("ld.shared.v4.f32 {%s, %s, %s, %s}, [%%redb+%d];" % (q[0], q[1], q[2], q[3], 16 * i))
+            self.e("ld.shared.v4.f32 {%s, %s, %s, %s}, [%%ub+%d];" % (q[0], q[1], q[2], q[3], OFF_RED + 16 * i))
             for x in q: self.e("add.f32 %s, %s, %s;" % (tot, tot, x))
         self.e("bar.sync 0;")
         tt = self.splat(tot)
@@ -806,28 +938,27 @@ class Kernel:
 
     def leaf_uload(self):
         """U[arg & 511] = scalar operand[arg >> 9], by thread 0"""
-        skip, lb = self.newlabel("ul"), self.newlabel("ul")
-        ui, oi, a, ptr, dt, pr, pb, v = self.r(), self.r(), self.r(), self.rd(), self.r(), self.p(), self.p(), self.f()
+        skip, lb, lst = self.newlabel("ul"), self.newlabel("ul"), self.newlabel("ul")
+        ui, oi, a, ptr, dt, pb, v = self.r(), self.r(), self.r(), self.rd(), self.r(), self.p(), self.f()
         self.e("and.b32 %s, %%arg, 511;" % ui)
         self.e("shr.u32 %s, %%arg, 9;" % oi)
         self.fetch()
-        self.e("setp.ne.u32 %s, %%tx, 0;" % pr)
-        self.e("@%s bra %s;" % (pr, skip))
+        self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
         self.e("shl.b32 %s, %s, 4;" % (a, oi))
-        self.e("add.u32 %s, %s, %%opb;" % (a, a))
-        self.e("ld.shared.u64 %s, [%s];" % (ptr, a))
-        self.e("ld.shared.u32 %s, [%s+12];" % (dt, a))
+        self.e("add.u32 %s, %s, %%ub;" % (a, a))
+        self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
+        self.e("ld.shared.u32 %s, [%s+%d];" % (dt, a, OFF_OPB + 12))
         self.e("setp.ne.u32 %s, %s, 0;" % (pb, dt))
         self.e("@%s bra %s;" % (pb, lb))
         self.e("ld.global.nc.f32 %s, [%s];" % (v, ptr))
-        self.e("bra %s;" % (skip + "_st"))
+        self.e("bra %s;" % lst)
         self.label(lb)
         hh, w = self.t("h"), self.r()
         self.e("ld.global.nc.u16 %s, [%s];" % (hh, ptr))
         self.e("cvt.u32.u16 %s, %s;" % (w, hh))
         self.e("shl.b32 %s, %s, 16;" % (w, w))
         self.e("mov.b32 %s, %s;" % (v, w))
-        self.label(skip + "_st")
+        self.label(lst)
         self.e("shl.b32 %s, %s, 2;" % (ui, ui))
         self.e("add.u32 %s, %s, %%ub;" % (ui, ui))
         self.e("st.shared.f32 [%s], %s;" % (ui, v))
@@ -836,17 +967,17 @@ class Kernel:
     def leaf_uconst(self):
         """U[arg] = the raw word that follows in the undecoded stream, by thread 0"""
         skip = self.newlabel("uc")
-        ui, idx, pr, ga, w = self.r(), self.r(), self.p(), self.rd(), self.r()
+        ui, idx, ga, w, cb = self.r(), self.r(), self.rd(), self.r(), self.r()
         self.e("shl.b32 %s, %%arg, 2;" % ui)
         self.e("add.u32 %s, %s, %%ub;" % (ui, ui))
-        self.e("sub.u32 %s, %%ip, %%codeb;" % idx)     # ip points at the literal's entry: 8 bytes per word
+        self.e("mov.u32 %s, dsm;" % cb)
+        self.e("sub.u32 %s, %%ip, %s;" % (idx, cb))    # ip points at the literal's entry: 8 bytes per word
         self.e("shr.u32 %s, %s, 1;" % (idx, idx))          # -> byte offset in the 4-byte stream
         self.e("add.u32 %ip, %ip, 8;")
         self.fetch()
-        self.e("setp.ne.u32 %s, %%tx, 0;" % pr)
-        self.e("@%s bra %s;" % (pr, skip))
+        self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
         self.e("cvt.u64.u32 %s, %s;" % (ga, idx))
-        self.e("add.u64 %s, %s, %%code;" % (ga, ga))
+        self.e("add.u64 %s, %s, %s;" % (ga, ga, self.param(P_CODE, "u64")))
         self.e("ld.global.nc.u32 %s, [%s];" % (w, ga))
         self.e("st.shared.u32 [%s], %s;" % (ui, w))
         self.label(skip)
@@ -854,47 +985,53 @@ class Kernel:
 
     def leaf_loop_end(self):
         out = self.newlabel("le")
-        pr = self.p()
-        self.e("add.s64 %tile, %tile, %gs;")
-        self.e("setp.ge.s64 %s, %%tile, %%ntiles;" % pr)
+        pr, cb = self.p(), self.r()
+        self.e("add.u32 %%tile, %%tile, %s;" % self.param(P_GRID))
+        self.e("setp.ge.u32 %s, %%tile, %s;" % (pr, self.param(P_NTILES)))
         self.e("@%s bra.uni %s;" % (pr, out))
         self.set_tile()
-        self.e("mov.u32 %ip, %loop_ip;")
+        self.e("mov.u32 %s, dsm;" % cb)
+        self.e("mad.lo.u32 %%ip, %s, 8, %s;" % (self.param(P_LOOPSTART), cb))
         self.label(out)
         self.fetch()
         self.jump()
 
+    def partial_index(self):
+        """arg * grid + cta (taken before the fetch)"""
+        o, t, cta = self.rd(), self.rd(), self.r()
+        self.e("mul.wide.u32 %s, %%arg, %s;" % (o, self.param(P_GRID)))
+        self.e("mov.u32 %s, %%ctaid.x;" % cta)
+        self.e("cvt.u64.u32 %s, %s;" % (t, cta))
+        self.e("add.u64 %s, %s, %s;" % (o, o, t))
+        return o
+
     def leaf_colout(self):
         """column partial sums: colpart[arg][cta][c] = acc"""
         A = self.A
-        o, t = self.rd(), self.rd()
-        self.e("mul.wide.u32 %s, %%arg, %%ncta;" % o)
+        o = self.partial_index()
         self.fetch()
-        self.e("cvt.u64.u32 %s, %%cta;" % t)
-        self.e("add.u64 %s, %s, %s;" % (o, o, t))
-        self.e("mul.lo.u64 %s, %s, %%cols64;" % (o, o))
-        self.e("add.u64 %s, %s, %%pos0_64;" % (o, o))
+        cols, c64 = self.param(P_COLS), self.rd()
+        self.e("cvt.u64.u32 %s, %s;" % (c64, cols))
+        self.e("mul.lo.u64 %s, %s, %s;" % (o, o, c64))
+        self.e("add.u64 %s, %s, %s;" % (o, o, self.pos0_64()))
         self.e("shl.b64 %s, %s, 2;" % (o, o))
-        self.e("add.u64 %s, %s, %%colpart;" % (o, o))
+        self.e("add.u64 %s, %s, %s;" % (o, o, self.param(P_COLPART, "u64")))
         sc = self.scalars(A)
         for j in range(V):
             pr = self.p()
-            self.e("setp.lt.s32 %s, %s, %%cols;" % (pr, self.lane_pos(j)))
+            self.e("setp.lt.u32 %s, %s, %s;" % (pr, self.lane_pos(j), cols))
             self.e("@%s st.global.f32 [%s+%d], %s;" % (pr, o, ((j >> 2) * NT * 4 + (j & 3)) * 4, sc[j]))
 
-    def leaf_scalout(self):
-        """scalar partial sum: scalpart[arg][cta] = block sum of acc in fp64"""
+    def leaf_scalout(self, values=None):
+        """scalar partial sum: scalpart[arg][cta] = block sum in fp64 of acc (or of the given scalars)"""
         A = self.A
-        o, t = self.rd(), self.rd()
-        self.e("mul.wide.u32 %s, %%arg, %%ncta;" % o)
+        o = self.partial_index()
         self.fetch()
-        self.e("cvt.u64.u32 %s, %%cta;" % t)
-        self.e("add.u64 %s, %s, %s;" % (o, o, t))
         self.e("shl.b64 %s, %s, 3;" % (o, o))
-        self.e("add.u64 %s, %s, %%scalpart;" % (o, o))
+        self.e("add.u64 %s, %s, %s;" % (o, o, self.param(P_SCALPART, "u64")))
         s = self.fd()
         self.e("mov.f64 %s, 0d0000000000000000;" % s)
-        for x in self.scalars(A):
+        for x in (values if values is not None else self.scalars(A)):
             d = self.fd()
             self.e("cvt.f64.f32 %s, %s;" % (d, x))
             self.e("add.f64 %s, %s, %s;" % (s, s, d))
@@ -905,21 +1042,20 @@ class Kernel:
             self.e("shfl.sync.bfly.b32 %s, %s, %d, 0x1f, 0xffffffff;" % (h2, hi, off))
             self.e("mov.b64 %s, {%s, %s};" % (d, l2, h2))
             self.e("add.f64 %s, %s, %s;" % (s, s, d))
+        warp, lane = self.warp_and_lane()
         pr, a = self.p(), self.r()
-        self.e("setp.eq.u32 %s, %%lane, 0;" % pr)
-        self.e("shl.b32 %s, %%warp, 3;" % a)
-        self.e("add.u32 %s, %s, %%redb;" % (a, a))
-        self.e("@%s st.shared.f64 [%s], %s;" % (pr, a, s))
+        self.e("setp.eq.u32 %s, %s, 0;" % (pr, lane))
+        self.e("shl.b32 %s, %s, 3;" % (a, warp))
+        self.e("add.u32 %s, %s, %%ub;" % (a, a))
+        self.e("@%s st.shared.f64 [%s+%d], %s;" % (pr, a, OFF_RED, s))
         self.e("bar.sync 0;")
         skip = self.newlabel("so")
-        p0 = self.p()
-        self.e("setp.ne.u32 %s, %%tx, 0;" % p0)
-        self.e("@%s bra %s;" % (p0, skip))
+        self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
         tot = self.fd()
         self.e("mov.f64 %s, 0d0000000000000000;" % tot)
         for i in range(NT // 32):
             d = self.fd()
-            self.e("ld.shared.f64 %s, [%%redb+%d];" % (d, 8 * i))
+            self.e("ld.shared.f64 %s, [%%ub+%d];" % (d, OFF_RED + 8 * i))
             self.e("add.f64 %s, %s, %s;" % (tot, tot, d))
         self.e("st.global.f64 [%s], %s;" % (o, tot))
         self.label(skip)
@@ -930,106 +1066,90 @@ class Kernel:
         nr = self.nr
         cases = []
         for op in JOINT:
-            for k in range(nr):
-                cases.append(("j", op, k))
+            for k in range(JOINT_STRIDE):
+                cases.append(("j", op, k) if k < nr else ("bad", op, k))
         for op in PLAIN:
             cases.append(("p", op, 0))
-        labels = ["$C_%s_%d" % (self.name, i) for i in range(len(cases))]
+        bad = "$BAD_%s" % self.name
+        labels = [bad if c[0] == "bad" else "$C_%s_%d" % (self.name, i) for i, c in enumerate(cases)]
         body = self.lines
-        # ---- prologue ----
         e = self.e
-        e("mov.u32 %tx, %tid.x;")
-        e("mov.u32 %cta, %ctaid.x;")
-        e("mov.u32 %ncta, %nctaid.x;")
-        e("and.b32 %lane, %tx, 31;")
-        e("shr.u32 %warp, %tx, 5;")
-        e("shl.b32 %pos0, %tx, 2;")
-        e("cvt.u64.u32 %pos0_64, %pos0;")
-        e("ld.param.u64 %%code, [VP+%d];" % P_CODE)
-        e("ld.param.s32 %%ncode, [VP+%d];" % P_NCODE)
-        e("ld.param.s32 %%rowmode, [VP+%d];" % P_ROWMODE)
-        e("ld.param.s64 %%n, [VP+%d];" % P_N)
-        e("ld.param.s32 %%cols, [VP+%d];" % P_COLS)
-        e("ld.param.s32 %%nspill, [VP+%d];" % P_NSPILL)
-        e("ld.param.u64 %%spb, [VP+%d];" % P_SPILL)
-        e("ld.param.u64 %%colpart, [VP+%d];" % P_COLPART)
-        e("ld.param.u64 %%scalpart, [VP+%d];" % P_SCALPART)
-        e("cvt.s64.s32 %cols64, %cols;")
-        e("setp.ne.s32 %prow, %rowmode, 0;")
-        e("cvt.u64.u32 %gs, %ncta;")
-        # shared memory: code | uniforms | reduction scratch | operand table | slots
-        e("mov.u32 %codeb, dsm;")
-        t0 = self.r()
-        e("add.s32 %s, %%ncode, 3;" % t0)
+        # ---- prologue ----
+        tx, ncode, t0 = self.r(), self.param(P_NCODE, "s32"), self.r()
+        e("mov.u32 %s, %%tid.x;" % tx)
+        e("shl.b32 %%pos0, %s, 2;" % tx)
+        # shared memory: decoded code | uniforms | reduction scratch | operand table | slots
+        e("add.s32 %s, %s, 3;" % (t0, ncode))
         e("and.b32 %s, %s, 0xfffffffc;" % (t0, t0))
         e("shl.b32 %s, %s, 3;" % (t0, t0))
-        e("add.u32 %%ub, %%codeb, %s;" % t0)
-        e("add.u32 %%redb, %%ub, %d;" % (MAX_UNIFORMS * 4))
-        e("add.u32 %opb, %redb, 512;")
-        e("add.u32 %%sa, %%opb, %d;" % (MAX_OPERANDS * 16))
-        t1 = self.r()
-        e("shl.b32 %s, %%tx, 4;" % t1)
-        e("add.u32 %%sa, %%sa, %s;" % t1)
+        e("mov.u32 %ub, dsm;")
+        e("add.u32 %%ub, %%ub, %s;" % t0)
+        e("mad.lo.u32 %%sa, %s, 16, %%ub;" % tx)
+        e("add.u32 %%sa, %%sa, %d;" % OFF_SLOTS)
         # operand table -> shared memory (one entry per thread)
         for i in range(MAX_OPERANDS):
             pr, ptr, k, d = self.p(), self.rd(), self.r(), self.r()
-            e("setp.eq.u32 %s, %%tx, %d;" % (pr, i))
+            e("setp.eq.u32 %s, %s, %d;" % (pr, tx, i))
             e("ld.param.u64 %s, [VP+%d];" % (ptr, P_OPERAND + 16 * i))
             e("ld.param.u32 %s, [VP+%d];" % (k, P_OPERAND + 16 * i + 8))
             e("ld.param.u32 %s, [VP+%d];" % (d, P_OPERAND + 16 * i + 12))
-            e("@%s st.shared.u64 [%%opb+%d], %s;" % (pr, 16 * i, ptr))
-            e("@%s st.shared.v2.u32 [%%opb+%d], {%s, %s};" % (pr, 16 * i + 8, k, d))
+            e("@%s st.shared.u64 [%%ub+%d], %s;" % (pr, OFF_OPB + 16 * i, ptr))
+            e("@%s st.shared.v2.u32 [%%ub+%d], {%s, %s};" % (pr, OFF_OPB + 16 * i + 8, k, d))
         # decode the instruction stream: {case id, argument} per word
         lp, ld_ = self.newlabel("dec"), self.newlabel("dec")
-        i_, pr, ga, w, c, a, sa = self.r(), self.p(), self.rd(), self.r(), self.r(), self.r(), self.r()
-        e("mov.u32 %s, %%tx;" % i_)
+        i_, pr, ga, w, c, a, sa, code = self.r(), self.p(), self.rd(), self.r(), self.r(), self.r(), self.r(), self.param(P_CODE, "u64")
+        e("mov.u32 %s, %s;" % (i_, tx))
         self.label(lp)
-        e("setp.ge.s32 %s, %s, %%ncode;" % (pr, i_))
+        e("setp.ge.s32 %s, %s, %s;" % (pr, i_, ncode))
         e("@%s bra %s;" % (pr, ld_))
         e("mul.wide.u32 %s, %s, 4;" % (ga, i_))
-        e("add.u64 %s, %s, %%code;" % (ga, ga))
+        e("add.u64 %s, %s, %s;" % (ga, ga, code))
         e("ld.global.nc.u32 %s, [%s];" % (w, ga))
         e("and.b32 %s, %s, 1023;" % (c, w))
         e("shr.u32 %s, %s, 14;" % (a, w))
-        e("shl.b32 %s, %s, 3;" % (sa, i_))
-        e("add.u32 %s, %s, %%codeb;" % (sa, sa))
+        e("mov.u32 %s, dsm;" % sa)
+        e("mad.lo.u32 %s, %s, 8, %s;" % (sa, i_, sa))
         e("st.shared.v2.u32 [%s], {%s, %s};" % (sa, c, a))
         e("add.u32 %s, %s, %d;" % (i_, i_, NT))
         e("bra %s;" % lp)
         self.label(ld_)
         e("bar.sync 0;")
         # per-CTA spill area: spill + cta * n_spill * TILE floats, this thread's 16 bytes
-        t2, t3 = self.rd(), self.rd()
-        e("mul.wide.u32 %s, %%cta, %d;" % (t2, SLOT_BYTES))
-        e("cvt.s64.s32 %s, %%nspill;" % t3)
-        e("mad.lo.u64 %%spb, %s, %s, %%spb;" % (t2, t3))
-        e("mul.wide.u32 %s, %%tx, 16;" % t2)
+        t2, t3, cta = self.rd(), self.rd(), self.r()
+        e("mov.u32 %s, %%ctaid.x;" % cta)
+        e("mul.wide.u32 %s, %s, %d;" % (t2, cta, SLOT_BYTES))
+        e("cvt.u64.u32 %s, %s;" % (t3, self.param(P_NSPILL)))
+        e("mad.lo.u64 %%spb, %s, %s, %s;" % (t2, t3, self.param(P_SPILL, "u64")))
+        e("mul.wide.u32 %s, %s, 16;" % (t2, tx))
         e("add.u64 %%spb, %%spb, %s;" % t2)
         for r_ in self.A + sum(self.R, []):
             e("mov.b64 %s, 0;" % r_)
-        # tiles
-        fl, dn = self.newlabel("nt"), self.newlabel("nt")
-        e("@!%%prow bra.uni %s;" % fl)
-        e("mov.s64 %ntiles, %n;")
-        e("bra.uni %s;" % dn)
-        self.label(fl)
-        e("add.s64 %%ntiles, %%n, %d;" % (TILE - 1))
-        e("shr.s64 %ntiles, %ntiles, 12;")
-        self.label(dn)
-        e("cvt.u64.u32 %tile, %cta;")
+        for r_ in self.S:
+            e("mov.f32 %s, 0f00000000;" % r_)
+        e("mov.u32 %%tile, %s;" % cta)
         self.set_tile()
-        e("mov.u32 %ip, %codeb;")
-        e("mov.u32 %loop_ip, %codeb;")
+        e("mov.u32 %ip, dsm;")
         self.fetch()
         e("JT_%s: .branchtargets %s;" % (self.name, ", ".join(labels)))
         self.jump()
         # ---- leaves ----
         for lab, (kind, op, k) in zip(labels, cases):
+            if kind == "bad":
+                continue
             self.label(lab)
             if kind == "j":
                 self.leaf_joint(op, k)
             else:
                 self.leaf_plain(op)
+        # a register slot this build does not have: report and stop (the host never emits one)
+        self.label(bad)
+        skip = self.newlabel("bad")
+        v = self.r()
+        e("@!%s bra %s;" % (self.tx_is_zero(), skip))
+        e("mov.u32 %s, -7;" % v)
+        e("st.global.u32 [%s], %s;" % (self.param(P_STATUS, "u64"), v))
+        self.label(skip)
+        e("exit;")
         # ---- assemble text ----
         head = []
         head.append(".const .align 8 .b64 KT_%s[%d] = {%s};" % (self.name, max(1, len(self.kt)), ", ".join("0x%016X" % w for w in self.kt) or "0"))
@@ -1040,16 +1160,16 @@ class Kernel:
         decl = []
         for kind, ty in (("f", ".f32"), ("r", ".b32"), ("rd", ".b64"), ("p", ".pred"), ("fd", ".f64"), ("h", ".b16")):
             if self.cnt[kind]:
-                decl.append("\t.reg %s %%%s<%d>;" % (ty, {"f": "f", "r": "r", "rd": "rd", "p": "p", "fd": "fd", "h": "h"}[kind], self.cnt[kind]))
-        decl.append("\t.reg .b32 %tx, %cta, %ncta, %lane, %warp, %pos0, %ncode, %rowmode, %cols, %nspill, %limit;")
-        decl.append("\t.reg .b32 %codeb, %ub, %redb, %opb, %sa, %ip, %loop_ip, %case, %arg;")
-        decl.append("\t.reg .b64 %pos0_64, %code, %n, %spb, %colpart, %scalpart, %cols64, %gs, %tile, %ntiles, %tbase, %tnext;")
-        decl.append("\t.reg .pred %prow, %pfull, %pvec, %pfirst, %pfast;")
+                decl.append("\t.reg %s %%%s<%d>;" % (ty, kind, self.cnt[kind]))
+        decl.append("\t.reg .b32 %pos0, %limit, %tnext, %tile, %ub, %sa, %ip, %case, %arg;")
+        decl.append("\t.reg .b64 %tb4, %spb;")
+        decl.append("\t.reg .pred %pfull;")
+        decl.append("\t.reg .f32 %s;" % ", ".join(self.S))
         decl.append("\t.reg .b64 %s;" % ", ".join(self.A + sum(self.R, [])))
         return "\n".join(head + decl + body + ["}"]) + "\n"
 
 
-VARIANTS = [("dragon_vm_r7", 7, 1)]
+VARIANTS = [("dragon_vm_wide", 7, 1), ("dragon_vm_dense", 3, 2)]   # name, register slots, CTAs per SM
 
 
 def generate():

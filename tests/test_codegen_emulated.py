@@ -15,7 +15,7 @@ def emulate(desc, inputs, outputs, feeds):
     assert f.num_launches() <= 2, f.describe()
     step = f.vm_step(0)
     shapes = {j: tuple(desc["tensors"][o]["shape"]) for j, o in enumerate(outputs)}
-    out, colout, scalout = run_step(step, feeds, shapes)
+    out, colout, scalout = run_step(step, feeds, shapes, nr=step["n_regs"])
     for kind, acc, pos in step["reduced"]:
         out[pos] = np.asarray(colout[acc] if kind == 0 else scalout[acc], dtype=np.float64).reshape(shapes[pos])
     return [out[j] for j in range(len(outputs))], f

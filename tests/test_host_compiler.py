@@ -168,7 +168,7 @@ def test_limits_are_reported_not_faulted():
     y2 = g2.add_tensor("y", B.F32, [4, 5000])
     g2.add_op(B.OPS["Tanh"], [x2], [y2])
     f = g2.function([x2], [y2])
-    assert "flat n=20000" in f.describe()
+    assert "vm[flat" in f.describe() and " n=20000 " in f.describe()
     # fetching the same tensor twice is refused
     with pytest.raises(B.DragonError):
         g2.function([x2], [y2, y2])

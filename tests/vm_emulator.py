@@ -5,11 +5,13 @@ thread layout play no role.  Arithmetic is float64; it checks the *program*, not
 Single-step functions only (feeds and fetches as memory operands)."""
 import numpy as np
 
-NR_DEFAULT = 7
-J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr"]
+STRIDE = 8   # case id of a register-operand instruction = index * STRIDE + register slot
+J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
+     "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3"]
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
-     "rdivps", "sin", "cos", "sincos", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
-     "rbf16", "rowsum", "gld", "gst", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout", "end"]
+     "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
+     "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
+     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "end"]
 
 
 def _bf16(a):
@@ -19,11 +21,12 @@ def _bf16(a):
     return r.view(np.float32).astype(np.float64)
 
 
-def run_step(step, feeds, fetch_shapes, nr=NR_DEFAULT):
+def run_step(step, feeds, fetch_shapes, nr=STRIDE):
     """step: dict from Function.vm_step; feeds: arrays by feed position; returns {fetch position: array}."""
     code, ops = step["code"], step["operands"]
     shape = (step["n"], step["cols"]) if step["row_mode"] else (step["n"],)
-    first_plain = len(J) * nr
+    first_plain = len(J) * STRIDE
+    A = [0.0] * 4   # scalar accumulators
 
     def divp(a, b):
         return a / (1 + np.abs(b))
@@ -48,7 +51,8 @@ def run_step(step, feeds, fetch_shapes, nr=NR_DEFAULT):
         w = code[pc]; pc += 1
         cs, arg = w & 1023, w >> 14
         if cs < first_plain:
-            name, k = J[cs // nr], cs % nr
+            name, k = J[cs // STRIDE], cs % STRIDE
+            assert k < nr, "register slot %d beyond the %d of this build" % (k, nr)
             if name == "ldr": acc = R[k].copy()
             elif name == "str": R[k] = acc.copy()
             elif name in binops: acc = binops[name](acc, R[k])
@@ -58,6 +62,11 @@ def run_step(step, feeds, fetch_shapes, nr=NR_DEFAULT):
             elif name == "stor": R[k] = S[arg].copy()
             elif name == "spillr": G[arg] = R[k].copy()
             elif name == "fillr": R[k] = G[arg].copy()
+            elif name == "gldr": acc = load(arg); R[k] = acc.copy()
+            elif name == "sincosr": R[k] = np.cos(acc); acc = np.sin(acc)
+            elif name == "cossinr": R[k] = np.sin(acc); acc = np.cos(acc)
+            elif name.startswith("macc"): A[int(name[4])] += float((acc * R[k]).sum())
+            else: raise ValueError(name)
             continue
         name = P[cs - first_plain]
         if name == "ldu": acc = np.full(shape, U[arg])
@@ -69,6 +78,7 @@ def run_step(step, feeds, fetch_shapes, nr=NR_DEFAULT):
         elif name == "sin": acc = np.sin(acc)
         elif name == "cos": acc = np.cos(acc)
         elif name == "sincos": S[arg] = np.cos(acc); acc = np.sin(acc)
+        elif name == "cossin": S[arg] = np.sin(acc); acc = np.cos(acc)
         elif name == "expc": acc = np.exp(np.clip(acc, -10, 10))
         elif name == "tanh": acc = np.tanh(acc)
         elif name == "sigmoid": acc = 1 / (1 + np.exp(-acc))
@@ -81,8 +91,8 @@ def run_step(step, feeds, fetch_shapes, nr=NR_DEFAULT):
         elif name == "divpgb": acc = -np.sign(acc) / (1 + np.abs(acc)) ** 2
         elif name == "rbf16": acc = _bf16(acc)
         elif name == "rowsum": acc = np.broadcast_to(acc.sum(axis=-1, keepdims=True), shape).copy()
-        elif name == "gld": acc = load(arg)
-        elif name == "gst":
+        elif name in ("gld", "gldf"): acc = load(arg)
+        elif name in ("gst", "gstf"):
             where, pos, kind, dtype = ops[arg]
             assert where == 1
             v = acc if kind == 0 else (acc[0] if kind == 1 else acc.reshape(-1)[0])
@@ -97,6 +107,8 @@ def run_step(step, feeds, fetch_shapes, nr=NR_DEFAULT):
         elif name in ("loop{", "}loop"): pass
         elif name == "colout": colout[arg] = acc.sum(axis=0)
         elif name == "scalout": scalout[arg] = acc.sum()
+        elif name.startswith("sacc"): A[int(name[4])] += float(acc.sum())
+        elif name.startswith("ascal"): scalout[arg] = A[int(name[5])]
         elif name == "end": break
         else: raise ValueError(name)
     return out, colout, scalout
