@@ -27,9 +27,10 @@ METRIC = "pruned-graph fwd+bwd elements/sec"
 UNIT = "elements/s"
 WORKLOAD = "config 2: f=x*sin(a*x+b), x fp32[2^26], fetch df/dx, df/da, df/db"
 ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
-# dram__bytes_read.sum + dram__bytes_write.sum of vm_kernel per element, from the ncu capture summarised in
-# profiles/vm_kernel_config2.md (taken at 2^25 elements; traffic is proportional to the element count)
-NCU_DRAM_BYTES_PER_ELEM = (134.377728e6 + 94.725632e6) / (1 << 25)
+# dram__bytes_read.sum + dram__bytes_write.sum of the VM kernel per element, from the ncu capture summarised in
+# profiles/vm_dense_config2.md (taken at 2^25 elements; traffic is proportional to the element count);
+# None while no capture of the current kernel exists
+NCU_DRAM_BYTES_PER_ELEM = None
 
 
 def measured_peak_gbs():
@@ -304,8 +305,8 @@ def main():
                 "e2e": {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                         "h2d_bytes_per_step": 4 * n + 8, "d2h_bytes_per_step": 4 * n + 8},
                 "gpu_launches": f.num_launches() * args.steps,
-                "roofline": {"bound": "hbm", "kernel": "vm_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": NCU_DRAM_BYTES_PER_ELEM * n,
+                "roofline": {"bound": "hbm", "kernel": "dragon_vm_dense", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                             "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": None if NCU_DRAM_BYTES_PER_ELEM is None else NCU_DRAM_BYTES_PER_ELEM * n,
                              "kernel_ms": kern_avg_ms, "frac_of_nominal_8TBs": achieved / 8000.0}}
         if not args.skip_cpu_baseline and world == 1:
             rate, sample, _ = oracle_rate()
