@@ -332,6 +332,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         p.n_tiles = (uint32_t)(sg.row_mode ? sg.n : (sg.n + kVmTile - 1) / kVmTile);
         p.loop_start = (uint32_t)sg.loop_start;
         p.grid = (uint32_t)sg.grid;
+        p.n_full_tiles = sg.row_mode ? (sg.cols == kVmTile ? p.n_tiles : 0u) : (uint32_t)(sg.n / kVmTile);
         p.spill = reinterpret_cast<float*>(ws + sg.spill_off);
         p.colpart = reinterpret_cast<float*>(ws + sg.colpart_off);
         p.scalpart = reinterpret_cast<double*>(ws + sg.scalpart_off);

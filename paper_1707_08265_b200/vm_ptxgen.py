@@ -32,7 +32,7 @@ MAX_UNIFORMS = 512
 
 # Params (csrc/vm_isa.h): byte offsets
 P_CODE, P_SPILL, P_COLPART, P_SCALPART, P_STATUS, P_N = 0, 8, 16, 24, 32, 40
-P_NCODE, P_ROWMODE, P_COLS, P_NSPILL, P_NTILES, P_LOOPSTART, P_GRID, P_OPERAND = 48, 52, 56, 60, 64, 68, 72, 80
+P_NCODE, P_ROWMODE, P_COLS, P_NSPILL, P_NTILES, P_LOOPSTART, P_GRID, P_NFULL, P_OPERAND = 48, 52, 56, 60, 64, 68, 72, 76, 80
 P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
 # shared memory behind the decoded instruction stream: uniforms | reduction scratch | operand table | slots
 OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
@@ -989,7 +989,21 @@ class Kernel:
         self.e("add.u32 %%tile, %%tile, %s;" % self.param(P_GRID))
         self.e("setp.ge.u32 %s, %%tile, %s;" % (pr, self.param(P_NTILES)))
         self.e("@%s bra.uni %s;" % (pr, out))
+        # a full tile (the common case) only moves the offsets on; a ragged one takes the general path
+        slow, join = self.newlabel("le"), self.newlabel("le")
+        pf, pn, nt, stride, gs, nfull = self.p(), self.p(), self.r(), self.rd(), self.param(P_GRID), self.param(P_NFULL)
+        self.e("setp.lt.u32 %s, %%tile, %s;" % (pf, nfull))
+        self.e("@!%s bra.uni %s;" % (pf, slow))
+        self.e("mul.wide.u32 %s, %s, %d;" % (stride, gs, SLOT_BYTES))
+        self.e("add.u64 %%tb4, %%tb4, %s;" % stride)
+        self.e("add.u32 %s, %%tile, %s;" % (nt, gs))
+        self.e("setp.lt.u32 %s, %s, %s;" % (pn, nt, nfull))
+        self.e("shl.b32 %s, %s, 12;" % (nt, gs))
+        self.e("selp.u32 %%tnext, %s, 0, %s;" % (nt, pn))
+        self.e("bra.uni %s;" % join)
+        self.label(slow)
         self.set_tile()
+        self.label(join)
         self.e("mov.u32 %s, dsm;" % cb)
         self.e("mad.lo.u32 %%ip, %s, 8, %s;" % (self.param(P_LOOPSTART), cb))
         self.label(out)
