@@ -37,7 +37,7 @@ struct Gen {
   Shape dom;
   std::vector<int> canon;
   std::map<int, VInfo> info;
-  std::vector<uint32_t> pro, body, epi;
+  std::vector<uint32_t> pro, preamble, body, epi;
   const int nr;                  // register slots of the kernel build this program is for
   const int n_smem_max;          // shared-memory slots that build can hold
   int reg_owner[kJointStride];   // value id, -1 free, -2 pinned accumulator
@@ -359,6 +359,50 @@ struct Gen {
     if (next_use(v, pos) == kFar) { release(v); acc_val = -1; }
   }
 
+  // Loads of fp32 tensors of the full domain shape are staged through free shared-memory slots:
+  // the copy of a tile starts one iteration ahead (P_GLDA after the slot's last read, P_GLDA0
+  // before the first iteration) and the read (P_LDSW / J_LDSWR) finds it on chip.
+  void stage_loads() {
+    const char* off = std::getenv("DRAGON_VM_STAGING");
+    if (off && std::string(off) == "0") return;
+    auto load_operand = [&](uint32_t w, int* k) -> int {   // operand of a short fp32 load, or -1
+      const uint32_t cs = w & 1023u;
+      *k = -1;
+      if (cs == (uint32_t)P_GLDF) return (int)(w >> 14);
+      if (cs >= (uint32_t)(J_GLDR * kJointStride) && cs < (uint32_t)(J_GLDR * kJointStride + nr)) { *k = (int)(cs - J_GLDR * kJointStride); return (int)(w >> 14); }
+      return -1;
+    };
+    std::map<int, int> slot_of;                 // operand -> staging slot
+    std::map<int, size_t> last_read;            // operand -> position of its last load in the body
+    for (size_t i = 0; i < body.size(); ++i) {
+      int k, opd = load_operand(body[i], &k);
+      if (opd < 0 || opd >= 64) continue;
+      if (!slot_of.count(opd)) {
+        if (seg->n_smem >= n_smem_max) continue;  // no free slot: this operand keeps its direct loads
+        slot_of[opd] = seg->n_smem++;
+      }
+      last_read[opd] = i;
+    }
+    if (slot_of.empty()) return;
+    std::vector<uint32_t> out;
+    std::map<int, bool> seen;
+    for (size_t i = 0; i < body.size(); ++i) {
+      int k, opd = load_operand(body[i], &k);
+      if (opd < 0 || !slot_of.count(opd)) { out.push_back(body[i]); continue; }
+      const uint32_t sl = (uint32_t)slot_of[opd], arg = (uint32_t)opd | (sl << 6);
+      if (!seen[opd]) {                          // first read of the iteration: wait for the copy
+        out.push_back(k < 0 ? encode(P_LDSW, 0, arg) : encode(J_LDSWR * kJointStride + k, 0, arg));
+        seen[opd] = true;
+      } else {                                   // the slot still holds the tile
+        out.push_back(encode(P_LDS, 0, sl));
+        if (k >= 0) out.push_back(encode(J_STR * kJointStride + k, 0, 0));
+      }
+      if (last_read[opd] == i) out.push_back(encode(P_GLDA, 0, arg));
+    }
+    body.swap(out);
+    for (auto& so : slot_of) preamble.push_back(encode(P_GLDA0, 0, (uint32_t)so.first | ((uint32_t)so.second << 6)));
+  }
+
   int run() {
     // 1. aliases (WIDEN) and the fused domain
     canon.resize(vals.size());
@@ -490,6 +534,7 @@ struct Gen {
       fused.push_back(w);
     }
     body.swap(fused);
+    stage_loads();
     // 6. epilogue: accumulators leave as per-CTA partial sums
     for (auto& a : accs) {
       const Item& it = items[idx[a.first]];
@@ -509,6 +554,7 @@ struct Gen {
     }
     seg->code = pro;
     seg->code.push_back(encode(P_LOOP_BEGIN, 0, 0));
+    seg->code.insert(seg->code.end(), preamble.begin(), preamble.end());
     seg->loop_start = (int)seg->code.size();
     seg->code.insert(seg->code.end(), body.begin(), body.end());
     seg->code.push_back(encode(P_LOOP_END, 0, 0));

@@ -38,6 +38,7 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   J_SINCOSR,   // R = cos(acc); acc = sin(acc)
   J_COSSINR,   // R = sin(acc); acc = cos(acc)
   J_MACC0, J_MACC1, J_MACC2, J_MACC3,   // A[i] += sum over this thread's valid lanes of acc * R   (acc unchanged)
+  J_LDSWR,     // R = acc = staged operand (P_LDSW)
   J_COUNT
 };
 // The kernel exists in two builds that share this encoding: "wide" (7 register slots, one CTA per
@@ -80,6 +81,14 @@ enum Plain : int {
   P_SCALOUT,            // scalar partial sum: scalpart[arg][cta] = block sum of acc in fp64
   P_SACC0, P_SACC1, P_SACC2, P_SACC3,       // A[i] += sum over this thread's valid lanes of acc
   P_ASCAL0, P_ASCAL1, P_ASCAL2, P_ASCAL3,   // scalpart[arg][cta] = block sum of A[i] in fp64
+  // Staged loads of an fp32 operand of the full domain shape (arg = operand | slot << 6): every thread
+  // copies its own 32 bytes of a tile into S[slot] with asynchronous copies one iteration ahead, so
+  // the latency of the global load is spent while the previous tile is computed.  A thread reads only
+  // what it copied itself, so no barrier is involved.
+  P_GLDA0,              // start the copy of the current tile (before the first iteration; full tiles only)
+  P_GLDA,               // start the copy of this CTA's next tile, if it has a whole one
+  P_LDSW,               // acc = the current tile: waits for this thread's copies and reads S[slot]
+                        // (a ragged tile was not staged and is loaded directly)
   P_END,
   P_COUNT_
 };

@@ -38,13 +38,13 @@ P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
 OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
-         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3"]
+         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr"]
 JOINT_STRIDE = 8    # case id of a joint instruction = index * JOINT_STRIDE + register slot
 N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "end"]
 
 
 def f32bits(x):
@@ -172,7 +172,10 @@ class Kernel:
         return d
 
     def jump(self):
-        self.e("brx.idx.uni %%case, JT_%s;" % self.name)
+        # every leaf leaves through the one dispatch block: the assembler gives each indexed branch
+        # its own table of branch instructions (about 2 KB per site), which with one site per leaf
+        # made the code image four times larger and scattered the hot leaves
+        self.e("bra.uni $DISPATCH_%s;" % self.name)
 
     # addresses that depend on the argument (taken before the fetch overwrites %arg)
     def slot_addr(self):
@@ -477,6 +480,58 @@ class Kernel:
             self.mov_v(copy_to, dst)
         self.jump()
 
+    # ---- staged loads: arg = operand | slot << 6 ------------------------------------------------
+    def staged_operand(self):
+        """-> (ptr u64 of the operand, shared address of this thread's 16 bytes of the slot); before the fetch"""
+        a, ptr, sl, sadr = self.r(), self.rd(), self.r(), self.r()
+        self.e("and.b32 %s, %%arg, 63;" % a)
+        self.e("shl.b32 %s, %s, 4;" % (a, a))
+        self.e("add.u32 %s, %s, %%ub;" % (a, a))
+        self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
+        self.e("shr.u32 %s, %%arg, 6;" % sl)
+        self.e("mad.lo.u32 %s, %s, %d, %%sa;" % (sadr, sl, SLOT_BYTES))
+        return ptr, sadr
+
+    def async_copy(self, sadr, gadr, pred):
+        """this thread's two 16-byte pieces of a tile: global -> shared, asynchronously"""
+        for h in range(2):
+            self.e("@%s cp.async.cg.shared.global [%s+%d], [%s+%d], 16;" % (pred, sadr, h * HALF_BYTES, gadr, h * HALF_BYTES))
+        self.e("cp.async.commit_group;")
+
+    def leaf_glda(self, first):
+        ptr, sadr = self.staged_operand()
+        self.fetch()
+        adr, pr = self.rd(), self.p()
+        self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
+        if first:
+            self.e("mov.pred %s, %%pfull;" % pr)
+        else:       # %tnext is non-zero only when the whole next tile exists
+            off = self.rd()
+            self.e("setp.ne.u32 %s, %%tnext, 0;" % pr)
+            self.e("mul.wide.u32 %s, %%tnext, 4;" % off)
+            self.e("add.u64 %s, %s, %s;" % (adr, adr, off))
+        self.async_copy(sadr, adr, pr)
+        self.jump()
+
+    def leaf_ldsw(self, dst, copy_to=None):
+        ptr, sadr = self.staged_operand()
+        self.fetch()
+        slow = self.newlabel("ldsw")
+        self.e("@!%%pfull bra.uni %s;" % slow)
+        self.e("cp.async.wait_all;")
+        self.lds_v(sadr, dst)
+        if copy_to:
+            self.mov_v(copy_to, dst)
+        self.jump()
+        self.label(slow)       # a ragged tile is never staged: load it and leave it in the slot for later reads
+        adr = self.rd()
+        self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
+        self.load_f32_slow(adr, dst)
+        self.sts_v(sadr, dst)
+        if copy_to:
+            self.mov_v(copy_to, dst)
+        self.jump()
+
     def load_f32_slow(self, adr, dst):
         pvec = self.pvec()
         for h in range(2):
@@ -686,6 +741,9 @@ class Kernel:
         elif op == "gldr":
             self.leaf_gldf(R, A)
             return
+        elif op == "ldswr":
+            self.leaf_ldsw(R, A)
+            return
         elif op in ("sincosr", "cossinr"):
             self.fetch()
             S, C = self.sincos(A)
@@ -857,6 +915,12 @@ class Kernel:
             self.leaf_gst(); return
         elif op == "gldf":
             self.leaf_gldf(A); return
+        elif op == "glda0":
+            self.leaf_glda(True); return
+        elif op == "glda":
+            self.leaf_glda(False); return
+        elif op == "ldsw":
+            self.leaf_ldsw(A); return
         elif op == "gstf":
             self.leaf_gstf(); return
         elif op == "fill":
@@ -1145,7 +1209,8 @@ class Kernel:
         e("mov.u32 %ip, dsm;")
         self.fetch()
         e("JT_%s: .branchtargets %s;" % (self.name, ", ".join(labels)))
-        self.jump()
+        self.label("$DISPATCH_%s" % self.name)
+        e("brx.idx.uni %%case, JT_%s;" % self.name)
         # ---- leaves ----
         for lab, (kind, op, k) in zip(labels, cases):
             if kind == "bad":
