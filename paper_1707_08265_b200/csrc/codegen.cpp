@@ -391,6 +391,11 @@ struct Gen {
       if (opd < 0 || !slot_of.count(opd)) { out.push_back(body[i]); continue; }
       const uint32_t sl = (uint32_t)slot_of[opd], arg = (uint32_t)opd | (sl << 6);
       if (!seen[opd]) {                          // first read of the iteration: wait for the copy
+        if (last_read[opd] == i) {               // the only read: the next copy starts in the same instruction
+          out.push_back(k < 0 ? encode(P_LDSWA, 0, arg) : encode(J_LDSWAR * kJointStride + k, 0, arg));
+          seen[opd] = true;
+          continue;
+        }
         out.push_back(k < 0 ? encode(P_LDSW, 0, arg) : encode(J_LDSWR * kJointStride + k, 0, arg));
         seen[opd] = true;
       } else {                                   // the slot still holds the tile

@@ -39,6 +39,7 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   J_COSSINR,   // R = sin(acc); acc = cos(acc)
   J_MACC0, J_MACC1, J_MACC2, J_MACC3,   // A[i] += sum over this thread's valid lanes of acc * R   (acc unchanged)
   J_LDSWR,     // R = acc = staged operand (P_LDSW)
+  J_LDSWAR,    // J_LDSWR, then P_GLDA for the same operand and slot
   J_COUNT
 };
 // The kernel exists in two builds that share this encoding: "wide" (7 register slots, one CTA per
@@ -89,6 +90,7 @@ enum Plain : int {
   P_GLDA,               // start the copy of this CTA's next tile, if it has a whole one
   P_LDSW,               // acc = the current tile: waits for this thread's copies and reads S[slot]
                         // (a ragged tile was not staged and is loaded directly)
+  P_LDSWA,              // P_LDSW, then P_GLDA for the same operand and slot (the tile is read once per iteration)
   P_END,
   P_COUNT_
 };

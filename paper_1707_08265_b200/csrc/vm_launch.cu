@@ -39,12 +39,23 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
     for (int g = 0; g < jb.grid; ++g) s += (double)part[(size_t)g * jb.cols + c];
     if (jb.dtype == DRAGON_F32) reinterpret_cast<float*>(jb.out)[c] = (float)s;
     else reinterpret_cast<unsigned short*>(jb.out)[c] = (unsigned short)vmmath::bf16_bits((float)s);
-  } else if (blockIdx.x == 0 && threadIdx.x == 0) {
+  } else if (blockIdx.x == 0) {
+    // one block per scalar: strided partial sums, then a tree in shared memory; the order is
+    // fixed by the thread count, so the result is the same on every run
+    __shared__ double sh[128];
     const double* part = reinterpret_cast<const double*>(jb.part);
     double s = 0.0;
-    for (int g = 0; g < jb.grid; ++g) s += part[g];
-    if (jb.dtype == DRAGON_F32) *reinterpret_cast<float*>(jb.out) = (float)s;
-    else *reinterpret_cast<unsigned short*>(jb.out) = (unsigned short)vmmath::bf16_bits((float)s);
+    for (int g = threadIdx.x; g < jb.grid; g += 128) s += part[g];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    for (int w = 64; w > 0; w >>= 1) {
+      if ((int)threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
+      __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+      if (jb.dtype == DRAGON_F32) *reinterpret_cast<float*>(jb.out) = (float)sh[0];
+      else *reinterpret_cast<unsigned short*>(jb.out) = (unsigned short)vmmath::bf16_bits((float)sh[0]);
+    }
   }
 }
 

@@ -38,13 +38,13 @@ P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
 OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
-         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr"]
+         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar"]
 JOINT_STRIDE = 8    # case id of a joint instruction = index * JOINT_STRIDE + register slot
 N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "end"]
 
 
 def f32bits(x):
@@ -513,7 +513,16 @@ class Kernel:
         self.async_copy(sadr, adr, pr)
         self.jump()
 
-    def leaf_ldsw(self, dst, copy_to=None):
+    def next_copy(self, ptr, sadr):
+        """start the copy of this CTA's next tile (when it has a whole one) into the slot"""
+        adr, off, pr = self.rd(), self.rd(), self.p()
+        self.e("setp.ne.u32 %s, %%tnext, 0;" % pr)
+        self.e("mul.wide.u32 %s, %%tnext, 4;" % off)
+        self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
+        self.e("add.u64 %s, %s, %s;" % (adr, adr, off))
+        self.async_copy(sadr, adr, pr)
+
+    def leaf_ldsw(self, dst, copy_to=None, then_copy=False):
         ptr, sadr = self.staged_operand()
         self.fetch()
         slow = self.newlabel("ldsw")
@@ -522,12 +531,15 @@ class Kernel:
         self.lds_v(sadr, dst)
         if copy_to:
             self.mov_v(copy_to, dst)
+        if then_copy:      # the slot has been read (the loads above are ahead of the copy in this thread's order)
+            self.next_copy(ptr, sadr)
         self.jump()
         self.label(slow)       # a ragged tile is never staged: load it and leave it in the slot for later reads
         adr = self.rd()
         self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
         self.load_f32_slow(adr, dst)
-        self.sts_v(sadr, dst)
+        if not then_copy:      # (read once: nothing to keep; a ragged tile is followed by ragged tiles only, never staged)
+            self.sts_v(sadr, dst)
         if copy_to:
             self.mov_v(copy_to, dst)
         self.jump()
@@ -744,6 +756,9 @@ class Kernel:
         elif op == "ldswr":
             self.leaf_ldsw(R, A)
             return
+        elif op == "ldswar":
+            self.leaf_ldsw(R, A, True)
+            return
         elif op in ("sincosr", "cossinr"):
             self.fetch()
             S, C = self.sincos(A)
@@ -921,6 +936,8 @@ class Kernel:
             self.leaf_glda(False); return
         elif op == "ldsw":
             self.leaf_ldsw(A); return
+        elif op == "ldswa":
+            self.leaf_ldsw(A, None, True); return
         elif op == "gstf":
             self.leaf_gstf(); return
         elif op == "fill":

@@ -7,11 +7,11 @@ import numpy as np
 
 STRIDE = 8   # case id of a register-operand instruction = index * STRIDE + register slot
 J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
-     "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr"]
+     "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar"]
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
-     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "end"]
+     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "end"]
 
 
 def _bf16(a):
@@ -63,7 +63,7 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
             elif name == "spillr": G[arg] = R[k].copy()
             elif name == "fillr": R[k] = G[arg].copy()
             elif name == "gldr": acc = load(arg); R[k] = acc.copy()
-            elif name == "ldswr": acc = load(arg & 63); R[k] = acc.copy(); S[arg >> 6] = acc.copy()
+            elif name in ("ldswr", "ldswar"): acc = load(arg & 63); R[k] = acc.copy(); S[arg >> 6] = acc.copy()
             elif name == "sincosr": R[k] = np.cos(acc); acc = np.sin(acc)
             elif name == "cossinr": R[k] = np.sin(acc); acc = np.cos(acc)
             elif name.startswith("macc"): A[int(name[4])] += float((acc * R[k]).sum())
@@ -109,7 +109,7 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
         elif name == "colout": colout[arg] = acc.sum(axis=0)
         elif name == "scalout": scalout[arg] = acc.sum()
         elif name in ("glda0", "glda"): pass      # the copy itself is modelled at the read
-        elif name == "ldsw": acc = load(arg & 63); S[arg >> 6] = acc.copy()
+        elif name in ("ldsw", "ldswa"): acc = load(arg & 63); S[arg >> 6] = acc.copy()
         elif name.startswith("sacc"): A[int(name[4])] += float(acc.sum())
         elif name.startswith("ascal"): scalout[arg] = A[int(name[5])]
         elif name == "end": break
