@@ -3,7 +3,7 @@
 //
 //   sin/cos : three-constant Cody-Waite reduction by pi/2 (fused multiply-adds), odd/even
 //             polynomials on [-pi/4, pi/4]
-//   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), scaled by 2^n
+//   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), n added to the exponent
 //   tanh    : x + x^3*T(x^2) below 0.6, 1 - 2/(exp(2|x|)+1) above
 //   sigmoid : 1/(1+exp(-x))
 // Polynomial coefficients are weighted least-squares fits on Chebyshev nodes, iteratively
@@ -108,7 +108,8 @@ VM_HD float cos_f(float x) {
   return ((q + 1) & 2) ? -v : v;
 }
 
-// exp for -100 <= x <= 88.7 (callers clamp)
+// exp for -86 <= x <= 88.7 (callers clamp), where the result is a normal number: e^x = p * 2^n with
+// the 2^n applied by adding n to the exponent field of p, which is exact, as the multiplication is
 VM_HD float exp_core(float x) {
   const float nb = fmaf(x, 1.44269504088896341f, 12582912.0f);   // round(x*log2 e) in the low mantissa bits
   const float n = nb - 12582912.0f;
@@ -119,14 +120,10 @@ VM_HD float exp_core(float x) {
   e = fmaf(r, e, 1.6666520673866728e-1f);
   e = fmaf(r, e, 4.9999993454926206e-1f);
   const float p = fmaf(r * r, e, r) + 1.0f;
-  // 2^n in two factors so that n = 128 and n below -126 stay in range
-  const int ni = (int)(f_bits(nb) << 10) >> 10;                   // sign-extended low 22 bits
-  const int h = ni >> 1;
-  const float s1 = f_from_bits((uint32_t)(h + 127) << 23), s2 = f_from_bits((uint32_t)(ni - h + 127) << 23);
-  return p * s1 * s2;
+  return f_from_bits(f_bits(p) + (f_bits(nb) << 23));
 }
 VM_HD float exp_clamped10(float x) { return exp_core(fminf(fmaxf(x, -10.0f), 10.0f)); }
-VM_HD float exp_wide(float x) { return exp_core(fminf(fmaxf(x, -100.0f), 88.7f)); }
+VM_HD float exp_wide(float x) { return exp_core(fminf(fmaxf(x, -86.0f), 88.7f)); }
 
 VM_HD float sigmoid_f(float x) { return f_rcp(1.0f + exp_wide(-x)); }
 

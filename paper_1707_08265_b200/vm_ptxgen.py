@@ -6,8 +6,9 @@ dispatch between them.  Both are written out here instruction by instruction ins
 them to a C++ compiler:
 
 * dispatch is one 64-bit shared-memory load of the pre-decoded {case, argument} pair, a pointer
-  increment and one uniform indexed branch (``brx.idx.uni``) over a table of leaf labels; the
-  fetch of the next pair is issued at the top of a leaf, ahead of its arithmetic;
+  increment and a jump to the one dispatch block, which holds the kernel's only indexed branch
+  (``brx.idx.uni`` over a table of leaf labels); the fetch of the next pair is issued at the top of
+  a leaf, ahead of its arithmetic;
 * every V-wide value lives in named registers as packed pairs (``.b64`` = two fp32), so additions,
   multiplications and fused multiply-adds are ``f32x2`` instructions: half the issue slots of
   scalar code for the same rounding (each lane is an IEEE fp32 operation);
