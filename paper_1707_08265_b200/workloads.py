@@ -184,3 +184,20 @@ def random_row_dag(rows, cols, seed, n_full=6, n_row=2, n_ops=1024, n_fetch=4):
     pick = rng.choice(len(sinks), size=min(n_fetch, len(sinks)), replace=False)
     fetch = [sinks[int(p)] for p in sorted(pick)]
     return g, inputs, fetch
+
+
+def updater(shape, kind="sgd"):
+    """The weight update as a graph of its own (Sec. 3.2 of the paper: the updater is split from the
+    training graph so that neither becomes cyclic).  sgd: W' = W - lr*g.  momentum: v' = mu*v + g,
+    W' = W - lr*v'.  lr and mu are scalar tensors; returns (graph, ids)."""
+    g = GraphDesc()
+    ids = {"W": g.tensor("W", shape), "g": g.tensor("g", shape), "lr": g.tensor("lr", [])}
+    if kind == "sgd":
+        step = g.op("Mul", [ids["lr"], ids["g"]], "step")
+    else:
+        ids["v"] = g.tensor("v", shape)
+        ids["mu"] = g.tensor("mu", [])
+        ids["v_new"] = g.op("Add", [g.op("Mul", [ids["mu"], ids["v"]], "mv"), ids["g"]], "v_new")
+        step = g.op("Mul", [ids["lr"], ids["v_new"]], "step")
+    ids["W_new"] = g.op("Sub", [ids["W"], step], "W_new")
+    return g, ids

@@ -1,0 +1,67 @@
+"""GPU checks that go beyond the benchmark graphs: the VM's elementary functions over dense sweeps
+of arguments (every binade, both signs, the switch points of the implementations), and the weight
+update run as a graph of its own (Sec. 3.2 of the paper), each against the fp64 oracle."""
+import numpy as np
+import pytest
+
+from oracle import interp
+from paper_1707_08265_b200 import workloads as wl
+from test_gpu_vm import run_gpu, check, TOL32
+
+pytestmark = pytest.mark.gpu
+
+
+def sweep(lo_exp, hi_exp, per_binade=64):
+    m = np.linspace(1.0, 2.0, per_binade, endpoint=False, dtype=np.float64)
+    mag = np.concatenate([m * 2.0 ** e for e in range(lo_exp, hi_exp)])
+    return np.concatenate([mag, -mag, [0.0, -0.0]]).astype(np.float32)
+
+
+@pytest.mark.parametrize("op,lo,hi,extra", [
+    ("Sin", -20, 22, [np.pi / 4, np.pi / 2, np.pi, 1e5 * np.pi, 6.4e6]),     # up to the documented 6.5e6
+    ("Exp", -20, 8, [10.0, -10.0, 9.9999, -9.9999, 10.0001, 88.0, -88.0]),   # clamp at +-10
+    ("Tanh", -20, 8, [0.6, 0.5999999, 0.6000001, 9.0, 20.0, 21.0, 90.0]),    # polynomial below 0.6
+    ("Sigmoid", -20, 8, [86.0, -86.0, 88.7, -88.7, 100.0, -100.0]),
+    ("Div", -20, 20, [1.0, -1.0]),
+])
+def test_elementary_functions_over_dense_sweeps(op, lo, hi, extra):
+    x = np.concatenate([sweep(lo, hi), np.asarray(extra, np.float32), -np.asarray(extra, np.float32)]).astype(np.float32)
+    n = x.size
+    gd = wl.GraphDesc()
+    xi = gd.tensor("x", [n])
+    ins = [xi]
+    feeds = [x]
+    if op == "Div":   # a / (1 + |b|): sweep b, a fixed to ones
+        one = gd.tensor("one", [n])
+        out = gd.op("Div", [one, xi], "out")
+        ins = [one, xi]
+        feeds = [np.ones(n, np.float32), x]
+    else:
+        out = gd.op(op, [xi], "out")
+    grads = gd.grad([out], [xi])     # Sin -> cos, Exp -> exp*mask, Tanh -> 1-y^2, Sigmoid -> y(1-y), Div -> d/db
+    got, _ = run_gpu(gd.desc, ins, [out] + grads, feeds)
+    ref = interp.run_function(gd.desc, ins, [out] + grads, feeds)
+    for gv, rv, what in zip(got, ref, ("value", "gradient")):
+        check(gv, rv, TOL32, "%s %s" % (op, what))
+
+
+@pytest.mark.parametrize("kind", ["sgd", "momentum"])
+@pytest.mark.parametrize("shape", [[5 * 4096 + 3], [300, 1000]])
+def test_updater_graph(kind, shape):
+    g, ids = wl.updater(shape, kind)
+    rng = np.random.default_rng(11)
+    W = rng.standard_normal(shape).astype(np.float32)
+    grad = (rng.standard_normal(shape) * 0.1).astype(np.float32)
+    lr, mu = np.float32(0.05), np.float32(0.9)
+    if kind == "sgd":
+        inputs, feeds, outs = [ids["W"], ids["g"], ids["lr"]], [W, grad, lr], [ids["W_new"]]
+    else:
+        v = (rng.standard_normal(shape) * 0.1).astype(np.float32)
+        inputs, feeds, outs = [ids["W"], ids["g"], ids["lr"], ids["v"], ids["mu"]], [W, grad, lr, v, mu], [ids["W_new"], ids["v_new"]]
+    got, f = run_gpu(g.desc, inputs, outs, feeds)
+    assert f.num_launches() == 1, f.describe()     # one fused VM launch for the whole update
+    ref = interp.run_function(g.desc, inputs, outs, feeds)
+    for gv, rv in zip(got, ref):
+        check(gv, rv, TOL32, kind)
+    if kind == "sgd":                              # and against the formula written out
+        assert np.allclose(got[0], W.astype(np.float64) - float(lr) * grad.astype(np.float64), rtol=0, atol=2e-6)
