@@ -40,6 +40,12 @@ OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIF
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
          "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar"]
+# Leaves that end in their own indexed branch instead of a jump to the shared dispatch block: one
+# taken branch less per dispatch.  Measured, not derived: every further site makes the assembler add
+# branch-table code and changes its register allocation, and larger sets ran slower on all three
+# large workloads (16 more short leaves: +3 % on the sin/cos graph, +3 % on the random DAG), so the
+# list holds the short arithmetic, store and staged-load leaves it was first tried with.
+HOT = {"fmau", "mul", "sacc0", "macc1", "fmaur", "gstf", "cossinr", "ldswar"}
 JOINT_STRIDE = 8    # case id of a joint instruction = index * JOINT_STRIDE + register slot
 N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
@@ -176,6 +182,9 @@ class Kernel:
         # every leaf leaves through the one dispatch block: the assembler gives each indexed branch
         # its own table of branch instructions (about 2 KB per site), which with one site per leaf
         # made the code image four times larger and scattered the hot leaves
+        if getattr(self, "own_brx", False):
+            self.e("brx.idx.uni %%case, JT_%s;" % self.name)
+            return
         self.e("bra.uni $DISPATCH_%s;" % self.name)
 
     # addresses that depend on the argument (taken before the fetch overwrites %arg)
@@ -1234,10 +1243,12 @@ class Kernel:
             if kind == "bad":
                 continue
             self.label(lab)
+            self.own_brx = op in HOT
             if kind == "j":
                 self.leaf_joint(op, k)
             else:
                 self.leaf_plain(op)
+            self.own_brx = False
         # a register slot this build does not have: report and stop (the host never emits one)
         self.label(bad)
         skip = self.newlabel("bad")
