@@ -174,7 +174,7 @@ int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* c
 int dragon_function_profile(dragon_function_t* f, int step, int capacity);
 int dragon_function_profile_read(dragon_function_t* f, double* total_ms, int* runs);
 
-/* Synchronises the stream of the last run and returns the device status word: DRAGON_OK,
+/* Synchronises the stream of the last run and returns the device status word of that run: DRAGON_OK,
  * DRAGON_ERR_TIMEOUT (a bounded wait gave up) or DRAGON_ERR_INVALID_ARG (bad label). */
 int dragon_function_status(dragon_function_t* f);
 

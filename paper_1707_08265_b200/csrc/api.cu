@@ -280,6 +280,7 @@ int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t by
   }
   f->workspace = dev_ptr;
   f->workspace_bytes = bytes;
+  f->status_ready = false;
   return DRAGON_OK;
 }
 
@@ -311,8 +312,17 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
     }
     f->uploaded = true;
   }
-  int* status = reinterpret_cast<int*>(ws + P.status_off);
-  cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
+  // this run's status word, and the other one, which it clears for the next run
+  int* const word0 = reinterpret_cast<int*>(ws + P.status_off);
+  cudaError_t e = cudaSuccess;
+  if (!f->status_ready) {
+    e = cudaMemsetAsync(word0, 0, 256, st);
+    f->status_ready = true;
+    f->run_parity = 0;
+  }
+  int* const status = word0 + 16 * f->run_parity;
+  int* const status_next = word0 + 16 * (f->run_parity ^ 1);
+  bool next_cleared = false;
   for (size_t si = 0; si < P.steps.size(); ++si) {
     const Step& s = P.steps[si];
     if (e != cudaSuccess) break;
@@ -337,6 +347,8 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         p.colpart = reinterpret_cast<float*>(ws + sg.colpart_off);
         p.scalpart = reinterpret_cast<double*>(ws + sg.scalpart_off);
         p.status = status;
+        p.status_clear = next_cleared ? nullptr : status_next;
+        next_cleared = true;
         for (size_t i = 0; i < sg.operand_mem.size(); ++i) {
           p.operand[i].ptr = ptr[sg.operand_mem[i]];
           p.operand[i].kind = sg.operand_kind[i];
@@ -352,7 +364,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         const MemRef &A = P.mems[s.mA], &C = P.mems[s.mC];
         const int kc = (int)(s.tA ? A.shape.d[0] : A.shape.d[1]);
         int rc = launch_gemm_bf16(ptr[s.mA], ptr[s.mB], ptr[s.mC], C.dtype, (int)C.shape.d[0], (int)C.shape.d[1], kc, s.tA, s.tB, status, st);
-        if (rc != DRAGON_OK) return rc;
+        if (rc != DRAGON_OK) { f->status_ready = false; return rc; }
         break;
       }
       case ST_TRANSPOSE:
@@ -377,9 +389,16 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
     }
   }
   if (e != cudaSuccess) {
+    f->status_ready = false;   // both status words are cleared again before the next run
     set_error("dragon_run: CUDA error: %s", cudaGetErrorString(e));
     return DRAGON_ERR_CUDA;
   }
+  if (!next_cleared && cudaMemsetAsync(status_next, 0, sizeof(int), st) != cudaSuccess) {
+    set_error("dragon_run: CUDA error: %s", cudaGetErrorString(cudaGetLastError()));
+    return DRAGON_ERR_CUDA;
+  }
+  f->last_status_word = f->run_parity;
+  f->run_parity ^= 1;
   f->last_stream = cuda_stream;
   return DRAGON_OK;
 }
@@ -474,7 +493,7 @@ int dragon_function_status(dragon_function_t* f) {
   int v = 0;
   cudaStream_t st = reinterpret_cast<cudaStream_t>(f->last_stream);
   if (cudaStreamSynchronize(st) != cudaSuccess ||
-      cudaMemcpy(&v, reinterpret_cast<char*>(f->workspace) + f->plan.status_off, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
+      cudaMemcpy(&v, reinterpret_cast<char*>(f->workspace) + f->plan.status_off + 64 * f->last_status_word, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess) {
     set_error("dragon_function_status: CUDA error: %s", cudaGetErrorString(cudaGetLastError()));
     return DRAGON_ERR_CUDA;
   }

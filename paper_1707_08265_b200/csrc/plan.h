@@ -127,6 +127,10 @@ struct dragon_function {
   size_t workspace_bytes = 0;
   void* last_stream = nullptr;
   bool uploaded = false;
+  // two status words used by alternate runs: a run reports into one and clears the other for the
+  // run after it, so that no run needs a memset of its own
+  bool status_ready = false;
+  int run_parity = 0, last_status_word = 0;
   // profiling ring (dragon_function_profile)
   int prof_step = -1, prof_used = 0;
   std::vector<void*> prof_ev;   // 2 * capacity cudaEvent_t

@@ -122,9 +122,11 @@ struct Params {             // kernel parameter block; the PTX generator (vm_ptx
   uint32_t loop_start;      // 68  index of the first instruction of the per-tile body
   uint32_t grid;            // 72  CTAs launched
   uint32_t n_full_tiles;    // 76  tiles [0, n_full_tiles) hold all kVmTile elements (row mode: rows of exactly kVmTile)
-  Operand operand[kMaxOperands];   // 80
+  int* status_clear;        // 80  word that CTA 0 sets to 0 (the status word of the next run), or null
+  unsigned long long reserved2;   // 88
+  Operand operand[kMaxOperands];   // 96
 };
-static_assert(sizeof(Operand) == 16 && sizeof(Params) == 80 + 16 * kMaxOperands, "layout shared with the PTX generator");
+static_assert(sizeof(Operand) == 16 && sizeof(Params) == 96 + 16 * kMaxOperands, "layout shared with the PTX generator");
 
 
 }  // namespace vm

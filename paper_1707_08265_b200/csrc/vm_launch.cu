@@ -30,6 +30,9 @@ struct FinishParams {
 };
 
 __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
+  // launched as a programmatic dependent of the VM kernel: its blocks may be resident before that
+  // kernel ends, and wait here until its partial sums are complete and visible
+  cudaGridDependencySynchronize();
   const FinishParams::Job& jb = fp.job[blockIdx.y];
   if (jb.kind == 0) {
     const int c = blockIdx.x * blockDim.x + threadIdx.x;
@@ -112,8 +115,16 @@ cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, 
     else o.part = ws + sg.scalpart_off + (size_t)j.acc * sg.grid * sizeof(double);
   }
   dim3 grid((max_cols + 127) / 128, fp.n_jobs);
-  vm::finish_kernel<<<grid, 128, 0, st>>>(fp);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = dim3(128);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, vm::finish_kernel, fp);
 }
 
 }  // namespace dragon

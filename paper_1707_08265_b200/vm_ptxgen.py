@@ -33,7 +33,7 @@ MAX_UNIFORMS = 512
 
 # Params (csrc/vm_isa.h): byte offsets
 P_CODE, P_SPILL, P_COLPART, P_SCALPART, P_STATUS, P_N = 0, 8, 16, 24, 32, 40
-P_NCODE, P_ROWMODE, P_COLS, P_NSPILL, P_NTILES, P_LOOPSTART, P_GRID, P_NFULL, P_OPERAND = 48, 52, 56, 60, 64, 68, 72, 76, 80
+P_NCODE, P_ROWMODE, P_COLS, P_NSPILL, P_NTILES, P_LOOPSTART, P_GRID, P_NFULL, P_STATUSCLEAR, P_OPERAND = 48, 52, 56, 60, 64, 68, 72, 76, 80, 96
 P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
 # shared memory behind the decoded instruction stream: uniforms | reduction scratch | operand table | slots
 OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
@@ -1231,6 +1231,17 @@ class Kernel:
             e("mov.b64 %s, 0;" % r_)
         for r_ in self.S:
             e("mov.f32 %s, 0f00000000;" % r_)
+        # CTA 0 clears the status word of the next run (the host alternates between two words)
+        skip_c = self.newlabel("sc")
+        pc, pz, sc_ptr, zero = self.p(), self.p(), self.param(P_STATUSCLEAR, "u64"), self.r()
+        e("or.b32 %s, %s, %s;" % (zero, cta, tx))
+        e("setp.ne.u32 %s, %s, 0;" % (pc, zero))
+        e("setp.eq.u64 %s, %s, 0;" % (pz, sc_ptr))
+        e("or.pred %s, %s, %s;" % (pc, pc, pz))
+        e("@%s bra %s;" % (pc, skip_c))
+        e("mov.u32 %s, 0;" % zero)
+        e("st.global.u32 [%s], %s;" % (sc_ptr, zero))
+        self.label(skip_c)
         e("mov.u32 %%tile, %s;" % cta)
         self.set_tile()
         e("mov.u32 %ip, dsm;")

@@ -15,7 +15,7 @@ import vm_ptxgen as gen  # noqa: E402
 
 FIELDS = {"code": "P_CODE", "spill": "P_SPILL", "colpart": "P_COLPART", "scalpart": "P_SCALPART", "status": "P_STATUS",
           "n": "P_N", "n_code": "P_NCODE", "row_mode": "P_ROWMODE", "cols": "P_COLS", "n_spill": "P_NSPILL",
-          "n_tiles": "P_NTILES", "loop_start": "P_LOOPSTART", "grid": "P_GRID", "n_full_tiles": "P_NFULL", "tile_stride_bytes": "P_STRIDE",
+          "n_tiles": "P_NTILES", "loop_start": "P_LOOPSTART", "grid": "P_GRID", "n_full_tiles": "P_NFULL", "status_clear": "P_STATUSCLEAR", "tile_stride_bytes": "P_STRIDE",
           "full_end_bytes": "P_FULLEND", "next_end_bytes": "P_NEXTEND", "all_end_bytes": "P_ALLEND", "operand": "P_OPERAND"}
 
 
