@@ -592,6 +592,12 @@ class Kernel:
         self.e("@%s bra.uni %s;" % (pbf, lbf))
         adr = self.rd()
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        slow = self.newlabel("gld")
+        self.e("@!%%pfull bra.uni %s;" % slow)     # a full tile: whole, aligned vectors (ROW operands too)
+        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s];" % (A[0], A[1], adr))
+        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (A[2], A[3], adr, HALF_BYTES))
+        self.jump()
+        self.label(slow)
         self.prefetch(adr, 4, pfullk)
         self.load_f32_slow(adr, A)
         self.jump()
@@ -600,6 +606,18 @@ class Kernel:
         adr = self.rd()
         self.e("shr.u64 %s, %s, 1;" % (off, off))
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        slowb = self.newlabel("gld")
+        self.e("@!%%pfull bra.uni %s;" % slowb)
+        for h in range(2):
+            w0, w1 = self.r(), self.r()
+            self.e("ld.global.nc.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, adr, h * NT * 8))
+            for i, w in enumerate((w0, w1)):
+                lo, hi = self.r(), self.r()
+                self.e("shl.b32 %s, %s, 16;" % (lo, w))
+                self.e("and.b32 %s, %s, 0xffff0000;" % (hi, w))
+                self.pack(lo, hi, A[2 * h + i])
+        self.jump()
+        self.label(slowb)
         self.prefetch(adr, 2, pfullk)
         pvec = self.pvec()
         for h in range(2):
@@ -688,6 +706,11 @@ class Kernel:
         self.e("@%s bra.uni %s;" % (pbf, lbf))
         adr = self.rd()
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        slow = self.newlabel("gst")
+        self.e("@!%%pfull bra.uni %s;" % slow)
+        self.stg_v(adr, A)
+        self.jump()
+        self.label(slow)
         self.store_f32_slow(adr)
         self.jump()
         # bf16 tensors
@@ -695,6 +718,16 @@ class Kernel:
         adr = self.rd()
         self.e("shr.u64 %s, %s, 1;" % (off, off))
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        slowb = self.newlabel("gst")
+        self.e("@!%%pfull bra.uni %s;" % slowb)
+        for h in range(2):
+            sc = self.unpack(A[2 * h]) + self.unpack(A[2 * h + 1])
+            w0, w1 = self.r(), self.r()
+            self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w0, sc[1], sc[0]))
+            self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w1, sc[3], sc[2]))
+            self.e("st.global.v2.u32 [%s+%d], {%s, %s};" % (adr, h * NT * 8, w0, w1))
+        self.jump()
+        self.label(slowb)
         pvec = self.pvec()
         for h in range(2):
             lv, ln = self.newlabel("gst"), self.newlabel("gst")
