@@ -127,6 +127,62 @@ __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdt
   }
 }
 
+// The same for rows that fit the CTA's registers (cols <= kChunks * 2048, a multiple of 8): the row
+// is read from memory once, the exponentials are computed once and kept.  Every thread owns the
+// same elements and adds them in the same order as in sce_kernel, so the results are identical.
+template <int kMode, int kChunks>
+__global__ void __launch_bounds__(kRowThreads) sce_row_kernel(const void* z, int zdtype, const int* labels, int rows, int cols,
+                                                              float* rowloss, void* dz, int dzdtype, const float* dl_ptr,
+                                                              float dl_imm, int* status) {
+  __shared__ float sh[kRowThreads / 32];
+  const int m = blockIdx.x;
+  const size_t off = (size_t)m * cols;
+  float v[kChunks][8];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    const int j = (c * kRowThreads + threadIdx.x) * 8;
+    if (j < cols) {
+      load8(z, zdtype, off + j, v[c]);
+#pragma unroll
+      for (int e = 0; e < 8; ++e) mx = fmaxf(mx, v[c][e]);
+    }
+  }
+  mx = block_reduce<true>(mx, sh);
+  float se = 0.f;
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c) {
+    const int j = (c * kRowThreads + threadIdx.x) * 8;
+    if (j < cols) {
+#pragma unroll
+      for (int e = 0; e < 8; ++e) { v[c][e] = vmmath::exp_wide(v[c][e] - mx); se += v[c][e]; }
+    }
+  }
+  se = block_reduce<false>(se, sh);
+  const int lab = __ldg(labels + m);
+  const bool ok = lab >= 0 && lab < cols;
+  if (!ok && threadIdx.x == 0) atomicExch(status, DRAGON_ERR_INVALID_ARG);
+  if (kMode == 0) {
+    if (threadIdx.x == 0) rowloss[m] = ok ? (logf(se) + mx - load_logit(z, zdtype, off + lab)) : 0.f;
+  } else {
+    const float dl = dl_ptr ? __ldg(dl_ptr) : dl_imm;
+    const float sc = dl / (float)rows, inv = 1.f / se;
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      const int j = (c * kRowThreads + threadIdx.x) * 8;
+      if (j < cols) {
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          float g = v[c][e] * inv;
+          if (j + e == lab) g -= 1.f;
+          v[c][e] = ok ? g * sc : 0.f;
+        }
+        store8(dz, dzdtype, off + j, v[c]);
+      }
+    }
+  }
+}
+
 __global__ void __launch_bounds__(kRowThreads) mean_kernel(const float* v, int n, float* out) {
   __shared__ double sh[kRowThreads];
   double s = 0.0;
@@ -161,14 +217,20 @@ __global__ void __launch_bounds__(256) transpose16_kernel(const unsigned short* 
 
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
                            int* status, cudaStream_t st) {
-  sce_kernel<0><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
+  if ((cols & 7) == 0 && cols <= 2 * kRowThreads * 8)
+    sce_row_kernel<0, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
+  else
+    sce_kernel<0><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
   mean_kernel<<<1, kRowThreads, 0, st>>>(rowloss, rows, out);
   return cudaGetLastError();
 }
 
 cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
                            const float* dl_ptr, float dl_imm, int* status, cudaStream_t st) {
-  sce_kernel<1><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status);
+  if ((cols & 7) == 0 && cols <= 2 * kRowThreads * 8)
+    sce_row_kernel<1, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status);
+  else
+    sce_kernel<1><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status);
   return cudaGetLastError();
 }
 
