@@ -11,7 +11,7 @@ namespace dragon {
 cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st);
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st);
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
-                           int* status, cudaStream_t st);
+                           int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm);
 cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
                            const float* dl_ptr, float dl_imm, int* status, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cudaStream_t st);
@@ -372,7 +372,8 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         break;
       case ST_SCE_FWD:
         e = launch_sce_fwd(ptr[s.mA], P.mems[s.mA].dtype, reinterpret_cast<const int*>(ptr[s.mB]), (int)P.mems[s.mA].shape.d[0],
-                           (int)P.mems[s.mA].shape.d[1], reinterpret_cast<float*>(ws + s.scratch_off), reinterpret_cast<float*>(ptr[s.mC]), status, st);
+                           (int)P.mems[s.mA].shape.d[1], reinterpret_cast<float*>(ws + s.scratch_off), reinterpret_cast<float*>(ptr[s.mC]), status, st,
+                           s.mD >= 0 ? ptr[s.mD] : nullptr, s.mD >= 0 ? P.mems[s.mD].dtype : 0, s.scale);
         break;
       case ST_SCE_BWD:
         e = launch_sce_bwd(ptr[s.mA], P.mems[s.mA].dtype, reinterpret_cast<const int*>(ptr[s.mB]), (int)P.mems[s.mA].shape.d[0],

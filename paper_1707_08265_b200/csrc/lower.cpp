@@ -459,9 +459,10 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
   // steps in execution order
   std::vector<int> seg_step(seg_items.size(), -1);
   plan->segs.resize(seg_items.size());
+  std::vector<bool> fused_away(items.size(), false);
   for (int i = 0; i < (int)items.size(); ++i) {
     const Item& it = items[i];
-    if (!it.live) continue;
+    if (!it.live || fused_away[i]) continue;
     if (it.kind == IT_MOP) {
       if (it.segment >= 0 && seg_step[it.segment] < 0) {
         seg_step[it.segment] = (int)plan->steps.size();
@@ -474,6 +475,20 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     st.kind = it.kind == IT_GEMM ? ST_GEMM : it.kind == IT_TRANSPOSE ? ST_TRANSPOSE : it.kind == IT_SCE_FWD ? ST_SCE_FWD
               : it.kind == IT_SCE_BWD ? ST_SCE_BWD : ST_COPY;
     st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
+    if (it.kind == IT_SCE_FWD) {
+      // the gradient with respect to the same logits, scaled by a constant, comes out of the same
+      // pass: the step then carries the gradient tensor in mD
+      st.mD = -1;
+      for (int j = i + 1; j < (int)items.size(); ++j) {
+        const Item& b = items[j];
+        if (b.live && b.kind == IT_SCE_BWD && b.mA == it.mA && b.mB == it.mB && b.mD < 0) {
+          st.mD = b.mC;
+          st.scale = b.scale;
+          fused_away[j] = true;
+          break;
+        }
+      }
+    }
     plan->steps.push_back(st);
   }
   for (size_t s = 0; s < seg_items.size(); ++s) {
@@ -550,7 +565,7 @@ std::string describe_plan(const Plan& p) {
       case ST_TRANSPOSE:
         snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);
         break;
-      case ST_SCE_FWD: snprintf(buf, sizeof(buf), "softmax_ce_fwd\n"); break;
+      case ST_SCE_FWD: snprintf(buf, sizeof(buf), st.mD >= 0 ? "softmax_ce_fwd+bwd\n" : "softmax_ce_fwd\n"); break;
       case ST_SCE_BWD: snprintf(buf, sizeof(buf), "softmax_ce_bwd\n"); break;
       default: snprintf(buf, sizeof(buf), "copy\n");
     }

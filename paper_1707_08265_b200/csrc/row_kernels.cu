@@ -61,7 +61,8 @@ __device__ __forceinline__ void store8(void* z, int dtype, size_t i, const float
   }
 }
 
-// mode 0: rowloss[m] = logsumexp(z[m,:]) - z[m,label];  mode 1: dz[m,j] = dL/M * (softmax - onehot).
+// mode 0: rowloss[m] = logsumexp(z[m,:]) - z[m,label];  mode 1: dz[m,j] = dL/M * (softmax - onehot);
+// mode 2: both in one pass over the logits.
 // Rows whose length is a multiple of 8 are read and written 8 elements (16 or 32 bytes) per thread.
 template <int kMode>
 __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdtype, const int* labels, int rows, int cols,
@@ -98,9 +99,10 @@ __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdt
   const int lab = __ldg(labels + m);
   const bool ok = lab >= 0 && lab < cols;
   if (!ok && threadIdx.x == 0) atomicExch(status, DRAGON_ERR_INVALID_ARG);
-  if (kMode == 0) {
+  if (kMode != 1) {
     if (threadIdx.x == 0) rowloss[m] = ok ? (logf(se) + mx - load_logit(z, zdtype, off + lab)) : 0.f;
-  } else {
+  }
+  if (kMode != 0) {
     const float dl = dl_ptr ? __ldg(dl_ptr) : dl_imm;
     const float sc = dl / (float)rows, inv = 1.f / se;
     if (vec) {
@@ -162,9 +164,10 @@ __global__ void __launch_bounds__(kRowThreads) sce_row_kernel(const void* z, int
   const int lab = __ldg(labels + m);
   const bool ok = lab >= 0 && lab < cols;
   if (!ok && threadIdx.x == 0) atomicExch(status, DRAGON_ERR_INVALID_ARG);
-  if (kMode == 0) {
+  if (kMode != 1) {
     if (threadIdx.x == 0) rowloss[m] = ok ? (logf(se) + mx - load_logit(z, zdtype, off + lab)) : 0.f;
-  } else {
+  }
+  if (kMode != 0) {
     const float dl = dl_ptr ? __ldg(dl_ptr) : dl_imm;
     const float sc = dl / (float)rows, inv = 1.f / se;
 #pragma unroll
@@ -216,8 +219,12 @@ __global__ void __launch_bounds__(256) transpose16_kernel(const unsigned short* 
 }  // namespace
 
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
-                           int* status, cudaStream_t st) {
-  if ((cols & 7) == 0 && cols <= 2 * kRowThreads * 8)
+                           int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm) {
+  const bool in_regs = (cols & 7) == 0 && cols <= 2 * kRowThreads * 8;
+  if (dz) {   // the gradient with respect to the logits in the same pass (dL is a constant)
+    if (in_regs) sce_row_kernel<2, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, dz, dzdtype, nullptr, dl_imm, status);
+    else sce_kernel<2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, dz, dzdtype, nullptr, dl_imm, status);
+  } else if (in_regs)
     sce_row_kernel<0, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
   else
     sce_kernel<0><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
@@ -288,7 +295,7 @@ extern "C" int dragon_softmax_ce_loss_static(const void* logits, int dtype, cons
   int* status = reinterpret_cast<int*>(scratch + kStaticMaxRows);
   // the status word must start at zero; the per-row losses are overwritten in full by every call
   cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
-  if (e == cudaSuccess) e = launch_sce_fwd(logits, dtype, labels, rows, cols, scratch, loss_out, status, st);
+  if (e == cudaSuccess) e = launch_sce_fwd(logits, dtype, labels, rows, cols, scratch, loss_out, status, st, nullptr, 0, 0.f);
   if (e != cudaSuccess) {
     set_error("dragon_softmax_ce_loss_static: CUDA error: %s", cudaGetErrorString(e));
     return DRAGON_ERR_CUDA;
