@@ -383,7 +383,6 @@ struct Gen {
       }
       last_read[opd] = i;
     }
-    if (slot_of.empty()) return;
     std::vector<uint32_t> out;
     std::map<int, bool> seen;
     for (size_t i = 0; i < body.size(); ++i) {
@@ -406,6 +405,19 @@ struct Gen {
     }
     body.swap(out);
     for (auto& so : slot_of) preamble.push_back(encode(P_GLDA0, 0, (uint32_t)so.first | ((uint32_t)so.second << 6)));
+    // bf16 operands of the full domain shape that the body reads exactly once
+    std::map<int, int> reads;
+    for (uint32_t w : body)
+      if ((w & 1023u) == (uint32_t)P_GLD) ++reads[(int)(w >> 14)];
+    for (uint32_t& w : body) {
+      const int opd = (int)(w >> 14);
+      if ((w & 1023u) != (uint32_t)P_GLD || opd >= 64 || reads[opd] != 1) continue;
+      if (seg->operand_kind[opd] != (uint32_t)K_FULL || mems[seg->operand_mem[opd]].dtype != DRAGON_BF16) continue;
+      if (seg->n_smem >= n_smem_max) break;
+      const uint32_t arg = (uint32_t)opd | ((uint32_t)seg->n_smem++ << 6);
+      w = encode(P_LDSWAH, 0, arg);
+      preamble.push_back(encode(P_GLDA0H, 0, arg));
+    }
   }
 
   int run() {

@@ -51,7 +51,7 @@ N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "glda0h", "ldswah", "end"]
 
 
 def f32bits(x):
@@ -532,6 +532,52 @@ class Kernel:
         self.e("add.u64 %s, %s, %s;" % (adr, adr, off))
         self.async_copy(sadr, adr, pr)
 
+    # bf16 operands, read once per iteration: 8 bytes per thread and half, converted at the read
+    def async_copy_h(self, sadr, gadr, pred):
+        for h in range(2):
+            self.e("@%s cp.async.ca.shared.global [%s+%d], [%s+%d], 8;" % (pred, sadr, h * HALF_BYTES, gadr, h * NT * 8))
+        self.e("cp.async.commit_group;")
+
+    def tile_adr_h(self, ptr):
+        adr, off = self.rd(), self.rd()
+        self.e("shr.u64 %s, %%tb4, 1;" % off)
+        self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
+        return adr
+
+    def leaf_glda0h(self):
+        ptr, sadr = self.staged_operand()
+        self.fetch()
+        pr = self.p()
+        self.e("mov.pred %s, %%pfull;" % pr)
+        self.async_copy_h(sadr, self.tile_adr_h(ptr), pr)
+        self.jump()
+
+    def leaf_ldswah(self):
+        A = self.A
+        ptr, sadr = self.staged_operand()
+        self.fetch()
+        adr = self.tile_adr_h(ptr)
+        slow = self.newlabel("ldswh")
+        self.e("@!%%pfull bra.uni %s;" % slow)
+        self.e("cp.async.wait_all;")
+        for h in range(2):
+            w0, w1 = self.r(), self.r()
+            self.e("ld.shared.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, sadr, h * HALF_BYTES))
+            for i, w in enumerate((w0, w1)):
+                lo, hi = self.r(), self.r()
+                self.e("shl.b32 %s, %s, 16;" % (lo, w))
+                self.e("and.b32 %s, %s, 0xffff0000;" % (hi, w))
+                self.pack(lo, hi, A[2 * h + i])
+        nadr, off, pr = self.rd(), self.rd(), self.p()      # the copy of the next tile, when it exists as a whole
+        self.e("setp.ne.u32 %s, %%tnext, 0;" % pr)
+        self.e("mul.wide.u32 %s, %%tnext, 2;" % off)
+        self.e("add.u64 %s, %s, %s;" % (nadr, adr, off))
+        self.async_copy_h(sadr, nadr, pr)
+        self.jump()
+        self.label(slow)       # a ragged tile is never staged
+        self.load_bf16_slow(adr, A)
+        self.jump()
+
     def leaf_ldsw(self, dst, copy_to=None, then_copy=False):
         ptr, sadr = self.staged_operand()
         self.fetch()
@@ -619,6 +665,10 @@ class Kernel:
         self.jump()
         self.label(slowb)
         self.prefetch(adr, 2, pfullk)
+        self.load_bf16_slow(adr, A)
+        self.jump()
+
+    def load_bf16_slow(self, adr, A):
         pvec = self.pvec()
         for h in range(2):
             lv, ln = self.newlabel("gld"), self.newlabel("gld")
@@ -648,7 +698,6 @@ class Kernel:
                 self.e("and.b32 %s, %s, 0xffff0000;" % (hi, w))
                 self.pack(lo, hi, A[2 * h + i])
             self.label(ln)
-        self.jump()
 
     def store_f32_slow(self, adr):
         A = self.A
@@ -981,6 +1030,10 @@ class Kernel:
             self.leaf_ldsw(A); return
         elif op == "ldswa":
             self.leaf_ldsw(A, None, True); return
+        elif op == "glda0h":
+            self.leaf_glda0h(); return
+        elif op == "ldswah":
+            self.leaf_ldswah(); return
         elif op == "gstf":
             self.leaf_gstf(); return
         elif op == "fill":
