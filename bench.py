@@ -142,6 +142,10 @@ def run_other_config(args):
         n = 1 << 27
         g, inputs, outputs = wl.random_dag(n, seeds["random_dag"]["seed"])
         units, what = n, "random 64-operator elementwise DAG, 4 x fp32[2^27], 2 fetches"
+    elif args.config == 6:   # not one of the five: the SGD weight update as a graph of its own, 12 bytes per element
+        n = 1 << 26
+        g, ids = wl.updater([n], "sgd")
+        inputs, outputs, units, what = [ids["W"], ids["g"], ids["lr"]], [ids["W_new"]], n, "SGD updater W - lr*g, fp32[2^26] (memory-bound: 12 B/element)"
     elif args.config == 4:
         g, ids = wl.mlp(8192, 4096, 4096, 4096)
         inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
@@ -187,8 +191,8 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU (default: the benchmark's 2^26)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5],
-                    help="2 (default) is the benchmark workload; the others print one summary line each")
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6],
+                    help="2 (default) is the benchmark workload; the others print one summary line each (6: SGD updater)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
