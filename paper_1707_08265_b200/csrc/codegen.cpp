@@ -574,7 +574,8 @@ struct Gen {
     seg->code.insert(seg->code.end(), preamble.begin(), preamble.end());
     seg->loop_start = (int)seg->code.size();
     seg->code.insert(seg->code.end(), body.begin(), body.end());
-    seg->code.push_back(encode(P_LOOP_END, 0, 0));
+    if (!body.empty() && (body.back() & 1023u) == (uint32_t)P_GSTF) seg->code.back() = encode(P_GSTFL, 0, body.back() >> 14);   // store and loop end in one instruction
+    else seg->code.push_back(encode(P_LOOP_END, 0, 0));
     seg->code.insert(seg->code.end(), epi.begin(), epi.end());
     seg->code.push_back(encode(P_END, 0, 0));
     seg->code.push_back(encode(P_END, 0, 0));  // the interpreter prefetches one word ahead

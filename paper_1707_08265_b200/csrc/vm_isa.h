@@ -91,6 +91,7 @@ enum Plain : int {
   P_LDSW,               // acc = the current tile: waits for this thread's copies and reads S[slot]
                         // (a ragged tile was not staged and is loaded directly)
   P_LDSWA,              // P_LDSW, then P_GLDA for the same operand and slot (the tile is read once per iteration)
+  P_GSTFL,              // P_GSTF followed by P_LOOP_END (a body that ends in a store)
   P_GLDA0H,             // P_GLDA0 for a bf16 operand (8 bytes per thread and half of the tile)
   P_LDSWAH,             // P_LDSWA for a bf16 operand: converts to fp32 at the read; such an operand is read once per iteration
   P_END,

@@ -45,13 +45,13 @@ JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "a
 # branch-table code and changes its register allocation, and larger sets ran slower on all three
 # large workloads (16 more short leaves: +3 % on the sin/cos graph, +3 % on the random DAG), so the
 # list holds the short arithmetic, store and staged-load leaves it was first tried with.
-HOT = {"fmau", "mul", "sacc0", "macc1", "fmaur", "gstf", "cossinr", "ldswar"}
+HOT = {"fmau", "mul", "sacc0", "macc1", "fmaur", "gstf", "gstfl", "cossinr", "ldswar"}
 JOINT_STRIDE = 8    # case id of a joint instruction = index * JOINT_STRIDE + register slot
 N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "glda0h", "ldswah", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "end"]
 
 
 def f32bits(x):
@@ -719,19 +719,27 @@ class Kernel:
             self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (adr, h * HALF_BYTES, A[2 * h], A[2 * h + 1]))
             self.label(ln)
 
-    def leaf_gstf(self):
-        """acc -> fp32 FULL operand"""
+    def leaf_gstf(self, then_loop_end=False):
+        """acc -> fp32 FULL operand (and, fused, the end of the per-tile body)"""
         ptr, _, _ = self.operand(False)
-        self.fetch()
+        if not then_loop_end:
+            self.fetch()
         adr = self.rd()
         self.e("add.u64 %s, %s, %%tb4;" % (adr, ptr))
-        slow = self.newlabel("gstf")
+        slow, done = self.newlabel("gstf"), self.newlabel("gstf")
         self.e("@!%%pfull bra.uni %s;" % slow)
         self.stg_v(adr, self.A)
-        self.jump()
+        if then_loop_end:
+            self.e("bra.uni %s;" % done)
+        else:
+            self.jump()
         self.label(slow)
         self.store_f32_slow(adr)
-        self.jump()
+        if then_loop_end:
+            self.label(done)
+            self.leaf_loop_end()
+        else:
+            self.jump()
 
     def leaf_gst(self):
         """acc -> any operand"""
@@ -1036,6 +1044,8 @@ class Kernel:
             self.leaf_ldswah(); return
         elif op == "gstf":
             self.leaf_gstf(); return
+        elif op == "gstfl":
+            self.leaf_gstf(True); return
         elif op == "fill":
             a = self.spill_addr(); self.fetch(); self.ldg_v(a, A)
         elif op == "spill":

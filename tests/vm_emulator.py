@@ -11,7 +11,7 @@ J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
-     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "glda0h", "ldswah", "end"]
+     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "end"]
 
 
 def _bf16(a):
@@ -93,7 +93,7 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
         elif name == "rbf16": acc = _bf16(acc)
         elif name == "rowsum": acc = np.broadcast_to(acc.sum(axis=-1, keepdims=True), shape).copy()
         elif name in ("gld", "gldf"): acc = load(arg)
-        elif name in ("gst", "gstf"):
+        elif name in ("gst", "gstf", "gstf}loop"):
             where, pos, kind, dtype = ops[arg]
             assert where == 1
             v = acc if kind == 0 else (acc[0] if kind == 1 else acc.reshape(-1)[0])
