@@ -551,6 +551,17 @@ struct Gen {
       fused.push_back(w);
     }
     body.swap(fused);
+    fused.clear();
+    for (size_t i = 0; i < body.size(); ++i) {   // "R[a] = acc; acc = R[b]" is one instruction
+      const uint32_t c0 = body[i] & 1023u, c1 = i + 1 < body.size() ? (body[i + 1] & 1023u) : ~0u;
+      if (c0 >= (uint32_t)(J_STR * kJointStride) && c0 < (uint32_t)(J_STR * kJointStride + nr) &&
+          c1 < (uint32_t)(J_LDR * kJointStride + nr)) {   // J_LDR is the first group: case ids [0, nr)
+        const int a = (int)(c0 - J_STR * kJointStride), b = (int)(c1 - J_LDR * kJointStride);
+        if (a != b) { fused.push_back(encode((J_STLD0 + a) * kJointStride + b, 0, 0)); ++i; continue; }
+      }
+      fused.push_back(body[i]);
+    }
+    body.swap(fused);
     stage_loads();
     // 6. epilogue: accumulators leave as per-CTA partial sums
     for (auto& a : accs) {

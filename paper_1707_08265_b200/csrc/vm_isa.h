@@ -40,6 +40,9 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   J_MACC0, J_MACC1, J_MACC2, J_MACC3,   // A[i] += sum over this thread's valid lanes of acc * R   (acc unchanged)
   J_LDSWR,     // R = acc = staged operand (P_LDSW)
   J_LDSWAR,    // J_LDSWR, then P_GLDA for the same operand and slot
+  // R[a] = acc; acc = R: the most frequent pair of instructions ("put this away, take that") as one,
+  // one group per a (the slot index of the case id is the register that is loaded)
+  J_STLD0, J_STLD1, J_STLD2, J_STLD3, J_STLD4, J_STLD5, J_STLD6, J_STLD7,
   J_COUNT
 };
 // The kernel exists in two builds that share this encoding: "wide" (7 register slots, one CTA per

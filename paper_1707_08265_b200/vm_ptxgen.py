@@ -39,7 +39,8 @@ P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
 OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
-         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar"]
+         "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
+         "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7"]
 # Leaves that end in their own indexed branch instead of a jump to the shared dispatch block: one
 # taken branch less per dispatch.  Measured, not derived: every further site makes the assembler add
 # branch-table code and changes its register allocation, and larger sets ran slower on all three
@@ -859,6 +860,10 @@ class Kernel:
         elif op == "ldswar":
             self.leaf_ldsw(R, A, True)
             return
+        elif op.startswith("stld"):     # R[a] = acc; acc = R[k]
+            self.fetch()
+            self.mov_v(self.R[int(op[4])], A)
+            self.mov_v(A, R)
         elif op in ("sincosr", "cossinr"):
             self.fetch()
             S, C = self.sincos(A)
@@ -1268,7 +1273,8 @@ class Kernel:
         cases = []
         for op in JOINT:
             for k in range(JOINT_STRIDE):
-                cases.append(("j", op, k) if k < nr else ("bad", op, k))
+                no_slot = op.startswith("stld") and int(op[4]) >= nr
+                cases.append(("j", op, k) if k < nr and not no_slot else ("bad", op, k))
         for op in PLAIN:
             cases.append(("p", op, 0))
         bad = "$BAD_%s" % self.name

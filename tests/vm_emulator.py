@@ -7,7 +7,8 @@ import numpy as np
 
 STRIDE = 8   # case id of a register-operand instruction = index * STRIDE + register slot
 J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
-     "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar"]
+     "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
+     "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7"]
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
@@ -67,6 +68,9 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
             elif name == "sincosr": R[k] = np.cos(acc); acc = np.sin(acc)
             elif name == "cossinr": R[k] = np.sin(acc); acc = np.cos(acc)
             elif name.startswith("macc"): A[int(name[4])] += float((acc * R[k]).sum())
+            elif name.startswith("stld"):
+                assert int(name[4]) < nr
+                R[int(name[4])] = acc.copy(); acc = R[k].copy()
             else: raise ValueError(name)
             continue
         name = P[cs - first_plain]
