@@ -562,6 +562,18 @@ struct Gen {
       fused.push_back(body[i]);
     }
     body.swap(fused);
+    {   // row sums alternate between scratch buffers so that each needs one barrier only; successive
+        // ones (the last of an iteration and the first of the next included) never share a buffer
+      std::vector<size_t> rs;
+      for (size_t i = 0; i < body.size(); ++i)
+        if ((body[i] & 1023u) == (uint32_t)P_ROWSUM) rs.push_back(i);
+      for (size_t j = 0; j < rs.size(); ++j) {
+        uint32_t arg = (uint32_t)(j & 1);
+        if (rs.size() == 1) arg = 4;                                   // alone in the body: barrier after the read too
+        else if ((rs.size() & 1) && j + 1 == rs.size()) arg = 2;        // odd count: the last one takes a third buffer
+        body[rs[j]] = encode(P_ROWSUM, 0, arg);
+      }
+    }
     stage_loads();
     // 6. epilogue: accumulators leave as per-CTA partial sums
     for (auto& a : accs) {

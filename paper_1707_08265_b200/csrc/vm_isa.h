@@ -70,7 +70,8 @@ enum Plain : int {
   P_YOMY,               // acc = acc * (1 - acc)
   P_DIVPGB,             // acc = -sgn(acc) / (1 + |acc|)^2
   P_RBF16,              // acc = float(bf16(acc)), round to nearest even
-  P_ROWSUM,             // acc = sum of acc over the whole row (all lanes, all threads), row mode only
+  P_ROWSUM,             // acc = sum of acc over the whole row (all lanes, all threads), row mode only;
+                        // arg bits 0..1: scratch buffer (successive row sums differ), bit 2: barrier after the read too
   P_GLD,                // acc = operand[arg] at this tile
   P_GST,                // operand[arg] at this tile = acc
   P_GLDF,               // P_GLD for an fp32 operand of the full domain shape

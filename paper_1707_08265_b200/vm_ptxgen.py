@@ -1026,9 +1026,14 @@ class Kernel:
                 self.e("shl.b32 %s, %s, 16;" % (l2, w))
                 self.e("and.b32 %s, %s, 0xffff0000;" % (h2, w))
                 self.pack(l2, h2, A[i])
-        elif op == "rowsum":
+        elif op == "rowsum":     # arg: scratch buffer (bits 0..1), barrier after the read as well (bit 2)
+            boff, t, psync = self.r(), self.r(), self.p()
+            self.e("and.b32 %s, %%arg, 3;" % boff)
+            self.e("shl.b32 %s, %s, 6;" % (boff, boff))
+            self.e("and.b32 %s, %%arg, 4;" % t)
+            self.e("setp.ne.u32 %s, %s, 0;" % (psync, t))
             self.fetch()
-            self.leaf_rowsum()
+            self.leaf_rowsum(boff, psync)
         elif op == "gld":
             self.leaf_gld(); return
         elif op == "gst":
@@ -1093,7 +1098,11 @@ class Kernel:
         self.e("shr.u32 %s, %s, 5;" % (warp, t))
         return warp, lane
 
-    def leaf_rowsum(self):
+    def leaf_rowsum(self, boff, psync):
+        """acc = sum of acc over the row.  Successive row sums write their per-warp partials to
+        different scratch buffers (the host alternates them), so one barrier per sum is enough: a
+        buffer is written again only after another row sum's barrier, which every warp passes after
+        it has read this one."""
         A = self.A
         full, go = self.newlabel("rs"), self.newlabel("rs")
         s = self.f()
@@ -1114,17 +1123,22 @@ class Kernel:
         warp, lane = self.warp_and_lane()
         pr, a = self.p(), self.r()
         self.e("setp.eq.u32 %s, %s, 0;" % (pr, lane))
+        base = self.r()
+        self.e("add.u32 %s, %%ub, %s;" % (base, boff))
         self.e("shl.b32 %s, %s, 2;" % (a, warp))
-        self.e("add.u32 %s, %s, %%ub;" % (a, a))
+        self.e("add.u32 %s, %s, %s;" % (a, a, base))
         self.e("@%s st.shared.f32 [%s+%d], %s;" % (pr, a, OFF_RED, s))
         self.e("bar.sync 0;")
         tot = self.f()
         self.e("mov.f32 %s, 0f00000000;" % tot)
         for i in range(NT // 128):
             q = [self.f() for _ in range(4)]
-            self.e("ld.shared.v4.f32 {%s, %s, %s, %s}, [%%ub+%d];" % (q[0], q[1], q[2], q[3], OFF_RED + 16 * i))
+            self.e("ld.shared.v4.f32 {%s, %s, %s, %s}, [%s+%d];" % (q[0], q[1], q[2], q[3], base, OFF_RED + 16 * i))
             for x in q: self.e("add.f32 %s, %s, %s;" % (tot, tot, x))
+        nosync = self.newlabel("rs")
+        self.e("@!%s bra.uni %s;" % (psync, nosync))
         self.e("bar.sync 0;")
+        self.label(nosync)
         tt = self.splat(tot)
         for i in range(NP): self.e("mov.b64 %s, %s;" % (A[i], tt))
 
@@ -1253,7 +1267,7 @@ class Kernel:
         self.e("setp.eq.u32 %s, %s, 0;" % (pr, lane))
         self.e("shl.b32 %s, %s, 3;" % (a, warp))
         self.e("add.u32 %s, %s, %%ub;" % (a, a))
-        self.e("@%s st.shared.f64 [%s+%d], %s;" % (pr, a, OFF_RED, s))
+        self.e("@%s st.shared.f64 [%s+%d], %s;" % (pr, a, OFF_RED + 256, s))
         self.e("bar.sync 0;")
         skip = self.newlabel("so")
         self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
@@ -1261,7 +1275,7 @@ class Kernel:
         self.e("mov.f64 %s, 0d0000000000000000;" % tot)
         for i in range(NT // 32):
             d = self.fd()
-            self.e("ld.shared.f64 %s, [%%ub+%d];" % (d, OFF_RED + 8 * i))
+            self.e("ld.shared.f64 %s, [%%ub+%d];" % (d, OFF_RED + 256 + 8 * i))
             self.e("add.f64 %s, %s, %s;" % (tot, tot, d))
         self.e("st.global.f64 [%s], %s;" % (o, tot))
         self.label(skip)
