@@ -1106,15 +1106,11 @@ class Kernel:
         A = self.A
         full, go = self.newlabel("rs"), self.newlabel("rs")
         s = self.f()
-        sc = self.scalars(A)
         self.e("@%%pfull bra.uni %s;" % full)
-        m = self.mask_tail(sc)
-        self.e("mov.f32 %s, 0f00000000;" % s)
-        for x in m: self.e("add.f32 %s, %s, %s;" % (s, s, x))
+        self.e("mov.f32 %s, %s;" % (s, self.lane_sum(self.packs(self.mask_tail(self.scalars(A))))))
         self.e("bra.uni %s;" % go)
         self.label(full)
-        self.e("mov.f32 %s, 0f00000000;" % s)
-        for x in sc: self.e("add.f32 %s, %s, %s;" % (s, s, x))
+        self.e("mov.f32 %s, %s;" % (s, self.lane_sum(A)))      # pairwise, with packed additions
         self.label(go)
         for o in (16, 8, 4, 2, 1):
             t = self.f()
@@ -1129,12 +1125,14 @@ class Kernel:
         self.e("add.u32 %s, %s, %s;" % (a, a, base))
         self.e("@%s st.shared.f32 [%s+%d], %s;" % (pr, a, OFF_RED, s))
         self.e("bar.sync 0;")
-        tot = self.f()
-        self.e("mov.f32 %s, 0f00000000;" % tot)
+        q = [self.rd() for _ in range(NT // 64)]       # the 16 per-warp partials as 8 packed pairs, summed pairwise
         for i in range(NT // 128):
-            q = [self.f() for _ in range(4)]
-            self.e("ld.shared.v4.f32 {%s, %s, %s, %s}, [%s+%d];" % (q[0], q[1], q[2], q[3], base, OFF_RED + 16 * i))
-            for x in q: self.e("add.f32 %s, %s, %s;" % (tot, tot, x))
+            self.e("ld.shared.v2.b64 {%s, %s}, [%s+%d];" % (q[2 * i], q[2 * i + 1], base, OFF_RED + 16 * i))
+        while len(q) > 1:
+            q = [self.add2(q[2 * i], q[2 * i + 1]) for i in range(len(q) // 2)]
+        lo, hi = self.unpack(q[0])
+        tot = self.f()
+        self.e("add.f32 %s, %s, %s;" % (tot, lo, hi))
         nosync = self.newlabel("rs")
         self.e("@!%s bra.uni %s;" % (psync, nosync))
         self.e("bar.sync 0;")
