@@ -160,7 +160,11 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
  * runs, and copies every fetched output to host_fetches[j], all asynchronously on cuda_stream
  * (the caller synchronises the stream before reading the results; pinned host memory makes the
  * copies truly asynchronous).  staging_dev: caller-owned device memory, 256-byte aligned, at
- * least dragon_function_staging_bytes() long.  Entries of pruned inputs may be NULL. */
+ * least dragon_function_staging_bytes() long.  Entries of pruned inputs may be NULL.
+ * A function that is a single elementwise launch over a large flat domain is run in chunks of
+ * the element range, with the copies of neighbouring chunks on two streams of the function's own
+ * so that copy-in, kernel and copy-out overlap; cuda_stream still orders the call as a whole (it
+ * waits for the last copy-out), so the caller sees the same behaviour. */
 size_t dragon_function_staging_bytes(const dragon_function_t* f);
 int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* const* host_fetches,
                     void* staging_dev, size_t staging_bytes, void* cuda_stream);

@@ -9,7 +9,7 @@
 
 namespace dragon {
 cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st);
-cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st);
+cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st, int chunks);
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
                            int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm);
 cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
@@ -193,6 +193,8 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
 void dragon_function_destroy(dragon_function_t* f) {
   if (!f) return;
   for (void* ev : f->prof_ev) cudaEventDestroy(reinterpret_cast<cudaEvent_t>(ev));
+  for (void* ev : f->h_event) cudaEventDestroy(reinterpret_cast<cudaEvent_t>(ev));
+  for (void* s : f->h_stream) if (s) cudaStreamDestroy(reinterpret_cast<cudaStream_t>(s));
   for (auto& sg : f->plan.segs)
     if (sg.d_code) cudaFree(sg.d_code);
   delete f;
@@ -357,7 +359,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used]), st);
         e = launch_vm(p, sg.grid, sg.n_smem, sg.dense, st);
         if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used + 1]), st);
-        if (e == cudaSuccess) e = launch_finish(sg, P.mems, ptr.data(), ws, st);
+        if (e == cudaSuccess) e = launch_finish(sg, P.mems, ptr.data(), ws, st, 1);
         break;
       }
       case ST_GEMM: {
@@ -412,6 +414,142 @@ size_t dragon_function_staging_bytes(const dragon_function_t* f) {
   return n;
 }
 
+namespace {
+
+// A function that is one flat elementwise VM launch over many tiles, whose tensors all have the
+// domain's shape or are scalars, can run in chunks of the element range: the copy-in of chunk c+1,
+// the kernel of chunk c and the copy-out of chunk c-1 then overlap (the link is full duplex).
+bool chunkable(const dragon_function_t* f) {
+  const Plan& P = f->plan;
+  if (P.steps.size() != 1 || P.steps[0].kind != ST_VM) return false;
+  const VmSegment& sg = P.segs[P.steps[0].seg];
+  if (sg.row_mode || sg.n_spill || sg.n_colacc) return false;
+  const long long tiles = (sg.n + kVmTile - 1) / kVmTile;
+  if (tiles / kHostChunks < sg.grid) return false;          // every chunk keeps all CTAs busy
+  for (uint32_t k : sg.operand_kind) if (k != vm::K_FULL && k != vm::K_SCALAR) return false;
+  for (int m : sg.operand_mem) if (P.mems[m].where == MEM_WORK) return false;
+  for (const FinishJob& j : sg.finish) if (j.kind != 1) return false;
+  for (const MemRef& m : P.mems)
+    if (m.live && m.where != MEM_WORK && m.shape.numel() != sg.n && m.shape.numel() != 1) return false;
+  return true;
+}
+
+#define HOST_TRY(call) do { cudaError_t e_ = (call); if (e_ != cudaSuccess) { f->status_ready = false; \
+  set_error("dragon_run_host: CUDA error: %s", cudaGetErrorString(e_)); return DRAGON_ERR_CUDA; } } while (0)
+
+int run_host_chunked(dragon_function_t* f, const std::vector<const void*>& dev_feeds, const std::vector<void*>& dev_fetches,
+                     const void* const* host_feeds, void* const* host_fetches, cudaStream_t st) {
+  Plan& P = f->plan;
+  VmSegment& sg = P.segs[P.steps[0].seg];
+  if (!f->workspace) { set_error("dragon_run_host: no workspace set (need %zu bytes)", P.workspace_bytes); return DRAGON_ERR_WORKSPACE; }
+  char* ws = reinterpret_cast<char*>(f->workspace);
+  if (!f->h_stream[0]) {
+    for (void*& s : f->h_stream) {
+      cudaStream_t ns;
+      HOST_TRY(cudaStreamCreateWithFlags(&ns, cudaStreamNonBlocking));
+      s = ns;
+    }
+    for (int i = 0; i < 2 * kHostChunks + 2; ++i) {
+      cudaEvent_t ev;
+      HOST_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+      f->h_event.push_back(ev);
+    }
+  }
+  cudaStream_t s_in = reinterpret_cast<cudaStream_t>(f->h_stream[0]), s_out = reinterpret_cast<cudaStream_t>(f->h_stream[1]);
+  auto ev = [&](int i) { return reinterpret_cast<cudaEvent_t>(f->h_event[i]); };
+  cudaEvent_t ev_start = ev(2 * kHostChunks), ev_done = ev(2 * kHostChunks + 1);
+  if (!f->uploaded) {
+    HOST_TRY(cudaMalloc(&sg.d_code, sg.code.size() * 4));
+    HOST_TRY(cudaMemcpy(sg.d_code, sg.code.data(), sg.code.size() * 4, cudaMemcpyHostToDevice));
+    f->uploaded = true;
+  }
+  int* const word0 = reinterpret_cast<int*>(ws + P.status_off);
+  if (!f->status_ready) {
+    HOST_TRY(cudaMemsetAsync(word0, 0, 256, st));
+    f->status_ready = true;
+    f->run_parity = 0;
+  }
+  int* const status = word0 + 16 * f->run_parity;
+  int* const status_next = word0 + 16 * (f->run_parity ^ 1);
+  // the copy-in stream starts after everything already queued on the caller's stream (the previous run reads the staging area)
+  HOST_TRY(cudaEventRecord(ev_start, st));
+  HOST_TRY(cudaStreamWaitEvent(s_in, ev_start, 0));
+  HOST_TRY(cudaStreamWaitEvent(s_out, ev_start, 0));
+  // scalars go first, whole
+  for (const MemRef& m : P.mems)
+    if (m.live && m.where == MEM_FEED && m.shape.numel() == 1 && sg.n != 1)
+      HOST_TRY(cudaMemcpyAsync(const_cast<void*>(dev_feeds[m.index]), host_feeds[m.index], m.bytes(), cudaMemcpyHostToDevice, s_in));
+  const long long tiles = (sg.n + kVmTile - 1) / kVmTile, base_tiles = tiles / kHostChunks, extra = tiles % kHostChunks;
+  long long tile0 = 0;
+  for (int c = 0; c < kHostChunks; ++c) {
+    const long long ntile = base_tiles + (c < extra ? 1 : 0);
+    const long long e0 = tile0 * kVmTile, e1 = std::min<long long>(sg.n, (tile0 + ntile) * kVmTile), cn = e1 - e0;
+    tile0 += ntile;
+    std::vector<uint8_t> done_in(f->n_in, 0), done_out(f->n_out, 0);
+    for (const MemRef& m : P.mems) {
+      if (!m.live || m.where != MEM_FEED || m.shape.numel() == 1 || done_in[m.index]) continue;
+      done_in[m.index] = 1;
+      const size_t es = m.dtype == DRAGON_BF16 ? 2 : 4;
+      HOST_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(const_cast<void*>(dev_feeds[m.index])) + e0 * es,
+                               reinterpret_cast<const char*>(host_feeds[m.index]) + e0 * es, (size_t)cn * es, cudaMemcpyHostToDevice, s_in));
+    }
+    HOST_TRY(cudaEventRecord(ev(c), s_in));
+    HOST_TRY(cudaStreamWaitEvent(st, ev(c), 0));
+    vm::Params p;
+    std::memset(&p, 0, sizeof(p));
+    p.code = sg.d_code;
+    p.n_code = (int)sg.code.size();
+    p.n = cn;
+    p.n_tiles = (uint32_t)ntile;
+    p.loop_start = (uint32_t)sg.loop_start;
+    p.grid = (uint32_t)sg.grid;
+    p.n_full_tiles = (uint32_t)(cn / kVmTile);
+    p.spill = reinterpret_cast<float*>(ws + sg.spill_off);
+    p.colpart = reinterpret_cast<float*>(ws + sg.colpart_off);
+    p.scalpart = reinterpret_cast<double*>(ws + sg.scalpart_off) + (size_t)c * sg.n_scalacc * sg.grid;
+    p.status = status;
+    p.status_clear = c == 0 ? status_next : nullptr;
+    for (size_t i = 0; i < sg.operand_mem.size(); ++i) {
+      const MemRef& m = P.mems[sg.operand_mem[i]];
+      char* q = reinterpret_cast<char*>(m.where == MEM_FEED ? const_cast<void*>(dev_feeds[m.index]) : dev_fetches[m.index]);
+      if (sg.operand_kind[i] == vm::K_FULL) q += e0 * (m.dtype == DRAGON_BF16 ? 2 : 4);
+      p.operand[i].ptr = q;
+      p.operand[i].kind = sg.operand_kind[i];
+      p.operand[i].dtype = (uint32_t)m.dtype;
+    }
+    HOST_TRY(launch_vm(p, sg.grid, sg.n_smem, sg.dense, st));
+    HOST_TRY(cudaEventRecord(ev(kHostChunks + c), st));
+    HOST_TRY(cudaStreamWaitEvent(s_out, ev(kHostChunks + c), 0));
+    for (const MemRef& m : P.mems) {
+      if (!m.live || m.where != MEM_FETCH || m.shape.numel() == 1 || done_out[m.index]) continue;
+      done_out[m.index] = 1;
+      const size_t es = m.dtype == DRAGON_BF16 ? 2 : 4;
+      HOST_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(host_fetches[m.index]) + e0 * es,
+                               reinterpret_cast<char*>(dev_fetches[m.index]) + e0 * es, (size_t)cn * es, cudaMemcpyDeviceToHost, s_out));
+    }
+  }
+  // sums over the whole domain: the partials of all chunks, then their copy to the host
+  std::vector<void*> mem_ptr(P.mems.size(), nullptr);
+  for (size_t m = 0; m < P.mems.size(); ++m)
+    if (P.mems[m].live && P.mems[m].where == MEM_FETCH) mem_ptr[m] = dev_fetches[P.mems[m].index];
+  HOST_TRY(launch_finish(sg, P.mems, mem_ptr.data(), ws, st, kHostChunks));
+  std::vector<uint8_t> done_out(f->n_out, 0);
+  for (const MemRef& m : P.mems) {
+    if (!m.live || m.where != MEM_FETCH || m.shape.numel() != 1 || done_out[m.index]) continue;
+    done_out[m.index] = 1;
+    HOST_TRY(cudaMemcpyAsync(host_fetches[m.index], dev_fetches[m.index], m.bytes(), cudaMemcpyDeviceToHost, st));
+  }
+  // the caller's stream ends after the last copy-out
+  HOST_TRY(cudaEventRecord(ev_done, s_out));
+  HOST_TRY(cudaStreamWaitEvent(st, ev_done, 0));
+  f->last_status_word = f->run_parity;
+  f->run_parity ^= 1;
+  f->last_stream = st;
+  return DRAGON_OK;
+}
+
+}  // namespace
+
 int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* const* host_fetches, void* staging_dev,
                     size_t staging_bytes, void* cuda_stream) {
   if (!f || !host_fetches || (f->n_in > 0 && !host_feeds)) { set_error("dragon_run_host: bad argument"); return DRAGON_ERR_INVALID_ARG; }
@@ -420,6 +558,7 @@ int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* c
     return DRAGON_ERR_WORKSPACE;
   }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const bool chunked = chunkable(f) && f->prof_step < 0;
   std::vector<const void*> feeds(f->n_in, nullptr);
   std::vector<void*> fetches(f->n_out, nullptr);
   char* base = reinterpret_cast<char*>(staging_dev);
@@ -431,7 +570,7 @@ int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* c
     if (m.where == MEM_FEED && !feeds[m.index]) {
       if (!host_feeds[m.index]) { set_error("dragon_run_host: feed %d is NULL", m.index); return DRAGON_ERR_INVALID_ARG; }
       feeds[m.index] = base + off;
-      if (cudaMemcpyAsync(base + off, host_feeds[m.index], m.bytes(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
+      if (!chunked && cudaMemcpyAsync(base + off, host_feeds[m.index], m.bytes(), cudaMemcpyHostToDevice, st) != cudaSuccess) {
         set_error("dragon_run_host: host-to-device copy failed: %s", cudaGetErrorString(cudaGetLastError()));
         return DRAGON_ERR_CUDA;
       }
@@ -441,6 +580,7 @@ int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* c
     }
     off += sz;
   }
+  if (chunked) return run_host_chunked(f, feeds, fetches, host_feeds, host_fetches, st);
   int rc = dragon_run(f, feeds.data(), fetches.data(), cuda_stream);
   if (rc != DRAGON_OK) return rc;
   std::vector<uint8_t> copied(f->n_out, 0);

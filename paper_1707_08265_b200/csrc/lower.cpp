@@ -505,7 +505,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
   for (auto& sg : plan->segs) {
     sg.spill_off = take((size_t)sg.grid * sg.n_spill * kVmTile * sizeof(float));
     sg.colpart_off = take((size_t)sg.n_colacc * sg.grid * sg.cols * sizeof(float));
-    sg.scalpart_off = take((size_t)sg.n_scalacc * sg.grid * sizeof(double));
+    sg.scalpart_off = take((size_t)kHostChunks * sg.n_scalacc * sg.grid * sizeof(double));   // a set per chunk of a chunked host run
   }
   for (auto& st : plan->steps)
     if (st.kind == ST_SCE_FWD) st.scratch_off = take((size_t)mems[st.mA].shape.d[0] * sizeof(float));

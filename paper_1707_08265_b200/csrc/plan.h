@@ -18,6 +18,7 @@ constexpr int kVmCodeMaxWords = 8 * 1024;     // instruction stream held in shar
 constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread (wide build: one CTA per SM)
 constexpr int kVmSmemSlotsDense = 6;          // the same for the dense build (two CTAs share the SM's shared memory)
 constexpr int kDefaultSmCount = 148;
+constexpr int kHostChunks = 16;               // dragon_run_host pipelines a large elementwise function in this many chunks
 
 enum MemWhere { MEM_FEED = 0, MEM_FETCH = 1, MEM_WORK = 2 };
 
@@ -131,6 +132,9 @@ struct dragon_function {
   // run after it, so that no run needs a memset of its own
   bool status_ready = false;
   int run_parity = 0, last_status_word = 0;
+  // dragon_run_host, chunked: copy-in and copy-out streams and the events that order them (made on first use)
+  void* h_stream[2] = {nullptr, nullptr};
+  std::vector<void*> h_event;
   // profiling ring (dragon_function_profile)
   int prof_step = -1, prof_used = 0;
   std::vector<void*> prof_ev;   // 2 * capacity cudaEvent_t

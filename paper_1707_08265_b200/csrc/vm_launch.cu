@@ -26,6 +26,7 @@ struct FinishParams {
     const void* part;  // float [grid][cols] or double [grid]
     void* out;
     int dtype, cols, grid;
+    int chunks, chunk_stride;              // scalar partials of a chunked run: one [accumulator][grid] set per chunk
   } job[8];
 };
 
@@ -48,7 +49,8 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
     __shared__ double sh[128];
     const double* part = reinterpret_cast<const double*>(jb.part);
     double s = 0.0;
-    for (int g = threadIdx.x; g < jb.grid; g += 128) s += part[g];
+    for (int c = 0; c < jb.chunks; ++c)
+      for (int g = threadIdx.x; g < jb.grid; g += 128) s += part[(size_t)c * jb.chunk_stride + g];
     sh[threadIdx.x] = s;
     __syncthreads();
     for (int w = 64; w > 0; w >>= 1) {
@@ -98,7 +100,7 @@ cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dens
   return cudaLaunchKernel(reinterpret_cast<const void*>(dense ? k.dense : k.wide), dim3(grid), dim3(kVmThreads), args, smem, st);
 }
 
-cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st) {
+cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st, int chunks) {
   if (sg.finish.empty()) return cudaSuccess;
   vm::FinishParams fp;
   fp.n_jobs = (int)sg.finish.size();
@@ -109,6 +111,8 @@ cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, 
     o.kind = j.kind;
     o.grid = sg.grid;
     o.cols = sg.cols;
+    o.chunks = chunks;
+    o.chunk_stride = sg.n_scalacc * sg.grid;
     o.dtype = mems[j.mem].dtype;
     o.out = mem_ptr[j.mem];
     if (j.kind == 0) { o.part = ws + sg.colpart_off + (size_t)j.acc * sg.grid * sg.cols * sizeof(float); max_cols = std::max(max_cols, sg.cols); }
