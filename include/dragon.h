@@ -121,6 +121,18 @@ int dragon_function_marked(const dragon_function_t* f, uint8_t* flag_per_tensor,
 int dragon_function_kept_ops(const dragon_function_t* f, dragon_id* fwd_ops, int cap_f, int* n_f,
                              dragon_id* grad_ops, uint32_t* grad_input_mask, int cap_g, int* n_g);
 
+/* In-place structures of the pruned graph (Sec. 2.4, Algorithm 3): ancestor[t] is the tensor whose
+ * memory tensor t may share - the first node, in creation order, of the path of nodes with exactly
+ * one child that leads to t (t itself when it starts a path), or -1 if t is not marked.  Marked
+ * tensors and kept forward operators take part (the paper renames after the prunes). */
+int dragon_function_rename_dictionary(const dragon_function_t* f, dragon_id* ancestor, int n_tensors);
+
+/* The tensors that cross kernels inside the caller's workspace, after memory sharing: up to cap
+ * quintuples {byte offset, bytes, first plan step that touches it, last one, 1 if it was placed over an
+ * input of its producing step (in place)}.  Returns their number.  Two tensors whose step ranges
+ * overlap never share bytes, except an in-place output and the input it replaces. */
+int dragon_function_workspace_tensors(const dragon_function_t* f, int64_t* out, int cap);
+
 /* One byte per listed input: 1 if the pruned function reads it. */
 int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flag_per_input, int n_in);
 

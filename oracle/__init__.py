@@ -3,7 +3,9 @@
 TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, node-at-a-time fp64
 restatement of what a compiled ``function(inputs, outputs)`` (Sec. 2.1) computes
 after the forward prune (Sec. 2.2, Algorithm 1) and the backward prune
-(Sec. 2.3, Algorithm 2).  It shares no code with the CUDA library, imports
+(Sec. 2.3, Algorithm 2), plus the in-place structures of the pruned graph
+(Sec. 2.4, Algorithm 3; oracle/inplace.py, pinned in tests/test_inplace.py by
+the definition written out on tiny DAGs).  It shares no code with the CUDA library, imports
 nothing from it, and must never be reached from the product path.  Only the
 tests, the smoke check and the benchmark's CPU-baseline leg may use it.
 

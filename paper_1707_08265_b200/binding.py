@@ -48,6 +48,8 @@ _SIGNATURES = {
     "dragon_function_staging_bytes": (_c.c_size_t, [_c.c_void_p]),
     "dragon_run_host": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_void_p), _c.POINTER(_c.c_void_p), _c.c_void_p,
                                    _c.c_size_t, _c.c_void_p]),
+    "dragon_function_rename_dictionary": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int]),
+    "dragon_function_workspace_tensors": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_int64), _c.c_int]),
     "dragon_function_profile": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_int]),
     "dragon_function_profile_read": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_double), _c.POINTER(_c.c_int)]),
     "dragon_softmax_ce_loss_static": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_void_p, _c.c_int, _c.c_int, _c.c_void_p, _c.c_void_p]),
@@ -224,6 +226,21 @@ class Function:
                 "n_spill": info[4], "n_smem": info[5], "n_regs": info[9],
                 "operands": [tuple(ops[4 * i:4 * i + 4]) for i in range(info[3])],
                 "reduced": [tuple(red[3 * i:3 * i + 3]) for i in range(info[8])]}
+
+    def rename_dictionary(self):
+        """Algorithm 3: per tensor id the ancestor it may be renamed to (-1: not marked)."""
+        rd = (_c.c_int32 * max(1, self.n_tensors))()
+        r = lib().dragon_function_rename_dictionary(self.h, rd, self.n_tensors)
+        if r < 0:
+            raise DragonError(r, "dragon_function_rename_dictionary")
+        return list(rd[:self.n_tensors])
+
+    def workspace_tensors(self):
+        """[(offset, bytes, first step, last step, in place)] of the tensors that cross kernels."""
+        n = lib().dragon_function_workspace_tensors(self.h, None, 0)
+        buf = (_c.c_int64 * max(5, 5 * n))()
+        lib().dragon_function_workspace_tensors(self.h, buf, n)
+        return [tuple(buf[5 * i:5 * i + 5]) for i in range(n)]
 
     def workspace_bytes(self):
         return lib().dragon_function_workspace_bytes(self.h)

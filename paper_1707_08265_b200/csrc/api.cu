@@ -187,6 +187,7 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
   f->n_out = n_out;
   if (prune_function(g->g, in, out, &f->prune) != DRAGON_OK) { delete f; return nullptr; }
   if (lower_function(g->g, f->prune, in, out, query_sm_count(), &f->plan) != DRAGON_OK) { delete f; return nullptr; }
+  f->rename = inplace_rename(g->g, f->prune);
   return f;
 }
 
@@ -223,6 +224,29 @@ int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flags, int 
   if (!f || (n_in > 0 && !flags) || n_in != f->n_in) { set_error("dragon_function_used_inputs: bad argument"); return DRAGON_ERR_INVALID_ARG; }
   if (n_in) std::memcpy(flags, f->prune.used_inputs.data(), (size_t)n_in);
   return DRAGON_OK;
+}
+
+int dragon_function_rename_dictionary(const dragon_function_t* f, dragon_id* ancestor, int n_tensors) {
+  if (!f || !ancestor || n_tensors != f->n_tensors) { set_error("dragon_function_rename_dictionary: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  for (int i = 0; i < n_tensors; ++i) ancestor[i] = f->rename[i];
+  return DRAGON_OK;
+}
+
+int dragon_function_workspace_tensors(const dragon_function_t* f, int64_t* out, int cap) {
+  if (!f || (cap > 0 && !out) || cap < 0) { set_error("dragon_function_workspace_tensors: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  int n = 0;
+  for (const MemRef& m : f->plan.mems) {
+    if (m.where != MEM_WORK || !m.live) continue;
+    if (n < cap) {
+      out[5 * n + 0] = (int64_t)m.offset;
+      out[5 * n + 1] = (int64_t)m.bytes();
+      out[5 * n + 2] = m.first_step;
+      out[5 * n + 3] = m.last_step;
+      out[5 * n + 4] = m.shares_input;
+    }
+    ++n;
+  }
+  return n;
 }
 
 int dragon_function_num_launches(const dragon_function_t* f) {

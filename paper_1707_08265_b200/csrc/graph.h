@@ -76,6 +76,10 @@ bool broadcast_shapes(const Shape& a, const Shape& b, Shape* out);
 // chains wrt ~> obj for one stage (Algorithm 2, all pairs at once)
 std::vector<uint8_t> backward_chain_marks(const Graph& g, const std::vector<int>& objs, const std::vector<int>& wrts);
 
+// in-place structures of the pruned forward graph (Sec. 2.4, Algorithm 3): per tensor the ancestor
+// it may be renamed to (itself when it starts a structure), -1 for an unmarked tensor
+std::vector<int> inplace_rename(const Graph& g, const PruneResult& pr);
+
 // both prunes over the two-stage DAG; returns a DRAGON_* code
 int prune_function(const Graph& g, const std::vector<int>& inputs, const std::vector<int>& outputs, PruneResult* out);
 

@@ -263,6 +263,8 @@ bool join_domain(Shape* dom, bool* has_dom, const Shape& s) {
 
 }  // namespace
 
+static size_t share_workspace(Plan* plan, size_t off);
+
 int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs,
                    const std::vector<int>& outputs, int sm_count, Plan* plan) {
   Lowerer L(g, pr, plan);
@@ -500,8 +502,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
   size_t off = 0;
   auto take = [&](size_t bytes) { size_t o = off; off += (bytes + 255) & ~(size_t)255; return o; };
   plan->status_off = take(256);
-  for (auto& m : mems)
-    if (m.where == MEM_WORK && m.live) m.offset = take(m.bytes());
+  off = share_workspace(plan, off);
   for (auto& sg : plan->segs) {
     sg.spill_off = take((size_t)sg.grid * sg.n_spill * kVmTile * sizeof(float));
     sg.colpart_off = take((size_t)sg.n_colacc * sg.grid * sg.cols * sizeof(float));
@@ -511,6 +512,122 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     if (st.kind == ST_SCE_FWD) st.scratch_off = take((size_t)mems[st.mA].shape.d[0] * sizeof(float));
   plan->workspace_bytes = off;
   return DRAGON_OK;
+}
+
+// Memory sharing between the tensors that cross kernels (the purpose of Sec. 2.4, at the granularity of
+// plan steps).  Every workspace tensor lives from the first step that touches it to the last one.
+//  * In place (the paper's in-place structure): the output of an elementwise VM step takes the region
+//    of an input of that step that dies there, when both have the domain's shape and the same element
+//    size and the program reads the input for the last time before it first writes the output, so
+//    every thread overwrites only what it has already read.
+//  * Otherwise a region is handed on once its tensor is dead: regions are taken in step order from
+//    the free list (smallest that fits, the remainder stays free), new space only when none fits.
+static size_t share_workspace(Plan* plan, size_t off) {
+  std::vector<MemRef>& mems = plan->mems;
+  const int n_steps = (int)plan->steps.size();
+  std::vector<std::vector<int>> reads(n_steps), writes(n_steps);
+  auto touch = [&](int si, int m, bool w) {
+    if (m < 0 || mems[m].where != MEM_WORK || !mems[m].live) return;
+    (w ? writes : reads)[si].push_back(m);
+    if (mems[m].first_step < 0) mems[m].first_step = si;
+    mems[m].last_step = si;
+  };
+  // positions of the last load and the first store of every operand of a VM program
+  struct Access { int last_load = -1, first_store = 1 << 30; };
+  std::vector<std::vector<Access>> acc(n_steps);
+  for (int si = 0; si < n_steps; ++si) {
+    const Step& st = plan->steps[si];
+    if (st.kind != ST_VM) {
+      touch(si, st.mA, false); touch(si, st.mB, false);
+      if (st.kind == ST_SCE_BWD) touch(si, st.mD, false);
+      if (st.kind == ST_SCE_FWD) touch(si, st.mD, true);
+      touch(si, st.mC, true);
+      continue;
+    }
+    const VmSegment& sg = plan->segs[st.seg];
+    acc[si].resize(sg.operand_mem.size());
+    for (int i = 0; i < (int)sg.code.size(); ++i) {
+      const uint32_t cs = sg.code[i] & 1023u, arg = sg.code[i] >> 14;
+      if (cs == (uint32_t)vm::P_UCONST) { ++i; continue; }
+      int opd = -1; bool store = false;
+      const uint32_t jg = cs / vm::kJointStride;
+      if (cs == (uint32_t)vm::P_GST || cs == (uint32_t)vm::P_GSTF || cs == (uint32_t)vm::P_GSTFL) { opd = (int)arg; store = true; }
+      else if (cs == (uint32_t)vm::P_GLD || cs == (uint32_t)vm::P_GLDF || (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_GLDR)) opd = (int)arg;
+      else if (cs == (uint32_t)vm::P_GLDA0 || cs == (uint32_t)vm::P_GLDA || cs == (uint32_t)vm::P_LDSW || cs == (uint32_t)vm::P_LDSWA ||
+               cs == (uint32_t)vm::P_GLDA0H || cs == (uint32_t)vm::P_LDSWAH ||
+               (cs < (uint32_t)vm::kFirstPlain && (jg == (uint32_t)vm::J_LDSWR || jg == (uint32_t)vm::J_LDSWAR))) opd = (int)(arg & 63u);
+      else if (cs == (uint32_t)vm::P_ULOAD) opd = (int)(arg >> 9);
+      if (opd < 0 || opd >= (int)acc[si].size()) continue;
+      if (store) acc[si][opd].first_store = std::min(acc[si][opd].first_store, i);
+      else acc[si][opd].last_load = i;
+    }
+    for (size_t i = 0; i < sg.operand_mem.size(); ++i) {
+      if (acc[si][i].last_load >= 0) touch(si, sg.operand_mem[i], false);
+      if (acc[si][i].first_store < (1 << 30)) touch(si, sg.operand_mem[i], true);
+    }
+    for (const FinishJob& j : sg.finish) touch(si, j.mem, true);
+  }
+  std::vector<std::pair<size_t, size_t>> free_list;   // (offset, bytes), 256-byte granules
+  auto round = [](size_t b) { return (b + 255) & ~(size_t)255; };
+  std::vector<char> placed(mems.size(), 0);
+  for (int si = 0; si < n_steps; ++si) {
+    const Step& st = plan->steps[si];
+    // 1. outputs of an elementwise step over inputs that die here
+    std::vector<int> taken;    // inputs whose region was handed to an output
+    if (st.kind == ST_VM) {
+      const VmSegment& sg = plan->segs[st.seg];
+      for (size_t o = 0; o < sg.operand_mem.size(); ++o) {
+        const int y = sg.operand_mem[o];
+        if (mems[y].where != MEM_WORK || !mems[y].live || placed[y] || mems[y].first_step != si) continue;
+        if (acc[si][o].first_store >= (1 << 30) || acc[si][o].last_load >= 0 || sg.operand_kind[o] != (uint32_t)vm::K_FULL) continue;
+        for (size_t i = 0; i < sg.operand_mem.size(); ++i) {
+          const int x = sg.operand_mem[i];
+          if (x == y || mems[x].where != MEM_WORK || !placed[x] || mems[x].last_step != si || sg.operand_kind[i] != (uint32_t)vm::K_FULL) continue;
+          if (std::find(taken.begin(), taken.end(), x) != taken.end()) continue;
+          if (mems[x].bytes() != mems[y].bytes() || mems[x].dtype != mems[y].dtype) continue;
+          if (acc[si][i].first_store < (1 << 30) || acc[si][i].last_load < 0 || acc[si][i].last_load > acc[si][o].first_store) continue;
+          mems[y].offset = mems[x].offset;
+          mems[y].shares_input = 1;
+          placed[y] = 1;
+          taken.push_back(x);
+          break;
+        }
+      }
+    }
+    // 2. everything else that starts here
+    for (int m : writes[si]) {
+      if (placed[m] || mems[m].first_step != si) continue;
+      const size_t need = round(mems[m].bytes());
+      int best = -1;
+      for (int k = 0; k < (int)free_list.size(); ++k)
+        if (free_list[k].second >= need && (best < 0 || free_list[k].second < free_list[best].second)) best = k;
+      if (best >= 0) {
+        mems[m].offset = free_list[best].first;
+        free_list[best].first += need;
+        free_list[best].second -= need;
+        if (free_list[best].second == 0) free_list.erase(free_list.begin() + best);
+      } else {
+        mems[m].offset = off;
+        off += need;
+      }
+      placed[m] = 1;
+    }
+    // 3. what dies here is free from the next step on (unless an output took it over)
+    for (int pass = 0; pass < 2; ++pass)
+      for (int m : (pass ? writes[si] : reads[si])) {
+        if (mems[m].last_step != si || !placed[m] || std::find(taken.begin(), taken.end(), m) != taken.end()) continue;
+        bool listed = false;
+        for (auto& fr : free_list) listed |= fr.first == mems[m].offset;
+        if (listed) continue;
+        bool inherited = false;   // a region that an in-place output still holds stays taken
+        for (size_t k = 0; k < mems.size(); ++k)
+          inherited |= (int)k != m && placed[k] && mems[k].where == MEM_WORK && mems[k].live && mems[k].offset == mems[m].offset && mems[k].last_step > si;
+        if (!inherited) free_list.emplace_back(mems[m].offset, round(mems[m].bytes()));
+      }
+  }
+  for (auto& m : mems)     // a live workspace tensor that no step touches keeps a region of its own
+    if (m.where == MEM_WORK && m.live && m.first_step < 0) { m.offset = off; off += round(m.bytes()); }
+  return off;
 }
 
 // one mnemonic per instruction word of a segment

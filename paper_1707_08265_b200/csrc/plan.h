@@ -29,6 +29,8 @@ struct MemRef {
   Shape shape;
   size_t offset = 0;     // byte offset inside the workspace (MEM_WORK)
   bool live = false;
+  int first_step = -1, last_step = -1;   // plan steps that touch it first and last (MEM_WORK)
+  int shares_input = 0;  // 1: written in place over an input of its producing step that dies there (Sec. 2.4)
   size_t bytes() const { return (size_t)shape.numel() * (dtype == DRAGON_BF16 ? 2 : 4); }
 };
 
@@ -123,6 +125,7 @@ std::string describe_plan(const Plan& p);
 struct dragon_function {
   dragon::PruneResult prune;
   dragon::Plan plan;
+  std::vector<int> rename;   // Algorithm 3 on the pruned graph (per tensor id)
   int n_tensors = 0, n_in = 0, n_out = 0;
   void* workspace = nullptr;
   size_t workspace_bytes = 0;

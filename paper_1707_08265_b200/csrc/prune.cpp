@@ -1,5 +1,6 @@
 // Forward prune (Algorithm 1) and backward prune (Algorithm 2) over the two-stage DAG of
 // Sec. 2.3, iterative (explicit stacks) so that graph depth is not limited by the call stack.
+#include <algorithm>
 #include <cstdarg>
 #include <cstdio>
 
@@ -169,6 +170,36 @@ int prune_function(const Graph& g, const std::vector<int>& inputs, const std::ve
       return DRAGON_ERR_MISSING_INPUT;
     }
   return DRAGON_OK;
+}
+
+// Algorithm 3 (Sec. 2.4).  A node with exactly one child hands its memory on to that child, so a
+// path of such nodes is one in-place structure named after its first node.  Nodes are taken in
+// creation order; from each node that has no name yet the walk follows only-children until it
+// meets a node with several (or no) children, or one that already has a name: every node is named
+// once, O(n + e).  Only marked tensors and kept forward operators take part (renaming comes after
+// the prunes: it would make the graph cyclic).
+std::vector<int> inplace_rename(const Graph& g, const PruneResult& pr) {
+  const int n = (int)g.tensors.size();
+  std::vector<std::vector<int>> child(n);
+  for (int k : pr.fwd_ops) {
+    const OpInfo& op = g.ops[k];
+    for (int i : op.in) {
+      if (!pr.marked[i]) continue;
+      for (int o : op.out)
+        if (pr.marked[o] && std::find(child[i].begin(), child[i].end(), o) == child[i].end()) child[i].push_back(o);
+    }
+  }
+  std::vector<int> rd(n, -1);
+  for (int start = 0; start < n; ++start) {
+    if (!pr.marked[start]) continue;
+    int x = start;
+    while (rd[x] < 0) {
+      rd[x] = start;
+      if (child[x].size() != 1) break;
+      x = child[x][0];
+    }
+  }
+  return rd;
 }
 
 }  // namespace dragon
