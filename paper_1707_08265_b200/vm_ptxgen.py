@@ -232,18 +232,48 @@ class Kernel:
             self.e("mov.b64 %s, %s;" % (dst[i], src[i]))
 
     # ---- elementary functions (csrc/vm_math.h, operation by operation) -----------------------
-    def reduce_pio2(self, x):
-        """x: packed pair -> (r packed, kb packed); the low bits of kb's lanes are the quadrant"""
-        lo, hi = self.unpack(x)
-        g = []
-        for s in (lo, hi):   # beyond 6.5e6 (and for inf/NaN) the argument becomes x - x: 0, or NaN
-            a, z, q, pr = self.f(), self.f(), self.f(), self.p()
-            self.e("abs.f32 %s, %s;" % (a, s))
-            self.e("setp.le.f32 %s, %s, %s;" % (pr, a, fc(6.5e6)))
-            self.e("sub.f32 %s, %s, %s;" % (z, s, s))
-            self.e("selp.f32 %s, %s, %s, %s;" % (q, s, z, pr))
-            g.append(q)
-        xg = self.pack(g[0], g[1])
+    def guard_range(self, xs):
+        """Copies of the packed pairs xs in which, when any lane of this thread lies beyond 6.5e6
+        in magnitude (or is inf/NaN), each such lane is replaced by x - x (0, or NaN): the
+        Cody-Waite reduction below is only good up to there.  The common case is one 3-input
+        maximum per two or three lanes and a branch that is not taken."""
+        out = [self.rd() for _ in xs]
+        lanes = []
+        for x, o in zip(xs, out):
+            self.e("mov.b64 %s, %s;" % (o, x))
+            for s in self.unpack(x):
+                a = self.f()
+                self.e("abs.f32 %s, %s;" % (a, s))
+                lanes.append(a)
+        m = lanes[0]
+        rest = lanes[1:]
+        while rest:
+            d = self.f()
+            if len(rest) >= 2:
+                self.e("max.NaN.f32 %s, %s, %s, %s;" % (d, m, rest[0], rest[1]))
+                rest = rest[2:]
+            else:
+                self.e("max.NaN.f32 %s, %s, %s;" % (d, m, rest[0]))
+                rest = rest[1:]
+            m = d
+        ok, done = self.p(), self.newlabel("rng")
+        self.e("setp.le.f32 %s, %s, %s;" % (ok, m, fc(6.5e6)))
+        self.e("@%s bra %s;" % (ok, done))
+        for x, o in zip(xs, out):
+            g = []
+            for s in self.unpack(x):
+                a, z, q, pr = self.f(), self.f(), self.f(), self.p()
+                self.e("abs.f32 %s, %s;" % (a, s))
+                self.e("setp.le.f32 %s, %s, %s;" % (pr, a, fc(6.5e6)))
+                self.e("sub.f32 %s, %s, %s;" % (z, s, s))
+                self.e("selp.f32 %s, %s, %s, %s;" % (q, s, z, pr))
+                g.append(q)
+            self.pack(g[0], g[1], o)
+        self.label(done)
+        return out
+
+    def reduce_pio2(self, xg):
+        """xg: packed pair within range -> (r packed, kb packed); the low bits of kb's lanes are the quadrant"""
         big = 12582912.0
         kb = self.fma2(xg, self.K(0.636619772367581343), self.K(big))
         k = self.add2(kb, self.K(-big))
@@ -264,31 +294,30 @@ class Kernel:
 
     def sincos(self, xs, want_sin=True, want_cos=True):
         S, C = [], []
-        for x in xs:
+        for x in self.guard_range(xs):
             r, kb = self.reduce_pio2(x)
             z = self.mul2(r, r)
-            ps, pc = self.unpack(self.sin_poly(r, z)), self.unpack(self.cos_poly(z))
+            sp = self.sin_poly(r, z)
+            ps, pc = self.unpack(sp), self.unpack(self.cos_poly(z))
+            # quadrant q = k mod 4: sin = (q0 ? pc : ps) * (-1)^q1, cos = (q0 ? -ps : pc) * (-1)^q1
+            nps = self.unpack(self.mul2(sp, self.K(-1.0))) if want_cos else None
             q = [self.r(), self.r()]
             self.e("mov.b64 {%s, %s}, %s;" % (q[0], q[1], kb))
             so, co = [], []
             for j in range(2):
-                b, pr = self.r(), self.p()
+                b, u, pr = self.r(), self.r(), self.p()
                 self.e("and.b32 %s, %s, 1;" % (b, q[j]))
                 self.e("setp.ne.u32 %s, %s, 0;" % (pr, b))
+                self.e("shl.b32 %s, %s, 30;" % (u, q[j]))
                 if want_sin:
-                    s, u = self.f(), self.r()
+                    s = self.f()
                     self.e("selp.f32 %s, %s, %s, %s;" % (s, pc[j], ps[j], pr))
-                    self.e("shl.b32 %s, %s, 30;" % (u, q[j]))
-                    self.e("and.b32 %s, %s, 0x80000000;" % (u, u))
-                    self.e("xor.b32 %s, %s, %s;" % (s, s, u))
+                    self.e("lop3.b32 %s, %s, %s, 0x80000000, 0x78;" % (s, s, u))   # s ^ (u & signbit)
                     so.append(s)
                 if want_cos:
-                    c, v = self.f(), self.r()
-                    self.e("selp.f32 %s, %s, %s, %s;" % (c, ps[j], pc[j], pr))
-                    self.e("add.u32 %s, %s, 1;" % (v, q[j]))
-                    self.e("shl.b32 %s, %s, 30;" % (v, v))
-                    self.e("and.b32 %s, %s, 0x80000000;" % (v, v))
-                    self.e("xor.b32 %s, %s, %s;" % (c, c, v))
+                    c = self.f()
+                    self.e("selp.f32 %s, %s, %s, %s;" % (c, nps[j], pc[j], pr))
+                    self.e("lop3.b32 %s, %s, %s, 0x80000000, 0x78;" % (c, c, u))
                     co.append(c)
             if want_sin:
                 S.append(self.pack(so[0], so[1]))

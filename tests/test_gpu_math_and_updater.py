@@ -65,3 +65,28 @@ def test_updater_graph(kind, shape):
         check(gv, rv, TOL32, kind)
     if kind == "sgd":                              # and against the formula written out
         assert np.allclose(got[0], W.astype(np.float64) - float(lr) * grad.astype(np.float64), rtol=0, atol=2e-6)
+
+
+def test_sine_beyond_the_reduction_range_leaves_its_neighbours_alone():
+    """Arguments beyond 6.5e6 in magnitude evaluate as sin(0), cos(0); inf and NaN give NaN; the
+    other elements of the same thread (and every other thread) are those of the oracle."""
+    n = 2 * 4096 + 100
+    x = np.random.default_rng(3).standard_normal(n).astype(np.float32)
+    odd = {5: 7.0e6, 6: -1.0e30, 2049: np.inf, 4096 + 17: -np.inf, 4096 + 2048 + 3: np.nan, n - 1: 3.0e8}
+    for k, v in odd.items():
+        x[k] = v
+    gd = wl.GraphDesc()
+    xi = gd.tensor("x", [n])
+    out = gd.op("Sin", [xi], "out")
+    grads = gd.grad([out], [xi])
+    (s, c), _ = run_gpu(gd.desc, [xi], [out] + grads, [x])
+    keep = np.ones(n, bool)
+    keep[list(odd)] = False
+    xd = x.astype(np.float64)
+    check(s[keep], np.sin(xd[keep]), TOL32, "sin")
+    check(c[keep], np.cos(xd[keep]), TOL32, "cos")
+    for k, v in odd.items():
+        if np.isfinite(v):
+            assert s[k] == 0.0 and c[k] == 1.0, (k, s[k], c[k])
+        else:
+            assert np.isnan(s[k]) and np.isnan(c[k]), (k, s[k], c[k])
