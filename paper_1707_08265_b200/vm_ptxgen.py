@@ -96,12 +96,10 @@ class Kernel:
     def fd(self): return self.t("fd")
 
     def K(self, x, y=None):
-        """packed constant {x, y} (y defaults to x) loaded from the constant table"""
+        """packed constant {x, y} (y defaults to x), an immediate the assembler places as it sees fit"""
         w = f32bits(x) | (f32bits(x if y is None else y) << 32)
-        if w not in self.kt:
-            self.kt.append(w)
         d = self.rd()
-        self.e("ld.const.b64 %s, [KT_%s+%d];" % (d, self.name, 8 * self.kt.index(w)))
+        self.e("mov.b64 %s, 0x%016X;" % (d, w))
         return d
 
     # ---- packed helpers --------------------------------------------------------------------
