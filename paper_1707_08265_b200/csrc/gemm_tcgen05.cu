@@ -128,6 +128,10 @@ struct GemmArgs {
   int M, N, K;
   int tiles_m, tiles_n;
   int* status;
+  // epilogue: C = act(acc + bias[col]); bias is a row vector of N elements (null: none)
+  const void* bias;
+  int bias_dtype;
+  int relu;
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -256,6 +260,47 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         tmem_ld32(tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(buf * kTileN + c), v);
         asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
         const int col0 = tn * kTileN + c;
+        if (g.bias != nullptr && col0 < g.N) {
+          // every lane of the warp reads the same 32 bias values (broadcast loads)
+          if (col0 + 32 <= g.N && (g.N & 7) == 0 && (reinterpret_cast<uintptr_t>(g.bias) & 15) == 0) {
+            if (g.bias_dtype == DRAGON_F32) {
+              const float4* b4 = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(g.bias) + col0);
+#pragma unroll
+              for (int j = 0; j < 8; ++j) {
+                const float4 b = __ldg(b4 + j);
+                v[4 * j] = __float_as_uint(__uint_as_float(v[4 * j]) + b.x);
+                v[4 * j + 1] = __float_as_uint(__uint_as_float(v[4 * j + 1]) + b.y);
+                v[4 * j + 2] = __float_as_uint(__uint_as_float(v[4 * j + 2]) + b.z);
+                v[4 * j + 3] = __float_as_uint(__uint_as_float(v[4 * j + 3]) + b.w);
+              }
+            } else {
+              const uint4* b8 = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(g.bias) + col0);
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint4 b = __ldg(b8 + j);
+                const uint32_t w[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  v[8 * j + 2 * k] = __float_as_uint(__uint_as_float(v[8 * j + 2 * k]) + __uint_as_float(w[k] << 16));
+                  v[8 * j + 2 * k + 1] = __float_as_uint(__uint_as_float(v[8 * j + 2 * k + 1]) + __uint_as_float(w[k] & 0xffff0000u));
+                }
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < g.N) {
+                const float b = g.bias_dtype == DRAGON_F32
+                                    ? __ldg(reinterpret_cast<const float*>(g.bias) + col0 + j)
+                                    : __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(g.bias) + col0 + j) << 16);
+                v[j] = __float_as_uint(__uint_as_float(v[j]) + b);
+              }
+          }
+        }
+        if (g.relu) {
+#pragma unroll
+          for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.f));
+        }
         if (row < g.M && col0 < g.N) {
           if (g.c_dtype == DRAGON_F32) {
             float* out = reinterpret_cast<float*>(g.C) + (size_t)row * g.N + col0;
@@ -337,8 +382,10 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_ro
 
 // C[M,N] = opA * opB^T with K the contraction length.  a_mn / b_mn: the operand is given as the
 // row-major matrix [K, M] (resp. [K, N]) instead of [M, K] (resp. [N, K]).
+// bias (may be null): row vector of N elements of type bias_dtype (fp32 or bf16), added to every
+// row of the product; relu: max(., 0) applied after it; both before the rounding to C's type.
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
-                     cudaStream_t st) {
+                     cudaStream_t st, const void* bias, int bias_dtype, bool relu) {
   const int a_inner = a_mn ? M : K, b_inner = b_mn ? N : K;
   if (M <= 0 || N <= 0 || K <= 0 || (a_inner & 7) || (b_inner & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
     set_error("InnerProduct: the contiguous extent of every operand must be a multiple of 8 and all pointers 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
@@ -356,7 +403,7 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
   cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
   if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
   const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
-  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status};
+  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0};
   static int sm_count = 0;
   if (!sm_count) {
     int dev = 0;

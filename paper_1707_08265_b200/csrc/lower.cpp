@@ -458,6 +458,67 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     }
   }
 
+  // A segment that only adds a row vector to the product of an InnerProduct, optionally clamps
+  // it at zero and rounds it, and stores the result, runs in the epilogue of that product: the
+  // fp32 product then never reaches memory.
+  for (size_t s = 0; s < seg_items.size(); ++s) {
+    std::vector<int> body;
+    for (int i : seg_items[s])
+      if (items[i].live && items[i].opc != M_WIDEN) body.push_back(i);
+    if (body.size() < 2 || body.size() > 4) continue;
+    auto root = [&](int v) {   // through the widenings to the value they show
+      for (bool again = true; again && v >= 0 && vals[v].kind == VK_OP;) {
+        again = false;
+        for (int i : seg_items[s])
+          if (items[i].opc == M_WIDEN && items[i].dst == v) { v = items[i].a; again = true; break; }
+      }
+      return v;
+    };
+    const Item& add = items[body[0]];
+    const Item& st = items[body.back()];
+    if (add.opc != M_ADD || st.opc != M_STORE) continue;
+    int prod = root(add.a), bias = root(add.b);
+    if (prod < 0 || bias < 0) continue;
+    if (!(vals[prod].kind == VK_MEM && vals[prod].shape.rank == 2)) std::swap(prod, bias);
+    if (vals[prod].kind != VK_MEM || vals[bias].kind != VK_MEM || vals[prod].shape.rank != 2) continue;
+    const int mP = vals[prod].mem, mBias = vals[bias].mem, mOut = st.mem;
+    const Shape& sp = mems[mP].shape;
+    const Shape& sb = mems[mBias].shape;
+    const bool row_vector = (sb.rank == 1 && sb.d[0] == sp.d[1]) || (sb.rank == 2 && sb.d[0] == 1 && sb.d[1] == sp.d[1]);
+    if (mems[mP].where != MEM_WORK || mems[mP].dtype != DRAGON_F32 || !row_vector || !(mems[mOut].shape == sp)) continue;
+    if (mems[mBias].dtype != DRAGON_F32 && mems[mBias].dtype != DRAGON_BF16) continue;
+    bool relu = false, rounded = false, chain = true;
+    int last = add.dst;
+    for (size_t k = 1; k + 1 < body.size() && chain; ++k) {
+      const Item& u = items[body[k]];
+      if (u.a != last) chain = false;
+      else if (u.opc == M_RELU && !relu && !rounded) relu = true;
+      else if (u.opc == M_RBF16 && !rounded) rounded = true;
+      else chain = false;
+      last = u.dst;
+    }
+    if (!chain || st.a != last) continue;
+    if (rounded != (mems[mOut].dtype == DRAGON_BF16) || (!rounded && mems[mOut].dtype != DRAGON_F32)) continue;
+    int producer = -1, readers = 0;
+    for (int i = 0; i < (int)items.size(); ++i) {
+      const Item& it = items[i];
+      if (!it.live) continue;
+      if (it.kind == IT_GEMM && it.mC == mP) producer = i;
+      if (it.kind != IT_MOP) { readers += (it.mA == mP) + (it.mB == mP) + (it.mD == mP); continue; }
+      if (it.opc == M_WIDEN) continue;
+      for (int v : {it.a, it.b})
+        if (v >= 0 && root(v) >= 0 && vals[root(v)].kind == VK_MEM && vals[root(v)].mem == mP) ++readers;
+    }
+    if (producer < 0 || producer > body[0] || readers != 1 || items[producer].mD >= 0) continue;
+    items[producer].mC = mOut;
+    items[producer].mD = mBias;
+    items[producer].relu = relu;
+    mems[mBias].live = true;
+    mems[mP].live = false;
+    for (int i : seg_items[s]) items[i].live = false;
+    seg_items[s].clear();
+  }
+
   // steps in execution order
   std::vector<int> seg_step(seg_items.size(), -1);
   plan->segs.resize(seg_items.size());
@@ -477,6 +538,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     st.kind = it.kind == IT_GEMM ? ST_GEMM : it.kind == IT_TRANSPOSE ? ST_TRANSPOSE : it.kind == IT_SCE_FWD ? ST_SCE_FWD
               : it.kind == IT_SCE_BWD ? ST_SCE_BWD : ST_COPY;
     st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
+    st.relu = it.relu;
     if (it.kind == IT_SCE_FWD) {
       // the gradient with respect to the same logits, scaled by a constant, comes out of the same
       // pass: the step then carries the gradient tensor in mD
@@ -494,6 +556,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     plan->steps.push_back(st);
   }
   for (size_t s = 0; s < seg_items.size(); ++s) {
+    if (seg_items[s].empty()) continue;   // ran in a product's epilogue
     int rc = codegen_segment(items, seg_items[s], vals, mems, sm_count, &plan->segs[s]);
     if (rc) return rc;
   }
@@ -676,9 +739,9 @@ std::string describe_plan(const Plan& p) {
         break;
       }
       case ST_GEMM:
-        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
-                 (long long)p.mems[st.mA].shape.d[st.tA ? 0 : 1], st.tA ? " A^T" : "", st.tB ? " B^T" : "",
-                 p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
+        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s%s%s -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
+                 (long long)p.mems[st.mA].shape.d[st.tA ? 0 : 1], st.tA ? " A^T" : "", st.tB ? " B^T" : "", st.mD >= 0 ? " +bias" : "",
+                 st.relu ? " relu" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
         break;
       case ST_TRANSPOSE:
         snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);

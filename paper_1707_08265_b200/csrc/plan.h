@@ -58,11 +58,13 @@ struct Item {
   int kind = IT_MOP;
   // IT_MOP
   int opc = 0, a = -1, b = -1, dst = -1, mem = -1;
-  // heavy items: memory operands.  GEMM: C = A * B^T; TRANSPOSE: C = A^T;
+  // heavy items: memory operands.  GEMM: C = act(A * B^T + D) with D an optional row vector and
+  // act the identity or max(., 0); TRANSPOSE: C = A^T;
   // SCE: A = logits, B = labels, C = out, D = scalar dL (gradient)
   int mA = -1, mB = -1, mC = -1, mD = -1;
   float scale = 1.f;                       // SCE_BWD: immediate dL when mD < 0
   bool tA = false, tB = false;             // GEMM: operand given transposed ([K, M] / [K, N] row-major)
+  bool relu = false;                       // GEMM: max(., 0) in the epilogue
   bool live = false;
   int segment = -1;
 };
@@ -99,6 +101,7 @@ struct Step {
   int mA = -1, mB = -1, mC = -1, mD = -1;
   float scale = 1.f;
   bool tA = false, tB = false;
+  bool relu = false;                     // ST_GEMM: epilogue max(., 0); its bias row vector is mD
   size_t scratch_off = 0;                // SCE_FWD: per-row losses
 };
 

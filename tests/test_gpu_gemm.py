@@ -95,3 +95,41 @@ def test_unsupported_contraction_length_is_an_error_not_a_fault():
     with pytest.raises(B.DragonError) as e:
         f.run_torch([to_dev(np.zeros((16, 12), np.float32), "bf16"), to_dev(np.zeros((8, 12), np.float32), "bf16")], [out])
     assert e.value.code == B.ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("m,n,k,bias_dt,relu,out_dt", [
+    (128, 128, 64, "f32", False, "f32"), (256, 384, 448, "bf16", True, "bf16"), (200, 136, 72, "bf16", True, "f32"),
+    (300, 520, 1000, "f32", True, "bf16"), (70, 40, 72, "bf16", False, "bf16"), (1024, 1024, 512, "bf16", True, "bf16")])
+def test_bias_and_relu_run_in_the_epilogue_of_the_product(m, n, k, bias_dt, relu, out_dt):
+    """Y = [ReLU](X W^T + b): one launch, the fp32 product never written; ragged tiles in m and n."""
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n], bias_dt)
+    Z = gd.op("InnerProduct", [X, W], "Z", [m, n], "f32")
+    last_dt = out_dt if not relu else "f32"
+    Y = gd.op("BiasAdd", [Z, b], "A", [m, n], last_dt)
+    if relu:
+        Y = gd.op("ReLU", [Y], "Y", out_dtype=out_dt)
+    rng = np.random.default_rng(m * 3 + n)
+    x = bf16able(rng.standard_normal((m, k))); w = bf16able(rng.standard_normal((n, k)) / np.sqrt(k))
+    bv = bf16able(rng.standard_normal(n))
+    (got,), f = run_gpu(gd.desc, [X, W, b], [Y], [x, w, bv])
+    assert f.num_launches() == 1 and "+bias" in f.describe() and ("relu" in f.describe()) == relu, f.describe()
+    (ref,) = interp.run_function(gd.desc, [X, W, b], [Y], [x, w, bv])
+    check(got, ref, TOLBF if out_dt == "bf16" else 2e-5, "Y")
+    if relu:
+        assert (got >= 0).all() and (got == 0).any() and (got > 0).any()
+
+
+def test_product_that_is_also_fetched_keeps_its_own_launch():
+    m, n, k = 128, 128, 64
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n], "f32")
+    Z = gd.op("InnerProduct", [X, W], "Z", [m, n], "f32")
+    Y = gd.op("BiasAdd", [Z, b], "Y", [m, n], "f32")
+    rng = np.random.default_rng(9)
+    feeds = [bf16able(rng.standard_normal((m, k))), bf16able(rng.standard_normal((n, k))), bf16able(rng.standard_normal(n))]
+    got, f = run_gpu(gd.desc, [X, W, b], [Y, Z], feeds)
+    assert "+bias" not in f.describe()
+    ref = interp.run_function(gd.desc, [X, W, b], [Y, Z], feeds)
+    check(got[0], ref[0], 2e-5, "Y")
+    check(got[1], ref[1], 2e-5, "Z")

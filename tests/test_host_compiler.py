@@ -172,3 +172,18 @@ def test_limits_are_reported_not_faulted():
     # fetching the same tensor twice is refused
     with pytest.raises(B.DragonError):
         g2.function([x2], [y2, y2])
+
+
+def test_bias_relu_after_a_product_fuse_into_its_epilogue():
+    """Lowering: a segment that only adds a row vector to an InnerProduct's result, clamps and rounds
+    it, becomes the product's epilogue; a second reader of the product prevents it."""
+    from paper_1707_08265_b200 import workloads as wl
+    g, ids = wl.mlp(256, 128, 192, 64)
+    inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
+    f = B.Graph.from_desc(g.desc).function(inputs, [ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")])
+    text = f.describe()
+    assert text.count("+bias") == 2 and text.count("relu") == 1, text
+    assert "gld" not in text.split("softmax")[0], text          # no elementwise launch before the loss
+    # the pre-activation fetched as well: the first product keeps a launch of its own
+    f2 = B.Graph.from_desc(g.desc).function(inputs, [ids["loss"], ids["z1"]])
+    assert f2.describe().count("+bias") == 1, f2.describe()
