@@ -634,9 +634,18 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
     else rc = DRAGON_ERR_UNSUPPORTED;
   }
   if (rc != DRAGON_OK) {
-    Gen gen(items, idx, vals, mems, seg, kVmRegsWide, kVmSmemSlots);
-    rc = gen.run();
-    if (rc) return rc;
+    // as many shared-memory slots as fit beside the instruction stream (whose length depends a
+    // little on the slot count: second attempt with the count that fits the first one's stream)
+    auto smem_of = [](const VmSegment& g, int slots) {
+      return (size_t)((g.code.size() + 3) & ~(size_t)3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)slots * kVmTile * 4;
+    };
+    for (int slots = kVmSmemSlots;; slots = kVmSmemSlotsLongCode) {
+      VmSegment trial = *seg;
+      Gen gen(items, idx, vals, mems, &trial, kVmRegsWide, slots);
+      rc = gen.run();
+      if (rc) return rc;
+      if (smem_of(trial, trial.n_smem) <= (size_t)227 * 1024 || slots == kVmSmemSlotsLongCode) { *seg = trial; break; }
+    }
     seg->dense = false;
   }
   long long tiles = seg->row_mode ? seg->n : (seg->n + kVmTile - 1) / kVmTile;

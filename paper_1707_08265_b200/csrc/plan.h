@@ -15,7 +15,8 @@ constexpr int kVmThreads = DRAGON_VM_THREADS;
 constexpr int kVmVec = DRAGON_VM_VEC;
 constexpr int kVmTile = kVmThreads * kVmVec;  // 4096
 constexpr int kVmCodeMaxWords = 8 * 1024;     // instruction stream held in shared memory (8 bytes per word once decoded)
-constexpr int kVmSmemSlots = 9;               // V-wide shared-memory slots per thread (wide build: one CTA per SM)
+constexpr int kVmSmemSlots = 13;              // V-wide shared-memory slots per thread at most (wide build: one CTA per SM, 227 KB)
+constexpr int kVmSmemSlotsLongCode = 9;       // the same when the instruction stream is too long for that many
 constexpr int kVmSmemSlotsDense = 6;          // the same for the dense build (two CTAs share the SM's shared memory)
 constexpr int kDefaultSmCount = 148;
 constexpr int kHostChunks = 16;               // dragon_run_host pipelines a large elementwise function in this many chunks
