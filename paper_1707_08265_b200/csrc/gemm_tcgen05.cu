@@ -132,6 +132,8 @@ struct GemmArgs {
   const void* bias;
   int bias_dtype;
   int relu;
+  // then multiplied by step(mask[row, col]) (1 where the bf16 mask element is > 0, else 0); null: none
+  const unsigned short* mask;
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -301,6 +303,25 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
 #pragma unroll
           for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(fmaxf(__uint_as_float(v[j]), 0.f));
         }
+        if (g.mask != nullptr && row < g.M && col0 < g.N) {
+          const unsigned short* mrow = g.mask + (size_t)row * g.N + col0;
+          if ((g.N & 7) == 0 && col0 + 32 <= g.N && (reinterpret_cast<uintptr_t>(g.mask) & 15) == 0) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 m = *reinterpret_cast<const uint4*>(mrow + 8 * j);
+              const uint32_t w[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                v[8 * j + 2 * k] = __float_as_uint(__uint_as_float(v[8 * j + 2 * k]) * (__uint_as_float(w[k] << 16) > 0.f ? 1.f : 0.f));
+                v[8 * j + 2 * k + 1] = __float_as_uint(__uint_as_float(v[8 * j + 2 * k + 1]) * (__uint_as_float(w[k] & 0xffff0000u) > 0.f ? 1.f : 0.f));
+              }
+            }
+          } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+              if (col0 + j < g.N) v[j] = __float_as_uint(__uint_as_float(v[j]) * (__uint_as_float((uint32_t)mrow[j] << 16) > 0.f ? 1.f : 0.f));
+          }
+        }
         if (row < g.M && col0 < g.N) {
           if (g.c_dtype == DRAGON_F32) {
             float* out = reinterpret_cast<float*>(g.C) + (size_t)row * g.N + col0;
@@ -383,9 +404,10 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_ro
 // C[M,N] = opA * opB^T with K the contraction length.  a_mn / b_mn: the operand is given as the
 // row-major matrix [K, M] (resp. [K, N]) instead of [M, K] (resp. [N, K]).
 // bias (may be null): row vector of N elements of type bias_dtype (fp32 or bf16), added to every
-// row of the product; relu: max(., 0) applied after it; both before the rounding to C's type.
+// row of the product; relu: max(., 0) applied after it; mask (may be null): bf16 [M, N], the result is
+// multiplied by 1 where the mask element is > 0 and by 0 elsewhere; all before the rounding to C's type.
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
-                     cudaStream_t st, const void* bias, int bias_dtype, bool relu) {
+                     cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask) {
   const int a_inner = a_mn ? M : K, b_inner = b_mn ? N : K;
   if (M <= 0 || N <= 0 || K <= 0 || (a_inner & 7) || (b_inner & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
     set_error("InnerProduct: the contiguous extent of every operand must be a multiple of 8 and all pointers 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
@@ -403,7 +425,7 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
   cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
   if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
   const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
-  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0};
+  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0, reinterpret_cast<const unsigned short*>(mask)};
   static int sm_count = 0;
   if (!sm_count) {
     int dev = 0;

@@ -387,7 +387,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     } else {
       it.live = mems[it.mC].live;
       if (it.live)
-        for (int m : {it.mA, it.mB, it.mD})
+        for (int m : {it.mA, it.mB, it.mD, it.mE})
           if (m >= 0) mems[m].live = true;
     }
   }
@@ -458,6 +458,24 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     }
   }
 
+  // a segment runs where its first item stands (items appended later for values that cross
+  // segments belong to the segment of the value's definition)
+  auto runs_at = [&](int i) {
+    const Item& it = items[i];
+    if (it.kind != IT_MOP || it.segment < 0 || seg_items[it.segment].empty()) return i;
+    return *std::min_element(seg_items[it.segment].begin(), seg_items[it.segment].end());
+  };
+  // position of the last live item that writes memory m (-1: a feed, or never written)
+  auto last_writer = [&](int m) {
+    int w = -1;
+    for (int i = 0; i < (int)items.size(); ++i) {
+      const Item& it = items[i];
+      if (!it.live) continue;
+      if (it.kind != IT_MOP) { if (it.mC == m || (it.kind == IT_SCE_FWD && it.mD == m)) w = std::max(w, i); }
+      else if ((it.opc == M_STORE || it.opc == M_ACCUM) && it.mem == m) w = std::max(w, runs_at(i));
+    }
+    return w;
+  };
   // A segment that only adds a row vector to the product of an InnerProduct, optionally clamps
   // it at zero and rounds it, and stores the result, runs in the epilogue of that product: the
   // fp32 product then never reaches memory.
@@ -509,7 +527,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
       for (int v : {it.a, it.b})
         if (v >= 0 && root(v) >= 0 && vals[root(v)].kind == VK_MEM && vals[root(v)].mem == mP) ++readers;
     }
-    if (producer < 0 || producer > body[0] || readers != 1 || items[producer].mD >= 0) continue;
+    if (producer < 0 || producer > runs_at(body[0]) || readers != 1 || items[producer].mD >= 0 || last_writer(mBias) > producer) continue;
     items[producer].mC = mOut;
     items[producer].mD = mBias;
     items[producer].relu = relu;
@@ -517,6 +535,67 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     mems[mP].live = false;
     for (int i : seg_items[s]) items[i].live = false;
     seg_items[s].clear();
+  }
+
+  // The backward of ReLU behind a product: a segment that multiplies the product by step(h), h a
+  // bf16 tensor of the same shape already in memory, stores that (and perhaps sums it as well),
+  // leaves the multiplication to the product's epilogue; what remains of the segment reads the
+  // stored result.
+  for (size_t s = 0; s < seg_items.size(); ++s) {
+    std::vector<int> body;
+    for (int i : seg_items[s])
+      if (items[i].live && items[i].opc != M_WIDEN) body.push_back(i);
+    int i_step = -1, i_mul = -1, i_store = -1, n_accum = 0, n_other = 0;
+    for (int i : body) {
+      const int opc = items[i].opc;
+      if (opc == M_STEP && i_step < 0) i_step = i;
+      else if (opc == M_MUL && i_mul < 0) i_mul = i;
+      else if (opc == M_STORE && i_store < 0) i_store = i;
+      else if (opc == M_ACCUM) ++n_accum;
+      else ++n_other;
+    }
+    if (i_step < 0 || i_mul < 0 || i_store < 0 || n_other) continue;
+    const Item& stp = items[i_step];
+    const Item& mul = items[i_mul];
+    if (vals[stp.a].kind != VK_MEM) continue;
+    int prod = mul.a == stp.dst ? mul.b : mul.b == stp.dst ? mul.a : -1;
+    if (prod < 0 || vals[prod].kind != VK_MEM) continue;
+    const int mH = vals[stp.a].mem, mP = vals[prod].mem, mOut = items[i_store].mem;
+    bool uses_ok = items[i_store].a == mul.dst;
+    for (int i : body)
+      if (items[i].opc == M_ACCUM) uses_ok &= items[i].a == mul.dst;
+    if (!uses_ok) continue;
+    if (mems[mP].where != MEM_WORK || mems[mP].shape.rank != 2 || !(mems[mH].shape == mems[mP].shape) || !(mems[mOut].shape == mems[mP].shape)) continue;
+    if (mems[mH].dtype != DRAGON_BF16 || mems[mP].dtype != mems[mOut].dtype) continue;
+    int producer = -1, readers = 0;
+    for (int i = 0; i < (int)items.size(); ++i) {
+      const Item& it = items[i];
+      if (!it.live) continue;
+      if (it.kind == IT_GEMM && it.mC == mP) producer = i;
+      if (it.kind != IT_MOP) {
+        readers += (it.mA == mP) + (it.mB == mP) + (it.mD == mP) + (it.mE == mP);
+        continue;
+      }
+      if (it.opc == M_WIDEN) continue;
+      for (int v : {it.a, it.b})
+        if (v >= 0 && vals[v].kind == VK_MEM && vals[v].mem == mP) ++readers;
+    }
+    if (producer < 0 || producer > runs_at(body[0]) || readers != 1 || items[producer].mE >= 0 || last_writer(mH) > producer) continue;
+    items[producer].mC = mOut;
+    items[producer].mE = mH;
+    mems[mH].live = true;
+    mems[mP].live = false;
+    items[i_step].live = items[i_mul].live = items[i_store].live = false;
+    Value nv; nv.kind = VK_MEM; nv.shape = mems[mOut].shape; nv.mem = mOut;
+    vals.push_back(nv);
+    std::vector<int> rest;
+    for (int i : seg_items[s]) {
+      if (!items[i].live) continue;
+      if (items[i].opc == M_ACCUM) { items[i].a = (int)vals.size() - 1; rest.push_back(i); }
+    }
+    for (int i : seg_items[s])
+      if (items[i].live && items[i].opc != M_ACCUM) items[i].live = false;   // widenings of what is gone
+    seg_items[s] = rest;
   }
 
   // steps in execution order
@@ -537,7 +616,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     Step st;
     st.kind = it.kind == IT_GEMM ? ST_GEMM : it.kind == IT_TRANSPOSE ? ST_TRANSPOSE : it.kind == IT_SCE_FWD ? ST_SCE_FWD
               : it.kind == IT_SCE_BWD ? ST_SCE_BWD : ST_COPY;
-    st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
+    st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.mE = it.mE; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
     st.relu = it.relu;
     if (it.kind == IT_SCE_FWD) {
       // the gradient with respect to the same logits, scaled by a constant, comes out of the same
@@ -602,7 +681,8 @@ static size_t share_workspace(Plan* plan, size_t off) {
     const Step& st = plan->steps[si];
     if (st.kind != ST_VM) {
       touch(si, st.mA, false); touch(si, st.mB, false);
-      if (st.kind == ST_SCE_BWD) touch(si, st.mD, false);
+      if (st.kind == ST_SCE_BWD || st.kind == ST_GEMM) touch(si, st.mD, false);
+      if (st.kind == ST_GEMM) touch(si, st.mE, false);
       if (st.kind == ST_SCE_FWD) touch(si, st.mD, true);
       touch(si, st.mC, true);
       continue;
@@ -739,9 +819,9 @@ std::string describe_plan(const Plan& p) {
         break;
       }
       case ST_GEMM:
-        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s%s%s -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
+        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s%s%s%s -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
                  (long long)p.mems[st.mA].shape.d[st.tA ? 0 : 1], st.tA ? " A^T" : "", st.tB ? " B^T" : "", st.mD >= 0 ? " +bias" : "",
-                 st.relu ? " relu" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
+                 st.relu ? " relu" : "", st.mE >= 0 ? " *step" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
         break;
       case ST_TRANSPOSE:
         snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);

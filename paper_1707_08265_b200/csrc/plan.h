@@ -59,10 +59,10 @@ struct Item {
   int kind = IT_MOP;
   // IT_MOP
   int opc = 0, a = -1, b = -1, dst = -1, mem = -1;
-  // heavy items: memory operands.  GEMM: C = act(A * B^T + D) with D an optional row vector and
-  // act the identity or max(., 0); TRANSPOSE: C = A^T;
+  // heavy items: memory operands.  GEMM: C = act(A * B^T + D) * step(E) with D an optional row
+  // vector, act the identity or max(., 0), E an optional bf16 tensor of C's shape; TRANSPOSE: C = A^T;
   // SCE: A = logits, B = labels, C = out, D = scalar dL (gradient)
-  int mA = -1, mB = -1, mC = -1, mD = -1;
+  int mA = -1, mB = -1, mC = -1, mD = -1, mE = -1;
   float scale = 1.f;                       // SCE_BWD: immediate dL when mD < 0
   bool tA = false, tB = false;             // GEMM: operand given transposed ([K, M] / [K, N] row-major)
   bool relu = false;                       // GEMM: max(., 0) in the epilogue
@@ -99,7 +99,7 @@ enum StepKind { ST_VM, ST_GEMM, ST_TRANSPOSE, ST_SCE_FWD, ST_SCE_BWD, ST_COPY };
 struct Step {
   int kind;
   int seg = -1;                          // ST_VM
-  int mA = -1, mB = -1, mC = -1, mD = -1;
+  int mA = -1, mB = -1, mC = -1, mD = -1, mE = -1;   // mE: ST_GEMM epilogue mask (step(E) multiplies the product)
   float scale = 1.f;
   bool tA = false, tB = false;
   bool relu = false;                     // ST_GEMM: epilogue max(., 0); its bias row vector is mD

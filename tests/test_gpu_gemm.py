@@ -133,3 +133,51 @@ def test_product_that_is_also_fetched_keeps_its_own_launch():
     ref = interp.run_function(gd.desc, [X, W, b], [Y, Z], feeds)
     check(got[0], ref[0], 2e-5, "Y")
     check(got[1], ref[1], 2e-5, "Z")
+
+
+@pytest.mark.parametrize("m,n,k", [(128, 256, 128), (200, 136, 72), (70, 40, 1000)])
+def test_relu_backward_runs_in_the_epilogue_of_the_product(m, n, k):
+    """H = ReLU(X W1^T + b) in bf16, Y = H W2^T, objective sum(Y * G): dZ1 = (G W2) * step(H) comes out of
+    the product's epilogue, db = column sums of dZ1, dW1 = dZ1^T X.  Ragged tiles in every extent."""
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W1 = gd.tensor("W1", [n, k], "bf16"); b = gd.tensor("b", [n], "bf16")
+    W2 = gd.tensor("W2", [n, n], "bf16"); G = gd.tensor("G", [m, n], "f32")
+    Z = gd.op("InnerProduct", [X, W1], "Z", [m, n], "f32")
+    A = gd.op("BiasAdd", [Z, b], "A", [m, n], "f32")
+    H = gd.op("ReLU", [A], "H", out_dtype="bf16")
+    Y = gd.op("InnerProduct", [H, W2], "Y", [m, n], "f32")
+    obj = gd.op("Mul", [Y, G], "obj")
+    dW1, db = gd.grad([obj], [W1, b])
+    rng = np.random.default_rng(n + k)
+    feeds = [bf16able(rng.standard_normal((m, k))), bf16able(rng.standard_normal((n, k)) / np.sqrt(k)),
+             bf16able(rng.standard_normal(n) * 0.1), bf16able(rng.standard_normal((n, n)) / np.sqrt(n)),
+             bf16able(rng.standard_normal((m, n)))]
+    ins = [X, W1, b, W2, G]
+    got, f = run_gpu(gd.desc, ins, [dW1, db], feeds)
+    assert "*step" in f.describe() and "step;" not in f.describe(), f.describe()
+    ref = interp.run_function(gd.desc, ins, [dW1, db], feeds)
+    check(got[0], ref[0], TOLBF, "dW1")
+    # dZ1 is kept in bf16 (it is an operand of the next product): db, a sum of m such values, is
+    # compared with the same sum of rounded values, and with the oracle within sqrt(m) roundings
+    (h_ref,) = interp.run_function(gd.desc, ins, [H], feeds)
+    dz = bf16able(feeds[4].astype(np.float64) @ feeds[3].astype(np.float64)) * (h_ref > 0)
+    check(got[1], dz.sum(axis=0), 6e-3, "db against the sum of bf16 values")
+    assert np.all(np.abs(got[1] - ref[1]) <= 4 * np.sqrt(m) * 2.0 ** -9 * (1 + np.abs(ref[1])))
+
+
+@pytest.mark.parametrize("bias_first", [True, False])
+def test_computed_bias_before_or_after_the_product(bias_first):
+    m, n, k = 64, 128, 64
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n], "f32")
+    if bias_first:
+        tb = gd.op("Tanh", [b], "tb")
+    Z = gd.op("InnerProduct", [X, W], "Z", [m, n], "f32")
+    if not bias_first:
+        tb = gd.op("Tanh", [b], "tb")
+    Y = gd.op("BiasAdd", [Z, tb], "Y", [m, n], "f32")
+    rng = np.random.default_rng(4)
+    feeds = [bf16able(rng.standard_normal((m, k))), bf16able(rng.standard_normal((n, k))), rng.standard_normal(n).astype(np.float32)]
+    (got,), f = run_gpu(gd.desc, [X, W, b], [Y], feeds)
+    (ref,) = interp.run_function(gd.desc, [X, W, b], [Y], feeds)
+    check(got, ref, 2e-5, "Y")

@@ -182,8 +182,26 @@ def test_bias_relu_after_a_product_fuse_into_its_epilogue():
     inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
     f = B.Graph.from_desc(g.desc).function(inputs, [ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")])
     text = f.describe()
-    assert text.count("+bias") == 2 and text.count("relu") == 1, text
+    assert text.count("+bias") == 2 and text.count("relu") == 1 and text.count("*step") == 1, text
+    assert " step;" not in text and " mul " not in text, text          # the mask is applied in the product's epilogue
     assert "gld" not in text.split("softmax")[0], text          # no elementwise launch before the loss
     # the pre-activation fetched as well: the first product keeps a launch of its own
     f2 = B.Graph.from_desc(g.desc).function(inputs, [ids["loss"], ids["z1"]])
     assert f2.describe().count("+bias") == 1, f2.describe()
+
+
+@pytest.mark.parametrize("bias_first", [True, False])
+def test_epilogue_fusion_needs_the_bias_in_memory_before_the_product_runs(bias_first):
+    from paper_1707_08265_b200 import workloads as wl
+    m, n, k = 64, 128, 64
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n], "f32")
+    if bias_first:
+        tb = gd.op("Tanh", [b], "tb")
+    Z = gd.op("InnerProduct", [X, W], "Z", [m, n], "f32")
+    if not bias_first:
+        tb = gd.op("Tanh", [b], "tb")
+    Y = gd.op("BiasAdd", [Z, tb], "Y", [m, n], "f32")
+    f = B.Graph.from_desc(gd.desc).function([X, W, b], [Y])
+    text = f.describe()
+    assert ("+bias" in text) == bias_first, text
