@@ -30,30 +30,39 @@ struct FinishParams {
   } job[8];
 };
 
+constexpr int kFinishThreads = 256;
+
 __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
   // launched as a programmatic dependent of the VM kernel: its blocks may be resident before that
   // kernel ends, and wait here until its partial sums are complete and visible
   cudaGridDependencySynchronize();
   const FinishParams::Job& jb = fp.job[blockIdx.y];
+  __shared__ double sh[kFinishThreads];
   if (jb.kind == 0) {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= jb.cols) return;
+    // a block owns 32 columns; its 8 warps each sum every 8th partial row (coalesced 128-byte
+    // reads), then warp 0 adds the 8 slices in order: the same order on every run
+    const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5, c = blockIdx.x * 32 + lane;
     const float* part = reinterpret_cast<const float*>(jb.part);
     double s = 0.0;
-    for (int g = 0; g < jb.grid; ++g) s += (double)part[(size_t)g * jb.cols + c];
-    if (jb.dtype == DRAGON_F32) reinterpret_cast<float*>(jb.out)[c] = (float)s;
-    else reinterpret_cast<unsigned short*>(jb.out)[c] = (unsigned short)vmmath::bf16_bits((float)s);
+    if (c < jb.cols)
+      for (int g = slice; g < jb.grid; g += kFinishThreads / 32) s += (double)part[(size_t)g * jb.cols + c];
+    sh[threadIdx.x] = s;
+    __syncthreads();
+    if (slice == 0 && c < jb.cols) {
+      for (int k = 1; k < kFinishThreads / 32; ++k) s += sh[k * 32 + lane];
+      if (jb.dtype == DRAGON_F32) reinterpret_cast<float*>(jb.out)[c] = (float)s;
+      else reinterpret_cast<unsigned short*>(jb.out)[c] = (unsigned short)vmmath::bf16_bits((float)s);
+    }
   } else if (blockIdx.x == 0) {
     // one block per scalar: strided partial sums, then a tree in shared memory; the order is
     // fixed by the thread count, so the result is the same on every run
-    __shared__ double sh[128];
     const double* part = reinterpret_cast<const double*>(jb.part);
     double s = 0.0;
     for (int c = 0; c < jb.chunks; ++c)
-      for (int g = threadIdx.x; g < jb.grid; g += 128) s += part[(size_t)c * jb.chunk_stride + g];
+      for (int g = threadIdx.x; g < jb.grid; g += kFinishThreads) s += part[(size_t)c * jb.chunk_stride + g];
     sh[threadIdx.x] = s;
     __syncthreads();
-    for (int w = 64; w > 0; w >>= 1) {
+    for (int w = kFinishThreads / 2; w > 0; w >>= 1) {
       if ((int)threadIdx.x < w) sh[threadIdx.x] += sh[threadIdx.x + w];
       __syncthreads();
     }
@@ -118,10 +127,10 @@ cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, 
     if (j.kind == 0) { o.part = ws + sg.colpart_off + (size_t)j.acc * sg.grid * sg.cols * sizeof(float); max_cols = std::max(max_cols, sg.cols); }
     else o.part = ws + sg.scalpart_off + (size_t)j.acc * sg.grid * sizeof(double);
   }
-  dim3 grid((max_cols + 127) / 128, fp.n_jobs);
+  dim3 grid((max_cols + 31) / 32, fp.n_jobs);
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = grid;
-  cfg.blockDim = dim3(128);
+  cfg.blockDim = dim3(vm::kFinishThreads);
   cfg.stream = st;
   cudaLaunchAttribute attr[1];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
