@@ -575,6 +575,23 @@ struct Gen {
       }
     }
     stage_loads();
+    {   // a staged load kept in a register slot followed by an affine map with adjacent uniforms
+      std::vector<uint32_t> out;
+      for (size_t i = 0; i < body.size(); ++i) {
+        const uint32_t w = body[i], cs = w & 1023u, nx = i + 1 < body.size() ? body[i + 1] : 0u;
+        if (cs >= (uint32_t)(J_LDSWAR * kJointStride) && cs < (uint32_t)(J_LDSWAR * kJointStride + nr) && i + 1 < body.size() &&
+            (nx & 1023u) == (uint32_t)P_FMAU) {
+          const uint32_t ui = (nx >> 14) & 511u, uj = nx >> 23, a = w >> 14;
+          if (uj == ui + 1 && ui < 256 && a < 1024) {
+            out.push_back(encode(J_LDSWARF * kJointStride + (int)(cs - J_LDSWAR * kJointStride), 0, a | (ui << 10)));
+            ++i;
+            continue;
+          }
+        }
+        out.push_back(w);
+      }
+      body.swap(out);
+    }
     // 6. epilogue: accumulators leave as per-CTA partial sums
     for (auto& a : accs) {
       const Item& it = items[idx[a.first]];
@@ -597,8 +614,17 @@ struct Gen {
     seg->code.insert(seg->code.end(), preamble.begin(), preamble.end());
     seg->loop_start = (int)seg->code.size();
     seg->code.insert(seg->code.end(), body.begin(), body.end());
-    if (!body.empty() && (body.back() & 1023u) == (uint32_t)P_GSTF) seg->code.back() = encode(P_GSTFL, 0, body.back() >> 14);   // store and loop end in one instruction
-    else seg->code.push_back(encode(P_LOOP_END, 0, 0));
+    if (!body.empty() && (body.back() & 1023u) == (uint32_t)P_GSTF) {   // store and loop end in one instruction
+      const uint32_t opd = body.back() >> 14, pv = body.size() > 1 ? body[body.size() - 2] : 0u, pc = pv & 1023u;
+      if (body.size() > 1 && pc >= (uint32_t)(J_FMAUR * kJointStride) && pc < (uint32_t)(J_FMAUR * kJointStride + nr) && (pv >> 14) < 512 && opd < 64) {
+        seg->code.pop_back();    // ... and the multiply-add before it as well
+        seg->code.back() = encode(J_FMAURSTL * kJointStride + (int)(pc - J_FMAUR * kJointStride), 0, (pv >> 14) | (opd << 9));
+      } else {
+        seg->code.back() = encode(P_GSTFL, 0, opd);
+      }
+    } else {
+      seg->code.push_back(encode(P_LOOP_END, 0, 0));
+    }
     seg->code.insert(seg->code.end(), epi.begin(), epi.end());
     seg->code.push_back(encode(P_END, 0, 0));
     seg->code.push_back(encode(P_END, 0, 0));  // the interpreter prefetches one word ahead

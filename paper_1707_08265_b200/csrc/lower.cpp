@@ -695,10 +695,11 @@ static size_t share_workspace(Plan* plan, size_t off) {
       int opd = -1; bool store = false;
       const uint32_t jg = cs / vm::kJointStride;
       if (cs == (uint32_t)vm::P_GST || cs == (uint32_t)vm::P_GSTF || cs == (uint32_t)vm::P_GSTFL) { opd = (int)arg; store = true; }
+      else if (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_FMAURSTL) { opd = (int)(arg >> 9); store = true; }
       else if (cs == (uint32_t)vm::P_GLD || cs == (uint32_t)vm::P_GLDF || (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_GLDR)) opd = (int)arg;
       else if (cs == (uint32_t)vm::P_GLDA0 || cs == (uint32_t)vm::P_GLDA || cs == (uint32_t)vm::P_LDSW || cs == (uint32_t)vm::P_LDSWA ||
                cs == (uint32_t)vm::P_GLDA0H || cs == (uint32_t)vm::P_LDSWAH ||
-               (cs < (uint32_t)vm::kFirstPlain && (jg == (uint32_t)vm::J_LDSWR || jg == (uint32_t)vm::J_LDSWAR))) opd = (int)(arg & 63u);
+               (cs < (uint32_t)vm::kFirstPlain && (jg == (uint32_t)vm::J_LDSWR || jg == (uint32_t)vm::J_LDSWAR || jg == (uint32_t)vm::J_LDSWARF))) opd = (int)(arg & 63u);
       else if (cs == (uint32_t)vm::P_ULOAD) opd = (int)(arg >> 9);
       if (opd < 0 || opd >= (int)acc[si].size()) continue;
       if (store) acc[si][opd].first_store = std::min(acc[si][opd].first_store, i);
@@ -777,7 +778,7 @@ static size_t share_workspace(Plan* plan, size_t off) {
 static std::string disassemble(const VmSegment& sg) {
   static const char* jn[] = {"ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
                              "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
-                             "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7"};
+                             "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurst}loop"};
   static const char* pn[] = {"ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls",
                              "divps", "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq",
                              "yomy", "divpgb", "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout",

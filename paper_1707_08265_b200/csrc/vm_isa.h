@@ -43,6 +43,9 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   // R[a] = acc; acc = R: the most frequent pair of instructions ("put this away, take that") as one,
   // one group per a (the slot index of the case id is the register that is loaded)
   J_STLD0, J_STLD1, J_STLD2, J_STLD3, J_STLD4, J_STLD5, J_STLD6, J_STLD7,
+  // two frequent pairs as one instruction each (one dispatch less per tile):
+  J_LDSWARF,   // J_LDSWAR (arg bits 0..9: operand | slot << 6), then acc = R * U[u] + U[u + 1], u = arg >> 10
+  J_FMAURSTL,  // J_FMAUR with U[arg & 511], then P_GSTFL to operand arg >> 9
   J_COUNT
 };
 // The kernel exists in two builds that share this encoding: "wide" (7 register slots, one CTA per

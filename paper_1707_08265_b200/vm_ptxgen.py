@@ -40,13 +40,13 @@ OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIF
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
          "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
-         "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7"]
+         "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurstl"]
 # Leaves that end in their own indexed branch instead of a jump to the shared dispatch block: one
 # taken branch less per dispatch.  Measured, not derived: every further site makes the assembler add
 # branch-table code and changes its register allocation, and larger sets ran slower on all three
 # large workloads (16 more short leaves: +3 % on the sin/cos graph, +3 % on the random DAG), so the
 # list holds the short arithmetic, store and staged-load leaves it was first tried with.
-HOT = {"fmau", "mul", "sacc0", "macc1", "fmaur", "gstf", "gstfl", "cossinr", "ldswar"}
+HOT = {"fmau", "mul", "sacc0", "macc1", "fmaur", "gstf", "gstfl", "cossinr", "ldswar", "ldswarf", "fmaurstl"}
 JOINT_STRIDE = 8    # case id of a joint instruction = index * JOINT_STRIDE + register slot
 N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
@@ -471,10 +471,10 @@ class Kernel:
         return out
 
     # ---- global loads and stores of one operand ----------------------------------------------
-    def operand(self, want_meta=True):
-        """-> (ptr u64, kind u32, dtype u32) of operand[%arg] from the shared-memory copy of the table"""
+    def operand(self, want_meta=True, idx_reg=None):
+        """-> (ptr u64, kind u32, dtype u32) of operand[%arg] (or [idx_reg]) from the shared-memory copy of the table"""
         a, ptr = self.r(), self.rd()
-        self.e("shl.b32 %s, %%arg, 4;" % a)
+        self.e("shl.b32 %s, %s, 4;" % (a, idx_reg or "%arg"))
         self.e("add.u32 %s, %s, %%ub;" % (a, a))
         self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
         if not want_meta:
@@ -525,14 +525,18 @@ class Kernel:
         self.jump()
 
     # ---- staged loads: arg = operand | slot << 6 ------------------------------------------------
-    def staged_operand(self):
-        """-> (ptr u64 of the operand, shared address of this thread's 16 bytes of the slot); before the fetch"""
+    def staged_operand(self, masked=False):
+        """-> (ptr u64 of the operand, shared address of this thread's 16 bytes of the slot); before the fetch.
+        masked: the slot is a 4-bit field (the argument carries more above it)"""
         a, ptr, sl, sadr = self.r(), self.rd(), self.r(), self.r()
         self.e("and.b32 %s, %%arg, 63;" % a)
         self.e("shl.b32 %s, %s, 4;" % (a, a))
         self.e("add.u32 %s, %s, %%ub;" % (a, a))
         self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
-        self.e("shr.u32 %s, %%arg, 6;" % sl)
+        if masked:
+            self.e("bfe.u32 %s, %%arg, 6, 4;" % sl)
+        else:
+            self.e("shr.u32 %s, %%arg, 6;" % sl)
         self.e("mad.lo.u32 %s, %s, %d, %%sa;" % (sadr, sl, SLOT_BYTES))
         return ptr, sadr
 
@@ -612,15 +616,34 @@ class Kernel:
         self.load_bf16_slow(adr, A)
         self.jump()
 
-    def leaf_ldsw(self, dst, copy_to=None, then_copy=False):
-        ptr, sadr = self.staged_operand()
+    def leaf_ldsw(self, dst, copy_to=None, then_copy=False, affine=False):
+        """affine: copy_to = dst * U[u] + U[u + 1] with u = arg >> 10 instead of a plain copy"""
+        ptr, sadr = self.staged_operand(masked=affine)
+        uu = vv = None
+        if affine:
+            iu, a = self.r(), self.r()
+            self.e("shr.u32 %s, %%arg, 10;" % iu)
+            self.e("shl.b32 %s, %s, 2;" % (a, iu))
+            self.e("add.u32 %s, %s, %%ub;" % (a, a))
+            u0, u1 = self.f(), self.f()
+            self.e("ld.shared.f32 %s, [%s];" % (u0, a))
+            self.e("ld.shared.f32 %s, [%s+4];" % (u1, a))
         self.fetch()
+        if affine:
+            uu, vv = self.splat(u0), self.splat(u1)
+
+        def copy():
+            if affine:
+                for i in range(NP):
+                    self.fma2(dst[i], uu, vv, copy_to[i])
+            elif copy_to:
+                self.mov_v(copy_to, dst)
+
         slow = self.newlabel("ldsw")
         self.e("@!%%pfull bra.uni %s;" % slow)
         self.e("cp.async.wait_all;")
         self.lds_v(sadr, dst)
-        if copy_to:
-            self.mov_v(copy_to, dst)
+        copy()
         if then_copy:      # the slot has been read (the loads above are ahead of the copy in this thread's order)
             self.next_copy(ptr, sadr)
         self.jump()
@@ -630,8 +653,7 @@ class Kernel:
         self.load_f32_slow(adr, dst)
         if not then_copy:      # (read once: nothing to keep; a ragged tile is followed by ragged tiles only, never staged)
             self.sts_v(sadr, dst)
-        if copy_to:
-            self.mov_v(copy_to, dst)
+        copy()
         self.jump()
 
     def load_f32_slow(self, adr, dst):
@@ -753,9 +775,10 @@ class Kernel:
             self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (adr, h * HALF_BYTES, A[2 * h], A[2 * h + 1]))
             self.label(ln)
 
-    def leaf_gstf(self, then_loop_end=False):
+    def leaf_gstf(self, then_loop_end=False, ptr=None):
         """acc -> fp32 FULL operand (and, fused, the end of the per-tile body)"""
-        ptr, _, _ = self.operand(False)
+        if ptr is None:
+            ptr, _, _ = self.operand(False)
         if not then_loop_end:
             self.fetch()
         adr = self.rd()
@@ -892,6 +915,20 @@ class Kernel:
             return
         elif op == "ldswar":
             self.leaf_ldsw(R, A, True)
+            return
+        elif op == "ldswarf":
+            self.leaf_ldsw(R, A, True, affine=True)
+            return
+        elif op == "fmaurstl":     # acc = acc * U[arg & 511] + R; store to operand arg >> 9; end of the body
+            iu, io = self.r(), self.r()
+            self.e("and.b32 %s, %%arg, 511;" % iu)
+            self.e("shr.u32 %s, %%arg, 9;" % io)
+            u = self.uniform(iu)
+            ptr, _, _ = self.operand(False, io)
+            uu = self.splat(u)
+            for i in range(NP):
+                self.fma2(A[i], uu, R[i], A[i])
+            self.leaf_gstf(True, ptr)
             return
         elif op.startswith("stld"):     # R[a] = acc; acc = R[k]
             self.fetch()

@@ -75,9 +75,9 @@ def test_programs_respect_the_builds_and_the_kernel_contracts():
                 if n.startswith("stld"):
                     assert int(n[4:]) < nr and int(n[4:]) != k
             # exactly one loop, closed either by "}loop" or by the fused store
-            assert names.count("loop{") == 1 and names.count("}loop") + names.count("gstf}loop") == 1
+            assert names.count("loop{") == 1 and names.count("}loop") + names.count("gstf}loop") + names.count("fmaurst}loop") == 1
             lo = names.index("loop{")
-            hi = names.index("}loop") if "}loop" in names else names.index("gstf}loop")
+            hi = [i for i, n in enumerate(names) if n.endswith("}loop")][0]
             body = ins[lo + 1:hi + 1]
             # successive row sums (the last of an iteration and the first of the next included) use
             # different scratch buffers; a single one asks for the barrier after its read
@@ -97,8 +97,8 @@ def test_programs_respect_the_builds_and_the_kernel_contracts():
             ordinary = {arg for n, _, arg in ins if n in ("sts", "rtos", "sincos", "cossin")}
             assert not (ordinary & set(staged.values()))
             for n, _, arg in body:
-                if n in ("ldsw", "ldswa", "ldswr", "ldswar", "glda", "ldswah"):
-                    assert staged.get(arg & 63) == arg >> 6, (n, arg)
+                if n in ("ldsw", "ldswa", "ldswr", "ldswar", "glda", "ldswah", "ldswarf"):
+                    assert staged.get(arg & 63) == (arg >> 6) & (15 if n == "ldswarf" else 0xFFF), (n, arg)
                 if n == "gldf":     # an unstaged fp32 load only when no slot was left
                     assert arg not in staged
             assert names[-1] == "end"

@@ -8,7 +8,7 @@ import numpy as np
 STRIDE = 8   # case id of a register-operand instruction = index * STRIDE + register slot
 J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
      "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
-     "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7"]
+     "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurst}loop"]
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
@@ -65,6 +65,14 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
             elif name == "fillr": R[k] = G[arg].copy()
             elif name == "gldr": acc = load(arg); R[k] = acc.copy()
             elif name in ("ldswr", "ldswar"): acc = load(arg & 63); R[k] = acc.copy(); S[arg >> 6] = acc.copy()
+            elif name == "ldswarf":
+                R[k] = load(arg & 63); S[(arg >> 6) & 15] = R[k].copy()
+                acc = R[k] * U[arg >> 10] + U[(arg >> 10) + 1]
+            elif name == "fmaurst}loop":
+                acc = acc * U[arg & 511] + R[k]
+                where, pos, kind, dtype = ops[arg >> 9]
+                assert where == 1 and kind == 0 and dtype == 0
+                out[pos] = np.array(acc, dtype=np.float64).reshape(fetch_shapes[pos])
             elif name == "sincosr": R[k] = np.cos(acc); acc = np.sin(acc)
             elif name == "cossinr": R[k] = np.sin(acc); acc = np.cos(acc)
             elif name.startswith("macc"): A[int(name[4])] += float((acc * R[k]).sum())
