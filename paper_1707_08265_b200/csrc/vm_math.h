@@ -1,7 +1,7 @@
 // Elementary functions of the graph VM, fp32, written for a few-ulp relative error so that
 // compositions of many operators stay within 1e-5 of an fp64 evaluation.
 //
-//   sin/cos : three-constant Cody-Waite reduction by pi/2 (fused multiply-adds), odd/even
+//   sin/cos : two-constant Cody-Waite reduction by pi/2 (fused multiply-adds), odd/even
 //             polynomials on [-pi/4, pi/4]
 //   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), n added to the exponent
 //   tanh    : x + x^3*T(x^2) below 0.6, 1 - 2/(exp(2|x|)+1) above
@@ -68,8 +68,9 @@ VM_HD float cos_poly(float r) {
 // costs two fused multiply-adds instead of a round and a float-to-int conversion on the
 // quarter-rate pipe; it is exact for |x*2/pi| < 2^22.  Each reduction step is one fused
 // multiply-add, so the first difference is exact while k*fl(pi/2) stays within 24 bits of x;
-// the later steps add an absolute error of a few 1e-7 at the largest arguments, far below the
-// spacing of fp32 numbers of that size.  Beyond |x| = 6.5e6 (and for inf/NaN) x - x is returned:
+// the second step and the part of pi/2 left out (1.7e-15 per quadrant, 7e-9 at the edge of the
+// range) add an absolute error of a few 1e-7 at the largest arguments, far below the spacing of
+// fp32 numbers of that size.  Beyond |x| = 6.5e6 (and for inf/NaN) x - x is returned:
 // 0, or NaN.
 VM_HD float reduce_pio2(float x, int* q) {
   const float big = 12582912.0f;                                  // 1.5 * 2^23
@@ -77,7 +78,6 @@ VM_HD float reduce_pio2(float x, int* q) {
   float k = kb - big;
   float r = fmaf(-k, 1.57079637050628662109375f, x);        // fl(pi/2)
   r = fmaf(-k, -4.371138828673793e-8f, r);                  // fl(pi/2 - c1)
-  r = fmaf(-k, -1.7151245100058819e-15f, r);                // fl(pi/2 - c1 - c2)
   int qi = (int)f_bits(kb);                                 // low bits = k (two's complement)
   if (!(fabsf(x) <= 6.5e6f)) { r = x - x; qi = 0; }
   *q = qi;
