@@ -592,6 +592,22 @@ struct Gen {
       }
       body.swap(out);
     }
+    {   // "R = acc; acc = S[slot]" and "row sum, times a uniform" (a mean) are one instruction each
+      std::vector<uint32_t> out;
+      for (size_t i = 0; i < body.size(); ++i) {
+        const uint32_t w = body[i], cs = w & 1023u, nx = i + 1 < body.size() ? body[i + 1] : 0u, nc = nx & 1023u;
+        if (i + 1 < body.size() && cs >= (uint32_t)(J_STR * kJointStride) && cs < (uint32_t)(J_STR * kJointStride + nr) && nc == (uint32_t)P_LDS) {
+          out.push_back(encode(J_STRLDS * kJointStride + (int)(cs - J_STR * kJointStride), 0, nx >> 14));
+          ++i;
+        } else if (i + 1 < body.size() && cs == (uint32_t)P_ROWSUM && nc == (uint32_t)P_MULU && (nx >> 14) < 512) {
+          out.push_back(encode(P_ROWSUMU, 0, ((w >> 14) & 7u) | ((nx >> 14) << 3)));
+          ++i;
+        } else {
+          out.push_back(w);
+        }
+      }
+      body.swap(out);
+    }
     // 6. epilogue: accumulators leave as per-CTA partial sums
     for (auto& a : accs) {
       const Item& it = items[idx[a.first]];

@@ -46,6 +46,7 @@ enum Joint : int {  // each occupies kJointStride consecutive case ids, one per 
   // two frequent pairs as one instruction each (one dispatch less per tile):
   J_LDSWARF,   // J_LDSWAR (arg bits 0..9: operand | slot << 6), then acc = R * U[u] + U[u + 1], u = arg >> 10
   J_FMAURSTL,  // J_FMAUR with U[arg & 511], then P_GSTFL to operand arg >> 9
+  J_STRLDS,    // R = acc; acc = S[arg]   (J_STR, then P_LDS)
   J_COUNT
 };
 // The kernel exists in two builds that share this encoding: "wide" (7 register slots, one CTA per
@@ -101,6 +102,7 @@ enum Plain : int {
   P_GSTFL,              // P_GSTF followed by P_LOOP_END (a body that ends in a store)
   P_GLDA0H,             // P_GLDA0 for a bf16 operand (8 bytes per thread and half of the tile)
   P_LDSWAH,             // P_LDSWA for a bf16 operand: converts to fp32 at the read; such an operand is read once per iteration
+  P_ROWSUMU,            // P_ROWSUM with arg & 7, then acc = acc * U[arg >> 3]   (a row mean)
   P_END,
   P_COUNT_
 };

@@ -40,7 +40,7 @@ OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIF
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
          "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
-         "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurstl"]
+         "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurstl", "strlds"]
 # Leaves that end in their own indexed branch instead of a jump to the shared dispatch block: one
 # taken branch less per dispatch.  Measured, not derived: every further site makes the assembler add
 # branch-table code and changes its register allocation, and larger sets ran slower on all three
@@ -52,7 +52,7 @@ N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "end"]
 
 
 def f32bits(x):
@@ -930,6 +930,11 @@ class Kernel:
                 self.fma2(A[i], uu, R[i], A[i])
             self.leaf_gstf(True, ptr)
             return
+        elif op == "strlds":            # R = acc; acc = S[arg]
+            a = self.slot_addr()
+            self.fetch()
+            self.mov_v(R, A)
+            self.lds_v(a, A)
         elif op.startswith("stld"):     # R[a] = acc; acc = R[k]
             self.fetch()
             self.mov_v(self.R[int(op[4])], A)
@@ -1104,6 +1109,16 @@ class Kernel:
             self.e("setp.ne.u32 %s, %s, 0;" % (psync, t))
             self.fetch()
             self.leaf_rowsum(boff, psync)
+        elif op == "rowsumu":    # the same with arg & 7, then acc = acc * U[arg >> 3]
+            boff, t, psync, iu = self.r(), self.r(), self.p(), self.r()
+            self.e("and.b32 %s, %%arg, 3;" % boff)
+            self.e("shl.b32 %s, %s, 6;" % (boff, boff))
+            self.e("and.b32 %s, %%arg, 4;" % t)
+            self.e("setp.ne.u32 %s, %s, 0;" % (psync, t))
+            self.e("shr.u32 %s, %%arg, 3;" % iu)
+            u = self.uniform(iu)
+            self.fetch()
+            self.leaf_rowsum(boff, psync, u)
         elif op == "gld":
             self.leaf_gld(); return
         elif op == "gst":
@@ -1168,8 +1183,8 @@ class Kernel:
         self.e("shr.u32 %s, %s, 5;" % (warp, t))
         return warp, lane
 
-    def leaf_rowsum(self, boff, psync):
-        """acc = sum of acc over the row.  Successive row sums write their per-warp partials to
+    def leaf_rowsum(self, boff, psync, scale=None):
+        """acc = sum of acc over the row (times the scalar register scale, if given).  Successive row sums write their per-warp partials to
         different scratch buffers (the host alternates them), so one barrier per sum is enough: a
         buffer is written again only after another row sum's barrier, which every warp passes after
         it has read this one."""
@@ -1207,6 +1222,8 @@ class Kernel:
         self.e("@!%s bra.uni %s;" % (psync, nosync))
         self.e("bar.sync 0;")
         self.label(nosync)
+        if scale:
+            self.e("mul.f32 %s, %s, %s;" % (tot, tot, scale))
         tt = self.splat(tot)
         for i in range(NP): self.e("mov.b64 %s, %s;" % (A[i], tt))
 

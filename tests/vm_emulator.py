@@ -8,11 +8,11 @@ import numpy as np
 STRIDE = 8   # case id of a register-operand instruction = index * STRIDE + register slot
 J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
      "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
-     "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurst}loop"]
+     "stld0", "stld1", "stld2", "stld3", "stld4", "stld5", "stld6", "stld7", "ldswarf", "fmaurst}loop", "strlds"]
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
-     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "end"]
+     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "end"]
 
 
 def _bf16(a):
@@ -65,6 +65,7 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
             elif name == "fillr": R[k] = G[arg].copy()
             elif name == "gldr": acc = load(arg); R[k] = acc.copy()
             elif name in ("ldswr", "ldswar"): acc = load(arg & 63); R[k] = acc.copy(); S[arg >> 6] = acc.copy()
+            elif name == "strlds": R[k] = acc.copy(); acc = S[arg].copy()
             elif name == "ldswarf":
                 R[k] = load(arg & 63); S[(arg >> 6) & 15] = R[k].copy()
                 acc = R[k] * U[arg >> 10] + U[(arg >> 10) + 1]
@@ -104,6 +105,7 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
         elif name == "divpgb": acc = -np.sign(acc) / (1 + np.abs(acc)) ** 2
         elif name == "rbf16": acc = _bf16(acc)
         elif name == "rowsum": acc = np.broadcast_to(acc.sum(axis=-1, keepdims=True), shape).copy()
+        elif name == "rowsumu": acc = np.broadcast_to(acc.sum(axis=-1, keepdims=True), shape).copy() * U[arg >> 3]
         elif name in ("gld", "gldf"): acc = load(arg)
         elif name in ("gst", "gstf", "gstf}loop"):
             where, pos, kind, dtype = ops[arg]
