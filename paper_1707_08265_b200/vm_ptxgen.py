@@ -375,33 +375,32 @@ class Kernel:
         return out
 
     def tanh(self, xs):
+        """x * P(x^2) / Q(x^2) on |x| <= 9 (a rational fit, about 5 ulp), clamped to [-1, 1]; NaN stays NaN"""
+        def clamp2(v, lim):
+            out = []
+            for s in self.unpack(v):
+                d = self.f()
+                self.e("max.NaN.f32 %s, %s, %s;" % (d, s, fc(-lim)))
+                self.e("min.NaN.f32 %s, %s, %s;" % (d, d, fc(lim)))
+                out.append(d)
+            return self.pack(out[0], out[1])
+        cs = [clamp2(x, 9.0) for x in xs]
+        z = [self.mul2(c, c) for c in cs]
+        k0, k1 = self.K(1.3442309683456469e-08), self.K(2.0679596671714183e-05)
+        p = [self.fma2(zi, k0, k1) for zi in z]
+        for c in (3.5001979607618507e-03, 1.3385017810927272e-01, 1.0):
+            k = self.K(c)
+            p = [self.fma2(zi, pi, k) for zi, pi in zip(z, p)]
+        k0, k1 = self.K(7.814557141497938e-07), self.K(3.2929435375013785e-04)
+        q = [self.fma2(zi, k0, k1) for zi in z]
+        for c in (2.5894861704209737e-02, 4.6718338985166813e-01, 1.0):
+            k = self.K(c)
+            q = [self.fma2(zi, qi, k) for zi, qi in zip(z, q)]
         out = []
-        for x in xs:
-            z = self.mul2(x, x)
-            p = self.fma2(z, self.K(-5.89516999486988e-3), self.K(2.079598263424288e-2))
-            p = self.fma2(z, p, self.K(-5.378383380013826e-2))
-            p = self.fma2(z, p, self.K(1.333192417199396e-1))
-            p = self.fma2(z, p, self.K(-3.3333298003965545e-1))
-            small = self.unpack(self.fma2(self.mul2(x, z), p, x))
-            xl = self.unpack(x)
-            ax, am = [], []
-            for s in xl:
-                a, m = self.f(), self.f()
-                self.e("abs.f32 %s, %s;" % (a, s))
-                self.e("min.f32 %s, %s, 0f41A00000;" % (m, a))   # 20
-                ax.append(a)
-                am.append(m)
-            e = self.exp_core(self.mul2(self.pack(am[0], am[1]), self.K(2.0)))
-            e1 = self.unpack(self.add2(e, self.K(1.0)))
-            big = self.unpack(self.fma2(self.pack(self.rcp(e1[0]), self.rcp(e1[1])), self.K(-2.0), self.K(1.0)))
-            res = []
-            for j in range(2):
-                b, pr, d = self.f(), self.p(), self.f()
-                self.e("copysign.f32 %s, %s, %s;" % (b, xl[j], big[j]))   # magnitude of big, sign of x
-                self.e("setp.lt.f32 %s, %s, %s;" % (pr, ax[j], fc(0.6)))
-                self.e("selp.f32 %s, %s, %s, %s;" % (d, small[j], b, pr))
-                res.append(d)
-            out.append(self.pack(res[0], res[1]))
+        for c, pi, qi in zip(cs, p, q):
+            ql, qh = self.unpack(qi)
+            y = self.mul2(self.mul2(c, pi), self.pack(self.rcp(ql), self.rcp(qh)))
+            out.append(clamp2(y, 1.0))
         return out
 
     def divp(self, num, den, dst):
