@@ -29,7 +29,7 @@ WORKLOAD = "config 2: f=x*sin(a*x+b), x fp32[2^26], fetch df/dx, df/da, df/db"
 ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
 # dram__bytes_read.sum + dram__bytes_write.sum of the VM kernel per element, from the ncu capture summarised in
 # profiles/vm_dense_config2.md (taken at 2^25 elements; traffic is proportional to the element count);
-NCU_DRAM_BYTES_PER_ELEM = (134.363904e6 + 92.452352e6) / (1 << 25)
+NCU_DRAM_BYTES_PER_ELEM = (134.344448e6 + 89.499136e6) / (1 << 25)
 
 
 def measured_peak_gbs():
