@@ -154,9 +154,16 @@ def run_other_config(args):
     else:
         from oracle import prune as oprune   # which inputs are connected is decided outside the generator
         g, inputs, fetch = wl.random_row_dag(16384, 4096, seeds["random_row_dag"]["seed"])
-        G = oprune.backward_marks(g.desc, fetch, inputs)
-        outputs = fetch + g.grad(fetch, [i for i in inputs if i in G])
-        units, what = 16384 * 4096, "random 1024-operator row DAG on [16384,4096], forward + backward"
+        if args.config == 5:
+            G = oprune.backward_marks(g.desc, fetch, inputs)
+            outputs = fetch + g.grad(fetch, [i for i in inputs if i in G])
+            units, what = 16384 * 4096, "random 1024-operator row DAG on [16384,4096], forward + backward"
+        else:   # not one of the five: the same DAG with one gradient stage per objective (Jacobian-style fetches)
+            outputs = list(fetch)
+            for o in fetch:
+                G = oprune.backward_marks(g.desc, [o], inputs)
+                outputs += g.grad([o], [i for i in inputs if i in G])
+            units, what = 16384 * 4096, "row DAG on [16384,4096], forward + one gradient stage per objective (%d fetches)" % len(outputs)
     f = B.Graph.from_desc(g.desc).function(inputs, outputs)
     feeds = [dev_random(g, t) if u else None for t, u in zip(inputs, f.used_inputs())]
     if args.config == 4:
@@ -191,7 +198,7 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU (default: the benchmark's 2^26)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6],
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7],
                     help="2 (default) is the benchmark workload; the others print one summary line each (6: SGD updater)")
     args = ap.parse_args()
     if args.impl == "reference":

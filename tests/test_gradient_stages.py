@@ -130,6 +130,23 @@ def test_emulated_jacobian_style_row_dag(seed):
         assert np.allclose(gv[ok], rv[ok], rtol=1e-7, atol=1e-7), o
 
 
+def test_emulated_per_objective_program_of_the_large_row_dag():
+    """The 1024-operator row DAG with one stage per objective, at its full row length: the emitted
+    program (wide build, shared-memory slots, a workspace spill slot, three column sums) evaluated in
+    fp64 by the emulator equals the oracle to rounding, ill-conditioned outputs included."""
+    import json
+    import os
+    seed = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "config_seeds.json")))["random_row_dag"]["seed"]
+    g, inputs, fetch = wl.random_row_dag(3, 4096, seed)
+    stages = attach_pairs(g, fetch, inputs)
+    outs = list(fetch) + [gid for (_, _, gids) in stages for gid in gids]
+    feeds = wl.normal_feeds([g.shape(i) for i in inputs], 5)
+    ref = interp.run_function(g.desc, inputs, outs, feeds)
+    _, got = emulate(g, inputs, outs, feeds)
+    for gv, rv, o in zip(got, ref, outs):
+        assert np.allclose(gv, rv, rtol=1e-9, atol=1e-9), o
+
+
 # ---- GPU ---------------------------------------------------------------------------------------
 
 @pytest.mark.gpu
@@ -174,3 +191,56 @@ def test_gpu_three_objectives_flat_with_ragged_tail():
     check(got[k + 1], np.cos(u), TOL32, "d o1 / d w")
     check(got[k + 4], np.sum(x * np.exp(a * x)), TOL32, "d o2 / d a")
     check(got[k + 6], np.sin(u) + w * np.cos(u), TOL32, "d o3 / d w")
+
+
+@pytest.mark.gpu
+def test_gpu_jacobian_style_row_dag_full_size():
+    """The row DAG of the fifth workload at [16384, 4096] with one gradient stage per objective, in the
+    launch configuration the benchmark times.  Rows are independent (row sums stay inside a row), so the
+    oracle evaluates a sample of rows on the same values; FULL-shaped outputs of those rows must match."""
+    import json
+    import os
+    import torch
+    from test_gpu_vm import check, TOL32
+    rows, cols = 16384, 4096
+    seed = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "config_seeds.json")))["random_row_dag"]["seed"]
+
+    def build(r):
+        g, inputs, fetch = wl.random_row_dag(r, cols, seed)
+        outs = list(fetch)
+        for o in fetch:
+            G = oprune.backward_marks(g.desc, [o], inputs)
+            outs += g.grad([o], [i for i in inputs if i in G])
+        return g, inputs, outs
+
+    g, inputs, outs_ids = build(rows)
+    f = B.Graph.from_desc(g.desc).function(inputs, outs_ids)
+    want = oprune.function_sets(g.desc, inputs, outs_ids)
+    fwd, gops, masks = f.kept_ops()
+    assert f.marked() == want["marked"] and fwd == want["fwd_ops"] and gops == [k for (_, k, _) in want["grad_ops"]]
+    gen = torch.Generator("cuda").manual_seed(seed)
+    gpu_in = [torch.empty(tuple(g.shape(i)), dtype=torch.float32, device="cuda").normal_(generator=gen) for i in inputs]
+    outs = [torch.full(tuple(g.shape(o)), float("nan"), dtype=torch.float32, device="cuda") for o in outs_ids]
+    f.run_torch([t if u else None for t, u in zip(gpu_in, f.used_inputs())], outs)
+    assert f.status() == 0
+    torch.cuda.synchronize()
+    pick = np.unique(np.concatenate([[0, 1, rows - 1], np.random.default_rng(2).integers(0, rows, 13)]))
+    tp = torch.from_numpy(pick).cuda()
+    sub = [t[tp].cpu().numpy() if t.dim() == 2 else t.cpu().numpy() for t in gpu_in]
+    gs, in_s, outs_s = build(len(pick))
+    ref = interp.run_function(gs.desc, in_s, outs_s, sub)
+    low = interp.run_function(gs.desc, in_s, outs_s, sub, dtype=np.float32)
+    n_full = n_tight = 0
+    for o, r, l, t in zip(outs, ref, low, outs_ids):
+        assert torch.isfinite(o).all()
+        if o.dim() == 2:
+            # One of the per-objective gradients is ill-conditioned in fp32: NumPy's own fp32 evaluation is
+            # 10 to 80 tolerances away from fp64 on it, and a mask behind a row sum flips for whole rows.  The
+            # emitted program for it is exact when run in fp64 (the emulated tests), so that tensor is left
+            # out of the comparison here; every other one is held to the tolerance.
+            floor = float(np.max(np.abs(l.astype(np.float64) - r) / (TOL32 * (1 + np.abs(r)))))
+            n_full += 1
+            if floor <= 0.25:
+                check(o[tp].cpu().numpy().astype(np.float64), r, TOL32, "tensor %d" % t)
+                n_tight += 1
+    assert n_full >= 4 and n_tight >= n_full - 1
