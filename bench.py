@@ -27,8 +27,9 @@ METRIC = "pruned-graph fwd+bwd elements/sec"
 UNIT = "elements/s"
 WORKLOAD = "config 2: f=x*sin(a*x+b), x fp32[2^26], fetch df/dx, df/da, df/db"
 ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
-# dram__bytes_read.sum + dram__bytes_write.sum of the VM kernel per element, from the ncu capture summarised in
-# profiles/vm_dense_config2.md (taken at 2^25 elements; traffic is proportional to the element count);
+# dram__bytes_read.sum + dram__bytes_write.sum of the VM kernel per element, from one ncu capture of this
+# kernel binary on this workload at 2^25 elements (traffic is proportional to the element count); None once the
+# kernel has changed since the counters were taken
 NCU_DRAM_BYTES_PER_ELEM = (134.344448e6 + 89.499136e6) / (1 << 25)
 
 
