@@ -48,6 +48,7 @@ struct Gen {
   std::vector<bool> done;        // item already produced by a fused instruction
   std::vector<std::pair<int, int>> accs;  // (item position of an accumulation, its pinned register)
   std::vector<std::pair<int, int>> saccs; // (item position of an accumulation to a scalar, its scalar accumulator)
+  std::vector<std::pair<int, int>> maccs; // (item position of an accumulation, its pinned shared-memory slot)
   int err = DRAGON_OK;
 
   Gen(const std::vector<Item>& it, const std::vector<int>& ix, const std::vector<Value>& v,
@@ -84,6 +85,7 @@ struct Gen {
   bool emit_accum(int q) {
     for (auto& a : accs) if (a.first == q) { emit(J_ACCUM * kJointStride + a.second); return true; }
     for (auto& a : saccs) if (a.first == q) { emit(P_SACC0 + a.second); return true; }
+    for (auto& a : maccs) if (a.first == q) { emit(P_ACCUMS, 0, (uint32_t)a.second); return true; }
     return false;
   }
   int scalar_acc_at(int q) const {
@@ -491,10 +493,27 @@ struct Gen {
           continue;
         }
         int k = (int)accs.size();
-        if (k >= nr - 2) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+        if (k >= nr - 2) {
+          // no register slot left to pin: the running sum lives in a shared-memory slot (two slots stay free for values)
+          int sl = (int)maccs.size() + 2 < n_smem_max ? free_smem() : -1;
+          if (sl < 0) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+          smem_owner[sl] = -2;
+          maccs.emplace_back(p, sl);
+          continue;
+        }
         reg_owner[k] = -2;
         accs.emplace_back(p, k);
       }
+    if (!maccs.empty()) {   // those slots start at zero
+      const float zero = 0.f;
+      const int uz = n_uni++;
+      pro.push_back(encode(P_UCONST, 0, uz));
+      uint32_t bits; std::memcpy(&bits, &zero, 4);
+      pro.push_back(bits);
+      preamble.push_back(encode(P_LDU, 0, uz));
+      for (auto& a : maccs) preamble.push_back(encode(P_STS, 0, (uint32_t)a.second));
+      if (n_uni > 511) { set_error("graph VM: too many scalars and constants"); return DRAGON_ERR_UNSUPPORTED; }
+    }
     // 4. body
     done.assign(idx.size(), false);
     for (int p = 0; p < (int)idx.size() && !err; ++p) {
@@ -619,6 +638,16 @@ struct Gen {
       else { set_error("graph VM: reduction target shape is not supported"); return DRAGON_ERR_UNSUPPORTED; }
       seg->finish.push_back(job);
     }
+    for (auto& a : maccs) {
+      const Item& it = items[idx[a.first]];
+      int cls = class_of(mems[it.mem].shape);
+      FinishJob job; job.mem = it.mem;
+      epi.push_back(encode(P_LDS, 0, (uint32_t)a.second));
+      if (cls == K_SCALAR) { job.kind = 1; job.acc = seg->n_scalacc++; epi.push_back(encode(P_SCALOUT, 0, job.acc)); }
+      else if (cls == K_ROW) { job.kind = 0; job.acc = seg->n_colacc++; epi.push_back(encode(P_COLOUT, 0, job.acc)); }
+      else { set_error("graph VM: reduction target shape is not supported"); return DRAGON_ERR_UNSUPPORTED; }
+      seg->finish.push_back(job);
+    }
     for (auto& a : saccs) {
       const Item& it = items[idx[a.first]];
       FinishJob job; job.mem = it.mem; job.kind = 1; job.acc = seg->n_scalacc++;
@@ -652,6 +681,7 @@ struct Gen {
       if (cs == P_UCONST) ++i;  // the next word is a literal
     }
     if ((int)seg->code.size() > kVmCodeMaxWords) { set_error("graph VM: instruction stream too long (%d words)", (int)seg->code.size()); return DRAGON_ERR_UNSUPPORTED; }
+    if ((int)seg->finish.size() > kVmScalarAccs + kVmRegsWide - 2 + kVmSmemSlots - 2) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
     if ((int)seg->operand_mem.size() > kMaxOperands) { set_error("graph VM: too many memory operands in one segment"); return DRAGON_ERR_UNSUPPORTED; }
     return DRAGON_OK;
   }

@@ -103,6 +103,8 @@ enum Plain : int {
   P_GLDA0H,             // P_GLDA0 for a bf16 operand (8 bytes per thread and half of the tile)
   P_LDSWAH,             // P_LDSWA for a bf16 operand: converts to fp32 at the read; such an operand is read once per iteration
   P_ROWSUMU,            // P_ROWSUM with arg & 7, then acc = acc * U[arg >> 3]   (a row mean)
+  P_ACCUMS,             // S[arg] = S[arg] + (lane valid ? acc : 0): a loop-carried accumulator kept in shared memory
+                        // (reduced outputs beyond the pinned register slots)
   P_END,
   P_COUNT_
 };

@@ -19,6 +19,10 @@ namespace vm {
 
 // ---- finishing reductions: per-CTA partials -> tensors (fixed order, fp64) ------------------
 
+// a segment reduces at most kVmScalarAccs sums in scalar accumulators, kVmRegsWide - 2 in pinned register
+// slots and kVmSmemSlots - 2 in pinned shared-memory slots
+constexpr int kMaxFinishJobs = kVmScalarAccs + kVmRegsWide - 2 + kVmSmemSlots - 2;
+
 struct FinishParams {
   int n_jobs;
   struct Job {
@@ -27,8 +31,10 @@ struct FinishParams {
     void* out;
     int dtype, cols, grid;
     int chunks, chunk_stride;              // scalar partials of a chunked run: one [accumulator][grid] set per chunk
-  } job[8];
+  } job[kMaxFinishJobs];
 };
+static_assert(kMaxFinishJobs >= kVmScalarAccs + kVmRegsDense - 2 + kVmSmemSlotsDense - 2 && sizeof(FinishParams) <= 4096,
+              "every build's reductions fit one finishing launch");
 
 constexpr int kFinishThreads = 256;
 
@@ -111,6 +117,7 @@ cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dens
 
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st, int chunks) {
   if (sg.finish.empty()) return cudaSuccess;
+  if ((int)sg.finish.size() > vm::kMaxFinishJobs) return cudaErrorInvalidValue;   // the code generator never emits more
   vm::FinishParams fp;
   fp.n_jobs = (int)sg.finish.size();
   int max_cols = 1;

@@ -52,7 +52,7 @@ N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "accums", "end"]
 
 
 def f32bits(x):
@@ -1166,6 +1166,18 @@ class Kernel:
             self.jump()
             self.label(tail)
             self.e("add.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(self.packs(self.mask_tail(self.scalars(A))))))
+        elif op == "accums":     # S[arg] += acc over the valid lanes
+            a = self.slot_addr(); self.fetch()
+            T = self.lds_v(a)
+            tail, st = self.newlabel("as"), self.newlabel("as")
+            self.e("@!%%pfull bra.uni %s;" % tail)
+            for i in range(NP): self.add2(T[i], A[i], T[i])
+            self.e("bra.uni %s;" % st)
+            self.label(tail)
+            m = self.packs(self.mask_tail(self.scalars(A)))
+            for i in range(NP): self.add2(T[i], m[i], T[i])
+            self.label(st)
+            self.sts_v(a, T)
         elif op.startswith("ascal"):
             self.leaf_scalout([self.S[int(op[5])]])
         elif op == "end":

@@ -205,3 +205,36 @@ def test_epilogue_fusion_needs_the_bias_in_memory_before_the_product_runs(bias_f
     f = B.Graph.from_desc(gd.desc).function([X, W, b], [Y])
     text = f.describe()
     assert ("+bias" in text) == bias_first, text
+
+
+@pytest.mark.parametrize("n_scalars", [8, 9, 10, 14, 30])
+def test_many_reduced_outputs_fit_the_finishing_launch_or_are_refused(n_scalars):
+    """Gradients with respect to k scalars are k sums over the whole domain.  One segment holds 4 scalar
+    accumulators, 5 pinned register slots and, beyond those, pinned shared-memory slots; the finishing
+    launch has a job table sized for all of them, so every count either compiles with exactly k jobs
+    (and computes the right sums, checked on the instruction-set emulator) or is refused at compile time."""
+    from vm_emulator import run_step
+    n = 3 * 4096 + 5
+    gd = wl.GraphDesc()
+    x = gd.tensor("x", [n])
+    ss = [gd.tensor("s%d" % k, []) for k in range(n_scalars)]
+    acc = None
+    for k, s in enumerate(ss):
+        t = gd.op("Mul", [s, gd.op("Sin" if k % 2 else "Tanh", [x], "u%d" % k)], "t%d" % k)
+        acc = t if acc is None else gd.op("Add", [acc, t], "a%d" % k)
+    grads = gd.grad([acc], ss)
+    try:
+        f = B.Graph.from_desc(gd.desc).function([x] + ss, grads)
+    except B.DragonError as e:
+        assert n_scalars > 20 and "reduced outputs" in str(e)
+        return
+    assert n_scalars <= 20
+    step = f.vm_step(0)
+    assert len(step["reduced"]) == n_scalars and f.vm_step(1) is None
+    rng = np.random.default_rng(n_scalars)
+    feeds = [rng.standard_normal(n)] + [rng.standard_normal() for _ in ss]
+    _, _, scal = run_step(step, feeds, {})
+    for k in range(n_scalars):
+        want = float(np.sum(np.sin(feeds[0]) if k % 2 else np.tanh(feeds[0])))
+        kind, accidx, pos = step["reduced"][[r[2] for r in step["reduced"]].index(k)]
+        assert kind == 1 and abs(scal[accidx] - want) <= 1e-9 * (1 + abs(want)), (k, scal[accidx], want)
