@@ -1,8 +1,8 @@
 // Elementary functions of the graph VM, fp32, written for a few-ulp relative error so that
 // compositions of many operators stay within 1e-5 of an fp64 evaluation.
 //
-//   sin/cos : two-constant Cody-Waite reduction by pi/2 (fused multiply-adds), odd/even
-//             polynomials on [-pi/4, pi/4]
+//   sin/cos : two-constant Cody-Waite reduction by pi/2 (fused multiply-adds) up to 2^20, an exact
+//             multi-word reduction beyond; odd/even polynomials on [-pi/4, pi/4]
 //   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), n added to the exponent
 //   tanh    : x*P(x^2)/Q(x^2) on |x| <= 9, clamped
 //   sigmoid : 1/(1+exp(-x))
@@ -63,15 +63,48 @@ VM_HD float cos_poly(float r) {
   return fmaf(z * z, p, fmaf(z, -0.5f, 1.0f));
 }
 
+// Reduction of a large finite argument (|x| > 2^20, where the two-constant reduction below starts to
+// lose bits) by multiplying with as many bits of 2/pi as the argument's exponent asks for.
+// x = m * 2^s with m a 24-bit integer.  Bits of 2/pi whose weight times 2^s is a multiple of 4 only
+// move the result by whole periods and are skipped; the next 96 bits are multiplied by m modulo 2^96:
+// the top two bits of that product are the quadrant, the 64 bits below them the fraction of a
+// quadrant, read as a signed number so that the remainder lies in [-pi/4, pi/4).  The bits left out
+// change the fraction by less than 2^-70, so r is exact to the rounding of the final conversion.
+// The table is 2/pi = 0x0.A2F9836E4E44... in 32-bit words behind one word of zeros (the integer part),
+// which covers every fp32 exponent: the window starts at bit s + 30 <= 134 and is 96 + 31 bits long.
+VM_HD float reduce_pio2_large(float x, int* q) {
+  const uint32_t two_over_pi[9] = {0x00000000u, 0xA2F9836Eu, 0x4E441529u, 0xFC2757D1u, 0xF534DDC0u,
+                                   0xDB629599u, 0x3C439041u, 0xFE5163ABu, 0xDEBBC561u};
+  const uint32_t ix = f_bits(x) & 0x7fffffffu;
+  const int s = (int)(ix >> 23) - 150;
+  const uint32_t m = (ix & 0x7fffffu) | 0x800000u;
+  const int start = s + 30, idx = start >> 5, sh = start & 31;
+  const uint32_t w0 = two_over_pi[idx], w1 = two_over_pi[idx + 1], w2 = two_over_pi[idx + 2], w3 = two_over_pi[idx + 3];
+  const uint32_t h2 = sh ? (w0 << sh) | (w1 >> (32 - sh)) : w0;
+  const uint32_t h1 = sh ? (w1 << sh) | (w2 >> (32 - sh)) : w1;
+  const uint32_t h0 = sh ? (w2 << sh) | (w3 >> (32 - sh)) : w2;
+  const uint64_t p0 = (uint64_t)m * h0;
+  const uint64_t p1 = (uint64_t)m * h1 + (p0 >> 32);
+  const uint32_t r2 = m * h2 + (uint32_t)(p1 >> 32), r1 = (uint32_t)p1, r0 = (uint32_t)p0;
+  int qi = (int)(r2 >> 30);
+  const uint64_t frac = ((uint64_t)((r2 << 2) | (r1 >> 30)) << 32) | (uint64_t)((r1 << 2) | (r0 >> 30));
+  const int64_t sf = (int64_t)frac;
+  if (sf < 0) qi += 1;                                             // nearest quadrant, remainder below zero
+  float r = (float)((double)sf * 8.5153039502163865e-20);          // pi/2 * 2^-64
+  if (x < 0.0f) { r = -r; qi = -qi; }
+  *q = qi & 3;
+  return r;
+}
+
 // r = x - k*pi/2 with |r| <= pi/4 (approximately), q = k mod 4.  k = round(x*2/pi) is taken
 // with the add-a-big-constant trick (1.5*2^23: the sum's low mantissa bits are the integer), which
 // costs two fused multiply-adds instead of a round and a float-to-int conversion on the
 // quarter-rate pipe; it is exact for |x*2/pi| < 2^22.  Each reduction step is one fused
 // multiply-add, so the first difference is exact while k*fl(pi/2) stays within 24 bits of x;
-// the second step and the part of pi/2 left out (1.7e-15 per quadrant, 7e-9 at the edge of the
-// range) add an absolute error of a few 1e-7 at the largest arguments, far below the spacing of
-// fp32 numbers of that size.  Beyond |x| = 6.5e6 (and for inf/NaN) x - x is returned:
-// 0, or NaN.
+// the part of pi/2 left out is 1.7e-15 per quadrant (1.1e-9 at 2^20), and the rounding of 2/pi moves
+// x*2/pi by at most 0.03 there, so |r| stays below 0.84.  Beyond |x| = 2^20 the exact reduction above
+// takes over (the rounded 2/pi would put r further and further outside the polynomials' interval);
+// inf and NaN give x - x = NaN.
 VM_HD float reduce_pio2(float x, int* q) {
   const float big = 12582912.0f;                                  // 1.5 * 2^23
   const float kb = fmaf(x, 0.636619772367581343f, big);
@@ -79,7 +112,10 @@ VM_HD float reduce_pio2(float x, int* q) {
   float r = fmaf(-k, 1.57079637050628662109375f, x);        // fl(pi/2)
   r = fmaf(-k, -4.371138828673793e-8f, r);                  // fl(pi/2 - c1)
   int qi = (int)f_bits(kb);                                 // low bits = k (two's complement)
-  if (!(fabsf(x) <= 6.5e6f)) { r = x - x; qi = 0; }
+  if (!(fabsf(x) <= 1048576.0f)) {
+    if ((f_bits(x) & 0x7fffffffu) >= 0x7f800000u) { r = x - x; qi = 0; }
+    else r = reduce_pio2_large(x, &qi);
+  }
   *q = qi;
   return r;
 }

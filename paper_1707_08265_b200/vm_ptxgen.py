@@ -67,6 +67,11 @@ class Kernel:
     def __init__(self, name, nr, ctas_per_sm):
         self.name, self.nr, self.ctas = name, nr, ctas_per_sm
         self.lines = []
+        self.ph_sites = []    # return labels of the sin/cos sites (reduce_pio2)
+        self.PX = ["%%PX%d" % i for i in range(NP)]
+        self.PR = ["%%PR%d" % i for i in range(NP)]
+        self.PK = ["%%PK%d" % i for i in range(NP)]
+        self.cold = []        # rarely executed blocks, placed behind all leaves so that the hot leaves stay short and close together
         self.cnt = {"f": 0, "r": 0, "rd": 0, "p": 0, "fd": 0, "h": 0}
         self.nlabel = 0
         self.kt = []          # packed constants (u64 words)
@@ -80,6 +85,12 @@ class Kernel:
 
     def label(self, s):
         self.lines.append(s + ":")
+
+    def begin_cold(self):
+        self.hot_lines, self.lines = self.lines, self.cold
+
+    def end_cold(self):
+        self.lines = self.hot_lines
 
     def newlabel(self, stem="L"):
         self.nlabel += 1
@@ -230,15 +241,20 @@ class Kernel:
             self.e("mov.b64 %s, %s;" % (dst[i], src[i]))
 
     # ---- elementary functions (csrc/vm_math.h, operation by operation) -----------------------
-    def guard_range(self, xs):
-        """Copies of the packed pairs xs in which, when any lane of this thread lies beyond 6.5e6
-        in magnitude (or is inf/NaN), each such lane is replaced by x - x (0, or NaN): the
-        Cody-Waite reduction below is only good up to there.  The common case is one 3-input
-        maximum per two or three lanes and a branch that is not taken."""
-        out = [self.rd() for _ in xs]
+    RANGE = 1048576.0     # 2^20: beyond it the two-constant reduction hands over to the exact one
+
+    def reduce_pio2(self, xs):
+        """-> (r, kb): remainders of the packed pairs xs modulo pi/2 and the words whose two low bits are
+        the quadrant.  Common case (every lane of this thread within 2^20 in magnitude: one 3-input
+        maximum per two or three lanes and a branch that is not taken): the two-constant reduction,
+        packed.  Otherwise the thread leaves for the one copy of the general reduction that the kernel
+        holds (emit_general_reduction), which returns here behind the packed code."""
+        big = 12582912.0
+        n = len(xs)
+        assert n == NP
+        r, kb = self.PR, self.PK
         lanes = []
-        for x, o in zip(xs, out):
-            self.e("mov.b64 %s, %s;" % (o, x))
+        for x in xs:
             for s in self.unpack(x):
                 a = self.f()
                 self.e("abs.f32 %s, %s;" % (a, s))
@@ -254,36 +270,139 @@ class Kernel:
                 self.e("max.NaN.f32 %s, %s, %s;" % (d, m, rest[0]))
                 rest = rest[1:]
             m = d
-        ok, done = self.p(), self.newlabel("rng")
-        self.e("setp.le.f32 %s, %s, %s;" % (ok, m, fc(6.5e6)))
-        self.e("@%s bra %s;" % (ok, done))
-        for x, o in zip(xs, out):
-            g = []
-            for s in self.unpack(x):
-                a, z, q, pr = self.f(), self.f(), self.f(), self.p()
-                self.e("abs.f32 %s, %s;" % (a, s))
-                self.e("setp.le.f32 %s, %s, %s;" % (pr, a, fc(6.5e6)))
-                self.e("sub.f32 %s, %s, %s;" % (z, s, s))
-                self.e("selp.f32 %s, %s, %s, %s;" % (q, s, z, pr))
-                g.append(q)
-            self.pack(g[0], g[1], o)
-        self.label(done)
-        return out
-
-    def sincos(self, xs, want_sin=True, want_cos=True):
-        """sin and cos of the packed pairs xs, stage by stage over all pairs.  Reduction by multiples of
-        pi/2 held in two parts: the part left out is 1.7e-15 per quadrant, 7e-9 at 6.5e6, the
-        edge of the range guard_range admits."""
-        xs = self.guard_range(xs)
-        big = 12582912.0
+        ok, stub, join = self.p(), self.newlabel("rng"), self.newlabel("rng")
+        self.e("setp.le.f32 %s, %s, %s;" % (ok, m, fc(self.RANGE)))
+        self.e("@!%s bra %s;" % (ok, stub))
+        self.begin_cold()
+        self.label(stub)
+        for i in range(n):
+            self.e("mov.b64 %s, %s;" % (self.PX[i], xs[i]))
+        self.e("mov.u32 %%phsite, %d;" % len(self.ph_sites))
+        self.e("bra $PH_%s;" % self.name)
+        self.end_cold()
+        self.ph_sites.append(join)
         c = self.K(0.636619772367581343); cb = self.K(big)
-        kb = [self.fma2(x, c, cb) for x in xs]
+        for x, d in zip(xs, kb):
+            self.fma2(x, c, cb, d)
         c = self.K(-big)
         k = [self.add2(t, c) for t in kb]
         c = self.K(-1.57079637050628662109375)
-        r = [self.fma2(ki, c, x) for ki, x in zip(k, xs)]
+        for ki, x, d in zip(k, xs, r):
+            self.fma2(ki, c, x, d)
         c = self.K(4.371138828673793e-8)
-        r = [self.fma2(ki, c, ri) for ki, ri in zip(k, r)]
+        for ki, d in zip(k, r):
+            self.fma2(ki, c, d, d)
+        self.label(join)
+        return list(r), list(kb)
+
+    def emit_general_reduction(self):
+        """The reduction modulo pi/2 for threads that hold a lane beyond 2^20, inf or NaN; one copy per
+        kernel, entered from every sin/cos site with the argument in %PX and the site's number in
+        %phsite, left through an indexed branch back to that site with r in %PR and the quadrant words
+        in %PK.  The eight lanes are walked in a loop over a small local array.  A lane within range
+        takes the two-constant reduction (the same operations as the packed code, hence the same
+        results); inf/NaN give r = x - x (NaN); a large finite lane takes the exact reduction of
+        csrc/vm_math.h (reduce_pio2_large): x = m * 2^s, a 96-bit window of 2/pi starting at bit
+        s + 30 of the table times m modulo 2^96, whose top two bits are the quadrant and whose next
+        64 the signed fraction of a quadrant."""
+        if not self.ph_sites:
+            return
+        big = 12582912.0
+        n = NP
+        self.e("PHRET_%s: .branchtargets %s;" % (self.name, ", ".join(self.ph_sites)))
+        self.label("$PH_%s" % self.name)
+        base = self.rd()
+        self.e("mov.u64 %s, PHBUF;" % base)
+        for i in range(n):
+            self.e("st.local.b64 [%s+%d], %s;" % (base, 8 * i, self.PX[i]))
+        loop, nxt, special, large = self.newlabel("rng"), self.newlabel("rng"), self.newlabel("rng"), self.newlabel("rng")
+        i_, adr = self.r(), self.rd()
+        self.e("mov.u32 %s, 0;" % i_)
+        self.label(loop)
+        xb, ax, pin, pnf = self.r(), self.r(), self.p(), self.p()
+        self.e("mad.wide.u32 %s, %s, 4, %s;" % (adr, i_, base))
+        self.e("ld.local.b32 %s, [%s];" % (xb, adr))
+        self.e("and.b32 %s, %s, 0x7fffffff;" % (ax, xb))
+        self.e("setp.le.u32 %s, %s, 0x%08X;" % (pin, ax, f32bits(self.RANGE)))
+        self.e("@!%s bra %s;" % (pin, large))
+        xs_, kbs, ks, rs = self.f(), self.f(), self.f(), self.f()
+        self.e("mov.b32 %s, %s;" % (xs_, xb))
+        self.e("fma.rn.f32 %s, %s, %s, %s;" % (kbs, xs_, fc(0.636619772367581343), fc(big)))
+        self.e("add.rn.f32 %s, %s, %s;" % (ks, kbs, fc(-big)))
+        self.e("fma.rn.f32 %s, %s, %s, %s;" % (rs, ks, fc(-1.57079637050628662109375), xs_))
+        self.e("fma.rn.f32 %s, %s, %s, %s;" % (rs, ks, fc(4.371138828673793e-8), rs))
+        self.e("st.local.f32 [%s+32], %s;" % (adr, rs))
+        self.e("st.local.f32 [%s+64], %s;" % (adr, kbs))
+        self.e("bra %s;" % nxt)
+        self.label(large)
+        self.e("setp.ge.u32 %s, %s, 0x7f800000;" % (pnf, ax))
+        self.e("@%s bra %s;" % (pnf, special))
+        # x = m * 2^s; window of 2/pi from bit s + 30
+        mm, st, idx, sh, tb = self.r(), self.r(), self.r(), self.r(), self.rd()
+        self.e("and.b32 %s, %s, 0x007fffff;" % (mm, ax))
+        self.e("or.b32 %s, %s, 0x00800000;" % (mm, mm))
+        self.e("shr.u32 %s, %s, 23;" % (st, ax))
+        self.e("sub.u32 %s, %s, 120;" % (st, st))            # (exponent - 150) + 30
+        self.e("shr.u32 %s, %s, 5;" % (idx, st))
+        self.e("and.b32 %s, %s, 31;" % (sh, st))
+        self.e("mov.u64 %s, TWO_OVER_PI;" % tb)
+        self.e("mad.wide.u32 %s, %s, 4, %s;" % (tb, idx, tb))
+        w = [self.r() for _ in range(4)]
+        for j in range(4):
+            self.e("ld.const.b32 %s, [%s+%d];" % (w[j], tb, 4 * j))
+        h2, h1, h0 = self.r(), self.r(), self.r()
+        self.e("shf.l.wrap.b32 %s, %s, %s, %s;" % (h2, w[1], w[0], sh))
+        self.e("shf.l.wrap.b32 %s, %s, %s, %s;" % (h1, w[2], w[1], sh))
+        self.e("shf.l.wrap.b32 %s, %s, %s, %s;" % (h0, w[3], w[2], sh))
+        p0, p1, t, c, r2, r1, r0 = self.rd(), self.rd(), self.rd(), self.r(), self.r(), self.r(), self.r()
+        self.e("mul.wide.u32 %s, %s, %s;" % (p0, mm, h0))
+        self.e("shr.u64 %s, %s, 32;" % (t, p0))
+        self.e("mad.wide.u32 %s, %s, %s, %s;" % (p1, mm, h1, t))
+        self.e("shr.u64 %s, %s, 32;" % (t, p1))
+        self.e("cvt.u32.u64 %s, %s;" % (c, t))
+        self.e("mad.lo.u32 %s, %s, %s, %s;" % (r2, mm, h2, c))
+        self.e("cvt.u32.u64 %s, %s;" % (r1, p1))
+        self.e("cvt.u32.u64 %s, %s;" % (r0, p0))
+        qi, fh, fl, frac, pneg, td, rf, px = self.r(), self.r(), self.r(), self.rd(), self.p(), self.fd(), self.f(), self.p()
+        self.e("shr.u32 %s, %s, 30;" % (qi, r2))
+        self.e("shf.l.wrap.b32 %s, %s, %s, 2;" % (fh, r1, r2))
+        self.e("shf.l.wrap.b32 %s, %s, %s, 2;" % (fl, r0, r1))
+        self.e("mov.b64 %s, {%s, %s};" % (frac, fl, fh))
+        self.e("setp.lt.s64 %s, %s, 0;" % (pneg, frac))
+        self.e("@%s add.u32 %s, %s, 1;" % (pneg, qi, qi))
+        self.e("cvt.rn.f64.s64 %s, %s;" % (td, frac))
+        self.e("mul.f64 %s, %s, 0d%016X;" % (td, td, struct.unpack("<Q", struct.pack("<d", 8.5153039502163865e-20))[0]))   # pi/2 * 2^-64
+        self.e("cvt.rn.f32.f64 %s, %s;" % (rf, td))
+        self.e("setp.ne.u32 %s, %s, %s;" % (px, xb, ax))     # sign bit set
+        self.e("@%s neg.f32 %s, %s;" % (px, rf, rf))
+        self.e("@%s neg.s32 %s, %s;" % (px, qi, qi))
+        self.e("and.b32 %s, %s, 3;" % (qi, qi))
+        self.e("or.b32 %s, %s, 0x%08X;" % (qi, qi, f32bits(big)))
+        self.e("st.local.f32 [%s+32], %s;" % (adr, rf))
+        self.e("st.local.b32 [%s+64], %s;" % (adr, qi))
+        self.e("bra %s;" % nxt)
+        self.label(special)
+        xf, z, kq = self.f(), self.f(), self.r()
+        self.e("mov.b32 %s, %s;" % (xf, xb))
+        self.e("sub.f32 %s, %s, %s;" % (z, xf, xf))
+        self.e("mov.u32 %s, 0x%08X;" % (kq, f32bits(big)))
+        self.e("st.local.f32 [%s+32], %s;" % (adr, z))
+        self.e("st.local.b32 [%s+64], %s;" % (adr, kq))
+        self.label(nxt)
+        plp = self.p()
+        self.e("add.u32 %s, %s, 1;" % (i_, i_))
+        self.e("setp.lt.u32 %s, %s, %d;" % (plp, i_, 2 * n))
+        self.e("@%s bra %s;" % (plp, loop))
+        for i in range(n):
+            self.e("ld.local.b64 %s, [%s+%d];" % (self.PR[i], base, 32 + 8 * i))
+            self.e("ld.local.b64 %s, [%s+%d];" % (self.PK[i], base, 64 + 8 * i))
+        self.e("brx.idx %%phsite, PHRET_%s;" % self.name)
+
+    def sincos(self, xs, want_sin=True, want_cos=True):
+        """sin and cos of the packed pairs xs, stage by stage over all pairs.  Reduction by multiples of
+        pi/2 held in two parts (the part left out is 1.7e-15 per quadrant, 1.1e-9 at 2^20); lanes
+        beyond 2^20 are redone exactly by fix_range."""
+        r, kb = self.reduce_pio2(xs)
         z = [self.mul2(ri, ri) for ri in r]
         c0, c1 = self.K(-1.9515285269243e-4), self.K(8.33216077944338e-3)
         p = [self.fma2(zi, c0, c1) for zi in z]
@@ -1481,6 +1600,8 @@ class Kernel:
         e("st.global.u32 [%s], %s;" % (self.param(P_STATUS, "u64"), v))
         self.label(skip)
         e("exit;")
+        self.lines.extend(self.cold)
+        self.emit_general_reduction()
         # ---- assemble text ----
         head = []
         head.append(".const .align 8 .b64 KT_%s[%d] = {%s};" % (self.name, max(1, len(self.kt)), ", ".join("0x%016X" % w for w in self.kt) or "0"))
@@ -1495,6 +1616,9 @@ class Kernel:
         decl.append("\t.reg .b32 %pos0, %limit, %tnext, %tile, %ub, %sa, %ip, %case, %arg;")
         decl.append("\t.reg .b64 %tb4, %spb;")
         decl.append("\t.reg .pred %pfull;")
+        decl.append("\t.local .align 8 .b8 PHBUF[96];")
+        decl.append("\t.reg .b64 %s;" % ", ".join(self.PX + self.PR + self.PK))
+        decl.append("\t.reg .b32 %phsite;")
         decl.append("\t.reg .f32 %s;" % ", ".join(self.S))
         decl.append("\t.reg .b64 %s;" % ", ".join(self.A + sum(self.R, [])))
         return "\n".join(head + decl + body + ["}"]) + "\n"
@@ -1504,7 +1628,9 @@ VARIANTS = [("dragon_vm_wide", 7, 1), ("dragon_vm_dense", 3, 2)]   # name, regis
 
 
 def generate():
-    out = [".version 8.8", ".target sm_100a", ".address_size 64", "", ".extern .shared .align 16 .b8 dsm[];", ""]
+    out = [".version 8.8", ".target sm_100a", ".address_size 64", "", ".extern .shared .align 16 .b8 dsm[];",
+           # 2/pi = 0x0.A2F9836E4E44... behind one word of zeros (its integer part), most significant word first
+           ".const .align 4 .b32 TWO_OVER_PI[9] = {0x00000000, 0xA2F9836E, 0x4E441529, 0xFC2757D1, 0xF534DDC0, 0xDB629599, 0x3C439041, 0xFE5163AB, 0xDEBBC561};", ""]
     for name, nr, ctas in VARIANTS:
         out.append(Kernel(name, nr, ctas).build())
     return "\n".join(out)

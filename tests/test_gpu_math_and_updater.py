@@ -18,7 +18,7 @@ def sweep(lo_exp, hi_exp, per_binade=64):
 
 
 @pytest.mark.parametrize("op,lo,hi,extra", [
-    ("Sin", -20, 22, [np.pi / 4, np.pi / 2, np.pi, 1e5 * np.pi, 6.4e6]),     # up to the documented 6.5e6
+    ("Sin", -20, 128, [np.pi / 4, np.pi / 2, np.pi, 1e5 * np.pi, 1048576.0, 1048577.0, 6.4e6, 3.4028235e38]),   # every finite binade
     ("Exp", -20, 8, [10.0, -10.0, 9.9999, -9.9999, 10.0001, 88.0, -88.0]),   # clamp at +-10
     ("Tanh", -20, 8, [0.6, 0.5999999, 0.6000001, 9.0, 20.0, 21.0, 90.0]),    # polynomial below 0.6
     ("Sigmoid", -20, 8, [86.0, -86.0, 88.7, -88.7, 100.0, -100.0]),
@@ -67,12 +67,14 @@ def test_updater_graph(kind, shape):
         assert np.allclose(got[0], W.astype(np.float64) - float(lr) * grad.astype(np.float64), rtol=0, atol=2e-6)
 
 
-def test_sine_beyond_the_reduction_range_leaves_its_neighbours_alone():
-    """Arguments beyond 6.5e6 in magnitude evaluate as sin(0), cos(0); inf and NaN give NaN; the
-    other elements of the same thread (and every other thread) are those of the oracle."""
+def test_sine_of_huge_arguments_is_exact_and_leaves_its_neighbours_alone():
+    """Arguments beyond 2^20 in magnitude take the exact multi-word reduction and match the oracle like
+    any other; inf and NaN give NaN; the other elements of the same thread (and of every other
+    thread) are untouched by the rare path."""
     n = 2 * 4096 + 100
     x = np.random.default_rng(3).standard_normal(n).astype(np.float32)
-    odd = {5: 7.0e6, 6: -1.0e30, 2049: np.inf, 4096 + 17: -np.inf, 4096 + 2048 + 3: np.nan, n - 1: 3.0e8}
+    odd = {5: 7.0e6, 6: -1.0e30, 7: 4.8e8, 8: -22026.0 * 22026.0, 2049: np.inf, 4096 + 17: -np.inf, 4096 + 2048 + 3: np.nan,
+           n - 1: 3.0e8, n - 2: 3.4028235e38, n - 3: -1048577.0}
     for k, v in odd.items():
         x[k] = v
     gd = wl.GraphDesc()
@@ -80,13 +82,31 @@ def test_sine_beyond_the_reduction_range_leaves_its_neighbours_alone():
     out = gd.op("Sin", [xi], "out")
     grads = gd.grad([out], [xi])
     (s, c), _ = run_gpu(gd.desc, [xi], [out] + grads, [x])
-    keep = np.ones(n, bool)
-    keep[list(odd)] = False
+    fin = np.isfinite(x)
     xd = x.astype(np.float64)
-    check(s[keep], np.sin(xd[keep]), TOL32, "sin")
-    check(c[keep], np.cos(xd[keep]), TOL32, "cos")
+    check(s[fin], np.sin(xd[fin]), TOL32, "sin")
+    check(c[fin], np.cos(xd[fin]), TOL32, "cos")
+    # far tighter than the tolerance: a few ulp, as for small arguments
+    assert np.max(np.abs(s[fin] - np.sin(xd[fin]))) < 3e-7 and np.max(np.abs(c[fin] - np.cos(xd[fin]))) < 3e-7
     for k, v in odd.items():
-        if np.isfinite(v):
-            assert s[k] == 0.0 and c[k] == 1.0, (k, s[k], c[k])
-        else:
+        if not np.isfinite(v):
             assert np.isnan(s[k]) and np.isnan(c[k]), (k, s[k], c[k])
+
+
+def test_sine_of_huge_arguments_in_every_lane_and_tail():
+    """Random bit patterns of every exponent from 2^20 up, in all eight lanes of a thread, in full tiles and
+    in a ragged tail, through the separate sin and cos instructions as well as the paired one."""
+    n = 3 * 4096 + 777
+    rng = np.random.default_rng(9)
+    e = rng.integers(147, 255, n).astype(np.uint32)
+    x = ((rng.integers(0, 2, n).astype(np.uint32) << 31) | (e << 23) | rng.integers(0, 1 << 23, n).astype(np.uint32)).view(np.float32)
+    x[::3] = rng.standard_normal(x[::3].size).astype(np.float32) * 100        # mixed with ordinary arguments
+    gd = wl.GraphDesc()
+    xi = gd.tensor("x", [n])
+    out = gd.op("Sin", [xi], "out")
+    (s,), _ = run_gpu(gd.desc, [xi], [out], [x])                               # sin alone
+    xd = x.astype(np.float64)
+    assert np.max(np.abs(s - np.sin(xd))) < 3e-7
+    grads = gd.grad([out], [xi])
+    (c,), _ = run_gpu(gd.desc, [xi], grads, [x])                               # cos alone
+    assert np.max(np.abs(c - np.cos(xd))) < 3e-7
