@@ -62,13 +62,19 @@ enum { DRAGON_F32 = 0, DRAGON_BF16 = 1, DRAGON_I32 = 2 };
  *   SOFTMAX_CROSS_ENTROPY(Z, labels)  scalar -(1/M) sum_m log softmax(Z[m,:])[labels[m]],
  *                          labels int32 in [0, N); an out-of-range label contributes 0 and
  *                          sets the function status to DRAGON_ERR_INVALID_ARG (no fault)
+ *   OPAQUE                 an operator the library knows only as an edge set: any number of inputs
+ *                          and of outputs (Sec. 2.2: an edge from every input to every output), output
+ *                          shapes as declared.  Both prunes treat it like any other operator; a
+ *                          function that keeps one compiles (marks, kept operators and masks can
+ *                          be read) but cannot run: dragon_run returns DRAGON_ERR_UNSUPPORTED.
  */
 enum {
   DRAGON_OP_ADD = 0, DRAGON_OP_SUB = 1, DRAGON_OP_MUL = 2, DRAGON_OP_DIV = 3,
   DRAGON_OP_SIN = 4, DRAGON_OP_EXP = 5, DRAGON_OP_TANH = 6, DRAGON_OP_SIGMOID = 7,
   DRAGON_OP_RELU = 8, DRAGON_OP_SUM = 9, DRAGON_OP_MEAN = 10,
   DRAGON_OP_INNER_PRODUCT = 11, DRAGON_OP_BIAS_ADD = 12, DRAGON_OP_SOFTMAX_CROSS_ENTROPY = 13,
-  DRAGON_OP_COUNT_ = 14
+  DRAGON_OP_OPAQUE = 16,
+  DRAGON_OP_COUNT_ = 17
 };
 
 /* ---- graph capture (Sec. 2.1: tensors are nodes; an operator connects each of its inputs
@@ -84,7 +90,8 @@ dragon_id dragon_add_tensor(dragon_graph_t* g, const char* name, int dtype, int 
 /* Appends an operator.  in/out: host arrays of tensor ids declared earlier.  Every output must
  * have no producer yet, must not be among the inputs and must not have been read already; its
  * declared shape must equal the inferred one (Sec. 4.3: a mistaken shape is caught before
- * executing).  attrs is reserved (pass NULL, 0).  Returns the operator id. */
+ * executing).  Every executable operator type has exactly one output; DRAGON_OP_OPAQUE takes
+ * n_out >= 1.  attrs is reserved (pass NULL, 0).  Returns the operator id. */
 dragon_id dragon_add_op(dragon_graph_t* g, int op_type, const dragon_id* in, int n_in,
                         const dragon_id* out, int n_out, const double* attrs, int n_attrs);
 
@@ -215,7 +222,12 @@ int dragon_function_status(dragon_function_t* f);
  * the current device); make that first call outside any stream capture.  All calls on a device
  * share the one array: it keeps the previous call's contents (the function clears what has to
  * start at zero), and two calls that overlap on the GPU -- different streams, no ordering --
- * race on it and give wrong results.  An out-of-range label contributes 0, as in the operator. */
+ * race on it and give wrong results.  An out-of-range label contributes 0 to the sum as in the
+ * operator, but is not reported: this entry point has no function whose status could be read, so
+ * validate labels beforehand if they can be wrong.  logits must be 16-byte aligned, labels and
+ * loss_out 4-byte aligned (DRAGON_ERR_INVALID_ARG otherwise).  The array's address is looked up
+ * once per device and kept; after a cudaDeviceReset() in the same process it is stale and this
+ * entry point must not be used any more. */
 int dragon_softmax_ce_loss_static(const void* logits, int dtype, const int32_t* labels, int rows, int cols,
                                   float* loss_out, void* cuda_stream);
 

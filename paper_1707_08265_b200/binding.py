@@ -16,7 +16,7 @@ ERR_NO_PATH, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8,
 F32, BF16, I32 = 0, 1, 2
 DTYPES = {"f32": F32, "bf16": BF16, "i32": I32}
 OPS = {"Add": 0, "Sub": 1, "Mul": 2, "Div": 3, "Sin": 4, "Exp": 5, "Tanh": 6, "Sigmoid": 7, "ReLU": 8,
-       "Sum": 9, "Mean": 10, "InnerProduct": 11, "BiasAdd": 12, "SoftmaxCrossEntropy": 13}
+       "Sum": 9, "Mean": 10, "InnerProduct": 11, "BiasAdd": 12, "SoftmaxCrossEntropy": 13, "Opaque": 16}
 
 _lib = None
 

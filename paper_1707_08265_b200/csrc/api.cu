@@ -107,27 +107,34 @@ dragon_id dragon_add_op(dragon_graph_t* g, int op_type, const dragon_id* in, int
     if (!valid_tensor(g, in[i])) { set_error("dragon_add_op: input id %d is not a tensor", in[i]); return DRAGON_ERR_INVALID_ARG; }
   for (int i = 0; i < n_out; ++i)
     if (!valid_tensor(g, out[i])) { set_error("dragon_add_op: output id %d is not a tensor", out[i]); return DRAGON_ERR_INVALID_ARG; }
-  if (n_out != 1) { set_error("dragon_add_op: every operator type of this library has one output"); return DRAGON_ERR_INVALID_ARG; }
+  if (n_out != 1 && op_type != DRAGON_OP_OPAQUE) { set_error("dragon_add_op: every executable operator type has one output (DRAGON_OP_OPAQUE takes several)"); return DRAGON_ERR_INVALID_ARG; }
   for (int i = 0; i < n_in; ++i)
     if (g->g.tensors[in[i]].grad_stage >= 0) { set_error("dragon_add_op: gradient tensors cannot be consumed by operators"); return DRAGON_ERR_UNSUPPORTED; }
-  TensorInfo& to = g->g.tensors[out[0]];
-  if (to.producer >= 0 || to.grad_stage >= 0) { set_error("dragon_add_op: tensor '%s' already has a producer", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
-  for (int i = 0; i < n_in; ++i)
-    if (in[i] == out[0]) { set_error("dragon_add_op: operator reads its own output '%s'", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
-  // a tensor that was read before it got a producer would let the new operator close a cycle
-  if (to.consumed) { set_error("dragon_add_op: tensor '%s' is already read by an earlier operator", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
-  Shape s;
-  int rc = infer_shape(g->g, op_type, in, n_in, &s);
-  if (rc != DRAGON_OK) return rc;
-  if (s != to.shape) { set_error("dragon_add_op: declared shape of '%s' differs from the inferred one", to.name.c_str()); return DRAGON_ERR_SHAPE; }
-  if (to.dtype == DRAGON_I32) { set_error("dragon_add_op: operators produce f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+  for (int j = 0; j < n_out; ++j) {
+    const TensorInfo& to = g->g.tensors[out[j]];
+    if (to.producer >= 0 || to.grad_stage >= 0) { set_error("dragon_add_op: tensor '%s' already has a producer", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+    for (int i = 0; i < n_in; ++i)
+      if (in[i] == out[j]) { set_error("dragon_add_op: operator reads its own output '%s'", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+    for (int i = 0; i < j; ++i)
+      if (out[i] == out[j]) { set_error("dragon_add_op: output '%s' is listed twice", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+    // a tensor that was read before it got a producer would let the new operator close a cycle
+    if (to.consumed) { set_error("dragon_add_op: tensor '%s' is already read by an earlier operator", to.name.c_str()); return DRAGON_ERR_NOT_SSA; }
+    if (to.dtype == DRAGON_I32) { set_error("dragon_add_op: operators produce f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
+  }
+  if (op_type != DRAGON_OP_OPAQUE) {
+    const TensorInfo& to = g->g.tensors[out[0]];
+    Shape s;
+    int rc = infer_shape(g->g, op_type, in, n_in, &s);
+    if (rc != DRAGON_OK) return rc;
+    if (s != to.shape) { set_error("dragon_add_op: declared shape of '%s' differs from the inferred one", to.name.c_str()); return DRAGON_ERR_SHAPE; }
+  }
   OpInfo op;
   op.type = op_type;
   op.in.assign(in, in + n_in);
   op.out.assign(out, out + n_out);
   g->g.ops.push_back(op);
   for (int i = 0; i < n_in; ++i) g->g.tensors[in[i]].consumed = true;
-  g->g.tensors[out[0]].producer = (int)g->g.ops.size() - 1;
+  for (int j = 0; j < n_out; ++j) g->g.tensors[out[j]].producer = (int)g->g.ops.size() - 1;
   return (dragon_id)g->g.ops.size() - 1;
 }
 
@@ -186,8 +193,15 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
   f->n_in = n_in;
   f->n_out = n_out;
   if (prune_function(g->g, in, out, &f->prune) != DRAGON_OK) { delete f; return nullptr; }
-  if (lower_function(g->g, f->prune, in, out, query_sm_count(), &f->plan) != DRAGON_OK) { delete f; return nullptr; }
   f->rename = inplace_rename(g->g, f->prune);
+  // a kept operator that is only an edge set (Sec. 2.2) can be pruned around but not executed: the
+  // function keeps its prune results and refuses to run
+  for (int k : f->prune.fwd_ops)
+    if (g->g.ops[k].type == DRAGON_OP_OPAQUE) {
+      f->not_executable = "the function keeps an opaque operator (operator " + std::to_string(k) + "): it can be pruned but not executed";
+      return f;
+    }
+  if (lower_function(g->g, f->prune, in, out, query_sm_count(), &f->plan) != DRAGON_OK) { delete f; return nullptr; }
   return f;
 }
 
@@ -262,7 +276,7 @@ int dragon_function_num_launches(const dragon_function_t* f) {
 
 int dragon_function_describe(const dragon_function_t* f, char* buf, int cap) {
   if (!f || !buf || cap <= 0) return DRAGON_ERR_INVALID_ARG;
-  std::string s = describe_plan(f->plan);
+  std::string s = f->not_executable.empty() ? describe_plan(f->plan) : "not executable: " + f->not_executable + "\n";
   std::strncpy(buf, s.c_str(), (size_t)cap - 1);
   buf[cap - 1] = 0;
   return DRAGON_OK;
@@ -313,6 +327,7 @@ int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t by
 int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetches, void* cuda_stream) {
   if (!f || !fetches || (f->n_in > 0 && !feeds)) { set_error("dragon_run: bad argument"); return DRAGON_ERR_INVALID_ARG; }
   Plan& P = f->plan;
+  if (!f->not_executable.empty()) { set_error("dragon_run: %s", f->not_executable.c_str()); return DRAGON_ERR_UNSUPPORTED; }
   if (!f->workspace) { set_error("dragon_run: no workspace set (need %zu bytes)", P.workspace_bytes); return DRAGON_ERR_WORKSPACE; }
   cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
   char* ws = reinterpret_cast<char*>(f->workspace);
@@ -579,6 +594,7 @@ int run_host_chunked(dragon_function_t* f, const std::vector<const void*>& dev_f
 int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* const* host_fetches, void* staging_dev,
                     size_t staging_bytes, void* cuda_stream) {
   if (!f || !host_fetches || (f->n_in > 0 && !host_feeds)) { set_error("dragon_run_host: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  if (!f->not_executable.empty()) { set_error("dragon_run_host: %s", f->not_executable.c_str()); return DRAGON_ERR_UNSUPPORTED; }
   if (!staging_dev || ((uintptr_t)staging_dev & 255) || staging_bytes < dragon_function_staging_bytes(f)) {
     set_error("dragon_run_host: staging area must be 256-byte aligned device memory of at least %zu bytes", dragon_function_staging_bytes(f));
     return DRAGON_ERR_WORKSPACE;

@@ -292,10 +292,6 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
     }
   }
   for (int k : pr.fwd_ops) {
-    if (g.ops[k].out.size() != 1) {
-      set_error("operators with several outputs can be pruned but not executed");
-      return DRAGON_ERR_UNSUPPORTED;
-    }
     L.lower_forward(k);
     if (L.err) return L.err;
   }

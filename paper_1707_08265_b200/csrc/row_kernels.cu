@@ -257,6 +257,9 @@ static __device__ __align__(256) float g_static_rowloss[kStaticMaxRows + 64];
 namespace {
 // device address of the scratch array, looked up once per device (index = CUDA device ordinal)
 float* static_scratch_for_current_device(int* err) {
+  // Filled without a lock: two threads that race here look up the same symbol on the same device and
+  // store the same address, so whichever write lands last changes nothing.  The address belongs to
+  // the device's primary context; it is not looked up again after a cudaDeviceReset().
   static float* cache[64] = {};
   int dev = -1;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = DRAGON_ERR_CUDA; return nullptr; }
@@ -282,6 +285,11 @@ extern "C" int dragon_softmax_ce_loss_static(const void* logits, int dtype, cons
   using namespace dragon;
   if (!logits || !labels || !loss_out || rows <= 0 || cols <= 0 || (dtype != DRAGON_F32 && dtype != DRAGON_BF16)) {
     set_error("dragon_softmax_ce_loss_static: bad argument");
+    return DRAGON_ERR_INVALID_ARG;
+  }
+  // the row kernels read the logits with 16-byte vector loads: a misaligned pointer must be an error code, not a fault
+  if (((uintptr_t)logits & 15) || ((uintptr_t)labels & 3) || ((uintptr_t)loss_out & 3)) {
+    set_error("dragon_softmax_ce_loss_static: logits must be 16-byte aligned, labels and loss_out 4-byte aligned");
     return DRAGON_ERR_INVALID_ARG;
   }
   if (rows > kStaticMaxRows) {

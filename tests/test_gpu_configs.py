@@ -1,8 +1,10 @@
-"""The five benchmark workloads at full size on the GPU, against the oracle.
+"""The five benchmark workloads at full size on the GPU, against the oracle, every element of every
+fetched tensor.
 
-Where the oracle cannot evaluate the whole tensor in seconds, it is evaluated on sampled elements
-(elementwise graphs) or sampled rows (row-reduction graph: rows are independent), and reductions
-over all elements are checked at full size where the oracle can afford it."""
+The two random graphs are too large for one pass of the NumPy interpreter, so the oracle runs over
+chunks of the leading axis on the host's cores (oracle/chunked.py: elements of an elementwise graph and
+rows of a row-reduction graph are independent; sums over that axis add up in fp64) and each chunk is
+compared where it is computed."""
 import json
 import os
 
@@ -10,10 +12,10 @@ import numpy as np
 import pytest
 import torch
 
-from oracle import interp, prune as oprune
+from oracle import chunked, interp, prune as oprune
 from paper_1707_08265_b200 import binding as B
 from paper_1707_08265_b200 import workloads as wl
-from test_gpu_vm import run_gpu, check, TOL32, TOLBF, to_dev
+from test_gpu_vm import run_gpu, check, TOL32, TOLBF, to_dev, FLOOR_OK, C_COND
 
 pytestmark = pytest.mark.gpu
 SEEDS = json.load(open(os.path.join(os.path.dirname(__file__), "golden", "config_seeds.json")))
@@ -69,17 +71,17 @@ def test_config3_random_elementwise_dag_full_size():
     f.run_torch([t if u else None for t, u in zip(gpu_in, f.used_inputs())], outs)
     assert f.status() == 0
     torch.cuda.synchronize()
-    # elementwise graph: the oracle evaluates a sample of positions (several whole tiles, the tail,
-    # and scattered elements) on the very same input values
-    rng = np.random.default_rng(0)
-    idx = np.unique(np.concatenate([np.arange(0, 3 * 4096), np.arange(n - 4099, n), rng.integers(0, n, 1 << 18)]))
-    tidx = torch.from_numpy(idx).cuda()
-    sample = [t[tidx].cpu().numpy() for t in gpu_in]
-    gs, _, fs = wl.random_dag(idx.size, seed)
-    ref = interp.run_function(gs.desc, inputs, fs, sample)
-    for o, r in zip(outs, ref):
+    for o in outs:
         assert torch.isfinite(o).all()
-        check(o[tidx].cpu().numpy().astype(np.float64), r, TOL32, "config 3")
+    # every element, in chunks of 2^21 over the host's cores, on the very same input values
+    host_in = [t.cpu().numpy() if u else None for t, u in zip(gpu_in, f.used_inputs())]
+    host_out = [o.cpu().numpy() for o in outs]
+    res = chunked.run_chunked(g.desc, inputs, fetch, host_in, n, 1 << 21, compare=host_out, tol=TOL32, with_floor=True)
+    for e, t in zip(res, fetch):
+        allowed = 1.0 if e[6] <= FLOOR_OK else C_COND * e[6]      # see test_gpu_vm.check_conditioned
+        print("config 3 tensor %d: worst error %.3g tolerances, CPU fp32 floor over all elements %.3g" % (t, e[1], e[6]))
+        assert e[0] == "err" and e[1] <= allowed, "config 3 tensor %d: worst normalised error %.3g at element %d (got %r ref %r, floor %.3g)" % (
+            t, e[1], e[2] + e[3], e[4], e[5], e[6])
 
 
 def test_config4_mlp_full_size():
@@ -119,27 +121,24 @@ def test_config5_row_dag_full_size():
     f.run_torch([t if u else None for t, u in zip(gpu_in, f.used_inputs())], outs)
     assert f.status() == 0
     torch.cuda.synchronize()
-    # rows are independent (row sums stay inside a row): the oracle evaluates a subset of rows on
-    # the same values; FULL-shaped outputs of those rows must match
-    pick = np.unique(np.concatenate([[0, 1, rows - 1], np.random.default_rng(1).integers(0, rows, 29)]))
-    sub_feeds = [t[torch.from_numpy(pick).cuda()].cpu().numpy() if t.dim() == 2 else t.cpu().numpy() for t in gpu_in]
-    gs, in_s, fetch_s = wl.random_row_dag(len(pick), cols, seed)
-    grads_s = gs.grad(fetch_s, wrts)
-    ref = interp.run_function(gs.desc, in_s, fetch_s + grads_s, sub_feeds)
-    for o, r, t in zip(outs, ref, outs_ids):
+    for o in outs:
         assert torch.isfinite(o).all()
-        if o.dim() == 2:
-            check(o[torch.from_numpy(pick).cuda()].cpu().numpy().astype(np.float64), r, TOL32, "config 5 tensor %d" % t)
-    # gradients of the [cols] inputs sum over all rows: checked against the oracle on a reduced row
-    # count (the first 256 rows of the same inputs), where the oracle can afford every row
-    r2 = 256
-    g2, in2, fetch2 = wl.random_row_dag(r2, cols, seed)
-    grads2 = g2.grad(fetch2, wrts)
-    small_in = [t[:r2].contiguous() if t.dim() == 2 else t for t in gpu_in]
-    f2 = B.Graph.from_desc(g2.desc).function(in2, fetch2 + grads2)
-    outs2 = [torch.full(tuple(g2.shape(o)), float("nan"), dtype=torch.float32, device="cuda") for o in fetch2 + grads2]
-    f2.run_torch([t if u else None for t, u in zip(small_in, f2.used_inputs())], outs2)
-    torch.cuda.synchronize()
-    ref2 = interp.run_function(g2.desc, in2, fetch2 + grads2, [t.cpu().numpy() for t in small_in])
-    for o, r, t in zip(outs2, ref2, fetch2 + grads2):
-        check(o.cpu().numpy().astype(np.float64), r, TOL32, "config 5 (256 rows) tensor %d" % t)
+    # rows are independent (row sums stay inside a row): the oracle runs over all 16384 rows in chunks of
+    # 256 on the host's cores.  FULL-shaped outputs are compared chunk by chunk; the gradients of the
+    # [cols] inputs are column sums over all rows: the chunks' shares are added in fp64 and compared whole.
+    host_in = [t.cpu().numpy() if u else None for t, u in zip(gpu_in, f.used_inputs())]
+    host_out = [o.cpu().numpy() if o.dim() == 2 else None for o in outs]
+    res = chunked.run_chunked(g.desc, inputs, outs_ids, host_in, rows, 256, compare=host_out, tol=TOL32, with_floor=True)
+    n_sums = 0
+    for e, o, t in zip(res, outs, outs_ids):
+        if e[0] == "err":
+            # over 2^26 elements the tail of fp32 rounding shows: a tensor on which NumPy's own fp32 evaluation
+            # leaves the tolerance somewhere is held to C_COND times that floor (test_gpu_vm.check_conditioned)
+            allowed = 1.0 if e[6] <= FLOOR_OK else C_COND * e[6]
+            print("config 5 tensor %d: worst error %.3g tolerances, CPU fp32 floor over all rows %.3g" % (t, e[1], e[6]))
+            assert e[1] <= allowed, "config 5 tensor %d: worst normalised error %.3g in the chunk at row %d, offset %d (got %r ref %r, floor %.3g)" % (
+                t, e[1], e[2], e[3], e[4], e[5], e[6])
+        else:
+            n_sums += 1
+            check(o.cpu().numpy().astype(np.float64), e[1], TOL32, "config 5 column sums over all rows, tensor %d" % t)
+    assert n_sums == sum(1 for w in wrts if len(g.shape(w)) == 1)

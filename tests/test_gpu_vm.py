@@ -82,15 +82,33 @@ def test_toy_gradients(n):
     assert np.array_equal(got2[1], got[0])
 
 
-def fp32_floor(desc, inputs, outputs, feeds):
+FLOOR_OK = 0.25   # CPU fp32 evaluation within a quarter of the tolerance: the tensor is held to the tolerance itself
+C_COND = 16.0     # otherwise (floor f, in tolerances): held to C_COND * f tolerances
+
+
+def fp32_floors(desc, inputs, outputs, feeds):
+    """Per fetched tensor: how far the oracle's own arithmetic, instantiated in fp32 on the CPU (same plain
+    loop, NumPy float32), lands from its fp64 result, in units of the tolerance.  A value above 1 says that
+    the graph amplifies fp32 rounding beyond 1e-5 whatever evaluates it; such a tensor cannot be held to
+    the plain tolerance, and is held to C_COND times its floor instead of not being compared at all."""
     ref = interp.run_function(desc, inputs, outputs, feeds)
     low = interp.run_function(desc, inputs, outputs, feeds, dtype=np.float32)
-    worst = 0.0
+    floors = []
     for r, l in zip(ref, low):
-        if not np.all(np.isfinite(r)):
-            return np.inf, ref
-        worst = max(worst, float(np.max(np.abs(l.astype(np.float64) - r) / (TOL32 * (1 + np.abs(r))))))
-    return worst, ref
+        assert np.all(np.isfinite(r)), "the fp64 reference itself is not finite"
+        floors.append(float(np.max(np.abs(l.astype(np.float64) - r) / (TOL32 * (1 + np.abs(r))))))
+    return floors, ref
+
+
+def check_conditioned(got, ref, floors, what):
+    """Every tensor against the oracle: at the tolerance where fp32 can reach it (floor <= FLOOR_OK), else
+    at C_COND * floor tolerances.  Returns the number of tensors held to the plain tolerance."""
+    tight = 0
+    for k, (gv, rv, fl) in enumerate(zip(got, ref, floors)):
+        scale = 1.0 if fl <= FLOOR_OK else C_COND * fl
+        tight += scale == 1.0
+        check(gv, rv, TOL32 * scale, "%s tensor %d (fp32 floor %.3g)" % (what, k, fl))
+    return tight
 
 
 @pytest.mark.parametrize("seed", range(24))
@@ -98,14 +116,11 @@ def test_random_elementwise_dags(seed):
     n = 2 * 4096 + 77
     g, inputs, fetch = wl.random_dag(n, 1000 + seed, n_ops=64)
     feeds = wl.normal_feeds([[n]] * 4, 2000 + seed)
-    floor, ref = fp32_floor(g.desc, inputs, fetch, feeds)
+    floors, ref = fp32_floors(g.desc, inputs, fetch, feeds)
     got, f = run_gpu(g.desc, inputs, fetch, feeds)
     want = oprune.function_sets(g.desc, inputs, fetch)
     assert f.marked() == want["marked"] and f.kept_ops()[0] == want["fwd_ops"]
-    if floor > 0.25:
-        pytest.skip("graph is ill-conditioned in fp32 on the CPU as well (floor %.3g)" % floor)
-    for gv, rv in zip(got, ref):
-        check(gv, rv, TOL32, "seed %d" % seed)
+    check_conditioned(got, ref, floors, "seed %d" % seed)
 
 
 @pytest.mark.parametrize("op", ["Add", "Sub", "Mul", "Div", "Sin", "Exp", "Tanh", "Sigmoid", "ReLU"])
@@ -162,15 +177,12 @@ def test_random_row_dags_with_gradients(seed):
     shapes = [g.shape(i) for i in inputs]
     feeds = [a * np.float32(0.5) for a in wl.normal_feeds(shapes, 4000 + seed)]
     outs = fetch + grads
-    floor, ref = fp32_floor(g.desc, inputs, outs, feeds)
+    floors, ref = fp32_floors(g.desc, inputs, outs, feeds)
     got, f = run_gpu(g.desc, inputs, outs, feeds)
     want = oprune.function_sets(g.desc, inputs, outs)
     fwd, gops, masks = f.kept_ops()
     assert f.marked() == want["marked"] and fwd == want["fwd_ops"] and gops == [k for (_, k, _) in want["grad_ops"]]
-    if floor > 0.25:
-        pytest.skip("graph is ill-conditioned in fp32 on the CPU as well (floor %.3g)" % floor)
-    for gv, rv, o in zip(got, ref, outs):
-        check(gv, rv, TOL32, "seed %d tensor %d" % (seed, o))
+    check_conditioned(got, ref, floors, "seed %d" % seed)
 
 
 def test_register_pressure_spills_to_shared_and_global():

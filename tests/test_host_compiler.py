@@ -238,3 +238,41 @@ def test_many_reduced_outputs_fit_the_finishing_launch_or_are_refused(n_scalars)
         want = float(np.sum(np.sin(feeds[0]) if k % 2 else np.tanh(feeds[0])))
         kind, accidx, pos = step["reduced"][[r[2] for r in step["reduced"]].index(k)]
         assert kind == 1 and abs(scal[accidx] - want) <= 1e-9 * (1 + abs(want)), (k, scal[accidx], want)
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_multi_output_operators_are_pruned_by_the_library_like_by_the_oracle(seed):
+    """Sec. 2.2: an operator connects each of its inputs to each of its outputs.  Tiny DAGs with one- and
+    two-output opaque operators and one or two gradient stages, replayed through the C ABI: marks, kept
+    operators, masks and used inputs equal the oracle's (which is itself pinned by path enumeration); a
+    function that keeps an opaque operator compiles and refuses to run."""
+    from test_oracle_prune import tiny_dag_with_stages
+    rng = np.random.default_rng(9000 + seed)
+    d, fetch = tiny_dag_with_stages(rng)
+    f = compare_sets(d, [0, 1, 2], fetch)
+    if f.kept_ops()[0]:
+        assert "not executable" in f.describe() and f.num_launches() == 0
+        with pytest.raises(B.DragonError) as e:
+            f.run([0, 0, 0], [0] * len(fetch))
+        assert e.value.code == B.ERR_UNSUPPORTED and "opaque" in str(e.value)
+
+
+def test_an_opaque_operator_that_is_pruned_away_does_not_stop_execution():
+    g = B.Graph()
+    x = g.add_tensor("x", B.F32, [100])
+    y = g.add_tensor("y", B.F32, [100])
+    u = g.add_tensor("u", B.F32, [7])
+    v = g.add_tensor("v", B.F32, [3, 3])
+    g.add_op(B.OPS["Tanh"], [x], [y])
+    g.add_op(B.OPS["Opaque"], [x, y], [u, v])                  # two outputs of arbitrary declared shapes
+    f = g.function([x], [y])
+    assert f.kept_ops()[0] == [0] and f.marked() == [1, 1, 0, 0] and "vm[" in f.describe()
+    f2 = g.function([x], [v])
+    assert f2.kept_ops()[0] == [0, 1] and f2.marked() == [1, 1, 0, 1]     # u is an un-colored output of a kept operator
+    with pytest.raises(B.DragonError) as e:
+        g.add_op(B.OPS["Tanh"], [x], [u, v])                   # executable types have one output
+    assert e.value.code == B.ERR_INVALID_ARG
+    w = g.add_tensor("w", B.F32, [7])
+    with pytest.raises(B.DragonError) as e:
+        g.add_op(B.OPS["Opaque"], [x], [w, w])
+    assert e.value.code == B.ERR_NOT_SSA

@@ -116,3 +116,57 @@ def test_gradient_without_path_is_rejected():
     g.grad([ids["y"]], [ids["b"]])                            # y = a*x does not depend on b
     with pytest.raises(ValueError):
         prune.function_sets(g.desc, [ids["x"], ids["a"], ids["b"]], [g.desc["grads"][0]["grad_ids"][0]])
+
+
+def tiny_dag_with_stages(rng):
+    """A tiny DAG (one- and two-output operators) with one or two gradient stages whose derivative targets
+    all have a chain to an objective, and a random set of fetched forward and gradient tensors."""
+    while True:
+        d = tiny_dag(rng, n_src=3, n_ops=int(rng.integers(3, 6)))
+        n = len(d["tensors"])
+        if n > 12:
+            continue
+        stages = []
+        for s in range(int(rng.integers(1, 3))):
+            objs = [int(t) for t in rng.choice(n, size=int(rng.integers(1, 3)), replace=False)]
+            cand = [w for w in range(n) if brute.backward_marks_bruteforce(d, set(objs), {w})]
+            if not cand:
+                break
+            wrts = [int(w) for w in rng.choice(cand, size=min(len(cand), int(rng.integers(1, 4))), replace=False)]
+            stages.append((objs, wrts))
+        else:
+            break
+    for s, (objs, wrts) in enumerate(stages):
+        gids = []
+        for w in wrts:
+            d["tensors"].append({"name": "grad%d/%d" % (s, w), "dtype": "f32", "shape": []})
+            gids.append(len(d["tensors"]) - 1)
+        d["grads"].append({"objs": objs, "wrts": wrts, "grad_ids": gids})
+    total = len(d["tensors"])
+    fetch = [int(t) for t in rng.choice(total, size=int(rng.integers(1, 4)), replace=False)]
+    return d, fetch
+
+
+@pytest.mark.parametrize("seed", range(120))
+def test_function_sets_equal_bruteforce_on_the_two_stage_dag(seed):
+    """oracle.prune.function_sets against the explicit two-stage DAG of Sec. 2.3 with every path that
+    ends in a fetched node walked edge by edge (anchor and seed edges written out): marks, kept
+    forward operators, kept gradient operators with the operand gradients they produce."""
+    rng = np.random.default_rng(7000 + seed)
+    d, fetch = tiny_dag_with_stages(rng)
+    inputs = [0, 1, 2]
+    got = prune.function_sets(d, inputs, fetch)
+    want = brute.function_sets_bruteforce(d, inputs, fetch)
+    assert got == want
+
+
+def test_bruteforce_function_sets_on_the_paper_example():
+    # the pin of the pin: fetching only df/db drops the a-side of Mul(a, x) (worked out by hand)
+    g, ids = wl.toy_function_grad(8)
+    inputs = [ids["x"], ids["a"], ids["b"]]
+    s = brute.function_sets_bruteforce(g.desc, inputs, [ids["db"]])
+    assert s["grad_ops"] == [(0, 3, (1,)), (0, 2, (0,)), (0, 1, (1,))]
+    assert s["marked"][ids["dx"]] == 0 and s["marked"][ids["da"]] == 0 and s["marked"][ids["db"]] == 1
+    assert s["fwd_ops"] == [0, 1, 2, 3] and s["used_inputs"] == [1, 1, 1]
+    s = brute.function_sets_bruteforce(g.desc, inputs, [ids["y"]])
+    assert s["fwd_ops"] == [0] and s["used_inputs"] == [1, 1, 0] and s["grad_ops"] == []

@@ -288,3 +288,40 @@ def test_fp32_instance_runs_in_float32():
     feeds = wl.normal_feeds([[64]] * 4, 3)
     outs = interp.run_function(g.desc, inputs, fetch, feeds, dtype=np.float32)
     assert all(o.dtype == np.float32 for o in outs)
+
+
+@pytest.mark.parametrize("workers", [1, 2])
+def test_chunked_evaluation_equals_the_plain_one(workers):
+    """oracle.chunked cuts the leading axis into independent chunks (rows of a row-reduction graph,
+    elements of an elementwise one); values equal the unchunked interpreter's, sums over the axis add up."""
+    from oracle import chunked, prune as oprune
+    from paper_1707_08265_b200 import workloads as wl
+    R, C = 23, 40
+    g, inputs, fetch = wl.random_row_dag(R, C, 3004, n_ops=48, n_fetch=2)
+    G = oprune.backward_marks(g.desc, fetch, inputs)
+    wrts = [i for i in inputs if i in G]
+    outs = fetch + g.grad(fetch, wrts)
+    feeds = [a * np.float32(0.5) for a in wl.normal_feeds([g.shape(i) for i in inputs], 7)]
+    ref = interp.run_function(g.desc, inputs, outs, feeds)
+    res = chunked.run_chunked(g.desc, inputs, outs, feeds, R, 5, workers=workers)
+    assert any(k == "sum" for k, *_ in res) and any(k == "val" for k, *_ in res)
+    for (kind, v), r in zip(res, ref):
+        assert np.allclose(v, r, rtol=1e-12, atol=1e-12), kind
+    # comparison mode: the reference handed in as "got" gives zero error, a planted mistake is found
+    cmp = [np.array(r) if len(np.shape(r)) == 2 else None for r in ref]
+    bad = next(k for k, c in enumerate(cmp) if c is not None)
+    cmp[bad][17, 3] += 1.0
+    res = chunked.run_chunked(g.desc, inputs, outs, feeds, R, 5, workers=workers, compare=cmp)
+    for k, e in enumerate(res):
+        if e[0] == "err":
+            assert (e[1] > 1 and e[2] == 15 and e[3] == 2 * C + 3) if k == bad else e[1] == 0.0
+            assert e[6] == 0.0          # no floor was asked for
+    # a flat elementwise graph with scalar gradients
+    n = 1000
+    g2, ids = wl.toy_function_grad(n)
+    x, a, b = wl.toy_feeds(n, 3)
+    ins, o2 = [ids["x"], ids["a"], ids["b"]], [ids["f"], ids["dx"], ids["da"], ids["db"]]
+    ref2 = interp.run_function(g2.desc, ins, o2, [x, a, b])
+    res2 = chunked.run_chunked(g2.desc, ins, o2, [x, a, b], n, 333, workers=workers)
+    for (kind, v), r in zip(res2, ref2):
+        assert np.allclose(v, r, rtol=1e-12, atol=1e-12)

@@ -34,7 +34,9 @@ def graph_loss(z, labels, dtype_name):
 def test_static_loss_matches_graph_loss_twice(dtype_name):
     tdt = torch.float32 if dtype_name == "f32" else torch.bfloat16
     gen = torch.Generator("cuda").manual_seed(11)
-    cases = [(777, 1000), (64, 4096)]          # second call: fewer rows than the first left behind
+    # second call: fewer rows than the first left behind; then a row length that is not a multiple of 8
+    # (element-wise loads), one beyond the in-register limit (looping kernel, vector loads), the row limit
+    cases = [(777, 1000), (64, 4096), (130, 1001), (33, 8200), (65536, 16)]
     for m, n in cases:
         z = (torch.randn(m, n, generator=gen, device="cuda") * 3).to(tdt)
         labels = torch.randint(0, n, (m,), generator=gen, device="cuda", dtype=torch.int32)
@@ -59,3 +61,11 @@ def test_static_loss_rejects_oversized_and_bad_arguments():
     with pytest.raises(B.DragonError) as e:
         B.softmax_ce_loss_static(0, B.F32, labels.data_ptr(), 8, 8, out.data_ptr())
     assert e.value.code == B.ERR_INVALID_ARG
+    # a view that starts 4 bytes into the buffer: refused on the host, nothing is launched
+    with pytest.raises(B.DragonError) as e:
+        B.softmax_ce_loss_static(z.data_ptr() + 4, B.F32, labels.data_ptr(), 7, 8, out.data_ptr())
+    assert e.value.code == B.ERR_INVALID_ARG and "aligned" in str(e.value)
+    with pytest.raises(B.DragonError) as e:
+        B.softmax_ce_loss_static(z.data_ptr(), B.F32, labels.data_ptr() + 2, 7, 8, out.data_ptr())
+    assert e.value.code == B.ERR_INVALID_ARG
+    torch.cuda.synchronize()
