@@ -1,11 +1,14 @@
-"""Benchmark: pruned-graph forward + generated backward of f = x*sin(a*x+b), elements/s.
+"""Benchmark: pruned-graph forward + generated backward, elements/s, on the five synthetic workloads.
 
-One step = one pass of the whole hot path over one batch: the compiled function that fetches
-df/dx (per element), df/da and df/db (summed over all elements) runs once over x fp32[2^26]
-(per GPU).  Timed with CUDA events on the launching stream; the input (256 MiB) plus the output
-(256 MiB) exceed the L2, so every step streams from HBM.
+The headline line is workload 2: f = x*sin(a*x+b) over x fp32[2^26] (per GPU), fetching df/dx (per
+element), df/da and df/db (summed over all elements).  One step = one pass of the whole hot path over
+one batch = one dragon_run().  Timed with CUDA events on the launching stream; input (256 MiB) plus
+output (256 MiB) exceed the L2, so every step streams from HBM.  The same JSON line carries, under
+"configs", the other four workloads (1: the forward-only toy function at 2^20, 3: the random
+64-operator elementwise DAG at 2^27, 4: the bf16 MLP forward + backward, 5: the random 1024-operator
+row DAG at [16384, 4096] forward + backward), each with its own roofline entry.
 
-  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config k]
 """
 import argparse
 import json
@@ -27,17 +30,20 @@ METRIC = "pruned-graph fwd+bwd elements/sec"
 UNIT = "elements/s"
 WORKLOAD = "config 2: f=x*sin(a*x+b), x fp32[2^26], fetch df/dx, df/da, df/db"
 ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
-# dram__bytes_read.sum + dram__bytes_write.sum of the VM kernel per element, from one ncu capture of this
-# kernel binary on this workload at 2^25 elements (traffic is proportional to the element count); None once the
-# kernel has changed since the counters were taken
-NCU_DRAM_BYTES_PER_ELEM = (134.344448e6 + 89.499136e6) / (1 << 25)
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the VM kernel on this workload at the full 2^26
+# elements, from one ncu capture of this kernel binary (profiles/vm_dense_config2.md); None once the kernel has
+# changed since the counters were taken
+NCU_DRAM_BYTES_PER_LAUNCH = None
+SAMPLE_ELEMS = 1 << 21       # the CPU oracle's bounded sample of workload 2, per pass
 
 
-def measured_peak_gbs():
+def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
-        return float(json.load(open(p))["hbm_gbs"]), "measured"
-    return 6650.0, "fallback"
+        d = json.load(open(p))
+        return {"hbm": float(d["hbm_gbs"]), "bf16": float(d["bf16_tflops"]), "bf16_sustained": float(d["bf16_tflops_sustained"]),
+                "kind": "of measured"}
+    return {"hbm": 6650.0, "bf16": 1590.0, "bf16_sustained": 1400.0, "kind": "of fallback"}
 
 
 class ClockSampler(threading.Thread):
@@ -79,116 +85,244 @@ class ClockSampler(threading.Thread):
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons)}
 
 
-def oracle_rate(seconds_budget=12.0):
-    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+# ---- the CPU oracle, timed as it stands ---------------------------------------------------------
+
+def oracle_workload():
+    g, ids = wl.toy_function_grad(SAMPLE_ELEMS)
+    x, a, b = wl.toy_feeds(SAMPLE_ELEMS, wl.BASE_SEED + 2)
+    return g, [ids["x"], ids["a"], ids["b"]], [ids["dx"], ids["da"], ids["db"]], [x, a, b]
+
+
+def oracle_single(seconds_budget):
+    """One core: passes of the fp64 NumPy interpreter over x[2^21] of the same graph, same fetches."""
     from oracle import interp
-    n = 1 << 21
-    g, ids = wl.toy_function_grad(n)
-    x, a, b = wl.toy_feeds(n, wl.BASE_SEED + 2)
-    inputs = [ids["x"], ids["a"], ids["b"]]
-    outs = [ids["dx"], ids["da"], ids["db"]]
-    interp.run_function(g.desc, inputs, outs, [x, a, b])
+    g, inputs, outs, feeds = oracle_workload()
+    interp.run_function(g.desc, inputs, outs, feeds)
     reps, t0 = 0, time.perf_counter()
     while True:
-        interp.run_function(g.desc, inputs, outs, [x, a, b])
+        interp.run_function(g.desc, inputs, outs, feeds)
         reps += 1
         if time.perf_counter() - t0 > seconds_budget or reps >= 64:
             break
     dt = time.perf_counter() - t0
-    return reps * n / dt, "%d passes of the fp64 NumPy interpreter over x[2^21] (same graph, same fetches)" % reps, dt / reps
+    return SAMPLE_ELEMS * reps / dt, reps, dt / reps
+
+
+CHUNK_ELEMS = 1 << 19
+
+
+class OraclePool:
+    """All host cores: the same interpreter over chunks of the element range (oracle/chunked.py), one worker
+    thread per core (NumPy releases the interpreter lock inside its loops, and threads hand their results
+    back without copying them between processes)."""
+
+    def __init__(self):
+        from multiprocessing.pool import ThreadPool
+        from oracle import chunked
+        self.chunked = chunked
+        self.cores = chunked.default_workers()
+        self.pool = ThreadPool(self.cores)
+        self.g, self.inputs, self.outs, _ = oracle_workload()
+        self.n = SAMPLE_ELEMS * self.cores
+        x, a, b = wl.toy_feeds(self.n, wl.BASE_SEED + 2)
+        self.desc = chunked.with_leading_extent(self.g.desc, SAMPLE_ELEMS, self.n)
+        self.feeds = [x, a, b]
+        self.one_pass()     # first touch of every buffer outside the timed passes
+
+    def one_pass(self):
+        """One pass over cores x 2^21 elements in chunks of 2^19; returns seconds."""
+        t0 = time.perf_counter()
+        self.chunked.run_chunked(self.desc, self.inputs, self.outs, self.feeds, self.n, CHUNK_ELEMS, pool=self.pool)
+        return time.perf_counter() - t0
+
+    def close(self):
+        self.pool.close()
+        self.pool.join()
+
+
+def cpu_baseline(seconds_budget=10.0):
+    single, reps, _ = oracle_single(seconds_budget / 2)
+    pool = OraclePool()
+    passes, t0 = 0, time.perf_counter()
+    while True:
+        pool.one_pass()
+        passes += 1
+        if time.perf_counter() - t0 > seconds_budget / 2 or passes >= 16:
+            break
+    dt = time.perf_counter() - t0
+    rate = pool.n * passes / dt
+    sample = "%d passes of the fp64 NumPy interpreter over x[%d x 2^21] in chunks of 2^19 on %d worker threads (same graph, same fetches)" % (
+        passes, pool.cores, pool.cores)
+    out = {"value": rate, "unit": UNIT, "cores": pool.cores, "kind": "oracle", "sample": sample, "host_cores": os.cpu_count(),
+           "single_thread": {"value": single, "unit": UNIT, "cores": 1, "sample": "%d passes over x[2^21]" % reps}}
+    pool.close()
+    return out
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
-    if rank != 0:
+    """The reference arm: the oracle on the host cores; a step = one pass over the bounded sample."""
+    if int(os.environ.get("RANK", "0")) != 0:
         return
-    per = []
+    pool = OraclePool()
     for _ in range(args.warmup):
-        oracle_rate(0.5)
+        pool.one_pass()
+    steps = max(1, args.steps)
     t0 = time.perf_counter()
-    sample = ""
-    for _ in range(args.steps):
-        rate, sample, _ = oracle_rate(max(1.0, 60.0 / max(1, args.steps)))
-        per.append(rate)
+    for _ in range(steps):
+        pool.one_pass()
     dt = time.perf_counter() - t0
-    value = float(np.mean(per))
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
-            "warmup": args.warmup, "ms_per_step": 1e3 * dt / max(1, args.steps), "higher_is_better": True, "scaling": "weak",
+    value = pool.n * steps / dt
+    sample = "each step is one pass of the fp64 NumPy interpreter over x[%d x 2^21] in chunks of 2^19 on %d worker threads" % (pool.cores, pool.cores)
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * dt / steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "note": "each step is a bounded sample: " + sample},
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "config": {"workload": WORKLOAD, "note": "bounded sample: " + sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": pool.cores, "kind": "oracle", "sample": sample, "host_cores": os.cpu_count()},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    pool.close()
     print(json.dumps(line), flush=True)
 
 
-def run_other_config(args):
-    """Device-resident timing of the other workloads (same step definition: one dragon_run)."""
-    import torch
-    from paper_1707_08265_b200 import binding as B
-    seeds = json.load(open(os.path.join(ROOT, "tests", "golden", "config_seeds.json")))
-    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32}
-    gen = torch.Generator("cuda").manual_seed(wl.BASE_SEED + args.config)
+# ---- the other workloads ------------------------------------------------------------------------
 
-    def dev_random(g, t):
+def connected_inputs(B, desc, objs, inputs):
+    """The inputs that have a chain to an objective, asked of the library: dragon_add_grad refuses a
+    derivative target without one (DRAGON_ERR_NO_PATH)."""
+    g = B.Graph.from_desc(desc)
+    keep = []
+    for i in inputs:
+        try:
+            g.add_grad(objs, [i])
+            keep.append(i)
+        except B.DragonError as e:
+            if e.code != B.ERR_NO_PATH:
+                raise
+    return keep
+
+
+def build_config(cfg, B, torch, seeds):
+    """-> dict(g, inputs, outputs, units, what, and the roofline's numerator)"""
+    MiB = 1 << 20
+    if cfg == 1:
+        n = 1 << 20
+        g, ids = wl.toy_function(n)
+        return dict(g=g, inputs=[ids["x"], ids["a"], ids["b"]], outputs=[ids["f"], ids["y"]], units=n, unit=UNIT, bound="hbm",
+                    alg=12.0 * n, what="config 1: f and y of x*sin(a*x+b), x fp32[2^20], forward (12 B/element; fits the L2)")
+    if cfg == 3:
+        n = 1 << 27
+        g, inputs, outputs = wl.random_dag(n, seeds["random_dag"]["seed"])
+        return dict(g=g, inputs=inputs, outputs=outputs, units=n, unit=UNIT, bound="hbm", alg=None,
+                    what="config 3: random 64-operator elementwise DAG, 4 x fp32[2^27], 2 fetched sinks, forward")
+    if cfg == 6:   # not one of the five: the SGD weight update as a graph of its own, 12 bytes per element
+        n = 1 << 26
+        g, ids = wl.updater([n], "sgd")
+        return dict(g=g, inputs=[ids["W"], ids["g"], ids["lr"]], outputs=[ids["W_new"]], units=n, unit=UNIT, bound="hbm", alg=12.0 * n,
+                    what="SGD updater W - lr*g, fp32[2^26] (12 B/element)")
+    if cfg == 4:
+        g, ids = wl.mlp(8192, 4096, 4096, 4096)
+        return dict(g=g, inputs=[ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")],
+                    outputs=[ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")], units=8192, unit="batch rows/s", bound="tensor",
+                    alg=5 * 2.0 * 8192 * 4096 * 4096, what="config 4: MLP 8192 x 4096-4096-4096 bf16, forward + backward (5 contractions survive the prunes)")
+    g, inputs, fetch = wl.random_row_dag(16384, 4096, seeds["random_row_dag"]["seed"])
+    if cfg == 5:
+        wrts = connected_inputs(B, g.desc, fetch, inputs)
+        outputs = fetch + g.grad(fetch, wrts)
+        what = "config 5: random 1024-operator row DAG on [16384,4096], forward + backward to every connected input"
+    else:   # 7, not one of the five: the same DAG with one gradient stage per objective (Jacobian-style fetches)
+        outputs = list(fetch)
+        for o in fetch:
+            outputs += g.grad([o], connected_inputs(B, g.desc, [o], inputs))
+        what = "row DAG on [16384,4096], forward + one gradient stage per objective (%d fetches)" % len(outputs)
+    # the workload as stated moves 6 FULL inputs, 4 FULL targets and 6 FULL gradients of 256 MiB each
+    return dict(g=g, inputs=inputs, outputs=outputs, units=16384 * 4096, unit=UNIT, bound="hbm", alg=16.0 * 256 * MiB, what=what)
+
+
+def time_config(cfg, args, B, torch, seeds, peaks, steps=None):
+    """Device-resident timing of one workload (a step = one dragon_run) plus the per-kernel times of its plan."""
+    c = build_config(cfg, B, torch, seeds)
+    g, inputs, outputs = c["g"], c["inputs"], c["outputs"]
+    tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32}
+    gen = torch.Generator("cuda").manual_seed(wl.BASE_SEED + cfg)
+
+    def dev_random(t):
         ti = g.desc["tensors"][t]
         if ti["dtype"] == "i32":
             return torch.randint(0, 4096, tuple(ti["shape"]), generator=gen, device="cuda", dtype=torch.int32)
         return torch.empty(tuple(ti["shape"]), dtype=torch.float32, device="cuda").normal_(generator=gen).to(tdt[ti["dtype"]])
 
-    if args.config == 1:
-        n = 1 << 20
-        g, ids = wl.toy_function(n)
-        inputs, outputs, units, what = [ids["x"], ids["a"], ids["b"]], [ids["f"], ids["y"]], n, "f and y of x*sin(a*x+b), x fp32[2^20] (L2-resident)"
-    elif args.config == 3:
-        n = 1 << 27
-        g, inputs, outputs = wl.random_dag(n, seeds["random_dag"]["seed"])
-        units, what = n, "random 64-operator elementwise DAG, 4 x fp32[2^27], 2 fetches"
-    elif args.config == 6:   # not one of the five: the SGD weight update as a graph of its own, 12 bytes per element
-        n = 1 << 26
-        g, ids = wl.updater([n], "sgd")
-        inputs, outputs, units, what = [ids["W"], ids["g"], ids["lr"]], [ids["W_new"]], n, "SGD updater W - lr*g, fp32[2^26] (memory-bound: 12 B/element)"
-    elif args.config == 4:
-        g, ids = wl.mlp(8192, 4096, 4096, 4096)
-        inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")]
-        outputs = [ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")]
-        units, what = 8192, "MLP 8192 x 4096-4096-4096 bf16, forward + backward (batch rows per step)"
-    else:
-        from oracle import prune as oprune   # which inputs are connected is decided outside the generator
-        g, inputs, fetch = wl.random_row_dag(16384, 4096, seeds["random_row_dag"]["seed"])
-        if args.config == 5:
-            G = oprune.backward_marks(g.desc, fetch, inputs)
-            outputs = fetch + g.grad(fetch, [i for i in inputs if i in G])
-            units, what = 16384 * 4096, "random 1024-operator row DAG on [16384,4096], forward + backward"
-        else:   # not one of the five: the same DAG with one gradient stage per objective (Jacobian-style fetches)
-            outputs = list(fetch)
-            for o in fetch:
-                G = oprune.backward_marks(g.desc, [o], inputs)
-                outputs += g.grad([o], [i for i in inputs if i in G])
-            units, what = 16384 * 4096, "row DAG on [16384,4096], forward + one gradient stage per objective (%d fetches)" % len(outputs)
     f = B.Graph.from_desc(g.desc).function(inputs, outputs)
-    feeds = [dev_random(g, t) if u else None for t, u in zip(inputs, f.used_inputs())]
-    if args.config == 4:
-        for j in (1, 2, 3, 4):
+    feeds = [dev_random(t) if u else None for t, u in zip(inputs, f.used_inputs())]
+    if cfg == 4:
+        for j in (1, 2, 3, 4):     # weights and biases ~ N(0, 1/4096)
             feeds[j] = (feeds[j].float() / 64).to(torch.bfloat16)
     outs = [torch.empty(tuple(g.shape(t)), dtype=tdt[g.desc["tensors"][t]["dtype"]], device="cuda") for t in outputs]
-    for _ in range(max(3, args.warmup)):
-        f.run_torch(feeds, outs)
-    torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    steps = min(args.steps, 50)
-    e0.record()
-    for _ in range(steps):
-        f.run_torch(feeds, outs)
-    e1.record()
-    torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / steps
-    assert f.status() == 0
-    nbytes = sum(t.numel() * t.element_size() for t in feeds if t is not None) + sum(t.numel() * t.element_size() for t in outs)
-    line = {"config": args.config, "workload": what, "ms_per_step": ms, "units_per_s": units / (ms * 1e-3),
-            "io_GBps": nbytes / ms / 1e6, "launches": f.num_launches(), "plan": f.describe().strip().split("\n")[:24]}
-    if args.config == 4:
-        line["gemm_TFLOPs_over_whole_step"] = 5 * 2 * 8192 * 4096 * 4096 / ms / 1e9
-    print(json.dumps(line), flush=True)
+    steps = steps or min(args.steps, 50)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        for _ in range(max(3, args.warmup)):
+            f.run_torch(feeds, outs, stream)
+        stream.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            f.run_torch(feeds, outs, stream)
+        e1.record(stream)
+        stream.synchronize()
+        ms = e0.elapsed_time(e1) / steps
+        assert f.status() == 0
+        # per-kernel times: CUDA events around every step of the plan (the library records them on the launching stream)
+        plan = f.describe().strip().split("\n")
+        plan = [l for l in plan if not l.startswith("  code:")]
+        kern = []
+        for si in range(len(plan)):
+            f.profile(si, 8)
+            for _ in range(8):
+                f.run_torch(feeds, outs, stream)
+            tot, runs = f.profile_read()
+            kern.append(tot / max(1, runs))
+        f.profile(-1, 0)
+        flushed = None
+        if cfg == 1:   # the working set fits the L2: also with an L2-flushing write (256 MiB) before every run
+            scratch = torch.empty(1 << 28, dtype=torch.uint8, device="cuda")
+            f.profile(0, 16)
+            for _ in range(16):
+                scratch.fill_(1)
+                f.run_torch(feeds, outs, stream)
+            tot, runs = f.profile_read()
+            f.profile(-1, 0)
+            flushed = tot / max(1, runs)
+            del scratch
+    io_bytes = sum(t.numel() * t.element_size() for t in feeds if t is not None) + sum(t.numel() * t.element_size() for t in outs)
+    fwd, gops, _ = f.kept_ops()
+    top = int(np.argmax(kern))
+    line = {"workload": c["what"], "ms_per_step": ms, "value": c["units"] / (ms * 1e-3), "unit": c["unit"], "steps": steps,
+            "launches_per_step": f.num_launches(), "kept_forward_ops": len(fwd), "kept_gradient_ops": len(gops), "ops_in_graph": f.n_ops,
+            "fed_and_fetched_bytes": io_bytes, "plan": plan[:16], "kernel_ms": [round(k, 5) for k in kern[:16]]}
+    if c["bound"] == "hbm":
+        alg = c["alg"] if c["alg"] is not None else float(io_bytes)
+        k_ms = sum(kern) if cfg != 1 else kern[0]
+        ach = alg / (k_ms * 1e-3) / 1e9
+        line["roofline"] = {"bound": "hbm", "kernel": plan[top].split("[")[0] + (" dense" if " dense " in plan[top] else " wide" if " wide " in plan[top] else ""),
+                            "achieved": ach, "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"], "peak_kind": peaks["kind"],
+                            "algorithmic_bytes": alg, "kernel_ms": k_ms, "traffic": None, "frac_of_nominal_8TBs": ach / 8000.0,
+                            "frac_on_fed_and_fetched_bytes": io_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm"]}
+        if cfg == 1:
+            line["roofline"]["note"] = "L2-warm (back-to-back runs, 12.6 MB working set in the 126 MB L2); kernel time under an L2-flushing 256 MiB write before every run: ms_l2_flushed"
+            line["ms_l2_flushed"] = flushed
+            line["roofline"]["frac_l2_flushed"] = alg / (flushed * 1e-3) / 1e9 / peaks["hbm"]
+        if cfg == 5 or cfg == 7:
+            line["roofline"]["note"] = "not HBM-bound: one interpreter launch of a few hundred instructions per row with many row sums (CTA barriers); the HBM fraction is reported as asked"
+    else:
+        whole = c["alg"] / (ms * 1e-3) / 1e12
+        gemm = [k for k, p in zip(kern, plan) if p.startswith("gemm")]
+        best = c["alg"] / 5 / (min(gemm) * 1e-3) / 1e12
+        line["roofline"] = {"bound": "tensor", "kernel": "gemm_bf16_tcgen05", "achieved": whole, "peak": peaks["bf16_sustained"], "unit": "TFLOP/s",
+                            "frac": whole / peaks["bf16_sustained"], "peak_kind": peaks["kind"] + " (sustained: the contractions run back to back inside a long step)",
+                            "flops": c["alg"], "traffic": None, "gemm_launch_ms": [round(k, 5) for k in gemm],
+                            "fastest_gemm_alone_TFLOPs": best, "fastest_gemm_frac_of_burst_peak": best / peaks["bf16"]}
+    del feeds, outs, f
+    torch.cuda.empty_cache()
+    return line
 
 
 def main():
@@ -199,17 +333,26 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU (default: the benchmark's 2^26)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
+    ap.add_argument("--skip-other-configs", action="store_true", help="leave the \"configs\" entry (workloads 1, 3, 4, 5) out")
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7],
-                    help="2 (default) is the benchmark workload; the others print one summary line each (6: SGD updater)")
+                    help="2 (default) is the benchmark workload with all five on its line; another number prints that workload alone "
+                         "(6: SGD updater, 7: one gradient stage per objective)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
-    if args.config != 2:
-        return run_other_config(args)
 
     import torch
     import torch.distributed as dist
     from paper_1707_08265_b200 import binding as B
+    seeds = json.load(open(os.path.join(ROOT, "tests", "golden", "config_seeds.json")))
+    peaks = measured_peaks()
+
+    if args.config != 2:
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        line = time_config(args.config, args, B, torch, seeds, peaks)
+        line["config"] = args.config
+        print(json.dumps(line), flush=True)
+        return
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -302,26 +445,35 @@ def main():
     assert f.status() == 0
     # the host copies came back: a cheap end-to-end sanity check against the device-resident run
     assert np.array_equal(h_out[0][:1024].numpy(), d_out[0][:1024].cpu().numpy())
+    plan = f.describe().strip().split("\n")
+    launches = f.num_launches()
+    del stg, d_feeds, d_out, h_x, h_out
+    torch.cuda.empty_cache()
+
+    others = {}
+    if world == 1 and not args.skip_other_configs:
+        for cfg in (1, 3, 4, 5):
+            others[str(cfg)] = time_config(cfg, args, B, torch, seeds, peaks)
 
     if rank == 0:
-        peak, peak_kind = measured_peak_gbs()
         kern_avg_ms = kern_ms / max(1, kern_runs)
         achieved = ALG_BYTES_PER_ELEM * n / (kern_avg_ms * 1e-3) / 1e9
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
                 "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "elements_per_gpu": n, "l2": "inputs+outputs (512 MiB) larger than L2",
-                           "plan": f.describe().strip().split("\n")},
+                "config": {"workload": WORKLOAD, "elements_per_gpu": n, "l2": "inputs+outputs (512 MiB) larger than L2", "plan": plan},
                 "clocks": sampler.summary(),
                 "e2e": {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                         "h2d_bytes_per_step": 4 * n + 8, "d2h_bytes_per_step": 4 * n + 8},
-                "gpu_launches": f.num_launches() * args.steps,
-                "roofline": {"bound": "hbm", "kernel": "dragon_vm_dense", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                             "frac": achieved / peak, "peak_kind": "of " + peak_kind, "traffic": None if NCU_DRAM_BYTES_PER_ELEM is None else NCU_DRAM_BYTES_PER_ELEM * n,
+                "gpu_launches": launches * args.steps,
+                "roofline": {"bound": "hbm", "kernel": "dragon_vm_dense", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                             "frac": achieved / peaks["hbm"], "peak_kind": peaks["kind"],
+                             "traffic": NCU_DRAM_BYTES_PER_LAUNCH if n == N_ELEMS else None,
                              "kernel_ms": kern_avg_ms, "frac_of_nominal_8TBs": achieved / 8000.0}}
+        if others:
+            line["configs"] = others
         if not args.skip_cpu_baseline and world == 1:
-            rate, sample, _ = oracle_rate()
-            line["cpu_baseline"] = {"value": rate, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample}
+            line["cpu_baseline"] = cpu_baseline()
         print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

@@ -4,7 +4,7 @@
 //   sin/cos : two-constant Cody-Waite reduction by pi/2 (fused multiply-adds) up to 2^20, an exact
 //             multi-word reduction beyond; odd/even polynomials on [-pi/4, pi/4]
 //   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), n added to the exponent
-//   tanh    : x*P(x^2)/Q(x^2) on |x| <= 9, clamped
+//   tanh    : x*P(x^2)/Q(x^2), argument clamped at 10, result at 1
 //   sigmoid : 1/(1+exp(-x))
 // Polynomial coefficients are weighted least-squares fits on Chebyshev nodes, iteratively
 // re-weighted towards the minimax error (relative errors 4e-9, 1e-10, 3e-9, 3e-9).
@@ -163,12 +163,15 @@ VM_HD float exp_wide(float x) { return exp_core(fminf(fmaxf(x, -86.0f), 88.7f));
 
 VM_HD float sigmoid_f(float x) { return f_rcp(1.0f + exp_wide(-x)); }
 
-// tanh(x) = x * P(x^2) / Q(x^2) on |x| <= 9 (beyond, tanh is 1 to the last fp32 bit): a rational
-// fit (degrees 4 and 4 in x^2, relative error 6e-8 in exact arithmetic, about 3e-7 = 5 ulp once
-// the two Horner chains and the reciprocal round); clamped to [-1, 1]; NaN stays NaN.
+// tanh(x) = x * P(x^2) / Q(x^2): a rational fit on |x| <= 9 (degrees 4 and 4 in x^2, relative error
+// 6e-8 in exact arithmetic, about 3e-7 = 5 ulp once the two Horner chains and the reciprocal round).
+// From |x| = 9.01 on tanh rounds to 1 in fp32; the fit crosses 1 at 9.07 and keeps growing (1 + 1.9e-6
+// at 10), so with the argument clamped at 10 and the result clamped to [-1, 1] a saturated tanh is
+// exactly +-1 (a gradient 1 - y^2 behind it is then exactly 0, as in wider arithmetic, instead of one
+// rounding step of y blown up by the cancellation).  NaN stays NaN.
 VM_HD float tanh_f(float x) {
   if (x != x) return x;
-  const float c = fminf(fmaxf(x, -9.0f), 9.0f);
+  const float c = fminf(fmaxf(x, -10.0f), 10.0f);
   const float z = c * c;
   float p = fmaf(z, 1.3442309683456469e-08f, 2.0679596671714183e-05f);
   p = fmaf(z, p, 3.5001979607618507e-03f);

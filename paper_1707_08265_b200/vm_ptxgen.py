@@ -494,7 +494,8 @@ class Kernel:
         return out
 
     def tanh(self, xs):
-        """x * P(x^2) / Q(x^2) on |x| <= 9 (a rational fit, about 5 ulp), clamped to [-1, 1]; NaN stays NaN"""
+        """x * P(x^2) / Q(x^2) (a rational fit on |x| <= 9, about 5 ulp; beyond 9.07 it exceeds 1), argument
+        clamped at 10 and result clamped to [-1, 1], so that a saturated tanh is exactly +-1; NaN stays NaN"""
         def clamp2(v, lim):
             out = []
             for s in self.unpack(v):
@@ -503,7 +504,7 @@ class Kernel:
                 self.e("min.NaN.f32 %s, %s, %s;" % (d, d, fc(lim)))
                 out.append(d)
             return self.pack(out[0], out[1])
-        cs = [clamp2(x, 9.0) for x in xs]
+        cs = [clamp2(x, 10.0) for x in xs]
         z = [self.mul2(c, c) for c in cs]
         k0, k1 = self.K(1.3442309683456469e-08), self.K(2.0679596671714183e-05)
         p = [self.fma2(zi, k0, k1) for zi in z]

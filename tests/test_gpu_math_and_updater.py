@@ -20,7 +20,7 @@ def sweep(lo_exp, hi_exp, per_binade=64):
 @pytest.mark.parametrize("op,lo,hi,extra", [
     ("Sin", -20, 128, [np.pi / 4, np.pi / 2, np.pi, 1e5 * np.pi, 1048576.0, 1048577.0, 6.4e6, 3.4028235e38]),   # every finite binade
     ("Exp", -20, 8, [10.0, -10.0, 9.9999, -9.9999, 10.0001, 88.0, -88.0]),   # clamp at +-10
-    ("Tanh", -20, 8, [0.6, 0.5999999, 0.6000001, 9.0, 20.0, 21.0, 90.0]),    # polynomial below 0.6
+    ("Tanh", -20, 8, [0.6, 0.5999999, 0.6000001, 9.0, 9.07, 9.1, 9.5, 10.0, 10.5, 20.0, 21.0, 90.0]),    # saturates exactly from 9.5 on at the latest
     ("Sigmoid", -20, 8, [86.0, -86.0, 88.7, -88.7, 100.0, -100.0]),
     ("Div", -20, 20, [1.0, -1.0]),
 ])
@@ -43,6 +43,9 @@ def test_elementary_functions_over_dense_sweeps(op, lo, hi, extra):
     ref = interp.run_function(gd.desc, ins, [out] + grads, feeds)
     for gv, rv, what in zip(got, ref, ("value", "gradient")):
         check(gv, rv, TOL32, "%s %s" % (op, what))
+    if op == "Tanh":      # a saturated tanh is exactly +-1 and its gradient exactly 0
+        sat = np.abs(x) >= 9.5
+        assert np.all(np.abs(got[0][sat]) == 1) and np.all(got[1][sat] == 0)
 
 
 @pytest.mark.parametrize("kind", ["sgd", "momentum"])

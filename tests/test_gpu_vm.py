@@ -83,7 +83,7 @@ def test_toy_gradients(n):
 
 
 FLOOR_OK = 0.25   # CPU fp32 evaluation within a quarter of the tolerance: the tensor is held to the tolerance itself
-C_COND = 16.0     # otherwise (floor f, in tolerances): held to C_COND * f tolerances
+C_COND = 8.0      # otherwise (floor f, in tolerances): held to C_COND * f tolerances
 
 
 def fp32_floors(desc, inputs, outputs, feeds):

@@ -225,19 +225,39 @@ def test_gpu_jacobian_style_row_dag_full_size():
     tp = torch.from_numpy(pick).cuda()
     sub = [t[tp].cpu().numpy() if t.dim() == 2 else t.cpu().numpy() for t in gpu_in]
     gs, in_s, outs_s = build(len(pick))
-    ref = interp.run_function(gs.desc, in_s, outs_s, sub)
-    low = interp.run_function(gs.desc, in_s, outs_s, sub, dtype=np.float32)
+    ref, v64, _ = interp.run_function(gs.desc, in_s, outs_s, sub, return_all=True)
+    low, v32, _ = interp.run_function(gs.desc, in_s, outs_s, sub, dtype=np.float32, return_all=True)
+    # Rows in which fp32 cannot decide a kink: an operand of ReLU (kink at 0), of Exp (the clamp at +-10) or the
+    # divisor of Div (|b| at 0) lies closer to the kink than 64 times the distance between the fp32 and the
+    # fp64 evaluation of that very operand (typically a row sum that cancels to almost nothing).  There the
+    # operator's value or derivative jumps, any fp32 evaluation may land on either side, and the whole row is
+    # affected through the row sums; such rows are set aside and counted, all others are compared.
+    undecided = np.zeros(len(pick), bool)
+    for k in oprune.function_sets(gs.desc, in_s, outs_s)["fwd_ops"]:
+        op = gs.desc["ops"][k]
+        kinks = {"ReLU": (0, [0.0]), "Div": (1, [0.0]), "Exp": (0, [-10.0, 10.0])}.get(op["type"])
+        if kinks is None:
+            continue
+        x64, x32 = v64[op["in"][kinks[0]]], v32[op["in"][kinks[0]]].astype(np.float64)
+        dev = np.abs(x32 - x64)
+        for c in kinks[1]:
+            near = (np.abs(x64 - c) <= 64 * dev) & (dev > 0)
+            if near.ndim == 2:
+                undecided |= near.any(axis=1)
+            elif near.any():
+                undecided[:] = True
+    assert undecided.sum() <= 2, "fp32 cannot decide a kink in %d of %d sampled rows" % (undecided.sum(), len(pick))
+    keep = ~undecided
     n_full = n_tight = 0
     for o, r, l, t in zip(outs, ref, low, outs_ids):
         assert torch.isfinite(o).all()
         if o.dim() == 2:
-            # One of the per-objective gradients is ill-conditioned in fp32: NumPy's own fp32 evaluation is
-            # 10 to 80 tolerances away from fp64 on it (a mask behind a row sum flips for whole rows).  The
-            # emitted program for it is exact when run in fp64 (the emulated tests); here it is held to
-            # C_COND times that floor, every other tensor to the tolerance itself.
-            floor = float(np.max(np.abs(l.astype(np.float64) - r) / (TOL32 * (1 + np.abs(r)))))
+            # A tensor on which NumPy's own fp32 evaluation leaves the tolerance is held to C_COND times that
+            # floor (the emitted program for it is exact when run in fp64: the emulated tests), every other
+            # tensor to the tolerance itself.
+            floor = float(np.max((np.abs(l.astype(np.float64) - r) / (TOL32 * (1 + np.abs(r))))[keep]))
             scale = 1.0 if floor <= FLOOR_OK else C_COND * floor
             n_full += 1
             n_tight += scale == 1.0
-            check(o[tp].cpu().numpy().astype(np.float64), r, TOL32 * scale, "tensor %d (fp32 floor %.3g)" % (t, floor))
+            check(o[tp].cpu().numpy().astype(np.float64)[keep], r[keep], TOL32 * scale, "tensor %d (fp32 floor %.3g)" % (t, floor))
     assert n_full >= 4 and n_tight >= n_full - 1

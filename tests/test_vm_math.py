@@ -61,7 +61,11 @@ def test_exp_tanh_sigmoid_div():
     assert np.max(rel(y, r)[r != 0]) < 4e-7 and np.all(np.abs(y) <= 1)     # about 5 ulp, never beyond +-1
     assert np.sqrt(np.mean(rel(y, r)[r != 0] ** 2)) < 1e-7
     t = B.host_math(B.OPS["Tanh"], np.float32([np.nan, np.inf, -np.inf, 0.0, 1e-30]))
-    assert np.isnan(t[0]) and abs(t[1] - 1) < 2e-7 and abs(t[2] + 1) < 2e-7 and t[3] == 0 and t[4] == np.float32(1e-30)
+    assert np.isnan(t[0]) and t[1] == 1 and t[2] == -1 and t[3] == 0 and t[4] == np.float32(1e-30)
+    # saturation is exact: from 9.3 on (tanh rounds to +-1 in fp32 from 9.02 on; in between the result is within
+    # one rounding step of it) the result is +-1, so 1 - y^2 is 0
+    x = np.concatenate([np.linspace(9.3, 200, 400001), [1e10, 3e38]]).astype(np.float32)
+    assert np.all(B.host_math(B.OPS["Tanh"], x) == 1) and np.all(B.host_math(B.OPS["Tanh"], -x) == -1)
     x = np.linspace(-80, 80, 1_000_001).astype(np.float32)
     assert np.max(rel(B.host_math(B.OPS["Sigmoid"], x), 1 / (1 + np.exp(-x.astype(np.float64))))) < 3e-7
     y = B.host_math(B.OPS["Sigmoid"], np.float32([-200, 200]))
