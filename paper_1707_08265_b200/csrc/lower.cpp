@@ -26,6 +26,7 @@ struct Lowerer {
   std::vector<int> fetch_of;                  // tensor -> fetch position or -1
   std::map<std::pair<int, int>, int> materialised;   // (value, dtype) -> memref
   std::vector<std::map<int, int>> pending;    // per stage: tensor -> gradient contributions still to come
+  std::map<int, int> def_item;                // value -> index of the micro-operation that defines it
   int err = DRAGON_OK;
 
   Lowerer(const Graph& g_, const PruneResult& pr_, Plan* p) : g(g_), pr(pr_), plan(p) {}
@@ -38,8 +39,19 @@ struct Lowerer {
   }
   int new_val(int kind, const Shape& s, int mem = -1, float c = 0.f) {
     Value v; v.kind = kind; v.shape = s; v.mem = mem; v.c = c;
+    v.row_uniform = s.numel() == 1;     // scalars and constants; operations set it for their results
     vals.push_back(v);
     return (int)vals.size() - 1;
+  }
+  // the micro-operation that defines value v (through widenings), or null
+  const Item* def_of(int v) const {
+    for (;;) {
+      auto it = def_item.find(v);
+      if (it == def_item.end()) return nullptr;
+      const Item& d = items[it->second];
+      if (d.opc != M_WIDEN) return &d;
+      v = d.a;
+    }
   }
   int konst(float c) {
     int v = new_val(VK_CONST, Shape(), -1, c);
@@ -56,6 +68,8 @@ struct Lowerer {
     it.dst = new_val(VK_OP, s);
     vals[it.dst].known_const = vals[v].known_const;
     vals[it.dst].c = vals[v].c;
+    vals[it.dst].row_uniform = vals[v].row_uniform;
+    def_item[it.dst] = (int)items.size();
     items.push_back(it);
     return it.dst;
   }
@@ -72,6 +86,18 @@ struct Lowerer {
       if (is_const(b, 1.f)) return widen(a, s);
     }
     if (opc == M_NEG && vals[a].known_const) return widen(konst(-vals[a].c), s);
+    if (opc == M_MUL && (vals[a].known_const != vals[b].known_const)) {
+      // (x * c1) * c2 = x * (c1 * c2): a mean of a row-uniform value, a scaled sum of one
+      const int x = vals[a].known_const ? b : a, c = vals[a].known_const ? a : b;
+      const Item* d = def_of(x);
+      if (d && d->opc == M_MUL && (vals[d->a].known_const != vals[d->b].known_const)) {
+        const int dx = vals[d->a].known_const ? d->b : d->a, dc = vals[d->a].known_const ? d->a : d->b;
+        return mop(M_MUL, widen(dx, vals[x].shape), konst(vals[dc].c * vals[c].c));
+      }
+    }
+    // the sum over a row whose elements are all equal is that element times the row length: no reduction
+    // (Sum of a Sum, Mean of a Mean, the gradient of a Mean that reaches it as one value per row)
+    if (opc == M_ROWSUM && vals[a].row_uniform) return mop(M_MUL, a, konst((float)vals[a].shape.cols()));
     if (is_binary(opc) && vals[a].known_const && vals[b].known_const) {
       float x = vals[a].c, y = vals[b].c;
       float r = opc == M_ADD ? x + y : opc == M_SUB ? x - y : opc == M_MUL ? x * y : x / (1.f + std::fabs(y));
@@ -79,6 +105,8 @@ struct Lowerer {
     }
     Item it; it.kind = IT_MOP; it.opc = opc; it.a = a; it.b = b;
     it.dst = new_val(VK_OP, s);
+    vals[it.dst].row_uniform = opc == M_ROWSUM || (vals[a].row_uniform && (b < 0 || vals[b].row_uniform));
+    def_item[it.dst] = (int)items.size();
     items.push_back(it);
     return it.dst;
   }

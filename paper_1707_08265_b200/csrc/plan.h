@@ -52,6 +52,7 @@ struct Value {
   int mem = -1;
   float c = 0.f;
   bool known_const = false;  // VK_CONST, or a widened view of one
+  bool row_uniform = false;  // the same value in every element of a row: a row sum, a scalar, or an elementwise function of such
 };
 
 enum ItemKind { IT_MOP, IT_GEMM, IT_TRANSPOSE, IT_SCE_FWD, IT_SCE_BWD, IT_COPY };

@@ -61,9 +61,11 @@ def test_random_row_programs(seed):
     outs = fetch + grads
     got, f = emulate(g.desc, inputs, outs, feeds)
     ref = interp.run_function(g.desc, inputs, outs, feeds)
+    # the emulator computes in fp64 but the program's constants are fp32 (1/24 is not representable: a mean is
+    # off by 3e-8 relative, and a row sum behind it multiplies that by up to the row length)
     for gv, rv in zip(got, ref):
         ok = np.isfinite(rv)
-        assert np.allclose(gv[ok], rv[ok], rtol=1e-7, atol=1e-7), f.describe()
+        assert np.allclose(gv[ok], rv[ok], rtol=2e-6, atol=1e-6), f.describe()
 
 
 def test_register_pressure_program():
