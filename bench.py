@@ -200,7 +200,7 @@ def connected_inputs(B, desc, objs, inputs):
     return keep
 
 
-def build_config(cfg, B, torch, seeds):
+def build_config(cfg, B, torch, seeds, rows=16384):
     """-> dict(g, inputs, outputs, units, what, and the roofline's numerator)"""
     MiB = 1 << 20
     if cfg == 1:
@@ -223,7 +223,7 @@ def build_config(cfg, B, torch, seeds):
         return dict(g=g, inputs=[ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels")],
                     outputs=[ids[k] for k in ("loss", "dW1", "db1", "dW2", "db2")], units=8192, unit="batch rows/s", bound="tensor",
                     alg=5 * 2.0 * 8192 * 4096 * 4096, what="config 4: MLP 8192 x 4096-4096-4096 bf16, forward + backward (5 contractions survive the prunes)")
-    g, inputs, fetch = wl.random_row_dag(16384, 4096, seeds["random_row_dag"]["seed"])
+    g, inputs, fetch = wl.random_row_dag(rows, 4096, seeds["random_row_dag"]["seed"])
     if cfg == 5:
         wrts = connected_inputs(B, g.desc, fetch, inputs)
         outputs = fetch + g.grad(fetch, wrts)
@@ -234,12 +234,12 @@ def build_config(cfg, B, torch, seeds):
             outputs += g.grad([o], connected_inputs(B, g.desc, [o], inputs))
         what = "row DAG on [16384,4096], forward + one gradient stage per objective (%d fetches)" % len(outputs)
     # the workload as stated moves 6 FULL inputs, 4 FULL targets and 6 FULL gradients of 256 MiB each
-    return dict(g=g, inputs=inputs, outputs=outputs, units=16384 * 4096, unit=UNIT, bound="hbm", alg=16.0 * 256 * MiB, what=what)
+    return dict(g=g, inputs=inputs, outputs=outputs, units=rows * 4096, unit=UNIT, bound="hbm", alg=16.0 * rows * 4096 * 4, what=what)
 
 
 def time_config(cfg, args, B, torch, seeds, peaks, steps=None):
     """Device-resident timing of one workload (a step = one dragon_run) plus the per-kernel times of its plan."""
-    c = build_config(cfg, B, torch, seeds)
+    c = build_config(cfg, B, torch, seeds, args.rows)
     g, inputs, outputs = c["g"], c["inputs"], c["outputs"]
     tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32}
     gen = torch.Generator("cuda").manual_seed(wl.BASE_SEED + cfg)
@@ -332,6 +332,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU (default: the benchmark's 2^26)")
+    ap.add_argument("--rows", type=int, default=16384, help="rows of workload 5 (default: its 16384; smaller for profiler captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-other-configs", action="store_true", help="leave the \"configs\" entry (workloads 1, 3, 4, 5) out")
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7],

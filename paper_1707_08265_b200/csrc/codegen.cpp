@@ -701,7 +701,7 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
     Gen gen(items, idx, vals, mems, &trial, kVmRegsDense, kVmSmemSlotsDense);
     rc = gen.run();
     // it must keep everything on chip, within half an SM's shared memory
-    const size_t smem = (size_t)((trial.code.size() + 3) & ~(size_t)3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)trial.n_smem * kVmTile * 4;
+    const size_t smem = (size_t)((trial.code.size() + 3) & ~(size_t)3) * 8 + kMaxUniforms * 4 + kVmReduceBytes + kMaxOperands * 16 + (size_t)trial.n_smem * kVmTile * 4;
     if (rc == DRAGON_OK && trial.n_spill == 0 && smem <= 113 * 1024) { *seg = trial; seg->dense = true; }
     else rc = DRAGON_ERR_UNSUPPORTED;
   }
@@ -709,7 +709,7 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
     // as many shared-memory slots as fit beside the instruction stream (whose length depends a
     // little on the slot count: second attempt with the count that fits the first one's stream)
     auto smem_of = [](const VmSegment& g, int slots) {
-      return (size_t)((g.code.size() + 3) & ~(size_t)3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)slots * kVmTile * 4;
+      return (size_t)((g.code.size() + 3) & ~(size_t)3) * 8 + kMaxUniforms * 4 + kVmReduceBytes + kMaxOperands * 16 + (size_t)slots * kVmTile * 4;
     };
     for (int slots = kVmSmemSlots;; slots = kVmSmemSlotsLongCode) {
       VmSegment trial = *seg;

@@ -18,6 +18,7 @@ constexpr int kVmCodeMaxWords = 8 * 1024;     // instruction stream held in shar
 constexpr int kVmSmemSlots = 13;              // V-wide shared-memory slots per thread at most (wide build: one CTA per SM, 227 KB)
 constexpr int kVmSmemSlotsLongCode = 9;       // the same when the instruction stream is too long for that many
 constexpr int kVmSmemSlotsDense = 6;          // the same for the dense build (two CTAs share the SM's shared memory)
+constexpr int kVmReduceBytes = 1024;          // shared memory for the per-warp partials of row sums and block sums
 constexpr int kDefaultSmCount = 148;
 constexpr int kHostChunks = 16;               // dragon_run_host pipelines a large elementwise function in this many chunks
 

@@ -81,7 +81,7 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
 
 // shared memory of one CTA: decoded instruction stream | uniforms | reduction scratch | operand table | slots
 size_t vm_smem_bytes(int n_code, int n_smem_slots) {
-  return (size_t)((n_code + 3) & ~3) * 8 + kMaxUniforms * 4 + 64 * 8 + kMaxOperands * 16 + (size_t)n_smem_slots * kVmTile * 4;
+  return (size_t)((n_code + 3) & ~3) * 8 + kMaxUniforms * 4 + kVmReduceBytes + kMaxOperands * 16 + (size_t)n_smem_slots * kVmTile * 4;
 }
 
 }  // namespace vm

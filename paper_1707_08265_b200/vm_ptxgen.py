@@ -22,12 +22,8 @@ Running this file writes the PTX to the path given as its first argument.
 import struct
 import sys
 
-NT = 512            # threads per CTA
-V = 8               # elements per thread
-NP = V // 2         # packed pairs per value
-TILE = NT * V       # 4096 elements
+TILE = 4096         # elements per tile = threads per CTA x elements per thread (512 x 8 or 1024 x 4)
 SLOT_BYTES = TILE * 4
-HALF_BYTES = NT * 16
 MAX_OPERANDS = 40
 MAX_UNIFORMS = 512
 
@@ -36,7 +32,8 @@ P_CODE, P_SPILL, P_COLPART, P_SCALPART, P_STATUS, P_N = 0, 8, 16, 24, 32, 40
 P_NCODE, P_ROWMODE, P_COLS, P_NSPILL, P_NTILES, P_LOOPSTART, P_GRID, P_NFULL, P_STATUSCLEAR, P_OPERAND = 48, 52, 56, 60, 64, 68, 72, 76, 80, 96
 P_SIZE = P_OPERAND + 16 * MAX_OPERANDS
 # shared memory behind the decoded instruction stream: uniforms | reduction scratch | operand table | slots
-OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + 512, MAX_UNIFORMS * 4 + 512 + MAX_OPERANDS * 16
+RED_BYTES = 1024    # per-warp partials of the row sums (three buffers of up to 32 floats) and of the fp64 block sums (32 doubles)
+OFF_RED, OFF_OPB, OFF_SLOTS = MAX_UNIFORMS * 4, MAX_UNIFORMS * 4 + RED_BYTES, MAX_UNIFORMS * 4 + RED_BYTES + MAX_OPERANDS * 16
 
 JOINT = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "fmaur", "rtos", "stor", "spillr", "fillr",
          "gldr", "sincosr", "cossinr", "macc0", "macc1", "macc2", "macc3", "ldswr", "ldswar",
@@ -64,19 +61,28 @@ def fc(x):
 
 
 class Kernel:
-    def __init__(self, name, nr, ctas_per_sm):
+    def __init__(self, name, nr, ctas_per_sm, threads=512):
         self.name, self.nr, self.ctas = name, nr, ctas_per_sm
+        # geometry: a thread owns V elements of a tile as V/4 groups of four consecutive ones (a group is one
+        # 16-byte vector, the groups of a warp are contiguous), held as NP = V/2 packed pairs
+        self.NT = threads
+        self.V = TILE // threads
+        self.NP = self.V // 2
+        self.NH = self.V // 4               # 16-byte groups per thread
+        self.HALF_BYTES = threads * 16      # distance between a thread's groups
+        self.red_shift = 6 if threads == 512 else 7     # log2 of the bytes of one buffer of per-warp row-sum partials
+        assert 3 * (threads // 32) * 4 <= 512 and 512 + (threads // 32) * 8 <= RED_BYTES
         self.lines = []
         self.ph_sites = []    # return labels of the sin/cos sites (reduce_pio2)
-        self.PX = ["%%PX%d" % i for i in range(NP)]
-        self.PR = ["%%PR%d" % i for i in range(NP)]
-        self.PK = ["%%PK%d" % i for i in range(NP)]
+        self.PX = ["%%PX%d" % i for i in range(self.NP)]
+        self.PR = ["%%PR%d" % i for i in range(self.NP)]
+        self.PK = ["%%PK%d" % i for i in range(self.NP)]
         self.cold = []        # rarely executed blocks, placed behind all leaves so that the hot leaves stay short and close together
         self.cnt = {"f": 0, "r": 0, "rd": 0, "p": 0, "fd": 0, "h": 0}
         self.nlabel = 0
         self.kt = []          # packed constants (u64 words)
-        self.A = ["%%A%d" % i for i in range(NP)]
-        self.R = [["%%R%d_%d" % (k, i) for i in range(NP)] for k in range(nr)]
+        self.A = ["%%A%d" % i for i in range(self.NP)]
+        self.R = [["%%R%d_%d" % (k, i) for i in range(self.NP)] for k in range(nr)]
         self.S = ["%%S%d" % i for i in range(N_SACC)]     # scalar accumulators (.f32)
 
     # ---- plumbing -------------------------------------------------------------------------
@@ -154,7 +160,7 @@ class Kernel:
         return out
 
     def packs(self, sc, dst=None):
-        return [self.pack(sc[2 * i], sc[2 * i + 1], dst[i] if dst else None) for i in range(NP)]
+        return [self.pack(sc[2 * i], sc[2 * i + 1], dst[i] if dst else None) for i in range(self.NP)]
 
     def rcp(self, x):
         d = self.f()
@@ -217,27 +223,27 @@ class Kernel:
         return u
 
     def lds_v(self, addr, dst=None):
-        d = dst or [self.rd() for _ in range(NP)]
-        self.e("ld.shared.v2.b64 {%s, %s}, [%s];" % (d[0], d[1], addr))
-        self.e("ld.shared.v2.b64 {%s, %s}, [%s+%d];" % (d[2], d[3], addr, HALF_BYTES))
+        d = dst or [self.rd() for _ in range(self.NP)]
+        for h in range(self.NH):
+            self.e("ld.shared.v2.b64 {%s, %s}, [%s+%d];" % (d[2 * h], d[2 * h + 1], addr, h * self.HALF_BYTES))
         return d
 
     def sts_v(self, addr, src):
-        self.e("st.shared.v2.b64 [%s], {%s, %s};" % (addr, src[0], src[1]))
-        self.e("st.shared.v2.b64 [%s+%d], {%s, %s};" % (addr, HALF_BYTES, src[2], src[3]))
+        for h in range(self.NH):
+            self.e("st.shared.v2.b64 [%s+%d], {%s, %s};" % (addr, h * self.HALF_BYTES, src[2 * h], src[2 * h + 1]))
 
     def ldg_v(self, addr, dst=None):
-        d = dst or [self.rd() for _ in range(NP)]
-        self.e("ld.global.v2.b64 {%s, %s}, [%s];" % (d[0], d[1], addr))
-        self.e("ld.global.v2.b64 {%s, %s}, [%s+%d];" % (d[2], d[3], addr, HALF_BYTES))
+        d = dst or [self.rd() for _ in range(self.NP)]
+        for h in range(self.NH):
+            self.e("ld.global.v2.b64 {%s, %s}, [%s+%d];" % (d[2 * h], d[2 * h + 1], addr, h * self.HALF_BYTES))
         return d
 
     def stg_v(self, addr, src):
-        self.e("st.global.v2.b64 [%s], {%s, %s};" % (addr, src[0], src[1]))
-        self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (addr, HALF_BYTES, src[2], src[3]))
+        for h in range(self.NH):
+            self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (addr, h * self.HALF_BYTES, src[2 * h], src[2 * h + 1]))
 
     def mov_v(self, dst, src):
-        for i in range(NP):
+        for i in range(self.NP):
             self.e("mov.b64 %s, %s;" % (dst[i], src[i]))
 
     # ---- elementary functions (csrc/vm_math.h, operation by operation) -----------------------
@@ -251,7 +257,7 @@ class Kernel:
         holds (emit_general_reduction), which returns here behind the packed code."""
         big = 12582912.0
         n = len(xs)
-        assert n == NP
+        assert n == self.NP
         r, kb = self.PR, self.PK
         lanes = []
         for x in xs:
@@ -308,7 +314,7 @@ class Kernel:
         if not self.ph_sites:
             return
         big = 12582912.0
-        n = NP
+        n = self.NP
         self.e("PHRET_%s: .branchtargets %s;" % (self.name, ", ".join(self.ph_sites)))
         self.label("$PH_%s" % self.name)
         base = self.rd()
@@ -331,8 +337,8 @@ class Kernel:
         self.e("add.rn.f32 %s, %s, %s;" % (ks, kbs, fc(-big)))
         self.e("fma.rn.f32 %s, %s, %s, %s;" % (rs, ks, fc(-1.57079637050628662109375), xs_))
         self.e("fma.rn.f32 %s, %s, %s, %s;" % (rs, ks, fc(4.371138828673793e-8), rs))
-        self.e("st.local.f32 [%s+32], %s;" % (adr, rs))
-        self.e("st.local.f32 [%s+64], %s;" % (adr, kbs))
+        self.e("st.local.f32 [%s+%d], %s;" % (adr, 8 * n, rs))
+        self.e("st.local.f32 [%s+%d], %s;" % (adr, 16 * n, kbs))
         self.e("bra %s;" % nxt)
         self.label(large)
         self.e("setp.ge.u32 %s, %s, 0x7f800000;" % (pnf, ax))
@@ -378,24 +384,24 @@ class Kernel:
         self.e("@%s neg.s32 %s, %s;" % (px, qi, qi))
         self.e("and.b32 %s, %s, 3;" % (qi, qi))
         self.e("or.b32 %s, %s, 0x%08X;" % (qi, qi, f32bits(big)))
-        self.e("st.local.f32 [%s+32], %s;" % (adr, rf))
-        self.e("st.local.b32 [%s+64], %s;" % (adr, qi))
+        self.e("st.local.f32 [%s+%d], %s;" % (adr, 8 * n, rf))
+        self.e("st.local.b32 [%s+%d], %s;" % (adr, 16 * n, qi))
         self.e("bra %s;" % nxt)
         self.label(special)
         xf, z, kq = self.f(), self.f(), self.r()
         self.e("mov.b32 %s, %s;" % (xf, xb))
         self.e("sub.f32 %s, %s, %s;" % (z, xf, xf))
         self.e("mov.u32 %s, 0x%08X;" % (kq, f32bits(big)))
-        self.e("st.local.f32 [%s+32], %s;" % (adr, z))
-        self.e("st.local.b32 [%s+64], %s;" % (adr, kq))
+        self.e("st.local.f32 [%s+%d], %s;" % (adr, 8 * n, z))
+        self.e("st.local.b32 [%s+%d], %s;" % (adr, 16 * n, kq))
         self.label(nxt)
         plp = self.p()
         self.e("add.u32 %s, %s, 1;" % (i_, i_))
         self.e("setp.lt.u32 %s, %s, %d;" % (plp, i_, 2 * n))
         self.e("@%s bra %s;" % (plp, loop))
         for i in range(n):
-            self.e("ld.local.b64 %s, [%s+%d];" % (self.PR[i], base, 32 + 8 * i))
-            self.e("ld.local.b64 %s, [%s+%d];" % (self.PK[i], base, 64 + 8 * i))
+            self.e("ld.local.b64 %s, [%s+%d];" % (self.PR[i], base, 8 * n + 8 * i))
+            self.e("ld.local.b64 %s, [%s+%d];" % (self.PK[i], base, 16 * n + 8 * i))
         self.e("brx.idx %%phsite, PHRET_%s;" % self.name)
 
     def sincos(self, xs, want_sin=True, want_cos=True):
@@ -525,7 +531,7 @@ class Kernel:
 
     def divp(self, num, den, dst):
         """dst = num / (1 + |den|), packed lists"""
-        for i in range(NP):
+        for i in range(self.NP):
             lo, hi = self.unpack(den[i])
             self.mul2(num[i], self.pack(self.rcp1pabs(lo), self.rcp1pabs(hi)), dst[i])
 
@@ -576,7 +582,7 @@ class Kernel:
     # position of element j of this thread inside the tile
     def lane_pos(self, j):
         d = self.r()
-        self.e("add.u32 %s, %%pos0, %d;" % (d, (j >> 2) * NT * 4 + (j & 3)))
+        self.e("add.u32 %s, %%pos0, %d;" % (d, (j >> 2) * self.NT * 4 + (j & 3)))
         return d
 
     def mask_tail(self, sc):
@@ -610,12 +616,12 @@ class Kernel:
             self.e("and.pred %s, %s, %s;" % (pr, pr, cond))
         self.e("mul.wide.u32 %s, %%tnext, %d;" % (off, esize))
         self.e("add.u64 %s, %s, %s;" % (pa, adr, off))
-        for h in range(2):
+        for h in range(self.NH):
             ph, ps = self.p(), self.r()
-            self.e("add.u32 %s, %%pos0, %d;" % (ps, h * NT * 4))
+            self.e("add.u32 %s, %%pos0, %d;" % (ps, h * self.NT * 4))
             self.e("setp.lt.u32 %s, %s, %%limit;" % (ph, ps))
             self.e("and.pred %s, %s, %s;" % (ph, ph, pr))
-            self.e("@%s prefetch.global.L2 [%s+%d];" % (ph, pa, h * NT * 4 * esize))
+            self.e("@%s prefetch.global.L2 [%s+%d];" % (ph, pa, h * self.NT * 4 * esize))
 
     def leaf_gldf(self, dst, copy_to=None):
         """fp32 FULL operand -> dst (and copy_to)"""
@@ -629,10 +635,10 @@ class Kernel:
         self.e("setp.ne.u32 %s, %%tnext, 0;" % pr)
         self.e("mul.wide.u32 %s, %%tnext, 4;" % off)
         self.e("add.u64 %s, %s, %s;" % (pa, adr, off))
-        self.e("@%s prefetch.global.L2 [%s];" % (pr, pa))
-        self.e("@%s prefetch.global.L2 [%s+%d];" % (pr, pa, HALF_BYTES))
-        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s];" % (dst[0], dst[1], adr))
-        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (dst[2], dst[3], adr, HALF_BYTES))
+        for h in range(self.NH):
+            self.e("@%s prefetch.global.L2 [%s+%d];" % (pr, pa, h * self.HALF_BYTES))
+        for h in range(self.NH):
+            self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (dst[2 * h], dst[2 * h + 1], adr, h * self.HALF_BYTES))
         if copy_to:
             self.mov_v(copy_to, dst)
         self.jump()
@@ -661,8 +667,8 @@ class Kernel:
 
     def async_copy(self, sadr, gadr, pred):
         """this thread's two 16-byte pieces of a tile: global -> shared, asynchronously"""
-        for h in range(2):
-            self.e("@%s cp.async.cg.shared.global [%s+%d], [%s+%d], 16;" % (pred, sadr, h * HALF_BYTES, gadr, h * HALF_BYTES))
+        for h in range(self.NH):
+            self.e("@%s cp.async.cg.shared.global [%s+%d], [%s+%d], 16;" % (pred, sadr, h * self.HALF_BYTES, gadr, h * self.HALF_BYTES))
         self.e("cp.async.commit_group;")
 
     def leaf_glda(self, first):
@@ -691,8 +697,8 @@ class Kernel:
 
     # bf16 operands, read once per iteration: 8 bytes per thread and half, converted at the read
     def async_copy_h(self, sadr, gadr, pred):
-        for h in range(2):
-            self.e("@%s cp.async.ca.shared.global [%s+%d], [%s+%d], 8;" % (pred, sadr, h * HALF_BYTES, gadr, h * NT * 8))
+        for h in range(self.NH):
+            self.e("@%s cp.async.ca.shared.global [%s+%d], [%s+%d], 8;" % (pred, sadr, h * self.HALF_BYTES, gadr, h * self.NT * 8))
         self.e("cp.async.commit_group;")
 
     def tile_adr_h(self, ptr):
@@ -717,9 +723,9 @@ class Kernel:
         slow = self.newlabel("ldswh")
         self.e("@!%%pfull bra.uni %s;" % slow)
         self.e("cp.async.wait_all;")
-        for h in range(2):
+        for h in range(self.NH):
             w0, w1 = self.r(), self.r()
-            self.e("ld.shared.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, sadr, h * HALF_BYTES))
+            self.e("ld.shared.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, sadr, h * self.HALF_BYTES))
             for i, w in enumerate((w0, w1)):
                 lo, hi = self.r(), self.r()
                 self.e("shl.b32 %s, %s, 16;" % (lo, w))
@@ -753,7 +759,7 @@ class Kernel:
 
         def copy():
             if affine:
-                for i in range(NP):
+                for i in range(self.NP):
                     self.fma2(dst[i], uu, vv, copy_to[i])
             elif copy_to:
                 self.mov_v(copy_to, dst)
@@ -777,10 +783,10 @@ class Kernel:
 
     def load_f32_slow(self, adr, dst):
         pvec = self.pvec()
-        for h in range(2):
+        for h in range(self.NH):
             lv, ln = self.newlabel("ld"), self.newlabel("ld")
             pv, pos3 = self.p(), self.r()
-            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
+            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * self.NT * 4 + 3))
             self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
             self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
@@ -789,13 +795,13 @@ class Kernel:
                 pe, d = self.p(), self.f()
                 self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
                 self.e("mov.f32 %s, 0f00000000;" % d)
-                self.e("@%s ld.global.nc.f32 %s, [%s+%d];" % (pe, d, adr, h * HALF_BYTES + 4 * e_))
+                self.e("@%s ld.global.nc.f32 %s, [%s+%d];" % (pe, d, adr, h * self.HALF_BYTES + 4 * e_))
                 sc.append(d)
             self.pack(sc[0], sc[1], dst[2 * h])
             self.pack(sc[2], sc[3], dst[2 * h + 1])
             self.e("bra %s;" % ln)
             self.label(lv)
-            self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (dst[2 * h], dst[2 * h + 1], adr, h * HALF_BYTES))
+            self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (dst[2 * h], dst[2 * h + 1], adr, h * self.HALF_BYTES))
             self.label(ln)
 
     def leaf_gld(self):
@@ -815,8 +821,8 @@ class Kernel:
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
         slow = self.newlabel("gld")
         self.e("@!%%pfull bra.uni %s;" % slow)     # a full tile: whole, aligned vectors (ROW operands too)
-        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s];" % (A[0], A[1], adr))
-        self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (A[2], A[3], adr, HALF_BYTES))
+        for h in range(self.NH):
+            self.e("ld.global.nc.v2.b64 {%s, %s}, [%s+%d];" % (A[2 * h], A[2 * h + 1], adr, h * self.HALF_BYTES))
         self.jump()
         self.label(slow)
         self.prefetch(adr, 4, pfullk)
@@ -829,9 +835,9 @@ class Kernel:
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
         slowb = self.newlabel("gld")
         self.e("@!%%pfull bra.uni %s;" % slowb)
-        for h in range(2):
+        for h in range(self.NH):
             w0, w1 = self.r(), self.r()
-            self.e("ld.global.nc.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, adr, h * NT * 8))
+            self.e("ld.global.nc.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, adr, h * self.NT * 8))
             for i, w in enumerate((w0, w1)):
                 lo, hi = self.r(), self.r()
                 self.e("shl.b32 %s, %s, 16;" % (lo, w))
@@ -845,10 +851,10 @@ class Kernel:
 
     def load_bf16_slow(self, adr, A):
         pvec = self.pvec()
-        for h in range(2):
+        for h in range(self.NH):
             lv, ln = self.newlabel("gld"), self.newlabel("gld")
             pv, pos3 = self.p(), self.r()
-            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
+            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * self.NT * 4 + 3))
             self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
             self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
@@ -857,7 +863,7 @@ class Kernel:
                 pe, d, hh = self.p(), self.r(), self.t("h")
                 self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
                 self.e("mov.b16 %s, 0;" % hh)
-                self.e("@%s ld.global.nc.u16 %s, [%s+%d];" % (pe, hh, adr, h * NT * 8 + 2 * e_))
+                self.e("@%s ld.global.nc.u16 %s, [%s+%d];" % (pe, hh, adr, h * self.NT * 8 + 2 * e_))
                 self.e("cvt.u32.u16 %s, %s;" % (d, hh))
                 self.e("shl.b32 %s, %s, 16;" % (d, d))
                 sc.append(d)
@@ -866,7 +872,7 @@ class Kernel:
             self.e("bra %s;" % ln)
             self.label(lv)
             w0, w1 = self.r(), self.r()
-            self.e("ld.global.nc.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, adr, h * NT * 8))
+            self.e("ld.global.nc.v2.u32 {%s, %s}, [%s+%d];" % (w0, w1, adr, h * self.NT * 8))
             for i, w in enumerate((w0, w1)):
                 lo, hi = self.r(), self.r()
                 self.e("shl.b32 %s, %s, 16;" % (lo, w))
@@ -877,10 +883,10 @@ class Kernel:
     def store_f32_slow(self, adr):
         A = self.A
         pvec = self.pvec()
-        for h in range(2):
+        for h in range(self.NH):
             lv, ln = self.newlabel("st"), self.newlabel("st")
             pv, pos3 = self.p(), self.r()
-            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
+            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * self.NT * 4 + 3))
             self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
             self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
@@ -888,10 +894,10 @@ class Kernel:
             for e_ in range(4):
                 pe = self.p()
                 self.e("setp.lt.u32 %s, %s, %%limit;" % (pe, self.lane_pos(4 * h + e_)))
-                self.e("@%s st.global.f32 [%s+%d], %s;" % (pe, adr, h * HALF_BYTES + 4 * e_, sc[e_]))
+                self.e("@%s st.global.f32 [%s+%d], %s;" % (pe, adr, h * self.HALF_BYTES + 4 * e_, sc[e_]))
             self.e("bra %s;" % ln)
             self.label(lv)
-            self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (adr, h * HALF_BYTES, A[2 * h], A[2 * h + 1]))
+            self.e("st.global.v2.b64 [%s+%d], {%s, %s};" % (adr, h * self.HALF_BYTES, A[2 * h], A[2 * h + 1]))
             self.label(ln)
 
     def leaf_gstf(self, then_loop_end=False, ptr=None):
@@ -953,23 +959,23 @@ class Kernel:
         self.e("add.u64 %s, %s, %s;" % (adr, ptr, off))
         slowb = self.newlabel("gst")
         self.e("@!%%pfull bra.uni %s;" % slowb)
-        for h in range(2):
+        for h in range(self.NH):
             sc = self.unpack(A[2 * h]) + self.unpack(A[2 * h + 1])
             w0, w1 = self.r(), self.r()
             self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w0, sc[1], sc[0]))
             self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w1, sc[3], sc[2]))
-            self.e("st.global.v2.u32 [%s+%d], {%s, %s};" % (adr, h * NT * 8, w0, w1))
+            self.e("st.global.v2.u32 [%s+%d], {%s, %s};" % (adr, h * self.NT * 8, w0, w1))
         self.jump()
         self.label(slowb)
         pvec = self.pvec()
-        for h in range(2):
+        for h in range(self.NH):
             lv, ln = self.newlabel("gst"), self.newlabel("gst")
             pv, pos3 = self.p(), self.r()
             sc = self.unpack(A[2 * h]) + self.unpack(A[2 * h + 1])
             w0, w1 = self.r(), self.r()
             self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w0, sc[1], sc[0]))
             self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w1, sc[3], sc[2]))
-            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * NT * 4 + 3))
+            self.e("add.u32 %s, %%pos0, %d;" % (pos3, h * self.NT * 4 + 3))
             self.e("setp.lt.u32 %s, %s, %%limit;" % (pv, pos3))
             self.e("and.pred %s, %s, %s;" % (pv, pv, pvec))
             self.e("@%s bra %s;" % (pv, lv))
@@ -980,10 +986,10 @@ class Kernel:
                     self.e("{ .reg .b16 %%lo; mov.b32 {%%lo, %s}, %s; }" % (hh, w))
                 else:
                     self.e("{ .reg .b16 %%hi; mov.b32 {%s, %%hi}, %s; }" % (hh, w))
-                self.e("@%s st.global.u16 [%s+%d], %s;" % (pe, adr, h * NT * 8 + 2 * e_, hh))
+                self.e("@%s st.global.u16 [%s+%d], %s;" % (pe, adr, h * self.NT * 8 + 2 * e_, hh))
             self.e("bra %s;" % ln)
             self.label(lv)
-            self.e("st.global.v2.u32 [%s+%d], {%s, %s};" % (adr, h * NT * 8, w0, w1))
+            self.e("st.global.v2.u32 [%s+%d], {%s, %s};" % (adr, h * self.NT * 8, w0, w1))
             self.label(ln)
         self.jump()
         # one scalar, written by thread 0
@@ -1004,8 +1010,11 @@ class Kernel:
 
     # ---- leaves -------------------------------------------------------------------------------
     def lane_sum(self, vals):
-        """sum of the 8 lanes of a packed V-wide value, as one scalar"""
-        lo, hi = self.unpack(self.add2(self.add2(vals[0], vals[1]), self.add2(vals[2], vals[3])))
+        """sum of the 8 lanes of a packed self.V-wide value, as one scalar"""
+        v = list(vals)
+        while len(v) > 1:
+            v = [self.add2(v[2 * i], v[2 * i + 1]) for i in range(len(v) // 2)]
+        lo, hi = self.unpack(v[0])
         d = self.f()
         self.e("add.f32 %s, %s, %s;" % (d, lo, hi))
         return d
@@ -1045,7 +1054,7 @@ class Kernel:
             u = self.uniform(iu)
             ptr, _, _ = self.operand(False, io)
             uu = self.splat(u)
-            for i in range(NP):
+            for i in range(self.NP):
                 self.fma2(A[i], uu, R[i], A[i])
             self.leaf_gstf(True, ptr)
             return
@@ -1069,7 +1078,7 @@ class Kernel:
             tail = self.newlabel("ma")
             self.e("@!%%pfull bra.uni %s;" % tail)
             t = self.mul2(A[0], R[0])
-            for i in range(1, NP): t = self.fma2(A[i], R[i], t)
+            for i in range(1, self.NP): t = self.fma2(A[i], R[i], t)
             lo, hi = self.unpack(t)
             self.e("add.f32 %s, %s, %s;" % (lo, lo, hi))
             self.e("add.f32 %s, %s, %s;" % (acc, acc, lo))
@@ -1077,7 +1086,7 @@ class Kernel:
             self.label(tail)
             m = self.packs(self.mask_tail(self.scalars(A)))
             t = self.mul2(m[0], R[0])
-            for i in range(1, NP): t = self.fma2(m[i], R[i], t)
+            for i in range(1, self.NP): t = self.fma2(m[i], R[i], t)
             lo, hi = self.unpack(t)
             self.e("add.f32 %s, %s, %s;" % (lo, lo, hi))
             self.e("add.f32 %s, %s, %s;" % (acc, acc, lo))
@@ -1085,7 +1094,7 @@ class Kernel:
             u = self.uniform()
             self.fetch()
             uu = self.splat(u)
-            for i in range(NP):
+            for i in range(self.NP):
                 self.fma2(A[i], uu, R[i], A[i])
         else:
             self.fetch()
@@ -1094,27 +1103,27 @@ class Kernel:
             elif op == "str":
                 self.mov_v(R, A)
             elif op == "add":
-                for i in range(NP): self.add2(A[i], R[i], A[i])
+                for i in range(self.NP): self.add2(A[i], R[i], A[i])
             elif op == "sub":
-                for i in range(NP): self.sub2(A[i], R[i], A[i])
+                for i in range(self.NP): self.sub2(A[i], R[i], A[i])
             elif op == "rsub":
-                for i in range(NP): self.sub2(R[i], A[i], A[i])
+                for i in range(self.NP): self.sub2(R[i], A[i], A[i])
             elif op == "mul":
-                for i in range(NP): self.mul2(A[i], R[i], A[i])
+                for i in range(self.NP): self.mul2(A[i], R[i], A[i])
             elif op == "divp":
                 self.divp(A, R, A)
             elif op == "rdivp":
                 self.divp(R, A, A)
             elif op == "addto":
-                for i in range(NP): self.add2(R[i], A[i], R[i])
+                for i in range(self.NP): self.add2(R[i], A[i], R[i])
             elif op == "accum":
                 tail = self.newlabel("acc")
                 self.e("@!%%pfull bra.uni %s;" % tail)
-                for i in range(NP): self.add2(R[i], A[i], R[i])
+                for i in range(self.NP): self.add2(R[i], A[i], R[i])
                 self.jump()
                 self.label(tail)
                 m = self.packs(self.mask_tail(self.scalars(A)))
-                for i in range(NP): self.add2(R[i], m[i], R[i])
+                for i in range(self.NP): self.add2(R[i], m[i], R[i])
             else:
                 raise ValueError(op)
         self.jump()
@@ -1128,8 +1137,8 @@ class Kernel:
                 u = self.rcp1pabs(u)
             uu = self.splat(u)
             if op == "rdivpu":
-                self.divp([uu] * NP, A, A)
-            for i in range(NP):
+                self.divp([uu] * self.NP, A, A)
+            for i in range(self.NP):
                 if op == "ldu": self.e("mov.b64 %s, %s;" % (A[i], uu))
                 elif op == "addu": self.add2(A[i], uu, A[i])
                 elif op == "subu": self.sub2(A[i], uu, A[i])
@@ -1142,7 +1151,7 @@ class Kernel:
             ua, ub = self.uniform(ia), self.uniform(ib)
             self.fetch()
             uu, vv = self.splat(ua), self.splat(ub)
-            for i in range(NP): self.fma2(A[i], uu, vv, A[i])
+            for i in range(self.NP): self.fma2(A[i], uu, vv, A[i])
         elif op == "lds":
             a = self.slot_addr(); self.fetch(); self.lds_v(a, A)
         elif op == "sts":
@@ -1150,7 +1159,7 @@ class Kernel:
         elif op in ("adds", "subs", "rsubs", "muls", "divps", "rdivps"):
             a = self.slot_addr(); self.fetch()
             T = self.lds_v(a)
-            for i in range(NP):
+            for i in range(self.NP):
                 if op == "adds": self.add2(A[i], T[i], A[i])
                 elif op == "subs": self.sub2(A[i], T[i], A[i])
                 elif op == "rsubs": self.sub2(T[i], A[i], A[i])
@@ -1202,18 +1211,18 @@ class Kernel:
         elif op == "neg":
             self.fetch()
             m = self.K(-1.0)
-            for i in range(NP): self.mul2(A[i], m, A[i])
+            for i in range(self.NP): self.mul2(A[i], m, A[i])
         elif op == "onemsq":
             self.fetch()
             m, one = self.K(-1.0), self.K(1.0)
-            for i in range(NP): self.fma2(self.mul2(A[i], m), A[i], one, A[i])
+            for i in range(self.NP): self.fma2(self.mul2(A[i], m), A[i], one, A[i])
         elif op == "yomy":
             self.fetch()
             m, one = self.K(-1.0), self.K(1.0)
-            for i in range(NP): self.mul2(A[i], self.fma2(A[i], m, one), A[i])
+            for i in range(self.NP): self.mul2(A[i], self.fma2(A[i], m, one), A[i])
         elif op == "rbf16":
             self.fetch()
-            for i in range(NP):
+            for i in range(self.NP):
                 lo, hi = self.unpack(A[i])
                 w, l2, h2 = self.r(), self.r(), self.r()
                 self.e("cvt.rn.bf16x2.f32 %s, %s, %s;" % (w, hi, lo))
@@ -1223,7 +1232,7 @@ class Kernel:
         elif op == "rowsum":     # arg: scratch buffer (bits 0..1), barrier after the read as well (bit 2)
             boff, t, psync = self.r(), self.r(), self.p()
             self.e("and.b32 %s, %%arg, 3;" % boff)
-            self.e("shl.b32 %s, %s, 6;" % (boff, boff))
+            self.e("shl.b32 %s, %s, %d;" % (boff, boff, self.red_shift))
             self.e("and.b32 %s, %%arg, 4;" % t)
             self.e("setp.ne.u32 %s, %s, 0;" % (psync, t))
             self.fetch()
@@ -1231,7 +1240,7 @@ class Kernel:
         elif op == "rowsumu":    # the same with arg & 7, then acc = acc * U[arg >> 3]
             boff, t, psync, iu = self.r(), self.r(), self.p(), self.r()
             self.e("and.b32 %s, %%arg, 3;" % boff)
-            self.e("shl.b32 %s, %s, 6;" % (boff, boff))
+            self.e("shl.b32 %s, %s, %d;" % (boff, boff, self.red_shift))
             self.e("and.b32 %s, %%arg, 4;" % t)
             self.e("setp.ne.u32 %s, %s, 0;" % (psync, t))
             self.e("shr.u32 %s, %%arg, 3;" % iu)
@@ -1291,11 +1300,11 @@ class Kernel:
             T = self.lds_v(a)
             tail, st = self.newlabel("as"), self.newlabel("as")
             self.e("@!%%pfull bra.uni %s;" % tail)
-            for i in range(NP): self.add2(T[i], A[i], T[i])
+            for i in range(self.NP): self.add2(T[i], A[i], T[i])
             self.e("bra.uni %s;" % st)
             self.label(tail)
             m = self.packs(self.mask_tail(self.scalars(A)))
-            for i in range(NP): self.add2(T[i], m[i], T[i])
+            for i in range(self.NP): self.add2(T[i], m[i], T[i])
             self.label(st)
             self.sts_v(a, T)
         elif op.startswith("ascal"):
@@ -1341,8 +1350,8 @@ class Kernel:
         self.e("add.u32 %s, %s, %s;" % (a, a, base))
         self.e("@%s st.shared.f32 [%s+%d], %s;" % (pr, a, OFF_RED, s))
         self.e("bar.sync 0;")
-        q = [self.rd() for _ in range(NT // 64)]       # the 16 per-warp partials as 8 packed pairs, summed pairwise
-        for i in range(NT // 128):
+        q = [self.rd() for _ in range(self.NT // 64)]       # the 16 per-warp partials as 8 packed pairs, summed pairwise
+        for i in range(self.NT // 128):
             self.e("ld.shared.v2.b64 {%s, %s}, [%s+%d];" % (q[2 * i], q[2 * i + 1], base, OFF_RED + 16 * i))
         while len(q) > 1:
             q = [self.add2(q[2 * i], q[2 * i + 1]) for i in range(len(q) // 2)]
@@ -1356,7 +1365,7 @@ class Kernel:
         if scale:
             self.e("mul.f32 %s, %s, %s;" % (tot, tot, scale))
         tt = self.splat(tot)
-        for i in range(NP): self.e("mov.b64 %s, %s;" % (A[i], tt))
+        for i in range(self.NP): self.e("mov.b64 %s, %s;" % (A[i], tt))
 
     def leaf_uload(self):
         """U[arg & 511] = scalar operand[arg >> 9], by thread 0"""
@@ -1453,10 +1462,10 @@ class Kernel:
         self.e("shl.b64 %s, %s, 2;" % (o, o))
         self.e("add.u64 %s, %s, %s;" % (o, o, self.param(P_COLPART, "u64")))
         sc = self.scalars(A)
-        for j in range(V):
+        for j in range(self.V):
             pr = self.p()
             self.e("setp.lt.u32 %s, %s, %s;" % (pr, self.lane_pos(j), cols))
-            self.e("@%s st.global.f32 [%s+%d], %s;" % (pr, o, ((j >> 2) * NT * 4 + (j & 3)) * 4, sc[j]))
+            self.e("@%s st.global.f32 [%s+%d], %s;" % (pr, o, ((j >> 2) * self.NT * 4 + (j & 3)) * 4, sc[j]))
 
     def leaf_scalout(self, values=None):
         """scalar partial sum: scalpart[arg][cta] = block sum in fp64 of acc (or of the given scalars)"""
@@ -1483,15 +1492,15 @@ class Kernel:
         self.e("setp.eq.u32 %s, %s, 0;" % (pr, lane))
         self.e("shl.b32 %s, %s, 3;" % (a, warp))
         self.e("add.u32 %s, %s, %%ub;" % (a, a))
-        self.e("@%s st.shared.f64 [%s+%d], %s;" % (pr, a, OFF_RED + 256, s))
+        self.e("@%s st.shared.f64 [%s+%d], %s;" % (pr, a, OFF_RED + 512, s))
         self.e("bar.sync 0;")
         skip = self.newlabel("so")
         self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
         tot = self.fd()
         self.e("mov.f64 %s, 0d0000000000000000;" % tot)
-        for i in range(NT // 32):
+        for i in range(self.NT // 32):
             d = self.fd()
-            self.e("ld.shared.f64 %s, [%%ub+%d];" % (d, OFF_RED + 256 + 8 * i))
+            self.e("ld.shared.f64 %s, [%%ub+%d];" % (d, OFF_RED + 512 + 8 * i))
             self.e("add.f64 %s, %s, %s;" % (tot, tot, d))
         self.e("st.global.f64 [%s], %s;" % (o, tot))
         self.label(skip)
@@ -1547,7 +1556,7 @@ class Kernel:
         e("mov.u32 %s, dsm;" % sa)
         e("mad.lo.u32 %s, %s, 8, %s;" % (sa, i_, sa))
         e("st.shared.v2.u32 [%s], {%s, %s};" % (sa, c, a))
-        e("add.u32 %s, %s, %d;" % (i_, i_, NT))
+        e("add.u32 %s, %s, %d;" % (i_, i_, self.NT))
         e("bra %s;" % lp)
         self.label(ld_)
         e("bar.sync 0;")
@@ -1607,7 +1616,7 @@ class Kernel:
         head = []
         head.append(".const .align 8 .b64 KT_%s[%d] = {%s};" % (self.name, max(1, len(self.kt)), ", ".join("0x%016X" % w for w in self.kt) or "0"))
         head.append(".visible .entry %s(.param .align 8 .b8 VP[%d])" % (self.name, P_SIZE))
-        head.append(".maxntid %d, 1, 1" % NT)
+        head.append(".maxntid %d, 1, 1" % self.NT)
         head.append(".minnctapersm %d" % self.ctas)
         head.append("{")
         decl = []
@@ -1625,15 +1634,20 @@ class Kernel:
         return "\n".join(head + decl + body + ["}"]) + "\n"
 
 
-VARIANTS = [("dragon_vm_wide", 7, 1), ("dragon_vm_dense", 3, 2)]   # name, register slots, CTAs per SM
+# name, register slots, CTAs per SM, threads per CTA.  The generator also takes 1024 threads (four elements per
+# thread, 32 warps per SM with the wide build's slots); measured on the row DAGs that was 13 % slower than 512
+# (the fixed cost of a dispatch is then spread over half the arithmetic), so no such kernel is built.  Loading the
+# instruction pairs two leaves ahead (so that the indexed branch of a short leaf never waits for shared memory)
+# was 4 % slower as well: the two register moves per dispatch cost more than the wait.
+VARIANTS = [("dragon_vm_wide", 7, 1, 512), ("dragon_vm_dense", 3, 2, 512)]
 
 
 def generate():
     out = [".version 8.8", ".target sm_100a", ".address_size 64", "", ".extern .shared .align 16 .b8 dsm[];",
            # 2/pi = 0x0.A2F9836E4E44... behind one word of zeros (its integer part), most significant word first
            ".const .align 4 .b32 TWO_OVER_PI[9] = {0x00000000, 0xA2F9836E, 0x4E441529, 0xFC2757D1, 0xF534DDC0, 0xDB629599, 0x3C439041, 0xFE5163AB, 0xDEBBC561};", ""]
-    for name, nr, ctas in VARIANTS:
-        out.append(Kernel(name, nr, ctas).build())
+    for name, nr, ctas, threads in VARIANTS:
+        out.append(Kernel(name, nr, ctas, threads).build())
     return "\n".join(out)
 
 

@@ -34,7 +34,9 @@ def test_instruction_lists_match_the_header():
     assert int(re.search(r"kJointStride = (\d+)", h).group(1)) == gen.JOINT_STRIDE
     assert int(re.search(r"kVmScalarAccs = (\d+)", h).group(1)) == gen.N_SACC
     wide, dense = re.search(r"kVmRegsWide = (\d+), kVmRegsDense = (\d+)", h).groups()
-    assert {(n, r, c) for n, r, c in gen.VARIANTS} == {("dragon_vm_wide", int(wide), 1), ("dragon_vm_dense", int(dense), 2)}
+    assert set(gen.VARIANTS) == {("dragon_vm_wide", int(wide), 1, 512), ("dragon_vm_dense", int(dense), 2, 512)}
+    threads, vec = re.search(r"DRAGON_VM_THREADS (\d+)", h).group(1), re.search(r"DRAGON_VM_VEC (\d+)", h).group(1)
+    assert int(threads) * int(vec) == gen.TILE
 
 
 def test_parameter_block_offsets(tmp_path):
