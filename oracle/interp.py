@@ -12,6 +12,7 @@ tensor per operator, no fusion, no reordering.
   Add, Sub, Mul      a+b, a-b, a*b with NumPy broadcasting
   Div(a, b)          a / (1 + |b|)
   Sin, Tanh, Sigmoid, ReLU   the usual; Exp(x) = exp(clip(x, -10, 10))
+  Sqrt, Reciprocal   sqrt(x), 1/x (the updaters of Sec. 3.2 divide by a root: RMSProp, Adam)
   Sum, Mean          over the last axis, result broadcast back to the operand's shape
   InnerProduct(X, W) X[M,K] @ W[N,K]^T; operands are rounded to bf16 first (the
                      contraction consumes bf16), products and sums are wide
@@ -21,7 +22,7 @@ tensor per operator, no fusion, no reordering.
 Gradient rules (dy = gradient of the output): Add (dy,dy); Sub (dy,-dy);
 Mul (dy*b, dy*a); Div (dy/(1+|b|), -dy*a*sgn(b)/(1+|b|)^2) with sgn(0)=0;
 Sin dy*cos x; Exp dy*y*[-10<=x<=10]; Tanh dy*(1-y^2); Sigmoid dy*y*(1-y);
-ReLU dy*[x>0]; Sum: row-sum of dy broadcast back; Mean: the same / C;
+ReLU dy*[x>0]; Sqrt dy/(2y); Reciprocal -dy*y^2; Sum: row-sum of dy broadcast back; Mean: the same / C;
 InnerProduct dX = dY@W, dW = dY^T@X (dY rounded to bf16 first);
 BiasAdd (dy, column sums of dy); SoftmaxCrossEntropy dZ = dL*(softmax - onehot)/M.
 A gradient with respect to a broadcast operand is summed over the broadcast
@@ -80,6 +81,10 @@ def _forward(op, ins, dtype, bf16_contraction=True):
         return 1 / (1 + np.exp(-ins[0]))
     if t == "ReLU":
         return np.maximum(ins[0], 0)
+    if t == "Sqrt":
+        return np.sqrt(ins[0])
+    if t == "Reciprocal":
+        return 1 / ins[0]
     if t == "Sum":
         return np.broadcast_to(ins[0].sum(axis=-1, keepdims=True), ins[0].shape).copy()
     if t == "Mean":
@@ -124,6 +129,10 @@ def _backward(op, ins, out, dy, pos, bf16_contraction=True):
         g[0] = dy * out * (1 - out)
     elif t == "ReLU":
         g[0] = dy * (ins[0] > 0)
+    elif t == "Sqrt":
+        g[0] = dy / (2 * out)
+    elif t == "Reciprocal":
+        g[0] = -dy * out * out
     elif t in ("Sum", "Mean"):
         r = np.broadcast_to(np.broadcast_to(dy, ins[0].shape).sum(axis=-1, keepdims=True), ins[0].shape)
         g[0] = r / ins[0].shape[-1] if t == "Mean" else r.copy()

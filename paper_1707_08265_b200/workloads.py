@@ -188,16 +188,47 @@ def random_row_dag(rows, cols, seed, n_full=6, n_row=2, n_ops=1024, n_fetch=4):
 
 def updater(shape, kind="sgd"):
     """The weight update as a graph of its own (Sec. 3.2 of the paper: the updater is split from the
-    training graph so that neither becomes cyclic).  sgd: W' = W - lr*g.  momentum: v' = mu*v + g,
-    W' = W - lr*v'.  lr and mu are scalar tensors; returns (graph, ids)."""
+    training graph so that neither becomes cyclic; it names Momentum, RMSProp and Adam).
+      sgd:      W' = W - lr*g
+      momentum: v' = mu*v + g,  W' = W - lr*v'
+      rmsprop:  v' = rho*v + (1-rho)*g*g,  W' = W - lr * g / (sqrt(v') + eps)
+      adam:     m' = beta1*m + (1-beta1)*g,  v' = beta2*v + (1-beta2)*g*g,  W' = W - lr * m' / (sqrt(v') + eps)
+                (lr and eps carry the bias corrections of the step: lr_t = lr*sqrt(1-beta2^t)/(1-beta1^t))
+    The hyper-parameters are scalar tensors, 1-x fed beside x; returns (graph, ids)."""
     g = GraphDesc()
-    ids = {"W": g.tensor("W", shape), "g": g.tensor("g", shape), "lr": g.tensor("lr", [])}
+    ids = {"W": g.tensor("W", shape), "g": g.tensor("g", shape)}
+
+    def scalars(*names):
+        for n in names:
+            ids[n] = g.tensor(n, [])
+
+    def decayed(state, keep, mix, value, name):      # keep*state + mix*value
+        return g.op("Add", [g.op("Mul", [ids[keep], ids[state]], name + "_keep"), g.op("Mul", [ids[mix], value], name + "_mix")], name)
+
     if kind == "sgd":
+        scalars("lr")
         step = g.op("Mul", [ids["lr"], ids["g"]], "step")
-    else:
+    elif kind == "momentum":
+        ids["lr"] = g.tensor("lr", [])
         ids["v"] = g.tensor("v", shape)
         ids["mu"] = g.tensor("mu", [])
         ids["v_new"] = g.op("Add", [g.op("Mul", [ids["mu"], ids["v"]], "mv"), ids["g"]], "v_new")
         step = g.op("Mul", [ids["lr"], ids["v_new"]], "step")
+    elif kind in ("rmsprop", "adam"):
+        if kind == "adam":
+            ids["m"] = g.tensor("m", shape)
+        ids["v"] = g.tensor("v", shape)
+        if kind == "adam":
+            scalars("lr", "beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "eps")
+            ids["m_new"] = decayed("m", "beta1", "one_minus_beta1", ids["g"], "m_new")
+            num, keep, mix = ids["m_new"], "beta2", "one_minus_beta2"
+        else:
+            scalars("lr", "rho", "one_minus_rho", "eps")
+            num, keep, mix = ids["g"], "rho", "one_minus_rho"
+        ids["v_new"] = decayed("v", keep, mix, g.op("Mul", [ids["g"], ids["g"]], "g2"), "v_new")
+        den = g.op("Add", [g.op("Sqrt", [ids["v_new"]], "root"), ids["eps"]], "den")
+        step = g.op("Mul", [g.op("Mul", [ids["lr"], num], "lr_num"), g.op("Reciprocal", [den], "inv")], "step")
+    else:
+        raise ValueError(kind)
     ids["W_new"] = g.op("Sub", [ids["W"], step], "W_new")
     return g, ids

@@ -73,6 +73,7 @@ KINKS = {"ReLU": [0.0], "Exp": [-10.0, 10.0]}
     ("Mul", [[3, 4], [3, 4]]), ("Div", [[3, 4], [4]]), ("Div", [[4], [3, 4]]), ("Sin", [[3, 4]]),
     ("Exp", [[3, 4]]), ("Tanh", [[3, 4]]), ("Sigmoid", [[3, 4]]), ("ReLU", [[3, 4]]),
     ("Sum", [[3, 4]]), ("Mean", [[3, 4]]), ("Sum", [[4]]), ("Mean", [[4]]),
+    ("Sqrt", [[3, 4]]), ("Reciprocal", [[3, 4]]),
 ])
 def test_operator_gradients_match_finite_differences(type_, shapes):
     rng = np.random.default_rng(11)
@@ -84,6 +85,8 @@ def test_operator_gradients_match_finite_differences(type_, shapes):
     gids = g.grad([obj], ins)
     scale = 6.0 if type_ == "Exp" else 2.0
     feeds = [rng.standard_normal(size=s) * scale for s in shapes] + [rng.standard_normal(size=g.shape(out))]
+    if type_ in ("Sqrt", "Reciprocal"):                      # positive arguments away from zero
+        feeds[0] = np.abs(feeds[0]) + 0.3
     for f, s in zip(feeds, shapes):                          # keep away from kinks
         for kpt in KINKS.get(type_, []) + ([0.0] if type_ == "Div" else []):
             f[np.abs(f - kpt) < 1e-2] += 0.05
@@ -93,6 +96,40 @@ def test_operator_gradients_match_finite_differences(type_, shapes):
         fd = interp.finite_difference(g.desc, inputs, feeds, [obj], wrt, h=1e-6)
         assert gv.shape == tuple(g.shape(wrt))
         assert np.allclose(gv, fd, rtol=2e-6, atol=2e-6), (type_, wrt, gv, fd)
+
+
+def test_sqrt_reciprocal_closed_forms_and_updaters():
+    # values: exact squares and powers of two; derivative of sqrt(x) * (1/x) = x^(-1/2) is -x^(-3/2)/2
+    g, ins, out = _single_op_graph("Sqrt", [[4]])
+    (v,) = interp.run_function(g.desc, ins, [out], [np.array([0.0, 1.0, 4.0, 2.25])])
+    assert np.array_equal(v, [0.0, 1.0, 2.0, 1.5])
+    g, ins, out = _single_op_graph("Reciprocal", [[3]])
+    (v,) = interp.run_function(g.desc, ins, [out], [np.array([1.0, -4.0, 0.125])])
+    assert np.array_equal(v, [1.0, -0.25, 8.0])
+    gd = wl.GraphDesc()
+    x = gd.tensor("x", [3])
+    y = gd.op("Mul", [gd.op("Sqrt", [x], "s"), gd.op("Reciprocal", [x], "r")], "y")
+    (dx,) = gd.grad([y], [x])
+    xv = np.array([0.5, 1.0, 9.0])
+    (got,) = interp.run_function(gd.desc, [x], [dx], [xv])
+    assert np.allclose(got, -0.5 * xv ** -1.5, rtol=1e-14)
+    # the updater graphs against their formulas written out (Sec. 3.2 names Momentum, RMSProp, Adam)
+    rng = np.random.default_rng(4)
+    W, gr, m, v = (rng.standard_normal(7) for _ in range(4))
+    v = np.abs(v)
+    lr, b1, b2, eps = 0.01, 0.9, 0.999, 1e-8
+    u, ids = wl.updater([7], "adam")
+    ins_ = [ids[k] for k in ("W", "g", "m", "v", "lr", "beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "eps")]
+    Wn, mn, vn = interp.run_function(u.desc, ins_, [ids["W_new"], ids["m_new"], ids["v_new"]],
+                                     [W, gr, m, v] + [np.asarray(c) for c in (lr, b1, 1 - b1, b2, 1 - b2, eps)])
+    m2, v2 = b1 * m + (1 - b1) * gr, b2 * v + (1 - b2) * gr * gr
+    assert np.allclose(mn, m2, rtol=1e-15) and np.allclose(vn, v2, rtol=1e-15)
+    assert np.allclose(Wn, W - lr * m2 / (np.sqrt(v2) + eps), rtol=1e-14)
+    u, ids = wl.updater([7], "rmsprop")
+    ins_ = [ids[k] for k in ("W", "g", "v", "lr", "rho", "one_minus_rho", "eps")]
+    Wn, vn = interp.run_function(u.desc, ins_, [ids["W_new"], ids["v_new"]], [W, gr, v] + [np.asarray(c) for c in (lr, 0.9, 0.1, eps)])
+    v2 = 0.9 * v + 0.1 * gr * gr
+    assert np.allclose(vn, v2, rtol=1e-15) and np.allclose(Wn, W - lr * gr / (np.sqrt(v2) + eps), rtol=1e-14)
 
 
 def test_same_operand_twice_and_fanout_accumulate():
