@@ -213,7 +213,13 @@ def build_config(cfg, B, torch, seeds, rows=16384):
         g, inputs, outputs = wl.random_dag(n, seeds["random_dag"]["seed"])
         return dict(g=g, inputs=inputs, outputs=outputs, units=n, unit=UNIT, bound="hbm", alg=None,
                     what="config 3: random 64-operator elementwise DAG, 4 x fp32[2^27], 2 fetched sinks, forward")
-    if cfg == 6:   # not one of the five: the SGD weight update as a graph of its own, 12 bytes per element
+    if cfg == 6:   # not one of the five: the Adam weight update as a graph of its own, 28 bytes per element
+        n = 1 << 26
+        g, ids = wl.updater([n], "adam")
+        names = ("W", "g", "m", "v", "lr", "beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "eps")
+        return dict(g=g, inputs=[ids[k] for k in names], outputs=[ids[k] for k in ("W_new", "m_new", "v_new")], units=n, unit=UNIT,
+                    bound="hbm", alg=28.0 * n, what="Adam updater, fp32[2^26]: W, g, m, v in; W, m, v out (28 B/element)")
+    if cfg == 8:   # not one of the five: the SGD weight update, 12 bytes per element
         n = 1 << 26
         g, ids = wl.updater([n], "sgd")
         return dict(g=g, inputs=[ids["W"], ids["g"], ids["lr"]], outputs=[ids["W_new"]], units=n, unit=UNIT, bound="hbm", alg=12.0 * n,
@@ -248,7 +254,10 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None):
         ti = g.desc["tensors"][t]
         if ti["dtype"] == "i32":
             return torch.randint(0, 4096, tuple(ti["shape"]), generator=gen, device="cuda", dtype=torch.int32)
-        return torch.empty(tuple(ti["shape"]), dtype=torch.float32, device="cuda").normal_(generator=gen).to(tdt[ti["dtype"]])
+        t_ = torch.empty(tuple(ti["shape"]), dtype=torch.float32, device="cuda").normal_(generator=gen)
+        if cfg == 6 and ti["name"] in ("v", "eps", "lr", "beta1", "beta2", "one_minus_beta1", "one_minus_beta2"):
+            t_ = t_.abs() * 0.01 + 1e-3     # second moments and hyper-parameters are positive
+        return t_.to(tdt[ti["dtype"]])
 
     f = B.Graph.from_desc(g.desc).function(inputs, outputs)
     feeds = [dev_random(t) if u else None for t, u in zip(inputs, f.used_inputs())]
@@ -335,9 +344,9 @@ def main():
     ap.add_argument("--rows", type=int, default=16384, help="rows of workload 5 (default: its 16384; smaller for profiler captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-other-configs", action="store_true", help="leave the \"configs\" entry (workloads 1, 3, 4, 5) out")
-    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7],
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8],
                     help="2 (default) is the benchmark workload with all five on its line; another number prints that workload alone "
-                         "(6: SGD updater, 7: one gradient stage per objective)")
+                         "(6: Adam updater, 7: one gradient stage per objective, 8: SGD updater)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)

@@ -55,6 +55,9 @@ enum { DRAGON_F32 = 0, DRAGON_BF16 = 1, DRAGON_I32 = 2 };
  *   ADD, SUB, MUL          a+b, a-b, a*b with right-aligned broadcasting among [], [C], [R,C]
  *   DIV                    a / (1 + |b|)
  *   EXP                    exp(min(max(x, -10), 10))
+ *   SQRT, RECIPROCAL       sqrt(x), 1/x (the RMSProp and Adam updaters of Sec. 3.2 divide by a root);
+ *                          approximate instructions of at most one unit in the last place, arguments
+ *                          below 2^-126 in magnitude count as zero
  *   SUM, MEAN              over the last axis, result broadcast back to the operand's shape
  *   INNER_PRODUCT(X, W)    Y[m,n] = sum_k X[m,k] * W[n,k]; operands are consumed as bf16,
  *                          accumulation is fp32
@@ -73,7 +76,7 @@ enum {
   DRAGON_OP_SIN = 4, DRAGON_OP_EXP = 5, DRAGON_OP_TANH = 6, DRAGON_OP_SIGMOID = 7,
   DRAGON_OP_RELU = 8, DRAGON_OP_SUM = 9, DRAGON_OP_MEAN = 10,
   DRAGON_OP_INNER_PRODUCT = 11, DRAGON_OP_BIAS_ADD = 12, DRAGON_OP_SOFTMAX_CROSS_ENTROPY = 13,
-  DRAGON_OP_OPAQUE = 16,
+  DRAGON_OP_SQRT = 14, DRAGON_OP_RECIPROCAL = 15, DRAGON_OP_OPAQUE = 16,
   DRAGON_OP_COUNT_ = 17
 };
 
@@ -139,6 +142,17 @@ int dragon_function_rename_dictionary(const dragon_function_t* f, dragon_id* anc
  * input of its producing step (in place)}.  Returns their number.  Two tensors whose step ranges
  * overlap never share bytes, except an in-place output and the input it replaces. */
 int dragon_function_workspace_tensors(const dragon_function_t* f, int64_t* out, int cap);
+
+/* In-place use.  The updater graphs of Sec. 3.2 overwrite their state (W, momentum, second moment), and
+ * Sec. 2.4 is about operators that write over their input.  Returns 1 if fetch position `output` may be
+ * given the very same device pointer as feed position `input` in dragon_run(), 0 if not, a negative
+ * code for bad positions.  It is 1 exactly when the function is a single elementwise launch over a
+ * flat domain, both tensors have the domain's shape and the same type, and the program reads the
+ * input for the last time before it first writes the output: every thread then overwrites only
+ * elements it has already read (the copy of a tile that is fetched ahead of time is never a tile that
+ * has been written).  The state of an update then stays in the caller's device memory from step to
+ * step.  Any other overlap between feeds and fetches is undefined. */
+int dragon_function_can_alias(const dragon_function_t* f, int input, int output);
 
 /* One byte per listed input: 1 if the pruned function reads it. */
 int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flag_per_input, int n_in);
@@ -232,7 +246,7 @@ int dragon_softmax_ce_loss_static(const void* logits, int dtype, const int32_t* 
                                   float* loss_out, void* cuda_stream);
 
 /* Host instantiation of the VM's elementary functions (fn: DRAGON_OP_SIN, _EXP, _TANH,
- * _SIGMOID; DRAGON_OP_DIV evaluates 1/(1+|x|); 100 + DRAGON_OP_SIN evaluates the cosine),
+ * _SIGMOID, _SQRT, _RECIPROCAL; DRAGON_OP_DIV evaluates 1/(1+|x|); 100 + DRAGON_OP_SIN evaluates the cosine),
  * for accuracy sweeps on machines without a GPU.  x, y: host arrays of n floats. */
 int dragon_host_math(int fn, const float* x, float* y, int n);
 

@@ -16,7 +16,8 @@ ERR_NO_PATH, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = -6, -7, -8,
 F32, BF16, I32 = 0, 1, 2
 DTYPES = {"f32": F32, "bf16": BF16, "i32": I32}
 OPS = {"Add": 0, "Sub": 1, "Mul": 2, "Div": 3, "Sin": 4, "Exp": 5, "Tanh": 6, "Sigmoid": 7, "ReLU": 8,
-       "Sum": 9, "Mean": 10, "InnerProduct": 11, "BiasAdd": 12, "SoftmaxCrossEntropy": 13, "Opaque": 16}
+       "Sum": 9, "Mean": 10, "InnerProduct": 11, "BiasAdd": 12, "SoftmaxCrossEntropy": 13, "Sqrt": 14,
+       "Reciprocal": 15, "Opaque": 16}
 
 _lib = None
 
@@ -37,6 +38,7 @@ _SIGNATURES = {
     "dragon_function_kept_ops": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int),
                                             _c.POINTER(_c.c_int32), _c.POINTER(_c.c_uint32), _c.c_int, _c.POINTER(_c.c_int)]),
     "dragon_function_used_inputs": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_uint8), _c.c_int]),
+    "dragon_function_can_alias": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_int]),
     "dragon_function_num_launches": (_c.c_int, [_c.c_void_p]),
     "dragon_function_describe": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_int]),
     "dragon_function_vm_step": (_c.c_int, [_c.c_void_p, _c.c_int, _c.POINTER(_c.c_int64), _c.POINTER(_c.c_uint32), _c.c_int,
@@ -204,6 +206,12 @@ class Function:
         if r < 0:
             raise DragonError(r, "dragon_function_used_inputs")
         return list(buf[:self.n_in])
+
+    def can_alias(self, input_pos, output_pos):
+        r = lib().dragon_function_can_alias(self.h, input_pos, output_pos)
+        if r < 0:
+            raise DragonError(r, "dragon_function_can_alias")
+        return bool(r)
 
     def num_launches(self):
         return lib().dragon_function_num_launches(self.h)

@@ -35,6 +35,7 @@ int infer_shape(const Graph& g, int type, const dragon_id* in, int n_in, Shape* 
       if (!broadcast_shapes(T(0).shape, T(1).shape, out)) { set_error("operands '%s' and '%s' do not broadcast", T(0).name.c_str(), T(1).name.c_str()); return DRAGON_ERR_SHAPE; }
       return DRAGON_OK;
     case DRAGON_OP_SIN: case DRAGON_OP_EXP: case DRAGON_OP_TANH: case DRAGON_OP_SIGMOID: case DRAGON_OP_RELU:
+    case DRAGON_OP_SQRT: case DRAGON_OP_RECIPROCAL:
     case DRAGON_OP_SUM: case DRAGON_OP_MEAN:
       if (n_in != 1) { set_error("unary operator takes 1 input"); return DRAGON_ERR_INVALID_ARG; }
       if (!is_float(0)) { set_error("elementwise operators take f32/bf16 tensors"); return DRAGON_ERR_DTYPE; }
@@ -238,6 +239,33 @@ int dragon_function_used_inputs(const dragon_function_t* f, uint8_t* flags, int 
   if (!f || (n_in > 0 && !flags) || n_in != f->n_in) { set_error("dragon_function_used_inputs: bad argument"); return DRAGON_ERR_INVALID_ARG; }
   if (n_in) std::memcpy(flags, f->prune.used_inputs.data(), (size_t)n_in);
   return DRAGON_OK;
+}
+
+int dragon_function_can_alias(const dragon_function_t* f, int input, int output) {
+  if (!f || input < 0 || input >= f->n_in || output < 0 || output >= f->n_out) { set_error("dragon_function_can_alias: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  const Plan& P = f->plan;
+  if (!f->not_executable.empty() || P.steps.size() != 1 || P.steps[0].kind != ST_VM) return 0;
+  const VmSegment& sg = P.segs[P.steps[0].seg];
+  if (sg.row_mode) return 0;
+  const std::vector<VmAccess> acc = vm_operand_accesses(sg);
+  int oi = -1, oo = -1;
+  for (size_t k = 0; k < sg.operand_mem.size(); ++k) {
+    const MemRef& m = P.mems[sg.operand_mem[k]];
+    if (sg.operand_kind[k] != (uint32_t)vm::K_FULL) continue;
+    if (m.where == MEM_FEED && m.index == input) oi = (int)k;
+    if (m.where == MEM_FETCH && m.index == output) oo = (int)k;
+  }
+  if (oi < 0 || oo < 0) return 0;
+  const MemRef &mi = P.mems[sg.operand_mem[oi]], &mo = P.mems[sg.operand_mem[oo]];
+  if (mi.dtype != mo.dtype || mi.shape.numel() != mo.shape.numel() || mi.shape.numel() != sg.n) return 0;
+  // several memrefs may name the same position: every load of the input, every store of the output
+  int last_load = -1, first_store = 1 << 30;
+  for (size_t k = 0; k < sg.operand_mem.size(); ++k) {
+    const MemRef& m = P.mems[sg.operand_mem[k]];
+    if (m.where == MEM_FEED && m.index == input) { if (sg.operand_kind[k] != (uint32_t)vm::K_FULL) return 0; last_load = std::max(last_load, acc[k].last_load); }
+    if (m.where == MEM_FETCH && m.index == output) { if (acc[k].last_load >= 0) return 0; first_store = std::min(first_store, acc[k].first_store); }
+  }
+  return (last_load >= 0 && last_load < first_store) ? 1 : 0;
 }
 
 int dragon_function_rename_dictionary(const dragon_function_t* f, dragon_id* ancestor, int n_tensors) {
@@ -693,6 +721,8 @@ int dragon_host_math(int fn, const float* x, float* y, int n) {
       case DRAGON_OP_TANH: y[i] = vmmath::tanh_f(x[i]); break;
       case DRAGON_OP_SIGMOID: y[i] = vmmath::sigmoid_f(x[i]); break;
       case DRAGON_OP_DIV: y[i] = vmmath::divp_f(1.f, x[i]); break;
+      case DRAGON_OP_SQRT: y[i] = vmmath::sqrt_f(x[i]); break;
+      case DRAGON_OP_RECIPROCAL: y[i] = vmmath::f_rcp(x[i]); break;
       default: set_error("dragon_host_math: unknown function %d", fn); return DRAGON_ERR_INVALID_ARG;
     }
   }

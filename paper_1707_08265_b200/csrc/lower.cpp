@@ -169,6 +169,8 @@ struct Lowerer {
       case DRAGON_OP_TANH: v = mop(M_TANH, in(0)); break;
       case DRAGON_OP_SIGMOID: v = mop(M_SIGMOID, in(0)); break;
       case DRAGON_OP_RELU: v = mop(M_RELU, in(0)); break;
+      case DRAGON_OP_SQRT: v = mop(M_SQRT, in(0)); break;
+      case DRAGON_OP_RECIPROCAL: v = mop(M_RCP, in(0)); break;
       case DRAGON_OP_SUM: v = mop(M_ROWSUM, in(0)); break;
       case DRAGON_OP_MEAN: v = mop(M_MUL, mop(M_ROWSUM, in(0)), konst(1.f / (float)to.shape.cols())); break;
       case DRAGON_OP_BIAS_ADD: v = mop(M_ADD, in(0), in(1)); break;
@@ -237,6 +239,8 @@ struct Lowerer {
       case DRAGON_OP_SIGMOID: add(0, mop(M_MUL, dy, mop(M_YOMY, fval[o]))); break;
       // [x > 0] = [relu(x) > 0]: reading the output keeps the input out of memory
       case DRAGON_OP_RELU: add(0, mop(M_MUL, dy, mop(M_STEP, fval[o]))); break;
+      case DRAGON_OP_SQRT: add(0, mop(M_MUL, dy, mop(M_MUL, konst(0.5f), mop(M_RCP, fval[o])))); break;      // dy / (2 y)
+      case DRAGON_OP_RECIPROCAL: add(0, mop(M_NEG, mop(M_MUL, dy, mop(M_MUL, fval[o], fval[o])))); break;     // -dy y^2
       case DRAGON_OP_SUM: case DRAGON_OP_MEAN: {
         int c = mop(M_ROWSUM, dy);
         if (op.type == DRAGON_OP_MEAN) c = mop(M_MUL, c, konst(1.f / (float)g.tensors[o].shape.cols()));
@@ -292,6 +296,28 @@ bool join_domain(Shape* dom, bool* has_dom, const Shape& s) {
 }  // namespace
 
 static size_t share_workspace(Plan* plan, size_t off);
+
+// per operand of a VM program: position (index into the code) of its last load and of its first store
+std::vector<VmAccess> vm_operand_accesses(const VmSegment& sg) {
+  std::vector<VmAccess> acc(sg.operand_mem.size());
+  for (int i = 0; i < (int)sg.code.size(); ++i) {
+    const uint32_t cs = sg.code[i] & 1023u, arg = sg.code[i] >> 14;
+    if (cs == (uint32_t)vm::P_UCONST) { ++i; continue; }
+    int opd = -1; bool store = false;
+    const uint32_t jg = cs / vm::kJointStride;
+    if (cs == (uint32_t)vm::P_GST || cs == (uint32_t)vm::P_GSTF || cs == (uint32_t)vm::P_GSTFL) { opd = (int)arg; store = true; }
+    else if (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_FMAURSTL) { opd = (int)(arg >> 9); store = true; }
+    else if (cs == (uint32_t)vm::P_GLD || cs == (uint32_t)vm::P_GLDF || (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_GLDR)) opd = (int)arg;
+    else if (cs == (uint32_t)vm::P_GLDA0 || cs == (uint32_t)vm::P_GLDA || cs == (uint32_t)vm::P_LDSW || cs == (uint32_t)vm::P_LDSWA ||
+             cs == (uint32_t)vm::P_GLDA0H || cs == (uint32_t)vm::P_LDSWAH ||
+             (cs < (uint32_t)vm::kFirstPlain && (jg == (uint32_t)vm::J_LDSWR || jg == (uint32_t)vm::J_LDSWAR || jg == (uint32_t)vm::J_LDSWARF))) opd = (int)(arg & 63u);
+    else if (cs == (uint32_t)vm::P_ULOAD) opd = (int)(arg >> 9);
+    if (opd < 0 || opd >= (int)acc.size()) continue;
+    if (store) acc[opd].first_store = std::min(acc[opd].first_store, i);
+    else acc[opd].last_load = i;
+  }
+  return acc;
+}
 
 int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs,
                    const std::vector<int>& outputs, int sm_count, Plan* plan) {
@@ -699,8 +725,7 @@ static size_t share_workspace(Plan* plan, size_t off) {
     mems[m].last_step = si;
   };
   // positions of the last load and the first store of every operand of a VM program
-  struct Access { int last_load = -1, first_store = 1 << 30; };
-  std::vector<std::vector<Access>> acc(n_steps);
+  std::vector<std::vector<VmAccess>> acc(n_steps);
   for (int si = 0; si < n_steps; ++si) {
     const Step& st = plan->steps[si];
     if (st.kind != ST_VM) {
@@ -712,23 +737,7 @@ static size_t share_workspace(Plan* plan, size_t off) {
       continue;
     }
     const VmSegment& sg = plan->segs[st.seg];
-    acc[si].resize(sg.operand_mem.size());
-    for (int i = 0; i < (int)sg.code.size(); ++i) {
-      const uint32_t cs = sg.code[i] & 1023u, arg = sg.code[i] >> 14;
-      if (cs == (uint32_t)vm::P_UCONST) { ++i; continue; }
-      int opd = -1; bool store = false;
-      const uint32_t jg = cs / vm::kJointStride;
-      if (cs == (uint32_t)vm::P_GST || cs == (uint32_t)vm::P_GSTF || cs == (uint32_t)vm::P_GSTFL) { opd = (int)arg; store = true; }
-      else if (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_FMAURSTL) { opd = (int)(arg >> 9); store = true; }
-      else if (cs == (uint32_t)vm::P_GLD || cs == (uint32_t)vm::P_GLDF || (cs < (uint32_t)vm::kFirstPlain && jg == (uint32_t)vm::J_GLDR)) opd = (int)arg;
-      else if (cs == (uint32_t)vm::P_GLDA0 || cs == (uint32_t)vm::P_GLDA || cs == (uint32_t)vm::P_LDSW || cs == (uint32_t)vm::P_LDSWA ||
-               cs == (uint32_t)vm::P_GLDA0H || cs == (uint32_t)vm::P_LDSWAH ||
-               (cs < (uint32_t)vm::kFirstPlain && (jg == (uint32_t)vm::J_LDSWR || jg == (uint32_t)vm::J_LDSWAR || jg == (uint32_t)vm::J_LDSWARF))) opd = (int)(arg & 63u);
-      else if (cs == (uint32_t)vm::P_ULOAD) opd = (int)(arg >> 9);
-      if (opd < 0 || opd >= (int)acc[si].size()) continue;
-      if (store) acc[si][opd].first_store = std::min(acc[si][opd].first_store, i);
-      else acc[si][opd].last_load = i;
-    }
+    acc[si] = vm_operand_accesses(sg);
     for (size_t i = 0; i < sg.operand_mem.size(); ++i) {
       if (acc[si][i].last_load >= 0) touch(si, sg.operand_mem[i], false);
       if (acc[si][i].first_store < (1 << 30)) touch(si, sg.operand_mem[i], true);
@@ -806,7 +815,7 @@ static std::string disassemble(const VmSegment& sg) {
   static const char* pn[] = {"ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls",
                              "divps", "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq",
                              "yomy", "divpgb", "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout",
-                             "scalout", "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "end"};
+                             "scalout", "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "end"};
   std::string s;
   char buf[64];
   for (size_t i = 0; i < sg.code.size(); ++i) {

@@ -39,7 +39,7 @@ struct MemRef {
 enum MOpc {
   M_ADD, M_SUB, M_MUL, M_DIVP,
   M_SIN, M_COS, M_EXPC, M_TANH, M_SIGMOID, M_RELU, M_NEG, M_STEP, M_CLAMPMASK, M_ONEMSQ, M_YOMY,
-  M_DIVPGB, M_RBF16, M_ROWSUM,
+  M_DIVPGB, M_RBF16, M_ROWSUM, M_SQRT, M_RCP,
   M_WIDEN,  // same value, wider logical shape (no instruction)
   M_STORE,  // write value a to memory mem
   M_ACCUM   // sum value a over the axes along which mem is smaller, write to mem
@@ -125,6 +125,10 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
                     const std::vector<MemRef>& mems, int sm_count, VmSegment* seg);
 
 std::string describe_plan(const Plan& p);
+
+// per operand of a VM program: position (index into the code) of its last load and of its first store
+struct VmAccess { int last_load = -1, first_store = 1 << 30; };
+std::vector<VmAccess> vm_operand_accesses(const VmSegment& sg);
 
 }  // namespace dragon
 

@@ -105,6 +105,8 @@ enum Plain : int {
   P_ROWSUMU,            // P_ROWSUM with arg & 7, then acc = acc * U[arg >> 3]   (a row mean)
   P_ACCUMS,             // S[arg] = S[arg] + (lane valid ? acc : 0): a loop-carried accumulator kept in shared memory
                         // (reduced outputs beyond the pinned register slots)
+  P_SQRT,               // acc = sqrt(acc)
+  P_RCP,                // acc = 1 / acc
   P_END,
   P_COUNT_
 };

@@ -35,6 +35,16 @@ VM_HD float f_rcp(float x) {
 #endif
 }
 
+VM_HD float sqrt_f(float x) {
+#if defined(__CUDA_ARCH__)
+  float r;
+  asm("sqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+  return r;
+#else
+  return sqrtf(x);
+#endif
+}
+
 VM_HD float f_from_bits(uint32_t u) {
 #if defined(__CUDA_ARCH__)
   return __uint_as_float(u);

@@ -49,7 +49,7 @@ N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "accums", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "end"]
 
 
 def f32bits(x):
@@ -1206,6 +1206,14 @@ class Kernel:
                     self.e("selp.f32 %s, 0fBF800000, %s, %s;" % (g, g, p1))
                     self.e("mul.f32 %s, %s, %s;" % (g, g, rr))
                     self.e("mul.f32 %s, %s, %s;" % (d, g, rr))
+                out.append(d)
+            self.packs(out, A)
+        elif op in ("sqrt", "rcp"):
+            self.fetch()
+            out = []
+            for s in self.scalars(A):
+                d = self.f()
+                self.e("%s.approx.ftz.f32 %s, %s;" % (op, d, s))
                 out.append(d)
             self.packs(out, A)
         elif op == "neg":

@@ -23,9 +23,15 @@ def sweep(lo_exp, hi_exp, per_binade=64):
     ("Tanh", -20, 8, [0.6, 0.5999999, 0.6000001, 9.0, 9.07, 9.1, 9.5, 10.0, 10.5, 20.0, 21.0, 90.0]),    # saturates exactly from 9.5 on at the latest
     ("Sigmoid", -20, 8, [86.0, -86.0, 88.7, -88.7, 100.0, -100.0]),
     ("Div", -20, 20, [1.0, -1.0]),
+    ("Sqrt", -40, 60, [1.0, 4.0, 2.0, 3.0e38]),                              # positive arguments only (see below)
+    ("Reciprocal", -60, 60, [1.0, -1.0, 3.0]),
 ])
 def test_elementary_functions_over_dense_sweeps(op, lo, hi, extra):
     x = np.concatenate([sweep(lo, hi), np.asarray(extra, np.float32), -np.asarray(extra, np.float32)]).astype(np.float32)
+    if op == "Sqrt":
+        x = np.abs(x[x != 0])
+    if op == "Reciprocal":
+        x = x[x != 0]
     n = x.size
     gd = wl.GraphDesc()
     xi = gd.tensor("x", [n])
@@ -46,6 +52,63 @@ def test_elementary_functions_over_dense_sweeps(op, lo, hi, extra):
     if op == "Tanh":      # a saturated tanh is exactly +-1 and its gradient exactly 0
         sat = np.abs(x) >= 9.5
         assert np.all(np.abs(got[0][sat]) == 1) and np.all(got[1][sat] == 0)
+
+
+def updater_case(kind, shape, seed=11):
+    g, ids = wl.updater(shape, kind)
+    rng = np.random.default_rng(seed)
+    W = rng.standard_normal(shape).astype(np.float32)
+    grad = (rng.standard_normal(shape) * 0.1).astype(np.float32)
+    m = (rng.standard_normal(shape) * 0.1).astype(np.float32)
+    v = (rng.standard_normal(shape) ** 2 * 0.01).astype(np.float32)
+    f32 = np.float32
+    if kind == "adam":
+        names = ("W", "g", "m", "v", "lr", "beta1", "one_minus_beta1", "beta2", "one_minus_beta2", "eps")
+        feeds = [W, grad, m, v, f32(0.01), f32(0.9), f32(1) - f32(0.9), f32(0.999), f32(1) - f32(0.999), f32(1e-8)]
+        outs = ("W_new", "m_new", "v_new")
+    else:
+        names = ("W", "g", "v", "lr", "rho", "one_minus_rho", "eps")
+        feeds = [W, grad, v, f32(0.01), f32(0.9), f32(1) - f32(0.9), f32(1e-8)]
+        outs = ("W_new", "v_new")
+    return g, [ids[k] for k in names], [ids[k] for k in outs], feeds
+
+
+@pytest.mark.parametrize("kind", ["rmsprop", "adam"])
+@pytest.mark.parametrize("shape", [[5 * 4096 + 3], [300, 1000]])
+def test_rmsprop_and_adam_updater_graphs(kind, shape):
+    """Sec. 3.2 names the RMSProp and Adam updaters: each is one fused VM launch, equal to the oracle."""
+    g, inputs, outs, feeds = updater_case(kind, shape)
+    got, f = run_gpu(g.desc, inputs, outs, feeds)
+    assert f.num_launches() == 1, f.describe()
+    ref = interp.run_function(g.desc, inputs, outs, feeds)
+    for gv, rv in zip(got, ref):
+        check(gv, rv, TOL32, kind)
+
+
+def test_adam_in_place_over_several_steps():
+    """The state of the update (W, m, v) stays in device memory: the fetch pointers are the feed pointers
+    (dragon_function_can_alias says that this function allows it), five steps with fresh gradients, against
+    the oracle run five times on its own fp64 state."""
+    import torch
+    from paper_1707_08265_b200 import binding as B
+    n = 7 * 4096 + 11
+    g, inputs, outs, feeds = updater_case("adam", [n])
+    f = B.Graph.from_desc(g.desc).function(inputs, outs)
+    assert f.can_alias(0, 0) and f.can_alias(2, 1) and f.can_alias(3, 2)     # W, m, v
+    assert not f.can_alias(3, 1)                                             # v is still read after m' has been written
+    dev = [torch.from_numpy(np.ascontiguousarray(a)).cuda() for a in feeds]
+    state64 = [feeds[0].astype(np.float64), feeds[2].astype(np.float64), feeds[3].astype(np.float64)]
+    rng = np.random.default_rng(5)
+    for step in range(5):
+        grad = (rng.standard_normal(n) * 0.1).astype(np.float32)
+        dev[1].copy_(torch.from_numpy(grad))
+        f.run_torch(dev, [dev[0], dev[2], dev[3]])
+        assert f.status() == 0
+        ref = interp.run_function(g.desc, inputs, outs, [state64[0], grad, state64[1], state64[2]] + feeds[4:])
+        state64 = [ref[0], ref[1], ref[2]]
+    torch.cuda.synchronize()
+    for t, r, name in zip((dev[0], dev[2], dev[3]), state64, ("W", "m", "v")):
+        check(t.cpu().numpy().astype(np.float64), r, 5 * TOL32, "after five steps: " + name)
 
 
 @pytest.mark.parametrize("kind", ["sgd", "momentum"])

@@ -12,7 +12,7 @@ J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
-     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "end"]
+     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "end"]
 
 
 def _bf16(a):
@@ -126,6 +126,8 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
         elif name == "ldswah": acc = load(arg & 63)
         elif name in ("ldsw", "ldswa"): acc = load(arg & 63); S[arg >> 6] = acc.copy()
         elif name == "accums": S[arg] = S[arg] + acc
+        elif name == "sqrt": acc = np.sqrt(acc)
+        elif name == "rcp": acc = 1 / acc
         elif name.startswith("sacc"): A[int(name[4])] += float(acc.sum())
         elif name.startswith("ascal"): scalout[arg] = A[int(name[5])]
         elif name == "end": break
