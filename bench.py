@@ -243,12 +243,18 @@ def build_config(cfg, B, torch, seeds, rows=16384):
     return dict(g=g, inputs=inputs, outputs=outputs, units=rows * 4096, unit=UNIT, bound="hbm", alg=16.0 * rows * 4096 * 4, what=what)
 
 
-def time_config(cfg, args, B, torch, seeds, peaks, steps=None):
-    """Device-resident timing of one workload (a step = one dragon_run) plus the per-kernel times of its plan."""
+def time_config(cfg, args, B, torch, seeds, peaks, steps=None, world=1, rank=0, dist=None):
+    """Device-resident timing of one workload (a step = one dragon_run) plus the per-kernel times of its plan.
+    world > 1: every rank runs the workload at its full per-GPU size on data of its own (weak scaling) as one
+    shard of a world-times larger problem; the outputs that are reductions over the sharded axis (sharding.py)
+    are all-reduced with NCCL inside every step."""
+    from paper_1707_08265_b200 import sharding
     c = build_config(cfg, B, torch, seeds, args.rows)
     g, inputs, outputs = c["g"], c["inputs"], c["outputs"]
+    extent = g.shape(inputs[0])[0]
+    kinds = sharding.classify_outputs(g.desc, outputs, extent)
     tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "i32": torch.int32}
-    gen = torch.Generator("cuda").manual_seed(wl.BASE_SEED + cfg)
+    gen = torch.Generator("cuda").manual_seed(wl.BASE_SEED + cfg + 1000 * rank)
 
     def dev_random(t):
         ti = g.desc["tensors"][t]
@@ -267,17 +273,35 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None):
     outs = [torch.empty(tuple(g.shape(t)), dtype=tdt[g.desc["tensors"][t]["dtype"]], device="cuda") for t in outputs]
     steps = steps or min(args.steps, 50)
     stream = torch.cuda.Stream()
+
+    def evaluate():
+        f.run_torch(feeds, outs, stream)
+        return outs
+
+    def one_step():
+        if world == 1:
+            evaluate()
+        else:
+            sharding.run_classified(evaluate, kinds, lambda t: dist.all_reduce(t), 1.0 / world)
+
     with torch.cuda.stream(stream):
         for _ in range(max(3, args.warmup)):
-            f.run_torch(feeds, outs, stream)
+            one_step()
         stream.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
         for _ in range(steps):
-            f.run_torch(feeds, outs, stream)
+            one_step()
         e1.record(stream)
         stream.synchronize()
         ms = e0.elapsed_time(e1) / steps
+        if world > 1:
+            t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ms = float(t.item())
         assert f.status() == 0
         # per-kernel times: CUDA events around every step of the plan (the library records them on the launching stream)
         plan = f.describe().strip().split("\n")
@@ -304,7 +328,8 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None):
     io_bytes = sum(t.numel() * t.element_size() for t in feeds if t is not None) + sum(t.numel() * t.element_size() for t in outs)
     fwd, gops, _ = f.kept_ops()
     top = int(np.argmax(kern))
-    line = {"workload": c["what"], "ms_per_step": ms, "value": c["units"] / (ms * 1e-3), "unit": c["unit"], "steps": steps,
+    line = {"workload": c["what"], "ms_per_step": ms, "value": world * c["units"] / (ms * 1e-3), "unit": c["unit"], "steps": steps,
+            "n_gpus": world, "scaling": "weak", "exchanged_outputs": [k for k in kinds if k in (sharding.SUM, sharding.MEAN)],
             "launches_per_step": f.num_launches(), "kept_forward_ops": len(fwd), "kept_gradient_ops": len(gops), "ops_in_graph": f.n_ops,
             "fed_and_fetched_bytes": io_bytes, "plan": plan[:16], "kernel_ms": [round(k, 5) for k in kern[:16]]}
     if c["bound"] == "hbm":
@@ -358,10 +383,16 @@ def main():
     peaks = measured_peaks()
 
     if args.config != 2:
-        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
-        line = time_config(args.config, args, B, torch, seeds, peaks)
+        world, rank, local = int(os.environ.get("WORLD_SIZE", "1")), int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0"))
+        torch.cuda.set_device(local)
+        if world > 1:
+            dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+        line = time_config(args.config, args, B, torch, seeds, peaks, world=world, rank=rank, dist=dist)
         line["config"] = args.config
-        print(json.dumps(line), flush=True)
+        if rank == 0:
+            print(json.dumps(line), flush=True)
+        if world > 1:
+            dist.destroy_process_group()
         return
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
