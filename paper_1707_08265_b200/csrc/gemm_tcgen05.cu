@@ -17,6 +17,7 @@
 
 #include <algorithm>
 #include <cstdint>
+#include <cstdlib>
 #include <mutex>
 
 #include "plan.h"
@@ -56,13 +57,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // bounded wait: false when the clock budget ran out (the caller records the failure and unwinds)
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, long long budget = kWaitBudgetCycles) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (;;) {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    if (clock64() - t0 > kWaitBudgetCycles) return false;
+    if (clock64() - t0 > budget) return false;
   }
 }
 
@@ -134,6 +135,11 @@ struct GemmArgs {
   int relu;
   // then multiplied by step(mask[row, col]) (1 where the bf16 mask element is > 0, else 0); null: none
   const unsigned short* mask;
+  // clock budget of the pipeline waits (the waits that let in-flight work finish during an unwind keep the
+  // full budget), and the failure-detection test's hook: the producer leaves out the loads of its first
+  // stage, so that the consumer's first wait is for a signal that nothing sends
+  long long wait_budget;
+  int drop_first_load;
 };
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
@@ -161,7 +167,8 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   uint64_t* bars = reinterpret_cast<uint64_t*>(tiles_ptr + (size_t)kStages * kStageBytes);
   const uint32_t bar_full = smem_u32(bars), bar_empty = bar_full + 8 * kStages;
   const uint32_t bar_acc_full = bar_empty + 8 * kStages, bar_acc_empty = bar_acc_full + 8 * kAccBufs;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccBufs);
+  const uint32_t bar_drain = bar_acc_empty + 8 * kAccBufs;     // used by an unwind only: "every MMA issued so far is done"
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * kStages + 2 * kAccBufs + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -171,6 +178,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   if (threadIdx.x == 0) {
     for (int s = 0; s < kStages; ++s) { mbar_init(bar_full + 8 * s, 1); mbar_init(bar_empty + 8 * s, 1); }
     for (int b = 0; b < kAccBufs; ++b) { mbar_init(bar_acc_full + 8 * b, 1); mbar_init(bar_acc_empty + 8 * b, 4); }
+    mbar_init(bar_drain, 1);
     abort_flag[0] = 0;
     abort_flag[1] = 0;   // a flag nobody sets, for waits that must not be cut short
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -184,16 +192,18 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *tmem_slot;
 
+  int issued = 0;          // thread 0 (the producer): stages handed to the TMA engine so far
+  int first_issued = 0;    // ... of which the first few may have been left out by the test hook
   if (warp == 0) {
     if (lane == 0) {  // TMA producer: one running stage counter across all tiles of this CTA
-      int issued = 0;
       bool ok = true;
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
         int tm, tn;
         tile_coords(t, g.tiles_m, g.tiles_n, &tm, &tn);
         for (int kt = 0; kt < k_tiles; ++kt, ++issued) {
           const int s = issued % kStages, it = issued / kStages;
-          if (!mbar_wait(bar_empty + 8 * s, (it & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+          if (!mbar_wait(bar_empty + 8 * s, (it & 1) ^ 1, abort_flag, g.wait_budget)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+          if (g.drop_first_load && issued == 0) { first_issued = 1; continue; }     // failure-detection test: this stage's signal never comes
           mbar_expect_tx(bar_full + 8 * s, kStageBytes);
           const uint32_t dst = tiles + (uint32_t)s * kStageBytes;
           if (!kAMn) {
@@ -210,10 +220,6 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
           }
         }
       }
-      if (*abort_flag) {  // let the copies that are still in flight land before the CTA goes away
-        for (int i = issued > kStages ? issued - kStages : 0; i < issued; ++i)
-          mbar_wait(bar_full + 8 * (i % kStages), (i / kStages) & 1, abort_flag + 1);
-      }
     }
   } else if (warp == 1) {
     if (lane == 0) {  // MMA issuer
@@ -223,12 +229,12 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
       for (int t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++local) {
         const int buf = local % kAccBufs, use = local / kAccBufs;
         // the epilogue must have drained this accumulator (first use passes at once)
-        if (!mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); break; }
+        if (!mbar_wait(bar_acc_empty + 8 * buf, (use & 1) ^ 1, abort_flag, g.wait_budget)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t d_tmem = tmem_base + (uint32_t)(buf * kTileN);
         for (int kt = 0; kt < k_tiles; ++kt, ++consumed) {
           const int s = consumed % kStages, it = consumed / kStages;
-          if (!mbar_wait(bar_full + 8 * s, it & 1, abort_flag)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
+          if (!mbar_wait(bar_full + 8 * s, it & 1, abort_flag, g.wait_budget)) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); ok = false; break; }
           asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
           const uint32_t a_addr = tiles + (uint32_t)s * kStageBytes, b_addr = a_addr + kStageBytesA;
           const uint64_t a_desc = kAMn ? make_smem_desc_mn(a_addr) : make_smem_desc(a_addr);
@@ -243,6 +249,10 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         if (ok) umma_commit(bar_acc_full + 8 * buf);   // accumulator complete
       }
+      if (*abort_flag) {   // unwinding: every MMA issued so far must be done before its operands and the TMEM go away
+        umma_commit(bar_drain);
+        mbar_wait(bar_drain, 0, abort_flag + 1);
+      }
     }
   } else {
     // epilogue: warp w owns TMEM lanes 32*(w%4) .. +31, i.e. rows 32*(w%4) + lane of the tile
@@ -252,7 +262,7 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
       const int buf = local % kAccBufs, use = local / kAccBufs;
       int tm, tn;
       tile_coords(t, g.tiles_m, g.tiles_n, &tm, &tn);
-      const bool ok = mbar_wait(bar_acc_full + 8 * buf, use & 1, abort_flag);
+      const bool ok = mbar_wait(bar_acc_full + 8 * buf, use & 1, abort_flag, g.wait_budget);
       if (!ok) { if (lane == 0) { *abort_flag = 1; atomicExch(g.status, DRAGON_ERR_TIMEOUT); } break; }
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int row = tm * kTileM + q * 32 + lane;
@@ -362,6 +372,15 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  if (*abort_flag) {
+    // an unwind: every role has stopped (barrier above).  The copies that the producer has handed to the TMA
+    // engine and that nobody consumed must land before the CTA's shared memory goes away; this wait keeps the
+    // full budget whatever the pipeline's budget is.
+    if (threadIdx.x == 0)
+      for (int i = std::max(first_issued, issued > kStages ? issued - kStages : 0); i < issued; ++i)
+        mbar_wait(bar_full + 8 * (i % kStages), (i / kStages) & 1, abort_flag + 1);
+    __syncthreads();
+  }
   if (warp == 1) {
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)(kAccBufs * kTileN)) : "memory");
   }
@@ -425,7 +444,12 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
   cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
   if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
   const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
-  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0, reinterpret_cast<const unsigned short*>(mask)};
+  GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0, reinterpret_cast<const unsigned short*>(mask),
+             kWaitBudgetCycles, 0};
+  // failure-detection test only: DRAGON_GEMM_WAIT_BUDGET=<clock cycles> shortens the pipeline waits and
+  // DRAGON_GEMM_DROP_FIRST_LOAD=1 makes the first of them wait for a signal that nothing sends
+  if (const char* e = std::getenv("DRAGON_GEMM_WAIT_BUDGET")) { const long long b = std::atoll(e); if (b > 0) g.wait_budget = std::min(b, kWaitBudgetCycles); }
+  if (const char* e = std::getenv("DRAGON_GEMM_DROP_FIRST_LOAD")) g.drop_first_load = e[0] == '1';
   static int sm_count = 0;
   if (!sm_count) {
     int dev = 0;

@@ -181,3 +181,33 @@ def test_computed_bias_before_or_after_the_product(bias_first):
     (got,), f = run_gpu(gd.desc, [X, W, b], [Y], feeds)
     (ref,) = interp.run_function(gd.desc, [X, W, b], [Y], feeds)
     check(got, ref, 2e-5, "Y")
+
+
+@pytest.mark.parametrize("k", [64, 320])
+def test_a_pipeline_wait_that_runs_out_is_reported_and_the_next_run_is_correct(k, monkeypatch):
+    """Failure detection without a fault: the producer of the contraction leaves out the loads of its first
+    stage (test hook), so the consumer's first wait is for a signal that nothing sends; with the pipeline's
+    budget shortened to about a millisecond the wait runs out, the kernel records DRAGON_ERR_TIMEOUT, lets
+    the copies that are in flight land (that wait keeps its full budget), frees its tensor memory and
+    returns by itself.  The context stays usable: the same function run again without the hook is correct."""
+    from paper_1707_08265_b200 import binding as B
+    m, n = 128, 256                                   # one output tile; k = 320: later stages are really loaded
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16")
+    Y = gd.op("InnerProduct", [X, W], "Y", [m, n], "f32")
+    rng = np.random.default_rng(k)
+    x = bf16able(rng.standard_normal((m, k))); w = bf16able(rng.standard_normal((n, k)) / np.sqrt(k))
+    f = B.Graph.from_desc(gd.desc).function([X, W], [Y])
+    dx, dw = torch.from_numpy(x).to(torch.bfloat16).cuda(), torch.from_numpy(w).to(torch.bfloat16).cuda()
+    out = torch.full((m, n), float("nan"), dtype=torch.float32, device="cuda")
+    monkeypatch.setenv("DRAGON_GEMM_WAIT_BUDGET", "2000000")
+    monkeypatch.setenv("DRAGON_GEMM_DROP_FIRST_LOAD", "1")
+    f.run_torch([dx, dw], [out])
+    assert f.status() == B.ERR_TIMEOUT
+    monkeypatch.delenv("DRAGON_GEMM_WAIT_BUDGET")
+    monkeypatch.delenv("DRAGON_GEMM_DROP_FIRST_LOAD")
+    f.run_torch([dx, dw], [out])
+    assert f.status() == 0
+    torch.cuda.synchronize()
+    (ref,) = interp.run_function(gd.desc, [X, W], [Y], [x, w])
+    check(out.cpu().numpy().astype(np.float64), ref, 2e-5, "Y after the timed-out run")
