@@ -8,7 +8,8 @@ import ctypes
 import os
 
 HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(HERE, "libdragon.so")
+# DRAGON_LIB names another build of the same library (the sanitizer build of build.build_sanitized)
+LIB_PATH = os.environ.get("DRAGON_LIB") or os.path.join(HERE, "libdragon.so")
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_DTYPE, ERR_NOT_SSA, ERR_MISSING_INPUT = -1, -2, -3, -4, -5

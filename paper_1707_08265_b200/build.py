@@ -71,5 +71,41 @@ def _generated_kernel_object(objdir, verbose, force):
     return obj
 
 
+HOST_SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp"]     # the host compiler: no CUDA in these
+SAN_LIB = os.path.join(HERE, "libdragon_san.so")
+
+
+def build_sanitized(verbose=False):
+    """libdragon_san.so: the same library with the host compiler (prunes, lowering, code generation) built
+    with -fsanitize=address,undefined.  Load it with DRAGON_LIB=<path> and the sanitizer runtime preloaded
+    (LD_PRELOAD=$(gcc -print-file-name=libasan.so)); used by tests/test_sanitized_host_compiler.py."""
+    build(verbose=verbose)
+    objdir = os.path.join(HERE, "_build")
+    headers = [os.path.join(CSRC, f) for f in os.listdir(CSRC) if f.endswith(".h")]
+    objs = []
+    for src in SOURCES:
+        if src not in HOST_SOURCES:
+            objs.append(os.path.join(objdir, src + ".o"))
+            continue
+        path, obj = os.path.join(CSRC, src), os.path.join(objdir, src + ".san.o")
+        objs.append(obj)
+        if _stale(obj, [path] + headers):
+            cmd = ["g++", "-std=c++17", "-O1", "-g", "-fPIC", "-fno-omit-frame-pointer", "-fsanitize=address,undefined",
+                   "-fno-sanitize-recover=undefined", "-Wall", "-c", path, "-o", obj]
+            if verbose:
+                print(" ".join(cmd), flush=True)
+            subprocess.run(cmd, check=True)
+    objs.append(os.path.join(objdir, "vm_gen_cubin.o"))
+    if _stale(SAN_LIB, objs):
+        cmd = [NVCC, "-shared", "-o", SAN_LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fsanitize=address", "-Xcompiler", "-fsanitize=undefined"]
+        if verbose:
+            print(" ".join(cmd), flush=True)
+        subprocess.run(cmd, check=True)
+    return SAN_LIB
+
+
 if __name__ == "__main__":
-    build(verbose=True, force="--force" in sys.argv, ptxas_info="--ptxas" in sys.argv)
+    if "--sanitize" in sys.argv:
+        print(build_sanitized(verbose=True))
+    else:
+        build(verbose=True, force="--force" in sys.argv, ptxas_info="--ptxas" in sys.argv)

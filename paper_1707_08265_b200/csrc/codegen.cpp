@@ -697,6 +697,7 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
   const char* force = std::getenv("DRAGON_VM_BUILD");
   const bool only_wide = force && std::string(force) == "wide", only_dense = force && std::string(force) == "dense";
   int rc = DRAGON_ERR_UNSUPPORTED;
+  (void)only_dense;      // the dense build is tried first anyway; a program that does not fit it goes to the wide one
   if (!only_wide) {
     VmSegment trial = *seg;
     Gen gen(items, idx, vals, mems, &trial, kVmRegsDense, kVmSmemSlotsDense);
