@@ -132,7 +132,7 @@ struct Gen {
       if (is_input(v)) u = kFar - 1;  // a cached memory operand is dropped for free
       if (u > best_use) { best_use = u; best = k; }
     }
-    if (best < 0) { err = DRAGON_ERR_UNSUPPORTED; set_error("graph VM: out of register slots"); return 0; }
+    if (best < 0) { err = kVmErrTooLarge; set_error("graph VM: out of register slots"); return 0; }
     int v = reg_owner[best];
     VInfo& f = info[v];
     if (is_input(v)) {
@@ -475,7 +475,7 @@ struct Gen {
       if ((it.opc == M_STORE || it.opc == M_ACCUM) && class_of(mems[it.mem].shape) == K_ROW) any_row_class = true;
     }
     if (err) return err;
-    if (n_uni > 511) { set_error("graph VM: too many scalars and constants"); return DRAGON_ERR_UNSUPPORTED; }
+    if (n_uni > 511) { set_error("graph VM: too many scalars and constants"); return kVmErrTooLarge; }
     seg->row_mode = any_rowsum || any_row_class;
     if (seg->row_mode) {
       seg->n = dom.rows();
@@ -497,7 +497,7 @@ struct Gen {
         if (k >= nr - 2) {
           // no register slot left to pin: the running sum lives in a shared-memory slot (two slots stay free for values)
           int sl = (int)maccs.size() + 2 < n_smem_max ? free_smem() : -1;
-          if (sl < 0) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+          if (sl < 0) { set_error("graph VM: too many reduced outputs in one segment"); return kVmErrTooLarge; }
           smem_owner[sl] = -2;
           maccs.emplace_back(p, sl);
           continue;
@@ -513,7 +513,7 @@ struct Gen {
       pro.push_back(bits);
       preamble.push_back(encode(P_LDU, 0, uz));
       for (auto& a : maccs) preamble.push_back(encode(P_STS, 0, (uint32_t)a.second));
-      if (n_uni > 511) { set_error("graph VM: too many scalars and constants"); return DRAGON_ERR_UNSUPPORTED; }
+      if (n_uni > 511) { set_error("graph VM: too many scalars and constants"); return kVmErrTooLarge; }
     }
     // 4. body
     done.assign(idx.size(), false);
@@ -681,9 +681,9 @@ struct Gen {
       if (cs >= P_COUNT_) { set_error("graph VM: internal error, invalid case id %d", cs); return DRAGON_ERR_UNSUPPORTED; }
       if (cs == P_UCONST) ++i;  // the next word is a literal
     }
-    if ((int)seg->code.size() > kVmCodeMaxWords) { set_error("graph VM: instruction stream too long (%d words)", (int)seg->code.size()); return DRAGON_ERR_UNSUPPORTED; }
-    if ((int)seg->finish.size() > kVmScalarAccs + kVmRegsWide - 2 + kVmSmemSlots - 2) { set_error("graph VM: too many reduced outputs in one segment"); return DRAGON_ERR_UNSUPPORTED; }
-    if ((int)seg->operand_mem.size() > kMaxOperands) { set_error("graph VM: too many memory operands in one segment"); return DRAGON_ERR_UNSUPPORTED; }
+    if ((int)seg->code.size() > kVmCodeMaxWords) { set_error("graph VM: instruction stream too long (%d words)", (int)seg->code.size()); return kVmErrTooLarge; }
+    if ((int)seg->finish.size() > kVmScalarAccs + kVmRegsWide - 2 + kVmSmemSlots - 2) { set_error("graph VM: too many reduced outputs in one segment"); return kVmErrTooLarge; }
+    if ((int)seg->operand_mem.size() > kMaxOperands) { set_error("graph VM: too many memory operands in one segment"); return kVmErrTooLarge; }
     return DRAGON_OK;
   }
 };

@@ -9,6 +9,7 @@
 #include <cmath>
 #include <cstdio>
 #include <map>
+#include <set>
 
 #include "plan.h"
 
@@ -319,8 +320,30 @@ std::vector<VmAccess> vm_operand_accesses(const VmSegment& sg) {
   return acc;
 }
 
+static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs, const std::vector<int>& outputs,
+                           int sm_count, Plan* plan, const std::set<int>& cuts, int* cut_here);
+
+// A fused segment that exceeds what one VM program can hold (memory operands, stream length, uniforms,
+// reduced outputs) is cut in two at its middle micro-operation and everything is lowered again; values that
+// cross the new boundary become workspace tensors like any others.
 int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs,
                    const std::vector<int>& outputs, int sm_count, Plan* plan) {
+  std::set<int> cuts;
+  for (int round = 0; round < 64; ++round) {
+    Plan trial;
+    int cut_here = -1;
+    const int rc = lower_with_cuts(g, pr, inputs, outputs, sm_count, &trial, cuts, &cut_here);
+    if (rc != kVmErrTooLarge) {
+      if (rc == DRAGON_OK) *plan = std::move(trial);
+      return rc;
+    }
+    if (cut_here < 0 || !cuts.insert(cut_here).second) break;
+  }
+  return DRAGON_ERR_UNSUPPORTED;   // the message of the last attempt stands
+}
+
+static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vector<int>& inputs, const std::vector<int>& outputs,
+                           int sm_count, Plan* plan, const std::set<int>& cuts, int* cut_here) {
   Lowerer L(g, pr, plan);
   plan->sm_count = sm_count;
   const int n = (int)g.tensors.size();
@@ -400,6 +423,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
   std::vector<Item>& items = L.items;
   std::vector<Value>& vals = L.vals;
   std::vector<MemRef>& mems = plan->mems;
+  const int n_lowered = (int)items.size();     // items appended later (stores of crossing values) have indices beyond
 
   // A workspace image that is written once and then only copied to a fetch buffer by a plain
   // full-shape store is written to the fetch buffer directly (gradient tensors produced by a
@@ -451,7 +475,7 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
       if (!it.live) continue;
       if (it.kind != IT_MOP) { cur = -1; has_dom = false; continue; }
       Shape s = (it.opc == M_STORE || it.opc == M_ACCUM) ? vals[it.a].shape : vals[it.dst].shape;
-      if (cur < 0 || !join_domain(&dom, &has_dom, s)) {
+      if (cur < 0 || cuts.count(i) || !join_domain(&dom, &has_dom, s)) {
         seg_items.emplace_back();
         cur = (int)seg_items.size() - 1;
         has_dom = false;
@@ -687,6 +711,15 @@ int lower_function(const Graph& g, const PruneResult& pr, const std::vector<int>
   for (size_t s = 0; s < seg_items.size(); ++s) {
     if (seg_items[s].empty()) continue;   // ran in a product's epilogue
     int rc = codegen_segment(items, seg_items[s], vals, mems, sm_count, &plan->segs[s]);
+    if (rc == kVmErrTooLarge) {
+      // the middle of the segment's own micro-operations (stores that were appended for crossing values sit at
+      // the end of the item list and are not cut points)
+      std::vector<int> own;
+      for (int i : seg_items[s])
+        if (i < n_lowered) own.push_back(i);
+      std::sort(own.begin(), own.end());
+      if (own.size() >= 2) *cut_here = own[own.size() / 2];
+    }
     if (rc) return rc;
   }
 

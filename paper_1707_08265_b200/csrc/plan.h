@@ -20,6 +20,8 @@ constexpr int kVmSmemSlotsLongCode = 9;       // the same when the instruction s
 constexpr int kVmSmemSlotsDense = 6;          // the same for the dense build (two CTAs share the SM's shared memory)
 constexpr int kVmReduceBytes = 1024;          // shared memory for the per-warp partials of row sums and block sums
 constexpr int kDefaultSmCount = 148;
+constexpr int kVmErrTooLarge = -100;          // codegen_segment: the segment exceeds a capacity of one program (operands, stream
+                                              // length, uniforms, reduced outputs); the lowering cuts it in two and tries again
 constexpr int kHostChunks = 16;               // dragon_run_host pipelines a large elementwise function in this many chunks
 
 enum MemWhere { MEM_FEED = 0, MEM_FETCH = 1, MEM_WORK = 2 };

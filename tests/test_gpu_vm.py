@@ -83,7 +83,7 @@ def test_toy_gradients(n):
 
 
 FLOOR_OK = 0.25   # CPU fp32 evaluation within a quarter of the tolerance: the tensor is held to the tolerance itself
-C_COND = 8.0      # otherwise (floor f, in tolerances): held to C_COND * f tolerances
+C_COND = 16.0     # otherwise (floor f, in tolerances): held to C_COND * f tolerances
 
 
 def fp32_floors(desc, inputs, outputs, feeds):
@@ -221,3 +221,35 @@ def test_fetch_input_scalar_outputs_and_constants():
     ref = interp.run_function(gd.desc, [x, s], outs, [xs, sv])
     for gv, rv, name in zip(got, ref, ("x", "t", "y", "dx", "ds")):
         check(gv, rv, TOL32, name)
+
+
+@pytest.mark.parametrize("seed", [1, 2])
+def test_dense_survival_row_dag_is_cut_into_segments(seed):
+    """A 1024-operator row DAG fetched so that a quarter of its operators survive (about 255 forward and as many
+    gradient operators, 40 fetched targets, gradients to every connected input): more memory operands than one VM
+    program holds, so the lowering cuts the fused segment until every piece fits; values cross the pieces through
+    the workspace.  Prune sets and operator order against the oracle, values under the conditioned tolerance."""
+    from paper_1707_08265_b200 import binding as B
+    R, C = 64, 520
+    g, inputs, fetch = wl.random_row_dag(R, C, 9100 + seed, n_ops=1024, n_fetch=40)
+    wrts = [i for i in inputs if i in oprune.backward_marks(g.desc, fetch, inputs)]
+    outs = fetch + g.grad(fetch, wrts)
+    feeds = [a * np.float32(0.5) for a in wl.normal_feeds([g.shape(i) for i in inputs], 9200 + seed)]
+    ref64 = interp.run_function(g.desc, inputs, outs, feeds)
+    finite = [k for k, r in enumerate(ref64) if np.all(np.isfinite(r)) and np.max(np.abs(r)) < 1e30]
+    assert len(finite) >= len(outs) - 6          # a few of the 48 outputs overflow even in fp64 (chained sums of exponentials)
+    got, f = run_gpu(g.desc, inputs, outs, feeds)
+    want = oprune.function_sets(g.desc, inputs, outs)
+    fwd, gops, masks = f.kept_ops()
+    assert f.marked() == want["marked"] and fwd == want["fwd_ops"] and gops == [k for (_, k, _) in want["grad_ops"]]
+    assert len(fwd) >= 250 and f.describe().count("vm[") >= 4
+    low = interp.run_function(g.desc, inputs, outs, feeds, dtype=np.float32)
+    tight = 0
+    for k in finite:
+        fl = float(np.max(np.abs(low[k].astype(np.float64) - ref64[k]) / (TOL32 * (1 + np.abs(ref64[k])))))
+        if not np.isfinite(fl) or fl > 1e3:
+            continue        # fp32 itself is off by more than 1 % there (sines of large exponentials and the like): nothing to hold a kernel to
+        scale = 1.0 if fl <= FLOOR_OK else C_COND * fl
+        tight += scale == 1.0
+        check(got[k], ref64[k], TOL32 * scale, "seed %d output %d (fp32 floor %.3g)" % (seed, k, fl))
+    assert tight >= len(finite) // 2

@@ -211,8 +211,8 @@ def test_epilogue_fusion_needs_the_bias_in_memory_before_the_product_runs(bias_f
 def test_many_reduced_outputs_fit_the_finishing_launch_or_are_refused(n_scalars):
     """Gradients with respect to k scalars are k sums over the whole domain.  One segment holds 4 scalar
     accumulators, 5 pinned register slots and, beyond those, pinned shared-memory slots; the finishing
-    launch has a job table sized for all of them, so every count either compiles with exactly k jobs
-    (and computes the right sums, checked on the instruction-set emulator) or is refused at compile time."""
+    launch has a job table sized for all of them.  Up to 20 sums are one program with exactly k jobs (and
+    compute the right sums, checked on the instruction-set emulator); more are cut into several programs."""
     from vm_emulator import run_step
     n = 3 * 4096 + 5
     gd = wl.GraphDesc()
@@ -223,14 +223,14 @@ def test_many_reduced_outputs_fit_the_finishing_launch_or_are_refused(n_scalars)
         t = gd.op("Mul", [s, gd.op("Sin" if k % 2 else "Tanh", [x], "u%d" % k)], "t%d" % k)
         acc = t if acc is None else gd.op("Add", [acc, t], "a%d" % k)
     grads = gd.grad([acc], ss)
-    try:
-        f = B.Graph.from_desc(gd.desc).function([x] + ss, grads)
-    except B.DragonError as e:
-        assert n_scalars > 20 and "reduced outputs" in str(e)
+    f = B.Graph.from_desc(gd.desc).function([x] + ss, grads)
+    steps = [st for st in (f.vm_step(i) for i in range(16)) if st]
+    assert sum(len(st["reduced"]) for st in steps) == n_scalars and all(len(st["reduced"]) <= 20 for st in steps)
+    if n_scalars > 20:      # more than one program holds: the lowering cut the segment in two
+        assert len(steps) >= 2
         return
-    assert n_scalars <= 20
-    step = f.vm_step(0)
-    assert len(step["reduced"]) == n_scalars and f.vm_step(1) is None
+    step = steps[0]
+    assert len(steps) == 1
     rng = np.random.default_rng(n_scalars)
     feeds = [rng.standard_normal(n)] + [rng.standard_normal() for _ in ss]
     _, _, scal = run_step(step, feeds, {})
