@@ -16,7 +16,8 @@ cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int row
                            const float* dl_ptr, float dl_imm, int* status, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cudaStream_t st);
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
-                     cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask);
+                     cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask,
+                     const std::vector<EpiSpec>& epi, const std::vector<MemRef>& mems, void* const* mem_ptr);
 }  // namespace dragon
 
 using namespace dragon;
@@ -434,7 +435,8 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         const MemRef &A = P.mems[s.mA], &C = P.mems[s.mC];
         const int kc = (int)(s.tA ? A.shape.d[0] : A.shape.d[1]);
         int rc = launch_gemm_bf16(ptr[s.mA], ptr[s.mB], ptr[s.mC], C.dtype, (int)C.shape.d[0], (int)C.shape.d[1], kc, s.tA, s.tB, status, st,
-                                  s.mD >= 0 ? ptr[s.mD] : nullptr, s.mD >= 0 ? P.mems[s.mD].dtype : DRAGON_F32, s.relu, s.mE >= 0 ? ptr[s.mE] : nullptr);
+                                  s.mD >= 0 ? ptr[s.mD] : nullptr, s.mD >= 0 ? P.mems[s.mD].dtype : DRAGON_F32, s.relu, s.mE >= 0 ? ptr[s.mE] : nullptr,
+                                  s.epi, P.mems, ptr.data());
         if (rc != DRAGON_OK) { f->status_ready = false; return rc; }
         break;
       }

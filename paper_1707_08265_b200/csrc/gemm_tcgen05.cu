@@ -123,6 +123,12 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* v) {
       : "r"(taddr) : "memory");
 }
 
+struct EpiArg {
+  int opc, operand, dtype;   // EpiOpc, EpiOperand, type of the memory operand
+  float c;                   // EO_CONST
+  const void* ptr;           // EO_SCALAR: one element; EO_ROW: N elements; EO_FULL: [M, N] row-major
+};
+
 struct GemmArgs {
   void* C;
   int c_dtype;
@@ -140,7 +146,66 @@ struct GemmArgs {
   // stage, so that the consumer's first wait is for a signal that nothing sends
   long long wait_budget;
   int drop_first_load;
+  // and then the epilogue program: n_epi operations on every element, in order (plan.h: EpiSpec)
+  int n_epi;
+  EpiArg epi[kMaxEpiOps];
 };
+
+__device__ __forceinline__ float epi_load(const void* p, int dtype, size_t i) {
+  return dtype == DRAGON_F32 ? __ldg(reinterpret_cast<const float*>(p) + i)
+                             : __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p) + i) << 16);
+}
+
+// one operation of the epilogue program on the 32 accumulator values of this thread (row `row`, columns col0..col0+31);
+// the elementary functions are those of the VM's leaves
+__device__ __forceinline__ void epi_apply(const EpiArg& e, uint32_t* v, int row, int col0, int M, int N) {
+  float x[32];
+  if (e.operand == EO_CONST || e.operand == EO_SCALAR) {
+    const float c = e.operand == EO_CONST ? e.c : epi_load(e.ptr, e.dtype, 0);
+#pragma unroll
+    for (int j = 0; j < 32; ++j) x[j] = c;
+  } else if (e.operand == EO_ROW || e.operand == EO_FULL) {
+    const size_t base = (e.operand == EO_FULL ? (size_t)(row < M ? row : 0) * N : 0) + col0;
+    const bool aligned = (N & 7) == 0 && col0 + 32 <= N && (reinterpret_cast<uintptr_t>(e.ptr) & 15) == 0;
+    if (aligned && e.dtype == DRAGON_F32) {
+      const float4* p4 = reinterpret_cast<const float4*>(reinterpret_cast<const float*>(e.ptr) + base);
+#pragma unroll
+      for (int j = 0; j < 8; ++j) { const float4 t = __ldg(p4 + j); x[4 * j] = t.x; x[4 * j + 1] = t.y; x[4 * j + 2] = t.z; x[4 * j + 3] = t.w; }
+    } else if (aligned) {
+      const uint4* p8 = reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned short*>(e.ptr) + base);
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const uint4 t = __ldg(p8 + j);
+        const uint32_t w[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { x[8 * j + 2 * k] = __uint_as_float(w[k] << 16); x[8 * j + 2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u); }
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < 32; ++j) x[j] = col0 + j < N ? epi_load(e.ptr, e.dtype, base + j) : 0.f;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < 32; ++j) {
+    float a = __uint_as_float(v[j]);
+    switch (e.opc) {
+      case E_ADD: a = a + x[j]; break;
+      case E_SUB: a = a - x[j]; break;
+      case E_RSUB: a = x[j] - a; break;
+      case E_MUL: a = a * x[j]; break;
+      case E_RELU: a = fmaxf(a, 0.f); break;
+      case E_TANH: a = vmmath::tanh_f(a); break;
+      case E_SIGMOID: a = vmmath::sigmoid_f(a); break;
+      case E_EXPC: a = vmmath::exp_clamped10(a); break;
+      case E_SIN: a = vmmath::sin_f(a); break;
+      case E_NEG: a = -a; break;
+      case E_SQRT: a = vmmath::sqrt_f(a); break;
+      case E_RCP: a = vmmath::f_rcp(a); break;
+      default: a = vmmath::round_bf16(a); break;    // E_RBF16
+    }
+    v[j] = __float_as_uint(a);
+  }
+}
 
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
@@ -332,6 +397,8 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
               if (col0 + j < g.N) v[j] = __float_as_uint(__uint_as_float(v[j]) * (__uint_as_float((uint32_t)mrow[j] << 16) > 0.f ? 1.f : 0.f));
           }
         }
+        if (col0 < g.N)
+          for (int e = 0; e < g.n_epi; ++e) epi_apply(g.epi[e], v, row, col0, g.M, g.N);
         if (row < g.M && col0 < g.N) {
           if (g.c_dtype == DRAGON_F32) {
             float* out = reinterpret_cast<float*>(g.C) + (size_t)row * g.N + col0;
@@ -422,11 +489,13 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_ro
 
 // C[M,N] = opA * opB^T with K the contraction length.  a_mn / b_mn: the operand is given as the
 // row-major matrix [K, M] (resp. [K, N]) instead of [M, K] (resp. [N, K]).
+// epi: the operations that follow on every element, in order (operands by memory id, pointers in mem_ptr).
 // bias (may be null): row vector of N elements of type bias_dtype (fp32 or bf16), added to every
 // row of the product; relu: max(., 0) applied after it; mask (may be null): bf16 [M, N], the result is
 // multiplied by 1 where the mask element is > 0 and by 0 elsewhere; all before the rounding to C's type.
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
-                     cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask) {
+                     cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask,
+                     const std::vector<EpiSpec>& epi, const std::vector<MemRef>& mems, void* const* mem_ptr) {
   const int a_inner = a_mn ? M : K, b_inner = b_mn ? N : K;
   if (M <= 0 || N <= 0 || K <= 0 || (a_inner & 7) || (b_inner & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
     set_error("InnerProduct: the contiguous extent of every operand must be a multiple of 8 and all pointers 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
@@ -445,7 +514,15 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
   if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
   const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
   GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0, reinterpret_cast<const unsigned short*>(mask),
-             kWaitBudgetCycles, 0};
+             kWaitBudgetCycles, 0, 0, {}};
+  if ((int)epi.size() > kMaxEpiOps) { set_error("InnerProduct: epilogue program too long"); return DRAGON_ERR_UNSUPPORTED; }
+  for (const EpiSpec& e : epi) {
+    EpiArg& a = g.epi[g.n_epi++];
+    a.opc = e.opc; a.operand = e.operand; a.c = e.c;
+    a.dtype = e.mem >= 0 ? mems[e.mem].dtype : DRAGON_F32;
+    a.ptr = e.mem >= 0 ? mem_ptr[e.mem] : nullptr;
+    if (e.operand != EO_NONE && e.operand != EO_CONST && !a.ptr) { set_error("InnerProduct: epilogue operand has no memory"); return DRAGON_ERR_INVALID_ARG; }
+  }
   // failure-detection test only: DRAGON_GEMM_WAIT_BUDGET=<clock cycles> shortens the pipeline waits and
   // DRAGON_GEMM_DROP_FIRST_LOAD=1 makes the first of them wait for a signal that nothing sends
   if (const char* e = std::getenv("DRAGON_GEMM_WAIT_BUDGET")) { const long long b = std::atoll(e); if (b > 0) g.wait_budget = std::min(b, kWaitBudgetCycles); }

@@ -611,6 +611,120 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
     seg_items[s].clear();
   }
 
+  // The general form of the above (a chain of elementwise operators behind an InnerProduct, Sec. 3.3's
+  // operator-at-a-time execution being what is avoided): a segment whose only tensor of the product's shape
+  // that it computes on is the product itself, each operation taking the running value and at most a
+  // constant, a scalar, a row vector or one more tensor of that shape, ending in one store, becomes the
+  // product's epilogue program; the arithmetic is that of the VM's leaves (vm_math.h) in the same order.
+  for (size_t s = 0; s < seg_items.size(); ++s) {
+    std::vector<int> body;
+    for (int i : seg_items[s])
+      if (items[i].live && items[i].opc != M_WIDEN) body.push_back(i);
+    if (body.size() < 2 || (int)body.size() > kMaxEpiOps + 1) continue;
+    auto root = [&](int v) {
+      for (bool again = true; again && v >= 0 && vals[v].kind == VK_OP;) {
+        again = false;
+        for (int i : seg_items[s])
+          if (items[i].opc == M_WIDEN && items[i].dst == v) { v = items[i].a; again = true; break; }
+      }
+      return v;
+    };
+    const Item& st = items[body.back()];
+    if (st.opc != M_STORE) continue;
+    // the product: the first operation's operand that is a rank-2 f32 workspace tensor written by a live contraction
+    const Item& first = items[body[0]];
+    int prod = -1;
+    for (int v : {root(first.a), first.b >= 0 ? root(first.b) : -1})
+      if (v >= 0 && vals[v].kind == VK_MEM && mems[vals[v].mem].where == MEM_WORK && mems[vals[v].mem].dtype == DRAGON_F32 &&
+          mems[vals[v].mem].shape.rank == 2 && prod < 0) {
+        for (const Item& it : items)
+          if (it.live && it.kind == IT_GEMM && it.mC == vals[v].mem) prod = v;
+      }
+    if (prod < 0) continue;
+    const int mP = vals[prod].mem, mOut = st.mem;
+    const Shape sp = mems[mP].shape;
+    if (!(mems[mOut].shape == sp)) continue;
+    int producer = -1, readers = 0;
+    for (int i = 0; i < (int)items.size(); ++i) {
+      const Item& it = items[i];
+      if (!it.live) continue;
+      if (it.kind == IT_GEMM && it.mC == mP) producer = i;
+      if (it.kind != IT_MOP) { readers += (it.mA == mP) + (it.mB == mP) + (it.mD == mP) + (it.mE == mP); continue; }
+      if (it.opc == M_WIDEN) continue;
+      for (int v : {it.a, it.b})
+        if (v >= 0 && root(v) >= 0 && vals[root(v)].kind == VK_MEM && vals[root(v)].mem == mP) ++readers;
+    }
+    if (producer < 0 || producer > runs_at(body[0]) || readers != 1 || items[producer].mD >= 0 || items[producer].mE >= 0 ||
+        !items[producer].epi.empty() || items[producer].relu) continue;
+    std::vector<EpiSpec> prog;
+    int cur = prod;
+    bool ok = true, rounded = false;
+    for (size_t k = 0; k + 1 < body.size() && ok; ++k) {
+      const Item& u = items[body[k]];
+      const int ua = root(u.a), ub = u.b >= 0 ? root(u.b) : -1;
+      EpiSpec e;
+      if (rounded) { ok = false; break; }                      // the rounding to bf16 is the last operation
+      if (u.b < 0) {
+        if (ua != cur) { ok = false; break; }
+        switch (u.opc) {
+          case M_RELU: e.opc = E_RELU; break;
+          case M_TANH: e.opc = E_TANH; break;
+          case M_SIGMOID: e.opc = E_SIGMOID; break;
+          case M_EXPC: e.opc = E_EXPC; break;
+          case M_SIN: e.opc = E_SIN; break;
+          case M_NEG: e.opc = E_NEG; break;
+          case M_SQRT: e.opc = E_SQRT; break;
+          case M_RCP: e.opc = E_RCP; break;
+          case M_RBF16: e.opc = E_RBF16; rounded = true; break;
+          default: ok = false;
+        }
+      } else {
+        if ((ua == cur) == (ub == cur)) { ok = false; break; }  // the running value exactly once
+        const bool value_first = ua == cur;
+        const int o = value_first ? ub : ua;
+        switch (u.opc) {
+          case M_ADD: e.opc = E_ADD; break;
+          case M_MUL: e.opc = E_MUL; break;
+          case M_SUB: e.opc = value_first ? E_SUB : E_RSUB; break;
+          default: ok = false;
+        }
+        if (!ok) break;
+        const Value& ov = vals[o];
+        if (ov.known_const) { e.operand = EO_CONST; e.c = ov.c; }
+        else if (ov.kind != VK_MEM) ok = false;
+        else {
+          const MemRef& om = mems[ov.mem];
+          const bool row_vector = (om.shape.rank == 1 && om.shape.d[0] == sp.d[1]) || (om.shape.rank == 2 && om.shape.d[0] == 1 && om.shape.d[1] == sp.d[1]);
+          if (om.dtype != DRAGON_F32 && om.dtype != DRAGON_BF16) ok = false;
+          else if (om.shape.numel() == 1) e.operand = EO_SCALAR;
+          else if (row_vector) e.operand = EO_ROW;
+          else if (om.shape == sp && ov.mem != mP) e.operand = EO_FULL;
+          else ok = false;
+          e.mem = ov.mem;
+          if (ok && last_writer(ov.mem) > producer) ok = false;   // it must be in memory before the product runs
+        }
+      }
+      if (!ok) break;
+      // nothing else may read an intermediate value of the chain
+      int uses = 0;
+      for (const Item& it : items)
+        if (it.live && it.kind == IT_MOP && it.opc != M_WIDEN)
+          uses += (it.a >= 0 && root(it.a) == u.dst) + (it.b >= 0 && root(it.b) == u.dst);
+      if (uses != 1) { ok = false; break; }
+      prog.push_back(e);
+      cur = u.dst;
+    }
+    if (!ok || root(st.a) != cur || prog.empty()) continue;
+    if (rounded != (mems[mOut].dtype == DRAGON_BF16) || (!rounded && mems[mOut].dtype != DRAGON_F32)) continue;
+    items[producer].mC = mOut;
+    items[producer].epi = prog;
+    for (const EpiSpec& e : prog)
+      if (e.mem >= 0) mems[e.mem].live = true;
+    mems[mP].live = false;
+    for (int i : seg_items[s]) items[i].live = false;
+    seg_items[s].clear();
+  }
+
   // The backward of ReLU behind a product: a segment that multiplies the product by step(h), h a
   // bf16 tensor of the same shape already in memory, stores that (and perhaps sums it as well),
   // leaves the multiplication to the product's epilogue; what remains of the segment reads the
@@ -692,6 +806,7 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
               : it.kind == IT_SCE_BWD ? ST_SCE_BWD : ST_COPY;
     st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.mE = it.mE; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
     st.relu = it.relu;
+    st.epi = it.epi;
     if (it.kind == IT_SCE_FWD) {
       // the gradient with respect to the same logits, scaled by a constant, comes out of the same
       // pass: the step then carries the gradient tensor in mD
@@ -765,6 +880,8 @@ static size_t share_workspace(Plan* plan, size_t off) {
       touch(si, st.mA, false); touch(si, st.mB, false);
       if (st.kind == ST_SCE_BWD || st.kind == ST_GEMM) touch(si, st.mD, false);
       if (st.kind == ST_GEMM) touch(si, st.mE, false);
+      if (st.kind == ST_GEMM)
+        for (const EpiSpec& e : st.epi) touch(si, e.mem, false);
       if (st.kind == ST_SCE_FWD) touch(si, st.mD, true);
       touch(si, st.mC, true);
       continue;
@@ -885,11 +1002,16 @@ std::string describe_plan(const Plan& p) {
         buf[0] = 0;
         break;
       }
-      case ST_GEMM:
-        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s%s%s%s -> %s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
+      case ST_GEMM: {
+        static const char* en[] = {"add", "sub", "rsub", "mul", "relu", "tanh", "sigmoid", "expc", "sin", "neg", "sqrt", "rcp", "rbf16"};
+        static const char* on[] = {"", "c", "s", "row", "full"};
+        std::string ep;
+        for (const EpiSpec& e : st.epi) ep += std::string(ep.empty() ? " epilogue: " : ", ") + en[e.opc] + (e.operand ? std::string(" ") + on[e.operand] : "");
+        snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s%s%s%s -> %s%s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
                  (long long)p.mems[st.mA].shape.d[st.tA ? 0 : 1], st.tA ? " A^T" : "", st.tB ? " B^T" : "", st.mD >= 0 ? " +bias" : "",
-                 st.relu ? " relu" : "", st.mE >= 0 ? " *step" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32");
+                 st.relu ? " relu" : "", st.mE >= 0 ? " *step" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32", ep.c_str());
         break;
+      }
       case ST_TRANSPOSE:
         snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);
         break;

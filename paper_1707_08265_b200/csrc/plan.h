@@ -58,6 +58,17 @@ struct Value {
   bool row_uniform = false;  // the same value in every element of a row: a row sum, a scalar, or an elementwise function of such
 };
 
+// One operation of a product's epilogue program: the running value v of an output element (the fp32
+// accumulator) becomes v op x, x a constant, a scalar tensor, a row vector of N elements or a tensor of the
+// product's shape, or f(v).  Sub and Div keep the operand order of the graph (R = the value is the second operand).
+enum EpiOpc { E_ADD, E_SUB, E_RSUB, E_MUL, E_RELU, E_TANH, E_SIGMOID, E_EXPC, E_SIN, E_NEG, E_SQRT, E_RCP, E_RBF16 };
+enum EpiOperand { EO_NONE, EO_CONST, EO_SCALAR, EO_ROW, EO_FULL };
+struct EpiSpec {
+  int opc = E_ADD, operand = EO_NONE, mem = -1;
+  float c = 0.f;
+};
+constexpr int kMaxEpiOps = 8;
+
 enum ItemKind { IT_MOP, IT_GEMM, IT_TRANSPOSE, IT_SCE_FWD, IT_SCE_BWD, IT_COPY };
 struct Item {
   int kind = IT_MOP;
@@ -70,6 +81,7 @@ struct Item {
   float scale = 1.f;                       // SCE_BWD: immediate dL when mD < 0
   bool tA = false, tB = false;             // GEMM: operand given transposed ([K, M] / [K, N] row-major)
   bool relu = false;                       // GEMM: max(., 0) in the epilogue
+  std::vector<EpiSpec> epi;                // GEMM: further elementwise operations on the accumulator, in order
   bool live = false;
   int segment = -1;
 };
@@ -107,6 +119,7 @@ struct Step {
   float scale = 1.f;
   bool tA = false, tB = false;
   bool relu = false;                     // ST_GEMM: epilogue max(., 0); its bias row vector is mD
+  std::vector<EpiSpec> epi;              // ST_GEMM: the epilogue program that follows bias / max / mask
   size_t scratch_off = 0;                // SCE_FWD: per-row losses
 };
 

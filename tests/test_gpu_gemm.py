@@ -211,3 +211,31 @@ def test_a_pipeline_wait_that_runs_out_is_reported_and_the_next_run_is_correct(k
     torch.cuda.synchronize()
     (ref,) = interp.run_function(gd.desc, [X, W], [Y], [x, w])
     check(out.cpu().numpy().astype(np.float64), ref, 2e-5, "Y after the timed-out run")
+
+
+@pytest.mark.parametrize("m,n,k", [(200, 136, 72), (256, 512, 128), (1, 8, 8), (300, 1000, 264)])
+def test_elementwise_chain_in_the_epilogue_of_a_product(m, n, k):
+    """InnerProduct -> Tanh -> bf16, and InnerProduct -> BiasAdd -> Sigmoid -> Mul(side tensor) -> scalar - (.),
+    each as ONE launch (the chain runs on the accumulator registers before the store), against the oracle at
+    ragged and at aligned sizes; bf16 and fp32 side operands."""
+    rng = np.random.default_rng(m + k)
+    x = bf16able(rng.standard_normal((m, k))); w = bf16able(rng.standard_normal((n, k)) / np.sqrt(k))
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16")
+    T = gd.op("Tanh", [gd.op("InnerProduct", [X, W], "Y", [m, n], "f32")], "T", out_dtype="bf16")
+    (got,), f = run_gpu(gd.desc, [X, W], [T], [x, w])
+    assert f.num_launches() == 1 and "epilogue" in f.describe()
+    (ref,) = interp.run_function(gd.desc, [X, W], [T], [x, w])
+    check(got, ref, TOLBF, "tanh in the epilogue")
+    for side_dtype in ("f32", "bf16"):
+        gd = wl.GraphDesc()
+        X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n], side_dtype)
+        side = gd.tensor("side", [m, n], side_dtype); s = gd.tensor("s", [])
+        A = gd.op("BiasAdd", [gd.op("InnerProduct", [X, W], "Z", [m, n], "f32"), b], "A", [m, n], "f32")
+        P = gd.op("Sub", [s, gd.op("Mul", [gd.op("Sigmoid", [A], "S"), side], "O")], "P")
+        feeds = [x, w, bf16able(rng.standard_normal(n)), bf16able(rng.standard_normal((m, n))), np.asarray(0.75, np.float32)]
+        (got,), f = run_gpu(gd.desc, [X, W, b, side, s], [P], feeds)
+        want = "epilogue: add row, sigmoid, mul %s, rsub s" % ("row" if m == 1 else "full")     # a one-row tensor is a row vector
+        assert f.num_launches() == 1 and want in f.describe(), f.describe()
+        (ref,) = interp.run_function(gd.desc, [X, W, b, side, s], [P], feeds)
+        check(got, ref, 2e-5, "bias, sigmoid, side operand, scalar in the epilogue (%s)" % side_dtype)

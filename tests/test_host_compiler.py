@@ -276,3 +276,34 @@ def test_an_opaque_operator_that_is_pruned_away_does_not_stop_execution():
     with pytest.raises(B.DragonError) as e:
         g.add_op(B.OPS["Opaque"], [x], [w, w])
     assert e.value.code == B.ERR_NOT_SSA
+
+
+def test_elementwise_chains_behind_a_product_run_in_its_epilogue():
+    """Lowering: a chain of elementwise operators whose only tensor of the product's shape is the product itself
+    (plus constants, scalars, row vectors and other tensors already in memory) becomes the contraction's
+    epilogue program: one launch, the fp32 product never reaches memory.  A second reader of the product, or an
+    operand that is computed after the product, keeps the separate elementwise launch."""
+    m, n, k = 200, 136, 72
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16")
+    T = gd.op("Tanh", [gd.op("InnerProduct", [X, W], "Y", [m, n], "f32")], "T", out_dtype="bf16")
+    f = B.Graph.from_desc(gd.desc).function([X, W], [T])
+    assert f.num_launches() == 1 and "epilogue: tanh, rbf16" in f.describe(), f.describe()
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n]); side = gd.tensor("side", [m, n])
+    s = gd.tensor("s", [])
+    A = gd.op("BiasAdd", [gd.op("InnerProduct", [X, W], "Z", [m, n], "f32"), b], "A", [m, n], "f32")
+    O = gd.op("Mul", [gd.op("Sigmoid", [A], "S"), side], "O")
+    P = gd.op("Sub", [s, O], "P")
+    f = B.Graph.from_desc(gd.desc).function([X, W, b, side, s], [P])
+    assert f.num_launches() == 1 and "epilogue: add row, sigmoid, mul full, rsub s" in f.describe(), f.describe()
+    f = B.Graph.from_desc(gd.desc).function([X, W, b, side, s], [P, A])          # A fetched too: two readers of the chain
+    assert "epilogue" not in f.describe() and f.num_launches() == 2, f.describe()
+    # the side operand is itself computed by a later step than the product: no fusion
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); raw = gd.tensor("raw", [m, n])
+    Y = gd.op("InnerProduct", [X, W], "Y", [m, n], "f32")
+    side = gd.op("Sum", [raw], "side")                                             # a row-mode segment of its own, after the product
+    O = gd.op("Mul", [gd.op("Tanh", [Y], "T"), side], "O")
+    f = B.Graph.from_desc(gd.desc).function([X, W, raw], [O])
+    assert "epilogue" not in f.describe(), f.describe()

@@ -72,17 +72,19 @@ def test_workspace_tensors_share_memory_only_when_one_is_dead(hidden):
 
 
 def test_regions_of_dead_tensors_are_used_again():
-    # products followed by Tanh (no epilogue form): every fp32 product dies in the step after it
+    # products read twice by what follows (so that it cannot run in their epilogue): every fp32 product dies in
+    # the step after it
     g = wl.GraphDesc()
     X = g.tensor("X", [128, 256], "bf16"); labels = g.tensor("labels", [128], "i32")
     cur = X
     for k in range(3):
         W = g.tensor("W%d" % k, [256, 256], "bf16")
         z = g.op("InnerProduct", [cur, W], "z%d" % k, [128, 256], "f32")
-        cur = g.op("Tanh", [z], "t%d" % k, out_dtype="bf16")
+        cur = g.op("Add", [g.op("Tanh", [z], "u%d" % k), g.op("Sin", [z], "v%d" % k)], "t%d" % k, out_dtype="bf16")
     loss = g.op("SoftmaxCrossEntropy", [cur, labels], "loss", [], "f32")
     ins = [t for t in range(len(g.desc["tensors"])) if g.desc["tensors"][t]["name"][0] in "XWl" and g.desc["tensors"][t]["name"] != "loss"]
     f = B.Graph.from_desc(g.desc).function(ins, [loss])
+    assert "epilogue" not in f.describe()
     check_sharing(f.workspace_tensors(), expect_reuse=True)
 
 
