@@ -11,13 +11,14 @@ namespace dragon {
 cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st);
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st, int chunks);
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
-                           int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm);
+                           int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm, float* colpart, int n_colpart);
 cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
-                           const float* dl_ptr, float dl_imm, int* status, cudaStream_t st);
+                           const float* dl_ptr, float dl_imm, int* status, cudaStream_t st, float* colpart, int n_colpart);
+cudaError_t launch_colsum_finish(const float* part, int n_part, int cols, void* out, int dtype, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int rows, int cols, cudaStream_t st);
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
                      cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask,
-                     const std::vector<EpiSpec>& epi, const std::vector<MemRef>& mems, void* const* mem_ptr);
+                     const std::vector<EpiSpec>& epi, const std::vector<MemRef>& mems, void* const* mem_ptr, float* colpart);
 }  // namespace dragon
 
 using namespace dragon;
@@ -297,8 +298,8 @@ int dragon_function_num_launches(const dragon_function_t* f) {
   int n = 0;
   for (const Step& st : f->plan.steps) {
     if (st.kind == ST_VM) n += 1 + (f->plan.segs[st.seg].finish.empty() ? 0 : 1);
-    else if (st.kind == ST_SCE_FWD) n += 2;
-    else if (st.kind != ST_COPY) n += 1;
+    else if (st.kind == ST_SCE_FWD) n += 2 + (st.mF >= 0 ? 1 : 0);
+    else if (st.kind != ST_COPY) n += 1 + (st.mF >= 0 ? 1 : 0);
   }
   return n;
 }
@@ -436,7 +437,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
         const int kc = (int)(s.tA ? A.shape.d[0] : A.shape.d[1]);
         int rc = launch_gemm_bf16(ptr[s.mA], ptr[s.mB], ptr[s.mC], C.dtype, (int)C.shape.d[0], (int)C.shape.d[1], kc, s.tA, s.tB, status, st,
                                   s.mD >= 0 ? ptr[s.mD] : nullptr, s.mD >= 0 ? P.mems[s.mD].dtype : DRAGON_F32, s.relu, s.mE >= 0 ? ptr[s.mE] : nullptr,
-                                  s.epi, P.mems, ptr.data());
+                                  s.epi, P.mems, ptr.data(), s.mF >= 0 ? reinterpret_cast<float*>(ws + s.colpart_off) : nullptr);
         if (rc != DRAGON_OK) { f->status_ready = false; return rc; }
         break;
       }
@@ -446,12 +447,14 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
       case ST_SCE_FWD:
         e = launch_sce_fwd(ptr[s.mA], P.mems[s.mA].dtype, reinterpret_cast<const int*>(ptr[s.mB]), (int)P.mems[s.mA].shape.d[0],
                            (int)P.mems[s.mA].shape.d[1], reinterpret_cast<float*>(ws + s.scratch_off), reinterpret_cast<float*>(ptr[s.mC]), status, st,
-                           s.mD >= 0 ? ptr[s.mD] : nullptr, s.mD >= 0 ? P.mems[s.mD].dtype : 0, s.scale);
+                           s.mD >= 0 ? ptr[s.mD] : nullptr, s.mD >= 0 ? P.mems[s.mD].dtype : 0, s.scale,
+                           s.mF >= 0 ? reinterpret_cast<float*>(ws + s.colpart_off) : nullptr, s.n_colpart);
         break;
       case ST_SCE_BWD:
         e = launch_sce_bwd(ptr[s.mA], P.mems[s.mA].dtype, reinterpret_cast<const int*>(ptr[s.mB]), (int)P.mems[s.mA].shape.d[0],
                            (int)P.mems[s.mA].shape.d[1], ptr[s.mC], P.mems[s.mC].dtype,
-                           s.mD >= 0 ? reinterpret_cast<const float*>(ptr[s.mD]) : nullptr, s.scale, status, st);
+                           s.mD >= 0 ? reinterpret_cast<const float*>(ptr[s.mD]) : nullptr, s.scale, status, st,
+                           s.mF >= 0 ? reinterpret_cast<float*>(ws + s.colpart_off) : nullptr, s.n_colpart);
         break;
       case ST_COPY:
         e = cudaMemcpyAsync(ptr[s.mC], ptr[s.mA], P.mems[s.mA].bytes(), cudaMemcpyDeviceToDevice, st);
@@ -461,6 +464,9 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
       if (s.kind != ST_VM) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used + 1]), st);
       ++f->prof_used;
     }
+    if (e == cudaSuccess && s.mF >= 0 && s.kind != ST_VM)     // the partial column sums that the kernel left -> the row vector
+      e = launch_colsum_finish(reinterpret_cast<const float*>(ws + s.colpart_off), s.n_colpart, (int)P.mems[s.mF].shape.d[0], ptr[s.mF],
+                               P.mems[s.mF].dtype, st);
   }
   if (e != cudaSuccess) {
     f->status_ready = false;   // both status words are cleared again before the next run

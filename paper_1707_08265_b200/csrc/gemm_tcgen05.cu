@@ -149,6 +149,9 @@ struct GemmArgs {
   // and then the epilogue program: n_epi operations on every element, in order (plan.h: EpiSpec)
   int n_epi;
   EpiArg epi[kMaxEpiOps];
+  // partial column sums of the values that are written (before their rounding to C's type), one row of N floats
+  // per 32 output rows: colpart[(row / 32)][col]; null: none.  A finishing kernel adds the rows in a fixed order.
+  float* colpart;
 };
 
 __device__ __forceinline__ float epi_load(const void* p, int dtype, size_t i) {
@@ -399,6 +402,24 @@ gemm_bf16_tcgen05(const __grid_constant__ CUtensorMap tmap_a, const __grid_const
         }
         if (col0 < g.N)
           for (int e = 0; e < g.n_epi; ++e) epi_apply(g.epi[e], v, row, col0, g.M, g.N);
+        if (g.colpart != nullptr && col0 < g.N) {
+          // sum over the 32 rows that this warp holds, for each of its 32 columns: a transposing butterfly (at
+          // every step a lane keeps one half of its values and receives the other lanes' share of that half):
+          // 31 shuffles, after which lane c holds the sum of column col0 + c
+          float t[32];
+#pragma unroll
+          for (int j = 0; j < 32; ++j) t[j] = row < g.M ? __uint_as_float(v[j]) : 0.f;
+#pragma unroll
+          for (int sft = 16; sft >= 1; sft >>= 1) {
+            const bool upper = (lane & sft) != 0;
+#pragma unroll
+            for (int j = 0; j < sft; ++j) {
+              const float send = upper ? t[j] : t[j + sft], keep = upper ? t[j + sft] : t[j];
+              t[j] = keep + __shfl_xor_sync(0xffffffffu, send, sft);
+            }
+          }
+          if (col0 + lane < g.N) g.colpart[(size_t)(tm * 4 + q) * g.N + col0 + lane] = t[0];
+        }
         if (row < g.M && col0 < g.N) {
           if (g.c_dtype == DRAGON_F32) {
             float* out = reinterpret_cast<float*>(g.C) + (size_t)row * g.N + col0;
@@ -485,6 +506,23 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_ro
             CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The encoding of a tensor map depends only on the pointer and the extents; a function runs with the same
+// workspace and, usually, the same feed pointers step after step, so the last few encodings are kept.
+bool cached_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_rows) {
+  struct Entry { const void* ptr; int rows, cols, box; CUtensorMap map; };
+  static std::mutex mu;
+  static Entry cache[64];
+  static int used = 0, next = 0;
+  std::lock_guard<std::mutex> lock(mu);
+  for (int i = 0; i < used; ++i)
+    if (cache[i].ptr == ptr && cache[i].rows == rows && cache[i].cols == cols && cache[i].box == box_rows) { *map = cache[i].map; return true; }
+  if (!make_tmap(map, ptr, rows, cols, box_rows)) return false;
+  cache[next] = Entry{ptr, rows, cols, box_rows, *map};
+  next = (next + 1) % 64;
+  used = std::min(used + 1, 64);
+  return true;
+}
+
 }  // namespace
 
 // C[M,N] = opA * opB^T with K the contraction length.  a_mn / b_mn: the operand is given as the
@@ -495,26 +533,42 @@ bool make_tmap(CUtensorMap* map, const void* ptr, int rows, int cols, int box_ro
 // multiplied by 1 where the mask element is > 0 and by 0 elsewhere; all before the rounding to C's type.
 int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, int N, int K, bool a_mn, bool b_mn, int* status,
                      cudaStream_t st, const void* bias, int bias_dtype, bool relu, const void* mask,
-                     const std::vector<EpiSpec>& epi, const std::vector<MemRef>& mems, void* const* mem_ptr) {
+                     const std::vector<EpiSpec>& epi, const std::vector<MemRef>& mems, void* const* mem_ptr, float* colpart) {
   const int a_inner = a_mn ? M : K, b_inner = b_mn ? N : K;
   if (M <= 0 || N <= 0 || K <= 0 || (a_inner & 7) || (b_inner & 7) || ((uintptr_t)A & 15) || ((uintptr_t)B & 15) || ((uintptr_t)C & 15)) {
     set_error("InnerProduct: the contiguous extent of every operand must be a multiple of 8 and all pointers 16-byte aligned (M=%d N=%d K=%d)", M, N, K);
     return DRAGON_ERR_UNSUPPORTED;
   }
   CUtensorMap ta, tb;
-  const bool ok_a = a_mn ? make_tmap(&ta, A, K, M, 64) : make_tmap(&ta, A, M, K, kTileM);
-  const bool ok_b = b_mn ? make_tmap(&tb, B, K, N, 64) : make_tmap(&tb, B, N, K, kTileN);
+  const bool ok_a = a_mn ? cached_tmap(&ta, A, K, M, 64) : cached_tmap(&ta, A, M, K, kTileM);
+  const bool ok_b = b_mn ? cached_tmap(&tb, B, K, N, 64) : cached_tmap(&tb, B, N, K, kTileN);
   if (!ok_a || !ok_b) {
     set_error("InnerProduct: cannot encode the TMA descriptors (no CUDA driver?)");
     return DRAGON_ERR_CUDA;
   }
   auto kern = a_mn ? gemm_bf16_tcgen05<true, true> : (b_mn ? gemm_bf16_tcgen05<false, true> : gemm_bf16_tcgen05<false, false>);
   if (a_mn && !b_mn) { set_error("InnerProduct: this operand layout combination is not built"); return DRAGON_ERR_UNSUPPORTED; }
-  cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
-  if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { set_error("InnerProduct: no current device"); return DRAGON_ERR_CUDA; }
+  // once per device and kernel variant: the shared-memory attribute and the SM count
+  static std::mutex mu;
+  static bool attr_set[64][3] = {};
+  static int sm_counts[64] = {};
+  const int variant = a_mn ? 2 : (b_mn ? 1 : 0);
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!attr_set[dev][variant]) {
+      cudaError_t attr_err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kGemmSmem);
+      if (attr_err != cudaSuccess) { set_error("InnerProduct: %s", cudaGetErrorString(attr_err)); return DRAGON_ERR_CUDA; }
+      attr_set[dev][variant] = true;
+    }
+    if (!sm_counts[dev] && (cudaDeviceGetAttribute(&sm_counts[dev], cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_counts[dev] <= 0))
+      sm_counts[dev] = kDefaultSmCount;
+  }
+  const int sm_count = sm_counts[dev];
   const int tiles_m = (M + kTileM - 1) / kTileM, tiles_n = (N + kTileN - 1) / kTileN;
   GemmArgs g{C, c_dtype, M, N, K, tiles_m, tiles_n, status, bias, bias_dtype, relu ? 1 : 0, reinterpret_cast<const unsigned short*>(mask),
-             kWaitBudgetCycles, 0, 0, {}};
+             kWaitBudgetCycles, 0, 0, {}, colpart};
   if ((int)epi.size() > kMaxEpiOps) { set_error("InnerProduct: epilogue program too long"); return DRAGON_ERR_UNSUPPORTED; }
   for (const EpiSpec& e : epi) {
     EpiArg& a = g.epi[g.n_epi++];
@@ -527,11 +581,6 @@ int launch_gemm_bf16(const void* A, const void* B, void* C, int c_dtype, int M, 
   // DRAGON_GEMM_DROP_FIRST_LOAD=1 makes the first of them wait for a signal that nothing sends
   if (const char* e = std::getenv("DRAGON_GEMM_WAIT_BUDGET")) { const long long b = std::atoll(e); if (b > 0) g.wait_budget = std::min(b, kWaitBudgetCycles); }
   if (const char* e = std::getenv("DRAGON_GEMM_DROP_FIRST_LOAD")) g.drop_first_load = e[0] == '1';
-  static int sm_count = 0;
-  if (!sm_count) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sm_count <= 0) sm_count = kDefaultSmCount;
-  }
   const int grid = std::min(tiles_m * tiles_n, sm_count);   // persistent CTAs, one per SM
   kern<<<grid, kGemmThreads, kGemmSmem, st>>>(ta, tb, g);
   cudaError_t e = cudaGetLastError();

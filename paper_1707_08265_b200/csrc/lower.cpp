@@ -463,6 +463,7 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
       if (it.live)
         for (int m : {it.mA, it.mB, it.mD, it.mE})
           if (m >= 0) mems[m].live = true;
+      // (mF is set by a later pass, from an accumulation that is live itself)
     }
   }
 
@@ -786,6 +787,32 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
     seg_items[s] = rest;
   }
 
+  // A segment that is nothing but the column sums of a tensor that a contraction or the softmax gradient has
+  // just written (a bias gradient) leaves the summing to that kernel: its CTAs write partial column sums of
+  // the values they hold anyway, and the fixed-order finishing kernel adds them.  The tensor is not read again.
+  for (size_t s = 0; s < seg_items.size(); ++s) {
+    std::vector<int> body;
+    for (int i : seg_items[s])
+      if (items[i].live && items[i].opc != M_WIDEN) body.push_back(i);
+    if (body.size() != 1 || items[body[0]].opc != M_ACCUM) continue;
+    const Item& ac = items[body[0]];
+    if (vals[ac.a].kind != VK_MEM) continue;
+    const int m = vals[ac.a].mem, mT = ac.mem;
+    const Shape& sm = mems[m].shape;
+    const Shape& stg = mems[mT].shape;
+    if (sm.rank != 2 || !(stg.rank == 1 && stg.d[0] == sm.d[1]) || (mems[mT].dtype != DRAGON_F32 && mems[mT].dtype != DRAGON_BF16)) continue;
+    int producer = -1;
+    for (int i = 0; i < (int)items.size(); ++i) {
+      const Item& it = items[i];
+      if (it.live && (it.kind == IT_GEMM || it.kind == IT_SCE_BWD) && it.mC == m) producer = i;
+    }
+    if (producer < 0 || producer > runs_at(body[0]) || items[producer].mF >= 0) continue;
+    if (items[producer].kind == IT_SCE_BWD && (sm.d[1] & 7 || sm.d[1] > 4096 || items[producer].mD >= 0)) continue;   // the in-register row kernel only
+    items[producer].mF = mT;
+    for (int i : seg_items[s]) items[i].live = false;
+    seg_items[s].clear();
+  }
+
   // steps in execution order
   std::vector<int> seg_step(seg_items.size(), -1);
   plan->segs.resize(seg_items.size());
@@ -807,6 +834,7 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
     st.mA = it.mA; st.mB = it.mB; st.mC = it.mC; st.mD = it.mD; st.mE = it.mE; st.scale = it.scale; st.tA = it.tA; st.tB = it.tB;
     st.relu = it.relu;
     st.epi = it.epi;
+    st.mF = it.mF;
     if (it.kind == IT_SCE_FWD) {
       // the gradient with respect to the same logits, scaled by a constant, comes out of the same
       // pass: the step then carries the gradient tensor in mD
@@ -816,6 +844,7 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
         if (b.live && b.kind == IT_SCE_BWD && b.mA == it.mA && b.mB == it.mB && b.mD < 0) {
           st.mD = b.mC;
           st.scale = b.scale;
+          st.mF = b.mF;
           fused_away[j] = true;
           break;
         }
@@ -848,8 +877,14 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
     sg.colpart_off = take((size_t)sg.n_colacc * sg.grid * sg.cols * sizeof(float));
     sg.scalpart_off = take((size_t)kHostChunks * sg.n_scalacc * sg.grid * sizeof(double));   // a set per chunk of a chunked host run
   }
-  for (auto& st : plan->steps)
+  for (auto& st : plan->steps) {
     if (st.kind == ST_SCE_FWD) st.scratch_off = take((size_t)mems[st.mA].shape.d[0] * sizeof(float));
+    if (st.mF >= 0) {   // partial column sums: one row per 32 output rows of a contraction, one per CTA of the softmax kernel
+      const Shape& sc = mems[st.kind == ST_SCE_FWD ? st.mD : st.mC].shape;
+      st.n_colpart = st.kind == ST_GEMM ? (int)((sc.d[0] + 127) / 128) * 4 : (int)std::min<int64_t>(sc.d[0], (int64_t)sm_count * 4);
+      st.colpart_off = take((size_t)st.n_colpart * sc.d[1] * sizeof(float));
+    }
+  }
   plan->workspace_bytes = off;
   return DRAGON_OK;
 }
@@ -884,6 +919,7 @@ static size_t share_workspace(Plan* plan, size_t off) {
         for (const EpiSpec& e : st.epi) touch(si, e.mem, false);
       if (st.kind == ST_SCE_FWD) touch(si, st.mD, true);
       touch(si, st.mC, true);
+      touch(si, st.mF, true);
       continue;
     }
     const VmSegment& sg = plan->segs[st.seg];
@@ -1009,14 +1045,15 @@ std::string describe_plan(const Plan& p) {
         for (const EpiSpec& e : st.epi) ep += std::string(ep.empty() ? " epilogue: " : ", ") + en[e.opc] + (e.operand ? std::string(" ") + on[e.operand] : "");
         snprintf(buf, sizeof(buf), "gemm[%lldx%lldx%lld%s%s%s%s%s -> %s%s]\n", (long long)p.mems[st.mC].shape.d[0], (long long)p.mems[st.mC].shape.d[1],
                  (long long)p.mems[st.mA].shape.d[st.tA ? 0 : 1], st.tA ? " A^T" : "", st.tB ? " B^T" : "", st.mD >= 0 ? " +bias" : "",
-                 st.relu ? " relu" : "", st.mE >= 0 ? " *step" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32", ep.c_str());
+                 st.relu ? " relu" : "", st.mE >= 0 ? " *step" : "", p.mems[st.mC].dtype == DRAGON_BF16 ? "bf16" : "f32",
+                 (ep + (st.mF >= 0 ? " +colsum" : "")).c_str());
         break;
       }
       case ST_TRANSPOSE:
         snprintf(buf, sizeof(buf), "transpose[%lldx%lld]\n", (long long)p.mems[st.mA].shape.d[0], (long long)p.mems[st.mA].shape.d[1]);
         break;
-      case ST_SCE_FWD: snprintf(buf, sizeof(buf), st.mD >= 0 ? "softmax_ce_fwd+bwd\n" : "softmax_ce_fwd\n"); break;
-      case ST_SCE_BWD: snprintf(buf, sizeof(buf), "softmax_ce_bwd\n"); break;
+      case ST_SCE_FWD: snprintf(buf, sizeof(buf), st.mD >= 0 ? "softmax_ce_fwd+bwd%s\n" : "softmax_ce_fwd%s\n", st.mF >= 0 ? " +colsum" : ""); break;
+      case ST_SCE_BWD: snprintf(buf, sizeof(buf), "softmax_ce_bwd%s\n", st.mF >= 0 ? " +colsum" : ""); break;
       default: snprintf(buf, sizeof(buf), "copy\n");
     }
     s += buf;

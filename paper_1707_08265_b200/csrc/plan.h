@@ -78,6 +78,7 @@ struct Item {
   // vector, act the identity or max(., 0), E an optional bf16 tensor of C's shape; TRANSPOSE: C = A^T;
   // SCE: A = logits, B = labels, C = out, D = scalar dL (gradient)
   int mA = -1, mB = -1, mC = -1, mD = -1, mE = -1;
+  int mF = -1;                             // GEMM, SCE_BWD: row vector that receives the column sums of the tensor written to mC
   float scale = 1.f;                       // SCE_BWD: immediate dL when mD < 0
   bool tA = false, tB = false;             // GEMM: operand given transposed ([K, M] / [K, N] row-major)
   bool relu = false;                       // GEMM: max(., 0) in the epilogue
@@ -120,6 +121,9 @@ struct Step {
   bool tA = false, tB = false;
   bool relu = false;                     // ST_GEMM: epilogue max(., 0); its bias row vector is mD
   std::vector<EpiSpec> epi;              // ST_GEMM: the epilogue program that follows bias / max / mask
+  int mF = -1;                           // ST_GEMM / ST_SCE_*: row vector receiving the column sums of the written tensor
+  int n_colpart = 0;                     // ... partial rows the kernel writes for it (fixed by the launch shape)
+  size_t colpart_off = 0;                // ... and where: float [n_colpart][cols] in the workspace
   size_t scratch_off = 0;                // SCE_FWD: per-row losses
 };
 

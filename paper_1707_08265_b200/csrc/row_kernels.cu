@@ -132,12 +132,20 @@ __global__ void __launch_bounds__(kRowThreads) sce_kernel(const void* z, int zdt
 // The same for rows that fit the CTA's registers (cols <= kChunks * 2048, a multiple of 8): the row
 // is read from memory once, the exponentials are computed once and kept.  Every thread owns the
 // same elements and adds them in the same order as in sce_kernel, so the results are identical.
+// colpart (may be null): the CTAs then walk the rows with the grid's stride, every thread keeps running sums of
+// the gradient values of its own columns (as computed, before their rounding to dz's type) and writes them to
+// colpart[blockIdx.x][.] at the end: partial column sums for the bias gradient behind the logits.
 template <int kMode, int kChunks>
 __global__ void __launch_bounds__(kRowThreads) sce_row_kernel(const void* z, int zdtype, const int* labels, int rows, int cols,
                                                               float* rowloss, void* dz, int dzdtype, const float* dl_ptr,
-                                                              float dl_imm, int* status) {
+                                                              float dl_imm, int* status, float* colpart) {
   __shared__ float sh[kRowThreads / 32];
-  const int m = blockIdx.x;
+  float cs[kChunks][8];
+#pragma unroll
+  for (int c = 0; c < kChunks; ++c)
+#pragma unroll
+    for (int e = 0; e < 8; ++e) cs[c][e] = 0.f;
+  for (int m = blockIdx.x; m < rows; m += gridDim.x) {
   const size_t off = (size_t)m * cols;
   float v[kChunks][8];
   float mx = -INFINITY;
@@ -179,8 +187,21 @@ __global__ void __launch_bounds__(kRowThreads) sce_row_kernel(const void* z, int
           float g = v[c][e] * inv;
           if (j + e == lab) g -= 1.f;
           v[c][e] = ok ? g * sc : 0.f;
+          cs[c][e] += v[c][e];
         }
         store8(dz, dzdtype, off + j, v[c]);
+      }
+    }
+  }
+  }
+  if (kMode != 0 && colpart != nullptr) {
+#pragma unroll
+    for (int c = 0; c < kChunks; ++c) {
+      const int j = (c * kRowThreads + threadIdx.x) * 8;
+      if (j < cols) {
+        float4* p = reinterpret_cast<float4*>(colpart + (size_t)blockIdx.x * cols + j);
+        p[0] = make_float4(cs[c][0], cs[c][1], cs[c][2], cs[c][3]);
+        p[1] = make_float4(cs[c][4], cs[c][5], cs[c][6], cs[c][7]);
       }
     }
   }
@@ -218,14 +239,16 @@ __global__ void __launch_bounds__(256) transpose16_kernel(const unsigned short* 
 
 }  // namespace
 
+// colpart / n_colpart (dz given, rows that fit the registers only): partial column sums of dz, n_colpart rows of cols floats
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
-                           int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm) {
+                           int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm, float* colpart, int n_colpart) {
   const bool in_regs = (cols & 7) == 0 && cols <= 2 * kRowThreads * 8;
+  if (colpart && !(dz && in_regs && n_colpart > 0 && n_colpart <= rows)) return cudaErrorInvalidValue;
   if (dz) {   // the gradient with respect to the logits in the same pass (dL is a constant)
-    if (in_regs) sce_row_kernel<2, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, dz, dzdtype, nullptr, dl_imm, status);
+    if (in_regs) sce_row_kernel<2, 2><<<colpart ? n_colpart : rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, dz, dzdtype, nullptr, dl_imm, status, colpart);
     else sce_kernel<2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, dz, dzdtype, nullptr, dl_imm, status);
   } else if (in_regs)
-    sce_row_kernel<0, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
+    sce_row_kernel<0, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status, nullptr);
   else
     sce_kernel<0><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, rowloss, nullptr, 0, nullptr, 0.f, status);
   mean_kernel<<<1, kRowThreads, 0, st>>>(rowloss, rows, out);
@@ -233,9 +256,11 @@ cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int row
 }
 
 cudaError_t launch_sce_bwd(const void* z, int zdtype, const int* labels, int rows, int cols, void* dz, int dzdtype,
-                           const float* dl_ptr, float dl_imm, int* status, cudaStream_t st) {
-  if ((cols & 7) == 0 && cols <= 2 * kRowThreads * 8)
-    sce_row_kernel<1, 2><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status);
+                           const float* dl_ptr, float dl_imm, int* status, cudaStream_t st, float* colpart, int n_colpart) {
+  const bool in_regs = (cols & 7) == 0 && cols <= 2 * kRowThreads * 8;
+  if (colpart && !(in_regs && n_colpart > 0 && n_colpart <= rows)) return cudaErrorInvalidValue;
+  if (in_regs)
+    sce_row_kernel<1, 2><<<colpart ? n_colpart : rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status, colpart);
   else
     sce_kernel<1><<<rows, kRowThreads, 0, st>>>(z, zdtype, labels, rows, cols, nullptr, dz, dzdtype, dl_ptr, dl_imm, status);
   return cudaGetLastError();
@@ -303,7 +328,7 @@ extern "C" int dragon_softmax_ce_loss_static(const void* logits, int dtype, cons
   int* status = reinterpret_cast<int*>(scratch + kStaticMaxRows);
   // the status word must start at zero; the per-row losses are overwritten in full by every call
   cudaError_t e = cudaMemsetAsync(status, 0, sizeof(int), st);
-  if (e == cudaSuccess) e = launch_sce_fwd(logits, dtype, labels, rows, cols, scratch, loss_out, status, st, nullptr, 0, 0.f);
+  if (e == cudaSuccess) e = launch_sce_fwd(logits, dtype, labels, rows, cols, scratch, loss_out, status, st, nullptr, 0, 0.f, nullptr, 0);
   if (e != cudaSuccess) {
     set_error("dragon_softmax_ce_loss_static: CUDA error: %s", cudaGetErrorString(e));
     return DRAGON_ERR_CUDA;

@@ -147,4 +147,28 @@ cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, 
   return cudaLaunchKernelEx(&cfg, vm::finish_kernel, fp);
 }
 
+// column sums of n_part partial rows (float [n_part][cols]) -> out[cols], fp64, fixed order
+cudaError_t launch_colsum_finish(const float* part, int n_part, int cols, void* out, int dtype, cudaStream_t st) {
+  vm::FinishParams fp;
+  fp.n_jobs = 1;
+  fp.job[0].kind = 0;
+  fp.job[0].part = part;
+  fp.job[0].out = out;
+  fp.job[0].dtype = dtype;
+  fp.job[0].cols = cols;
+  fp.job[0].grid = n_part;
+  fp.job[0].chunks = 1;
+  fp.job[0].chunk_stride = 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((cols + 31) / 32, 1);
+  cfg.blockDim = dim3(vm::kFinishThreads);
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, vm::finish_kernel, fp);
+}
+
 }  // namespace dragon
