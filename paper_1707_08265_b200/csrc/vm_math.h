@@ -3,7 +3,7 @@
 //
 //   sin/cos : two-constant Cody-Waite reduction by pi/2 (fused multiply-adds) up to 2^20, an exact
 //             multi-word reduction beyond; odd/even polynomials on [-pi/4, pi/4]
-//   exp     : n = rint(x*log2 e), r = x - n*ln2 (two constants), 1 + r + r^2*E(r), n added to the exponent
+//   exp     : 2^(x*log2 e) with the product held in two parts, the power of two by the hardware approximation
 //   tanh    : x*P(x^2)/Q(x^2), argument clamped at 10, result at 1
 //   sigmoid : 1/(1+exp(-x))
 // Polynomial coefficients are weighted least-squares fits on Chebyshev nodes, iteratively
@@ -154,19 +154,29 @@ VM_HD float cos_f(float x) {
   return ((q + 1) & 2) ? -v : v;
 }
 
-// exp for -86 <= x <= 88.7 (callers clamp), where the result is a normal number: e^x = p * 2^n with
-// the 2^n applied by adding n to the exponent field of p, which is exact, as the multiplication is
+// 2^t: the hardware approximation on the device (relative error at most 2^-22 over the whole range, results
+// below 2^-126 flushed to zero), exp2f on the host
+VM_HD float f_ex2(float t) {
+#if defined(__CUDA_ARCH__)
+  float r;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(t));
+  return r;
+#else
+  return exp2f(t);
+#endif
+}
+
+// exp for -86 <= x <= 88.7 (callers clamp), where the result is a normal number: e^x = 2^t with t = x * log2(e)
+// held as t_hi + e: t_hi the rounded product, e its exact residue (one fused multiply-add) plus x times the part
+// of log2(e) that fp32 leaves out; 2^t_hi by f_ex2, times 1 + e * ln 2.  About 2.5e-7 relative on the device.
 VM_HD float exp_core(float x) {
-  const float nb = fmaf(x, 1.44269504088896341f, 12582912.0f);   // round(x*log2 e) in the low mantissa bits
-  const float n = nb - 12582912.0f;
-  float r = fmaf(-n, 0.693145751953125f, x);                   // ln2, high part with a short mantissa
-  r = fmaf(-n, 1.428606765330187e-6f, r);                      // ln2 - high part
-  float e = fmaf(r, 1.3814663108745e-3f, 8.36871131029872e-3f);
-  e = fmaf(r, e, 4.16683865189979e-2f);
-  e = fmaf(r, e, 1.6666520673866728e-1f);
-  e = fmaf(r, e, 4.9999993454926206e-1f);
-  const float p = fmaf(r * r, e, r) + 1.0f;
-  return f_from_bits(f_bits(p) + (f_bits(nb) << 23));
+  const float l_hi = 1.44269502162933349609375f, l_lo = 1.9259629911266175e-8f;
+  const float t = x * l_hi;
+  float e = fmaf(x, l_hi, t * -1.0f);
+  e = fmaf(x, l_lo, e);
+  e = e * 0.693147180559945309f;
+  const float p = f_ex2(t);
+  return fmaf(p, e, p);
 }
 VM_HD float exp_clamped10(float x) { return exp_core(fminf(fmaxf(x, -10.0f), 10.0f)); }
 VM_HD float exp_wide(float x) { return exp_core(fminf(fmaxf(x, -86.0f), 88.7f)); }

@@ -455,25 +455,24 @@ class Kernel:
         return S, C
 
     def exp_core(self, x):
-        """x packed, already clamped so that the result is a normal number: e^x = p * 2^n with the
-        2^n applied by adding n to the exponent field of p (exact, as the multiplication is)"""
-        big = 12582912.0
-        nb = self.fma2(x, self.K(1.44269504088896341), self.K(big))
-        n = self.add2(nb, self.K(-big))
-        r = self.fma2(n, self.K(-0.693145751953125), x)
-        r = self.fma2(n, self.K(-1.428606765330187e-6), r)
-        e = self.fma2(r, self.K(1.3814663108745e-3), self.K(8.36871131029872e-3))
-        e = self.fma2(r, e, self.K(4.16683865189979e-2))
-        e = self.fma2(r, e, self.K(1.6666520673866728e-1))
-        e = self.fma2(r, e, self.K(4.9999993454926206e-1))
-        p = self.add2(self.fma2(self.mul2(r, r), e, r), self.K(1.0))
-        pb, nbb = [self.r(), self.r()], [self.r(), self.r()]
-        self.e("mov.b64 {%s, %s}, %s;" % (pb[0], pb[1], p))
-        self.e("mov.b64 {%s, %s}, %s;" % (nbb[0], nbb[1], nb))
-        for j in range(2):
-            self.e("shl.b32 %s, %s, 23;" % (nbb[j], nbb[j]))
-            self.e("add.u32 %s, %s, %s;" % (pb[j], pb[j], nbb[j]))
-        return self.pack(pb[0], pb[1])
+        """x packed, already clamped so that the result is a normal number: e^x = 2^t with t = x * log2(e) held as
+        t_hi + e: t_hi the rounded product, e its exact residue (one fused multiply-add) plus x times the part of
+        log2(e) that fp32 leaves out; 2^t_hi by the hardware approximation (relative error 2^-22 at most over the
+        whole range), times 1 + e * ln 2"""
+        l_hi, l_lo = 1.44269502162933349609375, 1.9259629911266175e-8
+        kl, kn = self.K(l_hi), self.K(-1.0)
+        t = self.mul2(x, kl)
+        e = self.fma2(x, kl, self.mul2(t, kn))
+        e = self.fma2(x, self.K(l_lo), e)
+        e = self.mul2(e, self.K(0.693147180559945309))
+        lo, hi = self.unpack(t)
+        p = []
+        for s in (lo, hi):
+            d = self.f()
+            self.e("ex2.approx.ftz.f32 %s, %s;" % (d, s))
+            p.append(d)
+        pp = self.pack(p[0], p[1])
+        return self.fma2(pp, e, pp)
 
     def clamp(self, s, lo, hi):
         d = self.f()

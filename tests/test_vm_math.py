@@ -1,6 +1,7 @@
 """Accuracy sweep of the VM's elementary functions (host instantiation of csrc/vm_math.h, reached
-through dragon_host_math) against fp64.  The device build differs only in the reciprocal
-(rcp.approx, about one ulp); the polynomials, reductions and constants are the same code."""
+through dragon_host_math) against fp64.  The device build differs only in the reciprocal and the
+power of two (rcp.approx, about one ulp; ex2.approx, 2^-22 relative: swept on the GPU in
+tests/test_gpu_math_and_updater.py); the polynomials, reductions and constants are the same code."""
 import numpy as np
 
 from paper_1707_08265_b200 import binding as B
