@@ -33,7 +33,7 @@ ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the VM kernel on this workload at the full 2^26
 # elements, from one ncu capture of this kernel binary (profiles/vm_dense_config2.md); None once the kernel has
 # changed since the counters were taken
-NCU_DRAM_BYTES_PER_LAUNCH = None
+NCU_DRAM_BYTES_PER_LAUNCH = 268571648 + 222234880
 SAMPLE_ELEMS = 1 << 21       # the CPU oracle's bounded sample of workload 2, per pass
 
 
@@ -200,7 +200,7 @@ def connected_inputs(B, desc, objs, inputs):
     return keep
 
 
-def build_config(cfg, B, torch, seeds, rows=16384):
+def build_config(cfg, B, torch, seeds, rows=16384, elements=None):
     """-> dict(g, inputs, outputs, units, what, and the roofline's numerator)"""
     MiB = 1 << 20
     if cfg == 1:
@@ -209,7 +209,7 @@ def build_config(cfg, B, torch, seeds, rows=16384):
         return dict(g=g, inputs=[ids["x"], ids["a"], ids["b"]], outputs=[ids["f"], ids["y"]], units=n, unit=UNIT, bound="hbm",
                     alg=12.0 * n, what="config 1: f and y of x*sin(a*x+b), x fp32[2^20], forward (12 B/element; fits the L2)")
     if cfg == 3:
-        n = 1 << 27
+        n = elements or 1 << 27
         g, inputs, outputs = wl.random_dag(n, seeds["random_dag"]["seed"])
         return dict(g=g, inputs=inputs, outputs=outputs, units=n, unit=UNIT, bound="hbm", alg=None,
                     what="config 3: random 64-operator elementwise DAG, 4 x fp32[2^27], 2 fetched sinks, forward")
@@ -249,7 +249,7 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None, world=1, rank=0, 
     shard of a world-times larger problem; the outputs that are reductions over the sharded axis (sharding.py)
     are all-reduced with NCCL inside every step."""
     from paper_1707_08265_b200 import sharding
-    c = build_config(cfg, B, torch, seeds, args.rows)
+    c = build_config(cfg, B, torch, seeds, args.rows, args.elements if args.elements != N_ELEMS else None)
     g, inputs, outputs = c["g"], c["inputs"], c["outputs"]
     extent = g.shape(inputs[0])[0]
     kinds = sharding.classify_outputs(g.desc, outputs, extent)
@@ -365,7 +365,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours")
-    ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU (default: the benchmark's 2^26)")
+    ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU of workload 2 (default: its 2^26) or 3 (default 2^27); smaller for profiler captures")
     ap.add_argument("--rows", type=int, default=16384, help="rows of workload 5 (default: its 16384; smaller for profiler captures)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-other-configs", action="store_true", help="leave the \"configs\" entry (workloads 1, 3, 4, 5) out")

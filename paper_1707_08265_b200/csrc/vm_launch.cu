@@ -50,8 +50,19 @@ __global__ void finish_kernel(const __grid_constant__ FinishParams fp) {
     const int lane = threadIdx.x & 31, slice = threadIdx.x >> 5, c = blockIdx.x * 32 + lane;
     const float* part = reinterpret_cast<const float*>(jb.part);
     double s = 0.0;
-    if (c < jb.cols)
-      for (int g = slice; g < jb.grid; g += kFinishThreads / 32) s += (double)part[(size_t)g * jb.cols + c];
+    if (c < jb.cols) {
+      // four partial rows in flight per warp (independent running sums, added in a fixed order afterwards)
+      constexpr int kStep = kFinishThreads / 32;
+      double s1 = 0.0, s2 = 0.0, s3 = 0.0;
+      int g = slice;
+      for (; g + 3 * kStep < jb.grid; g += 4 * kStep) {
+        const float a0 = part[(size_t)g * jb.cols + c], a1 = part[(size_t)(g + kStep) * jb.cols + c];
+        const float a2 = part[(size_t)(g + 2 * kStep) * jb.cols + c], a3 = part[(size_t)(g + 3 * kStep) * jb.cols + c];
+        s += (double)a0; s1 += (double)a1; s2 += (double)a2; s3 += (double)a3;
+      }
+      for (; g < jb.grid; g += kStep) s += (double)part[(size_t)g * jb.cols + c];
+      s = (s + s1) + (s2 + s3);
+    }
     sh[threadIdx.x] = s;
     __syncthreads();
     if (slice == 0 && c < jb.cols) {
