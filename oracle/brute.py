@@ -91,7 +91,11 @@ def function_sets_bruteforce(desc, inputs, outputs):
     """What function(inputs, outputs) keeps, from the definition alone: a node of the two-stage DAG is
     marked iff it lies on some path that ends in a fetched node (Algorithm 1 as prose: "can affect a
     target").  Every path is walked edge by edge, no reachability sets.  Same result layout as
-    oracle.prune.function_sets."""
+    oracle.prune.function_sets.  A listed input is given (Sec. 3.1: fed by name), so the operator that
+    would have produced it loses it as an output: no edge of the function's graph ends in it."""
+    given = set(inputs)
+    desc = {"tensors": desc["tensors"], "grads": desc.get("grads", []),
+            "ops": [dict(op, out=[y for y in op["out"] if y not in given]) for op in desc["ops"]]}
     tensors, ops, grads = desc["tensors"], desc["ops"], desc.get("grads", [])
     edges = sorted(two_stage_dag(desc))
     alias = {}

@@ -24,6 +24,13 @@ dY for outputs Y in G (plus forward tensors through its anchor, Sec. 3.3) and
 writes dX for inputs X in G.  The targets of a function are its fetched
 outputs; Algorithm 1 runs over the two-stage DAG from them.  The seed d(obj)
 has the objective itself as parent, so an objective of a live stage is marked.
+
+Fed intermediates (Sec. 3.1: any tensor of the workspace can be fed by name;
+Sec. 2.1: the inputs of a function are pushed in).  A tensor listed among the
+inputs of a function is given, not solved: in that function's graph no edge
+leads into it, so the operator that would have produced it is no parent of
+it.  Every set above is then taken on the graph without those edges; a
+gradient whose derivative target has lost all its chains cannot be fetched.
 """
 
 
@@ -49,6 +56,15 @@ def _reach(start, nbrs):
         seen.add(x)
         stack.extend(nbrs[x])
     return seen
+
+
+def without_edges_into(desc, fed):
+    """The graph of a function whose inputs are ``fed``: every operator loses the fed tensors from its
+    outputs (operator ids stay as they are; an operator left without outputs has no edge at all)."""
+    fed = set(fed)
+    ops = [{"type": op["type"], "in": list(op["in"]), "out": [o for o in op["out"] if o not in fed]}
+           for op in desc["ops"]]
+    return {"tensors": desc["tensors"], "ops": ops, "grads": desc.get("grads", [])}
 
 
 def forward_marks(desc, targets):
@@ -79,6 +95,7 @@ def function_sets(desc, inputs, outputs):
                     stage, inverse creation order inside a stage (Sec. 3.2)
       used_inputs : 0/1 per listed input
     """
+    desc = without_edges_into(desc, inputs)
     tensors, ops, grads = desc["tensors"], desc["ops"], desc.get("grads", [])
     n = len(tensors)
     grad_node = {}  # tensor id of a gradient tensor -> (stage, wrt)
@@ -87,8 +104,9 @@ def function_sets(desc, inputs, outputs):
             grad_node[gid] = (s, w)
 
     G = [backward_marks(desc, g["objs"], g["wrts"]) for g in grads]
-    for s, g in enumerate(grads):
-        for w in g["wrts"]:
+    for t in outputs:
+        if t in grad_node:
+            s, w = grad_node[t]
             if w not in G[s]:
                 raise ValueError("no path from tensor %d to any objective of stage %d" % (w, s))
     producer = {}

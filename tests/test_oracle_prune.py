@@ -170,3 +170,57 @@ def test_bruteforce_function_sets_on_the_paper_example():
     assert s["fwd_ops"] == [0, 1, 2, 3] and s["used_inputs"] == [1, 1, 1]
     s = brute.function_sets_bruteforce(g.desc, inputs, [ids["y"]])
     assert s["fwd_ops"] == [0] and s["used_inputs"] == [1, 1, 0] and s["grad_ops"] == []
+
+
+# ---- fed intermediates (Sec. 3.1: any tensor can be fed by name) -----------------------------------
+
+@pytest.mark.parametrize("seed", range(120))
+def test_function_sets_with_fed_intermediates_equal_bruteforce(seed):
+    """The same brute-force comparison when some of the listed inputs are tensors that an operator
+    produces: the walk over explicit edges simply has no edge into a given tensor.  Fetched gradients
+    whose derivative target keeps no chain are rejected by both."""
+    rng = np.random.default_rng(9000 + seed)
+    d, fetch = tiny_dag_with_stages(rng)
+    n_fwd = len(d["tensors"]) - sum(len(st["wrts"]) for st in d["grads"])
+    fed = [int(t) for t in rng.choice(np.arange(3, n_fwd), size=int(rng.integers(1, 3)), replace=False)]
+    inputs = [0, 1, 2] + fed
+    alias = {gid: (s, w) for s, st in enumerate(d["grads"]) for w, gid in zip(st["wrts"], st["grad_ids"])}
+    given = set(inputs)
+    cut = {"tensors": d["tensors"], "grads": d["grads"],
+           "ops": [dict(op, out=[y for y in op["out"] if y not in given]) for op in d["ops"]]}
+    dead = [t for t in fetch if t in alias and
+            not brute.backward_marks_bruteforce(cut, set(d["grads"][alias[t][0]]["objs"]), {alias[t][1]})]
+    if dead:
+        with pytest.raises(ValueError):
+            prune.function_sets(d, inputs, fetch)
+        fetch = [t for t in fetch if t not in dead]
+        if not fetch:
+            return
+    got = prune.function_sets(d, inputs, fetch)
+    want = brute.function_sets_bruteforce(d, inputs, fetch)
+    assert got == want
+    # no operator is kept for the sake of a given tensor alone, and a given tensor has no marked parent through it
+    for k in got["fwd_ops"]:
+        assert any(got["marked"][y] for y in d["ops"][k]["out"] if y not in given)
+
+
+def test_feeding_the_argument_of_the_sine_by_hand():
+    """The function of Sec. 2.2 with t2 = a*x + b given instead of computed (worked out by hand):
+    f = x*sin(t2) needs x and t2 only, so Mul(a, x) and Add(y, b) go and a, b are never read; df/dx keeps
+    the one chain x -> f (the chain through y is cut), so only the gradient operator of the last Mul
+    stays and it produces the x side alone; df/da and df/db have no chain left."""
+    g, ids = wl.toy_function_grad(8)
+    inputs = [ids["x"], ids["a"], ids["b"], ids["t2"]]
+    s = prune.function_sets(g.desc, inputs, [ids["f"], ids["dx"]])
+    assert s["fwd_ops"] == [2, 3] and s["used_inputs"] == [1, 0, 0, 1]
+    assert s["grad_ops"] == [(0, 3, (0,))]
+    assert [s["marked"][ids[k]] for k in ("y", "t2", "t3", "f", "dx", "da", "db")] == [0, 1, 1, 1, 1, 0, 0]
+    assert s == brute.function_sets_bruteforce(g.desc, inputs, [ids["f"], ids["dx"]])
+    for dead in ("da", "db"):
+        with pytest.raises(ValueError):
+            prune.function_sets(g.desc, inputs, [ids[dead]])
+    # given y instead: the chain b -> t2 -> t3 -> f is alive, a's is not
+    inputs = [ids["x"], ids["a"], ids["b"], ids["y"]]
+    s = prune.function_sets(g.desc, inputs, [ids["db"], ids["dx"]])
+    assert s["fwd_ops"] == [1, 2, 3] and s["used_inputs"] == [1, 0, 1, 1]
+    assert s["grad_ops"] == [(0, 3, (0, 1)), (0, 2, (0,)), (0, 1, (1,))]

@@ -68,6 +68,34 @@ def _single_op_graph(type_, shapes):
 KINKS = {"ReLU": [0.0], "Exp": [-10.0, 10.0]}
 
 
+def test_fed_intermediate_closed_forms():
+    """Sec. 3.1 (any tensor can be fed): with t2 given, f = x*sin(t2) whatever a and b are (they are not
+    read), df/dx = sin(t2) alone (the chain through a*x is cut), and the gradient with respect to the
+    given tensor is x*cos(t2).  With y given, df/db = sum x*cos(y+b)."""
+    n = 257
+    g = wl.toy_function(n)[0]
+    ids = {t["name"]: i for i, t in enumerate(g.desc["tensors"])}
+    dx, dt2, db = g.grad([ids["f"]], [ids["x"], ids["t2"], ids["b"]])
+    x, a, b = wl.toy_feeds(n, 11)
+    xd = x.astype(np.float64)
+    t2 = np.random.default_rng(5).uniform(-3, 3, n)
+    inputs = [ids["x"], ids["a"], ids["b"], ids["t2"]]
+    f, gx, gt = interp.run_function(g.desc, inputs, [ids["f"], dx, dt2], [x, None, None, t2])
+    assert np.allclose(f, xd * np.sin(t2), rtol=1e-15, atol=0)
+    assert np.allclose(gx, np.sin(t2), rtol=1e-15, atol=0)
+    assert np.allclose(gt, xd * np.cos(t2), rtol=1e-15, atol=0)
+    with pytest.raises(ValueError):
+        interp.run_function(g.desc, inputs, [db], [x, a, b, t2])
+    yv = np.random.default_rng(6).uniform(-3, 3, n)
+    inputs = [ids["x"], ids["a"], ids["b"], ids["y"]]
+    (gb,) = interp.run_function(g.desc, inputs, [db], [x, None, b, yv])
+    assert math.isclose(float(gb), math.fsum(xd * np.cos(yv + float(b))), rel_tol=1e-12)
+    # feeding what the function itself would have computed changes nothing downstream
+    full = interp.run_function(g.desc, inputs[:3], [ids["y"], ids["f"]], [x, a, b])
+    (f2,) = interp.run_function(g.desc, inputs, [ids["f"]], [x, None, b, full[0]])
+    assert np.array_equal(f2, full[1])
+
+
 @pytest.mark.parametrize("type_,shapes", [
     ("Add", [[3, 4], [4]]), ("Sub", [[3, 4], [4]]), ("Sub", [[4], [3, 4]]), ("Mul", [[3, 4], []]),
     ("Mul", [[3, 4], [3, 4]]), ("Div", [[3, 4], [4]]), ("Div", [[4], [3, 4]]), ("Sin", [[3, 4]]),
