@@ -32,6 +32,7 @@ extern "C" {
 
 typedef struct dragon_graph dragon_graph_t;       /* host-only graph under construction   */
 typedef struct dragon_function dragon_function_t; /* pruned + compiled function           */
+typedef struct dragon_workspace dragon_workspace_t; /* named tensors in device memory (Sec. 3.1) */
 typedef int32_t dragon_id;
 
 enum {
@@ -111,10 +112,14 @@ int dragon_graph_num_ops(const dragon_graph_t* g);
 
 /* ---- compile: prune + instruction streams (Sec. 2.2, 2.3, 3.2) -------------------------- */
 
-/* Builds f = function(inputs, outputs).  inputs must be source tensors (no producer); an input
- * that the targets do not need is legal, is reported as pruned, and its feed pointer is never
- * read (the redundant b of Sec. 2.2).  Works without a GPU.  The graph may be destroyed
- * afterwards.  Returns NULL on error. */
+/* Builds f = function(inputs, outputs).  An input that the targets do not need is legal, is
+ * reported as pruned, and its feed pointer is never read (the redundant b of Sec. 2.2).  An input
+ * may also be a tensor that an operator produces (Sec. 3.1: any tensor can be fed): in this
+ * function it is given, the operator that would have produced it is not its parent, both prunes
+ * run on the graph without the edges into it, and a chain objective -> derivative target counts
+ * only if it avoids those edges; fetching a gradient whose derivative target has no chain left
+ * fails with DRAGON_ERR_NO_PATH.  Gradient tensors cannot be fed.  Works without a GPU.  The
+ * graph is not changed and may be destroyed afterwards.  Returns NULL on error. */
 dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, int n_in,
                                    const dragon_id* outputs, int n_out);
 void dragon_function_destroy(dragon_function_t* f); /* NULL is allowed */
@@ -201,6 +206,46 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
 size_t dragon_function_staging_bytes(const dragon_function_t* f);
 int dragon_run_host(dragon_function_t* f, const void* const* host_feeds, void* const* host_fetches,
                     void* staging_dev, size_t staging_bytes, void* cuda_stream);
+
+/* ---- workspace (Sec. 3.1: the workspace owns every tensor; any of them can be fed or fetched by
+ *      name; Sec. 3.2: the state of an updater lives there between runs) ------------------------ */
+
+/* A workspace owns device memory for named tensors and for the scratch areas of the functions run
+ * against it.  It is used from one host thread and with one stream at a time; destroying it frees
+ * everything it allocated (no run that uses it may still be in flight). */
+dragon_workspace_t* dragon_workspace_create(void);
+void dragon_workspace_destroy(dragon_workspace_t* w); /* NULL is allowed */
+
+/* Feed by name.  The first feed of a name creates the tensor (type, rank 0..2 and shape as given,
+ * contents zero); later feeds must repeat type and shape (DRAGON_ERR_DTYPE / DRAGON_ERR_SHAPE).
+ * src: host or device memory holding the tensor contiguously, or NULL to create without copying;
+ * the copy is asynchronous on cuda_stream (pageable host memory makes it synchronous). */
+int dragon_workspace_feed(dragon_workspace_t* w, const char* name, int dtype, int rank, const int64_t* shape,
+                          const void* src, void* cuda_stream);
+
+/* Fetch by name: copies the tensor's bytes to dst (host or device memory, caller-owned) asynchronously
+ * on cuda_stream.  bytes must equal the tensor's size.  DRAGON_ERR_MISSING_INPUT for an unknown name. */
+int dragon_workspace_fetch(dragon_workspace_t* w, const char* name, void* dst, size_t bytes, void* cuda_stream);
+
+/* Device address of a named tensor as of now (a later run that rebinds the name may change it), with its
+ * type, rank and shape (each may be NULL; shape receives rank extents).  NULL for an unknown name. */
+void* dragon_workspace_tensor(dragon_workspace_t* w, const char* name, int* dtype, int* rank, int64_t* shape);
+
+/* Bytes of device memory the workspace holds. */
+size_t dragon_workspace_bytes(const dragon_workspace_t* w);
+
+/* Runs f against the workspace: every input that the pruned function reads is the workspace tensor with
+ * the input's graph name (DRAGON_ERR_MISSING_INPUT if it was never fed, DRAGON_ERR_DTYPE /
+ * DRAGON_ERR_SHAPE if it does not fit: Sec. 4.3, a mistaken shape is caught before executing); output j
+ * is written to the tensor named output_names[j], or, where output_names or its entry is NULL, to the one
+ * named like the output in the graph; missing tensors are created.  An output may be bound to the name
+ * of an input (W' -> W in the updater of Sec. 3.2): it overwrites the input in place where
+ * dragon_function_can_alias() allows, otherwise it is written to a second buffer that the name points
+ * to once the run is enqueued (the old buffer is kept for the next such run), so a later run or fetch on
+ * the same stream sees the new contents.  If f has no scratch area yet, the workspace allocates one.
+ * Asynchronous on cuda_stream; errors as for dragon_run(). */
+int dragon_workspace_run(dragon_workspace_t* w, dragon_function_t* f, const char* const* output_names,
+                         void* cuda_stream);
 
 /* Device-side timing of one launch step of the plan (step index as listed by
  * dragon_function_describe, one line per step; for a graph-VM step the VM kernel alone is

@@ -35,6 +35,15 @@ _SIGNATURES = {
     "dragon_graph_num_ops": (_c.c_int, [_c.c_void_p]),
     "dragon_function": (_c.c_void_p, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int32), _c.c_int]),
     "dragon_function_destroy": (None, [_c.c_void_p]),
+    "dragon_workspace_create": (_c.c_void_p, []),
+    "dragon_workspace_destroy": (None, [_c.c_void_p]),
+    "dragon_workspace_feed": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_int, _c.c_int, _c.POINTER(_c.c_int64), _c.c_void_p,
+                                         _c.c_void_p]),
+    "dragon_workspace_fetch": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_void_p, _c.c_size_t, _c.c_void_p]),
+    "dragon_workspace_tensor": (_c.c_void_p, [_c.c_void_p, _c.c_char_p, _c.POINTER(_c.c_int), _c.POINTER(_c.c_int),
+                                              _c.POINTER(_c.c_int64)]),
+    "dragon_workspace_bytes": (_c.c_size_t, [_c.c_void_p]),
+    "dragon_workspace_run": (_c.c_int, [_c.c_void_p, _c.c_void_p, _c.POINTER(_c.c_char_p), _c.c_void_p]),
     "dragon_function_marked": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_uint8), _c.c_int]),
     "dragon_function_kept_ops": (_c.c_int, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int),
                                             _c.POINTER(_c.c_int32), _c.POINTER(_c.c_uint32), _c.c_int, _c.POINTER(_c.c_int)]),
@@ -306,6 +315,56 @@ class Function:
         self.ensure_workspace()
         s = stream if stream is not None else torch.cuda.current_stream()
         self.run([0 if t is None else t.data_ptr() for t in feeds], [t.data_ptr() for t in fetches], s.cuda_stream)
+
+
+class Workspace:
+    """dragon_workspace_t: named tensors that stay in device memory between runs (feed, fetch, run by name)."""
+
+    def __init__(self):
+        self.h = lib().dragon_workspace_create()
+        if not self.h:
+            raise DragonError(-1, "dragon_workspace_create")
+
+    def close(self):
+        if self.h:
+            lib().dragon_workspace_destroy(self.h)
+            self.h = None
+
+    __del__ = close
+
+    def feed(self, name, dtype, shape, src_ptr, stream=0):
+        """src_ptr: address of host or device memory holding the tensor (0 creates it zero-filled)."""
+        arr = (_c.c_int64 * max(1, len(shape)))(*shape)
+        r = lib().dragon_workspace_feed(self.h, name.encode(), dtype, len(shape), arr, src_ptr or None, stream)
+        if r < 0:
+            raise DragonError(r, "dragon_workspace_feed")
+
+    def fetch(self, name, dst_ptr, nbytes, stream=0):
+        r = lib().dragon_workspace_fetch(self.h, name.encode(), dst_ptr, nbytes, stream)
+        if r < 0:
+            raise DragonError(r, "dragon_workspace_fetch")
+
+    def tensor(self, name):
+        """(device address, dtype, shape) of a named tensor."""
+        dt, rk = _c.c_int(), _c.c_int()
+        shp = (_c.c_int64 * 2)()
+        p = lib().dragon_workspace_tensor(self.h, name.encode(), _c.byref(dt), _c.byref(rk), shp)
+        if not p:
+            raise DragonError(-1, "dragon_workspace_tensor")
+        return p, dt.value, list(shp[:rk.value])
+
+    def nbytes(self):
+        return lib().dragon_workspace_bytes(self.h)
+
+    def run(self, function, output_names=None, stream=0):
+        """output_names: None, or one name (or None) per output of the function."""
+        names = None
+        if output_names is not None:
+            assert len(output_names) == function.n_out
+            names = (_c.c_char_p * function.n_out)(*[None if n is None else n.encode() for n in output_names])
+        r = lib().dragon_workspace_run(self.h, function.h, names, stream)
+        if r < 0:
+            raise DragonError(r, "dragon_workspace_run")
 
 
 def softmax_ce_loss_static(logits_ptr, dtype, labels_ptr, rows, cols, loss_ptr, stream=0):

@@ -1,6 +1,7 @@
 // C ABI of libdragon.so: graph capture, compile (prune + lower), run.
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstring>
 #include <new>
 
@@ -184,7 +185,7 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
   std::vector<uint8_t> seen(g->g.tensors.size(), 0);
   for (int t : in) {
     if (!valid_tensor(g, t)) { set_error("dragon_function: input id %d is not a tensor", t); return nullptr; }
-    if (g->g.tensors[t].producer >= 0 || g->g.tensors[t].grad_stage >= 0) { set_error("dragon_function: input '%s' is not a source tensor", g->g.tensors[t].name.c_str()); return nullptr; }
+    if (g->g.tensors[t].grad_stage >= 0) { set_error("dragon_function: input '%s' is a gradient tensor and cannot be fed", g->g.tensors[t].name.c_str()); return nullptr; }
     if (seen[t]) { set_error("dragon_function: input '%s' is listed twice", g->g.tensors[t].name.c_str()); return nullptr; }
     seen[t] = 1;
   }
@@ -195,16 +196,36 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
   f->n_tensors = (int)g->g.tensors.size();
   f->n_in = n_in;
   f->n_out = n_out;
-  if (prune_function(g->g, in, out, &f->prune) != DRAGON_OK) { delete f; return nullptr; }
-  f->rename = inplace_rename(g->g, f->prune);
+  for (int t : in) f->in_info.push_back(g->g.tensors[t]);
+  for (int t : out) f->out_info.push_back(g->g.tensors[t]);
+  // A listed input that an operator produces is given, not solved (Sec. 3.1: any tensor can be fed): in
+  // this function's graph it is a source, and the operator that would have produced it loses it as an
+  // output.  The cut is made on a copy; the caller's graph stays as it is.
+  const dragon::Graph* fg = &g->g;
+  dragon::Graph cut;
+  bool feeds_intermediate = false;
+  for (int t : in) feeds_intermediate |= g->g.tensors[t].producer >= 0;
+  if (feeds_intermediate) {
+    cut = g->g;
+    for (int t : in) {
+      const int p = cut.tensors[t].producer;
+      if (p < 0) continue;
+      auto& o = cut.ops[p].out;
+      o.erase(std::remove(o.begin(), o.end(), t), o.end());
+      cut.tensors[t].producer = -1;
+    }
+    fg = &cut;
+  }
+  if (prune_function(*fg, in, out, &f->prune) != DRAGON_OK) { delete f; return nullptr; }
+  f->rename = inplace_rename(*fg, f->prune);
   // a kept operator that is only an edge set (Sec. 2.2) can be pruned around but not executed: the
   // function keeps its prune results and refuses to run
   for (int k : f->prune.fwd_ops)
-    if (g->g.ops[k].type == DRAGON_OP_OPAQUE) {
+    if (fg->ops[k].type == DRAGON_OP_OPAQUE) {
       f->not_executable = "the function keeps an opaque operator (operator " + std::to_string(k) + "): it can be pruned but not executed";
       return f;
     }
-  if (lower_function(g->g, f->prune, in, out, query_sm_count(), &f->plan) != DRAGON_OK) { delete f; return nullptr; }
+  if (lower_function(*fg, f->prune, in, out, query_sm_count(), &f->plan) != DRAGON_OK) { delete f; return nullptr; }
   return f;
 }
 

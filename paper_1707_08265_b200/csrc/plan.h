@@ -157,6 +157,7 @@ struct dragon_function {
   std::vector<int> rename;   // Algorithm 3 on the pruned graph (per tensor id)
   std::string not_executable;   // non-empty: why dragon_run refuses this function (it still answers every prune query)
   int n_tensors = 0, n_in = 0, n_out = 0;
+  std::vector<dragon::TensorInfo> in_info, out_info;   // name, type and shape of every listed input and output
   void* workspace = nullptr;
   size_t workspace_bytes = 0;
   void* last_stream = nullptr;

@@ -104,6 +104,14 @@ int prune_function(const Graph& g, const std::vector<int>& inputs, const std::ve
       gop[s][k] = o_in && i_in;
     }
   }
+  // a fetched gradient needs a chain; feeding an intermediate tensor can have cut the last one
+  for (int t : outputs) {
+    const TensorInfo& ti = g.tensors[t];
+    if (ti.grad_stage >= 0 && !out->in_G[ti.grad_stage][ti.grad_wrt]) {
+      set_error("no chain is left from '%s' to any objective of its gradient stage in this function", g.tensors[ti.grad_wrt].name.c_str());
+      return DRAGON_ERR_NO_PATH;
+    }
+  }
   std::vector<std::vector<int>> consumers(n);
   for (int k = 0; k < n_ops; ++k)
     for (int i : g.ops[k].in)

@@ -72,6 +72,32 @@ def test_mlp_forward_backward(shape):
         assert np.max(np.abs(gv - rv)) <= 0.03 * scale + 1e-12, (name, np.max(np.abs(gv - rv)), scale)
 
 
+def test_mlp_with_the_hidden_activations_given():
+    """Sec. 3.1: feeding h (the output of the first layer) makes it a source of the function: the first
+    contraction, its bias and ReLU go, X, W1 and b1 are never read, the second layer's loss and gradients
+    are computed from the given h, and the gradient with respect to h itself can be fetched."""
+    batch, d_in, d_hid, d_out = 256, 192, 320, 136
+    g, ids = wl.mlp(batch, d_in, d_hid, d_out)
+    (dh,) = g.grad([ids["loss"]], [ids["h"]])
+    feeds = list(wl.mlp_feeds(batch, d_in, d_hid, d_out, 77))
+    hv = bf16able(np.abs(np.random.default_rng(8).standard_normal((batch, d_hid))))
+    inputs = [ids[k] for k in ("X", "W1", "b1", "W2", "b2", "labels", "h")]
+    outs = [ids["loss"], ids["dW2"], ids["db2"], dh]
+    fd = [None, None, None, feeds[3], feeds[4], feeds[5], hv]
+    got, f = run_gpu(g.desc, inputs, outs, fd)
+    assert f.used_inputs() == [0, 0, 0, 1, 1, 1, 1] and f.kept_ops()[0] == [4, 5, 6]
+    assert f.describe().count("gemm") == 3, f.describe()                       # z2, dW2, dh
+    ref = interp.run_function(g.desc, inputs, outs, fd)
+    for gv, rv, name in zip(got, ref, ("loss", "dW2", "db2", "dh")):
+        check(gv, rv, TOLBF, name)
+        assert np.max(np.abs(gv - rv)) <= 0.03 * np.max(np.abs(rv)) + 1e-12, name
+    # the first layer's gradients have lost their chain in this function
+    from paper_1707_08265_b200 import binding as B
+    with pytest.raises(B.DragonError) as e:
+        B.Graph.from_desc(g.desc).function(inputs, [ids["dW1"]])
+    assert "no chain is left" in str(e.value)
+
+
 def test_mlp_out_of_range_label_sets_status_and_does_not_fault():
     g, ids, inputs, outs, feeds = mlp_case(128, 128, 128, 128, seed=3)
     feeds[5] = feeds[5].copy(); feeds[5][7] = 4096

@@ -185,6 +185,33 @@ def test_random_row_dags_with_gradients(seed):
     check_conditioned(got, ref, floors, "seed %d" % seed)
 
 
+@pytest.mark.parametrize("seed", range(8))
+def test_random_row_dags_with_fed_intermediates(seed):
+    """Sec. 3.1: any tensor can be fed.  Up to three tensors that operators produce (a full tensor, a broadcast
+    row sum, whatever the draw gives) are listed among the inputs and fed with fresh values; forward values and
+    the gradients with respect to the sources that keep a chain and to the given tensors themselves against the
+    oracle, prune sets included."""
+    R, C = 37, 520
+    g, inputs, fetch = wl.random_row_dag(R, C, 3000 + seed, n_ops=48, n_fetch=2)
+    kept = oprune.function_sets(g.desc, inputs, fetch)["fwd_ops"]
+    rng = np.random.default_rng(seed)
+    fed = sorted({g.desc["ops"][int(k)]["out"][0] for k in rng.choice(kept, size=min(3, len(kept)), replace=False)} - set(fetch))
+    all_in = inputs + fed
+    G = oprune.backward_marks(oprune.without_edges_into(g.desc, all_in), fetch, all_in)
+    wrts = [i for i in all_in if i in G]
+    grads = g.grad(fetch, wrts) if wrts else []
+    feeds = [a * np.float32(0.5) for a in wl.normal_feeds([g.shape(i) for i in all_in], 4100 + seed)]
+    outs = fetch + grads
+    want = oprune.function_sets(g.desc, all_in, outs)
+    feeds = [a if u else None for a, u in zip(feeds, want["used_inputs"])]
+    floors, ref = fp32_floors(g.desc, all_in, outs, feeds)
+    got, f = run_gpu(g.desc, all_in, outs, feeds)
+    fwd, gops, masks = f.kept_ops()
+    assert f.marked() == want["marked"] and fwd == want["fwd_ops"] and gops == [k for (_, k, _) in want["grad_ops"]]
+    assert f.used_inputs() == want["used_inputs"]
+    check_conditioned(got, ref, floors, "seed %d" % seed)
+
+
 def test_register_pressure_spills_to_shared_and_global():
     # a wide fan-in: 40 live values force shared-memory slots and workspace spill slots
     n = 3 * 4096 + 9

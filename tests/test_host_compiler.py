@@ -118,8 +118,13 @@ def test_error_codes():
     with pytest.raises(B.DragonError):
         g.function([r], [y])                                                           # x is needed but not listed
     assert b"not among the inputs" in B.lib().dragon_last_error()
+    f = g.function([x, r, y], [y])                                                     # y is given: nothing is computed
+    assert f.used_inputs() == [0, 0, 1] and f.kept_ops()[0] == []
     with pytest.raises(B.DragonError):
-        g.function([x, r, y], [y])                                                     # y is not a source
+        g.function([x, r, dr], [y])                                                    # a gradient tensor cannot be fed
+    with pytest.raises(B.DragonError) as e:
+        g.function([x, r, y], [dr])                                                    # the only chain r -> y is cut
+    assert "no chain is left" in str(e.value)
     f = g.function([x, r, bad], [y, dr])
     assert f.used_inputs() == [1, 1, 0]
     assert f.workspace_bytes() > 0 and f.num_launches() >= 1
@@ -255,6 +260,43 @@ def test_multi_output_operators_are_pruned_by_the_library_like_by_the_oracle(see
         with pytest.raises(B.DragonError) as e:
             f.run([0, 0, 0], [0] * len(fetch))
         assert e.value.code == B.ERR_UNSUPPORTED and "opaque" in str(e.value)
+
+
+@pytest.mark.parametrize("seed", range(60))
+def test_fed_intermediates_are_pruned_by_the_library_like_by_the_oracle(seed):
+    """Sec. 3.1: any tensor can be fed.  The same tiny DAGs with one or two produced tensors among the inputs:
+    the library's sets equal the oracle's (pinned by path enumeration on the graph without the edges into the
+    given tensors), and a fetched gradient that has lost its chains is refused with NO_PATH by both."""
+    from test_oracle_prune import tiny_dag_with_stages
+    rng = np.random.default_rng(9000 + seed)
+    d, fetch = tiny_dag_with_stages(rng)
+    n_fwd = len(d["tensors"]) - sum(len(st["wrts"]) for st in d["grads"])
+    fed = [int(t) for t in rng.choice(np.arange(3, n_fwd), size=int(rng.integers(1, 3)), replace=False)]
+    inputs = [0, 1, 2] + fed
+    try:
+        oprune.function_sets(d, inputs, fetch)
+    except ValueError:
+        with pytest.raises(B.DragonError) as e:
+            B.Graph.from_desc(d).function(inputs, fetch)
+        assert "no chain is left" in str(e.value)
+        return
+    compare_sets(d, inputs, fetch)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_fed_intermediates_in_random_row_dags_with_gradients(seed):
+    g, inputs, fetch = wl.random_row_dag(8, 16, seed, n_ops=60)
+    kept = oprune.function_sets(g.desc, inputs, fetch)["fwd_ops"]
+    rng = np.random.default_rng(seed)
+    fed = sorted({g.desc["ops"][int(k)]["out"][0] for k in rng.choice(kept, size=min(3, len(kept)), replace=False)} - set(fetch))
+    G = oprune.backward_marks(oprune.without_edges_into(g.desc, inputs + fed), fetch, inputs + fed)
+    wrts = [i for i in inputs + fed if i in G]
+    grads = g.grad(fetch, wrts) if wrts else []
+    f = compare_sets(g.desc, inputs + fed, fetch + grads)
+    assert "not executable" not in f.describe()
+    for t in fed:                                       # what produced a given tensor is kept only for other readers
+        k = next(k for k, op in enumerate(g.desc["ops"]) if t in op["out"])
+        assert k not in f.kept_ops()[0]
 
 
 def test_an_opaque_operator_that_is_pruned_away_does_not_stop_execution():
