@@ -180,6 +180,25 @@ int dragon_function_describe(const dragon_function_t* f, char* buf, int cap);
 int dragon_function_vm_step(const dragon_function_t* f, int step, int64_t* info, uint32_t* code, int cap_code,
                             int64_t* operands, int cap_operands, int64_t* reduced, int cap_reduced);
 
+/* Execution tier of the graph-VM programs of f.  By default (mode 1) every program is turned, at the
+ * function's first run, into a kernel of its own: the leaves of its instructions in program order as
+ * straight-line PTX with every decoded field a constant, assembled by the driver (a fraction of a second
+ * per program).  It computes what the interpreter computes, bit for bit (every leaf uses explicitly
+ * rounded operations), without fetch, decode and dispatch.  The paper has one kernel per operator
+ * (Sec. 3.3); this is the other end: one kernel per pruned function segment.  mode 0 holds f to the
+ * interpreter kernel; mode 2 specialises now and returns the number of programs specialised, or
+ * DRAGON_ERR_CUDA (with the assembler's message in dragon_last_error()) if that is not possible.  In
+ * mode 1 a program whose kernel cannot be made stays interpreted and dragon_function_describe() says so.
+ * dragon_function_num_specialized(): programs of f that currently run as specialised kernels.  The
+ * environment variable DRAGON_VM_TIER=0 makes mode 0 the default of functions created afterwards. */
+int dragon_function_specialize(dragon_function_t* f, int mode);
+int dragon_function_num_specialized(const dragon_function_t* f);
+
+/* The PTX text of the specialised kernel of a graph-VM step (step index as for dragon_function_vm_step),
+ * for tools and tests; works without a GPU.  Copies up to cap - 1 characters and a NUL into buf (buf may be
+ * NULL if cap is 0) and returns the full length, or a negative code. */
+int dragon_function_vm_ptx(const dragon_function_t* f, int step, char* buf, int cap);
+
 /* Scratch memory (partial sums, tensors that cross kernels, spilled values, a status word).
  * dev_ptr: device memory, 256-byte aligned, at least dragon_function_workspace_bytes() long,
  * owned by the caller and not touched by anyone else while a run is in flight. */

@@ -35,6 +35,9 @@ _SIGNATURES = {
     "dragon_graph_num_ops": (_c.c_int, [_c.c_void_p]),
     "dragon_function": (_c.c_void_p, [_c.c_void_p, _c.POINTER(_c.c_int32), _c.c_int, _c.POINTER(_c.c_int32), _c.c_int]),
     "dragon_function_destroy": (None, [_c.c_void_p]),
+    "dragon_function_specialize": (_c.c_int, [_c.c_void_p, _c.c_int]),
+    "dragon_function_num_specialized": (_c.c_int, [_c.c_void_p]),
+    "dragon_function_vm_ptx": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_char_p, _c.c_int]),
     "dragon_workspace_create": (_c.c_void_p, []),
     "dragon_workspace_destroy": (None, [_c.c_void_p]),
     "dragon_workspace_feed": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_int, _c.c_int, _c.POINTER(_c.c_int64), _c.c_void_p,
@@ -244,6 +247,25 @@ class Function:
                 "n_spill": info[4], "n_smem": info[5], "n_regs": info[9],
                 "operands": [tuple(ops[4 * i:4 * i + 4]) for i in range(info[3])],
                 "reduced": [tuple(red[3 * i:3 * i + 3]) for i in range(info[8])]}
+
+    def specialize(self, mode=2):
+        """0: interpreter; 1: specialised kernels from the first run on (default); 2: specialise now."""
+        r = lib().dragon_function_specialize(self.h, mode)
+        if r < 0:
+            raise DragonError(r, "dragon_function_specialize")
+        return r
+
+    def num_specialized(self):
+        return lib().dragon_function_num_specialized(self.h)
+
+    def vm_ptx(self, step):
+        """PTX text of the specialised kernel of a graph-VM step (no GPU needed)."""
+        n = lib().dragon_function_vm_ptx(self.h, step, None, 0)
+        if n < 0:
+            raise DragonError(n, "dragon_function_vm_ptx")
+        buf = _c.create_string_buffer(n + 1)
+        lib().dragon_function_vm_ptx(self.h, step, buf, n + 1)
+        return buf.value.decode()
 
     def rename_dictionary(self):
         """Algorithm 3: per tensor id the ancestor it may be renamed to (-1: not marked)."""

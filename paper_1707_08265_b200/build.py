@@ -8,7 +8,7 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdragon.so")
-SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "api.cu", "workspace.cu", "vm_launch.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
+SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "specialize.cpp", "api.cu", "workspace.cu", "vm_launch.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr", "-Xcompiler", "-Wall"] + os.environ.get("DRAGON_NVCC_DEFS", "").split()
@@ -37,6 +37,7 @@ def build(verbose=False, force=False, ptxas_info=False):
                 print(" ".join(cmd), flush=True)
             subprocess.run(cmd, check=True)
     objs.append(_generated_kernel_object(objdir, verbose, force or ptxas_info))
+    objs.append(_generated_templates_object(objdir, verbose, force))
     if force or _stale(LIB, objs):
         cmd = [NVCC, "-shared", "-o", LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a"]
         if verbose:
@@ -71,7 +72,21 @@ def _generated_kernel_object(objdir, verbose, force):
     return obj
 
 
-HOST_SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp"]     # the host compiler: no CUDA in these
+def _generated_templates_object(objdir, verbose, force):
+    """vm_ptxgen.py -> the leaves of the VM kernel as PTX text (C++ string tables) for csrc/specialize.cpp."""
+    from paper_1707_08265_b200 import vm_ptxgen
+    cpp, obj = os.path.join(objdir, "vm_templates.cpp"), os.path.join(objdir, "vm_templates.o")
+    if not (force or _stale(obj, [vm_ptxgen.__file__, os.path.join(CSRC, "vm_templates.h")])):
+        return obj
+    open(cpp, "w").write(vm_ptxgen.templates_source())
+    cmd = ["g++", "-std=c++17", "-O0", "-fPIC", "-I", CSRC, "-c", cpp, "-o", obj]
+    if verbose:
+        print(" ".join(cmd), flush=True)
+    subprocess.run(cmd, check=True)
+    return obj
+
+
+HOST_SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "specialize.cpp"]     # the host compiler: no CUDA in these
 SAN_LIB = os.path.join(HERE, "libdragon_san.so")
 
 
@@ -96,6 +111,7 @@ def build_sanitized(verbose=False):
                 print(" ".join(cmd), flush=True)
             subprocess.run(cmd, check=True)
     objs.append(os.path.join(objdir, "vm_gen_cubin.o"))
+    objs.append(os.path.join(objdir, "vm_templates.o"))
     if _stale(SAN_LIB, objs):
         cmd = [NVCC, "-shared", "-o", SAN_LIB] + objs + ["-gencode", "arch=compute_100a,code=sm_100a", "-Xcompiler", "-fsanitize=address", "-Xcompiler", "-fsanitize=undefined"]
         if verbose:

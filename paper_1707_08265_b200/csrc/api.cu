@@ -2,6 +2,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -9,7 +10,9 @@
 #include "vm_math.h"
 
 namespace dragon {
-cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st);
+cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st, void* spec_kernel);
+void load_specialized(VmSegment* sg);
+void unload_specialized(VmSegment* sg);
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st, int chunks);
 cudaError_t launch_sce_fwd(const void* z, int zdtype, const int* labels, int rows, int cols, float* rowloss, float* out,
                            int* status, cudaStream_t st, void* dz, int dzdtype, float dl_imm, float* colpart, int n_colpart);
@@ -196,6 +199,7 @@ dragon_function_t* dragon_function(dragon_graph_t* g, const dragon_id* inputs, i
   f->n_tensors = (int)g->g.tensors.size();
   f->n_in = n_in;
   f->n_out = n_out;
+  if (const char* tier = std::getenv("DRAGON_VM_TIER")) f->tier = tier[0] == '0' ? 0 : 1;
   for (int t : in) f->in_info.push_back(g->g.tensors[t]);
   for (int t : out) f->out_info.push_back(g->g.tensors[t]);
   // A listed input that an operator produces is given, not solved (Sec. 3.1: any tensor can be fed): in
@@ -234,8 +238,10 @@ void dragon_function_destroy(dragon_function_t* f) {
   for (void* ev : f->prof_ev) cudaEventDestroy(reinterpret_cast<cudaEvent_t>(ev));
   for (void* ev : f->h_event) cudaEventDestroy(reinterpret_cast<cudaEvent_t>(ev));
   for (void* s : f->h_stream) if (s) cudaStreamDestroy(reinterpret_cast<cudaStream_t>(s));
-  for (auto& sg : f->plan.segs)
+  for (auto& sg : f->plan.segs) {
     if (sg.d_code) cudaFree(sg.d_code);
+    unload_specialized(&sg);
+  }
   delete f;
 }
 
@@ -328,6 +334,9 @@ int dragon_function_num_launches(const dragon_function_t* f) {
 int dragon_function_describe(const dragon_function_t* f, char* buf, int cap) {
   if (!f || !buf || cap <= 0) return DRAGON_ERR_INVALID_ARG;
   std::string s = f->not_executable.empty() ? describe_plan(f->plan) : "not executable: " + f->not_executable + "\n";
+  for (size_t k = 0; k < f->plan.steps.size(); ++k)
+    if (f->plan.steps[k].kind == ST_VM && f->plan.segs[f->plan.steps[k].seg].spec_state < 0)
+      s += "note: the program of step " + std::to_string(k) + " runs interpreted: " + f->plan.segs[f->plan.steps[k].seg].spec_log + "\n";
   std::strncpy(buf, s.c_str(), (size_t)cap - 1);
   buf[cap - 1] = 0;
   return DRAGON_OK;
@@ -375,6 +384,62 @@ int dragon_function_set_workspace(dragon_function_t* f, void* dev_ptr, size_t by
   return DRAGON_OK;
 }
 
+// First run: device copies of the instruction streams and, unless the function is held to the interpreter,
+// the kernels specialised for them.  A program whose specialised kernel cannot be made (no assembler in
+// the driver, an assembler error) stays with the interpreter; dragon_function_describe() says why.
+static int upload_programs(dragon_function_t* f) {
+  for (auto& sg : f->plan.segs) {
+    if (sg.code.empty()) continue;
+    if (!sg.d_code && (cudaMalloc(&sg.d_code, sg.code.size() * 4) != cudaSuccess ||
+                       cudaMemcpy(sg.d_code, sg.code.data(), sg.code.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess)) {
+      set_error("dragon_run: cannot upload the instruction stream: %s", cudaGetErrorString(cudaGetLastError()));
+      sg.d_code = nullptr;
+      return DRAGON_ERR_CUDA;
+    }
+    if (f->tier && sg.spec_state == 0) load_specialized(&sg);
+  }
+  f->uploaded = true;
+  return DRAGON_OK;
+}
+
+int dragon_function_specialize(dragon_function_t* f, int mode) {
+  if (!f || mode < 0 || mode > 2) { set_error("dragon_function_specialize: bad argument"); return DRAGON_ERR_INVALID_ARG; }
+  f->tier = mode ? 1 : 0;
+  if (mode != 2) return DRAGON_OK;
+  if (!f->not_executable.empty()) { set_error("dragon_function_specialize: %s", f->not_executable.c_str()); return DRAGON_ERR_UNSUPPORTED; }
+  int n = 0;
+  for (auto& sg : f->plan.segs) {
+    if (sg.code.empty()) continue;
+    if (sg.spec_state == 0) load_specialized(&sg);
+    if (sg.spec_state != 1) { set_error("dragon_function_specialize: %s", sg.spec_log.c_str()); return DRAGON_ERR_CUDA; }
+    ++n;
+  }
+  return n;
+}
+
+int dragon_function_num_specialized(const dragon_function_t* f) {
+  if (!f) { set_error("dragon_function_num_specialized: NULL function"); return DRAGON_ERR_INVALID_ARG; }
+  int n = 0;
+  for (const auto& sg : f->plan.segs) n += f->tier && sg.spec_state == 1;
+  return n;
+}
+
+int dragon_function_vm_ptx(const dragon_function_t* f, int step, char* buf, int cap) {
+  if (!f || step < 0 || step >= (int)f->plan.steps.size() || f->plan.steps[step].kind != ST_VM || cap < 0 || (cap > 0 && !buf)) {
+    set_error("dragon_function_vm_ptx: not a graph-VM step");
+    return DRAGON_ERR_INVALID_ARG;
+  }
+  std::string ptx;
+  const int rc = specialize_ptx(f->plan.segs[f->plan.steps[step].seg], "dragon_vm_spec", &ptx);
+  if (rc != DRAGON_OK) return rc;
+  if (cap > 0) {
+    const size_t k = std::min(ptx.size(), (size_t)cap - 1);
+    std::memcpy(buf, ptx.data(), k);
+    buf[k] = 0;
+  }
+  return (int)ptx.size();
+}
+
 int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetches, void* cuda_stream) {
   if (!f || !fetches || (f->n_in > 0 && !feeds)) { set_error("dragon_run: bad argument"); return DRAGON_ERR_INVALID_ARG; }
   Plan& P = f->plan;
@@ -394,17 +459,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
     }
     ptr[m] = q;
   }
-  if (!f->uploaded) {  // first run: device copies of the instruction streams
-    for (auto& sg : P.segs) {
-      if (sg.code.empty()) continue;
-      if (cudaMalloc(&sg.d_code, sg.code.size() * 4) != cudaSuccess ||
-          cudaMemcpy(sg.d_code, sg.code.data(), sg.code.size() * 4, cudaMemcpyHostToDevice) != cudaSuccess) {
-        set_error("dragon_run: cannot upload the instruction stream: %s", cudaGetErrorString(cudaGetLastError()));
-        return DRAGON_ERR_CUDA;
-      }
-    }
-    f->uploaded = true;
-  }
+  if (upload_programs(f) != DRAGON_OK) return DRAGON_ERR_CUDA;
   // this run's status word, and the other one, which it clears for the next run
   int* const word0 = reinterpret_cast<int*>(ws + P.status_off);
   cudaError_t e = cudaSuccess;
@@ -448,7 +503,7 @@ int dragon_run(dragon_function_t* f, const void* const* feeds, void* const* fetc
           p.operand[i].dtype = (uint32_t)P.mems[sg.operand_mem[i]].dtype;
         }
         if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used]), st);
-        e = launch_vm(p, sg.grid, sg.n_smem, sg.dense, st);
+        e = launch_vm(p, sg.grid, sg.n_smem, sg.dense, st, f->tier ? sg.spec_kernel : nullptr);
         if (prof) cudaEventRecord(reinterpret_cast<cudaEvent_t>(f->prof_ev[2 * f->prof_used + 1]), st);
         if (e == cudaSuccess) e = launch_finish(sg, P.mems, ptr.data(), ws, st, 1);
         break;
@@ -556,11 +611,7 @@ int run_host_chunked(dragon_function_t* f, const std::vector<const void*>& dev_f
   cudaStream_t s_in = reinterpret_cast<cudaStream_t>(f->h_stream[0]), s_out = reinterpret_cast<cudaStream_t>(f->h_stream[1]);
   auto ev = [&](int i) { return reinterpret_cast<cudaEvent_t>(f->h_event[i]); };
   cudaEvent_t ev_start = ev(2 * kHostChunks), ev_done = ev(2 * kHostChunks + 1);
-  if (!f->uploaded) {
-    HOST_TRY(cudaMalloc(&sg.d_code, sg.code.size() * 4));
-    HOST_TRY(cudaMemcpy(sg.d_code, sg.code.data(), sg.code.size() * 4, cudaMemcpyHostToDevice));
-    f->uploaded = true;
-  }
+  if (upload_programs(f) != DRAGON_OK) return DRAGON_ERR_CUDA;
   int* const word0 = reinterpret_cast<int*>(ws + P.status_off);
   if (!f->status_ready) {
     HOST_TRY(cudaMemsetAsync(word0, 0, 256, st));
@@ -615,7 +666,7 @@ int run_host_chunked(dragon_function_t* f, const std::vector<const void*>& dev_f
       p.operand[i].kind = sg.operand_kind[i];
       p.operand[i].dtype = (uint32_t)m.dtype;
     }
-    HOST_TRY(launch_vm(p, sg.grid, sg.n_smem, sg.dense, st));
+    HOST_TRY(launch_vm(p, sg.grid, sg.n_smem, sg.dense, st, f->tier ? sg.spec_kernel : nullptr));
     HOST_TRY(cudaEventRecord(ev(kHostChunks + c), st));
     HOST_TRY(cudaStreamWaitEvent(s_out, ev(kHostChunks + c), 0));
     for (const MemRef& m : P.mems) {

@@ -110,6 +110,11 @@ struct VmSegment {
   uint32_t* d_code = nullptr;       // device copy
   int n_instr_body = 0;
   int loop_start = 0;               // index in code of the first instruction of the per-tile body
+  // the kernel specialised for this instruction stream (specialize.cpp), made from PTX at the first run
+  int spec_state = 0;               // 0 not tried yet, 1 loaded, -1 failed (the interpreter runs the program)
+  void* spec_lib = nullptr;         // cudaLibrary_t
+  void* spec_kernel = nullptr;      // cudaKernel_t
+  std::string spec_log;             // why it failed
 };
 
 enum StepKind { ST_VM, ST_GEMM, ST_TRANSPOSE, ST_SCE_FWD, ST_SCE_BWD, ST_COPY };
@@ -145,6 +150,9 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
 
 std::string describe_plan(const Plan& p);
 
+// specialize.cpp: PTX of the kernel that runs sg's instruction stream as straight-line code
+int specialize_ptx(const VmSegment& sg, const char* entry, std::string* ptx);
+
 // per operand of a VM program: position (index into the code) of its last load and of its first store
 struct VmAccess { int last_load = -1, first_store = 1 << 30; };
 std::vector<VmAccess> vm_operand_accesses(const VmSegment& sg);
@@ -157,6 +165,7 @@ struct dragon_function {
   std::vector<int> rename;   // Algorithm 3 on the pruned graph (per tensor id)
   std::string not_executable;   // non-empty: why dragon_run refuses this function (it still answers every prune query)
   int n_tensors = 0, n_in = 0, n_out = 0;
+  int tier = 1;              // 1: graph-VM programs run as specialised kernels (made at the first run), 0: interpreted
   std::vector<dragon::TensorInfo> in_info, out_info;   // name, type and shape of every listed input and output
   void* workspace = nullptr;
   size_t workspace_bytes = 0;

@@ -117,13 +117,50 @@ static const VmKernels& vm_kernels() {
   return k;
 }
 
-cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st) {
-  const VmKernels& k = vm_kernels();
-  if (k.err != cudaSuccess) return k.err;
+// spec_kernel: the kernel specialised for this program (same parameters, same launch shape), or nullptr for the interpreter
+cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dense, cudaStream_t st, void* spec_kernel) {
+  const void* fn = spec_kernel;
+  if (!fn) {
+    const VmKernels& k = vm_kernels();
+    if (k.err != cudaSuccess) return k.err;
+    fn = reinterpret_cast<const void*>(dense ? k.dense : k.wide);
+  }
   const size_t smem = vm::vm_smem_bytes(p.n_code, n_smem_slots);
   if (smem > (size_t)(dense ? 113 : 227) * 1024) return cudaErrorInvalidConfiguration;
   void* args[] = {const_cast<vm::Params*>(&p)};
-  return cudaLaunchKernel(reinterpret_cast<const void*>(dense ? k.dense : k.wide), dim3(grid), dim3(kVmThreads), args, smem, st);
+  return cudaLaunchKernel(fn, dim3(grid), dim3(kVmThreads), args, smem, st);
+}
+
+// Hands the PTX of a specialised kernel to the driver's assembler and fetches the kernel.  On failure the
+// assembler's messages (or the runtime's error) are left in sg->spec_log and the interpreter keeps the program.
+void load_specialized(VmSegment* sg) {
+  static const char* kEntry = "dragon_vm_spec";
+  sg->spec_state = -1;
+  std::string ptx;
+  if (specialize_ptx(*sg, kEntry, &ptx) != DRAGON_OK) { sg->spec_log = last_error(); return; }
+  char log[4096] = "";
+  cudaJitOption opt[] = {cudaJitErrorLogBuffer, cudaJitErrorLogBufferSizeBytes};
+  void* val[] = {log, reinterpret_cast<void*>(sizeof(log))};
+  cudaLibrary_t lib = nullptr;
+  cudaKernel_t kernel = nullptr;
+  cudaError_t e = cudaLibraryLoadData(&lib, ptx.c_str(), opt, val, 2, nullptr, nullptr, 0);
+  if (e == cudaSuccess) e = cudaLibraryGetKernel(&kernel, lib, kEntry);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (sg->dense ? 113 : 227) * 1024);
+  if (e != cudaSuccess) {
+    sg->spec_log = std::string(cudaGetErrorString(e)) + (log[0] ? std::string(": ") + log : std::string());
+    cudaGetLastError();
+    if (lib) cudaLibraryUnload(lib);
+    return;
+  }
+  sg->spec_lib = lib;
+  sg->spec_kernel = kernel;
+  sg->spec_state = 1;
+}
+
+void unload_specialized(VmSegment* sg) {
+  if (sg->spec_lib) cudaLibraryUnload(reinterpret_cast<cudaLibrary_t>(sg->spec_lib));
+  sg->spec_lib = sg->spec_kernel = nullptr;
+  sg->spec_state = 0;
 }
 
 cudaError_t launch_finish(const VmSegment& sg, const std::vector<MemRef>& mems, void* const* mem_ptr, char* ws, cudaStream_t st, int chunks) {

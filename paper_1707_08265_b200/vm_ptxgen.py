@@ -61,8 +61,12 @@ def fc(x):
 
 
 class Kernel:
-    def __init__(self, name, nr, ctas_per_sm, threads=512):
+    def __init__(self, name, nr, ctas_per_sm, threads=512, template=False):
         self.name, self.nr, self.ctas = name, nr, ctas_per_sm
+        # template mode: every leaf is generated on its own, with placeholders (#...#) where the interpreter
+        # fetches and dispatches; csrc/specialize.cpp strings such leaves together for one instruction stream
+        self.template = template
+        self.leaf_sites = []  # template mode: return labels of the sin/cos sites of the leaf being generated
         # geometry: a thread owns V elements of a tile as V/4 groups of four consecutive ones (a group is one
         # 16-byte vector, the groups of a warp are contiguous), held as NP = V/2 packed pairs
         self.NT = threads
@@ -100,7 +104,7 @@ class Kernel:
 
     def newlabel(self, stem="L"):
         self.nlabel += 1
-        return "$%s_%s_%d" % (stem, self.name, self.nlabel)
+        return "$%s_%s_%d%s" % (stem, self.name, self.nlabel, "_#I#" if self.template else "")
 
     def t(self, kind):
         self.cnt[kind] += 1
@@ -130,15 +134,33 @@ class Kernel:
         self.e("mul.rn.f32x2 %s, %s, %s;" % (d, a, b))
         return d
 
+    # In a specialised kernel a packed product of one leaf can meet a packed sum of the next, and the
+    # assembler was seen to contract such a pair into one fused multiply-add although both name their
+    # rounding (a*b + c*d then differed from the interpreter in the last place; so did the sum written as
+    # a*1 + b).  The scalar forms with an explicit rounding are never contracted, so there the packed sums
+    # and differences are written as two scalar ones: the same bits as add.rn.f32x2 / sub.rn.f32x2.
     def add2(self, a, b, d=None):
         d = d or self.rd()
-        self.e("add.rn.f32x2 %s, %s, %s;" % (d, a, b))
+        if self.template:
+            self.scalar_pair("add", a, b, d)
+        else:
+            self.e("add.rn.f32x2 %s, %s, %s;" % (d, a, b))
         return d
 
     def sub2(self, a, b, d=None):
         d = d or self.rd()
-        self.e("sub.rn.f32x2 %s, %s, %s;" % (d, a, b))
+        if self.template:
+            self.scalar_pair("sub", a, b, d)
+        else:
+            self.e("sub.rn.f32x2 %s, %s, %s;" % (d, a, b))
         return d
+
+    def scalar_pair(self, op, a, b, d):
+        (al, ah), (bl, bh) = self.unpack(a), self.unpack(b)
+        lo, hi = self.f(), self.f()
+        self.e("%s.rn.f32 %s, %s, %s;" % (op, lo, al, bl))
+        self.e("%s.rn.f32 %s, %s, %s;" % (op, hi, ah, bh))
+        self.e("mov.b64 %s, {%s, %s};" % (d, lo, hi))
 
     def unpack(self, a):
         lo, hi = self.f(), self.f()
@@ -171,11 +193,14 @@ class Kernel:
         """1 / (1 + |x|)"""
         a = self.f()
         self.e("abs.f32 %s, %s;" % (a, x))
-        self.e("add.f32 %s, %s, 0f3F800000;" % (a, a))
+        self.e("add.rn.f32 %s, %s, 0f3F800000;" % (a, a))
         return self.rcp(a)
 
     # ---- dispatch ---------------------------------------------------------------------------
     def fetch(self):
+        if self.template:       # the next instruction's argument is a constant of the specialised kernel
+            self.e("mov.u32 %arg, #NEXTARG#;")
+            return
         self.e("ld.shared.v2.u32 {%case, %arg}, [%ip];")
         self.e("add.u32 %ip, %ip, 8;")
 
@@ -198,6 +223,9 @@ class Kernel:
         # every leaf leaves through the one dispatch block: the assembler gives each indexed branch
         # its own table of branch instructions (about 2 KB per site), which with one site per leaf
         # made the code image four times larger and scattered the hot leaves
+        if self.template:       # straight to the next instruction's leaf (the assembler drops a branch to the next line)
+            self.e("bra.uni #NEXT#;")
+            return
         if getattr(self, "own_brx", False):
             self.e("brx.idx.uni %%case, JT_%s;" % self.name)
             return
@@ -283,7 +311,11 @@ class Kernel:
         self.label(stub)
         for i in range(n):
             self.e("mov.b64 %s, %s;" % (self.PX[i], xs[i]))
-        self.e("mov.u32 %%phsite, %d;" % len(self.ph_sites))
+        if self.template:
+            self.e("mov.u32 %%phsite, #SITE%d#;" % len(self.leaf_sites))
+            self.leaf_sites.append(join)
+        else:
+            self.e("mov.u32 %%phsite, %d;" % len(self.ph_sites))
         self.e("bra $PH_%s;" % self.name)
         self.end_cold()
         self.ph_sites.append(join)
@@ -315,7 +347,7 @@ class Kernel:
             return
         big = 12582912.0
         n = self.NP
-        self.e("PHRET_%s: .branchtargets %s;" % (self.name, ", ".join(self.ph_sites)))
+        self.e("PHRET_%s: .branchtargets %s;" % (self.name, "#PHRET#" if self.template else ", ".join(self.ph_sites)))
         self.label("$PH_%s" % self.name)
         base = self.rd()
         self.e("mov.u64 %s, PHBUF;" % base)
@@ -390,7 +422,7 @@ class Kernel:
         self.label(special)
         xf, z, kq = self.f(), self.f(), self.r()
         self.e("mov.b32 %s, %s;" % (xf, xb))
-        self.e("sub.f32 %s, %s, %s;" % (z, xf, xf))
+        self.e("sub.rn.f32 %s, %s, %s;" % (z, xf, xf))
         self.e("mov.u32 %s, 0x%08X;" % (kq, f32bits(big)))
         self.e("st.local.f32 [%s+%d], %s;" % (adr, 8 * n, z))
         self.e("st.local.b32 [%s+%d], %s;" % (adr, 16 * n, kq))
@@ -1015,7 +1047,7 @@ class Kernel:
             v = [self.add2(v[2 * i], v[2 * i + 1]) for i in range(len(v) // 2)]
         lo, hi = self.unpack(v[0])
         d = self.f()
-        self.e("add.f32 %s, %s, %s;" % (d, lo, hi))
+        self.e("add.rn.f32 %s, %s, %s;" % (d, lo, hi))
         return d
 
     def leaf_joint(self, op, k):
@@ -1079,16 +1111,16 @@ class Kernel:
             t = self.mul2(A[0], R[0])
             for i in range(1, self.NP): t = self.fma2(A[i], R[i], t)
             lo, hi = self.unpack(t)
-            self.e("add.f32 %s, %s, %s;" % (lo, lo, hi))
-            self.e("add.f32 %s, %s, %s;" % (acc, acc, lo))
+            self.e("add.rn.f32 %s, %s, %s;" % (lo, lo, hi))
+            self.e("add.rn.f32 %s, %s, %s;" % (acc, acc, lo))
             self.jump()
             self.label(tail)
             m = self.packs(self.mask_tail(self.scalars(A)))
             t = self.mul2(m[0], R[0])
             for i in range(1, self.NP): t = self.fma2(m[i], R[i], t)
             lo, hi = self.unpack(t)
-            self.e("add.f32 %s, %s, %s;" % (lo, lo, hi))
-            self.e("add.f32 %s, %s, %s;" % (acc, acc, lo))
+            self.e("add.rn.f32 %s, %s, %s;" % (lo, lo, hi))
+            self.e("add.rn.f32 %s, %s, %s;" % (acc, acc, lo))
         elif op == "fmaur":
             u = self.uniform()
             self.fetch()
@@ -1203,8 +1235,8 @@ class Kernel:
                     self.e("setp.lt.f32 %s, %s, 0f00000000;" % (p2, s))
                     self.e("selp.f32 %s, 0f3F800000, 0f00000000, %s;" % (g, p2))      # -sgn
                     self.e("selp.f32 %s, 0fBF800000, %s, %s;" % (g, g, p1))
-                    self.e("mul.f32 %s, %s, %s;" % (g, g, rr))
-                    self.e("mul.f32 %s, %s, %s;" % (d, g, rr))
+                    self.e("mul.rn.f32 %s, %s, %s;" % (g, g, rr))
+                    self.e("mul.rn.f32 %s, %s, %s;" % (d, g, rr))
                 out.append(d)
             self.packs(out, A)
         elif op in ("sqrt", "rcp"):
@@ -1298,10 +1330,10 @@ class Kernel:
             acc = self.S[int(op[4])]
             tail = self.newlabel("sa")
             self.e("@!%%pfull bra.uni %s;" % tail)
-            self.e("add.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(A)))
+            self.e("add.rn.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(A)))
             self.jump()
             self.label(tail)
-            self.e("add.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(self.packs(self.mask_tail(self.scalars(A))))))
+            self.e("add.rn.f32 %s, %s, %s;" % (acc, acc, self.lane_sum(self.packs(self.mask_tail(self.scalars(A))))))
         elif op == "accums":     # S[arg] += acc over the valid lanes
             a = self.slot_addr(); self.fetch()
             T = self.lds_v(a)
@@ -1347,7 +1379,7 @@ class Kernel:
         for o in (16, 8, 4, 2, 1):
             t = self.f()
             self.e("shfl.sync.bfly.b32 %s, %s, %d, 0x1f, 0xffffffff;" % (t, s, o))
-            self.e("add.f32 %s, %s, %s;" % (s, s, t))
+            self.e("add.rn.f32 %s, %s, %s;" % (s, s, t))
         warp, lane = self.warp_and_lane()
         pr, a = self.p(), self.r()
         self.e("setp.eq.u32 %s, %s, 0;" % (pr, lane))
@@ -1364,13 +1396,13 @@ class Kernel:
             q = [self.add2(q[2 * i], q[2 * i + 1]) for i in range(len(q) // 2)]
         lo, hi = self.unpack(q[0])
         tot = self.f()
-        self.e("add.f32 %s, %s, %s;" % (tot, lo, hi))
+        self.e("add.rn.f32 %s, %s, %s;" % (tot, lo, hi))
         nosync = self.newlabel("rs")
         self.e("@!%s bra.uni %s;" % (psync, nosync))
         self.e("bar.sync 0;")
         self.label(nosync)
         if scale:
-            self.e("mul.f32 %s, %s, %s;" % (tot, tot, scale))
+            self.e("mul.rn.f32 %s, %s, %s;" % (tot, tot, scale))
         tt = self.splat(tot)
         for i in range(self.NP): self.e("mov.b64 %s, %s;" % (A[i], tt))
 
@@ -1408,6 +1440,14 @@ class Kernel:
         ui, idx, ga, w, cb = self.r(), self.r(), self.rd(), self.r(), self.r()
         self.e("shl.b32 %s, %%arg, 2;" % ui)
         self.e("add.u32 %s, %s, %%ub;" % (ui, ui))
+        if self.template:       # the literal is a constant; "next" is the instruction behind it
+            self.fetch()
+            self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
+            self.e("mov.u32 %s, #LITERAL#;" % w)
+            self.e("st.shared.u32 [%s], %s;" % (ui, w))
+            self.label(skip)
+            self.jump()
+            return
         self.e("mov.u32 %s, dsm;" % cb)
         self.e("sub.u32 %s, %%ip, %s;" % (idx, cb))    # ip points at the literal's entry: 8 bytes per word
         self.e("shr.u32 %s, %s, 1;" % (idx, idx))          # -> byte offset in the 4-byte stream
@@ -1442,8 +1482,12 @@ class Kernel:
         self.label(slow)
         self.set_tile()
         self.label(join)
-        self.e("mov.u32 %s, dsm;" % cb)
-        self.e("mad.lo.u32 %%ip, %s, 8, %s;" % (self.param(P_LOOPSTART), cb))
+        if self.template:
+            self.e("mov.u32 %arg, #LOOPARG#;")
+            self.e("bra.uni #LOOP#;")
+        else:
+            self.e("mov.u32 %s, dsm;" % cb)
+            self.e("mad.lo.u32 %%ip, %s, 8, %s;" % (self.param(P_LOOPSTART), cb))
         self.label(out)
         self.fetch()
         self.jump()
@@ -1514,29 +1558,30 @@ class Kernel:
         self.e("bar.sync 0;")
 
     # ---- the kernel ---------------------------------------------------------------------------
-    def build(self):
-        nr = self.nr
-        cases = []
+    def cases(self):
+        """case id -> ("j", op, slot) | ("p", op, 0) | ("bad", op, slot)"""
+        out = []
         for op in JOINT:
             for k in range(JOINT_STRIDE):
-                no_slot = op.startswith("stld") and int(op[4]) >= nr
-                cases.append(("j", op, k) if k < nr and not no_slot else ("bad", op, k))
+                no_slot = op.startswith("stld") and int(op[4]) >= self.nr
+                out.append(("j", op, k) if k < self.nr and not no_slot else ("bad", op, k))
         for op in PLAIN:
-            cases.append(("p", op, 0))
-        bad = "$BAD_%s" % self.name
-        labels = [bad if c[0] == "bad" else "$C_%s_%d" % (self.name, i) for i, c in enumerate(cases)]
-        body = self.lines
+            out.append(("p", op, 0))
+        return out
+
+    def prologue(self):
         e = self.e
-        # ---- prologue ----
-        tx, ncode, t0 = self.r(), self.param(P_NCODE, "s32"), self.r()
+        tx = self.r()
         e("mov.u32 %s, %%tid.x;" % tx)
         e("shl.b32 %%pos0, %s, 2;" % tx)
         # shared memory: decoded code | uniforms | reduction scratch | operand table | slots
-        e("add.s32 %s, %s, 3;" % (t0, ncode))
-        e("and.b32 %s, %s, 0xfffffffc;" % (t0, t0))
-        e("shl.b32 %s, %s, 3;" % (t0, t0))
         e("mov.u32 %ub, dsm;")
-        e("add.u32 %%ub, %%ub, %s;" % t0)
+        if not self.template:       # a specialised kernel holds no instruction stream: its uniforms start the area
+            ncode, t0 = self.param(P_NCODE, "s32"), self.r()
+            e("add.s32 %s, %s, 3;" % (t0, ncode))
+            e("and.b32 %s, %s, 0xfffffffc;" % (t0, t0))
+            e("shl.b32 %s, %s, 3;" % (t0, t0))
+            e("add.u32 %%ub, %%ub, %s;" % t0)
         e("mad.lo.u32 %%sa, %s, 16, %%ub;" % tx)
         e("add.u32 %%sa, %%sa, %d;" % OFF_SLOTS)
         # operand table -> shared memory (one entry per thread)
@@ -1548,24 +1593,26 @@ class Kernel:
             e("ld.param.u32 %s, [VP+%d];" % (d, P_OPERAND + 16 * i + 12))
             e("@%s st.shared.u64 [%%ub+%d], %s;" % (pr, OFF_OPB + 16 * i, ptr))
             e("@%s st.shared.v2.u32 [%%ub+%d], {%s, %s};" % (pr, OFF_OPB + 16 * i + 8, k, d))
-        # decode the instruction stream: {case id, argument} per word
-        lp, ld_ = self.newlabel("dec"), self.newlabel("dec")
-        i_, pr, ga, w, c, a, sa, code = self.r(), self.p(), self.rd(), self.r(), self.r(), self.r(), self.r(), self.param(P_CODE, "u64")
-        e("mov.u32 %s, %s;" % (i_, tx))
-        self.label(lp)
-        e("setp.ge.s32 %s, %s, %s;" % (pr, i_, ncode))
-        e("@%s bra %s;" % (pr, ld_))
-        e("mul.wide.u32 %s, %s, 4;" % (ga, i_))
-        e("add.u64 %s, %s, %s;" % (ga, ga, code))
-        e("ld.global.nc.u32 %s, [%s];" % (w, ga))
-        e("and.b32 %s, %s, 1023;" % (c, w))
-        e("shr.u32 %s, %s, 14;" % (a, w))
-        e("mov.u32 %s, dsm;" % sa)
-        e("mad.lo.u32 %s, %s, 8, %s;" % (sa, i_, sa))
-        e("st.shared.v2.u32 [%s], {%s, %s};" % (sa, c, a))
-        e("add.u32 %s, %s, %d;" % (i_, i_, self.NT))
-        e("bra %s;" % lp)
-        self.label(ld_)
+        if not self.template:
+            # decode the instruction stream: {case id, argument} per word
+            ncode = self.param(P_NCODE, "s32")
+            lp, ld_ = self.newlabel("dec"), self.newlabel("dec")
+            i_, pr, ga, w, c, a, sa, code = self.r(), self.p(), self.rd(), self.r(), self.r(), self.r(), self.r(), self.param(P_CODE, "u64")
+            e("mov.u32 %s, %s;" % (i_, tx))
+            self.label(lp)
+            e("setp.ge.s32 %s, %s, %s;" % (pr, i_, ncode))
+            e("@%s bra %s;" % (pr, ld_))
+            e("mul.wide.u32 %s, %s, 4;" % (ga, i_))
+            e("add.u64 %s, %s, %s;" % (ga, ga, code))
+            e("ld.global.nc.u32 %s, [%s];" % (w, ga))
+            e("and.b32 %s, %s, 1023;" % (c, w))
+            e("shr.u32 %s, %s, 14;" % (a, w))
+            e("mov.u32 %s, dsm;" % sa)
+            e("mad.lo.u32 %s, %s, 8, %s;" % (sa, i_, sa))
+            e("st.shared.v2.u32 [%s], {%s, %s};" % (sa, c, a))
+            e("add.u32 %s, %s, %d;" % (i_, i_, self.NT))
+            e("bra %s;" % lp)
+            self.label(ld_)
         e("bar.sync 0;")
         # per-CTA spill area: spill + cta * n_spill * TILE floats, this thread's 16 bytes
         t2, t3, cta = self.rd(), self.rd(), self.r()
@@ -1592,6 +1639,29 @@ class Kernel:
         self.label(skip_c)
         e("mov.u32 %%tile, %s;" % cta)
         self.set_tile()
+
+    def declarations(self):
+        decl = []
+        for kind, ty in (("f", ".f32"), ("r", ".b32"), ("rd", ".b64"), ("p", ".pred"), ("fd", ".f64"), ("h", ".b16")):
+            if self.cnt[kind]:
+                decl.append("\t.reg %s %%%s<%d>;" % (ty, kind, self.cnt[kind]))
+        decl.append("\t.reg .b32 %pos0, %limit, %tnext, %tile, %ub, %sa, %ip, %case, %arg;")
+        decl.append("\t.reg .b64 %tb4, %spb;")
+        decl.append("\t.reg .pred %pfull;")
+        decl.append("\t.local .align 8 .b8 PHBUF[96];")
+        decl.append("\t.reg .b64 %s;" % ", ".join(self.PX + self.PR + self.PK))
+        decl.append("\t.reg .b32 %phsite;")
+        decl.append("\t.reg .f32 %s;" % ", ".join(self.S))
+        decl.append("\t.reg .b64 %s;" % ", ".join(self.A + sum(self.R, [])))
+        return decl
+
+    def build(self):
+        cases = self.cases()
+        bad = "$BAD_%s" % self.name
+        labels = [bad if c[0] == "bad" else "$C_%s_%d" % (self.name, i) for i, c in enumerate(cases)]
+        body = self.lines
+        e = self.e
+        self.prologue()
         e("mov.u32 %ip, dsm;")
         self.fetch()
         e("JT_%s: .branchtargets %s;" % (self.name, ", ".join(labels)))
@@ -1626,19 +1696,34 @@ class Kernel:
         head.append(".maxntid %d, 1, 1" % self.NT)
         head.append(".minnctapersm %d" % self.ctas)
         head.append("{")
-        decl = []
-        for kind, ty in (("f", ".f32"), ("r", ".b32"), ("rd", ".b64"), ("p", ".pred"), ("fd", ".f64"), ("h", ".b16")):
-            if self.cnt[kind]:
-                decl.append("\t.reg %s %%%s<%d>;" % (ty, kind, self.cnt[kind]))
-        decl.append("\t.reg .b32 %pos0, %limit, %tnext, %tile, %ub, %sa, %ip, %case, %arg;")
-        decl.append("\t.reg .b64 %tb4, %spb;")
-        decl.append("\t.reg .pred %pfull;")
-        decl.append("\t.local .align 8 .b8 PHBUF[96];")
-        decl.append("\t.reg .b64 %s;" % ", ".join(self.PX + self.PR + self.PK))
-        decl.append("\t.reg .b32 %phsite;")
-        decl.append("\t.reg .f32 %s;" % ", ".join(self.S))
-        decl.append("\t.reg .b64 %s;" % ", ".join(self.A + sum(self.R, [])))
-        return "\n".join(head + decl + body + ["}"]) + "\n"
+        return "\n".join(head + self.declarations() + body + ["}"]) + "\n"
+
+    def build_templates(self):
+        """-> dict(head, prologue, leaves = {case id: (text, cold text, [site return labels])}, reduction):
+        the pieces of a kernel that runs one instruction stream as straight-line code.  Placeholders:
+        #I# (number of the instruction, makes labels unique), #NEXT# / #NEXTARG# (label and argument of the
+        instruction that follows), #LOOP# / #LOOPARG# (of the first instruction of the per-tile body),
+        #LITERAL# (the word behind a uconst), #SITEk# (number of the leaf's k-th sin/cos site among all
+        sites of the kernel), #PHRET# (the return labels of all sites)."""
+        assert self.template
+
+        def capture(fn):
+            self.lines, self.cold, self.leaf_sites = [], [], []
+            fn()
+            return "\n".join(self.lines) + "\n", "\n".join(self.cold) + ("\n" if self.cold else ""), list(self.leaf_sites)
+
+        prologue = capture(self.prologue)[0].replace("#I#", "P")
+        leaves = {}
+        for i, (kind, op, k) in enumerate(self.cases()):
+            if kind == "bad":
+                continue
+            leaves[i] = capture((lambda: self.leaf_joint(op, k)) if kind == "j" else (lambda: self.leaf_plain(op)))
+        self.ph_sites = ["x"]
+        reduction = capture(self.emit_general_reduction)[0].replace("#I#", "R")
+        head = [".visible .entry #ENTRY#(.param .align 8 .b8 VP[%d])" % P_SIZE, ".maxntid %d, 1, 1" % self.NT,
+                ".minnctapersm %d" % self.ctas, "{"] + self.declarations()
+        assert not self.kt, "packed constants are immediates"
+        return dict(head="\n".join(head) + "\n", prologue=prologue, leaves=leaves, reduction=reduction)
 
 
 # name, register slots, CTAs per SM, threads per CTA.  The generator also takes 1024 threads (four elements per
@@ -1649,17 +1734,99 @@ class Kernel:
 VARIANTS = [("dragon_vm_wide", 7, 1, 512), ("dragon_vm_dense", 3, 2, 512)]
 
 
+MODULE_HEAD = [".version 8.8", ".target sm_100a", ".address_size 64", "", ".extern .shared .align 16 .b8 dsm[];",
+               # 2/pi = 0x0.A2F9836E4E44... behind one word of zeros (its integer part), most significant word first
+               ".const .align 4 .b32 TWO_OVER_PI[9] = {0x00000000, 0xA2F9836E, 0x4E441529, 0xFC2757D1, 0xF534DDC0, 0xDB629599, 0x3C439041, 0xFE5163AB, 0xDEBBC561};", ""]
+
+
 def generate():
-    out = [".version 8.8", ".target sm_100a", ".address_size 64", "", ".extern .shared .align 16 .b8 dsm[];",
-           # 2/pi = 0x0.A2F9836E4E44... behind one word of zeros (its integer part), most significant word first
-           ".const .align 4 .b32 TWO_OVER_PI[9] = {0x00000000, 0xA2F9836E, 0x4E441529, 0xFC2757D1, 0xF534DDC0, 0xDB629599, 0x3C439041, 0xFE5163AB, 0xDEBBC561};", ""]
+    out = list(MODULE_HEAD)
     for name, nr, ctas, threads in VARIANTS:
         out.append(Kernel(name, nr, ctas, threads).build())
     return "\n".join(out)
 
 
+def specialise(template, code, loop_start, entry="dragon_vm_spec"):
+    """Python twin of csrc/specialize.cpp (used by the tests to check the C++ stitcher and the templates):
+    the PTX of the kernel that runs the instruction words ``code`` as straight-line code."""
+    n = len(code)
+    uconst = JOINT_STRIDE * len(JOINT) + PLAIN.index("uconst")
+    body, cold, sites = [], [], []
+    pc = 0
+
+    def label(i):
+        return "$I_%d" % i if i < n else "$I_END"
+
+    while pc < n:
+        case, arg = code[pc] & 1023, code[pc] >> 14
+        text, cold_text, leaf_sites = template["leaves"][case]
+        nxt = pc + 2 if case == uconst else pc + 1
+        sub = {"I": str(pc), "NEXT": label(nxt), "NEXTARG": str(code[nxt] >> 14 if nxt < n else 0), "LOOP": label(loop_start),
+               "LOOPARG": str(code[loop_start] >> 14), "LITERAL": str(code[pc + 1]) if case == uconst else "0"}
+        for k in range(len(leaf_sites)):
+            sub["SITE%d" % k] = str(len(sites) + k)
+
+        def fill(t):
+            parts = t.split("#")
+            return "".join(p if i % 2 == 0 else sub[p] for i, p in enumerate(parts))
+
+        sites += [fill(l) for l in leaf_sites]
+        body.append(label(pc) + ":\n" + fill(text))
+        cold.append(fill(cold_text))
+        pc = nxt
+    out = "\n".join(MODULE_HEAD) + "\n" + template["head"].replace("#ENTRY#", entry) + template["prologue"]
+    out += "\tmov.u32 %%arg, %d;\n" % (code[0] >> 14) + "".join(body) + "$I_END:\n\texit;\n" + "".join(cold)
+    if sites:
+        out += template["reduction"].replace("#PHRET#", ", ".join(sites))
+    return out + "}\n"
+
+
+def templates_source():
+    """C++ source of the leaf templates of both builds, compiled into the library for csrc/specialize.cpp."""
+    out = ["// generated by vm_ptxgen.py: the leaves of the graph-VM kernel as PTX text with placeholders", "#include \"vm_templates.h\"", "",
+           "namespace dragon {", "namespace vmt {", ""]
+
+    def lit(text):
+        # raw string literals in pieces: some compilers limit the length of one literal
+        chunks, cur, size = [], [], 0
+        for line in text.splitlines(True):
+            cur.append(line)
+            size += len(line)
+            if size > 12000:
+                chunks.append("".join(cur)); cur, size = [], 0
+        if cur or not chunks:
+            chunks.append("".join(cur))
+        return "\n".join('R"PTX(%s)PTX"' % c for c in chunks)
+
+    out.append("const char* const kModuleHead = %s;" % lit("\n".join(MODULE_HEAD) + "\n"))
+    names = []
+    for name, nr, ctas, threads in VARIANTS:
+        t = Kernel(name, nr, ctas, threads, template=True).build_templates()
+        n_cases = JOINT_STRIDE * len(JOINT) + len(PLAIN)
+        tag = name.replace("dragon_vm_", "")
+        out.append("static const Leaf kLeaves_%s[%d] = {" % (tag, n_cases))
+        for i in range(n_cases):
+            if i in t["leaves"]:
+                text, cold, sites = t["leaves"][i]
+                out.append("  {%s,\n   %s,\n   %d, \"%s\"}," % (lit(text), lit(cold), len(sites), ",".join(sites)))
+            else:
+                out.append("  {nullptr, nullptr, 0, nullptr},")
+        out.append("};")
+        names.append((tag, nr, n_cases, t))
+    out.append("const Variant kVariants[%d] = {" % len(names))
+    for tag, nr, n_cases, t in names:
+        out.append("  {%d, %d, %s,\n   %s,\n   %s,\n   kLeaves_%s}," % (nr, n_cases, lit(t["head"]), lit(t["prologue"]), lit(t["reduction"]), tag))
+    out.append("};")
+    out.append("const int kNumVariants = %d;" % len(names))
+    out += ["", "}  // namespace vmt", "}  // namespace dragon", ""]
+    return "\n".join(out)
+
+
+
+
 if __name__ == "__main__":
-    text = generate()
+    text = templates_source() if "--templates" in sys.argv[1:] else generate()
+    sys.argv = [a for a in sys.argv if a != "--templates"]
     if len(sys.argv) > 1:
         open(sys.argv[1], "w").write(text)
     else:
