@@ -30,10 +30,10 @@ METRIC = "pruned-graph fwd+bwd elements/sec"
 UNIT = "elements/s"
 WORKLOAD = "config 2: f=x*sin(a*x+b), x fp32[2^26], fetch df/dx, df/da, df/db"
 ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the VM kernel on this workload at the full 2^26
-# elements, from one ncu capture of this kernel binary (profiles/vm_dense_config2.md); None once the kernel has
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the specialised VM kernel of this workload at the
+# full 2^26 elements, from one ncu capture (profiles/vm_config2.md); None once the generator of that kernel has
 # changed since the counters were taken
-NCU_DRAM_BYTES_PER_LAUNCH = 268571648 + 222234880
+NCU_DRAM_BYTES_PER_LAUNCH = 268459264 + 218289408
 SAMPLE_ELEMS = 1 << 21       # the CPU oracle's bounded sample of workload 2, per pass
 
 
@@ -266,6 +266,7 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None, world=1, rank=0, 
         return t_.to(tdt[ti["dtype"]])
 
     f = B.Graph.from_desc(g.desc).function(inputs, outputs)
+    f.specialize(0 if args.interpreter else 1)
     feeds = [dev_random(t) if u else None for t, u in zip(inputs, f.used_inputs())]
     if cfg == 4:
         for j in (1, 2, 3, 4):     # weights and biases ~ N(0, 1/4096)
@@ -331,12 +332,14 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None, world=1, rank=0, 
     line = {"workload": c["what"], "ms_per_step": ms, "value": world * c["units"] / (ms * 1e-3), "unit": c["unit"], "steps": steps,
             "n_gpus": world, "scaling": "weak", "exchanged_outputs": [k for k in kinds if k in (sharding.SUM, sharding.MEAN)],
             "launches_per_step": f.num_launches(), "kept_forward_ops": len(fwd), "kept_gradient_ops": len(gops), "ops_in_graph": f.n_ops,
-            "fed_and_fetched_bytes": io_bytes, "plan": plan[:16], "kernel_ms": [round(k, 5) for k in kern[:16]]}
+            "fed_and_fetched_bytes": io_bytes, "plan": plan[:16], "kernel_ms": [round(k, 5) for k in kern[:16]],
+            "vm_tier": "specialised kernels" if f.num_specialized() else ("interpreter" if any(p_.startswith("vm[") for p_ in plan) else "no graph-VM program in the plan")}
     if c["bound"] == "hbm":
         alg = c["alg"] if c["alg"] is not None else float(io_bytes)
         k_ms = sum(kern) if cfg != 1 else kern[0]
         ach = alg / (k_ms * 1e-3) / 1e9
-        line["roofline"] = {"bound": "hbm", "kernel": plan[top].split("[")[0] + (" dense" if " dense " in plan[top] else " wide" if " wide " in plan[top] else ""),
+        build = "dense" if " dense " in plan[top] else "wide" if " wide " in plan[top] else ""
+        line["roofline"] = {"bound": "hbm", "kernel": ("dragon_vm_spec (specialised, %s build)" % build) if f.num_specialized() else "dragon_vm_" + build,
                             "achieved": ach, "peak": peaks["hbm"], "unit": "GB/s", "frac": ach / peaks["hbm"], "peak_kind": peaks["kind"],
                             "algorithmic_bytes": alg, "kernel_ms": k_ms, "traffic": None, "frac_of_nominal_8TBs": ach / 8000.0,
                             "frac_on_fed_and_fetched_bytes": io_bytes / (k_ms * 1e-3) / 1e9 / peaks["hbm"]}
@@ -345,7 +348,7 @@ def time_config(cfg, args, B, torch, seeds, peaks, steps=None, world=1, rank=0, 
             line["ms_l2_flushed"] = flushed
             line["roofline"]["frac_l2_flushed"] = alg / (flushed * 1e-3) / 1e9 / peaks["hbm"]
         if cfg == 5 or cfg == 7:
-            line["roofline"]["note"] = "not HBM-bound: one interpreter launch of a few hundred instructions per row with many row sums (CTA barriers); the HBM fraction is reported as asked"
+            line["roofline"]["note"] = "achieved = the workload's nominal 16 FULL tensors over the kernel time; frac_on_fed_and_fetched_bytes counts what the pruned function really reads and writes; one launch of a few hundred VM instructions per row with several row sums (CTA barriers) at 16 warps per SM"
     else:
         whole = c["alg"] / (ms * 1e-3) / 1e12
         gemm = [k for k, p in zip(kern, plan) if p.startswith("gemm")]
@@ -367,6 +370,7 @@ def main():
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--elements", type=int, default=N_ELEMS, help="elements per GPU of workload 2 (default: its 2^26) or 3 (default 2^27); smaller for profiler captures")
     ap.add_argument("--rows", type=int, default=16384, help="rows of workload 5 (default: its 16384; smaller for profiler captures)")
+    ap.add_argument("--interpreter", action="store_true", help="hold the graph-VM programs to the interpreter kernel (default: specialised kernels)")
     ap.add_argument("--skip-cpu-baseline", action="store_true")
     ap.add_argument("--skip-other-configs", action="store_true", help="leave the \"configs\" entry (workloads 1, 3, 4, 5) out")
     ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5, 6, 7, 8],
@@ -411,6 +415,7 @@ def main():
     inputs = [ids["x"], ids["a"], ids["b"]]
     outputs = [ids["dx"], ids["da"], ids["db"]]
     f = B.Graph.from_desc(g.desc).function(inputs, outputs)
+    f.specialize(0 if args.interpreter else 1)
     f.ensure_workspace()
     stream = torch.cuda.Stream()
     d_feeds = [torch.from_numpy(np.ascontiguousarray(v)).cuda() for v in (x, a, b)]
@@ -488,6 +493,7 @@ def main():
     assert np.array_equal(h_out[0][:1024].numpy(), d_out[0][:1024].cpu().numpy())
     plan = f.describe().strip().split("\n")
     launches = f.num_launches()
+    specialised = f.num_specialized() > 0
     del stg, d_feeds, d_out, h_x, h_out
     torch.cuda.empty_cache()
 
@@ -502,14 +508,15 @@ def main():
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warm,
                 "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "f32", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "elements_per_gpu": n, "l2": "inputs+outputs (512 MiB) larger than L2", "plan": plan},
+                "config": {"workload": WORKLOAD, "elements_per_gpu": n, "l2": "inputs+outputs (512 MiB) larger than L2", "plan": plan,
+                           "vm_tier": "specialised kernel" if specialised else "interpreter"},
                 "clocks": sampler.summary(),
                 "e2e": {"value": world * n * e2e_steps / (e2e_ms * 1e-3), "unit": UNIT,
                         "h2d_bytes_per_step": 4 * n + 8, "d2h_bytes_per_step": 4 * n + 8},
                 "gpu_launches": launches * args.steps,
-                "roofline": {"bound": "hbm", "kernel": "dragon_vm_dense", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
+                "roofline": {"bound": "hbm", "kernel": "dragon_vm_spec (specialised, dense build)" if specialised else "dragon_vm_dense", "achieved": achieved, "peak": peaks["hbm"], "unit": "GB/s",
                              "frac": achieved / peaks["hbm"], "peak_kind": peaks["kind"],
-                             "traffic": NCU_DRAM_BYTES_PER_LAUNCH if n == N_ELEMS else None,
+                             "traffic": NCU_DRAM_BYTES_PER_LAUNCH if n == N_ELEMS and specialised else None,
                              "kernel_ms": kern_avg_ms, "frac_of_nominal_8TBs": achieved / 8000.0}}
         if others:
             line["configs"] = others

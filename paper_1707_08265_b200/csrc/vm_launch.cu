@@ -5,6 +5,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 
 #include "plan.h"
@@ -136,6 +137,10 @@ cudaError_t launch_vm(const vm::Params& p, int grid, int n_smem_slots, bool dens
 void load_specialized(VmSegment* sg) {
   static const char* kEntry = "dragon_vm_spec";
   sg->spec_state = -1;
+  // test hook: behave as if the driver had no assembler, so that the fall-back to the interpreter can be exercised
+  if (const char* off = std::getenv("DRAGON_VM_NO_ASSEMBLER")) {
+    if (off[0] == '1') { sg->spec_log = "no assembler (DRAGON_VM_NO_ASSEMBLER=1)"; return; }
+  }
   std::string ptx;
   if (specialize_ptx(*sg, kEntry, &ptx) != DRAGON_OK) { sg->spec_log = last_error(); return; }
   char log[4096] = "";

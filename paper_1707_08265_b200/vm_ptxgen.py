@@ -631,6 +631,17 @@ class Kernel:
         """-> (ptr u64, kind u32, dtype u32) of operand[%arg] (or [idx_reg]) from the shared-memory copy of the table"""
         a, ptr = self.r(), self.rd()
         self.e("shl.b32 %s, %s, 4;" % (a, idx_reg or "%arg"))
+        if self.template:       # the index is a constant there: the entry is read straight from the kernel's parameters
+            a64, base = self.rd(), self.rd()
+            self.e("cvt.u64.u32 %s, %s;" % (a64, a))
+            self.e("mov.u64 %s, VP;" % base)
+            self.e("add.u64 %s, %s, %s;" % (base, base, a64))
+            self.e("ld.param.u64 %s, [%s+%d];" % (ptr, base, P_OPERAND))
+            if not want_meta:
+                return ptr, None, None
+            kind, dt = self.r(), self.r()
+            self.e("ld.param.v2.u32 {%s, %s}, [%s+%d];" % (kind, dt, base, P_OPERAND + 8))
+            return ptr, kind, dt
         self.e("add.u32 %s, %s, %%ub;" % (a, a))
         self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
         if not want_meta:
@@ -687,8 +698,15 @@ class Kernel:
         a, ptr, sl, sadr = self.r(), self.rd(), self.r(), self.r()
         self.e("and.b32 %s, %%arg, 63;" % a)
         self.e("shl.b32 %s, %s, 4;" % (a, a))
-        self.e("add.u32 %s, %s, %%ub;" % (a, a))
-        self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
+        if self.template:
+            a64, base = self.rd(), self.rd()
+            self.e("cvt.u64.u32 %s, %s;" % (a64, a))
+            self.e("mov.u64 %s, VP;" % base)
+            self.e("add.u64 %s, %s, %s;" % (base, base, a64))
+            self.e("ld.param.u64 %s, [%s+%d];" % (ptr, base, P_OPERAND))
+        else:
+            self.e("add.u32 %s, %s, %%ub;" % (a, a))
+            self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
         if masked:
             self.e("bfe.u32 %s, %%arg, 6, 4;" % sl)
         else:

@@ -143,3 +143,28 @@ def test_host_buffer_run_in_chunks_same_bits():
         res.append([o.clone() for o in outs])
     for k in range(3):
         assert np.array_equal(bits(res[0][k]), bits(res[1][k])), k
+
+
+def test_without_an_assembler_the_interpreter_runs_and_says_so(monkeypatch):
+    """A driver without the PTX assembler (simulated on the host): in the default mode the program stays with
+    the interpreter, the plan says why, the results are the oracle's; asking for specialisation outright fails."""
+    from oracle import interp
+    monkeypatch.setenv("DRAGON_VM_NO_ASSEMBLER", "1")
+    n = 3 * 4096 + 5
+    g, ids = wl.toy_function_grad(n)
+    inputs, outputs = [ids["x"], ids["a"], ids["b"]], [ids["dx"], ids["da"], ids["db"]]
+    x, a, b = wl.toy_feeds(n, 3)
+    f = B.Graph.from_desc(g.desc).function(inputs, outputs)
+    f.specialize(1)
+    dev = [torch.from_numpy(np.ascontiguousarray(v)).cuda() for v in (x, a, b)]
+    outs = [torch.full(tuple(g.shape(o)), float("nan"), device="cuda") for o in outputs]
+    f.run_torch(dev, outs)
+    assert f.status() == 0 and f.num_specialized() == 0
+    assert "runs interpreted: no assembler" in f.describe()
+    ref = interp.run_function(g.desc, inputs, outputs, [x, a, b])
+    for o, r in zip(outs, ref):
+        assert np.all(np.abs(o.cpu().numpy() - r) <= 1e-5 * (1 + np.abs(r)))
+    f2 = B.Graph.from_desc(g.desc).function(inputs, outputs)
+    with pytest.raises(B.DragonError) as e:
+        f2.specialize(2)
+    assert e.value.code == B.ERR_CUDA and "no assembler" in str(e.value)
