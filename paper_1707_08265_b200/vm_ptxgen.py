@@ -1432,10 +1432,13 @@ class Kernel:
         self.e("shr.u32 %s, %%arg, 9;" % oi)
         self.fetch()
         self.e("@!%s bra %s;" % (self.tx_is_zero(), skip))
-        self.e("shl.b32 %s, %s, 4;" % (a, oi))
-        self.e("add.u32 %s, %s, %%ub;" % (a, a))
-        self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
-        self.e("ld.shared.u32 %s, [%s+%d];" % (dt, a, OFF_OPB + 12))
+        if self.template:
+            ptr, _, dt = self.operand(idx_reg=oi)
+        else:
+            self.e("shl.b32 %s, %s, 4;" % (a, oi))
+            self.e("add.u32 %s, %s, %%ub;" % (a, a))
+            self.e("ld.shared.u64 %s, [%s+%d];" % (ptr, a, OFF_OPB))
+            self.e("ld.shared.u32 %s, [%s+%d];" % (dt, a, OFF_OPB + 12))
         self.e("setp.ne.u32 %s, %s, 0;" % (pb, dt))
         self.e("@%s bra %s;" % (pb, lb))
         self.e("ld.global.nc.f32 %s, [%s];" % (v, ptr))
@@ -1602,8 +1605,9 @@ class Kernel:
             e("add.u32 %%ub, %%ub, %s;" % t0)
         e("mad.lo.u32 %%sa, %s, 16, %%ub;" % tx)
         e("add.u32 %%sa, %%sa, %d;" % OFF_SLOTS)
-        # operand table -> shared memory (one entry per thread)
-        for i in range(MAX_OPERANDS):
+        # operand table -> shared memory (one entry per thread); a specialised kernel reads its entries, whose
+        # indices are constants there, straight from the parameters
+        for i in range(0 if self.template else MAX_OPERANDS):
             pr, ptr, k, d = self.p(), self.rd(), self.r(), self.r()
             e("setp.eq.u32 %s, %s, %d;" % (pr, tx, i))
             e("ld.param.u64 %s, [VP+%d];" % (ptr, P_OPERAND + 16 * i))
