@@ -45,9 +45,11 @@ def test_library_rename_dictionary_matches_the_oracle(seed):
     f = B.Graph.from_desc(g.desc).function(inputs, fetch)
     want = oprune.function_sets(g.desc, inputs, fetch)
     marked = [t for t, m in enumerate(want["marked"]) if m]
-    rd = inplace.rename_dictionary(g.desc, marked, want["fwd_ops"])
+    # the definition written out (no shared walk state), not the step-by-step form the library also follows
+    rd = inplace.rename_dictionary_bruteforce(g.desc, marked, want["fwd_ops"])
     got = f.rename_dictionary()
     assert got == [rd.get(t, -1) for t in range(len(got))]
+    assert rd == inplace.rename_dictionary(g.desc, marked, want["fwd_ops"])
 
 
 def test_toy_function_structures():
