@@ -199,6 +199,18 @@ int dragon_function_num_specialized(const dragon_function_t* f);
  * NULL if cap is 0) and returns the full length, or a negative code. */
 int dragon_function_vm_ptx(const dragon_function_t* f, int step, char* buf, int cap);
 
+/* Static check of a graph-VM instruction stream (encoding: csrc/vm_isa.h): every case id exists in the
+ * kernel build with register_slots slots (3 or 7), every register slot, shared-memory slot, uniform,
+ * memory operand, spill slot and accumulator an instruction names lies inside the given limits, row sums
+ * occur only in row programs, and the stream is loop_begin ... body from loop_start ... one loop end ...
+ * end.  A program is immutable once compiled, so this check on the host stands for a range check in every
+ * leaf of the kernel; the compiler runs it on each program it emits (a failure there is
+ * DRAGON_ERR_UNSUPPORTED at dragon_function) and this entry point exposes it to tools and tests.
+ * code: host array of n_code words.  Returns DRAGON_OK or DRAGON_ERR_INVALID_ARG (dragon_last_error()
+ * names the word and the index).  The paper has no counterpart: its operators are separate kernels. */
+int dragon_verify_vm_program(const uint32_t* code, int n_code, int loop_start, int register_slots, int n_operands,
+                             int n_smem_slots, int n_spill_slots, int n_column_accs, int n_scalar_accs, int row_mode);
+
 /* Scratch memory (partial sums, tensors that cross kernels, spilled values, a status word).
  * dev_ptr: device memory, 256-byte aligned, at least dragon_function_workspace_bytes() long,
  * owned by the caller and not touched by anyone else while a run is in flight. */

@@ -38,6 +38,8 @@ _SIGNATURES = {
     "dragon_function_specialize": (_c.c_int, [_c.c_void_p, _c.c_int]),
     "dragon_function_num_specialized": (_c.c_int, [_c.c_void_p]),
     "dragon_function_vm_ptx": (_c.c_int, [_c.c_void_p, _c.c_int, _c.c_char_p, _c.c_int]),
+    "dragon_verify_vm_program": (_c.c_int, [_c.POINTER(_c.c_uint32), _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int, _c.c_int,
+                                            _c.c_int, _c.c_int, _c.c_int]),
     "dragon_workspace_create": (_c.c_void_p, []),
     "dragon_workspace_destroy": (None, [_c.c_void_p]),
     "dragon_workspace_feed": (_c.c_int, [_c.c_void_p, _c.c_char_p, _c.c_int, _c.c_int, _c.POINTER(_c.c_int64), _c.c_void_p,
@@ -387,6 +389,15 @@ class Workspace:
         r = lib().dragon_workspace_run(self.h, function.h, names, stream)
         if r < 0:
             raise DragonError(r, "dragon_workspace_run")
+
+
+def verify_vm_program(code, loop_start, register_slots, n_operands, n_smem, n_spill, n_colacc, n_scalacc, row_mode):
+    """dragon_verify_vm_program: raises DragonError (INVALID_ARG) naming the first bad word."""
+    arr = (_c.c_uint32 * max(1, len(code)))(*code)
+    r = lib().dragon_verify_vm_program(arr, len(code), loop_start, register_slots, n_operands, n_smem, n_spill, n_colacc,
+                                       n_scalacc, int(bool(row_mode)))
+    if r < 0:
+        raise DragonError(r, "dragon_verify_vm_program")
 
 
 def softmax_ce_loss_static(logits_ptr, dtype, labels_ptr, rows, cols, loss_ptr, stream=0):

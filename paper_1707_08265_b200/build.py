@@ -8,7 +8,7 @@ sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libdragon.so")
-SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "specialize.cpp", "api.cu", "workspace.cu", "vm_launch.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
+SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "specialize.cpp", "verify.cpp", "api.cu", "workspace.cu", "vm_launch.cu", "row_kernels.cu", "gemm_tcgen05.cu"]
 NVCC = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
 FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-Xcompiler", "-fPIC",
          "--expt-relaxed-constexpr", "-Xcompiler", "-Wall"] + os.environ.get("DRAGON_NVCC_DEFS", "").split()
@@ -86,7 +86,7 @@ def _generated_templates_object(objdir, verbose, force):
     return obj
 
 
-HOST_SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "specialize.cpp"]     # the host compiler: no CUDA in these
+HOST_SOURCES = ["prune.cpp", "lower.cpp", "codegen.cpp", "specialize.cpp", "verify.cpp"]     # the host compiler: no CUDA in these
 SAN_LIB = os.path.join(HERE, "libdragon_san.so")
 
 

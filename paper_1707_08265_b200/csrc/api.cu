@@ -424,6 +424,12 @@ int dragon_function_num_specialized(const dragon_function_t* f) {
   return n;
 }
 
+int dragon_verify_vm_program(const uint32_t* code, int n_code, int loop_start, int register_slots, int n_operands,
+                             int n_smem_slots, int n_spill_slots, int n_column_accs, int n_scalar_accs, int row_mode) {
+  return verify_program(code, n_code, loop_start, register_slots, n_operands, n_smem_slots, n_spill_slots, n_column_accs,
+                        n_scalar_accs, row_mode != 0);
+}
+
 int dragon_function_vm_ptx(const dragon_function_t* f, int step, char* buf, int cap) {
   if (!f || step < 0 || step >= (int)f->plan.steps.size() || f->plan.steps[step].kind != ST_VM || cap < 0 || (cap > 0 && !buf)) {
     set_error("dragon_function_vm_ptx: not a graph-VM step");

@@ -725,6 +725,8 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
   long long tiles = seg->row_mode ? seg->n : (seg->n + kVmTile - 1) / kVmTile;
   if (tiles >= (1LL << 31)) { set_error("graph VM: more than 2^31 tiles"); return DRAGON_ERR_UNSUPPORTED; }
   seg->grid = (int)std::max<long long>(1, std::min<long long>(tiles, (long long)sm_count * (seg->dense ? 2 : 1)));
+  // no program leaves here unverified: an index that a leaf would use out of range is a compiler error, not a fault
+  if (verify_segment(*seg) != DRAGON_OK) return DRAGON_ERR_UNSUPPORTED;
   return DRAGON_OK;
 }
 

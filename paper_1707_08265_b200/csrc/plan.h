@@ -150,6 +150,11 @@ int codegen_segment(const std::vector<Item>& items, const std::vector<int>& idx,
 
 std::string describe_plan(const Plan& p);
 
+// verify.cpp: static range check of every index an instruction stream uses, and of its structure
+int verify_program(const uint32_t* code, int n, int loop_start, int register_slots, int n_operands, int n_smem,
+                   int n_spill, int n_colacc, int n_scalacc, bool row_mode);
+int verify_segment(const VmSegment& sg);
+
 // specialize.cpp: PTX of the kernel that runs sg's instruction stream as straight-line code
 int specialize_ptx(const VmSegment& sg, const char* entry, std::string* ptx);
 
