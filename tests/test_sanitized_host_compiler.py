@@ -1,5 +1,5 @@
 """The host compiler (both prunes, lowering, segmentation, slot allocation, code generation) under
-AddressSanitizer and UndefinedBehaviorSanitizer: the library is rebuilt with those three sources
+AddressSanitizer and UndefinedBehaviorSanitizer: the library is rebuilt with the host-only sources (prune, lower, codegen, specialize, verify)
 instrumented and the host-side tests run against it in a child process with the sanitizer runtime
 preloaded.  Any report (heap overflow, use after free, signed overflow, misaligned access, ...) fails."""
 import os
@@ -22,7 +22,7 @@ def test_host_compiler_tests_are_clean_under_asan_and_ubsan():
                ASAN_OPTIONS="detect_leaks=0:abort_on_error=0:exitcode=99", UBSAN_OPTIONS="print_stacktrace=1:halt_on_error=1:exitcode=98")
     r = subprocess.run([sys.executable, "-m", "pytest", "-x", "-q", "-m", "not gpu", "-p", "no:cacheprovider",
                         "tests/test_host_compiler.py", "tests/test_codegen_emulated.py", "tests/test_codegen_invariants.py",
-                        "tests/test_inplace.py", "tests/test_gradient_stages.py"],
+                        "tests/test_inplace.py", "tests/test_gradient_stages.py", "tests/test_verify_program.py", "tests/test_specialize.py"],
                        cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
     out = r.stdout + r.stderr
     assert "AddressSanitizer" not in out and "runtime error:" not in out, out[-4000:]
