@@ -33,7 +33,7 @@ ALG_BYTES_PER_ELEM = 8.0     # read x once, write df/dx once
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the specialised VM kernel of this workload at the
 # full 2^26 elements, from one ncu capture (profiles/vm_config2.md); None once the generator of that kernel has
 # changed since the counters were taken
-NCU_DRAM_BYTES_PER_LAUNCH = None
+NCU_DRAM_BYTES_PER_LAUNCH = 268458752 + 218547968
 SAMPLE_ELEMS = 1 << 21       # the CPU oracle's bounded sample of workload 2, per pass
 
 
