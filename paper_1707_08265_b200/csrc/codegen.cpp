@@ -299,7 +299,7 @@ struct Gen {
     static const std::map<int, int> op = {{M_SIN, P_SIN}, {M_COS, P_COS}, {M_EXPC, P_EXPC}, {M_TANH, P_TANH},
       {M_SIGMOID, P_SIGMOID}, {M_RELU, P_RELU}, {M_NEG, P_NEG}, {M_STEP, P_STEP}, {M_CLAMPMASK, P_CLAMPMASK},
       {M_ONEMSQ, P_ONEMSQ}, {M_YOMY, P_YOMY}, {M_DIVPGB, P_DIVPGB}, {M_RBF16, P_RBF16}, {M_ROWSUM, P_ROWSUM},
-      {M_SQRT, P_SQRT}, {M_RCP, P_RCP}};
+      {M_SQRT, P_SQRT}, {M_RCP, P_RCP}, {M_TANHB, P_TANHB}, {M_SIGMOIDB, P_SIGMOIDB}, {M_EXPCB, P_EXPCB}};
     const int a = C(it.a), d = C(it.dst);
     load_acc(a, pos, a);
     // sin and cos of the same value share one range reduction

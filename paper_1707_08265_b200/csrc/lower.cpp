@@ -57,6 +57,7 @@ struct Lowerer {
   int konst(float c) {
     int v = new_val(VK_CONST, Shape(), -1, c);
     vals[v].known_const = true;
+    vals[v].lo = vals[v].hi = c;
     return v;
   }
   bool is_const(int v, float c) const { return vals[v].known_const && vals[v].c == c; }
@@ -70,9 +71,49 @@ struct Lowerer {
     vals[it.dst].known_const = vals[v].known_const;
     vals[it.dst].c = vals[v].c;
     vals[it.dst].row_uniform = vals[v].row_uniform;
+    vals[it.dst].lo = vals[v].lo;
+    vals[it.dst].hi = vals[v].hi;
     def_item[it.dst] = (int)items.size();
     items.push_back(it);
     return it.dst;
+  }
+
+  // [lo, hi] of the result of a micro-operation from those of its operands (NaN aside); anything not known is
+  // the whole line.  The bounds are rounded outwards by a relative 1e-6 so that fp32 rounding cannot breach them.
+  void set_range(int dst, int opc, const Value& A, const Value* B) {
+    const float inf = std::numeric_limits<float>::infinity();
+    float lo = -inf, hi = inf;
+    auto corners = [&](float (*f)(float, float)) {
+      const float c[4] = {f(A.lo, B->lo), f(A.lo, B->hi), f(A.hi, B->lo), f(A.hi, B->hi)};
+      lo = inf; hi = -inf;
+      for (float x : c) {
+        if (x != x) { lo = -inf; hi = inf; return; }      // 0 * inf, inf - inf: nothing is known
+        lo = std::min(lo, x); hi = std::max(hi, x);
+      }
+    };
+    const float m = std::max(std::fabs(A.lo), std::fabs(A.hi));
+    switch (opc) {
+      case M_ADD: corners([](float x, float y) { return x + y; }); break;
+      case M_SUB: corners([](float x, float y) { return x - y; }); break;
+      case M_MUL: corners([](float x, float y) { return x * y; }); break;
+      case M_DIVP: lo = std::min(A.lo, 0.f); hi = std::max(A.hi, 0.f); break;          // |a / (1 + |b|)| <= |a|, same sign
+      case M_SIN: case M_COS: case M_TANH: case M_TANHB: case M_DIVPGB: lo = -1.f; hi = 1.f; break;
+      case M_SIGMOID: case M_SIGMOIDB: case M_STEP: case M_CLAMPMASK: lo = 0.f; hi = 1.f; break;
+      case M_EXPC: case M_EXPCB: lo = 4.5e-5f; hi = 22027.f; break;                    // e^-10 .. e^10
+      case M_RELU: lo = std::max(A.lo, 0.f); hi = std::max(A.hi, 0.f); break;
+      case M_NEG: lo = -A.hi; hi = -A.lo; break;
+      case M_ONEMSQ: hi = 1.f; lo = m < 1e18f ? 1.f - m * m : -inf; break;              // 1 - y^2
+      case M_YOMY: hi = 0.25f;                                                          // y (1 - y), concave
+        lo = m < 1e18f ? std::min(A.lo * (1.f - A.lo), A.hi * (1.f - A.hi)) : -inf; break;
+      case M_RBF16: lo = A.lo - std::fabs(A.lo) / 128.f; hi = A.hi + std::fabs(A.hi) / 128.f; break;
+      case M_ROWSUM: { const float n = (float)A.shape.cols(); lo = std::min(A.lo * n, A.lo); hi = std::max(A.hi * n, A.hi); break; }
+      case M_SQRT: lo = std::sqrt(std::max(A.lo, 0.f)); hi = A.hi >= 0.f ? std::sqrt(A.hi) : 0.f; break;
+      case M_RCP: if (A.lo > 0.f || A.hi < 0.f) { lo = 1.f / A.hi; hi = 1.f / A.lo; } break;
+      default: break;
+    }
+    if (lo != lo || hi != hi) { lo = -inf; hi = inf; }
+    vals[dst].lo = lo - std::fabs(lo) * 1e-6f;
+    vals[dst].hi = hi + std::fabs(hi) * 1e-6f;
   }
 
   int mop(int opc, int a, int b = -1) {
@@ -104,8 +145,15 @@ struct Lowerer {
       float r = opc == M_ADD ? x + y : opc == M_SUB ? x - y : opc == M_MUL ? x * y : x / (1.f + std::fabs(y));
       return widen(konst(r), s);
     }
+    // clamps that cannot act are left out: tanh keeps its argument inside [-10, 10] and its result inside [-1, 1]
+    // (the rational fit stays below 1 well beyond |x| = 4), sigmoid and exp keep the exponential in range
+    const float mag = std::max(std::fabs(vals[a].lo), std::fabs(vals[a].hi));
+    if (opc == M_TANH && mag <= 4.01f) opc = M_TANHB;
+    if (opc == M_SIGMOID && mag <= 80.f) opc = M_SIGMOIDB;
+    if (opc == M_EXPC && mag <= 9.99f) opc = M_EXPCB;
     Item it; it.kind = IT_MOP; it.opc = opc; it.a = a; it.b = b;
     it.dst = new_val(VK_OP, s);
+    set_range(it.dst, opc, vals[a], b >= 0 ? &vals[b] : nullptr);
     vals[it.dst].row_uniform = opc == M_ROWSUM || (vals[a].row_uniform && (b < 0 || vals[b].row_uniform));
     def_item[it.dst] = (int)items.size();
     items.push_back(it);
@@ -669,9 +717,9 @@ static int lower_with_cuts(const Graph& g, const PruneResult& pr, const std::vec
         if (ua != cur) { ok = false; break; }
         switch (u.opc) {
           case M_RELU: e.opc = E_RELU; break;
-          case M_TANH: e.opc = E_TANH; break;
-          case M_SIGMOID: e.opc = E_SIGMOID; break;
-          case M_EXPC: e.opc = E_EXPC; break;
+          case M_TANH: case M_TANHB: e.opc = E_TANH; break;          // the epilogue keeps the clamped forms
+          case M_SIGMOID: case M_SIGMOIDB: e.opc = E_SIGMOID; break;
+          case M_EXPC: case M_EXPCB: e.opc = E_EXPC; break;
           case M_SIN: e.opc = E_SIN; break;
           case M_NEG: e.opc = E_NEG; break;
           case M_SQRT: e.opc = E_SQRT; break;
@@ -1001,7 +1049,7 @@ static std::string disassemble(const VmSegment& sg) {
   static const char* pn[] = {"ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls",
                              "divps", "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq",
                              "yomy", "divpgb", "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout",
-                             "scalout", "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "end"};
+                             "scalout", "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "tanhb", "sigmoidb", "expcb", "end"};
   std::string s;
   char buf[64];
   for (size_t i = 0; i < sg.code.size(); ++i) {

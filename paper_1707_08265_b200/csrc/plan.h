@@ -2,6 +2,7 @@
 // (lower.cpp builds the micro-operation list from the kept operators, codegen.cpp turns each
 // fused segment into a VM instruction stream).
 #pragma once
+#include <limits>
 #include <string>
 #include <vector>
 
@@ -42,6 +43,7 @@ enum MOpc {
   M_ADD, M_SUB, M_MUL, M_DIVP,
   M_SIN, M_COS, M_EXPC, M_TANH, M_SIGMOID, M_RELU, M_NEG, M_STEP, M_CLAMPMASK, M_ONEMSQ, M_YOMY,
   M_DIVPGB, M_RBF16, M_ROWSUM, M_SQRT, M_RCP,
+  M_TANHB, M_SIGMOIDB, M_EXPCB,   // the same functions where the argument is proven inside the range in which the clamps do nothing
   M_WIDEN,  // same value, wider logical shape (no instruction)
   M_STORE,  // write value a to memory mem
   M_ACCUM   // sum value a over the axes along which mem is smaller, write to mem
@@ -56,6 +58,8 @@ struct Value {
   float c = 0.f;
   bool known_const = false;  // VK_CONST, or a widened view of one
   bool row_uniform = false;  // the same value in every element of a row: a row sum, a scalar, or an elementwise function of such
+  // every element lies in [lo, hi] whatever is fed (NaN aside): interval arithmetic over the micro-operations
+  float lo = -std::numeric_limits<float>::infinity(), hi = std::numeric_limits<float>::infinity();
 };
 
 // One operation of a product's epilogue program: the running value v of an output element (the fp32

@@ -107,6 +107,9 @@ enum Plain : int {
                         // (reduced outputs beyond the pinned register slots)
   P_SQRT,               // acc = sqrt(acc)
   P_RCP,                // acc = 1 / acc
+  // tanh, sigmoid and clamped exp without their clamps, for arguments that the host's interval analysis has
+  // proven inside the range where the clamps do nothing (|x| <= 4.01, |x| <= 80, |x| <= 9.99)
+  P_TANHB, P_SIGMOIDB, P_EXPCB,
   P_END,
   P_COUNT_
 };

@@ -178,8 +178,9 @@ VM_HD float exp_core(float x) {
   const float p = f_ex2(t);
   return fmaf(p, e, p);
 }
-VM_HD float exp_clamped10(float x) { return exp_core(fminf(fmaxf(x, -10.0f), 10.0f)); }
-VM_HD float exp_wide(float x) { return exp_core(fminf(fmaxf(x, -86.0f), 88.7f)); }
+// the clamps keep a NaN a NaN, as the kernel's max.NaN / min.NaN do (fminf / fmaxf alone would drop it)
+VM_HD float exp_clamped10(float x) { return x != x ? x : exp_core(fminf(fmaxf(x, -10.0f), 10.0f)); }
+VM_HD float exp_wide(float x) { return x != x ? x : exp_core(fminf(fmaxf(x, -86.0f), 88.7f)); }
 
 VM_HD float sigmoid_f(float x) { return f_rcp(1.0f + exp_wide(-x)); }
 

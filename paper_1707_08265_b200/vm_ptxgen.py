@@ -49,7 +49,7 @@ N_SACC = 4          # scalar accumulators
 PLAIN = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
          "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
          "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop_begin", "loop_end", "colout", "scalout",
-         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "end"]
+         "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstfl", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "tanhb", "sigmoidb", "expcb", "end"]
 
 
 def f32bits(x):
@@ -508,29 +508,39 @@ class Kernel:
 
     def clamp(self, s, lo, hi):
         d = self.f()
-        self.e("max.f32 %s, %s, %s;" % (d, s, fc(lo)))
-        self.e("min.f32 %s, %s, %s;" % (d, d, fc(hi)))
+        self.e("max.NaN.f32 %s, %s, %s;" % (d, s, fc(lo)))      # a NaN stays a NaN (as in the reference arithmetic)
+        self.e("min.NaN.f32 %s, %s, %s;" % (d, d, fc(hi)))
         return d
 
     EXP_LO, EXP_HI = -86.0, 88.7   # e^x stays a normal fp32 number on this range
 
-    def expc(self, xs):
+    # The "b" forms of expc, sigmoid and tanh (bounded=True) leave the clamps out: the host emits them only where
+    # its interval analysis has proven the argument inside the range in which the clamps do nothing.
+    def expc(self, xs, bounded=False):
         out = []
         for x in xs:
+            if bounded:
+                out.append(self.exp_core(x))
+                continue
             lo, hi = self.unpack(x)
             out.append(self.exp_core(self.pack(self.clamp(lo, -10.0, 10.0), self.clamp(hi, -10.0, 10.0))))
         return out
 
-    def sigmoid(self, xs):
+    def sigmoid(self, xs, bounded=False):
         out = []
         for x in xs:
+            if bounded:
+                e = self.exp_core(self.mul2(x, self.K(-1.0)))
+                l2, h2 = self.unpack(self.add2(e, self.K(1.0)))
+                out.append(self.pack(self.rcp(l2), self.rcp(h2)))
+                continue
             lo, hi = self.unpack(self.mul2(x, self.K(-1.0)))
             e = self.exp_core(self.pack(self.clamp(lo, self.EXP_LO, self.EXP_HI), self.clamp(hi, self.EXP_LO, self.EXP_HI)))
             l2, h2 = self.unpack(self.add2(e, self.K(1.0)))
             out.append(self.pack(self.rcp(l2), self.rcp(h2)))
         return out
 
-    def tanh(self, xs):
+    def tanh(self, xs, bounded=False):
         """x * P(x^2) / Q(x^2) (a rational fit on |x| <= 9, about 5 ulp; beyond 9.07 it exceeds 1), argument
         clamped at 10 and result clamped to [-1, 1], so that a saturated tanh is exactly +-1; NaN stays NaN"""
         def clamp2(v, lim):
@@ -541,7 +551,7 @@ class Kernel:
                 self.e("min.NaN.f32 %s, %s, %s;" % (d, d, fc(lim)))
                 out.append(d)
             return self.pack(out[0], out[1])
-        cs = [clamp2(x, 10.0) for x in xs]
+        cs = list(xs) if bounded else [clamp2(x, 10.0) for x in xs]
         z = [self.mul2(c, c) for c in cs]
         k0, k1 = self.K(1.3442309683456469e-08), self.K(2.0679596671714183e-05)
         p = [self.fma2(zi, k0, k1) for zi in z]
@@ -557,7 +567,7 @@ class Kernel:
         for c, pi, qi in zip(cs, p, q):
             ql, qh = self.unpack(qi)
             y = self.mul2(self.mul2(c, pi), self.pack(self.rcp(ql), self.rcp(qh)))
-            out.append(clamp2(y, 1.0))
+            out.append(y if bounded else clamp2(y, 1.0))
         return out
 
     def divp(self, num, den, dst):
@@ -1230,6 +1240,12 @@ class Kernel:
             self.fetch(); self.mov_v(A, self.tanh(A))
         elif op == "sigmoid":
             self.fetch(); self.mov_v(A, self.sigmoid(A))
+        elif op == "expcb":
+            self.fetch(); self.mov_v(A, self.expc(A, bounded=True))
+        elif op == "tanhb":
+            self.fetch(); self.mov_v(A, self.tanh(A, bounded=True))
+        elif op == "sigmoidb":
+            self.fetch(); self.mov_v(A, self.sigmoid(A, bounded=True))
         elif op in ("relu", "step", "clampmask", "divpgb"):
             self.fetch()
             out = []

@@ -180,3 +180,42 @@ def test_sine_of_huge_arguments_in_every_lane_and_tail():
     grads = gd.grad([out], [xi])
     (c,), _ = run_gpu(gd.desc, [xi], grads, [x])                               # cos alone
     assert np.max(np.abs(c - np.cos(xd))) < 3e-7
+
+
+@pytest.mark.parametrize("outer,inner,scale", [("Tanh", "Sigmoid", 1), ("Tanh", "Sin", 1), ("Tanh", "Tanh", 4), ("Exp", "Tanh", 8),
+                                               ("Sigmoid", "Sin", 64), ("Exp", "Sin", 16)])
+def test_forms_without_clamps_over_their_whole_proven_range(outer, inner, scale):
+    """outer(scale * inner(x)): the lowering proves |argument| <= scale and, where that is inside the range in which
+    the clamps of outer do nothing, emits the form without them (tanhb up to 4, sigmoidb up to 80, expcb up to 9.99).
+    Values and gradients against the oracle over a dense sweep of x that drives the inner function to both ends of
+    its range, inf and NaN included; scale 16 > 9.99 keeps the clamped exponential (and its mask) in the comparison."""
+    gd = wl.GraphDesc()
+    xs = np.concatenate([sweep(-12, 8, 48), np.linspace(-20, 20, 4001).astype(np.float32), [np.inf, -np.inf, np.nan]]).astype(np.float32)
+    n = xs.size
+    x = gd.tensor("x", [n]); w = gd.tensor("w", [n])
+    v = gd.op(inner, [x], "inner")
+    k = 1
+    while k < scale:                                   # scale * v by doubling
+        v = gd.op("Add", [v, v], "v%d" % k); k *= 2
+    y = gd.op(outer, [v], "outer")
+    (dx,) = gd.grad([gd.op("Mul", [y, w], "obj")], [x])
+    ws = np.random.default_rng(3).standard_normal(n).astype(np.float32)
+    got, f = run_gpu(gd.desc, [x, w], [y, dx], [xs, ws])
+    want_b = {"Tanh": scale <= 4, "Sigmoid": scale <= 80, "Exp": scale <= 9}[outer]
+    name = {"Tanh": "tanh", "Sigmoid": "sigmoid", "Exp": "expc"}[outer]
+    # the inner function may itself be one of the three: look at the last occurrence
+    plan = f.describe()
+    assert (name + "b") in plan if want_b else (name + ";") in plan.replace(name + "b", "#"), plan
+    from test_gpu_vm import FLOOR_OK, C_COND
+    fin = np.isfinite(xs)
+    with np.errstate(all="ignore"):
+        ref = interp.run_function(gd.desc, [x, w], [y, dx], [xs, ws])
+        low = interp.run_function(gd.desc, [x, w], [y, dx], [xs, ws], dtype=np.float32)
+    for gv, rv, lv, what in zip(got, ref, low, ("value", "gradient")):
+        # a composition that saturates amplifies fp32 rounding (e^(8 tanh x) near its ends): held to the plain
+        # tolerance where the CPU fp32 instance of the same graph reaches it, else to C_COND times that floor
+        floor = float(np.max(np.abs(lv[fin].astype(np.float64) - rv[fin]) / (TOL32 * (1 + np.abs(rv[fin])))))
+        tol = TOL32 if floor <= FLOOR_OK else TOL32 * C_COND * floor
+        check(gv[fin], rv[fin], tol, "%s(%d*%s) %s (fp32 floor %.3g)" % (outer, scale, inner, what, floor))
+        if what == "value":
+            assert np.isnan(gv[np.isnan(xs)]).all(), what             # NaN in, NaN out

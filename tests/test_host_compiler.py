@@ -349,3 +349,35 @@ def test_elementwise_chains_behind_a_product_run_in_its_epilogue():
     O = gd.op("Mul", [gd.op("Tanh", [Y], "T"), side], "O")
     f = B.Graph.from_desc(gd.desc).function([X, W, raw], [O])
     assert "epilogue" not in f.describe(), f.describe()
+
+
+def test_clamps_are_left_out_only_where_the_argument_is_proven_in_range():
+    """Interval analysis over the micro-operations: tanh of a sigmoid, of a sine, of a product of two bounded values
+    takes the form without clamps, tanh of a fed tensor or of a sum that can exceed the range does not; the clamped
+    exponential of a bounded argument likewise, and of 12 * tanh(x) (up to 12 > 10) not."""
+    def plan(build):
+        gd = wl.GraphDesc()
+        x = gd.tensor("x", [5000]); y = gd.tensor("y", [5000])
+        out = build(gd, x, y)
+        return B.Graph.from_desc(gd.desc).function([x, y], [out]).describe()
+
+    def twelve(gd, v):      # 12 * v as a sum of doublings, no constant operand needed
+        v2 = gd.op("Add", [v, v], "v2"); v4 = gd.op("Add", [v2, v2], "v4"); v8 = gd.op("Add", [v4, v4], "v8")
+        return gd.op("Add", [v8, v4], "v12")
+
+    assert "tanhb" in plan(lambda gd, x, y: gd.op("Tanh", [gd.op("Sigmoid", [x], "s")], "t"))
+    assert "tanhb" in plan(lambda gd, x, y: gd.op("Tanh", [gd.op("Sin", [x], "s")], "t"))
+    assert "tanhb" in plan(lambda gd, x, y: gd.op("Tanh", [gd.op("Mul", [gd.op("Sin", [x], "s"), gd.op("Tanh", [y], "u")], "p")], "t"))
+    p = plan(lambda gd, x, y: gd.op("Tanh", [x], "t"))
+    assert "tanh;" in p and "tanhb" not in p
+    p = plan(lambda gd, x, y: gd.op("Tanh", [gd.op("Add", [gd.op("Sin", [x], "s"), y], "a")], "t"))
+    assert "tanhb" not in p
+    p = plan(lambda gd, x, y: gd.op("Tanh", [twelve(gd, gd.op("Sin", [x], "s"))], "t"))
+    assert "tanhb" not in p                                              # |12 sin x| <= 12 > 4
+    assert "sigmoidb" in plan(lambda gd, x, y: gd.op("Sigmoid", [twelve(gd, gd.op("Sin", [x], "s"))], "t"))     # 12 <= 80
+    assert "expcb" in plan(lambda gd, x, y: gd.op("Exp", [gd.op("Tanh", [x], "s")], "t"))
+    p = plan(lambda gd, x, y: gd.op("Exp", [twelve(gd, gd.op("Tanh", [x], "s"))], "t"))
+    assert "expcb" not in p and "expc;" in p
+    # a ReLU keeps the upper bound open, a division by 1 + |b| keeps the numerator's bound
+    assert "tanhb" not in plan(lambda gd, x, y: gd.op("Tanh", [gd.op("ReLU", [x], "r")], "t"))
+    assert "tanhb" in plan(lambda gd, x, y: gd.op("Tanh", [gd.op("Div", [gd.op("Sigmoid", [x], "s"), y], "d")], "t"))

@@ -156,7 +156,7 @@ def test_random_single_word_damage_is_caught_or_harmless(seed):
     """Flip the argument field of one word of a real program to a huge value: either the verifier refuses the
     stream, or the instruction takes no argument (its leaf never looks at the field)."""
     takes_no_arg = {plain(n) for n in ("sin", "cos", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy",
-                                       "divpgb", "rbf16", "loop_begin", "loop_end", "end", "sacc0", "sacc1", "sacc2", "sacc3", "sqrt", "rcp")}
+                                       "divpgb", "rbf16", "loop_begin", "loop_end", "end", "sacc0", "sacc1", "sacc2", "sacc3", "sqrt", "rcp", "tanhb", "sigmoidb", "expcb")}
     for j in ("ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum", "sincosr", "cossinr", "macc0", "macc1", "macc2",
               "macc3") + tuple("stld%d" % k for k in range(8)):
         takes_no_arg |= {joint(j, s) for s in range(8)}

@@ -12,7 +12,7 @@ J = ["ldr", "str", "add", "sub", "rsub", "mul", "divp", "rdivp", "addto", "accum
 P = ["ldu", "addu", "subu", "rsubu", "mulu", "divpu", "rdivpu", "fmau", "lds", "sts", "adds", "subs", "rsubs", "muls", "divps",
      "rdivps", "sin", "cos", "sincos", "cossin", "expc", "tanh", "sigmoid", "relu", "neg", "step", "clampmask", "onemsq", "yomy", "divpgb",
      "rbf16", "rowsum", "gld", "gst", "gldf", "gstf", "fill", "spill", "uload", "uconst", "loop{", "}loop", "colout", "scalout",
-     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "end"]
+     "sacc0", "sacc1", "sacc2", "sacc3", "ascal0", "ascal1", "ascal2", "ascal3", "glda0", "glda", "ldsw", "ldswa", "gstf}loop", "glda0h", "ldswah", "rowsumu", "accums", "sqrt", "rcp", "tanhb", "sigmoidb", "expcb", "end"]
 
 
 def _bf16(a):
@@ -95,6 +95,15 @@ def run_step(step, feeds, fetch_shapes, nr=STRIDE):
         elif name == "cossin": S[arg] = np.sin(acc); acc = np.cos(acc)
         elif name == "expc": acc = np.exp(np.clip(acc, -10, 10))
         elif name == "tanh": acc = np.tanh(acc)
+        elif name == "tanhb":
+            assert np.all(np.abs(acc[np.isfinite(acc)]) <= 4.01), "tanhb outside its proven range"
+            acc = np.tanh(acc)
+        elif name == "sigmoidb":
+            assert np.all(np.abs(acc[np.isfinite(acc)]) <= 80.0), "sigmoidb outside its proven range"
+            acc = 1 / (1 + np.exp(-acc))
+        elif name == "expcb":
+            assert np.all(np.abs(acc[np.isfinite(acc)]) <= 10.0), "expcb outside its proven range"
+            acc = np.exp(acc)
         elif name == "sigmoid": acc = 1 / (1 + np.exp(-acc))
         elif name == "relu": acc = np.maximum(acc, 0)
         elif name == "neg": acc = -acc
