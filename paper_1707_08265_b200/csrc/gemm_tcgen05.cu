@@ -1,8 +1,9 @@
 // InnerProduct contraction C[M,N] = A[M,K] * B[N,K]^T: bf16 operands, fp32 accumulation in
 // tensor memory, fp32 or bf16 output.  Hand-written for sm_100a:
-//   - operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) into a
-//     ring of shared-memory stages guarded by full/empty mbarriers;
-//   - one elected thread issues tcgen05.mma (cta_group::1, kind::f16, 128 x 256 x 16) with the
+//   - operands are staged by TMA (cp.async.bulk.tensor, 128-byte swizzle; every CTA loads its own
+//     tiles) into a ring of shared-memory stages guarded by full/empty mbarriers;
+//   - one elected thread issues tcgen05.mma (kind::f16; cta_group::1 with 128 x 256 x 16, or, in the
+//     pair kernel, cta_group::2 with 256 x 256 x 16 over the two CTAs of a cluster) with the
 //     accumulator in TMEM; tcgen05.commit releases stages and signals the epilogue;
 //   - four epilogue warps read their 32-lane TMEM quadrants with tcgen05.ld and write C;
 //   - CTAs are persistent (one per SM) and walk the 128 x 256 output tiles in an L2-friendly
@@ -143,7 +144,7 @@ __device__ __forceinline__ void mbar_arrive_remote(uint32_t bar) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 // TMA copy of one CTA of a pair into its own shared memory; the bytes are counted on the mbarrier `bar` (a
-// shared::cluster address: the first CTA's), no multicast
+// shared::cluster address: the first CTA's); each CTA copies only what it reads itself
 __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
