@@ -263,3 +263,25 @@ def test_elementwise_chain_in_the_epilogue_of_a_product(m, n, k):
         assert f.num_launches() == 1 and want in f.describe(), f.describe()
         (ref,) = interp.run_function(gd.desc, [X, W, b, side, s], [P], feeds)
         check(got, ref, 2e-5, "bias, sigmoid, side operand, scalar in the epilogue (%s)" % side_dtype)
+
+
+@pytest.mark.parametrize("pair", ["0", "1"])
+@pytest.mark.parametrize("m,n,k", [(136, 104, 64), (264, 256, 72), (520, 264, 136), (128, 256, 64), (1024, 136, 200)])
+def test_both_kernel_forms_at_the_edges_of_a_pair_tile(m, n, k, pair, monkeypatch):
+    """The product kernel exists for one CTA per 128 x 256 tile and for a pair of CTAs per 256 x 256 tile.  Shapes that
+    leave the pair's second CTA eight rows of A, no row of B at all (n <= 128), or a last tile that is mostly empty, in
+    both forms, forward with bias and ReLU and all three gradients (the transposed-operand variants and the column
+    sums of the bias gradient), against the oracle."""
+    monkeypatch.setenv("DRAGON_GEMM_PAIR", pair)
+    gd = wl.GraphDesc()
+    X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16"); b = gd.tensor("b", [n], "f32"); G = gd.tensor("G", [m, n], "f32")
+    Y = gd.op("ReLU", [gd.op("BiasAdd", [gd.op("InnerProduct", [X, W], "Z", [m, n], "f32"), b], "A", [m, n], "f32")], "Y")
+    obj = gd.op("Mul", [Y, G], "obj")
+    dX, dW, db = gd.grad([obj], [X, W, b])
+    rng = np.random.default_rng(m + n + k)
+    feeds = [bf16able(rng.standard_normal((m, k))), bf16able(rng.standard_normal((n, k)) / np.sqrt(k)), bf16able(rng.standard_normal(n)),
+             bf16able(rng.standard_normal((m, n)))]
+    got, f = run_gpu(gd.desc, [X, W, b, G], [Y, dX, dW, db], feeds)
+    ref = interp.run_function(gd.desc, [X, W, b, G], [Y, dX, dW, db], feeds)
+    for gv, rv, name in zip(got, ref, ("Y", "dX", "dW", "db")):
+        check(gv, rv, 1e-4 if name != "Y" else 2e-5, "%s (pair=%s)" % (name, pair))
