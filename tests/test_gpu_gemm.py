@@ -207,15 +207,18 @@ def test_computed_bias_before_or_after_the_product(bias_first):
     check(got, ref, 2e-5, "Y")
 
 
+@pytest.mark.parametrize("m", [128, 256])             # one CTA per tile; a pair of CTAs on one tile
 @pytest.mark.parametrize("k", [64, 320])
-def test_a_pipeline_wait_that_runs_out_is_reported_and_the_next_run_is_correct(k, monkeypatch):
+def test_a_pipeline_wait_that_runs_out_is_reported_and_the_next_run_is_correct(k, m, monkeypatch):
     """Failure detection without a fault: the producer of the contraction leaves out the loads of its first
     stage (test hook), so the consumer's first wait is for a signal that nothing sends; with the pipeline's
     budget shortened to about a millisecond the wait runs out, the kernel records DRAGON_ERR_TIMEOUT, lets
     the copies that are in flight land (that wait keeps its full budget), frees its tensor memory and
     returns by itself.  The context stays usable: the same function run again without the hook is correct."""
     from paper_1707_08265_b200 import binding as B
-    m, n = 128, 256                                   # one output tile; k = 320: later stages are really loaded
+    n = 256                                           # one output tile; k = 320: later stages are really loaded
+    # m = 256: the pair kernel; both CTAs leave out their first loads, the first CTA's consumer gives up, the second
+    # CTA's epilogue gives up on its own budget, both meet at the cluster barrier and free their tensor memory
     gd = wl.GraphDesc()
     X = gd.tensor("X", [m, k], "bf16"); W = gd.tensor("W", [n, k], "bf16")
     Y = gd.op("InnerProduct", [X, W], "Y", [m, n], "f32")
